@@ -1,0 +1,155 @@
+/*
+ * rrm.h - C ABI of the B200 (sm_100a) Recurrent Residual Module library.
+ *
+ * The Recurrent Residual Module (RRM) runs a CNN on video by keeping, for every linear
+ * layer l, the previous frame's input I_{t-1,l} and projection P_{t-1,l} = F_l*I_{t-1,l} + b_l,
+ * and evaluating each new frame as  P_{t,l} = P_{t-1,l} + F_l * (I_{t,l} - I_{t-1,l}),
+ * I_{t,l+1} = f(P_{t,l})  (Eq. 4-5, Algorithm 1).  Only the non-zero part of the input
+ * delta is visited (Sec. 3.5), so the cost follows the delta density (Table 1) while the
+ * result equals a dense recompute of the frame.
+ *
+ * Conventions
+ *   - Every function returns an int status (RRM_OK or a negative RRM_ERR_*), never throws,
+ *     never aborts.  Nothing synchronises the stream unless stated.
+ *   - "dev" pointers are device pointers on the current CUDA device, "host" pointers are
+ *     host memory.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Activation layouts at this boundary, N = number of independent video streams:
+ *       RRM_F32 : float   [N][C][H][W]
+ *       RRM_I8  : int8_t  [N][C][H][W]     (values in [-127,127]; layer inputs in [0,127]
+ *                                           or any range whose frame-to-frame delta fits int8)
+ *       RRM_BIN : uint32_t[N][H][W][ceil(C/32)]  bit i of word k = channel 32k+i, 1 = +1, 0 = -1,
+ *                                           unused high bits zero
+ *       raw int32 projections: int32_t [N][C][H][W]
+ *     Filters: [C_out][C_in][kh][kw] row-major; float for RRM_F32, int8_t for RRM_I8 and
+ *     RRM_BIN (+1 / -1).  Bias: float (RRM_F32) or int32_t.  Weights and bias are copied and
+ *     repacked into library-owned device memory at create time; the caller may free its copy.
+ *   - One object may be used from one stream at a time.
+ */
+#ifndef RRM_H
+#define RRM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rrm_net rrm_net;     /* a stack of linear layers with their RRM state */
+typedef struct rrm_net rrm_layer;   /* a single layer is a stack of one */
+
+enum {
+    RRM_OK = 0,
+    RRM_ERR_INVALID_ARG = -1,
+    RRM_ERR_SHAPE = -2,
+    RRM_ERR_DTYPE = -3,
+    RRM_ERR_ALLOC = -4,
+    RRM_ERR_CAPACITY = -5,
+    RRM_ERR_TIMEOUT = -6,
+    RRM_ERR_CUDA = -7,
+    RRM_ERR_UNSUPPORTED = -8
+};
+
+enum { RRM_CONV = 0, RRM_FC = 1 };
+enum { RRM_F32 = 0, RRM_I8 = 1, RRM_BIN = 2 };
+enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2 };
+/* how F*dI is evaluated; AUTO picks per layer */
+enum { RRM_VARIANT_AUTO = 0, RRM_VARIANT_GATHER = 1, RRM_VARIANT_TENSOR = 2, RRM_VARIANT_DENSE = 3 };
+
+/*
+ * One linear layer and the nonlinear map f that follows it (Eq. 1).
+ * f, in order: [requant by `shift`: q = clamp((P + 2^(shift-1)) >> shift, -127, 127)] ->
+ * [+ residual tensor] -> act -> max-pool; with act == SIGN the pool comes first and the
+ * output bit is (pooled P >= theta).  shift < 0 on an integer layer emits the raw int32
+ * projection (no act other than SIGN allowed then).  RRM_F32 ignores shift/theta.
+ * An FC layer has h = w = kh = kw = 1, stride 1, pad 0.
+ */
+typedef struct {
+    int32_t kind;        /* RRM_CONV | RRM_FC */
+    int32_t dtype;       /* type of the layer's input and weights */
+    int32_t n;           /* independent streams processed per call (same for all layers) */
+    int32_t c_in, h, w;  /* input tensor */
+    int32_t c_out, kh, kw, stride, pad;
+    int32_t act;         /* RRM_ACT_* */
+    int32_t pool_k, pool_s, pool_p;   /* pool_k == 0: no pooling */
+    int32_t shift, theta;
+    int32_t src;         /* stacks only: index of the tensor this layer reads (0 = frame, l+1 = output of layer l) */
+    int32_t res;         /* stacks only: tensor added before act, or -1 */
+    int32_t variant;     /* RRM_VARIANT_* */
+} rrm_layer_desc;
+
+/* Counters of the most recent step of one layer (delta density as defined for Table 1). */
+typedef struct {
+    int64_t in_elems;          /* elements of the layer input (all streams) */
+    int64_t nnz_elems;         /* non-zero delta elements: rho = nnz_elems / in_elems */
+    int64_t in_pixels;         /* spatial positions of the input (FC: groups of 32 inputs) */
+    int64_t active_in_pixels;  /* positions with at least one non-zero delta */
+    int64_t out_pixels;        /* spatial positions of the projection */
+    int64_t active_out_pixels; /* positions whose projection was updated */
+    int64_t active_macs;       /* exact multiply-accumulates the non-zero deltas imply */
+    int64_t dense_macs;        /* multiply-accumulates of a dense pass */
+    int32_t variant;           /* RRM_VARIANT_* actually used */
+    int32_t error_word;        /* device-side error flags, 0 = none */
+} rrm_stats;
+
+/* ---- single layer (Eq. 2-5) ------------------------------------------------------- */
+
+/* Creates a layer with state I_prev = 0, P_prev = bias (Algorithm 1, line 1), so a first
+ * rrm_step without keyframe equals a dense pass.  W_dev / bias_dev: device pointers in the
+ * layouts above (bias_dev may be NULL = zeros).  Allocates device memory. */
+int rrm_layer_create(rrm_layer** out, const rrm_layer_desc* desc, const void* W_dev, const void* bias_dev);
+int rrm_layer_destroy(rrm_layer* layer);
+
+/* Dense ("precise") inference of X0 that resets the state: I_prev = X0, P_prev = F*X0 + b
+ * (the re-start that clears accumulated error, Sec. 3.4).  Y0_dev may be NULL; otherwise it
+ * receives f(P) like rrm_step.  Asynchronous on `stream`. */
+int rrm_keyframe(rrm_layer* layer, const void* X0_dev, void* Y0_dev, void* stream);
+
+/* One RRM frame (Eq. 5): D = X_t - I_prev, compact its non-zeros, P_prev += F*D (no bias),
+ * I_prev = X_t, Y_t = f(P_prev).  X_t is read-only and caller-owned; Y_t (caller-owned, may
+ * be NULL) is written in full in the boundary layout.  Asynchronous on `stream`; no host
+ * synchronisation inside. */
+int rrm_step(rrm_layer* layer, const void* Xt_dev, void* Yt_dev, void* stream);
+
+/* The same layer evaluated densely, Y = f(F*X + b), without reading or changing the RRM
+ * state: the library's own dense path (the denominator of its delta-path speedup). */
+int rrm_dense(rrm_layer* layer, const void* X_dev, void* Y_dev, void* stream);
+
+/* rrm_step with HOST buffers: copies X_t to the device, steps, copies Y_t back, all on
+ * `stream`; returns after the stream has been synchronised. */
+int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* stream);
+
+/* Synchronises the layer's last stream and fills `host_out`. */
+int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out);
+
+/* Copies the stored projection P_prev (float or int32, [N][C_out][OH][OW]) to P_dev. */
+int rrm_layer_projection(rrm_layer* layer, void* P_dev, void* stream);
+
+/* ---- layer stack (Algorithm 1) ---------------------------------------------------- */
+
+/* descs[l].src / .res give the topology; tensor 0 is the frame, tensor l+1 = f(P_l).
+ * W_dev[l] / bias_dev[l] as for rrm_layer_create. */
+int rrm_net_create(rrm_net** out, const rrm_layer_desc* descs, int n_layers,
+                   const void* const* W_dev, const void* const* bias_dev);
+int rrm_net_destroy(rrm_net* net);
+
+/* Dense pass over the whole stack that resets every layer's state. out_dev may be NULL. */
+int rrm_net_keyframe(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
+/* Algorithm 1, one iteration of the frame loop; out_dev receives the last tensor. */
+int rrm_net_step(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
+/* Dense evaluation of the stack without touching the RRM state. */
+int rrm_net_dense(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
+int rrm_net_step_host(rrm_net* net, const void* frame_host, void* out_host, void* stream);
+
+int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* host_out);
+/* Copies P_prev of `layer` / the current value of tensor `t` (boundary layout) to dst_dev. */
+int rrm_net_projection(rrm_net* net, int layer, void* P_dev, void* stream);
+int rrm_net_tensor(rrm_net* net, int t, void* dst_dev, void* stream);
+/* Bytes rrm_net_tensor / the out_dev argument need for tensor `t` (negative = error). */
+int64_t rrm_net_tensor_bytes(const rrm_net* net, int t);
+
+const char* rrm_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RRM_H */

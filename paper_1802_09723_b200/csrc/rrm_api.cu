@@ -1,0 +1,347 @@
+// C ABI of the RRM library: object construction, validation and the per-frame launch sequences.
+#include "rrm_common.cuh"
+#include <new>
+#include <cstring>
+
+using namespace rrm;
+
+namespace {
+
+int tensor_bytes_boundary(const Tensor& T, int64_t* out)
+{
+    if (T.dtype == T_BIN) *out = (int64_t)T.pixels() * T.cs * 4;
+    else *out = (int64_t)T.n * T.c * T.h * T.w * (T.dtype == T_I8 ? 1 : 4);
+    return RRM_OK;
+}
+
+int validate_desc(const rrm_layer_desc& d, int l, int n_layers)
+{
+    if (d.kind != RRM_CONV && d.kind != RRM_FC) return RRM_ERR_INVALID_ARG;
+    if (d.dtype != RRM_F32 && d.dtype != RRM_I8 && d.dtype != RRM_BIN) return RRM_ERR_DTYPE;
+    if (d.n < 1 || d.c_in < 1 || d.c_out < 1 || d.h < 1 || d.w < 1) return RRM_ERR_SHAPE;
+    if (d.kh < 1 || d.kw < 1 || d.stride < 1 || d.pad < 0) return RRM_ERR_SHAPE;
+    if (d.kind == RRM_FC && (d.h != 1 || d.w != 1 || d.kh != 1 || d.kw != 1 || d.stride != 1 || d.pad != 0))
+        return RRM_ERR_SHAPE;
+    if (d.h + 2 * d.pad < d.kh || d.w + 2 * d.pad < d.kw) return RRM_ERR_SHAPE;
+    if (d.pad >= d.kh || d.pad >= d.kw) return RRM_ERR_SHAPE;
+    if (d.act != RRM_ACT_NONE && d.act != RRM_ACT_RELU && d.act != RRM_ACT_SIGN) return RRM_ERR_INVALID_ARG;
+    if (d.dtype == RRM_F32 && d.act == RRM_ACT_SIGN) return RRM_ERR_UNSUPPORTED;
+    if (d.dtype != RRM_F32 && d.shift < 0 && d.act == RRM_ACT_RELU) return RRM_ERR_UNSUPPORTED;
+    if (d.shift > 30) return RRM_ERR_INVALID_ARG;
+    if (d.pool_k < 0 || (d.pool_k > 0 && (d.pool_s < 1 || d.pool_p < 0 || d.pool_p >= d.pool_k))) return RRM_ERR_SHAPE;
+    if (d.src < 0 || d.src > l) return RRM_ERR_INVALID_ARG;
+    if (d.res > l) return RRM_ERR_INVALID_ARG;
+    if (d.res >= 0 && (d.pool_k > 0 || d.act == RRM_ACT_SIGN)) return RRM_ERR_UNSUPPORTED;
+    if (d.res >= 0 && d.dtype != RRM_F32 && d.shift < 0) return RRM_ERR_UNSUPPORTED;
+    if (d.variant < RRM_VARIANT_AUTO || d.variant > RRM_VARIANT_DENSE) return RRM_ERR_INVALID_ARG;
+    (void)n_layers;
+    return RRM_OK;
+}
+
+int dev_alloc(rrm_net* net, void** p, size_t bytes)
+{
+    if (bytes == 0) bytes = 16;
+    if (cudaMalloc(p, bytes) != cudaSuccess) { *p = nullptr; cudaGetLastError(); return RRM_ERR_ALLOC; }
+    net->allocs.push_back(*p);
+    if (cudaMemset(*p, 0, bytes) != cudaSuccess) return RRM_ERR_CUDA;
+    return RRM_OK;
+}
+
+void set_tensor(Tensor& T, int dtype, int n, int c, int h, int w)
+{
+    T.dtype = dtype; T.n = n; T.c = c; T.h = h; T.w = w;
+    if (dtype == T_I8) { T.cs = round_up(c, 4); T.unit_bytes = 1; }
+    else if (dtype == T_BIN) { T.cs = ceil_div(c, 32); T.unit_bytes = 4; }
+    else { T.cs = c; T.unit_bytes = 4; }
+}
+
+int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const void* const* W, const void* const* B)
+{
+    const int n = descs[0].n;
+    net->n = n;
+    net->tensors.resize(n_layers + 1);
+    net->layers.resize(n_layers);
+    {
+        const rrm_layer_desc& d0 = descs[0];
+        if (d0.src != 0) return RRM_ERR_INVALID_ARG;
+        set_tensor(net->tensors[0], d0.dtype == RRM_F32 ? T_F32 : (d0.dtype == RRM_I8 ? T_I8 : T_BIN), n, d0.c_in, d0.h, d0.w);
+    }
+    for (int l = 0; l < n_layers; ++l) {
+        const rrm_layer_desc& d = descs[l];
+        RRM_TRY(validate_desc(d, l, n_layers));
+        if (d.n != n) return RRM_ERR_SHAPE;
+        if (!W[l]) return RRM_ERR_INVALID_ARG;
+        Layer& L = net->layers[l];
+        L.d = d;
+        L.oh = (d.h + 2 * d.pad - d.kh) / d.stride + 1;
+        L.ow = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+        L.th = L.oh; L.tw = L.ow;
+        if (d.pool_k > 0) {
+            if (L.oh + 2 * d.pool_p < d.pool_k || L.ow + 2 * d.pool_p < d.pool_k) return RRM_ERR_SHAPE;
+            L.th = (L.oh + 2 * d.pool_p - d.pool_k) / d.pool_s + 1;
+            L.tw = (L.ow + 2 * d.pool_p - d.pool_k) / d.pool_s + 1;
+        }
+        const Tensor& in = net->tensors[d.src];
+        const int want = d.dtype == RRM_F32 ? T_F32 : (d.dtype == RRM_I8 ? T_I8 : T_BIN);
+        if (in.dtype != want) return RRM_ERR_DTYPE;
+        if (in.c != d.c_in || in.h != d.h || in.w != d.w) return RRM_ERR_SHAPE;
+        int ot;
+        if (d.dtype == RRM_F32) ot = T_F32;
+        else if (d.act == RRM_ACT_SIGN) ot = T_BIN;
+        else if (d.shift >= 0) ot = T_I8;
+        else ot = T_I32;
+        set_tensor(net->tensors[l + 1], ot, n, d.c_out, L.th, L.tw);
+        if (d.res >= 0) {
+            const Tensor& r = net->tensors[d.res];
+            if (r.dtype != ot || r.c != d.c_out || r.h != L.th || r.w != L.tw) return RRM_ERR_SHAPE;
+        }
+        if ((long long)n * L.oh * L.ow * (long long)d.c_out > (1ll << 31) - 1) return RRM_ERR_CAPACITY;
+        if ((long long)n * d.h * d.w * (long long)in.cs > (1ll << 31) - 1) return RRM_ERR_CAPACITY;
+    }
+    // the fused FC kernel serves a lone int8 FC layer that reads the external input
+    bool fused = false;
+    if (n_layers == 1 && descs[0].kind == RRM_FC && descs[0].dtype == RRM_I8 && descs[0].pool_k == 0 &&
+        descs[0].act != RRM_ACT_SIGN && descs[0].variant != RRM_VARIANT_DENSE) {
+        const int s = fc_fused_create(net, net->layers[0], W[0], B ? B[0] : nullptr);
+        if (s == RRM_OK) fused = true;
+        else if (s != RRM_ERR_UNSUPPORTED) return s;
+    }
+    RRM_TRY(dev_alloc(net, (void**)&net->errw, 16));
+    if (fused) return RRM_OK;
+
+    // tensors
+    size_t cleared = 0;
+    for (auto& T : net->tensors) {
+        RRM_TRY(dev_alloc(net, &T.X, T.bytes()));
+        RRM_TRY(dev_alloc(net, &T.D, T.bytes()));
+        RRM_TRY(dev_alloc(net, (void**)&T.pnnz, (size_t)T.pixels() * 4));
+        cleared += (size_t)T.act_words() * 4;
+    }
+    for (auto& L : net->layers) cleared += (size_t)ceil_div(L.opixels(), 32) * 4;
+    cleared = (cleared + 15) & ~(size_t)15;
+    const size_t counters_off = cleared;
+    cleared += net->tensors.size() * 16 + net->layers.size() * 16;
+    RRM_TRY(dev_alloc(net, &net->cleared, cleared));
+    net->cleared_bytes = cleared;
+    char* base = reinterpret_cast<char*>(net->cleared);
+    size_t off = 0;
+    for (auto& T : net->tensors) { T.act = reinterpret_cast<uint32_t*>(base + off); off += (size_t)T.act_words() * 4; }
+    for (auto& L : net->layers) { L.oact = reinterpret_cast<uint32_t*>(base + off); off += (size_t)ceil_div(L.opixels(), 32) * 4; }
+    off = counters_off;
+    for (auto& T : net->tensors) {
+        T.nnz = reinterpret_cast<unsigned long long*>(base + off);
+        T.npix = reinterpret_cast<unsigned long long*>(base + off + 8);
+        off += 16;
+    }
+    for (auto& L : net->layers) {
+        L.macs = reinterpret_cast<unsigned long long*>(base + off);
+        L.ocount = reinterpret_cast<int*>(base + off + 8);
+        off += 16;
+    }
+    for (int l = 0; l < n_layers; ++l) RRM_TRY(conv_layer_create(net, net->layers[l], W[l], B ? B[l] : nullptr));
+    for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
+    RRM_TRY(reset_state(net, nullptr));
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
+    return RRM_OK;
+}
+
+int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
+{
+    if (!net || !frame) return RRM_ERR_INVALID_ARG;
+    net->last_stream = st;
+    if (net->layers[0].fc_fused) return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
+    if (!stateless) RRM_CUDA_TRY(cudaMemsetAsync(net->cleared, 0, net->cleared_bytes, st));
+    RRM_TRY(launch_import(net, frame, !dense, stateless, st));
+    for (int l = 0; l < (int)net->layers.size(); ++l) RRM_TRY(launch_layer(net, l, dense, stateless, st));
+    if (out) RRM_TRY(launch_export_tensor(net, (int)net->layers.size(), out, stateless, st));
+    return RRM_OK;
+}
+
+int ensure_stage(rrm_net* net)
+{
+    if (net->stage_in) return RRM_OK;
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    RRM_TRY(dev_alloc(net, &net->stage_in, (size_t)bi));
+    RRM_TRY(dev_alloc(net, &net->stage_out, (size_t)bo));
+    return RRM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rrm_net_create(rrm_net** out, const rrm_layer_desc* descs, int n_layers,
+                   const void* const* W_dev, const void* const* bias_dev)
+{
+    if (!out || !descs || n_layers < 1 || !W_dev) return RRM_ERR_INVALID_ARG;
+    *out = nullptr;
+    rrm_net* net = new (std::nothrow) rrm_net();
+    if (!net) return RRM_ERR_ALLOC;
+    int s;
+    try {
+        s = build_net(net, descs, n_layers, W_dev, bias_dev);
+    } catch (...) {
+        s = RRM_ERR_ALLOC;
+    }
+    if (s != RRM_OK) {
+        for (void* p : net->allocs) cudaFree(p);
+        delete net;
+        cudaGetLastError();
+        return s;
+    }
+    *out = net;
+    return RRM_OK;
+}
+
+int rrm_net_destroy(rrm_net* net)
+{
+    if (!net) return RRM_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    for (void* p : net->allocs) cudaFree(p);
+    delete net;
+    return RRM_OK;
+}
+
+int rrm_layer_create(rrm_layer** out, const rrm_layer_desc* desc, const void* W_dev, const void* bias_dev)
+{
+    if (!out || !desc) return RRM_ERR_INVALID_ARG;
+    rrm_layer_desc d = *desc;
+    d.src = 0;
+    d.res = -1;
+    const void* W[1] = {W_dev};
+    const void* B[1] = {bias_dev};
+    return rrm_net_create(out, &d, 1, W, B);
+}
+
+int rrm_layer_destroy(rrm_layer* layer) { return rrm_net_destroy(layer); }
+
+int rrm_net_keyframe(rrm_net* net, const void* frame_dev, void* out_dev, void* stream)
+{
+    return run(net, frame_dev, out_dev, (cudaStream_t)stream, true, false);
+}
+int rrm_net_step(rrm_net* net, const void* frame_dev, void* out_dev, void* stream)
+{
+    return run(net, frame_dev, out_dev, (cudaStream_t)stream, false, false);
+}
+int rrm_net_dense(rrm_net* net, const void* frame_dev, void* out_dev, void* stream)
+{
+    return run(net, frame_dev, out_dev, (cudaStream_t)stream, true, true);
+}
+int rrm_keyframe(rrm_layer* layer, const void* X0_dev, void* Y0_dev, void* stream)
+{
+    return rrm_net_keyframe(layer, X0_dev, Y0_dev, stream);
+}
+int rrm_step(rrm_layer* layer, const void* Xt_dev, void* Yt_dev, void* stream)
+{
+    return rrm_net_step(layer, Xt_dev, Yt_dev, stream);
+}
+int rrm_dense(rrm_layer* layer, const void* X_dev, void* Y_dev, void* stream)
+{
+    return rrm_net_dense(layer, X_dev, Y_dev, stream);
+}
+
+int rrm_net_step_host(rrm_net* net, const void* frame_host, void* out_host, void* stream)
+{
+    if (!net || !frame_host) return RRM_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    RRM_TRY(ensure_stage(net));
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    RRM_CUDA_TRY(cudaMemcpyAsync(net->stage_in, frame_host, (size_t)bi, cudaMemcpyHostToDevice, st));
+    RRM_TRY(run(net, net->stage_in, out_host ? net->stage_out : nullptr, st, false, false));
+    if (out_host) RRM_CUDA_TRY(cudaMemcpyAsync(out_host, net->stage_out, (size_t)bo, cudaMemcpyDeviceToHost, st));
+    RRM_CUDA_TRY(cudaStreamSynchronize(st));
+    return RRM_OK;
+}
+int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* stream)
+{
+    return rrm_net_step_host(layer, Xt_host, Yt_host, stream);
+}
+
+int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
+{
+    if (!net || !h || layer < 0 || layer >= (int)net->layers.size()) return RRM_ERR_INVALID_ARG;
+    RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
+    std::memset(h, 0, sizeof(*h));
+    const Layer& L = net->layers[layer];
+    const rrm_layer_desc& d = L.d;
+    const int oh = (d.h + 2 * d.pad - d.kh) / d.stride + 1, ow = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+    h->in_elems = (int64_t)d.n * d.c_in * d.h * d.w;
+    h->out_pixels = (int64_t)d.n * oh * ow;
+    h->dense_macs = h->out_pixels * d.c_out * d.c_in * d.kh * d.kw;
+    int errw = 0;
+    RRM_CUDA_TRY(cudaMemcpy(&errw, net->errw, 4, cudaMemcpyDeviceToHost));
+    h->error_word = errw;
+    if (L.fc_fused) {
+        unsigned long long tot[2] = {0, 0};
+        std::vector<unsigned long long> v((size_t)d.n * 2);
+        RRM_CUDA_TRY(cudaMemcpy(v.data(), L.fc_nnz, v.size() * 8, cudaMemcpyDeviceToHost));
+        for (int s = 0; s < d.n; ++s) { tot[0] += v[s * 2]; tot[1] += v[s * 2 + 1]; }
+        h->nnz_elems = (int64_t)tot[0];
+        h->in_pixels = (int64_t)d.n * ((d.c_in + 31) / 32);
+        h->active_in_pixels = (int64_t)tot[1];
+        h->active_out_pixels = tot[0] ? d.n : 0;
+        h->active_macs = (int64_t)tot[0] * d.c_out;
+        h->variant = RRM_VARIANT_GATHER;
+        return RRM_OK;
+    }
+    const Tensor& in = net->tensors[d.src];
+    unsigned long long v[2] = {0, 0};
+    RRM_CUDA_TRY(cudaMemcpy(v, in.nnz, 16, cudaMemcpyDeviceToHost));
+    h->nnz_elems = (int64_t)v[0];
+    h->active_in_pixels = (int64_t)v[1];
+    h->in_pixels = in.pixels();
+    unsigned long long m = 0;
+    int oc = 0;
+    RRM_CUDA_TRY(cudaMemcpy(&m, L.macs, 8, cudaMemcpyDeviceToHost));
+    RRM_CUDA_TRY(cudaMemcpy(&oc, L.ocount, 4, cudaMemcpyDeviceToHost));
+    h->active_macs = (int64_t)m;
+    h->active_out_pixels = oc;
+    h->variant = RRM_VARIANT_GATHER;
+    return RRM_OK;
+}
+int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out) { return rrm_net_get_stats(layer, 0, host_out); }
+
+int rrm_net_projection(rrm_net* net, int layer, void* P_dev, void* stream)
+{
+    if (!net || !P_dev || layer < 0 || layer >= (int)net->layers.size()) return RRM_ERR_INVALID_ARG;
+    if (net->layers[layer].fc_fused) return fc_fused_projection(net, net->layers[layer], P_dev, (cudaStream_t)stream);
+    return launch_export_projection(net, layer, P_dev, (cudaStream_t)stream);
+}
+int rrm_layer_projection(rrm_layer* layer, void* P_dev, void* stream) { return rrm_net_projection(layer, 0, P_dev, stream); }
+
+int rrm_net_tensor(rrm_net* net, int t, void* dst_dev, void* stream)
+{
+    if (!net || !dst_dev || t < 0 || t >= (int)net->tensors.size()) return RRM_ERR_INVALID_ARG;
+    if (net->layers[0].fc_fused) return RRM_ERR_UNSUPPORTED;
+    return launch_export_tensor(net, t, dst_dev, false, (cudaStream_t)stream);
+}
+
+int64_t rrm_net_tensor_bytes(const rrm_net* net, int t)
+{
+    if (!net || t < 0 || t >= (int)net->tensors.size()) return RRM_ERR_INVALID_ARG;
+    int64_t b = 0;
+    tensor_bytes_boundary(net->tensors[t], &b);
+    return b;
+}
+
+const char* rrm_strerror(int status)
+{
+    switch (status) {
+        case RRM_OK: return "ok";
+        case RRM_ERR_INVALID_ARG: return "invalid argument";
+        case RRM_ERR_SHAPE: return "shape mismatch";
+        case RRM_ERR_DTYPE: return "dtype mismatch";
+        case RRM_ERR_ALLOC: return "device allocation failed";
+        case RRM_ERR_CAPACITY: return "size exceeds the library's index range";
+        case RRM_ERR_TIMEOUT: return "bounded device wait ran out";
+        case RRM_ERR_CUDA: return "CUDA runtime error";
+        case RRM_ERR_UNSUPPORTED: return "unsupported combination";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

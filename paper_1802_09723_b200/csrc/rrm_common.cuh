@@ -1,0 +1,110 @@
+// Internal declarations shared by the translation units of the RRM library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <vector>
+#include "../../include/rrm.h"
+
+#define RRM_CUDA_TRY(expr)                                   \
+    do {                                                     \
+        cudaError_t e__ = (expr);                            \
+        if (e__ != cudaSuccess) return RRM_ERR_CUDA;         \
+    } while (0)
+
+#define RRM_TRY(expr)                                        \
+    do {                                                     \
+        int s__ = (expr);                                    \
+        if (s__ != RRM_OK) return s__;                       \
+    } while (0)
+
+namespace rrm {
+
+// storage type of a tensor inside the library (always pixel-major: [n][h][w][cs])
+enum { T_F32 = 0, T_I8 = 1, T_BIN = 2, T_I32 = 3 };
+
+// device error flags (rrm_stats.error_word)
+enum { ERRW_BOUNDS = 1, ERRW_TIMEOUT = 2, ERRW_CAPACITY = 4 };
+
+// tile shape of the CUDA-core implicit GEMM (units: float, 4 x int8, or 32 sign bits)
+constexpr int GEMM_TN = 64;   // output channels per CTA
+constexpr int GEMM_TK = 16;   // K units per stage
+
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
+
+struct Tensor {
+    int dtype = T_F32;
+    int n = 0, c = 0, h = 0, w = 0;
+    int cs = 0;                       // storage units per pixel (f32/i32: c; i8: c rounded up to 4; bin: words)
+    int unit_bytes = 4;               // bytes per storage unit (i8: 1)
+    void* X = nullptr;                // current value (= snapshot of the previous frame before a step)
+    void* D = nullptr;                // delta rows, valid only for pixels whose `act` bit is set
+    uint32_t* act = nullptr;          // bitmap over n*h*w pixels (cleared every step)
+    int* pnnz = nullptr;              // per-pixel count of non-zero delta elements (valid where act is set)
+    unsigned long long* nnz = nullptr;      // total non-zero delta elements (cleared every step)
+    unsigned long long* npix = nullptr;     // active pixels (cleared every step)
+    void* X2 = nullptr;               // value buffer of the stateless dense path
+    bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
+    int pixels() const { return n * h * w; }
+    size_t row_bytes() const { return (size_t)cs * unit_bytes; }
+    size_t bytes() const { return (size_t)pixels() * row_bytes(); }
+    int act_words() const { return ceil_div(pixels(), 32); }
+};
+
+struct Layer {
+    rrm_layer_desc d;
+    int oh = 0, ow = 0;               // projection spatial size
+    int th = 0, tw = 0;               // output tensor spatial size (after pooling)
+    int u_in = 0;                     // storage units per input pixel
+    int ku = 0, kup = 0;              // K in units, and padded to GEMM_TK
+    int np = 0;                       // c_out padded to GEMM_TN
+    void* Wk = nullptr;               // packed filters [kup][np] units
+    void* bias = nullptr;             // float or int32 [c_out]
+    void* P = nullptr;                // projection [n*oh*ow][c_out] float or int32
+    void* P2 = nullptr;               // projection buffer of the stateless dense path
+    uint32_t* oact = nullptr;         // bitmap of updated projection pixels (cleared every step)
+    int* olist = nullptr;             // compacted ids of those pixels
+    int* ocount = nullptr;            // their number (cleared every step)
+    unsigned long long* macs = nullptr;     // exact active multiply-accumulates (cleared every step)
+    int opixels() const { return d.n * oh * ow; }
+    // fused FC path (int8 FC reading the external input)
+    bool fc_fused = false;
+    int8_t* Wt = nullptr;             // [c_in][c_out] transposed weights
+    int8_t* xs[2] = {nullptr, nullptr};     // ping-pong input snapshots [n][c_in]
+    int xs_cur = 0;
+    unsigned int* fc_counters = nullptr;    // arrival counters per (stream, output slice)
+    unsigned long long* fc_nnz = nullptr;   // [0] nnz elements, [1] active groups of 32 (cleared by the kernel's last CTA)
+};
+
+}  // namespace rrm
+
+struct rrm_net {
+    std::vector<rrm::Layer> layers;
+    std::vector<rrm::Tensor> tensors;
+    int n = 1;
+    void* cleared = nullptr;          // arena zeroed at the start of every step
+    size_t cleared_bytes = 0;
+    int* errw = nullptr;              // device error word
+    cudaStream_t last_stream = nullptr;
+    void* stage_in = nullptr;         // device staging for the *_host entry points
+    void* stage_out = nullptr;
+    std::vector<void*> allocs;        // everything to free
+};
+
+namespace rrm {
+
+// ---- rrm_fc.cu
+int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);
+int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool dense, bool stateless,
+                 cudaStream_t st);
+int fc_fused_projection(rrm_net* net, Layer& L, void* P_dev, cudaStream_t st);
+
+// ---- rrm_conv.cu
+int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);
+int launch_import(rrm_net* net, const void* frame_dev, bool delta, bool stateless, cudaStream_t st);
+int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st);
+int launch_export_tensor(rrm_net* net, int t, void* dst_dev, bool stateless, cudaStream_t st);
+int launch_export_projection(rrm_net* net, int l, void* dst_dev, cudaStream_t st);
+int reset_state(rrm_net* net, cudaStream_t st);
+
+}  // namespace rrm

@@ -1,0 +1,207 @@
+"""GPU parity of the convolution path (single layers and layer stacks) against the CPU oracle.
+Integer and binary layers must match bit for bit; fp32 layers within 1e-4 * max|P_dense| per
+frame (the accumulated projection is compared at every frame, so drift would show)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from workloads.nets import LayerSpec, out_hw
+from oracle import rrm_oracle as orc
+from helpers import dev, pack_bits_nhwc, unpack_bits_nhwc
+
+pytestmark = pytest.mark.gpu
+F32_TOL = 1e-4
+
+
+def _rrm():
+    import paper_1802_09723_b200 as rrm
+    return rrm
+
+
+def _frame_to_dev(specs, frame):
+    if specs[0].dtype == "bin":
+        return dev(pack_bits_nhwc(frame).view(np.int32))
+    return dev(frame)
+
+
+def _out_kind(s):
+    if s.dtype == "f32":
+        return "f32"
+    if s.act == "sign":
+        return "bin"
+    return "i8" if s.shift >= 0 else "i32"
+
+
+def _compare(specs, net, frame, t, check_tensors=True):
+    tens_d, P_d = orc.dense_forward(specs, frame)
+    for l, s in enumerate(specs):
+        P = net.projection(l).cpu().numpy()
+        if s.dtype == "f32":
+            scale = float(np.abs(P_d[l]).max())
+            err = float(np.abs(P.astype(np.float64) - P_d[l]).max())
+            assert err <= F32_TOL * scale, f"frame {t} layer {l} ({s.name}): err {err:.3e} scale {scale:.3e}"
+        else:
+            np.testing.assert_array_equal(P.astype(np.int64), P_d[l], err_msg=f"frame {t} layer {l} ({s.name})")
+        if not check_tensors:
+            continue
+        T = net.tensor(l + 1).cpu().numpy()
+        kind = _out_kind(s)
+        if kind == "bin":
+            np.testing.assert_array_equal(unpack_bits_nhwc(T.view(np.uint32), s.c_out), tens_d[l + 1],
+                                          err_msg=f"frame {t} tensor {l + 1}")
+        elif kind == "f32":
+            scale = max(1e-30, float(np.abs(tens_d[l + 1]).max()))
+            assert float(np.abs(T - tens_d[l + 1]).max()) <= F32_TOL * max(scale, float(np.abs(P_d[l]).max()))
+        else:
+            np.testing.assert_array_equal(T.astype(np.int64), tens_d[l + 1], err_msg=f"frame {t} tensor {l + 1}")
+
+
+def _run(specs, video, n=1, check_frames=None, stats=False, keyframe_at=(), variant="auto"):
+    rrm = _rrm()
+    net = rrm.net_from_specs(specs, n=n, variant=variant)
+    out = net.new_output()
+    rec = orc.Recurrence(specs, n=n) if stats else None
+    if rec is not None:
+        # a fresh library state is the stack's response to the all-zero input pattern (all -1 for a
+        # binary input); bring the literal recurrence to the same state
+        rec.step(np.full_like(video[0], -1 if specs[0].dtype == "bin" else 0))
+    for t in range(video.shape[0]):
+        x = _frame_to_dev(specs, video[t])
+        if t in keyframe_at:
+            net.keyframe(x, out)
+        else:
+            net.step(x, out)
+        if rec is not None:
+            rec.step(video[t])
+            if t not in keyframe_at:
+                for l in range(len(specs)):
+                    st = net.stats(l)
+                    assert st["error_word"] == 0
+                    if specs[0].dtype != "f32" or l == 0:
+                        assert st["nnz_elems"] == rec.nnz[l], (t, l, st, rec.nnz[l])
+                        assert st["active_macs"] == rec.macs[l], (t, l, st, rec.macs[l])
+        if check_frames is None or t in check_frames:
+            _compare(specs, net, video[t], t)
+            # the caller-owned output equals the last tensor
+            last = net.tensor(len(specs))
+            assert torch.equal(out, last)
+    net.close()
+
+
+# ------------------------------------------------------------------ config 1
+def test_cfg1_single_conv_fp32_all_frames():
+    specs = wl.single_conv_f32()
+    video = wl.block_redraw_sequence()
+    _run(specs, video, stats=True)
+
+
+def _spec(dtype, c_in, hw, c_out, k, s, p, rng, **kw):
+    sp = LayerSpec("conv", dtype, c_in, hw[0], hw[1], c_out, k, k, s, p, src=0, **kw)
+    if dtype == "f32":
+        sp.weight = rng.standard_normal((c_out, c_in, k, k)).astype(np.float32) * np.float32(0.1)
+        sp.bias = rng.standard_normal(c_out).astype(np.float32)
+    elif dtype == "i8":
+        sp.weight = rng.integers(-127, 128, size=(c_out, c_in, k, k)).astype(np.int8)
+        sp.bias = rng.integers(-500, 501, size=c_out).astype(np.int32)
+    else:
+        sp.weight = (rng.integers(0, 2, size=(c_out, c_in, k, k)) * 2 - 1).astype(np.int8)
+        sp.bias = rng.integers(-5, 6, size=c_out).astype(np.int32)
+    return sp
+
+
+def _video(dtype, c, hw, frames, n, rng):
+    kind = {"f32": "f32_relu", "i8": "i8", "bin": "pm1"}[dtype]
+    h, w = hw
+    seq = wl.block_redraw_sequence(frames=frames, c=c, hw=max(h, w), frac=0.08, block=3, dtype=kind,
+                                   seed=int(rng.integers(1, 1 << 30)), n=n)[:, :, :, :h, :w].copy()
+    seq[2] = seq[1]                                  # zero delta
+    if dtype == "bin":
+        seq[3] = -seq[2]                             # every element changes
+    elif dtype == "i8":
+        seq[3] = 127 - seq[2]
+    else:
+        seq[3] = seq[2] + np.float32(0.5)
+    return seq
+
+
+@pytest.mark.parametrize("dtype", ["f32", "i8", "bin"])
+@pytest.mark.parametrize("c_in,c_out,hw,k,s,p", [
+    (3, 5, (9, 11), 3, 1, 1), (16, 70, (13, 13), 3, 1, 1), (8, 12, (17, 15), 5, 2, 2), (5, 9, (12, 12), 1, 1, 0),
+    (4, 8, (20, 19), 1, 2, 0), (3, 6, (35, 35), 11, 4, 0), (3, 8, (30, 30), 7, 2, 3), (40, 33, (7, 7), 3, 1, 0),
+    (64, 16, (10, 10), 3, 1, 1)])
+def test_single_layer_shapes(dtype, c_in, c_out, hw, k, s, p):
+    rng = np.random.default_rng(c_in * 1000 + c_out * 10 + k)
+    sp = _spec(dtype, c_in, hw, c_out, k, s, p, rng)
+    video = _video(dtype, c_in, hw, 5, 2, rng)
+    _run([sp], video, n=2, stats=True)
+
+
+@pytest.mark.parametrize("dtype,act,pool,shift", [
+    ("f32", "relu", (3, 2, 0), -1), ("f32", "relu", (3, 2, 1), -1), ("f32", "none", (2, 2, 0), -1),
+    ("i8", "relu", (3, 2, 0), 9), ("i8", "none", None, 10), ("i8", "sign", (3, 2, 0), -1), ("i8", "none", (3, 2, 1), -1),
+    ("bin", "sign", None, -1), ("bin", "sign", (3, 2, 0), -1), ("bin", "none", (3, 2, 0), -1)])
+def test_single_layer_nonlinearities(dtype, act, pool, shift):
+    rng = np.random.default_rng(77)
+    sp = _spec(dtype, 12, (15, 14), 40, 3, 1, 1, rng, act=act, pool=pool, shift=shift, theta=3)
+    video = _video(dtype, 12, (15, 14), 5, 1, rng)
+    _run([sp], video, n=1, stats=True)
+
+
+def test_keyframe_resets_state_and_dense_path_is_stateless():
+    rrm = _rrm()
+    specs = wl.single_conv_f32(c_in=8, c_out=8, hw=20)
+    video = wl.block_redraw_sequence(frames=6, c=8, hw=20, seed=3)
+    _run(specs, video, keyframe_at=(0, 3))
+    net = rrm.net_from_specs(specs)
+    out, outd = net.new_output(), net.new_output()
+    net.step(dev(video[0]), out)
+    net.dense(dev(video[4]), outd)
+    ref = orc.dense_forward(specs, video[4])[0][1]
+    assert np.abs(outd.cpu().numpy() - ref).max() <= F32_TOL * np.abs(ref).max()
+    net.step(dev(video[1]), out)
+    ref = orc.dense_forward(specs, video[1])[0][1]
+    assert np.abs(out.cpu().numpy() - ref).max() <= F32_TOL * np.abs(ref).max()
+    net.close()
+
+
+# ------------------------------------------------------------------ small stacks, every frame, with stats
+@pytest.mark.parametrize("name", ["alex_f32", "alex_i8", "resnet_i8", "xnor"])
+def test_small_stacks_every_frame(name):
+    if name == "alex_f32":
+        specs, dt, hw = wl.alexnet_convs("f32", hw=99, scale=8), "f32", 99
+    elif name == "alex_i8":
+        specs, dt, hw = wl.alexnet_convs("i8", hw=99, scale=8), "i8", 99
+    elif name == "resnet_i8":
+        specs, dt, hw = wl.resnet18_convs(hw=96, scale=8), "i8", 96
+    else:
+        specs, dt, hw = wl.xnor_alexnet_convs(hw=99, scale=8), "i8", 99
+    n = 2 if name == "resnet_i8" else 1
+    video = wl.moving_rect_video(frames=6, hw=hw, dtype=dt, seed=9, n=n, side=(12, 24),
+                                 bg_redraw=0.02 if name == "resnet_i8" else 0.0)
+    _run(specs, video, n=n, stats=True, keyframe_at=(4,))
+
+
+# ------------------------------------------------------------------ full-size configs, sampled frames
+def test_cfg3_alexnet_fp32_full_size():
+    specs = wl.alexnet_convs("f32")
+    video = wl.moving_rect_video(frames=64, hw=227, dtype="f32", seed=31)
+    _run(specs, video, check_frames={0, 1, 2, 17, 63})
+
+
+def test_cfg3_alexnet_int8_full_size():
+    specs = wl.alexnet_convs("i8")
+    video = wl.moving_rect_video(frames=64, hw=227, dtype="i8", seed=32)
+    _run(specs, video, check_frames={0, 1, 30, 63})
+
+
+def test_cfg4_resnet18_int8_batch4():
+    specs = wl.resnet18_convs()
+    video = wl.moving_rect_video(frames=64, hw=224, dtype="i8", seed=41, n=4, bg_redraw=0.02)
+    _run(specs, video, n=4, check_frames={0, 1, 63})
+
+
+def test_cfg5_xnor_alexnet_128_frames():
+    specs = wl.xnor_alexnet_convs()
+    video = wl.moving_rect_video(frames=128, hw=227, dtype="i8", seed=51)
+    _run(specs, video, check_frames={0, 1, 64, 127})

@@ -1,0 +1,105 @@
+"""GPU parity of the fused delta-FC path against the CPU oracle (bit-exact int32)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from workloads.nets import LayerSpec
+from oracle import rrm_oracle as orc
+from helpers import dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _rrm():
+    import paper_1802_09723_b200 as rrm
+    return rrm
+
+
+def _run_sequence(spec, seq, n, keyframe_first=False):
+    rrm = _rrm()
+    layer = rrm.layer_from_spec(spec, n=n)
+    rec = orc.Recurrence([spec], n=n)
+    Y = layer.new_output()
+    for t in range(seq.shape[0]):
+        x = dev(seq[t])
+        if t == 0 and keyframe_first:
+            layer.keyframe(x, Y)
+        else:
+            layer.step(x, Y)
+        tens_d, P_d = orc.dense_forward([spec], seq[t])
+        got = Y.cpu().numpy().astype(np.int64)
+        np.testing.assert_array_equal(got, tens_d[1].astype(np.int64), err_msg=f"frame {t}")
+        np.testing.assert_array_equal(layer.projection(0).cpu().numpy().astype(np.int64), P_d[0])
+        rec.step(seq[t])
+        if not (t == 0 and keyframe_first):
+            st = layer.stats(0)
+            assert st["nnz_elems"] == rec.nnz[0], (t, st)
+            assert st["active_macs"] == rec.macs[0]
+            assert st["error_word"] == 0
+    layer.close()
+
+
+@pytest.mark.parametrize("rho", [0.01, 0.05, 0.20])
+def test_fc6_int8_all_frames_bit_exact(rho):
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=32, rho=rho, seed=21)
+    _run_sequence(spec, seq, 1)
+
+
+def test_fc6_keyframe_then_steps_and_two_streams():
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=6, rho=0.05, seed=22, n=2)
+    _run_sequence(spec, seq, 2, keyframe_first=True)
+
+
+@pytest.mark.parametrize("c_in,c_out,shift,act", [(64, 48, -1, "none"), (160, 528, 6, "relu"),
+                                                  (1024 + 32, 16, 5, "none"), (32, 1040, -1, "none")])
+def test_fc_small_and_ragged_shapes(c_in, c_out, shift, act):
+    rng = np.random.default_rng(c_in + c_out)
+    spec = LayerSpec("fc", "i8", c_in, 1, 1, c_out, act=act, shift=shift, src=0)
+    spec.weight = rng.integers(-127, 128, size=(c_out, c_in, 1, 1)).astype(np.int8)
+    spec.bias = rng.integers(-500, 501, size=c_out).astype(np.int32)
+    seq = wl.fc_run_sequence(frames=5, c_in=c_in, rho=0.25, run=8, seed=c_in, n=3)
+    seq[3] = seq[2]                       # a frame with zero delta
+    seq[4] = 127 - seq[3]                 # every entry changes, deltas up to +-127
+    _run_sequence(spec, seq, 3)
+
+
+def test_fc_full_range_inputs_need_split_deltas():
+    """Inputs spanning [-127,127] give deltas up to +-254, beyond one int8 factor."""
+    rng = np.random.default_rng(9)
+    spec = LayerSpec("fc", "i8", 96, 1, 1, 64, src=0)
+    spec.weight = rng.integers(-127, 128, size=(64, 96, 1, 1)).astype(np.int8)
+    spec.bias = np.zeros(64, dtype=np.int32)
+    a = rng.integers(-127, 128, size=(1, 96)).astype(np.int8)
+    seq = np.stack([a, (-a).astype(np.int8), a])
+    seq[1, 0, :4] = [127, -127, 127, -127]
+    seq[2, 0, :4] = [-127, 127, -127, 127]
+    _run_sequence(spec, seq, 1)
+
+
+def test_fc_dense_path_leaves_state_untouched():
+    rrm = _rrm()
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=3, rho=0.05, seed=23)
+    layer = rrm.layer_from_spec(spec)
+    Y, Yd = layer.new_output(), layer.new_output()
+    layer.step(dev(seq[0]), Y)
+    layer.dense(dev(seq[2]), Yd)          # unrelated frame through the dense path
+    np.testing.assert_array_equal(Yd.cpu().numpy(), orc.dense_forward([spec], seq[2])[0][1])
+    layer.step(dev(seq[1]), Y)            # state must still be that of frame 0
+    np.testing.assert_array_equal(Y.cpu().numpy(), orc.dense_forward([spec], seq[1])[0][1])
+    layer.close()
+
+
+def test_fc_step_host_matches_device_call():
+    rrm = _rrm()
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=3, rho=0.2, seed=24)
+    layer = rrm.layer_from_spec(spec)
+    out = torch.empty((1, 4096, 1, 1), dtype=torch.int32).pin_memory()
+    for t in range(3):
+        layer.step_host(torch.from_numpy(seq[t]).pin_memory(), out)
+        np.testing.assert_array_equal(out.numpy(), orc.dense_forward([spec], seq[t])[0][1])
+    layer.close()
