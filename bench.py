@@ -234,7 +234,7 @@ def main():
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     xh = [torch.from_numpy(seq[t]).pin_memory() for t in range(FRAMES)]
     yh = torch.empty((1, C_OUT, 1, 1), dtype=torch.int32).pin_memory()
-    e2e_steps = min(args.steps, 310)
+    e2e_steps = 10 if args.quick else min(args.steps, 310)
     for i in range(5):
         layer.step_host(xh[order[(i + 1) % len(order)]], yh)
     barrier()
@@ -275,7 +275,7 @@ def main():
 
     # ---- CPU oracle on the host cores (rank 0, N = 1 only): a bounded sample of the same workload
     cpu = None
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.quick:
         from oracle import rrm_oracle as orc
         rec = orc.Recurrence([spec])
         rec.step(seq[0])

@@ -1,25 +1,38 @@
 // Fused delta-FC step for int8 layers (Algorithm 1, FC branch; Sec. 3.5 column products).
 //
-// One launch does the whole frame of one FC layer:
-//   1. every CTA scans X_t against the snapshot with 128-bit loads and builds, by ballot-free
-//      per-chunk counts + a block prefix sum, the ordered list of non-zero delta entries;
-//   2. the list is split evenly over the CTAs of a column group; each CTA gathers only the
-//      weight columns W[:, j] of its entries (weights are stored transposed, one contiguous
-//      C_out-byte row per input j) and accumulates d_j * W[:, j] in int32;
-//   3. partial sums are added into the stored projection P with integer atomics (exact,
-//      order-independent);
-//   4. the last CTA to finish an output slice applies f and writes Y_t; CTA 0 of a stream
-//      writes the new snapshot into the other half of a ping-pong pair.
+// One launch does the whole frame of one FC layer.  The grid is made of clusters of FC_CL CTAs;
+// a cluster owns FC_OW consecutive outputs of one stream:
+//   1. every CTA scans X_t against the snapshot with 128-bit loads (all loads issued up front) and
+//      finds, by per-thread counts and a block prefix sum, its share of the ordered list of
+//      non-zero delta entries (the list is split evenly over the CTAs of the cluster);
+//   2. each CTA gathers only the weight columns W[:, j] of its entries (weights are stored
+//      transposed, one contiguous C_out-byte row per input j) and accumulates d_j * W[:, j] in int32;
+//   3. partial sums are reduced inside the CTA, then across the cluster through distributed shared
+//      memory; CTA 0 of the cluster adds them onto the stored projection P (owner computes, no
+//      atomics), applies f and writes Y_t;
+//   4. one CTA per stream writes the new snapshot into the other half of a ping-pong pair.
 // Cost is HBM-bound: nnz * C_out weight bytes per frame.
 #include "rrm_common.cuh"
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
+
+// Optional phase timestamps for tuning builds (-DRRM_FC_TIMING): CTA (0,0,0) stores clock64() per phase.
+#ifdef RRM_FC_TIMING
+__device__ long long rrm_fc_phase_clock[16];
+#define RRM_FC_PHASE(i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) rrm_fc_phase_clock[i] = clock64(); } while (0)
+#else
+#define RRM_FC_PHASE(i) do { } while (0)
+#endif
 
 namespace rrm {
 
 constexpr int FC_THREADS = 256;
-constexpr int FC_OW = 512;                 // outputs per CTA (32 lanes x 16 bytes)
-constexpr int FC_GROUPS = FC_THREADS / 32; // column groups working in parallel inside a CTA
-constexpr int FC_LCAP = 1024;              // list entries one CTA can own
-constexpr int FC_MAX_CHUNKS = 4096;        // 16-byte chunks of one input row (C_in <= 65536)
+constexpr int FC_CL = 8;                   // CTAs per cluster = split of the non-zero list
+constexpr int FC_OW = 128;                 // outputs per cluster (8 lanes x 16 bytes)
+constexpr int FC_GROUPS = FC_THREADS / 8;  // columns gathered in parallel inside a CTA
+constexpr int FC_LCAP = 2048;              // list entries one CTA can own  (C_in <= FC_CL * FC_LCAP)
+constexpr int FC_PT = 4;                   // 16-byte chunks scanned per thread (C_in <= 16 * FC_PT * FC_THREADS)
 
 struct FcParams {
     const int8_t* xt;        // [n][c_in]
@@ -28,9 +41,8 @@ struct FcParams {
     const int8_t* Wt;        // [c_in][c_out]
     int32_t* P;              // [n][c_out]
     void* Y;                 // [n][c_out] int32 or int8, or nullptr
-    unsigned int* counters;  // [n][slices]
     unsigned long long* stat;// [n][2]: nnz elements, active groups of 32 inputs (or nullptr)
-    int c_in, c_out, ksplit, shift, act;
+    int c_in, c_out, shift, act;
 };
 
 __device__ __forceinline__ int fc_apply_f(int v, int shift, int act) {
@@ -40,37 +52,77 @@ __device__ __forceinline__ int fc_apply_f(int v, int shift, int act) {
     return v;
 }
 
-__global__ void __launch_bounds__(FC_THREADS) fc_delta_i8_kernel(FcParams p)
+// Split cluster barrier.  Every thread alternates arrive and wait; a thread may exit after an arrive.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+__global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_delta_i8_kernel(FcParams p)
 {
     __shared__ int s_warp[FC_THREADS / 32];
-    __shared__ int s_list_j[FC_LCAP];
-    __shared__ int s_list_d[FC_LCAP];
-    __shared__ int s_red[FC_GROUPS][FC_OW];
-    __shared__ int s_flag;
+    __shared__ int s_off[FC_THREADS];
+    __shared__ unsigned long long s_mask[FC_THREADS];
+    __shared__ unsigned short s_list_j[FC_LCAP];   // C_in <= 16384 fits 16 bits
+    __shared__ __align__(16) int8_t s_xt[16 * FC_PT * FC_THREADS];
+    __shared__ __align__(16) int8_t s_xp[16 * FC_PT * FC_THREADS];
+    __shared__ int s_red[FC_THREADS / 32][FC_OW];
+    __shared__ int s_part[FC_CL][FC_OW];          // used in rank 0 only: partial sums pushed by every rank
 
-    const int tid = threadIdx.x;
-    const int kg = blockIdx.x, slice = blockIdx.y, s = blockIdx.z;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int kg = blockIdx.x;                       // rank inside the cluster (cluster spans x)
+    const int slice = blockIdx.y, s = blockIdx.z;
     const int C = p.c_in, K = p.c_out;
     const int nchunks = C >> 4;
     const uint4* xt4 = reinterpret_cast<const uint4*>(p.xt + (size_t)s * C);
     const uint4* xp4 = p.xprev ? reinterpret_cast<const uint4*>(p.xprev + (size_t)s * C) : nullptr;
+    int32_t* Ps = p.P + (size_t)s * K + slice * FC_OW;
+    const int width = min(FC_OW, K - slice * FC_OW);
 
-    // ---- 1. count non-zero delta bytes per 16-byte chunk; each thread owns a contiguous range of chunks
-    const int per_thread = (nchunks + FC_THREADS - 1) / FC_THREADS;
-    const int c_begin = min(nchunks, tid * per_thread), c_end = min(nchunks, c_begin + per_thread);
-    int local = 0;
-    for (int c = c_begin; c < c_end; ++c) {
-        if (xp4) {
-            const uint4 a = __ldg(xt4 + c), b = __ldg(xp4 + c);
-            // a byte differs <=> its delta is non-zero
-            auto nzb = [](unsigned v) { v |= v >> 4; v |= v >> 2; v |= v >> 1; return __popc(v & 0x01010101u); };
-            local += nzb(a.x ^ b.x) + nzb(a.y ^ b.y) + nzb(a.z ^ b.z) + nzb(a.w ^ b.w);
-        } else {
-            local += 16;
+    RRM_FC_PHASE(0);
+    cluster_arrive_relaxed();                        // waited for just before the first remote store
+    // stored projection of this slice: fetched now, needed at the very end
+    int p_old = 0;
+    if (kg == 0 && tid < width) p_old = Ps[tid];
+
+    // ---- 1. non-zero delta bytes per 16-byte chunk; each thread owns FC_PT consecutive chunks
+    const int c_begin = tid * FC_PT;
+    uint4 xa[FC_PT], xb[FC_PT];
+    #pragma unroll
+    for (int i = 0; i < FC_PT; ++i) {
+        xa[i] = make_uint4(0, 0, 0, 0);
+        xb[i] = xa[i];
+        if (c_begin + i < nchunks) {
+            xa[i] = __ldg(xt4 + c_begin + i);
+            if (xp4) xb[i] = __ldg(xp4 + c_begin + i);
         }
     }
+    RRM_FC_PHASE(1);
+    // raw bytes to shared memory (the gather looks the delta of an entry up there) and a 64-bit mask
+    // of the non-zero delta bytes of this thread's 64 inputs (a byte differs <=> its delta is non-zero)
+    unsigned long long m = 0;
+    #pragma unroll
+    for (int i = 0; i < FC_PT; ++i) {
+        if (c_begin + i < nchunks) {
+            reinterpret_cast<uint4*>(s_xt)[c_begin + i] = xa[i];
+            reinterpret_cast<uint4*>(s_xp)[c_begin + i] = xb[i];
+            unsigned cm;
+            if (xp4) {
+                auto nib = [](unsigned v) {           // one flag bit per non-zero byte, packed into 4 bits
+                    v |= v >> 4; v |= v >> 2; v |= v >> 1;
+                    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
+                };
+                cm = nib(xa[i].x ^ xb[i].x) | nib(xa[i].y ^ xb[i].y) << 4 | nib(xa[i].z ^ xb[i].z) << 8 |
+                     nib(xa[i].w ^ xb[i].w) << 12;
+            } else {
+                cm = 0xffffu;
+            }
+            m |= (unsigned long long)cm << (16 * i);
+        }
+    }
+    const int local = __popcll(m);
     // block exclusive scan of `local`
-    const int lane = tid & 31, warp = tid >> 5;
     int incl = local;
     #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -86,144 +138,140 @@ __global__ void __launch_bounds__(FC_THREADS) fc_delta_i8_kernel(FcParams p)
         if (w < warp) warp_off += v;
         total += v;
     }
-    int offset = warp_off + incl - local;          // index of this thread's first entry in the global list
+    int offset = warp_off + incl - local;          // index of this thread's first entry in the ordered list
 
-    // ---- 2. this CTA's share of the ordered list
-    const int per_cta = (total + p.ksplit - 1) / p.ksplit;
+    s_off[tid] = offset;
+    s_mask[tid] = m;
+    __syncthreads();
+    RRM_FC_PHASE(2);
+    // ---- 2. this CTA's share of the list, one entry per thread: find the thread that scanned entry e
+    // (largest t with s_off[t] <= e) and pick the matching set bit of its mask
+    const int per_cta = (total + FC_CL - 1) / FC_CL;
     const int lo = kg * per_cta, hi = min(total, lo + per_cta);
-    const int mine = max(0, hi - lo);              // <= FC_LCAP by the host's choice of ksplit
-    if (offset < hi && offset + local > lo) {
-        for (int c = c_begin; c < c_end; ++c) {
-            uint4 a = __ldg(xt4 + c);
-            uint4 b = xp4 ? __ldg(xp4 + c) : make_uint4(0, 0, 0, 0);
-            const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-            #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                int av = (int)(int8_t)(aw[i >> 2] >> ((i & 3) * 8));
-                int bv = (int)(int8_t)(bw[i >> 2] >> ((i & 3) * 8));
-                bool on = xp4 ? (av != bv) : true;
-                if (on) {
-                    if (offset >= lo && offset < hi) {
-                        s_list_j[offset - lo] = c * 16 + i;
-                        s_list_d[offset - lo] = av - bv;
-                    }
-                    ++offset;
-                }
-            }
-        }
+    const int mine = max(0, hi - lo);              // <= FC_LCAP: checked on the host
+    for (int e = lo + tid; e < hi; e += FC_THREADS) {
+        int t = 0;
+        #pragma unroll
+        for (int step = FC_THREADS / 2; step > 0; step >>= 1)
+            if (s_off[t + step] <= e) t += step;
+        const unsigned long long mk = s_mask[t];
+        const int r = e - s_off[t];                  // r-th set bit (0-based) of mk
+        const unsigned lo32 = (unsigned)mk, hi32 = (unsigned)(mk >> 32);
+        const int cl = __popc(lo32);
+        const int bit = r < cl ? (int)__fns(lo32, 0, r + 1) : 32 + (int)__fns(hi32, 0, r - cl + 1);
+        s_list_j[e - lo] = (unsigned short)(t * (16 * FC_PT) + bit);
     }
-    // new snapshot and statistics: one CTA per stream
-    if (kg == 0 && slice == 0) {
-        int groups32 = 0;
-        for (int base = 0; base < nchunks; base += FC_THREADS) {      // uniform trip count: shuffles inside
-            const int c = base + tid;
-            const bool in = c < nchunks;
-            uint4 a = make_uint4(0, 0, 0, 0), b = a;
-            if (in) {
-                a = __ldg(xt4 + c);
-                if (p.xnext) reinterpret_cast<uint4*>(p.xnext + (size_t)s * C)[c] = a;
-                if (xp4) b = __ldg(xp4 + c);
-            }
-            const unsigned diff = (a.x ^ b.x) | (a.y ^ b.y) | (a.z ^ b.z) | (a.w ^ b.w);
-            // a group of 32 inputs spans two chunks held by neighbouring lanes
-            const unsigned other = __shfl_xor_sync(0xffffffffu, diff, 1);
-            groups32 += in && ((c & 1) == 0) && ((diff | other) != 0);
-        }
-        if (p.stat) {
+    // new snapshot: in the clusters of slice 0, CTA r stores the chunks scanned by its warp r
+    if (slice == 0 && p.xnext && warp == kg) {
+        #pragma unroll
+        for (int i = 0; i < FC_PT; ++i)
+            if (c_begin + i < nchunks) reinterpret_cast<uint4*>(p.xnext + (size_t)s * C)[c_begin + i] = xa[i];
+    }
+    // statistics: one CTA per stream
+    if (kg == 0 && slice == 0 && p.stat) {
+        int groups32 = __popc((unsigned)((m | m >> 16) & 0xffffu) != 0) + __popc((unsigned)(((m >> 32) | (m >> 48)) & 0xffffu) != 0);
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) groups32 += __shfl_down_sync(0xffffffffu, groups32, o);
+        __shared__ int s_grp[FC_THREADS / 32];
+        if (lane == 0) s_grp[warp] = groups32;
+        __syncthreads();
+        if (tid == 0) {
+            int g = 0;
             #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) groups32 += __shfl_down_sync(0xffffffffu, groups32, o);
-            if (lane == 0 && groups32) atomicAdd(&p.stat[s * 2 + 1], (unsigned long long)groups32);
-            if (tid == 0) atomicAdd(&p.stat[s * 2 + 0], (unsigned long long)total);
+            for (int w = 0; w < FC_THREADS / 32; ++w) g += s_grp[w];
+            p.stat[s * 2 + 0] = (unsigned long long)total;
+            p.stat[s * 2 + 1] = (unsigned long long)g;
         }
     }
     __syncthreads();
 
-    // ---- 3. gather the columns of the owned entries: lane -> 16 outputs, warp -> column group
-    const int o0 = slice * FC_OW + lane * 16;
+    RRM_FC_PHASE(3);
+    // ---- 3. gather the columns of the owned entries: 8 lanes x 16 bytes span the slice, 32 columns in flight
+    const int sub = tid & 7, grp = tid >> 3;
+    const int o0 = slice * FC_OW + sub * 16;
     const bool o_ok = o0 < K;                       // K is a multiple of 16
     int acc[16];
     #pragma unroll
     for (int i = 0; i < 16; ++i) acc[i] = 0;
     const int8_t* wbase = p.Wt + o0;
-    // acc[i] += w_i * d for the 16 int8 weights in w.  dp4a against a selector that holds d in
-    // one byte lane; a delta outside int8 range (|d| <= 254) is split into two in-range halves.
+    // acc[i] += w_i * d for the 16 int8 weights in w: dp4a against a selector that holds d in one
+    // byte lane; a delta outside int8 range (|d| <= 254) is split into two in-range halves.
     auto fma16 = [&](const uint4& w, int d) {
         const unsigned ww[4] = {w.x, w.y, w.z, w.w};
-        if (d >= -128 && d <= 127) {                 // warp-uniform: d belongs to the column
-            const unsigned db = (unsigned)d & 0xffu;
+        const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
+        const int dl = d - dh;
+        const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
+        #pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            #pragma unroll
+            for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
+        }
+        if (dh != 0) {
             #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(db << (8 * b)), acc[q * 4 + b]);
-            }
-        } else {
-            const int dh = d / 2, dl = d - dh;
-            const unsigned hb = (unsigned)dh & 0xffu, lb = (unsigned)dl & 0xffu;
-            #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
-                    acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
-                }
+                for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
             }
         }
     };
     if (o_ok) {
-        int e = warp;
-        for (; e + 3 * FC_GROUPS < mine; e += 4 * FC_GROUPS) {
-            const int j0 = s_list_j[e], j1 = s_list_j[e + FC_GROUPS], j2 = s_list_j[e + 2 * FC_GROUPS],
-                      j3 = s_list_j[e + 3 * FC_GROUPS];
-            const uint4 w0 = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)j0 * K));
-            const uint4 w1 = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)j1 * K));
-            const uint4 w2 = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)j2 * K));
-            const uint4 w3 = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)j3 * K));
-            fma16(w0, s_list_d[e]);
-            fma16(w1, s_list_d[e + FC_GROUPS]);
-            fma16(w2, s_list_d[e + 2 * FC_GROUPS]);
-            fma16(w3, s_list_d[e + 3 * FC_GROUPS]);
-        }
-        for (; e < mine; e += FC_GROUPS) {
-            const uint4 w0 = __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)s_list_j[e] * K));
-            fma16(w0, s_list_d[e]);
-        }
-    }
-    #pragma unroll
-    for (int i = 0; i < 16; ++i) s_red[warp][lane * 16 + i] = acc[i];
-    __syncthreads();
-
-    // ---- 4. add into the stored projection (exact integer atomics)
-    int32_t* Ps = p.P + (size_t)s * K + slice * FC_OW;
-    const int width = min(FC_OW, K - slice * FC_OW);
-    if (mine > 0) {
-        for (int o = tid; o < width; o += FC_THREADS) {
-            int v = 0;
+        constexpr int U = 8;                           // columns in flight per thread
+        for (int e = grp; e < mine; e += U * FC_GROUPS) {
+            int j[U];
+            uint4 w[U];
             #pragma unroll
-            for (int g = 0; g < FC_GROUPS; ++g) v += s_red[g][o];
-            if (v) atomicAdd(&Ps[o], v);
+            for (int u = 0; u < U; ++u) {
+                const int eu = e + u * FC_GROUPS;
+                j[u] = eu < mine ? s_list_j[eu] : -1;
+            }
+            #pragma unroll
+            for (int u = 0; u < U; ++u)
+                w[u] = j[u] >= 0 ? __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)j[u] * K)) : make_uint4(0, 0, 0, 0);
+            #pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (j[u] >= 0) fma16(w[u], (int)s_xt[j[u]] - (int)s_xp[j[u]]);
         }
     }
-
-    // ---- 5. last CTA of this (stream, slice) applies f and writes Y_t
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        unsigned int* ctr = &p.counters[s * gridDim.y + slice];
-        const unsigned int ticket = atomicAdd(ctr, 1u);
-        const int last = (ticket == (unsigned)p.ksplit - 1);
-        if (last) *ctr = 0;                          // ready for the next launch (stream-ordered)
-        s_flag = last;
+    RRM_FC_PHASE(4);
+    // ---- 4. reduce: the 4 column groups of a warp by shuffles, the 8 warps through shared memory
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 8);
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
+    }
+    if (lane < 8) {
+        #pragma unroll
+        for (int i = 0; i < 16; ++i) s_red[warp][lane * 16 + i] = acc[i];
     }
     __syncthreads();
-    if (s_flag && p.Y) {
-        __threadfence();
-        for (int o = tid; o < width; o += FC_THREADS) {
-            const int v = __ldcg(&Ps[o]);
-            const size_t oi = (size_t)s * K + slice * FC_OW + o;
+    // ---- 5. across the cluster: every CTA pushes its partial sums into rank 0's shared memory, then
+    // arrives at the cluster barrier; only rank 0 waits, adds them onto the projection slice it owns
+    // (owner computes, no atomics), applies f and writes Y_t.
+    RRM_FC_PHASE(5);
+    cluster_wait();                                  // pairs with the arrive at kernel entry: all CTAs are running
+    if (tid < FC_OW) {
+        int v = 0;
+        #pragma unroll
+        for (int w = 0; w < FC_THREADS / 32; ++w) v += s_red[w][tid];
+        *cluster.map_shared_rank(&s_part[kg][tid], 0) = v;
+    }
+    RRM_FC_PHASE(6);
+    cluster_arrive_release();
+    if (kg != 0) return;                             // nobody reads a non-zero rank's shared memory
+    cluster_wait_acquire();
+    RRM_FC_PHASE(7);
+    if (tid < width) {
+        int v = p_old;
+        #pragma unroll
+        for (int r = 0; r < FC_CL; ++r) v += s_part[r][tid];
+        if (total > 0) Ps[tid] = v;
+        if (p.Y) {
+            const size_t oi = (size_t)s * K + slice * FC_OW + tid;
             if (p.shift < 0) reinterpret_cast<int32_t*>(p.Y)[oi] = v;
             else reinterpret_cast<int8_t*>(p.Y)[oi] = (int8_t)fc_apply_f(v, p.shift, p.act);
         }
     }
+    RRM_FC_PHASE(8);
 }
 
 // P[s][o] = bias[o]; optionally zero a snapshot
@@ -250,19 +298,10 @@ __global__ void fc_transpose_kernel(const int8_t* W, int8_t* Wt, int K, int C)
     }
 }
 
-static int fc_ksplit(const Layer& L)
-{
-    const int slices = ceil_div(L.d.c_out, FC_OW);
-    int ks = ceil_div(2 * 148, slices * L.d.n);
-    ks = ks < 1 ? 1 : ks;
-    const int need = ceil_div(L.d.c_in, FC_LCAP);      // a CTA's share must fit its list
-    return ks < need ? need : ks;
-}
-
 int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev)
 {
     const int C = L.d.c_in, K = L.d.c_out, n = L.d.n;
-    if (C % 16 || K % 16 || C / 16 > FC_MAX_CHUNKS * 4) return RRM_ERR_UNSUPPORTED;
+    if (C % 16 || K % 16 || C > FC_CL * FC_LCAP || C > 16 * FC_PT * FC_THREADS) return RRM_ERR_UNSUPPORTED;
     auto alloc = [&](void** p, size_t bytes) -> int {
         if (cudaMalloc(p, bytes) != cudaSuccess) return RRM_ERR_ALLOC;
         net->allocs.push_back(*p);
@@ -275,9 +314,7 @@ int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_
     RRM_TRY(alloc((void**)&L.P, (size_t)n * K * 4));
     RRM_TRY(alloc((void**)&L.P2, (size_t)n * K * 4));
     RRM_TRY(alloc((void**)&L.bias, (size_t)K * 4));
-    RRM_TRY(alloc((void**)&L.fc_counters, (size_t)n * slices * 4 * 2));
     RRM_TRY(alloc((void**)&L.fc_nnz, (size_t)n * 2 * 8));
-    RRM_CUDA_TRY(cudaMemset(L.fc_counters, 0, (size_t)n * slices * 4 * 2));
     RRM_CUDA_TRY(cudaMemset(L.fc_nnz, 0, (size_t)n * 2 * 8));
     if (bias_dev) RRM_CUDA_TRY(cudaMemcpy(L.bias, bias_dev, (size_t)K * 4, cudaMemcpyDeviceToDevice));
     else RRM_CUDA_TRY(cudaMemset(L.bias, 0, (size_t)K * 4));
@@ -303,7 +340,6 @@ int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool de
     p.xt = reinterpret_cast<const int8_t*>(X_dev);
     p.Wt = L.Wt;
     p.c_in = C; p.c_out = K; p.shift = L.d.shift; p.act = L.d.act;
-    p.ksplit = fc_ksplit(L);
     p.Y = Y_dev;
     const int tot = n * (K > C ? K : C);
     if (dense) {
@@ -312,19 +348,16 @@ int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool de
         p.xprev = nullptr;
         p.P = Pd;
         p.stat = nullptr;
-        p.counters = L.fc_counters + (stateless ? n * slices : 0);
         if (stateless) p.xnext = nullptr;
         else { p.xnext = L.xs[L.xs_cur ^ 1]; L.xs_cur ^= 1; }
     } else {
-        cudaMemsetAsync(L.fc_nnz, 0, (size_t)n * 2 * 8, st);
         p.xprev = L.xs[L.xs_cur];
         p.xnext = L.xs[L.xs_cur ^ 1];
         L.xs_cur ^= 1;
         p.P = reinterpret_cast<int32_t*>(L.P);
         p.stat = L.fc_nnz;
-        p.counters = L.fc_counters;
     }
-    dim3 grid(p.ksplit, slices, n);
+    dim3 grid(FC_CL, slices, n);
     fc_delta_i8_kernel<<<grid, FC_THREADS, 0, st>>>(p);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
@@ -337,3 +370,10 @@ int fc_fused_projection(rrm_net* net, Layer& L, void* P_dev, cudaStream_t st)
 }
 
 }  // namespace rrm
+
+#ifdef RRM_FC_TIMING
+extern "C" int rrm_fc_phase_clocks(long long* host16)
+{
+    return cudaMemcpyFromSymbol(host16, rrm_fc_phase_clock, sizeof(long long) * 16) == cudaSuccess ? 0 : -7;
+}
+#endif
