@@ -72,7 +72,7 @@ struct Layer {
     int8_t* Wt = nullptr;             // [c_in][c_out] transposed weights
     int8_t* xs[2] = {nullptr, nullptr};     // ping-pong input snapshots [n][c_in]
     int xs_cur = 0;
-    unsigned int* fc_counters = nullptr;    // arrival counters per (stream, output slice)
+    void* fc_scratch = nullptr;             // per-stream non-zero lists of the two-kernel form
     unsigned long long* fc_nnz = nullptr;   // [0] nnz elements, [1] active groups of 32 (cleared by the kernel's last CTA)
 };
 

@@ -32,6 +32,7 @@ constexpr int FC_CL = 8;                   // CTAs per cluster = split of the no
 constexpr int FC_OW = 128;                 // outputs per cluster (8 lanes x 16 bytes)
 constexpr int FC_GROUPS = FC_THREADS / 8;  // columns gathered in parallel inside a CTA
 constexpr int FC_LCAP = 2048;              // list entries one CTA can own  (C_in <= FC_CL * FC_LCAP)
+constexpr int FC_TWO_KERNEL_MIN_STREAMS = 3;   // from this many streams per call on, build the list once per stream
 constexpr int FC_PT = 4;                   // 16-byte chunks scanned per thread (C_in <= 16 * FC_PT * FC_THREADS)
 
 struct FcParams {
@@ -274,6 +275,181 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
     RRM_FC_PHASE(8);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Two-kernel form of the same step, used when many streams are processed per call: the list of
+// non-zero delta entries is built once per stream into global scratch memory instead of once per
+// CTA, and the gather kernel needs no cross-CTA reduction (one CTA owns FC_OW outputs of a stream).
+//   scratch layout: count[n] (int), then entries[n][c_in] (uint32: input index | (delta + 256) << 16)
+// ------------------------------------------------------------------------------------------------
+__host__ __device__ inline size_t fc_scratch_bytes(int n, int c_in) { return ((size_t)n * 4 + 15) / 16 * 16 + (size_t)n * c_in * 4; }
+__host__ __device__ inline uint32_t* fc_scratch_entries(void* scratch, int n) {
+    return reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(scratch) + ((size_t)n * 4 + 15) / 16 * 16);
+}
+
+__global__ void __launch_bounds__(FC_THREADS) fc_scan_kernel(FcParams p, void* scratch, int n)
+{
+    __shared__ int s_warp[FC_THREADS / 32];
+    __shared__ int s_off[FC_THREADS];
+    __shared__ unsigned long long s_mask[FC_THREADS];
+    __shared__ __align__(16) int8_t s_xt[16 * FC_PT * FC_THREADS];
+    __shared__ __align__(16) int8_t s_xp[16 * FC_PT * FC_THREADS];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int s = blockIdx.x;
+    const int C = p.c_in;
+    const int nchunks = C >> 4;
+    const uint4* xt4 = reinterpret_cast<const uint4*>(p.xt + (size_t)s * C);
+    const uint4* xp4 = p.xprev ? reinterpret_cast<const uint4*>(p.xprev + (size_t)s * C) : nullptr;
+    const int c_begin = tid * FC_PT;
+    unsigned long long m = 0;
+    #pragma unroll
+    for (int i = 0; i < FC_PT; ++i) {
+        if (c_begin + i < nchunks) {
+            const uint4 a = __ldg(xt4 + c_begin + i);
+            const uint4 b = xp4 ? xp4[c_begin + i] : make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4*>(s_xt)[c_begin + i] = a;
+            reinterpret_cast<uint4*>(s_xp)[c_begin + i] = b;
+            // the thread that read a chunk of the snapshot is the one that overwrites it: in place is safe
+            if (p.xnext) reinterpret_cast<uint4*>(p.xnext + (size_t)s * C)[c_begin + i] = a;
+            unsigned cm = 0xffffu;
+            if (xp4) {
+                auto nib = [](unsigned v) {
+                    v |= v >> 4; v |= v >> 2; v |= v >> 1;
+                    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
+                };
+                cm = nib(a.x ^ b.x) | nib(a.y ^ b.y) << 4 | nib(a.z ^ b.z) << 8 | nib(a.w ^ b.w) << 12;
+            }
+            m |= (unsigned long long)cm << (16 * i);
+        }
+    }
+    const int local = __popcll(m);
+    int incl = local;
+    #pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int warp_off = 0, total = 0;
+    #pragma unroll
+    for (int w = 0; w < FC_THREADS / 32; ++w) {
+        int v = s_warp[w];
+        if (w < warp) warp_off += v;
+        total += v;
+    }
+    s_off[tid] = warp_off + incl - local;
+    s_mask[tid] = m;
+    __syncthreads();
+    uint32_t* entries = fc_scratch_entries(scratch, n) + (size_t)s * C;
+    for (int e = tid; e < total; e += FC_THREADS) {
+        int t = 0;
+        #pragma unroll
+        for (int step = FC_THREADS / 2; step > 0; step >>= 1)
+            if (s_off[t + step] <= e) t += step;
+        const unsigned long long mk = s_mask[t];
+        const int r = e - s_off[t];
+        const unsigned lo32 = (unsigned)mk, hi32 = (unsigned)(mk >> 32);
+        const int cl = __popc(lo32);
+        const int bit = r < cl ? (int)__fns(lo32, 0, r + 1) : 32 + (int)__fns(hi32, 0, r - cl + 1);
+        const int j = t * (16 * FC_PT) + bit;
+        const int d = (int)s_xt[j] - (int)s_xp[j];
+        entries[e] = (uint32_t)j | ((uint32_t)(d + 256) << 16);
+    }
+    if (tid == 0) reinterpret_cast<int*>(scratch)[s] = total;
+    if (p.stat) {
+        int groups32 = __popc((unsigned)((m | m >> 16) & 0xffffu) != 0) + __popc((unsigned)(((m >> 32) | (m >> 48)) & 0xffffu) != 0);
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) groups32 += __shfl_down_sync(0xffffffffu, groups32, o);
+        if (lane == 0) s_warp[warp] = groups32;      // s_warp is free again: every thread is past its reads
+        __syncthreads();
+        if (tid == 0) {
+            int g = 0;
+            #pragma unroll
+            for (int w = 0; w < FC_THREADS / 32; ++w) g += s_warp[w];
+            p.stat[s * 2 + 0] = (unsigned long long)total;
+            p.stat[s * 2 + 1] = (unsigned long long)g;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(FC_THREADS) fc_gather_kernel(FcParams p, const void* scratch, int n)
+{
+    __shared__ int s_red[FC_THREADS / 32][FC_OW];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int slice = blockIdx.x, s = blockIdx.y;
+    const int C = p.c_in, K = p.c_out;
+    const int total = reinterpret_cast<const int*>(scratch)[s];
+    const uint32_t* entries = fc_scratch_entries(const_cast<void*>(scratch), n) + (size_t)s * C;
+    int32_t* Ps = p.P + (size_t)s * K + slice * FC_OW;
+    const int width = min(FC_OW, K - slice * FC_OW);
+    int p_old = 0;
+    if (tid < width) p_old = Ps[tid];
+    const int sub = tid & 7, grp = tid >> 3;
+    const int o0 = slice * FC_OW + sub * 16;
+    int acc[16];
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0;
+    const int8_t* wbase = p.Wt + o0;
+    auto fma16 = [&](const uint4& w, int d) {
+        const unsigned ww[4] = {w.x, w.y, w.z, w.w};
+        const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
+        const int dl = d - dh;
+        const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
+        #pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            #pragma unroll
+            for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
+        }
+        if (dh != 0) {
+            #pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                #pragma unroll
+                for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
+            }
+        }
+    };
+    if (o0 < K) {
+        constexpr int U = 8;
+        for (int e = grp; e < total; e += U * FC_GROUPS) {
+            uint32_t ent[U];
+            uint4 w[U];
+            #pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int eu = e + u * FC_GROUPS;
+                ent[u] = eu < total ? __ldg(entries + eu) : 0xffffffffu;
+            }
+            #pragma unroll
+            for (int u = 0; u < U; ++u)
+                w[u] = ent[u] != 0xffffffffu ? __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(ent[u] & 0xffffu) * K))
+                                             : make_uint4(0, 0, 0, 0);
+            #pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (ent[u] != 0xffffffffu) fma16(w[u], (int)(ent[u] >> 16) - 256);
+        }
+    }
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 8);
+        acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
+    }
+    if (lane < 8) {
+        #pragma unroll
+        for (int i = 0; i < 16; ++i) s_red[warp][lane * 16 + i] = acc[i];
+    }
+    __syncthreads();
+    if (tid < width) {
+        int v = p_old;
+        #pragma unroll
+        for (int w = 0; w < FC_THREADS / 32; ++w) v += s_red[w][tid];
+        if (total > 0) Ps[tid] = v;
+        if (p.Y) {
+            const size_t oi = (size_t)s * K + slice * FC_OW + tid;
+            if (p.shift < 0) reinterpret_cast<int32_t*>(p.Y)[oi] = v;
+            else reinterpret_cast<int8_t*>(p.Y)[oi] = (int8_t)fc_apply_f(v, p.shift, p.act);
+        }
+    }
+}
+
 // P[s][o] = bias[o]; optionally zero a snapshot
 __global__ void fc_init_kernel(int32_t* P, const int32_t* bias, int n, int K, int8_t* snap, int C)
 {
@@ -315,6 +491,7 @@ int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_
     RRM_TRY(alloc((void**)&L.P2, (size_t)n * K * 4));
     RRM_TRY(alloc((void**)&L.bias, (size_t)K * 4));
     RRM_TRY(alloc((void**)&L.fc_nnz, (size_t)n * 2 * 8));
+    RRM_TRY(alloc((void**)&L.fc_scratch, fc_scratch_bytes(n, C)));
     RRM_CUDA_TRY(cudaMemset(L.fc_nnz, 0, (size_t)n * 2 * 8));
     if (bias_dev) RRM_CUDA_TRY(cudaMemcpy(L.bias, bias_dev, (size_t)K * 4, cudaMemcpyDeviceToDevice));
     else RRM_CUDA_TRY(cudaMemset(L.bias, 0, (size_t)K * 4));
@@ -357,8 +534,13 @@ int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool de
         p.P = reinterpret_cast<int32_t*>(L.P);
         p.stat = L.fc_nnz;
     }
-    dim3 grid(FC_CL, slices, n);
-    fc_delta_i8_kernel<<<grid, FC_THREADS, 0, st>>>(p);
+    if (n < FC_TWO_KERNEL_MIN_STREAMS) {
+        dim3 grid(FC_CL, slices, n);
+        fc_delta_i8_kernel<<<grid, FC_THREADS, 0, st>>>(p);
+    } else {
+        fc_scan_kernel<<<n, FC_THREADS, 0, st>>>(p, L.fc_scratch, n);
+        fc_gather_kernel<<<dim3(slices, n), FC_THREADS, 0, st>>>(p, L.fc_scratch, n);
+    }
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }

@@ -53,6 +53,13 @@ def test_fc6_keyframe_then_steps_and_two_streams():
     _run_sequence(spec, seq, 2, keyframe_first=True)
 
 
+def test_fc6_many_streams_take_the_two_kernel_form():
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=5, rho=0.05, seed=25, n=5)
+    seq[3, 2] = seq[2, 2]                 # one stream with zero delta in one frame
+    _run_sequence(spec, seq, 5, keyframe_first=True)
+
+
 @pytest.mark.parametrize("c_in,c_out,shift,act", [(64, 48, -1, "none"), (160, 528, 6, "relu"),
                                                   (1024 + 32, 16, 5, "none"), (32, 1040, -1, "none")])
 def test_fc_small_and_ragged_shapes(c_in, c_out, shift, act):
