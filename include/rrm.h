@@ -147,6 +147,42 @@ int rrm_net_tensor(rrm_net* net, int t, void* dst_dev, void* stream);
 /* Bytes rrm_net_tensor / the out_dev argument need for tensor `t` (negative = error). */
 int64_t rrm_net_tensor_bytes(const rrm_net* net, int t);
 
+/* ---- allocation-free delta-FC step --------------------------------------------------
+ * (The paper has no counterpart; this is a deployment aid of this library.)
+ *
+ * Some callers of this library are not allowed to allocate device memory: plug-ins whose
+ * host hands them a fixed memory budget up front and forbids cudaMalloc afterwards, real-time
+ * loops that must not wait on the allocator's lock or on the device-wide synchronisation a
+ * cudaFree implies, and processes that share a GPU under a hard memory cap.  This entry point does one int8 delta-FC frame - what rrm_step
+ * does for a lone RRM_FC / RRM_I8 layer - without calling cudaMalloc, cudaFree or any
+ * allocating routine: the caller owns the whole RRM state, and the one piece of working
+ * memory the kernels need (the per-stream lists of non-zero delta entries) is a fixed
+ * array compiled into the library, RRM_FC_NOALLOC_MAX_STREAMS * RRM_FC_NOALLOC_MAX_C_IN * 4
+ * bytes (1 MiB) plus a 64-byte header.  Every GPU that loads the library keeps that array until
+ * the process exits.
+ *
+ *   Wt_dev    [c_in][c_out] int8   the layer's weights TRANSPOSED (one contiguous row per input)
+ *   Xt_dev    [n][c_in]     int8   frame t, read-only
+ *   Xprev_dev [n][c_in]     int8   in/out: frame t-1 on entry, frame t on return (start with zeros)
+ *   P_dev     [n][c_out]    int32  in/out: stored projection (start with the bias in every row)
+ *   Y_dev     [n][c_out]    int32 if shift < 0, else int8 = f(P) as for rrm_step; may be NULL
+ * All pointers are device pointers; Wt_dev, Xt_dev and Xprev_dev must be 16-byte aligned; c_in
+ * and c_out must be multiples of 16.  act is RRM_ACT_NONE or RRM_ACT_RELU.
+ *
+ * Errors: RRM_ERR_CAPACITY if n > RRM_FC_NOALLOC_MAX_STREAMS or c_in > RRM_FC_NOALLOC_MAX_C_IN;
+ * RRM_ERR_SHAPE / RRM_ERR_INVALID_ARG for the other violations; nothing is launched then.
+ *
+ * The first call on a device looks up the array's device address (one cudaGetSymbolAddress,
+ * no allocation); make that first call before starting any stream capture.  All calls on a
+ * device share the one array and it keeps the previous call's contents; nothing in it has to
+ * start at zero (each call rewrites every count and entry it later reads), but for the same
+ * reason two calls that overlap on the GPU (different streams, no ordering) race on it:
+ * serialise them.  Asynchronous on `stream`. */
+#define RRM_FC_NOALLOC_MAX_STREAMS 16
+#define RRM_FC_NOALLOC_MAX_C_IN 16384
+int rrm_fc_step_noalloc(const int8_t* Wt_dev, const int8_t* Xt_dev, int8_t* Xprev_dev, int32_t* P_dev,
+                        void* Y_dev, int n, int c_in, int c_out, int shift, int act, void* stream);
+
 const char* rrm_strerror(int status);
 
 #ifdef __cplusplus

@@ -75,6 +75,8 @@ def lib():
         f = getattr(L, name)
         f.argtypes = args
         f.restype = ctypes.c_int
+    L.rrm_fc_step_noalloc.argtypes = [_P, _P, _P, _P, _P] + [ctypes.c_int] * 5 + [_P]
+    L.rrm_fc_step_noalloc.restype = ctypes.c_int
     L.rrm_net_tensor_bytes.argtypes = [_P, ctypes.c_int]
     L.rrm_net_tensor_bytes.restype = ctypes.c_int64
     L.rrm_strerror.argtypes = [ctypes.c_int]
@@ -206,6 +208,14 @@ class Net:
 
 
 Layer = Net   # a single layer is a stack of one
+
+
+def fc_step_noalloc(Wt, Xt, Xprev, P, Y, n, c_in, c_out, shift=-1, act="none", stream=None):
+    """rrm_fc_step_noalloc: one int8 delta-FC frame on caller-owned state, for callers that may
+    not allocate device memory.  Returns the status code instead of raising, so that a caller
+    can test the documented limits."""
+    return lib().rrm_fc_step_noalloc(_ptr(Wt), _ptr(Xt), _ptr(Xprev), _ptr(P), _ptr(Y), n, c_in, c_out, shift,
+                                     ACT[act], _stream(stream))
 
 
 def net_from_specs(specs, n=1, variant="auto", device="cuda"):

@@ -14,6 +14,7 @@
 // Cost is HBM-bound: nnz * C_out weight bytes per frame.
 #include "rrm_common.cuh"
 #include <cooperative_groups.h>
+#include <mutex>
 
 namespace cg = cooperative_groups;
 
@@ -552,6 +553,70 @@ int fc_fused_projection(rrm_net* net, Layer& L, void* P_dev, cudaStream_t st)
 }
 
 }  // namespace rrm
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free delta-FC step.  The per-stream non-zero lists live in a fixed array that is part
+// of the loaded module, so the call needs no device allocation at all.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int NOALLOC_MAX_STREAMS = RRM_FC_NOALLOC_MAX_STREAMS;
+constexpr int NOALLOC_MAX_C_IN = RRM_FC_NOALLOC_MAX_C_IN;
+constexpr size_t NOALLOC_BYTES = ((size_t)NOALLOC_MAX_STREAMS * 4 + 15) / 16 * 16 +
+                                 (size_t)NOALLOC_MAX_STREAMS * NOALLOC_MAX_C_IN * 4;
+
+// Every GPU that loads the library holds this array until the process exits.
+static __device__ __align__(256) unsigned char g_fc_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+void* g_noalloc_ptr[NOALLOC_MAX_DEVICES];          // device address of the array, per device
+std::mutex g_noalloc_mutex;
+
+// In host code the array's name is only a handle: the address a kernel can use has to be asked for,
+// once per device, with that device current.
+int noalloc_scratch(void** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return RRM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_fc_noalloc_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return RRM_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return RRM_OK;
+}
+
+}  // namespace
+
+extern "C" int rrm_fc_step_noalloc(const int8_t* Wt_dev, const int8_t* Xt_dev, int8_t* Xprev_dev, int32_t* P_dev,
+                                   void* Y_dev, int n, int c_in, int c_out, int shift, int act, void* stream)
+{
+    using namespace rrm;
+    if (!Wt_dev || !Xt_dev || !Xprev_dev || !P_dev) return RRM_ERR_INVALID_ARG;
+    if (n < 1 || c_in < 1 || c_out < 1) return RRM_ERR_SHAPE;
+    if (n > NOALLOC_MAX_STREAMS || c_in > NOALLOC_MAX_C_IN) return RRM_ERR_CAPACITY;
+    if (c_in % 16 || c_out % 16) return RRM_ERR_SHAPE;
+    if (act != RRM_ACT_NONE && act != RRM_ACT_RELU) return RRM_ERR_INVALID_ARG;
+    if (shift > 30 || (shift < 0 && act != RRM_ACT_NONE)) return RRM_ERR_INVALID_ARG;
+    if (((uintptr_t)Wt_dev | (uintptr_t)Xt_dev | (uintptr_t)Xprev_dev) & 15) return RRM_ERR_INVALID_ARG;
+    if (((uintptr_t)P_dev & 3) || (Y_dev && shift < 0 && ((uintptr_t)Y_dev & 3))) return RRM_ERR_INVALID_ARG;
+    void* scratch = nullptr;
+    RRM_TRY(noalloc_scratch(&scratch));
+    FcParams p;
+    p.xt = Xt_dev; p.xprev = Xprev_dev; p.xnext = Xprev_dev;   // snapshot updated in place
+    p.Wt = Wt_dev; p.P = P_dev; p.Y = Y_dev; p.stat = nullptr;
+    p.c_in = c_in; p.c_out = c_out; p.shift = shift; p.act = act;
+    cudaStream_t st = (cudaStream_t)stream;
+    fc_scan_kernel<<<n, FC_THREADS, 0, st>>>(p, scratch, n);
+    fc_gather_kernel<<<dim3(ceil_div(c_out, FC_OW), n), FC_THREADS, 0, st>>>(p, scratch, n);
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
 
 #ifdef RRM_FC_TIMING
 extern "C" int rrm_fc_phase_clocks(long long* host16)
