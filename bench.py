@@ -3,10 +3,13 @@
 
 Workload: the int8 delta-FC configuration (AlexNet-fc6 shape 9216 -> 4096, int32 accumulation,
 32-frame sequences whose frames differ in a fraction rho of the inputs, changed entries in runs
-of 32).  One "step" = one frame through the whole hot path of the layer (delta + compaction,
-column-gather product, accumulate + snapshot + output), i.e. one rrm_step call.
+of 32).  One "step" = one chunk of 32 consecutive frames of one stream through the whole hot path
+of the layer (delta + compaction, column-gather product, accumulate + snapshot + output for every
+frame), i.e. one rrm_step_seq call = one kernel launch; the reported value is frames per second.
+Secondary numbers: the same with one frame per call (rrm_step), the library's dense path, other
+densities, several streams per call.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--rho 0.05] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--rho 0.05] [--chunk 32] [--impl ours|reference]
 
 Timing: every timed step is preceded by an untimed L2 flush (a 256 MiB device write), and is
 bracketed by its own CUDA event pair on the launching stream; ms_per_step is the mean of those
@@ -48,8 +51,8 @@ def measured_peaks():
 
 
 def committed_traffic(rho):
-    """DRAM bytes per launch of the delta-FC kernel from the committed ncu summary, if present."""
-    p = os.path.join(ROOT, "profiles", "fc_delta_i8_fc6.txt")
+    """DRAM bytes per launch of the chunk delta-FC kernel from the committed ncu summary, if present."""
+    p = os.path.join(ROOT, "profiles", "fc_seq_fc6_chunk32.txt")
     if not os.path.exists(p):
         return None
     for line in open(p):
@@ -103,7 +106,8 @@ class ClockSampler:
 
 
 def run_reference(args, rank, world):
-    """The CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    """The CPU oracle, as it stands, on the host cores (rank 0 only).  One reference step is a bounded
+    sample of the GPU arm's step: ONE frame of the chunk; ms_per_step is scaled to a whole chunk."""
     if rank != 0:
         return
     import workloads as wl
@@ -122,12 +126,15 @@ def run_reference(args, rank, world):
     fps = args.steps / dt
     print(json.dumps({
         "impl": "reference", "metric": "frames_per_sec", "value": fps, "unit": "frames/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps * args.chunk,
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "i8", "data": "synthetic",
-        "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream"},
+        "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream; one step = one chunk "
+                               f"of {args.chunk} consecutive frames", "frames_per_step": args.chunk},
         "dense_equiv_gmacs": fps * DENSE_MACS / 1e9,
         "cpu_baseline": {"value": fps, "unit": "frames/s", "cores": orc.threads(), "kind": "oracle",
-                         "sample": f"{args.steps} frames of the same sequence through the oracle's Algorithm-1 recurrence"},
+                         "sample": f"1 frame per step ({args.steps} frames of the same sequence) through the oracle's "
+                                   f"Algorithm-1 recurrence; ms_per_step scaled to {args.chunk} frames"},
         "e2e": {"value": fps, "unit": "frames/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -135,9 +142,10 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=992)
-    ap.add_argument("--warmup", type=int, default=62)
+    ap.add_argument("--steps", type=int, default=310, help="timed steps; one step = one chunk of --chunk frames")
+    ap.add_argument("--warmup", type=int, default=31)
     ap.add_argument("--rho", type=float, default=0.05)
+    ap.add_argument("--chunk", type=int, default=FRAMES, help="frames per rrm_step_seq call")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="skip the secondary sweeps (profiling runs)")
     args = ap.parse_args()
@@ -145,8 +153,6 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
-        if args.steps == 992:
-            args.steps, args.warmup = 310, 31
         run_reference(args, rank, world)
         return
 
@@ -165,8 +171,10 @@ def main():
     W = torch.from_numpy(spec.weight).cuda()
     B = torch.from_numpy(spec.bias).cuda()
     order = pingpong(FRAMES)
+    period = len(order)                                  # 62 frames, then the walk repeats
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
+    T = args.chunk
 
     def barrier():
         torch.cuda.synchronize()
@@ -174,29 +182,49 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    def reduce_max(ms):
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
     def make(rho, n=1):
+        """Layer + the endless back-and-forth walk over the 32-frame sequence, laid out so that chunk k
+        is rows [k*T, (k+1)*T) of one device array (whole number of periods, so it wraps seamlessly)."""
         desc = rrm.desc_from_spec(spec, n=n)
         layer = rrm.Net([desc], [W], [B])
         seq = wl.fc_run_sequence(frames=FRAMES, rho=rho, seed=21 + rank, n=n)
-        frames = [torch.from_numpy(seq[t]).cuda() for t in range(FRAMES)]
-        nnz = [int(np.count_nonzero(seq[order[(i + 1) % len(order)]] != seq[order[i % len(order)]]))
-               for i in range(len(order))]
-        return layer, seq, frames, float(np.mean(nnz))
+        total = period * T // np.gcd(period, T)
+        walk = np.stack([seq[order[(i + 1) % period]] for i in range(total)])      # frame i+1 of the walk
+        nnz = np.array([np.count_nonzero(seq[order[(i + 1) % period]] != seq[order[i % period]]) / n
+                        for i in range(period)])
+        # distinct weight columns one chunk touches (what a cold L2 must fetch), mean over the chunks, stream 0
+        uniq = []
+        for k in range(total // T):
+            touched = np.zeros(C_IN, dtype=bool)
+            for i in range(k * T, (k + 1) * T):
+                touched |= seq[order[(i + 1) % period]][0] != seq[order[i % period]][0]
+            uniq.append(int(touched.sum()))
+        return layer, seq, walk, torch.from_numpy(walk).cuda(), float(nnz.mean()), float(np.mean(uniq))
 
-    def timed(layer, frames, steps, warmup, cold, dense=False):
-        """Returns (mean ms per step, launches).  cold: flush L2 before each step, time each step alone."""
-        Y = layer.new_output()
-        layer.keyframe(frames[0], Y)
-        call = layer.dense if dense else layer.step
+    def timed_chunks(layer, seq, walk_dev, steps, warmup, cold, dense=False, frames_per_call=None):
+        """Mean ms per call of rrm_step_seq (or rrm_dense_seq) over chunks of the walk."""
+        tc = T if frames_per_call is None else frames_per_call
+        nchunks = walk_dev.shape[0] // tc
+        Y = layer.new_output(frames=tc)
+        layer.keyframe(torch.from_numpy(seq[order[0]]).cuda(), None)
+        call = layer.dense_seq if dense else layer.step_seq
         for i in range(warmup):
-            call(frames[order[(i + 1) % len(order)]], Y)
+            call(walk_dev[(i % nchunks) * tc:(i % nchunks + 1) * tc], Y, tc)
         barrier()
         if cold:
             evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
             for i in range(steps):
+                k = (warmup + i) % nchunks
                 flush.fill_(i & 0xff)
                 evs[i][0].record(stream)
-                call(frames[order[(warmup + i + 1) % len(order)]], Y)
+                call(walk_dev[k * tc:(k + 1) * tc], Y, tc)
                 evs[i][1].record(stream)
             barrier()
             ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
@@ -204,72 +232,100 @@ def main():
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
             for i in range(steps):
-                call(frames[order[(warmup + i + 1) % len(order)]], Y)
+                k = (warmup + i) % nchunks
+                call(walk_dev[k * tc:(k + 1) * tc], Y, tc)
             b.record(stream)
             barrier()
             ms = a.elapsed_time(b) / steps
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms, steps * (2 if dense else 1)
+        return reduce_max(ms)
 
-    def algorithmic_bytes(nnz_mean):
-        # gathered weight columns + read/modify/write of P + output + X_t, snapshot read, snapshot write
+    def timed_single(layer, seq, frames, steps, warmup, cold, dense=False):
+        """Mean ms per rrm_step (one frame per call)."""
+        Y = layer.new_output()
+        layer.keyframe(frames[0], Y)
+        call = layer.dense if dense else layer.step
+        for i in range(warmup):
+            call(frames[order[(i + 1) % period]], Y)
+        barrier()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps):
+            if cold:
+                flush.fill_(i & 0xff)
+            evs[i][0].record(stream)
+            call(frames[order[(warmup + i + 1) % period]], Y)
+            evs[i][1].record(stream)
+        barrier()
+        return reduce_max(float(np.mean([a.elapsed_time(b) for a, b in evs])))
+
+    def frame_bytes(nnz_mean):
+        # per frame: gathered weight columns + read/modify/write of P + output + X_t, snapshot read, snapshot write
         return nnz_mean * C_OUT + 8 * C_OUT + 4 * C_OUT + 3 * C_IN
+
+    def chunk_cold_bytes(uniq_cols, frames):
+        # what one chunk launch must fetch with a cold L2: every distinct column once, the frames, per-frame
+        # projection deltas (write + read) and outputs, the stored projection
+        return uniq_cols * C_OUT + (frames + 2) * C_IN + frames * 12 * C_OUT + 8 * C_OUT
 
     peak, peak_kind = measured_peaks()
 
-    # ---- primary: one stream, rho as asked, cold L2, per-step events
-    layer, seq, frames, nnz_mean = make(args.rho)
+    # ---- primary: one stream per GPU, chunks of T frames per call, rho as asked, cold L2, per-step events
+    layer, seq, walk, walk_dev, nnz_mean, uniq_mean = make(args.rho)
     sampler = ClockSampler(local)
     sampler.start()
-    ms, launches = timed(layer, frames, args.steps, args.warmup, cold=True)
+    ms = timed_chunks(layer, seq, walk_dev, args.steps, args.warmup, cold=True)
     clocks = sampler.stop()
-    fps = world * 1e3 / ms
-    bytes_step = algorithmic_bytes(nnz_mean)
-    achieved = bytes_step / (ms * 1e-3) / 1e9
+    fps = world * T * 1e3 / ms
+    bytes_launch = frame_bytes(nnz_mean) * T
+    achieved = bytes_launch / (ms * 1e-3) / 1e9
+    achieved_unique = chunk_cold_bytes(uniq_mean, T) / (ms * 1e-3) / 1e9
     st = layer.stats(0)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
-    xh = [torch.from_numpy(seq[t]).pin_memory() for t in range(FRAMES)]
-    yh = torch.empty((1, C_OUT, 1, 1), dtype=torch.int32).pin_memory()
+    nchunks = walk.shape[0] // T
+    xh = torch.from_numpy(walk).pin_memory()
+    yh = torch.empty((T, 1, C_OUT, 1, 1), dtype=torch.int32).pin_memory()
     e2e_steps = 10 if args.quick else min(args.steps, 310)
+    layer.keyframe(torch.from_numpy(seq[order[0]]).cuda(), None)
     for i in range(5):
-        layer.step_host(xh[order[(i + 1) % len(order)]], yh)
+        layer.step_seq_host(xh[(i % nchunks) * T:(i % nchunks + 1) * T], yh, T)
     barrier()
     t0 = time.perf_counter()
     for i in range(e2e_steps):
-        layer.step_host(xh[order[(5 + i + 1) % len(order)]], yh)
+        k = (5 + i) % nchunks
+        layer.step_seq_host(xh[k * T:(k + 1) * T], yh, T)
     torch.cuda.synchronize()
-    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = reduce_max((time.perf_counter() - t0) * 1e3 / e2e_steps)
     layer.close()
 
     extra = {}
     if not args.quick:
         by_rho = {}
         for rho in RHOS:
-            L2, _, fr, nz = make(rho)
-            c_ms, _ = timed(L2, fr, 310, 31, cold=True)
-            w_ms, _ = timed(L2, fr, 310, 31, cold=False)
-            d_ms, _ = timed(L2, fr, 124, 10, cold=True, dense=True)
+            L2, sq, wk, wd, nz, un = make(rho)
+            fr = [torch.from_numpy(sq[t]).cuda() for t in range(FRAMES)]
+            c_ms = timed_chunks(L2, sq, wd, 124, 10, cold=True)
+            w_ms = timed_chunks(L2, sq, wd, 124, 10, cold=False)
+            d_ms = timed_chunks(L2, sq, wd, 31, 3, cold=True, dense=True)
+            s_ms = timed_single(L2, sq, fr, 310, 31, cold=True)
+            sd_ms = timed_single(L2, sq, fr, 124, 10, cold=True, dense=True)
             by_rho[f"{rho:g}"] = {
-                "nnz_mean": nz, "cold_us": c_ms * 1e3, "warm_us": w_ms * 1e3, "dense_cold_us": d_ms * 1e3,
-                "fps_cold": 1e3 / c_ms, "gmacs_dense_equiv_cold": DENSE_MACS / c_ms / 1e6,
-                "speedup_vs_own_dense": d_ms / c_ms,
-                "roofline_frac_cold": algorithmic_bytes(nz) / (c_ms * 1e-3) / 1e9 / peak}
+                "nnz_mean_per_frame": nz, "distinct_columns_per_chunk": un,
+                "chunk_cold_us": c_ms * 1e3, "chunk_warm_us": w_ms * 1e3, "dense_chunk_cold_us": d_ms * 1e3,
+                "fps_cold": T * 1e3 / c_ms, "gmacs_dense_equiv_cold": T * DENSE_MACS / c_ms / 1e6,
+                "speedup_vs_own_dense_chunk": d_ms / c_ms,
+                "roofline_frac_per_frame_bytes": frame_bytes(nz) * T / (c_ms * 1e-3) / 1e9 / peak,
+                "roofline_frac_distinct_bytes": chunk_cold_bytes(un, T) / (c_ms * 1e-3) / 1e9 / peak,
+                "single_frame_call_cold_us": s_ms * 1e3, "single_frame_dense_cold_us": sd_ms * 1e3,
+                "single_frame_speedup_vs_own_dense": sd_ms / s_ms,
+                "single_frame_roofline_frac": frame_bytes(nz) / (s_ms * 1e-3) / 1e9 / peak}
             L2.close()
         extra["by_rho"] = by_rho
         streams = {}
-        for n in (16, 64):
-            L3, _, fr, nz = make(args.rho, n=n)
-            c_ms, _ = timed(L3, fr, 124, 10, cold=True)
-            streams[str(n)] = {"cold_us_per_step": c_ms * 1e3, "fps_cold": n * 1e3 / c_ms,
-                               "algorithmic_gbs": (nz * C_OUT + n * (12 * C_OUT + 3 * C_IN)) / (c_ms * 1e-3) / 1e9}
+        for n in (4, 16):
+            L3, sq, wk, wd, nz, un = make(args.rho, n=n)
+            c_ms = timed_chunks(L3, sq, wd, 62, 5, cold=True)
+            streams[str(n)] = {"chunk_cold_us": c_ms * 1e3, "fps_cold": n * T * 1e3 / c_ms,
+                               "per_frame_bytes_gbs": n * T * frame_bytes(nz) / (c_ms * 1e-3) / 1e9}
             L3.close()
         extra["streams_per_call"] = streams
 
@@ -281,8 +337,8 @@ def main():
         rec.step(seq[0])
         t0 = time.perf_counter()
         cnt = 0
-        while cnt < 2 * len(order) and time.perf_counter() - t0 < 20.0:
-            rec.step(seq[order[(cnt + 1) % len(order)]])
+        while cnt < 2 * period and time.perf_counter() - t0 < 20.0:
+            rec.step(seq[order[(cnt + 1) % period]])
             cnt += 1
         dt = time.perf_counter() - t0
         cpu = {"value": cnt / dt, "unit": "frames/s", "cores": orc.threads(), "kind": "oracle",
@@ -293,18 +349,25 @@ def main():
             "metric": "frames_per_sec", "value": fps, "unit": "frames/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "i8", "data": "synthetic",
-            "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream per GPU, "
-                                   f"{FRAMES}-frame sequence replayed back and forth",
+            "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream per GPU; one step = "
+                                   f"one chunk of {T} consecutive frames (one rrm_step_seq call) of the {FRAMES}-frame "
+                                   f"sequence walked back and forth",
+                       "frames_per_step": T,
                        "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair",
-                       "measured_nnz_mean": nnz_mean, "measured_density": nnz_mean / C_IN},
+                       "measured_nnz_mean_per_frame": nnz_mean, "measured_density": nnz_mean / C_IN,
+                       "distinct_columns_per_chunk": uniq_mean},
             "dense_equiv_gmacs": fps * DENSE_MACS / 1e9,
             "clocks": clocks,
-            "e2e": {"value": world * 1e3 / e2e_ms, "unit": "frames/s", "h2d_bytes_per_step": C_IN,
-                    "d2h_bytes_per_step": 4 * C_OUT},
-            "gpu_launches": launches,
+            "e2e": {"value": world * T * 1e3 / e2e_ms, "unit": "frames/s", "h2d_bytes_per_step": T * C_IN,
+                    "d2h_bytes_per_step": T * 4 * C_OUT},
+            "gpu_launches": args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": committed_traffic(args.rho), "peak_kind": f"of {peak_kind}",
-                         "kernel": "fc_delta_i8_kernel", "algorithmic_bytes_per_launch": bytes_step},
+                         "kernel": "fc_seq_kernel", "algorithmic_bytes_per_launch": bytes_launch,
+                         "achieved_distinct": achieved_unique, "frac_distinct": achieved_unique / peak,
+                         "distinct_bytes_per_launch": chunk_cold_bytes(uniq_mean, T),
+                         "note": "algorithmic bytes = per-frame bytes x frames per launch; frames of a chunk share "
+                                 "weight columns through L2, so DRAM traffic is the smaller 'distinct' figure"},
             "cpu_baseline": cpu,
             "last_step_stats": st,
         }

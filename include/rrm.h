@@ -118,6 +118,23 @@ int rrm_dense(rrm_layer* layer, const void* X_dev, void* Y_dev, void* stream);
  * `stream`; returns after the stream has been synchronised. */
 int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* stream);
 
+/* A chunk of T consecutive frames in one call: the frame loop of Algorithm 1 for frames t0 .. t0+T-1
+ * (Sec. 3.3 notes that a video may be cut into chunks that are processed on their own).  The result
+ * and the state afterwards are exactly those of T rrm_step calls in a row.
+ *   X_dev  [T] frames, each in the layer's input layout, back to back; read-only
+ *   Y_dev  [T] outputs f(P_t), each in the layer's output layout, back to back; may be NULL
+ * For a lone int8 FC layer all T input deltas are known up front (dI_t = X_t - X_{t-1}), so the T
+ * sparse products W dI_t run in ONE launch and only the running sum P_t = P_{t-1} + W dI_t is
+ * serial; other layers and stacks are stepped frame by frame on `stream`.  The first call with a
+ * larger T than any before allocates scratch memory (T * N * c_out * 4 bytes); later calls do not.
+ * T * N must not exceed 65535.  Asynchronous on `stream`.  After the call rrm_get_stats reports the
+ * counters summed over the chunk's frames. */
+int rrm_step_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream);
+/* T frames through the dense path, each on its own (Y_t = f(F*X_t + b)); RRM state untouched. */
+int rrm_dense_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream);
+/* rrm_step_seq with HOST buffers (copies in, steps, copies out, synchronises `stream`). */
+int rrm_step_seq_host(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream);
+
 /* Synchronises the layer's last stream and fills `host_out`. */
 int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out);
 
@@ -139,6 +156,10 @@ int rrm_net_step(rrm_net* net, const void* frame_dev, void* out_dev, void* strea
 /* Dense evaluation of the stack without touching the RRM state. */
 int rrm_net_dense(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
 int rrm_net_step_host(rrm_net* net, const void* frame_host, void* out_host, void* stream);
+/* Chunks of T frames, as rrm_step_seq / rrm_dense_seq / rrm_step_seq_host; outs = [T] last tensors. */
+int rrm_net_step_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream);
+int rrm_net_dense_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream);
+int rrm_net_step_seq_host(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream);
 
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* host_out);
 /* Copies P_prev of `layer` / the current value of tensor `t` (boundary layout) to dst_dev. */

@@ -67,6 +67,12 @@ def lib():
         "rrm_net_step": [_P, _P, _P, _P],
         "rrm_net_dense": [_P, _P, _P, _P],
         "rrm_net_step_host": [_P, _P, _P, _P],
+        "rrm_step_seq": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_dense_seq": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_step_seq_host": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_net_step_seq": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_net_dense_seq": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_net_step_seq_host": [_P, _P, _P, ctypes.c_int, _P],
         "rrm_net_get_stats": [_P, ctypes.c_int, ctypes.POINTER(Stats)],
         "rrm_net_projection": [_P, ctypes.c_int, _P, _P],
         "rrm_net_tensor": [_P, ctypes.c_int, _P, _P],
@@ -158,6 +164,19 @@ class Net:
         _check(lib().rrm_net_step_host(self._h, _ptr(frame_host), _ptr(out_host), _stream(stream)),
                "rrm_net_step_host")
 
+    def step_seq(self, frames, outs=None, T=None, stream=None):
+        T = frames.shape[0] if T is None else T
+        _check(lib().rrm_net_step_seq(self._h, _ptr(frames), _ptr(outs), T, _stream(stream)), "rrm_net_step_seq")
+
+    def dense_seq(self, frames, outs=None, T=None, stream=None):
+        T = frames.shape[0] if T is None else T
+        _check(lib().rrm_net_dense_seq(self._h, _ptr(frames), _ptr(outs), T, _stream(stream)), "rrm_net_dense_seq")
+
+    def step_seq_host(self, frames_host, outs_host=None, T=None, stream=None):
+        T = frames_host.shape[0] if T is None else T
+        _check(lib().rrm_net_step_seq_host(self._h, _ptr(frames_host), _ptr(outs_host), T, _stream(stream)),
+               "rrm_net_step_seq_host")
+
     def stats(self, layer=0):
         s = Stats()
         _check(lib().rrm_net_get_stats(self._h, layer, ctypes.byref(s)), "rrm_net_get_stats")
@@ -189,8 +208,10 @@ class Net:
             return torch.int32, (n, h, w, (c + 31) // 32)
         return {"f32": torch.float32, "i8": torch.int8, "i32": torch.int32}[kind], (n, c, h, w)
 
-    def new_output(self, t=None):
+    def new_output(self, t=None, frames=None):
         dt, shape = self._tensor_meta(self.n_layers if t is None else t)
+        if frames is not None:
+            shape = (frames,) + tuple(shape)
         return torch.empty(shape, dtype=dt, device="cuda")
 
     def tensor(self, t, stream=None):

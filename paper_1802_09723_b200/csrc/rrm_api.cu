@@ -157,14 +157,35 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
     return RRM_OK;
 }
 
-int ensure_stage(rrm_net* net)
+// T consecutive frames: one launch for the fused FC layer, the per-frame launch sequence otherwise
+int run_seq(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t st, bool dense, bool stateless)
 {
-    if (net->stage_in) return RRM_OK;
+    if (!net || !frames || T < 1) return RRM_ERR_INVALID_ARG;
+    Layer& L0 = net->layers[0];
+    // (a chunk too small to fill the machine goes frame by frame through the split-list kernel instead)
+    if (L0.fc_fused && fc_seq_supported(L0) && T * net->n >= 4) {
+        net->last_stream = st;
+        return fc_seq_run(net, L0, frames, outs, T, dense, stateless, st);
+    }
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
-    RRM_TRY(dev_alloc(net, &net->stage_in, (size_t)bi));
-    RRM_TRY(dev_alloc(net, &net->stage_out, (size_t)bo));
+    for (int t = 0; t < T; ++t)
+        RRM_TRY(run(net, reinterpret_cast<const char*>(frames) + (size_t)t * bi,
+                    outs ? reinterpret_cast<char*>(outs) + (size_t)t * bo : nullptr, st, dense, stateless));
+    return RRM_OK;
+}
+
+// device staging of the *_host entry points, grown on demand to `frames` frames
+int ensure_stage(rrm_net* net, int frames = 1)
+{
+    if (net->stage_in && frames <= net->stage_frames) return RRM_OK;
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    RRM_TRY(dev_alloc(net, &net->stage_in, (size_t)bi * frames));
+    RRM_TRY(dev_alloc(net, &net->stage_out, (size_t)bo * frames));
+    net->stage_frames = frames;
     return RRM_OK;
 }
 
@@ -261,6 +282,41 @@ int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* st
     return rrm_net_step_host(layer, Xt_host, Yt_host, stream);
 }
 
+int rrm_net_step_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream)
+{
+    return run_seq(net, frames_dev, outs_dev, T, (cudaStream_t)stream, false, false);
+}
+int rrm_net_dense_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream)
+{
+    return run_seq(net, frames_dev, outs_dev, T, (cudaStream_t)stream, true, true);
+}
+int rrm_step_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream)
+{
+    return rrm_net_step_seq(layer, X_dev, Y_dev, T, stream);
+}
+int rrm_dense_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream)
+{
+    return rrm_net_dense_seq(layer, X_dev, Y_dev, T, stream);
+}
+int rrm_net_step_seq_host(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream)
+{
+    if (!net || !frames_host || T < 1) return RRM_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    RRM_TRY(ensure_stage(net, T));
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    RRM_CUDA_TRY(cudaMemcpyAsync(net->stage_in, frames_host, (size_t)bi * T, cudaMemcpyHostToDevice, st));
+    RRM_TRY(run_seq(net, net->stage_in, outs_host ? net->stage_out : nullptr, T, st, false, false));
+    if (outs_host) RRM_CUDA_TRY(cudaMemcpyAsync(outs_host, net->stage_out, (size_t)bo * T, cudaMemcpyDeviceToHost, st));
+    RRM_CUDA_TRY(cudaStreamSynchronize(st));
+    return RRM_OK;
+}
+int rrm_step_seq_host(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream)
+{
+    return rrm_net_step_seq_host(layer, X_host, Y_host, T, stream);
+}
+
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
 {
     if (!net || !h || layer < 0 || layer >= (int)net->layers.size()) return RRM_ERR_INVALID_ARG;
@@ -277,13 +333,22 @@ int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
     h->error_word = errw;
     if (L.fc_fused) {
         unsigned long long tot[2] = {0, 0};
-        std::vector<unsigned long long> v((size_t)d.n * 2);
-        RRM_CUDA_TRY(cudaMemcpy(v.data(), L.fc_nnz, v.size() * 8, cudaMemcpyDeviceToHost));
-        for (int s = 0; s < d.n; ++s) { tot[0] += v[s * 2]; tot[1] += v[s * 2 + 1]; }
+        int frames = 1;
+        if (L.seq_last_T > 0) {                  // the last call was a chunk: counters cover all its frames
+            frames = L.seq_last_T;
+            RRM_TRY(fc_seq_stats(net->layers[layer], &tot[0], &tot[1]));
+            h->in_elems *= frames;
+            h->out_pixels *= frames;
+            h->dense_macs *= frames;
+        } else {
+            std::vector<unsigned long long> v((size_t)d.n * 2);
+            RRM_CUDA_TRY(cudaMemcpy(v.data(), L.fc_nnz, v.size() * 8, cudaMemcpyDeviceToHost));
+            for (int s = 0; s < d.n; ++s) { tot[0] += v[s * 2]; tot[1] += v[s * 2 + 1]; }
+        }
         h->nnz_elems = (int64_t)tot[0];
-        h->in_pixels = (int64_t)d.n * ((d.c_in + 31) / 32);
+        h->in_pixels = (int64_t)frames * d.n * ((d.c_in + 31) / 32);
         h->active_in_pixels = (int64_t)tot[1];
-        h->active_out_pixels = tot[0] ? d.n : 0;
+        h->active_out_pixels = tot[0] ? (int64_t)frames * d.n : 0;
         h->active_macs = (int64_t)tot[0] * d.c_out;
         h->variant = RRM_VARIANT_GATHER;
         return RRM_OK;

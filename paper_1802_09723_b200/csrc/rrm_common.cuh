@@ -74,6 +74,13 @@ struct Layer {
     int xs_cur = 0;
     void* fc_scratch = nullptr;             // per-stream non-zero lists of the two-kernel form
     unsigned long long* fc_nnz = nullptr;   // [0] nnz elements, [1] active groups of 32 (cleared by the kernel's last CTA)
+    // chunk-of-frames form of the fused FC path
+    int32_t* seq_dP = nullptr;              // [seq_cap][n][c_out] per-frame projection deltas
+    unsigned* seq_stat = nullptr;           // [seq_cap * n][2] per frame and stream: non-zeros, active groups of 32
+    unsigned* seq_counters = nullptr;       // [n][slices] arrival counters (zero between launches)
+    int seq_cap = 0;                        // frames the scratch arrays hold
+    int seq_lanes = 0;                      // 0: pick the slice width per call; 8 / 16 / 32: forced (tuning)
+    int seq_last_T = 0;                     // frames of the most recent chunk (0: last call was a single-frame step)
 };
 
 }  // namespace rrm
@@ -88,6 +95,7 @@ struct rrm_net {
     cudaStream_t last_stream = nullptr;
     void* stage_in = nullptr;         // device staging for the *_host entry points
     void* stage_out = nullptr;
+    int stage_frames = 0;             // frames the staging buffers hold
     std::vector<void*> allocs;        // everything to free
 };
 
@@ -98,6 +106,13 @@ int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_
 int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool dense, bool stateless,
                  cudaStream_t st);
 int fc_fused_projection(rrm_net* net, Layer& L, void* P_dev, cudaStream_t st);
+
+// ---- rrm_fc_seq.cu
+int fc_seq_create(rrm_net* net, Layer& L);
+bool fc_seq_supported(const Layer& L);
+int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool dense, bool stateless,
+               cudaStream_t st);
+int fc_seq_stats(Layer& L, unsigned long long* nnz, unsigned long long* groups);
 
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);

@@ -505,6 +505,7 @@ int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_
     RRM_CUDA_TRY(cudaDeviceSynchronize());
     L.xs_cur = 0;
     L.fc_fused = true;
+    RRM_TRY(fc_seq_create(net, L));
     return RRM_OK;
 }
 
@@ -534,6 +535,7 @@ int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool de
         L.xs_cur ^= 1;
         p.P = reinterpret_cast<int32_t*>(L.P);
         p.stat = L.fc_nnz;
+        L.seq_last_T = 0;
     }
     if (n < FC_TWO_KERNEL_MIN_STREAMS) {
         dim3 grid(FC_CL, slices, n);

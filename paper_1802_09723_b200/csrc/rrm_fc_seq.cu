@@ -1,0 +1,423 @@
+// Delta-FC over a chunk of T consecutive frames in one launch (Algorithm 1, FC branch, with the
+// frame loop moved inside the kernel).
+//
+// For a lone linear layer the deltas of all frames of a chunk are known up front:
+//   dI_t = X_t - X_{t-1}   (X_{-1} = the stored snapshot),     dP_t = W dI_t   (Eq. 4),
+//   P_t  = P_{t-1} + dP_t  (Eq. 5) is a running sum over t,    Y_t = f(P_t).
+// So the T sparse products are independent and only the running sum is serial.  One launch,
+// one CTA per (512-output slice, frame, stream):
+//   1. the CTA scans X_t against X_{t-1} with 128-bit loads (all issued up front) and compacts the
+//      non-zero delta entries (index, delta) into a list in shared memory: a 16-bit mask per
+//      16-byte chunk, a warp prefix sum, one shared-memory atomic per warp to reserve list space
+//      (the list is unordered; integer sums do not depend on the order, so results stay bit-exact);
+//   2. each warp takes every 8th list entry and loads the 512-byte slice of that entry's weight
+//      column (weights are stored transposed: one contiguous C_out-byte row per input) with one
+//      fully coalesced 128-bit load per lane, many columns in flight, accumulating d_j * W[:, j];
+//   3. the 8 warps' partial sums are added through shared memory into the slice of dP_t (scratch);
+//   4. the CTA that finishes LAST for a given (stream, slice) - found with one atomic counter,
+//      nobody waits - adds the T slices onto the stored projection in frame order, applies f and
+//      writes Y_0 .. Y_{T-1}.
+// Cost: the weight columns of the non-zero entries (HBM; frames of a chunk share columns through L2).
+#include "rrm_common.cuh"
+
+namespace rrm {
+
+constexpr int SQ_THREADS = 256;
+constexpr int SQ_WARPS = SQ_THREADS / 32;
+constexpr int SQ_TAIL = 16;                    // frames one thread of the closing sum holds (chunks of up to 2 * SQ_TAIL frames)
+constexpr int SQ_PT = 4;                       // 16-byte chunks scanned per thread
+constexpr int SQ_MAX_C_IN = 16 * SQ_PT * SQ_THREADS;   // 16384 (entry format: 14-bit index)
+
+struct FcSeqParams {
+    const int8_t* x;         // [T][n][c_in] frames of the chunk
+    const int8_t* xprev;     // [n][c_in] snapshot = frame before the chunk; nullptr: every entry active, d = x
+    int8_t* xnext;           // [n][c_in] receives frame T-1, or nullptr
+    const int8_t* Wt;        // [c_in][c_out]
+    const int32_t* bias;     // non-null: frames are independent, P_t = bias + dP_t (dense evaluation)
+    int32_t* P;              // [n][c_out] stored projection (chained mode: read and updated), may be nullptr with bias
+    int32_t* dP;             // [T][n][c_out] scratch
+    void* Y;                 // [T][n][c_out] int32 (shift < 0) or int8, or nullptr
+    unsigned* counters;      // [n][slices], zero on entry, zero again on exit
+    unsigned* stat;          // [T*n][2]: non-zero entries / active groups of 32 inputs per frame, or nullptr
+    int T, n, c_in, c_out, shift, act;
+};
+
+__device__ __forceinline__ int seq_apply_f(int v, int shift, int act)
+{
+    if (shift > 0) v = (v + (1 << (shift - 1))) >> shift;
+    v = max(-127, min(127, v));
+    if (act == RRM_ACT_RELU) v = max(v, 0);
+    return v;
+}
+
+// one flag bit per non-zero byte of v, packed into the low 4 bits
+__device__ __forceinline__ unsigned nonzero_bytes(unsigned v)
+{
+    v |= v >> 4; v |= v >> 2; v |= v >> 1;
+    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
+}
+
+// acc[i] += w_i * d for the 16 int8 weights in w: dp4a against a selector holding d in one byte
+// lane; a delta outside int8 range (|d| <= 254) is split into two in-range halves.
+__device__ __forceinline__ void fma16(int (&acc)[16], const uint4& w, int d)
+{
+    const unsigned ww[4] = {w.x, w.y, w.z, w.w};
+    const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
+    const int dl = d - dh;
+    const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
+    #pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        #pragma unroll
+        for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
+    }
+    if (dh != 0) {
+        #pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            #pragma unroll
+            for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
+        }
+    }
+}
+
+// LANES: lanes of a warp that span one column slice (16 bytes each): the CTA owns OW = 16 * LANES
+// outputs and a warp-wide load fetches 32 / LANES columns.  Narrow slices mean more CTAs and fewer
+// list entries per lane (a shorter chain of dependent memory round trips); wide slices mean fewer
+// redundant scans.  The host picks LANES from the size of the chunk.
+// DEEP: 16 instead of 8 loads in flight per lane at 2 instead of 3 CTAs per SM; pays when the whole
+// grid is resident at once (each CTA's chain of round trips is what the launch waits for).
+template <int LANES, bool DEEP>
+__global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqParams p)
+{
+    constexpr int OW = 16 * LANES;                 // outputs per CTA
+    constexpr int CPW = 32 / LANES;                // columns per warp-wide load
+    constexpr int CPR = CPW * SQ_WARPS;            // columns per CTA-wide round
+    constexpr int SQ_U = DEEP ? 16 : 8;            // rounds in flight (16-byte loads per lane)
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    int* s_red = reinterpret_cast<int*>(s_dyn);                                   // [SQ_WARPS][OW]
+    uint32_t* s_list = reinterpret_cast<uint32_t*>(s_dyn + SQ_WARPS * OW * 4);     // [c_in] index | (delta + 256) << 16
+    __shared__ int s_count, s_groups, s_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int slice = blockIdx.x;
+    const int t = blockIdx.y / p.n, s = blockIdx.y - t * p.n;
+    const int C = p.c_in, K = p.c_out;
+    const int nchunks = C >> 4;
+    const int slices = gridDim.x;
+    const int width = min(OW, K - slice * OW);
+
+    if (tid == 0) { s_count = 0; s_groups = 0; }
+    // ---- 1. scan: chunk i*256 + tid for i < SQ_PT, all loads first
+    const uint4* xt4 = reinterpret_cast<const uint4*>(p.x + ((size_t)t * p.n + s) * C);
+    const uint4* xp4 = nullptr;
+    if (p.xprev) xp4 = reinterpret_cast<const uint4*>(t > 0 ? p.x + ((size_t)(t - 1) * p.n + s) * C : p.xprev + (size_t)s * C);
+    uint4 a[SQ_PT], b[SQ_PT];
+    #pragma unroll
+    for (int i = 0; i < SQ_PT; ++i) {
+        const int chunk = i * SQ_THREADS + tid;
+        a[i] = make_uint4(0, 0, 0, 0);
+        b[i] = a[i];
+        if (chunk < nchunks) {
+            a[i] = __ldg(xt4 + chunk);
+            if (xp4) b[i] = __ldg(xp4 + chunk);
+        }
+    }
+    // while the frame is on its way: touch one line in every 2 MiB of the weights, so that the
+    // address translations the gather will need are fetched now instead of on its first loads
+    {
+        const size_t wbytes = (size_t)C * K;
+        const size_t off = (size_t)tid << 21;
+        if (off < wbytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.Wt + off));
+        // likewise the stored projection (or the bias), which only the closing sum reads
+        const int32_t* pp = p.bias ? p.bias + slice * OW : p.P + (size_t)s * K + slice * OW;
+        if (t == 0 && tid * 32 < width) asm volatile("prefetch.global.L2 [%0];" ::"l"(pp + tid * 32));
+    }
+    __syncthreads();                                         // s_count is initialised
+    int groups = 0;
+    #pragma unroll
+    for (int i = 0; i < SQ_PT; ++i) {
+        const int chunk = i * SQ_THREADS + tid;
+        if (i * SQ_THREADS >= nchunks) break;                // uniform
+        unsigned m = 0;
+        if (chunk < nchunks)
+            m = xp4 ? (nonzero_bytes(a[i].x ^ b[i].x) | nonzero_bytes(a[i].y ^ b[i].y) << 4 |
+                       nonzero_bytes(a[i].z ^ b[i].z) << 8 | nonzero_bytes(a[i].w ^ b[i].w) << 12)
+                    : 0xffffu;
+        const int local = __popc(m);
+        int incl = local;
+        #pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int wtot = __shfl_sync(0xffffffffu, incl, 31);
+        if (wtot == 0) continue;                             // uniform inside the warp
+        int base = 0;
+        if (lane == 31) base = atomicAdd(&s_count, wtot);
+        base = __shfl_sync(0xffffffffu, base, 31);
+        // groups of 32 inputs = pairs of neighbouring chunks (an even/odd lane pair)
+        const unsigned other = __shfl_xor_sync(0xffffffffu, m, 1);
+        groups += ((lane & 1) == 0 && (m | other)) ? 1 : 0;
+        if (m) {
+            int off = base + incl - local;
+            const unsigned aw[4] = {a[i].x, a[i].y, a[i].z, a[i].w}, bw[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
+            #pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                if (m >> k & 1u) {
+                    const int xa = (int)(int8_t)(aw[k >> 2] >> (8 * (k & 3)));
+                    const int xb = (int)(int8_t)(bw[k >> 2] >> (8 * (k & 3)));
+                    s_list[off++] = (uint32_t)(chunk * 16 + k) | (uint32_t)(xa - xb + 256) << 16;
+                }
+            }
+        }
+    }
+    // the new snapshot is the chunk's last frame; the CTAs of slice 0 store it
+    if (p.xnext && t == p.T - 1 && slice == 0) {
+        #pragma unroll
+        for (int i = 0; i < SQ_PT; ++i) {
+            const int chunk = i * SQ_THREADS + tid;
+            if (chunk < nchunks) reinterpret_cast<uint4*>(p.xnext + (size_t)s * C)[chunk] = a[i];
+        }
+    }
+    if (p.stat && slice == 0) {
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) groups += __shfl_down_sync(0xffffffffu, groups, o);
+        if (lane == 0 && groups) atomicAdd(&s_groups, groups);
+    }
+    __syncthreads();
+    const int total = s_count;
+    if (p.stat && slice == 0 && tid == 0) {
+        p.stat[blockIdx.y * 2 + 0] = (unsigned)total;
+        p.stat[blockIdx.y * 2 + 1] = (unsigned)s_groups;
+    }
+
+    // ---- 2. gather: LANES lanes x 16 bytes span the slice; SQ_U rounds of CPR columns in flight
+    const int sub = lane % LANES, grp = warp * CPW + lane / LANES;
+    const int o0 = slice * OW + sub * 16;
+    int acc[16];
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0;
+    if (o0 < K) {                                            // K is a multiple of 16
+        const int8_t* wbase = p.Wt + o0;
+        for (int e = grp; e < total; e += SQ_U * CPR) {
+            uint32_t ent[SQ_U];
+            uint4 w[SQ_U];
+            #pragma unroll
+            for (int u = 0; u < SQ_U; ++u) {
+                const int eu = e + u * CPR;
+                ent[u] = eu < total ? s_list[eu] : 0xffffffffu;
+            }
+            #pragma unroll
+            for (int u = 0; u < SQ_U; ++u)
+                w[u] = ent[u] != 0xffffffffu
+                           ? __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(ent[u] & 0xffffu) * K))
+                           : make_uint4(0, 0, 0, 0);
+            #pragma unroll
+            for (int u = 0; u < SQ_U; ++u)
+                if (ent[u] != 0xffffffffu) fma16(acc, w[u], (int)(ent[u] >> 16) - 256);
+        }
+    }
+    // ---- 3. add the partial sums: the column groups of a warp by shuffles, the warps through shared memory
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        #pragma unroll
+        for (int o = LANES; o < 32; o <<= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+    }
+    if (lane < LANES) {
+        #pragma unroll
+        for (int i = 0; i < 16; i += 4)
+            *reinterpret_cast<int4*>(&s_red[warp * OW + lane * 16 + i]) = make_int4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+    }
+    __syncthreads();
+    for (int o = tid; o < width; o += SQ_THREADS) {
+        int v = 0;
+        #pragma unroll
+        for (int w = 0; w < SQ_WARPS; ++w) v += s_red[w * OW + o];
+        p.dP[((size_t)t * p.n + s) * K + slice * OW + o] = v;
+    }
+    // ---- 4. whoever finishes last for this (stream, slice) runs the sum over the frames
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned old = atomicAdd(&p.counters[s * slices + slice], 1u);
+        s_last = (old == (unsigned)(p.T - 1));
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // every thread owns 4 neighbouring outputs and a contiguous share of the frames: it sums its
+    // share (all loads in flight), the shares are chained through shared memory, then it writes
+    // its frames' outputs.  FS = threads per output group = frame shares.
+    constexpr int OG = OW / 4;                                // output groups of 4
+    constexpr int FS = SQ_THREADS / OG;                       // frame shares (2 for OW = 512 ... 8 for OW = 128)
+    const int og = tid % OG, fs = tid / OG;
+    const int per = (p.T + FS - 1) / FS;
+    const int tb = fs * per, te = min(p.T, tb + per);
+    const int o = slice * OW + og * 4;
+    const bool live = og * 4 < width;                         // width is a multiple of 16
+    const size_t stride = (size_t)p.n * K;
+    const int32_t* dp = p.dP + (size_t)s * K + o;
+    // the frames of this share stay in registers between the two steps (host guarantees per <= SQ_TAIL)
+    int4 d[SQ_TAIL];
+    int4 sum = make_int4(0, 0, 0, 0);
+    #pragma unroll
+    for (int u = 0; u < SQ_TAIL; ++u) {
+        d[u] = (live && tb + u < te) ? __ldcg(reinterpret_cast<const int4*>(dp + (size_t)(tb + u) * stride)) : make_int4(0, 0, 0, 0);
+    }
+    #pragma unroll
+    for (int u = 0; u < SQ_TAIL; ++u) { sum.x += d[u].x; sum.y += d[u].y; sum.z += d[u].z; sum.w += d[u].w; }
+    int4* s_share = reinterpret_cast<int4*>(s_dyn);           // [FS][OG], reuses the reduction buffer
+    __syncthreads();
+    s_share[fs * OG + og] = sum;
+    __syncthreads();
+    if (!live) return;
+    int4 v;
+    if (p.bias) {
+        v = *reinterpret_cast<const int4*>(p.bias + o);
+    } else {
+        v = *reinterpret_cast<const int4*>(p.P + (size_t)s * K + o);
+        for (int f = 0; f < fs; ++f) {
+            const int4 q = s_share[f * OG + og];
+            v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+    }
+    const int4 bias4 = v;
+    #pragma unroll
+    for (int u = 0; u < SQ_TAIL; ++u) {
+        if (tb + u < te) {
+            if (p.bias) v = make_int4(bias4.x + d[u].x, bias4.y + d[u].y, bias4.z + d[u].z, bias4.w + d[u].w);
+            else { v.x += d[u].x; v.y += d[u].y; v.z += d[u].z; v.w += d[u].w; }
+            if (p.Y) {
+                const size_t oi = ((size_t)(tb + u) * p.n + s) * K + o;
+                if (p.shift < 0) {
+                    *reinterpret_cast<int4*>(reinterpret_cast<int32_t*>(p.Y) + oi) = v;
+                } else {
+                    char4 q;
+                    q.x = (signed char)seq_apply_f(v.x, p.shift, p.act); q.y = (signed char)seq_apply_f(v.y, p.shift, p.act);
+                    q.z = (signed char)seq_apply_f(v.z, p.shift, p.act); q.w = (signed char)seq_apply_f(v.w, p.shift, p.act);
+                    *reinterpret_cast<char4*>(reinterpret_cast<int8_t*>(p.Y) + oi) = q;
+                }
+            }
+        }
+    }
+    // the share that holds the last frame stores the projection
+    if (p.P && te == p.T && tb < te) *reinterpret_cast<int4*>(p.P + (size_t)s * K + o) = v;
+    if (tid == 0) p.counters[s * slices + slice] = 0;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+static size_t seq_dyn_smem(int c_in, int lanes) { return (size_t)SQ_WARPS * 16 * lanes * 4 + (size_t)c_in * 4; }
+
+static int seq_ensure(rrm_net* net, Layer& L, int T)
+{
+    if (T <= L.seq_cap) return RRM_OK;
+    const int K = L.d.c_out, n = L.d.n;
+    void* dP = nullptr;
+    void* stat = nullptr;
+    if (cudaMalloc(&dP, (size_t)T * n * K * 4) != cudaSuccess) { cudaGetLastError(); return RRM_ERR_ALLOC; }
+    if (cudaMalloc(&stat, (size_t)T * n * 2 * 4) != cudaSuccess) { cudaFree(dP); cudaGetLastError(); return RRM_ERR_ALLOC; }
+    net->allocs.push_back(dP);
+    net->allocs.push_back(stat);
+    L.seq_dP = reinterpret_cast<int32_t*>(dP);
+    L.seq_stat = reinterpret_cast<unsigned*>(stat);
+    L.seq_cap = T;
+    return RRM_OK;
+}
+
+int fc_seq_create(rrm_net* net, Layer& L)
+{
+    const int K = L.d.c_out, n = L.d.n;
+    const int slices = ceil_div(K, 16 * 8);                  // the narrowest slice the kernel is built for
+    void* c = nullptr;
+    if (cudaMalloc(&c, (size_t)n * slices * 4) != cudaSuccess) { cudaGetLastError(); return RRM_ERR_ALLOC; }
+    net->allocs.push_back(c);
+    RRM_CUDA_TRY(cudaMemset(c, 0, (size_t)n * slices * 4));
+    L.seq_counters = reinterpret_cast<unsigned*>(c);
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 16)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 8)));
+    return seq_ensure(net, L, 1);
+}
+
+bool fc_seq_supported(const Layer& L) { return L.fc_fused && L.d.c_in <= SQ_MAX_C_IN; }
+
+// T frames of every stream in one launch.  dense: every entry is visited and frames are independent
+// (P_t = b + W X_t); stateless: the RRM state (snapshot, stored projection) is left untouched.
+int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool dense, bool stateless, cudaStream_t st)
+{
+    const int C = L.d.c_in, K = L.d.c_out, n = L.d.n;
+    if (T < 1) return RRM_ERR_INVALID_ARG;
+    if ((long long)T * n > 65535) return RRM_ERR_CAPACITY;
+    RRM_TRY(seq_ensure(net, L, T));
+    FcSeqParams p;
+    p.x = reinterpret_cast<const int8_t*>(X_dev);
+    p.Wt = L.Wt;
+    p.dP = L.seq_dP;
+    p.Y = Y_dev;
+    p.counters = L.seq_counters;
+    p.T = T; p.n = n; p.c_in = C; p.c_out = K; p.shift = L.d.shift; p.act = L.d.act;
+    if (dense) {
+        p.xprev = nullptr;
+        p.bias = reinterpret_cast<const int32_t*>(L.bias);
+        p.stat = nullptr;
+        if (stateless) { p.xnext = nullptr; p.P = nullptr; }
+        else { p.xnext = L.xs[L.xs_cur ^ 1]; L.xs_cur ^= 1; p.P = reinterpret_cast<int32_t*>(L.P); }
+    } else {
+        p.xprev = L.xs[L.xs_cur];
+        p.xnext = L.xs[L.xs_cur ^ 1];
+        L.xs_cur ^= 1;
+        p.bias = nullptr;
+        p.P = reinterpret_cast<int32_t*>(L.P);
+        p.stat = L.seq_stat;
+        L.seq_last_T = T;
+    }
+    // slice width: the widest (fewest redundant scans, one wave of CTAs with a short chain of dependent
+    // round trips each), narrowed while the grid would leave a good part of the machine idle
+    int lanes = L.seq_lanes;
+    if (lanes == 0) {
+        lanes = 32;
+        while (lanes > 8 && (long long)ceil_div(K, 16 * lanes) * T * n < 200) lanes /= 2;
+    }
+    // the closing sum keeps SQ_TAIL frames per thread: longer chunks go out in pieces, each piece
+    // taking the frame before it (still in X) as its "previous" frame
+    const int piece_max = SQ_TAIL * (SQ_THREADS / (4 * lanes));
+    const int8_t* snapshot = p.xprev;
+    int8_t* const xnext = p.xnext;
+    const size_t ybytes = (size_t)n * K * (L.d.shift < 0 ? 4 : 1);
+    for (int t0 = 0; t0 < T; t0 += piece_max) {
+        const int piece = T - t0 < piece_max ? T - t0 : piece_max;
+        p.x = reinterpret_cast<const int8_t*>(X_dev) + (size_t)t0 * n * C;
+        p.xprev = dense ? nullptr : (t0 == 0 ? snapshot : p.x - (size_t)n * C);
+        p.xnext = t0 + piece == T ? xnext : nullptr;
+        p.Y = Y_dev ? reinterpret_cast<char*>(Y_dev) + (size_t)t0 * ybytes : nullptr;
+        p.stat = dense ? nullptr : L.seq_stat + (size_t)t0 * n * 2;
+        p.T = piece;
+        dim3 grid(ceil_div(K, 16 * lanes), piece * n);
+        const size_t dyn = seq_dyn_smem(C, lanes);
+        if (lanes == 32 && grid.x * grid.y <= 2 * 148) fc_seq_kernel<32, true><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else if (lanes == 32) fc_seq_kernel<32, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else if (lanes == 16) fc_seq_kernel<16, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else fc_seq_kernel<8, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+    }
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
+// Sums the per-frame counters of the last chunk: non-zero delta entries and active groups of 32 inputs.
+int fc_seq_stats(Layer& L, unsigned long long* nnz, unsigned long long* groups)
+{
+    const size_t cnt = (size_t)L.seq_last_T * L.d.n * 2;
+    std::vector<unsigned> h(cnt);
+    RRM_CUDA_TRY(cudaMemcpy(h.data(), L.seq_stat, cnt * 4, cudaMemcpyDeviceToHost));
+    *nnz = 0; *groups = 0;
+    for (size_t i = 0; i < cnt; i += 2) { *nnz += h[i]; *groups += h[i + 1]; }
+    return RRM_OK;
+}
+
+}  // namespace rrm

@@ -110,3 +110,110 @@ def test_fc_step_host_matches_device_call():
         layer.step_host(torch.from_numpy(seq[t]).pin_memory(), out)
         np.testing.assert_array_equal(out.numpy(), orc.dense_forward([spec], seq[t])[0][1])
     layer.close()
+
+
+# ------------------------------------------------------------------ chunks of frames in one call
+def _run_chunks(spec, seq, n, chunks):
+    """Feeds `seq` ([F][n][c_in]) in chunks of the given lengths and checks every frame's output,
+    the stored projection after each chunk and the summed counters against the oracle."""
+    rrm = _rrm()
+    layer = rrm.layer_from_spec(spec, n=n)
+    rec = orc.Recurrence([spec], n=n)
+    frames = dev(seq)
+    t0 = 0
+    for T in chunks:
+        Y = layer.new_output(frames=T)
+        layer.step_seq(frames[t0:t0 + T], Y, T)
+        got = Y.cpu().numpy().astype(np.int64)
+        nnz = macs = 0
+        for i in range(T):
+            tens_d, P_d = orc.dense_forward([spec], seq[t0 + i])
+            np.testing.assert_array_equal(got[i], tens_d[1].astype(np.int64), err_msg=f"frame {t0 + i}")
+            rec.step(seq[t0 + i])
+            nnz += rec.nnz[0]
+            macs += rec.macs[0]
+        np.testing.assert_array_equal(layer.projection(0).cpu().numpy().astype(np.int64), P_d[0])
+        st = layer.stats(0)
+        assert st["nnz_elems"] == nnz and st["active_macs"] == macs and st["error_word"] == 0, st
+        assert st["in_elems"] == T * n * spec.c_in
+        t0 += T
+    # a single-frame step after the chunks continues from the same state
+    if t0 < seq.shape[0]:
+        Y1 = layer.new_output()
+        layer.step(frames[t0], Y1)
+        np.testing.assert_array_equal(Y1.cpu().numpy().astype(np.int64),
+                                      orc.dense_forward([spec], seq[t0])[0][1].astype(np.int64))
+    layer.close()
+
+
+@pytest.mark.parametrize("rho", [0.01, 0.05, 0.20])
+def test_fc6_chunk_of_32_frames_bit_exact(rho):
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=32, rho=rho, seed=21)
+    _run_chunks(spec, seq, 1, [32])
+
+
+def test_fc6_chunks_of_uneven_length_and_streams():
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=14, rho=0.05, seed=26, n=3)
+    seq[5, 1] = seq[4, 1]                 # one stream with zero delta in one frame
+    seq[9] = seq[8]                       # a frame with zero delta in every stream
+    _run_chunks(spec, seq, 3, [1, 7, 2, 3])
+
+
+@pytest.mark.parametrize("c_in,c_out,shift,act", [(64, 48, -1, "none"), (160, 528, 6, "relu"),
+                                                  (1024 + 32, 16, 5, "none"), (32, 1040, -1, "none"),
+                                                  (16384, 128, -1, "none")])
+def test_fc_chunks_small_and_ragged_shapes(c_in, c_out, shift, act):
+    rng = np.random.default_rng(c_in + c_out + 1)
+    spec = LayerSpec("fc", "i8", c_in, 1, 1, c_out, act=act, shift=shift, src=0)
+    spec.weight = rng.integers(-127, 128, size=(c_out, c_in, 1, 1)).astype(np.int8)
+    spec.bias = rng.integers(-500, 501, size=c_out).astype(np.int32)
+    seq = wl.fc_run_sequence(frames=7, c_in=c_in, rho=0.25, run=8, seed=c_in, n=2)
+    seq[3] = seq[2]                       # zero delta
+    seq[4] = 127 - seq[3]                 # every entry changes
+    seq[5] = -seq[4]                      # deltas up to +-254 (split into two int8 factors)
+    _run_chunks(spec, seq, 2, [3, 3])
+
+
+def test_fc_chunk_equals_single_frame_steps_and_dense_chunk_is_stateless():
+    rrm = _rrm()
+    spec = wl.fc6_i8(c_in=2048, c_out=1024)[0]
+    seq = wl.fc_run_sequence(frames=9, c_in=2048, rho=0.1, seed=27, n=2)
+    a, b = rrm.layer_from_spec(spec, n=2), rrm.layer_from_spec(spec, n=2)
+    frames = dev(seq)
+    Ya, Yb = a.new_output(frames=8), b.new_output()
+    a.step_seq(frames[:8], Ya, 8)
+    for t in range(8):
+        b.step(frames[t], Yb)
+        assert torch.equal(Ya[t], Yb), t
+    assert torch.equal(a.projection(0), b.projection(0))
+    # dense chunk: every frame on its own, state untouched
+    Yd = a.new_output(frames=3)
+    a.dense_seq(frames[2:5], Yd, 3)
+    for i in range(3):
+        np.testing.assert_array_equal(Yd[i].cpu().numpy(), orc.dense_forward([spec], seq[2 + i])[0][1])
+    Y1 = a.new_output()
+    a.step(frames[8], Y1)
+    np.testing.assert_array_equal(Y1.cpu().numpy(), orc.dense_forward([spec], seq[8])[0][1])
+    a.close(); b.close()
+
+
+def test_fc_chunk_host_entry_point():
+    rrm = _rrm()
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=6, rho=0.05, seed=28)
+    layer = rrm.layer_from_spec(spec)
+    xin = torch.from_numpy(seq).pin_memory()
+    out = torch.empty((6, 1, 4096, 1, 1), dtype=torch.int32).pin_memory()
+    layer.step_seq_host(xin, out, 6)
+    for t in range(6):
+        np.testing.assert_array_equal(out[t].numpy(), orc.dense_forward([spec], seq[t])[0][1])
+    layer.close()
+
+
+def test_fc6_chunk_longer_than_one_launch_holds():
+    """40 frames exceed what one launch's closing sum keeps per thread: the call goes out in pieces."""
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=41, rho=0.01, seed=29)
+    _run_chunks(spec, seq, 1, [40])
