@@ -139,6 +139,95 @@ def run_reference(args, rank, world):
     }))
 
 
+# ------------------------------------------------------------------------------------------------
+# Secondary workloads (the convolution configurations): python bench.py --workload cfg1|cfg3_f32|...
+# One step = one frame through rrm_net_step (Algorithm 1, one iteration of the frame loop).
+# ------------------------------------------------------------------------------------------------
+CONV_WORKLOADS = ("cfg1", "cfg3_f32", "cfg3_i8", "cfg4", "cfg5")
+FFMA_TMACS, DP4A_TMACS, POPC_TBITMACS = 37.2, 74.5, 148.9      # derived ALU peaks: lanes x clock
+
+
+def conv_workload(name, frames=None):
+    import workloads as wl
+    if name == "cfg1":
+        return wl.single_conv_f32(), wl.block_redraw_sequence(frames=frames or 8), 1, "f32"
+    if name == "cfg3_f32":
+        return wl.alexnet_convs("f32"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="f32", seed=31), 1, "f32"
+    if name == "cfg3_i8":
+        return wl.alexnet_convs("i8"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="i8", seed=32), 1, "i8"
+    if name == "cfg4":
+        return (wl.resnet18_convs(), wl.moving_rect_video(frames=frames or 64, hw=224, dtype="i8", seed=41, n=4,
+                                                          bg_redraw=0.02), 4, "i8")
+    if name == "cfg5":
+        return wl.xnor_alexnet_convs(), wl.moving_rect_video(frames=frames or 128, hw=227, dtype="i8", seed=51), 1, "i8+bin"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def run_conv(args):
+    import torch
+    import workloads as wl
+    import paper_1802_09723_b200 as rrm
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    specs, video, n, dtype = conv_workload(args.workload, args.frames)
+    F = video.shape[0]
+    net = rrm.net_from_specs(specs, n=n, variant=args.variant)
+    frames = [torch.from_numpy(np.ascontiguousarray(video[t])).cuda() for t in range(F)]
+    order = pingpong(F)
+    period = len(order)
+    out = net.new_output()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    dense_macs = wl.dense_macs(specs) * n
+
+    def timed(call, steps, warmup, cold=True):
+        net.keyframe(frames[order[0]], out)
+        for i in range(warmup):
+            call(frames[order[(i + 1) % period]], out)
+        torch.cuda.synchronize()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps):
+            if cold:
+                flush.fill_(i & 0xff)
+            evs[i][0].record(stream)
+            call(frames[order[(warmup + i + 1) % period]], out)
+            evs[i][1].record(stream)
+        torch.cuda.synchronize()
+        return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    ms = timed(net.step, args.steps, args.warmup)
+    clocks = sampler.stop()
+    per_layer = []
+    tot_active = 0
+    for l, sp in enumerate(specs):
+        st = net.stats(l)
+        tot_active += st["active_macs"]
+        per_layer.append({"layer": sp.name, "rho": st["nnz_elems"] / max(1, st["in_elems"]),
+                          "active_in_pixels": st["active_in_pixels"] / max(1, st["in_pixels"]),
+                          "active_out_pixels": st["active_out_pixels"] / max(1, st["out_pixels"]),
+                          "active_macs": st["active_macs"], "dense_macs": st["dense_macs"], "variant": st["variant"]})
+    ms_warm = timed(net.step, args.steps, args.warmup, cold=False)
+    ms_dense = timed(net.dense, max(8, args.steps // 4), 3)
+    line = {
+        "metric": "frames_per_sec", "value": n * 1e3 / ms, "unit": "frames/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": dtype, "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {len(specs)} conv layers, {n} stream(s), {F}-frame video walked back and forth; "
+                               f"one step = one frame of every stream through rrm_net_step", "variant": args.variant,
+                   "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair"},
+        "dense_equiv_gmacs": n * 1e3 / ms * (dense_macs / n) / 1e9,
+        "ms_per_step_warm": ms_warm, "ms_per_step_dense_path": ms_dense, "speedup_vs_own_dense": ms_dense / ms,
+        "active_macs_last_step": tot_active, "dense_macs_per_step": dense_macs,
+        "active_gmacs_per_s": tot_active / ms / 1e6,
+        "clocks": clocks, "per_layer_last_step": per_layer,
+    }
+    print(json.dumps(line))
+    net.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -148,7 +237,16 @@ def main():
     ap.add_argument("--chunk", type=int, default=FRAMES, help="frames per rrm_step_seq call")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="skip the secondary sweeps (profiling runs)")
+    ap.add_argument("--workload", default="cfg2", choices=("cfg2",) + CONV_WORKLOADS,
+                    help="cfg2 (default) is the contract line; the others are secondary convolution workloads")
+    ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense"])
+    ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
     args = ap.parse_args()
+    if args.workload != "cfg2":
+        if args.steps == 310:
+            args.steps, args.warmup = 60, 5
+        run_conv(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

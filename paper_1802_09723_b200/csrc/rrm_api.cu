@@ -50,7 +50,8 @@ int dev_alloc(rrm_net* net, void** p, size_t bytes)
 void set_tensor(Tensor& T, int dtype, int n, int c, int h, int w)
 {
     T.dtype = dtype; T.n = n; T.c = c; T.h = h; T.w = w;
-    if (dtype == T_I8) { T.cs = round_up(c, 4); T.unit_bytes = 1; }
+    // int8 rows are padded to whole 32-byte K chunks of the tensor-core path (tiny channel counts: to 4)
+    if (dtype == T_I8) { T.cs = c <= 4 ? 4 : round_up(c, 32); T.unit_bytes = 1; }
     else if (dtype == T_BIN) { T.cs = ceil_div(c, 32); T.unit_bytes = 4; }
     else { T.cs = c; T.unit_bytes = 4; }
 }
@@ -365,7 +366,7 @@ int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
     RRM_CUDA_TRY(cudaMemcpy(&oc, L.ocount, 4, cudaMemcpyDeviceToHost));
     h->active_macs = (int64_t)m;
     h->active_out_pixels = oc;
-    h->variant = RRM_VARIANT_GATHER;
+    h->variant = L.tc_ready ? RRM_VARIANT_TENSOR : RRM_VARIANT_GATHER;
     return RRM_OK;
 }
 int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out) { return rrm_net_get_stats(layer, 0, host_out); }

@@ -74,6 +74,11 @@ struct Layer {
     int xs_cur = 0;
     void* fc_scratch = nullptr;             // per-stream non-zero lists of the two-kernel form
     unsigned long long* fc_nnz = nullptr;   // [0] nnz elements, [1] active groups of 32 (cleared by the kernel's last CTA)
+    // tensor-core variant (int8 / binary layers whose input rows are whole 32-byte K chunks)
+    bool tc_ready = false;
+    int8_t* tc_Wimg = nullptr;              // [n_tiles][slabs][bn * 128] shared-memory images of the filter tiles
+    int tc_kpp = 0;                         // K bytes per tap (padded channels per pixel)
+    int tc_bn = 0, tc_ntiles = 0, tc_slabs = 0;
     // chunk-of-frames form of the fused FC path
     int32_t* seq_dP = nullptr;              // [seq_cap][n][c_out] per-frame projection deltas
     unsigned* seq_stat = nullptr;           // [seq_cap * n][2] per frame and stream: non-zeros, active groups of 32
@@ -113,6 +118,11 @@ bool fc_seq_supported(const Layer& L);
 int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool dense, bool stateless,
                cudaStream_t st);
 int fc_seq_stats(Layer& L, unsigned long long* nnz, unsigned long long* groups);
+
+// ---- rrm_conv_tc.cu
+bool conv_tc_eligible(const rrm_net* net, const Layer& L);
+int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev);
+int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st);
 
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);

@@ -596,6 +596,7 @@ int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bia
                                                     d.dtype == RRM_F32 ? T_F32 : (d.dtype == RRM_I8 ? T_I8 : T_BIN),
                                                     d.c_in, d.c_out, d.kh, d.kw, L.u_in, L.kup, L.np);
     RRM_CUDA_TRY(cudaGetLastError());
+    if (d.variant != RRM_VARIANT_GATHER && conv_tc_eligible(net, L)) RRM_TRY(conv_tc_create(net, L, W_dev));
     return RRM_OK;
 }
 
@@ -700,7 +701,8 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
     dim3 grid(ceil_div(L.opixels(), TM), L.np / TN);
     const bool vec = (L.u_in % 4) == 0;
-    if (d.dtype == RRM_F32) { if (dense) launch_gemm<T_F32, true>(p, vec, grid, st); else launch_gemm<T_F32, false>(p, vec, grid, st); }
+    if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, dense, stateless, st));
+    else if (d.dtype == RRM_F32) { if (dense) launch_gemm<T_F32, true>(p, vec, grid, st); else launch_gemm<T_F32, false>(p, vec, grid, st); }
     else if (d.dtype == RRM_I8) { if (dense) launch_gemm<T_I8, true>(p, vec, grid, st); else launch_gemm<T_I8, false>(p, vec, grid, st); }
     else { if (dense) launch_gemm<T_BIN, true>(p, vec, grid, st); else launch_gemm<T_BIN, false>(p, vec, grid, st); }
 
