@@ -2,6 +2,7 @@
 #include "rrm_common.cuh"
 #include <new>
 #include <cstring>
+#include <cstdlib>
 
 using namespace rrm;
 
@@ -140,9 +141,35 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         off += 16;
     }
     for (int l = 0; l < n_layers; ++l) RRM_TRY(conv_layer_create(net, net->layers[l], W[l], B ? B[l] : nullptr));
+    {
+        const char* e = getenv("RRM_NO_GRAPH");
+        net->graph_off = e && e[0] == '1';
+    }
     for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
     RRM_TRY(reset_state(net, nullptr));
     RRM_CUDA_TRY(cudaDeviceSynchronize());
+    return RRM_OK;
+}
+
+int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
+
+// Captures the delta step's launch sequence into a graph (on a private stream: a capture cannot start
+// on the legacy default stream) so that later steps cost one graph launch on the host.
+int build_step_graph(rrm_net* net)
+{
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    RRM_TRY(dev_alloc(net, &net->frame_buf, (size_t)bi));
+    RRM_TRY(dev_alloc(net, &net->out_buf, (size_t)bo));
+    RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
+    RRM_CUDA_TRY(cudaStreamBeginCapture(net->cap_stream, cudaStreamCaptureModeThreadLocal));
+    const int s = launch_sequence(net, net->frame_buf, net->out_buf, net->cap_stream, false, false);
+    cudaGraph_t g = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(net->cap_stream, &g);
+    if (s != RRM_OK || e != cudaSuccess || !g) { if (g) cudaGraphDestroy(g); cudaGetLastError(); return s != RRM_OK ? s : RRM_ERR_CUDA; }
+    net->step_graph = g;
+    RRM_CUDA_TRY(cudaGraphInstantiate(&net->step_exec, g, 0));
     return RRM_OK;
 }
 
@@ -151,6 +178,26 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
     if (!net || !frame) return RRM_ERR_INVALID_ARG;
     net->last_stream = st;
     if (net->layers[0].fc_fused) return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
+    if (!dense && !stateless && !net->graph_off) {
+        if (!net->step_exec) {
+            const int s = build_step_graph(net);
+            if (s != RRM_OK) { net->graph_off = true; if (s == RRM_ERR_ALLOC) return s; }
+        }
+        if (net->step_exec) {
+            int64_t bi = 0, bo = 0;
+            tensor_bytes_boundary(net->tensors.front(), &bi);
+            tensor_bytes_boundary(net->tensors.back(), &bo);
+            RRM_CUDA_TRY(cudaMemcpyAsync(net->frame_buf, frame, (size_t)bi, cudaMemcpyDeviceToDevice, st));
+            RRM_CUDA_TRY(cudaGraphLaunch(net->step_exec, st));
+            if (out) RRM_CUDA_TRY(cudaMemcpyAsync(out, net->out_buf, (size_t)bo, cudaMemcpyDeviceToDevice, st));
+            return RRM_OK;
+        }
+    }
+    return launch_sequence(net, frame, out, st, dense, stateless);
+}
+
+int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
+{
     if (!stateless) RRM_CUDA_TRY(cudaMemsetAsync(net->cleared, 0, net->cleared_bytes, st));
     RRM_TRY(launch_import(net, frame, !dense, stateless, st));
     for (int l = 0; l < (int)net->layers.size(); ++l) RRM_TRY(launch_layer(net, l, dense, stateless, st));
@@ -221,6 +268,9 @@ int rrm_net_destroy(rrm_net* net)
 {
     if (!net) return RRM_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
+    if (net->step_exec) cudaGraphExecDestroy(net->step_exec);
+    if (net->step_graph) cudaGraphDestroy(net->step_graph);
+    if (net->cap_stream) cudaStreamDestroy(net->cap_stream);
     for (void* p : net->allocs) cudaFree(p);
     delete net;
     return RRM_OK;

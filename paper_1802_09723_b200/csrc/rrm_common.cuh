@@ -101,6 +101,13 @@ struct rrm_net {
     void* stage_in = nullptr;         // device staging for the *_host entry points
     void* stage_out = nullptr;
     int stage_frames = 0;             // frames the staging buffers hold
+    // the per-frame launch sequence of rrm_net_step, captured once and replayed (fixed frame / output buffers)
+    cudaGraph_t step_graph = nullptr;
+    cudaGraphExec_t step_exec = nullptr;
+    cudaStream_t cap_stream = nullptr;
+    void* frame_buf = nullptr;        // the step's input frame, boundary layout
+    void* out_buf = nullptr;          // the step's last tensor, boundary layout
+    bool graph_off = false;           // RRM_NO_GRAPH=1: launch kernel by kernel (debugging)
     std::vector<void*> allocs;        // everything to free
 };
 

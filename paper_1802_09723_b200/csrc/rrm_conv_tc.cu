@@ -8,13 +8,14 @@
 //   depth   K = taps x input channels, cut into slabs of 128 bytes (4 MMA steps of 32 int8 each).
 // A (activations) is gathered: each row of a slab is 128 contiguous bytes of one input pixel's delta
 // row (zero when the pixel is outside the image or did not change), copied by four producer warps with
-// 128-bit loads into shared memory in the 128-byte-swizzled K-major layout the MMA reads.  Binary
-// layers expand their bit-packed rows on the way: delta = +2 / -2 / 0 per changed bit (dense: +1 / -1).
+// asynchronous 16-byte copies into shared memory in the 128-byte-swizzled K-major layout the MMA reads.
+// Binary layers expand their bit-packed rows on the way: delta = +2 / -2 / 0 per changed bit (dense: +1 / -1).
 // B (filters) is packed once at create time as the exact shared-memory image of every (N tile, slab),
 // so one bulk copy (cp.async.bulk, completion on an mbarrier) stages a slab.  One thread issues the
 // MMAs; tcgen05.commit releases a stage when the tensor core has read it.  The K range can be split
-// over CTAs (grid.z); partial sums are then added onto the stored projection with integer atomics,
-// which keeps the result exact.  (Pixel tile x tap) blocks with no changed input are skipped.
+// over CTAs (grid.z); every accumulator row leaves through shared memory as one bulk store or one bulk
+// integer add-reduction onto the stored projection, which keeps the result exact in any order.
+// (Pixel tile x tap) blocks with no changed input are skipped.
 //
 // Every wait on an mbarrier is bounded; a wait that runs out sets ERRW_TIMEOUT in the net's error
 // word and the CTA leaves through the common exit, which frees its tensor memory.
@@ -24,7 +25,7 @@ namespace rrm {
 
 constexpr int TC_M = 128;
 constexpr int TC_SLAB = 128;                  // bytes of K per stage
-constexpr int TC_STAGES = 4;
+constexpr int TC_STAGES = 3;
 constexpr int TC_THREADS = 192;               // warps 0-3: A producers + epilogue, warp 4: MMA, warp 5: B loader
 constexpr int TC_MAX_BN = 128;
 constexpr unsigned TC_SPIN_LIMIT = 1u << 20;
@@ -123,14 +124,25 @@ struct TcSmemTail {
     unsigned long long full[TC_STAGES], empty[TC_STAGES], done;
     uint32_t tmem_base;
     int fail;
-    unsigned long long tap_mask[2];           // taps with at least one changed input under this tile (up to 128 taps)
-    int q[TC_M], nbase[TC_M], iy0[TC_M], ix0[TC_M];
+    unsigned long long tap_mask[2];           // taps with a usable input under at least one row of this tile (up to 128 taps)
+    unsigned long long rmask[TC_M][2];        // per row: taps whose input pixel is inside the image (and changed, delta mode)
+    int q[TC_M], pix0[TC_M];                  // projection pixel of the row; input pixel under tap (0,0) (may be outside)
 };
 constexpr size_t TC_STAGE_BYTES = (size_t)TC_M * TC_SLAB + (size_t)TC_MAX_BN * TC_SLAB;
 constexpr size_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + sizeof(TcSmemTail);
+constexpr int TC_LAG = TC_STAGES - 1;         // slabs whose asynchronous copies may still be in flight
+constexpr int TC_ROW_WORDS = TC_MAX_BN + 4;   // epilogue row buffers: 16-byte aligned rows, staggered over the banks
+static_assert((size_t)TC_M * TC_ROW_WORDS * 4 <= TC_STAGES * TC_STAGE_BYTES, "epilogue rows reuse the stage buffers");
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <bool BIN, bool DENSE>
-__global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(TcParams p)
+__global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
 {
     extern __shared__ unsigned char tc_smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -151,58 +163,80 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(TcParams p)
         }
         mbar_init(smem_u32(&S->done), 1);
         S->fail = 0;
-        S->tap_mask[0] = S->tap_mask[1] = DENSE ? ~0ull : 0ull;
+        S->tap_mask[0] = S->tap_mask[1] = 0ull;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (tid < TC_M) {
-        const int r = tile * TC_M + tid;
-        int q = -1;
-        if (r < count) q = DENSE ? r : p.olist[r];
-        S->q[tid] = q;
-        if (q >= 0) {
-            const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
-            S->nbase[tid] = ns * p.h * p.w;
-            S->iy0[tid] = oy * p.stride - p.pad;
-            S->ix0[tid] = ox * p.stride - p.pad;
-        } else {
-            S->nbase[tid] = 0; S->iy0[tid] = -(1 << 20); S->ix0[tid] = -(1 << 20);
-        }
     }
     if (warp == 4) {                                        // tensor memory for the accumulator tile
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&S->tmem_base)), "r"((uint32_t)TC_MAX_BN) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    __syncthreads();                                        // tap_mask is zero before the rows add to it
+    if (tid < TC_M) {
+        // row -> projection pixel, and per tap: is its input pixel inside the image (and changed)?
+        const int r = tile * TC_M + tid;
+        int q = -1;
+        if (r < count) q = DENSE ? r : p.olist[r];
+        S->q[tid] = q;
+        unsigned long long m0 = 0, m1 = 0;
+        int pix0 = 0;
+        if (q >= 0) {
+            const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
+            const int y0 = oy * p.stride - p.pad, x0 = ox * p.stride - p.pad;
+            pix0 = ns * p.h * p.w + y0 * p.w + x0;
+            for (int t0 = 0; t0 < p.taps; t0 += 8) {          // 8 taps at a time: all bitmap loads first
+                uint32_t word[8];
+                int sh[8];
+                #pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int t = t0 + u, ky = t / p.kw, kx = t - ky * p.kw;
+                    const int iy = y0 + ky, ix = x0 + kx;
+                    const bool in = t < p.taps && iy >= 0 && iy < p.h && ix >= 0 && ix < p.w;
+                    const int pix = pix0 + ky * p.w + kx;
+                    sh[u] = in ? (pix & 31) : -1;
+                    word[u] = DENSE ? 0xffffffffu : (in ? p.in_act[pix >> 5] : 0u);
+                }
+                #pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (sh[u] >= 0 && ((word[u] >> sh[u]) & 1u)) {
+                        const int t = t0 + u;
+                        if (t < 64) m0 |= 1ull << t; else m1 |= 1ull << (t - 64);
+                    }
+                }
+            }
+        }
+        S->pix0[tid] = pix0;
+        S->rmask[tid][0] = m0; S->rmask[tid][1] = m1;
+        // OR over the warp first (32-bit halves), then one shared-memory atomic per warp and half
+        const unsigned a0 = __reduce_or_sync(0xffffffffu, (unsigned)m0), a1 = __reduce_or_sync(0xffffffffu, (unsigned)(m0 >> 32));
+        const unsigned a2 = __reduce_or_sync(0xffffffffu, (unsigned)m1), a3 = __reduce_or_sync(0xffffffffu, (unsigned)(m1 >> 32));
+        if (lane == 0) {
+            unsigned* tm = reinterpret_cast<unsigned*>(S->tap_mask);
+            if (a0) atomicOr(tm + 0, a0);
+            if (a1) atomicOr(tm + 1, a1);
+            if (a2) atomicOr(tm + 2, a2);
+            if (a3) atomicOr(tm + 3, a3);
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S->tmem_base;
-
-    // taps that see a changed input pixel under any row of this tile
-    if (!DENSE && tid < TC_M && S->q[tid] >= 0) {
-        const int nb = S->nbase[tid], y0 = S->iy0[tid], x0 = S->ix0[tid];
-        unsigned long long m0 = 0, m1 = 0;
-        for (int t = 0; t < p.taps; ++t) {
-            const int iy = y0 + t / p.kw, ix = x0 + t % p.kw;
-            if (iy < 0 || iy >= p.h || ix < 0 || ix >= p.w) continue;
-            const int pix = nb + iy * p.w + ix;
-            if ((p.in_act[pix >> 5] >> (pix & 31)) & 1u) { if (t < 64) m0 |= 1ull << t; else m1 |= 1ull << (t - 64); }
-        }
-        if (m0) atomicOr(&S->tap_mask[0], m0);
-        if (m1) atomicOr(&S->tap_mask[1], m1);
-    }
-    __syncthreads();
     const unsigned long long tm0 = S->tap_mask[0], tm1 = S->tap_mask[1];
 
-    // this CTA's share of the slabs
+    // this CTA's share of the slabs; a slab none of whose taps is usable under any row is skipped
     const int per = (p.slabs + p.ksplit - 1) / p.ksplit;
     const int s_begin = split * per, s_end = min(p.slabs, s_begin + per);
     const int cpt = p.chunks_per_tap;
-    auto slab_live = [&](int ks) -> bool {                  // any tap of the slab's 4 chunks changed?
+    auto slab_live = [&](int ks) -> bool {
         const int t_lo = (ks * 4) / cpt, t_hi = min(p.taps - 1, (ks * 4 + 3) / cpt);
         for (int t = t_lo; t <= t_hi; ++t)
             if (t < 64 ? (tm0 >> t) & 1ull : (tm1 >> (t - 64)) & 1ull) return true;
         return false;
+    };
+    auto next_live = [&](int ks) -> int {                   // first live slab >= ks, or s_end
+        while (ks < s_end && !slab_live(ks)) ++ks;
+        return ks;
     };
     const uint32_t tile_b_bytes = (uint32_t)p.bn * TC_SLAB;
     bool ok = true;
@@ -211,64 +245,113 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(TcParams p)
     if (warp < 4) {
         // ================= A producers: 8 lanes x 16 bytes = one 128-byte row; 4 rows per warp pass
         const int piece = lane & 7, rsub = lane >> 3;
-        const uint32_t* Au = reinterpret_cast<const uint32_t*>(p.A);
-        const uint32_t* Nu = reinterpret_cast<const uint32_t*>(p.Anew);
         int it = 0;
-        for (int ks = s_begin; ks < s_end; ++ks) {
-            if (!slab_live(ks)) continue;
-            const int stage = it % TC_STAGES;
-            if (ok && !mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) ok = false;
-            if (!ok) break;
-            unsigned char* As = base + stage * TC_STAGE_BYTES;
-            const int kc = ks * 4 + (piece >> 1);           // this lane's 32-byte chunk of K
-            const int tap = kc / cpt, cc = kc - tap * cpt;
-            const int ky = tap / p.kw, kx = tap - ky * p.kw;
-            const bool tap_ok = tap < p.taps;
-            #pragma unroll 4
-            for (int i = 0; i < 8; ++i) {
-                const int r = warp * 32 + i * 4 + rsub;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                const int iy = S->iy0[r] + ky, ix = S->ix0[r] + kx;
-                if (tap_ok && iy >= 0 && iy < p.h && ix >= 0 && ix < p.w) {
-                    const int pix = S->nbase[r] + iy * p.w + ix;
-                    if (DENSE || ((p.in_act[pix >> 5] >> (pix & 31)) & 1u)) {
-                        if (!BIN) {
-                            v = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.A) +
-                                                                (size_t)pix * p.row_units + cc * 32 + (piece & 1) * 16);
-                        } else {
-                            // 16 channels of word cc: bits -> bytes
-                            const uint32_t nw = Nu[(size_t)pix * p.row_units + cc] >> ((piece & 1) * 16);
-                            uint32_t valid = 0xffffu;
-                            const int c_base = cc * 32 + (piece & 1) * 16;
-                            if (c_base + 16 > p.c_in) valid = c_base >= p.c_in ? 0u : ((1u << (p.c_in - c_base)) - 1u);
-                            uint32_t pos, neg;                 // channels that contribute +1 / -1 (dense) or +2 / -2 (delta)
-                            if (DENSE) { pos = nw & valid; neg = ~nw & valid; }
-                            else {
-                                const uint32_t ch = (Au[(size_t)pix * p.row_units + cc] >> ((piece & 1) * 16)) & valid;
-                                pos = ch & nw; neg = ch & ~nw;
-                            }
-                            const uint32_t pm = DENSE ? 0x01u : 0x02u, nm = DENSE ? 0xffu : 0xfeu;
-                            v.x = spread4(pos) * pm + spread4(neg) * nm;
-                            v.y = spread4(pos >> 4) * pm + spread4(neg >> 4) * nm;
-                            v.z = spread4(pos >> 8) * pm + spread4(neg >> 8) * nm;
-                            v.w = spread4(pos >> 12) * pm + spread4(neg >> 12) * nm;
-                        }
+        if (!BIN) {
+            // int8 rows are copied as they are: asynchronous 16-byte copies (zero-filled where the input
+            // pixel is unusable); a slab is handed to the tensor core TC_LAG slabs later, when its copies landed
+            const unsigned char* Ab = reinterpret_cast<const unsigned char*>(p.A);
+            for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
+                const int stage = it % TC_STAGES;
+                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
+                const uint32_t As = base_u32 + stage * (uint32_t)TC_STAGE_BYTES;
+                const int kc = ks * 4 + (piece >> 1);       // this lane's 32-byte chunk of K
+                const int tap = kc / cpt, cc = kc - tap * cpt;
+                const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                const int tap_off = ky * p.w + kx;
+                const int byte_off = cc * 32 + (piece & 1) * 16;
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = warp * 32 + i * 4 + rsub;
+                    const bool use = tap < p.taps && ((S->rmask[r][tap >> 6] >> (tap & 63)) & 1ull);
+                    const unsigned char* src = use ? Ab + (size_t)(S->pix0[r] + tap_off) * p.row_units + byte_off : Ab;
+                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
+                    cp_async16(As + off, src, use ? 16u : 0u);
+                }
+                cp_async_commit();
+                if (it >= TC_LAG) {
+                    cp_async_wait<TC_LAG>();                 // the copies of slab it - TC_LAG have landed
+                    fence_async_smem();
+                    mbar_arrive(smem_u32(&S->full[(it - TC_LAG) % TC_STAGES]));
+                }
+                ++it;
+            }
+            cp_async_wait<0>();
+            fence_async_smem();
+            if (ok) for (int j = max(0, it - TC_LAG); j < it; ++j) mbar_arrive(smem_u32(&S->full[j % TC_STAGES]));
+        } else {
+            // binary rows are expanded from bits to bytes on the way: the words of the next slab are
+            // fetched into registers while the current slab is expanded and stored
+            const uint32_t* Cu = reinterpret_cast<const uint32_t*>(p.A);
+            const uint32_t* Nu = reinterpret_cast<const uint32_t*>(p.Anew);
+            uint32_t nw[8], cw[8];
+            unsigned usemask = 0;
+            int half_valid = 0;
+            auto fetch = [&](int ks) {
+                const int kc = ks * 4 + (piece >> 1);
+                const int tap = kc / cpt, cc = kc - tap * cpt;
+                const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                const int tap_off = ky * p.w + kx;
+                const int c_base = cc * 32 + (piece & 1) * 16;
+                half_valid = c_base >= p.c_in ? 0 : (c_base + 16 > p.c_in ? (int)((1u << (p.c_in - c_base)) - 1u) : 0xffff);
+                usemask = 0;
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = warp * 32 + i * 4 + rsub;
+                    const bool use = tap < p.taps && ((S->rmask[r][tap >> 6] >> (tap & 63)) & 1ull);
+                    nw[i] = 0; cw[i] = 0;
+                    if (use) {
+                        const size_t wi = (size_t)(S->pix0[r] + tap_off) * p.row_units + cc;
+                        nw[i] = Nu[wi];
+                        if (!DENSE) cw[i] = Cu[wi];
+                        usemask |= 1u << i;
                     }
                 }
-                const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
-                *reinterpret_cast<uint4*>(As + off) = v;
+            };
+            int ks = next_live(s_begin);
+            if (ks < s_end) fetch(ks);
+            while (ks < s_end) {
+                // keep this slab's words, start fetching the next one
+                uint32_t n_cur[8], c_cur[8];
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) { n_cur[i] = nw[i]; c_cur[i] = cw[i]; }
+                const unsigned use_cur = usemask;
+                const uint32_t valid = (uint32_t)half_valid;
+                const int ks_next = next_live(ks + 1);
+                if (ks_next < s_end) fetch(ks_next);
+                const int stage = it % TC_STAGES;
+                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
+                unsigned char* As = base + stage * TC_STAGE_BYTES;
+                const int shift = (piece & 1) * 16;
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = warp * 32 + i * 4 + rsub;
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (use_cur >> i & 1u) {
+                        const uint32_t nb = n_cur[i] >> shift;
+                        uint32_t pos, neg;                 // channels that contribute +1 / -1 (dense) or +2 / -2 (delta)
+                        if (DENSE) { pos = nb & valid; neg = ~nb & valid; }
+                        else { const uint32_t ch = (c_cur[i] >> shift) & valid; pos = ch & nb; neg = ch & ~nb; }
+                        const uint32_t pm = DENSE ? 0x01u : 0x02u, nm = DENSE ? 0xffu : 0xfeu;
+                        v.x = spread4(pos) * pm + spread4(neg) * nm;
+                        v.y = spread4(pos >> 4) * pm + spread4(neg >> 4) * nm;
+                        v.z = spread4(pos >> 8) * pm + spread4(neg >> 8) * nm;
+                        v.w = spread4(pos >> 12) * pm + spread4(neg >> 12) * nm;
+                    }
+                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(As + off) = v;
+                }
+                fence_async_smem();                          // generic-proxy stores -> visible to the tensor core
+                mbar_arrive(smem_u32(&S->full[stage]));
+                ++it;
+                ks = ks_next;
             }
-            fence_async_smem();                              // generic-proxy stores -> visible to the tensor core
-            mbar_arrive(smem_u32(&S->full[stage]));
-            ++it;
         }
         n_issued = it;
     } else if (warp == 5) {
         // ================= B loader: one bulk copy per slab
         if (lane == 0) {
             int it = 0;
-            for (int ks = s_begin; ks < s_end; ++ks) {
-                if (!slab_live(ks)) continue;
+            for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
                 const int stage = it % TC_STAGES;
                 if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
                 const uint32_t bar = smem_u32(&S->full[stage]);
@@ -283,8 +366,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(TcParams p)
         if (lane == 0) {
             const uint32_t idesc = tc_instr_desc(p.bn);
             int it = 0;
-            for (int ks = s_begin; ks < s_end; ++ks) {
-                if (!slab_live(ks)) continue;
+            for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
                 const int stage = it % TC_STAGES;
                 if (!mbar_wait(smem_u32(&S->full[stage]), (it / TC_STAGES) & 1)) { ok = false; break; }
                 tc_fence_after();
@@ -297,52 +379,85 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(TcParams p)
                 ++it;
             }
             if (ok) tc_commit(smem_u32(&S->done));          // all MMAs of this CTA have completed
-            n_issued = it;
         }
     }
     if (!ok) { S->fail = 1; atomicOr(p.errw, ERRW_TIMEOUT); }
 
-    // ================= epilogue: warps 0-3 read their 32 accumulator rows and update the projection
+    // ================= epilogue: each of the 128 threads of warps 0-3 owns one accumulator row.  It copies
+    // the row from tensor memory into shared memory (the stage buffers are free now) and hands it to the
+    // copy engine as ONE bulk operation on the row's c_out-contiguous slice of the projection: a bulk
+    // store for a dense pass that owns its outputs, a bulk integer add-reduction otherwise (exact in any
+    // order).  Channel counts that are not a multiple of 4 take the element-wise path.
     if (warp < 4) {
         ok = __all_sync(0xffffffffu, ok);                   // the tensor-memory loads below need the whole warp
-        bool have = n_issued > 0;                           // identical for all producer threads
+        const bool have = n_issued > 0;                     // identical for all producer threads
         if (ok && have && !mbar_wait(smem_u32(&S->done), 0)) { ok = false; S->fail = 1; atomicOr(p.errw, ERRW_TIMEOUT); }
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
-        const int r = warp * 32 + lane;
-        const int q = S->q[r];
         const bool atomic = p.ksplit > 1;
         const int n0 = ntile * p.bn;
+        const int r = warp * 32 + lane;
+        const int q = S->q[r];
+        const int ncols = min(p.bn, p.c_out - n0);
+        const bool bulk = (p.c_out & 3) == 0;
+        int* row = reinterpret_cast<int*>(base) + r * TC_ROW_WORDS;
         if (ok && (have || DENSE)) {
-            for (int c0 = 0; c0 < p.bn; c0 += 16) {
-                uint32_t v[16];
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                uint32_t v[32];
                 if (have) {
                     asm volatile(
-                        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                         : "r"(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0));
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 } else {
                     #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0;
+                    for (int j = 0; j < 32; ++j) v[j] = 0;
                 }
                 if (q < 0) continue;
-                int32_t* Pq = p.P + (size_t)q * p.c_out + n0 + c0;
-                #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int co = n0 + c0 + j;
-                    if (co >= p.c_out) break;
-                    const int val = (int)v[j];
-                    if (DENSE) {
-                        // split 0 carries the bias; with a split K the projection was zeroed beforehand
-                        const int b = (split == 0 && p.bias) ? p.bias[co] : 0;
-                        if (atomic) atomicAdd(Pq + j, val + b); else Pq[j] = val + b;
-                    } else if (val != 0) {
-                        if (atomic) atomicAdd(Pq + j, val); else Pq[j] += val;
+                if (bulk) {
+                    #pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        int4 o = make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]);
+                        if (DENSE && split == 0 && p.bias && c0 + j < ncols) {   // split 0 carries the bias
+                            const int4 bb = *reinterpret_cast<const int4*>(p.bias + n0 + c0 + j);
+                            o.x += bb.x; o.y += bb.y; o.z += bb.z; o.w += bb.w;
+                        }
+                        *reinterpret_cast<int4*>(row + c0 + j) = o;
+                    }
+                } else {
+                    #pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int co = n0 + c0 + j;
+                        if (co >= p.c_out) break;
+                        const int val = (int)v[j];
+                        int32_t* dst = p.P + (size_t)q * p.c_out + co;
+                        if (DENSE) {
+                            const int b = (split == 0 && p.bias) ? p.bias[co] : 0;
+                            if (atomic) atomicAdd(dst, val + b); else *dst = val + b;
+                        } else if (val != 0) {
+                            atomicAdd(dst, val);
+                        }
                     }
                 }
+            }
+            if (bulk && q >= 0) {
+                fence_async_smem();                          // this thread's row -> visible to the copy engine
+                int32_t* dst = p.P + (size_t)q * p.c_out + n0;
+                const uint32_t bytes = (uint32_t)ncols * 4u;
+                if (DENSE && !atomic)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 ::"l"(dst), "r"(smem_u32(row)), "r"(bytes) : "memory");
+                else                                         // with a split K of a dense pass the projection was zeroed beforehand
+                    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.s32 [%0], [%1], %2;"
+                                 ::"l"(dst), "r"(smem_u32(row)), "r"(bytes) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the row buffer may be released
             }
         }
     }
@@ -445,9 +560,12 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.chunks_per_tap = L.tc_kpp / 32;
     p.slabs = L.tc_slabs; p.bn = L.tc_bn;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
-    // split K until the grid covers the machine (a split needs at least 2 slabs to be worth a CTA)
-    int ksplit = 1;
-    while (m_tiles * L.tc_ntiles * ksplit < 148 && ksplit * 2 <= L.tc_slabs / 2) ksplit *= 2;
+    // split K so that a CTA's slabs all fit in its pipeline at once (its gather is then one round trip
+    // instead of a chain of them), as long as the grid stays within a few waves of the machine
+    int ksplit = ceil_div(L.tc_slabs, TC_STAGES);
+    const int max_ctas = 148 * 2 * 4;
+    while (ksplit > 1 && (long long)m_tiles * L.tc_ntiles * ksplit > max_ctas) --ksplit;
+    ksplit = ceil_div(L.tc_slabs, ceil_div(L.tc_slabs, ksplit));   // no empty shares
     p.ksplit = ksplit;
     if (dense && ksplit > 1) {
         const long long tot = (long long)L.opixels() * d.c_out;
