@@ -30,6 +30,7 @@ int validate_desc(const rrm_layer_desc& d, int l, int n_layers)
     if (d.dtype != RRM_F32 && d.shift < 0 && d.act == RRM_ACT_RELU) return RRM_ERR_UNSUPPORTED;
     if (d.shift > 30) return RRM_ERR_INVALID_ARG;
     if (d.pool_k < 0 || (d.pool_k > 0 && (d.pool_s < 1 || d.pool_p < 0 || d.pool_p >= d.pool_k))) return RRM_ERR_SHAPE;
+    if (d.pool_k > 3) return RRM_ERR_UNSUPPORTED;
     if (d.src < 0 || d.src > l) return RRM_ERR_INVALID_ARG;
     if (d.res > l) return RRM_ERR_INVALID_ARG;
     if (d.res >= 0 && (d.pool_k > 0 || d.act == RRM_ACT_SIGN)) return RRM_ERR_UNSUPPORTED;
@@ -146,6 +147,19 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         net->graph_off = e && e[0] == '1';
     }
     for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
+    // who reads which tensor: as input (filter footprint) or as shortcut (1x1)
+    for (int l = 0; l < n_layers; ++l) {
+        Layer& L = net->layers[l];
+        const rrm_layer_desc& d = L.d;
+        auto add = [&](int t, Reader r) -> int {
+            Readers& R = net->tensors[t].readers;
+            if (R.n >= MAX_READERS) return RRM_ERR_UNSUPPORTED;
+            R.r[R.n++] = r;
+            return RRM_OK;
+        };
+        RRM_TRY(add(d.src, Reader{L.oact, L.oh, L.ow, d.kh, d.kw, d.stride, d.pad, d.c_out, L.macs}));
+        if (d.res >= 0) RRM_TRY(add(d.res, Reader{L.oact, L.oh, L.ow, 1, 1, 1, 0, d.c_out, nullptr}));
+    }
     RRM_TRY(reset_state(net, nullptr));
     RRM_CUDA_TRY(cudaDeviceSynchronize());
     return RRM_OK;

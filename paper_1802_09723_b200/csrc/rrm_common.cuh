@@ -32,6 +32,15 @@ constexpr int GEMM_TK = 16;   // K units per stage
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
 
+// A layer that reads a tensor, as its input (filter footprint) or as its shortcut (1x1 footprint).
+struct Reader {
+    uint32_t* oact;                   // the reading layer's bitmap of projection pixels to update
+    int oh, ow, kh, kw, stride, pad, c_out;
+    unsigned long long* macs;         // the reading layer's counter of exact multiply-accumulates; nullptr for a shortcut reader
+};
+constexpr int MAX_READERS = 4;
+struct Readers { Reader r[MAX_READERS]; int n; };
+
 struct Tensor {
     int dtype = T_F32;
     int n = 0, c = 0, h = 0, w = 0;
@@ -45,6 +54,7 @@ struct Tensor {
     unsigned long long* npix = nullptr;     // active pixels (cleared every step)
     void* X2 = nullptr;               // value buffer of the stateless dense path
     bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
+    Readers readers{};                // the layers that read it
     int pixels() const { return n * h * w; }
     size_t row_bytes() const { return (size_t)cs * unit_bytes; }
     size_t bytes() const { return (size_t)pixels() * row_bytes(); }
@@ -62,9 +72,9 @@ struct Layer {
     void* bias = nullptr;             // float or int32 [c_out]
     void* P = nullptr;                // projection [n*oh*ow][c_out] float or int32
     void* P2 = nullptr;               // projection buffer of the stateless dense path
-    uint32_t* oact = nullptr;         // bitmap of updated projection pixels (cleared every step)
-    int* olist = nullptr;             // compacted ids of those pixels
-    int* ocount = nullptr;            // their number (cleared every step)
+    uint32_t* oact = nullptr;         // bitmap of projection pixels to update (cleared every step, set by the
+                                      // kernels that produce the layer's input and shortcut tensors)
+    int* ocount = nullptr;            // their number (cleared every step, written by the convolution kernel)
     unsigned long long* macs = nullptr;     // exact active multiply-accumulates (cleared every step)
     int opixels() const { return d.n * oh * ow; }
     // fused FC path (int8 FC reading the external input)

@@ -4,18 +4,20 @@
 // four int8 channels, or 32 sign bits.  Per frame and layer:
 //   import_delta   (layer input = the external frame only)  D = X_t - X_prev, per-pixel activity
 //                  bitmap, X_prev := X_t in place for changed pixels;
-//   active_pixels  dilates the input activity by the filter footprint into the set of projection
-//                  pixels that can change, compacts it with warp ballots into a list, and counts
-//                  the exact multiply-accumulates the non-zero deltas imply (Table 1);
-//   delta_conv     implicit GEMM over the compacted pixels: rows = listed pixels, K = taps x input
+//   delta_conv     implicit GEMM over the projection pixels that can change: every CTA finds its
+//                  rows by a prefix sum over the layer's bitmap of such pixels; K = taps x input
 //                  units gathered from the delta rows of active input pixels (zero otherwise),
 //                  N = output channels; P_prev += result (owner computes: no float atomics);
 //   epilogue       recomputes f only where its window touches an updated projection pixel,
 //                  compares with the stored activation and emits the next layer's delta rows,
 //                  activity bitmap and snapshot update in one pass.
+// A kernel that finds a changed pixel of a tensor (import, epilogue) also marks, in the bitmap of every
+// layer that reads the tensor, the projection pixels whose filter footprint covers it, and counts the
+// exact multiply-accumulates the non-zero deltas imply (Table 1): no separate pass over the activity.
 // The same GEMM kernel with DENSE=true (all pixels, input values instead of deltas, bias added)
 // is the library's dense path and the keyframe.
 #include "rrm_common.cuh"
+#include "rrm_rows.cuh"
 #include <type_traits>
 
 namespace rrm {
@@ -29,8 +31,8 @@ struct ConvParams {
     const void* D;            // delta rows (delta mode) / unused (dense)
     const void* X;            // input values (dense mode; binary delta mode: new sign bits)
     const uint32_t* in_act;   // input activity bitmap (delta mode)
-    const int* olist;         // compacted projection pixels (delta mode)
-    const int* ocount;
+    const uint32_t* oact;     // projection pixels to update (delta mode)
+    int* ocount;              // receives their number
     const void* Wk;           // [kup][np] units
     const void* bias;
     void* P;                  // [opixels][c_out]
@@ -53,18 +55,19 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     __shared__ __align__(16) uint32_t Bs[TK][TN];
     __shared__ int s_q[TM], s_nbase[TM], s_iy0[TM], s_ix0[TM];
     __shared__ int s_rowsum[TM];
+    __shared__ int s_tmp[33];
 
     const int tid = threadIdx.x;
     const int tile = blockIdx.x, n0 = blockIdx.y * TN;
-    int count = p.opixels;
     if (!DENSE) {
-        count = *p.ocount;
+        // this CTA's rows: the tile-th group of TM set bits of the layer's update bitmap
+        const int count = select_rows<TM>(p.oact, (p.opixels + 31) >> 5, tile, s_q, s_tmp);
+        if (tile == 0 && blockIdx.y == 0 && tid == 0) *p.ocount = count;
         if (tile * TM >= count) return;
     }
     if (tid < TM) {
         const int r = tile * TM + tid;
-        int q = -1;
-        if (r < count) q = DENSE ? r : p.olist[r];
+        const int q = DENSE ? (r < p.opixels ? r : -1) : s_q[tid];
         s_q[tid] = q;
         s_rowsum[tid] = 0;
         if (q >= 0) {
@@ -251,7 +254,7 @@ template <typename T, bool DELTA>
 __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ src, T* X, T* D, uint32_t* act,
                                                           int* pnnz, unsigned long long* nnz,
                                                           unsigned long long* npix, int* errw,
-                                                          int c, int cs, int hw)
+                                                          int c, int cs, int hw, int w, Readers readers)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* s_x = reinterpret_cast<T*>(smem_raw);               // [IMP_TP][cs + 1]
@@ -310,12 +313,30 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
             atomicAdd(npix, (unsigned long long)__popc(m));
         }
     }
+    // every changed pixel marks the projection pixels of the reading layers that it touches
+    __shared__ unsigned long long s_macs[MAX_READERS];
+    if (tid < MAX_READERS) s_macs[tid] = 0;
+    __syncthreads();
+    for (int pl = warp; pl < IMP_TP; pl += 8) {
+        const int cnt = (pix0 + pl < hw) ? s_cnt[pl] : 0;
+        if (cnt == 0) continue;
+        const int pix = pix0 + pl;
+        unsigned long long macs[MAX_READERS];
+        scatter_changed(readers, ns, pix / w, pix % w, cnt, lane, macs);
+        if (lane == 0) {
+            #pragma unroll
+            for (int i = 0; i < MAX_READERS; ++i) if (macs[i]) atomicAdd(&s_macs[i], macs[i]);
+        }
+    }
+    __syncthreads();
+    if (tid < readers.n && s_macs[tid]) atomicAdd(readers.r[tid].macs, s_macs[tid]);
 }
 
 // Binary frames arrive already pixel-major and bit-packed: one thread per pixel.
 template <bool DELTA>
 __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X, uint32_t* D, uint32_t* act,
-                                  int* pnnz, unsigned long long* nnz, unsigned long long* npix, int cw, int pixels)
+                                  int* pnnz, unsigned long long* nnz, unsigned long long* npix, int cw, int pixels,
+                                  int h, int w, Readers readers)
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x;
     int cnt = 0;
@@ -343,76 +364,30 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
         atomicAdd(nnz, (unsigned long long)tot);
         atomicAdd(npix, (unsigned long long)__popc(m));
     }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Active projection pixels: q is active iff some input pixel under its filter footprint is active,
-// or the residual tensor changed at q.  Warp ballots give the bitmap word and the compacted list.
-// The second half counts the exact multiply-accumulates implied by the non-zero deltas.
-// ------------------------------------------------------------------------------------------------
-struct ActiveParams {
-    const uint32_t* in_act;
-    const int* in_pnnz;
-    const uint32_t* res_act;      // or nullptr
-    uint32_t* oact;
-    int* olist;
-    int* ocount;
-    unsigned long long* macs;
-    int n, h, w, oh, ow, kh, kw, stride, pad, c_out;
-};
-
-__global__ void __launch_bounds__(256) active_pixels_kernel(ActiveParams p)
-{
-    const int q = blockIdx.x * blockDim.x + threadIdx.x;
-    const int opix = p.n * p.oh * p.ow, ipix = p.n * p.h * p.w;
+    // every changed pixel marks the projection pixels of the reading layers that it touches
     const int lane = threadIdx.x & 31;
-    bool on = false;
-    if (q < opix) {
-        const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
-        const int base = ns * p.h * p.w;
-        for (int ky = 0; ky < p.kh && !on; ++ky) {
-            const int iy = oy * p.stride - p.pad + ky;
-            if (iy < 0 || iy >= p.h) continue;
-            for (int kx = 0; kx < p.kw; ++kx) {
-                const int ix = ox * p.stride - p.pad + kx;
-                if (ix < 0 || ix >= p.w) continue;
-                if (bit_test(p.in_act, base + iy * p.w + ix)) { on = true; break; }
-            }
-        }
-        if (!on && p.res_act) on = bit_test(p.res_act, q);
-    }
-    const unsigned m = __ballot_sync(0xffffffffu, on);
-    if (m) {
-        int slot = 0;
-        if (lane == 0) {
-            slot = atomicAdd(p.ocount, __popc(m));
-            p.oact[q >> 5] = m;                       // q of lane 0 is a multiple of 32
-        }
-        slot = __shfl_sync(0xffffffffu, slot, 0);
-        if (on) p.olist[slot + __popc(m & ((1u << lane) - 1u))] = q;
-    }
-    // exact active MACs: every non-zero delta element at (y,x) meets ty(y)*tx(x) filter taps
-    unsigned long long macs = 0;
-    if (q < ipix && bit_test(p.in_act, q)) {
-        const int x = q % p.w, y = (q / p.w) % p.h;
-        int ty = 0, tx = 0;
-        for (int ky = 0; ky < p.kh; ++ky) {
-            const int t = y + p.pad - ky;
-            ty += (t >= 0 && t % p.stride == 0 && t / p.stride < p.oh);
-        }
-        for (int kx = 0; kx < p.kw; ++kx) {
-            const int t = x + p.pad - kx;
-            tx += (t >= 0 && t % p.stride == 0 && t / p.stride < p.ow);
-        }
-        macs = (unsigned long long)p.in_pnnz[q] * ty * tx * p.c_out;
-    }
+    unsigned long long wsum[MAX_READERS];
     #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) macs += __shfl_down_sync(0xffffffffu, macs, o);
-    if (lane == 0 && macs) atomicAdd(p.macs, macs);
+    for (int i = 0; i < MAX_READERS; ++i) wsum[i] = 0;
+    for (unsigned mm = m; mm; mm &= mm - 1) {
+        const int src_lane = __ffs(mm) - 1;
+        const int pix = __shfl_sync(0xffffffffu, gp, src_lane), c = __shfl_sync(0xffffffffu, cnt, src_lane);
+        const int x = pix % w, y = (pix / w) % h, ns = pix / (w * h);
+        unsigned long long macs[MAX_READERS];
+        scatter_changed(readers, ns, y, x, c, lane, macs);
+        #pragma unroll
+        for (int i = 0; i < MAX_READERS; ++i) wsum[i] += macs[i];
+    }
+    if (lane == 0) {
+        #pragma unroll
+        for (int i = 0; i < MAX_READERS; ++i) if (i < readers.n && wsum[i]) atomicAdd(readers.r[i].macs, wsum[i]);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
-// Epilogue: f on the stored projection, next layer's delta.  One warp per output-tensor pixel.
+// Epilogue: f on the stored projection, next layer's delta.  One warp per output-tensor pixel; a lane
+// owns 4 neighbouring channels at a time, so the 4-channel words of all window positions are fetched
+// with independent 128-bit loads (one memory round trip per 128 channels).
 // ------------------------------------------------------------------------------------------------
 struct EpiParams {
     const void* P;            // [opixels][c_out] float / int
@@ -426,120 +401,173 @@ struct EpiParams {
     unsigned long long* npix;
     int* errw;
     int n, oh, ow, th, tw, c_out, cs, pool_k, pool_s, pool_p, act_fn, shift, theta;
+    Readers readers;          // layers that read the output tensor
 };
 
-// PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.
-template <int PT, int OT, bool DENSE>
+// PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.  KW: pool window edge (1 = no pool).
+template <int PT, int OT, bool DENSE, int KW>
 __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
 {
+    using pt = typename std::conditional<PT == T_F32, float, int>::type;
+    __shared__ unsigned long long s_macs[MAX_READERS];
+    __shared__ unsigned int s_nnz, s_npix;
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x < MAX_READERS) s_macs[threadIdx.x] = 0;
+    if (threadIdx.x == 0) { s_nnz = 0; s_npix = 0; }
+    __syncthreads();
     const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int tpix = p.n * p.th * p.tw;
-    if (r >= tpix) return;
     const int tx = r % p.tw, ty = (r / p.tw) % p.th, ns = r / (p.tw * p.th);
-    const int k = p.pool_k > 0 ? p.pool_k : 1, st = p.pool_k > 0 ? p.pool_s : 1, pp = p.pool_k > 0 ? p.pool_p : 0;
+    const int st = KW > 1 ? p.pool_s : 1, pp = KW > 1 ? p.pool_p : 0;
     const int y0 = ty * st - pp, x0 = tx * st - pp;
     const int qbase = ns * p.oh * p.ow;
-    if (!DENSE) {
-        bool on = false;
-        for (int wy = 0; wy < k && !on; ++wy) {
-            const int y = y0 + wy;
-            if (y < 0 || y >= p.oh) continue;
-            for (int wx = 0; wx < k; ++wx) {
-                const int x = x0 + wx;
-                if (x < 0 || x >= p.ow) continue;
-                if (bit_test(p.oact, qbase + y * p.ow + x)) { on = true; break; }
-            }
+    // window positions inside the projection (bit wy * KW + wx), and whether any of them was updated
+    unsigned inside = 0;
+    bool on = false;
+    if (r < tpix) {
+        bool mine = false, upd = false;
+        if (lane < KW * KW) {
+            const int y = y0 + lane / KW, x = x0 + lane % KW;
+            mine = y >= 0 && y < p.oh && x >= 0 && x < p.ow;
+            if (mine && !DENSE) { const int q = qbase + y * p.ow + x; upd = (p.oact[q >> 5] >> (q & 31)) & 1u; }
         }
-        if (!on) return;
+        inside = __ballot_sync(0xffffffffu, mine);
+        on = DENSE ? true : (__ballot_sync(0xffffffffu, upd) != 0);
     }
-    using pt = typename std::conditional<PT == T_F32, float, int>::type;
-    const pt* P = reinterpret_cast<const pt*>(p.P);
     int cnt = 0;
-    const int c_iter = (OT == T_BIN) ? p.cs * 32 : p.cs;
-    for (int c0 = 0; c0 < c_iter; c0 += 32) {
-        const int c = c0 + lane;
-        const bool live = c < p.c_out;
-        // pooled value of channel c (before sign / after requant+residual+act for int8)
-        pt best = 0;
-        bool have = false;
-        if (live) {
-            for (int wy = 0; wy < k; ++wy) {
-                const int y = y0 + wy;
-                if (y < 0 || y >= p.oh) continue;
-                for (int wx = 0; wx < k; ++wx) {
-                    const int x = x0 + wx;
-                    if (x < 0 || x >= p.ow) continue;
-                    pt v = P[(size_t)(qbase + y * p.ow + x) * p.c_out + c];
+    if (on) {
+        const pt* P = reinterpret_cast<const pt*>(p.P);
+        const bool vec = (p.c_out & 3) == 0;
+        const int c_iter = (OT == T_BIN) ? p.cs * 32 : p.cs;
+        for (int c0 = 0; c0 < c_iter; c0 += 128) {
+            const int c = c0 + lane * 4;
+            // ---- the 4-channel words of every window position
+            pt v[KW * KW][4];
+            #pragma unroll
+            for (int wi = 0; wi < KW * KW; ++wi) {
+                v[wi][0] = v[wi][1] = v[wi][2] = v[wi][3] = 0;
+                if (!(inside >> wi & 1u) || c >= p.c_out) continue;
+                const size_t o = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out + c;
+                if (vec) {
+                    if (PT == T_F32) { const float4 t = *reinterpret_cast<const float4*>(P + o); v[wi][0] = (pt)t.x; v[wi][1] = (pt)t.y; v[wi][2] = (pt)t.z; v[wi][3] = (pt)t.w; }
+                    else { const int4 t = *reinterpret_cast<const int4*>(P + o); v[wi][0] = (pt)t.x; v[wi][1] = (pt)t.y; v[wi][2] = (pt)t.z; v[wi][3] = (pt)t.w; }
+                } else {
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) if (c + j < p.c_out) v[wi][j] = P[o + j];
+                }
+            }
+            // ---- f: [requant] -> [+ shortcut] -> act -> max over the window (sign: max first, threshold last)
+            pt best[4];
+            #pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool live = c + j < p.c_out;
+                pt res = 0;
+                if (live && p.resX) {
+                    if (PT == T_F32) res = (pt)reinterpret_cast<const float*>(p.resX)[(size_t)r * p.cs + c + j];
+                    else if (OT == T_I8) res = (pt)reinterpret_cast<const int8_t*>(p.resX)[(size_t)r * p.cs + c + j];
+                }
+                bool have = false;
+                pt b = 0;
+                #pragma unroll
+                for (int wi = 0; wi < KW * KW; ++wi) {
+                    if (!(inside >> wi & 1u)) continue;
+                    pt x = v[wi][j];
                     if (PT == T_F32) {
-                        if (p.resX) v += reinterpret_cast<const float*>(p.resX)[(size_t)r * p.cs + c];
-                        if (p.act_fn == RRM_ACT_RELU) v = v > 0 ? v : 0;
+                        x += res;
+                        if (p.act_fn == RRM_ACT_RELU) x = x > 0 ? x : 0;
                     } else if (OT == T_I8) {
-                        int iv = (int)v;
+                        int iv = (int)x;
                         if (p.shift > 0) iv = (iv + (1 << (p.shift - 1))) >> p.shift;
                         iv = max(-127, min(127, iv));
-                        if (p.resX) iv += (int)reinterpret_cast<const int8_t*>(p.resX)[(size_t)r * p.cs + c];
+                        iv += (int)res;
                         iv = (p.act_fn == RRM_ACT_RELU) ? max(0, min(127, iv)) : max(-127, min(127, iv));
-                        v = (pt)iv;
+                        x = (pt)iv;
                     }
-                    if (!have || v > best) { best = v; have = true; }
+                    if (!have || x > b) { b = x; have = true; }
                 }
+                best[j] = live ? b : (pt)0;
             }
-        }
-        const size_t o = (size_t)r * p.cs + (OT == T_BIN ? (c0 >> 5) : c);
-        if (OT == T_BIN) {
-            const unsigned word = __ballot_sync(0xffffffffu, live && (int)best >= p.theta);
-            if (lane == 0) {
-                uint32_t* X = reinterpret_cast<uint32_t*>(p.X);
-                if (DENSE) X[o] = word;
-                else {
-                    const uint32_t ch = word ^ X[o];
-                    reinterpret_cast<uint32_t*>(p.D)[o] = ch;
-                    X[o] = word;
-                    cnt += __popc(ch);
+            // ---- compare with the stored activation, emit delta row and snapshot
+            if (OT == T_BIN) {
+                unsigned bits = 0;
+                #pragma unroll
+                for (int j = 0; j < 4; ++j) if (c + j < p.c_out && (int)best[j] >= p.theta) bits |= 1u << j;
+                unsigned word = bits << (4 * (lane & 7));
+                word |= __shfl_xor_sync(0xffffffffu, word, 1);
+                word |= __shfl_xor_sync(0xffffffffu, word, 2);
+                word |= __shfl_xor_sync(0xffffffffu, word, 4);
+                const int wd = (c0 >> 5) + (lane >> 3);
+                if ((lane & 7) == 0 && wd < p.cs) {
+                    uint32_t* X = reinterpret_cast<uint32_t*>(p.X);
+                    const size_t o = (size_t)r * p.cs + wd;
+                    if (DENSE) X[o] = word;
+                    else {
+                        const uint32_t ch = word ^ X[o];
+                        reinterpret_cast<uint32_t*>(p.D)[o] = ch;
+                        X[o] = word;
+                        cnt += __popc(ch);
+                    }
                 }
-            }
-        } else if (c < p.cs) {
-            if (OT == T_F32) {
-                float* X = reinterpret_cast<float*>(p.X);
-                const float v = live ? (float)best : 0.f;
-                if (DENSE) X[o] = v;
-                else {
-                    const float old = X[o];
-                    reinterpret_cast<float*>(p.D)[o] = v - old;
-                    if (v != old) { X[o] = v; ++cnt; }
-                }
-            } else if (OT == T_I32) {
-                int* X = reinterpret_cast<int*>(p.X);
-                const int v = live ? (int)best : 0;
-                if (DENSE) X[o] = v;
-                else {
-                    const int old = X[o];
-                    reinterpret_cast<int*>(p.D)[o] = v - old;
-                    if (v != old) { X[o] = v; ++cnt; }
-                }
-            } else {   // T_I8
-                int8_t* X = reinterpret_cast<int8_t*>(p.X);
-                const int v = live ? (int)best : 0;
-                if (DENSE) X[o] = (int8_t)v;
-                else {
-                    const int old = X[o];
-                    const int d = v - old;
-                    if (p.errw && (d < -128 || d > 127)) atomicOr(p.errw, ERRW_BOUNDS);
-                    reinterpret_cast<int8_t*>(p.D)[o] = (int8_t)d;
-                    if (v != old) { X[o] = (int8_t)v; ++cnt; }
+            } else if (c < p.cs) {
+                const size_t o = (size_t)r * p.cs + c;
+                if (OT == T_I8) {            // cs is a multiple of 4: one 4-channel word per lane
+                    const uint32_t nw = ((uint32_t)(int)best[0] & 0xffu) | ((uint32_t)(int)best[1] & 0xffu) << 8 |
+                                        ((uint32_t)(int)best[2] & 0xffu) << 16 | ((uint32_t)(int)best[3] & 0xffu) << 24;
+                    uint32_t* X = reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.X) + o);
+                    if (DENSE) *X = nw;
+                    else {
+                        const uint32_t ow_ = *X;
+                        uint32_t dw = 0;
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int nv = (int)(int8_t)(nw >> (8 * j)), ov = (int)(int8_t)(ow_ >> (8 * j));
+                            const int d = nv - ov;
+                            if (p.errw && (d < -128 || d > 127)) atomicOr(p.errw, ERRW_BOUNDS);
+                            dw |= ((uint32_t)d & 0xffu) << (8 * j);
+                            cnt += nv != ov;
+                        }
+                        *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.D) + o) = dw;
+                        if (nw != ow_) *X = nw;
+                    }
+                } else {
+                    pt* X = reinterpret_cast<pt*>(p.X);
+                    pt* Dp = reinterpret_cast<pt*>(p.D);
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (c + j >= p.cs) break;
+                        if (DENSE) X[o + j] = best[j];
+                        else {
+                            const pt old = X[o + j];
+                            Dp[o + j] = best[j] - old;
+                            if (best[j] != old) { X[o + j] = best[j]; ++cnt; }
+                        }
+                    }
                 }
             }
         }
     }
     if (DENSE) return;
     #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, o);
-    if (lane == 0 && cnt) {
-        atomicOr(&p.act[r >> 5], 1u << (r & 31));
-        p.pnnz[r] = cnt;
-        atomicAdd(p.nnz, (unsigned long long)cnt);
-        atomicAdd(p.npix, 1ull);
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (cnt) {                                               // uniform inside the warp
+        if (lane == 0) {
+            atomicOr(&p.act[r >> 5], 1u << (r & 31));
+            p.pnnz[r] = cnt;
+            atomicAdd(&s_nnz, (unsigned)cnt);
+            atomicAdd(&s_npix, 1u);
+        }
+        unsigned long long macs[MAX_READERS];
+        scatter_changed(p.readers, ns, ty, tx, cnt, lane, macs);
+        if (lane == 0) {
+            #pragma unroll
+            for (int i = 0; i < MAX_READERS; ++i) if (macs[i]) atomicAdd(&s_macs[i], macs[i]);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < p.readers.n && s_macs[threadIdx.x]) atomicAdd(p.readers.r[threadIdx.x].macs, s_macs[threadIdx.x]);
+    if (threadIdx.x == 0 && s_npix) {
+        atomicAdd(p.nnz, (unsigned long long)s_nnz);
+        atomicAdd(p.npix, (unsigned long long)s_npix);
     }
 }
 
@@ -589,7 +617,6 @@ int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bia
     RRM_TRY(dev_alloc(net, &L.Wk, (size_t)L.kup * L.np * 4));
     RRM_TRY(dev_alloc(net, &L.bias, (size_t)d.c_out * 4));
     RRM_TRY(dev_alloc(net, &L.P, (size_t)L.opixels() * d.c_out * 4));
-    RRM_TRY(dev_alloc(net, (void**)&L.olist, (size_t)L.opixels() * 4));
     if (bias_dev) RRM_CUDA_TRY(cudaMemcpy(L.bias, bias_dev, (size_t)d.c_out * 4, cudaMemcpyDeviceToDevice));
     const int tot = L.kup * L.np;
     pack_weights_kernel<<<ceil_div(tot, 256), 256>>>(W_dev, reinterpret_cast<uint32_t*>(L.Wk),
@@ -628,9 +655,11 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
     if (T.dtype == T_BIN) {
         const int blocks = ceil_div(T.pixels(), 256);
         if (delta) import_bin_kernel<true><<<blocks, 256, 0, st>>>((const uint32_t*)frame, (uint32_t*)X, (uint32_t*)T.D,
-                                                                  T.act, T.pnnz, T.nnz, T.npix, T.cs, T.pixels());
+                                                                  T.act, T.pnnz, T.nnz, T.npix, T.cs, T.pixels(),
+                                                                  T.h, T.w, T.readers);
         else import_bin_kernel<false><<<blocks, 256, 0, st>>>((const uint32_t*)frame, (uint32_t*)X, nullptr, nullptr,
-                                                              nullptr, nullptr, nullptr, T.cs, T.pixels());
+                                                              nullptr, nullptr, nullptr, T.cs, T.pixels(), T.h, T.w,
+                                                              Readers{});
     } else {
         dim3 grid(ceil_div(hw, IMP_TP), T.n);
         const size_t smem = (size_t)IMP_TP * (T.cs + 1) * T.unit_bytes;
@@ -642,16 +671,16 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                 cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             }
             if (delta) kd<<<grid, 256, smem, st>>>((const float*)frame, (float*)X, (float*)T.D, T.act, T.pnnz, T.nnz,
-                                                   T.npix, net->errw, T.c, T.cs, hw);
+                                                   T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers);
             else kn<<<grid, 256, smem, st>>>((const float*)frame, (float*)X, nullptr, nullptr, nullptr, nullptr,
-                                             nullptr, net->errw, T.c, T.cs, hw);
+                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{});
         } else {
             auto kd = import_nchw_kernel<int8_t, true>;
             auto kn = import_nchw_kernel<int8_t, false>;
             if (delta) kd<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, (int8_t*)T.D, T.act, T.pnnz,
-                                                   T.nnz, T.npix, net->errw, T.c, T.cs, hw);
+                                                   T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers);
             else kn<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, nullptr, nullptr, nullptr, nullptr,
-                                             nullptr, net->errw, T.c, T.cs, hw);
+                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{});
         }
     }
     RRM_CUDA_TRY(cudaGetLastError());
@@ -665,14 +694,26 @@ static void launch_gemm(const ConvParams& p, bool vec, dim3 grid, cudaStream_t s
     else conv_gemm_kernel<DT, DENSE, false><<<grid, CONV_THREADS, 0, st>>>(p);
 }
 
-template <int PT, bool DENSE>
-static void launch_epi(const EpiParams& e, int ot, int blocks, cudaStream_t st)
+template <int PT, int OT, bool DENSE>
+static int launch_epi_k(const EpiParams& e, int blocks, cudaStream_t st)
 {
+    switch (e.pool_k > 0 ? e.pool_k : 1) {
+        case 1: epilogue_kernel<PT, OT, DENSE, 1><<<blocks, 256, 0, st>>>(e); break;
+        case 2: epilogue_kernel<PT, OT, DENSE, 2><<<blocks, 256, 0, st>>>(e); break;
+        case 3: epilogue_kernel<PT, OT, DENSE, 3><<<blocks, 256, 0, st>>>(e); break;
+        default: return RRM_ERR_UNSUPPORTED;                 // pool windows are 2x2 or 3x3
+    }
+    return RRM_OK;
+}
+
+template <int PT, bool DENSE>
+static int launch_epi(const EpiParams& e, int ot, int blocks, cudaStream_t st)
+{
+    if (PT == T_F32) return launch_epi_k<PT, T_F32, DENSE>(e, blocks, st);
     switch (ot) {
-        case T_F32: epilogue_kernel<PT, T_F32, DENSE><<<blocks, 256, 0, st>>>(e); break;
-        case T_I8: epilogue_kernel<PT, T_I8, DENSE><<<blocks, 256, 0, st>>>(e); break;
-        case T_BIN: epilogue_kernel<PT, T_BIN, DENSE><<<blocks, 256, 0, st>>>(e); break;
-        default: epilogue_kernel<PT, T_I32, DENSE><<<blocks, 256, 0, st>>>(e); break;
+        case T_I8: return launch_epi_k<PT, T_I8, DENSE>(e, blocks, st);
+        case T_BIN: return launch_epi_k<PT, T_BIN, DENSE>(e, blocks, st);
+        default: return launch_epi_k<PT, T_I32, DENSE>(e, blocks, st);
     }
 }
 
@@ -684,17 +725,8 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     Tensor& out = net->tensors[l + 1];
     Tensor* res = d.res >= 0 ? &net->tensors[d.res] : nullptr;
 
-    if (!dense) {
-        ActiveParams a;
-        a.in_act = in.act; a.in_pnnz = in.pnnz; a.res_act = res ? res->act : nullptr;
-        a.oact = L.oact; a.olist = L.olist; a.ocount = L.ocount; a.macs = L.macs;
-        a.n = d.n; a.h = d.h; a.w = d.w; a.oh = L.oh; a.ow = L.ow; a.kh = d.kh; a.kw = d.kw;
-        a.stride = d.stride; a.pad = d.pad; a.c_out = d.c_out;
-        const int work = L.opixels() > in.pixels() ? L.opixels() : in.pixels();
-        active_pixels_kernel<<<ceil_div(work, 256), 256, 0, st>>>(a);
-    }
     ConvParams p;
-    p.D = in.D; p.X = stateless ? in.X2 : in.X; p.in_act = in.act; p.olist = L.olist; p.ocount = L.ocount;
+    p.D = in.D; p.X = stateless ? in.X2 : in.X; p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
     p.Wk = L.Wk; p.bias = L.bias; p.P = stateless ? L.P2 : L.P;
     p.n = d.n; p.c_in = d.c_in; p.h = d.h; p.w = d.w; p.u_in = L.u_in; p.oh = L.oh; p.ow = L.ow;
     p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.c_out = d.c_out; p.np = L.np;
@@ -713,9 +745,12 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     e.npix = out.npix; e.errw = out.has_consumer ? net->errw : nullptr;
     e.n = d.n; e.oh = L.oh; e.ow = L.ow; e.th = L.th; e.tw = L.tw; e.c_out = d.c_out; e.cs = out.cs;
     e.pool_k = d.pool_k; e.pool_s = d.pool_s; e.pool_p = d.pool_p; e.act_fn = d.act; e.shift = d.shift; e.theta = d.theta;
+    e.readers = dense ? Readers{} : out.readers;
     const int blocks = ceil_div(out.pixels(), 8);
-    if (proj_type(L) == T_F32) { if (dense) launch_epi<T_F32, true>(e, out.dtype, blocks, st); else launch_epi<T_F32, false>(e, out.dtype, blocks, st); }
-    else { if (dense) launch_epi<T_I32, true>(e, out.dtype, blocks, st); else launch_epi<T_I32, false>(e, out.dtype, blocks, st); }
+    int es;
+    if (proj_type(L) == T_F32) es = dense ? launch_epi<T_F32, true>(e, out.dtype, blocks, st) : launch_epi<T_F32, false>(e, out.dtype, blocks, st);
+    else es = dense ? launch_epi<T_I32, true>(e, out.dtype, blocks, st) : launch_epi<T_I32, false>(e, out.dtype, blocks, st);
+    RRM_TRY(es);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }

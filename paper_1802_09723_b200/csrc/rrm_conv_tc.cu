@@ -20,6 +20,7 @@
 // Every wait on an mbarrier is bounded; a wait that runs out sets ERRW_TIMEOUT in the net's error
 // word and the CTA leaves through the common exit, which frees its tensor memory.
 #include "rrm_common.cuh"
+#include "rrm_rows.cuh"
 
 namespace rrm {
 
@@ -34,8 +35,8 @@ struct TcParams {
     const void* A;            // int8: delta rows (delta) or values (dense); binary: changed bits (delta) / unused
     const void* Anew;         // binary: current sign bits
     const uint32_t* in_act;   // input activity bitmap (delta mode)
-    const int* olist;         // compacted projection pixels (delta mode)
-    const int* ocount;
+    const uint32_t* oact;     // projection pixels to update (delta mode)
+    int* ocount;              // receives their number
     const int8_t* Wimg;       // [n_tiles][slabs][bn * 128] swizzled tile images
     const int32_t* bias;
     int32_t* P;               // [opixels][c_out]
@@ -147,14 +148,17 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     extern __shared__ unsigned char tc_smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x, ntile = blockIdx.y, split = blockIdx.z;
-    int count = p.opixels;
-    if (!DENSE) {
-        count = *p.ocount;
-        if (tile * TC_M >= count) return;                   // before anything is allocated
-    }
     unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
     TcSmemTail* S = reinterpret_cast<TcSmemTail*>(base + TC_STAGES * TC_STAGE_BYTES);
     const uint32_t base_u32 = smem_u32(base);
+    __shared__ int s_tmp[33];
+    int count = p.opixels;
+    if (!DENSE) {
+        // this CTA's rows: the tile-th group of 128 set bits of the layer's update bitmap
+        count = select_rows<TC_M>(p.oact, (p.opixels + 31) >> 5, tile, S->q, s_tmp);
+        if (tile == 0 && ntile == 0 && split == 0 && tid == 0) *p.ocount = count;
+        if (tile * TC_M >= count) return;                   // before anything is allocated
+    }
 
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) {
@@ -175,8 +179,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     if (tid < TC_M) {
         // row -> projection pixel, and per tap: is its input pixel inside the image (and changed)?
         const int r = tile * TC_M + tid;
-        int q = -1;
-        if (r < count) q = DENSE ? r : p.olist[r];
+        const int q = DENSE ? (r < count ? r : -1) : S->q[tid];
         S->q[tid] = q;
         unsigned long long m0 = 0, m1 = 0;
         int pix0 = 0;
@@ -550,7 +553,7 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     const void* X = stateless ? in.X2 : in.X;
     p.A = bin ? in.D : (dense ? X : in.D);
     p.Anew = X;
-    p.in_act = in.act; p.olist = L.olist; p.ocount = L.ocount;
+    p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
     p.Wimg = L.tc_Wimg; p.bias = reinterpret_cast<const int32_t*>(L.bias);
     p.P = reinterpret_cast<int32_t*>(stateless ? L.P2 : L.P);
     p.errw = net->errw;
