@@ -10,6 +10,8 @@ namespace rrm {
 // covers the pixel (a layer that adds the tensor as its shortcut is a 1x1 reader), and returns in
 // macs[i] (same value in every lane) the exact multiply-accumulates the pixel implies in reader i:
 // nnz x (output, tap) pairs that meet it x output channels (Table 1 without its border approximation).
+// The projection pixels that meet (y, x) form a rectangle [oy_lo, oy_hi] x [ox_lo, ox_hi]: lane j marks
+// row oy_lo + j as one run of bits (one or two word-wide atomic ORs).
 __device__ __forceinline__ void scatter_changed(const Readers& R, int ns, int y, int x, int nnz, int lane,
                                                 unsigned long long (&macs)[MAX_READERS])
 {
@@ -18,21 +20,23 @@ __device__ __forceinline__ void scatter_changed(const Readers& R, int ns, int y,
         macs[i] = 0;
         if (i >= R.n) continue;
         const Reader& c = R.r[i];
-        const int taps = c.kh * c.kw;
-        int hits = 0;
-        for (int t = lane; t < taps; t += 32) {
-            const int ky = t / c.kw, kx = t - ky * c.kw;
-            const int ty = y + c.pad - ky, tx = x + c.pad - kx;
-            if (ty < 0 || tx < 0 || ty % c.stride || tx % c.stride) continue;
-            const int oy = ty / c.stride, ox = tx / c.stride;
-            if (oy >= c.oh || ox >= c.ow) continue;
-            const int q = (ns * c.oh + oy) * c.ow + ox;
-            atomicOr(&c.oact[q >> 5], 1u << (q & 31));
-            ++hits;
+        // o * stride - pad + k = coordinate, 0 <= k < kernel  <=>  ceil((coord + pad - kernel + 1) / stride) <= o <= floor((coord + pad) / stride)
+        const int ay = y + c.pad, ax = x + c.pad;
+        const int oy_lo = max(0, (ay - c.kh + c.stride) / c.stride), oy_hi = min(c.oh - 1, ay / c.stride);
+        const int ox_lo = max(0, (ax - c.kw + c.stride) / c.stride), ox_hi = min(c.ow - 1, ax / c.stride);
+        const int rows = oy_hi - oy_lo + 1, cols = ox_hi - ox_lo + 1;
+        if (rows <= 0 || cols <= 0) continue;
+        for (int j = lane; j < rows; j += 32) {
+            const int q0 = (ns * c.oh + oy_lo + j) * c.ow + ox_lo;       // first bit of the run, `cols` bits long
+            int done = 0;
+            while (done < cols) {
+                const int bit = (q0 + done) & 31, take = min(32 - bit, cols - done);
+                const uint32_t m = (take == 32 ? 0xffffffffu : ((1u << take) - 1u)) << bit;
+                atomicOr(&c.oact[(q0 + done) >> 5], m);
+                done += take;
+            }
         }
-        #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) hits += __shfl_xor_sync(0xffffffffu, hits, o);
-        if (c.macs) macs[i] = (unsigned long long)nnz * hits * c.c_out;
+        if (c.macs) macs[i] = (unsigned long long)nnz * rows * cols * c.c_out;
     }
 }
 
