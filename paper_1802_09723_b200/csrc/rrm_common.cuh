@@ -27,7 +27,7 @@ enum { ERRW_BOUNDS = 1, ERRW_TIMEOUT = 2, ERRW_CAPACITY = 4 };
 
 // tile shape of the CUDA-core implicit GEMM (units: float, 4 x int8, or 32 sign bits)
 constexpr int GEMM_TN = 64;   // output channels per CTA
-constexpr int GEMM_TK = 16;   // K units per stage
+constexpr int GEMM_TK = 32;   // K units per stage
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline int round_up(int a, int b) { return ceil_div(a, b) * b; }

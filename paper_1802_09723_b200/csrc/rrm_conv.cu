@@ -36,28 +36,72 @@ struct ConvParams {
     const void* Wk;           // [kup][np] units
     const void* bias;
     void* P;                  // [opixels][c_out]
+    int* errw;
     int n, c_in, h, w, u_in, oh, ow, kh, kw, stride, pad, c_out, np, ku, kup, opixels;
 };
 
 __device__ __forceinline__ bool bit_test(const uint32_t* bm, int i) { return (bm[i >> 5] >> (i & 31)) & 1u; }
 
 // ------------------------------------------------------------------------------------------------
-// Implicit GEMM.  DT: T_F32 (float FMA), T_I8 (dp4a on 4-channel words), T_BIN (popcount on 32-channel
-// words: sum(d*w) = 2*(popc(changed) - 2*popc(changed & (new ^ wbits))), dense: valid instead of changed
-// and no factor 2).  VEC: units per pixel divisible by 4 -> 128-bit gathers.
+// Implicit GEMM on the CUDA cores.  DT: T_F32 (float FMA), T_I8 (dp4a on 4-channel words), T_BIN
+// (popcount on 32-channel words: sum(d*w) = 2*(popc(changed) - 2*popc(changed & (new ^ wbits))), dense:
+// valid instead of changed and no factor 2).
+//
+// A CTA owns TM projection pixels x TN output channels and walks K = taps x input units in stages of
+// TK units through a ring of GEMM_STAGES shared-memory buffers:
+//   - the filter slice of a stage ([TK][TN] words, contiguous in the packed filters) is staged with one
+//     bulk copy (cp.async.bulk) that completes on an mbarrier;
+//   - the activation slice is gathered with asynchronous copies (16 bytes = 4 K units of one row at a
+//     time when the units per pixel allow it, 8 lanes covering 128 contiguous bytes of a pixel row; else
+//     4 bytes), zero-filled where the input pixel is outside the image or did not change; which taps
+//     are usable is decided once per row (a 128-bit mask in shared memory), so the gather addresses
+//     depend on no further load;
+//   - stages none of whose taps is usable under any row of the tile are skipped.
+// Copies of later stages are in flight while the current one is multiplied (4x4 outputs per thread).
 // ------------------------------------------------------------------------------------------------
+constexpr int GEMM_STAGES = 3;
+constexpr unsigned GEMM_SPIN_LIMIT = 1u << 20;
+constexpr int GEMM_LDA = TK + 4;                   // words per activation row in shared memory (16-byte aligned, bank-staggered)
+constexpr int GEMM_A_WORDS = TM * GEMM_LDA, GEMM_B_WORDS = TK * TN;
+
+__device__ __forceinline__ uint32_t g_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void g_cp_async4(uint32_t dst, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void g_cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ bool g_mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (unsigned i = 0; i < GEMM_SPIN_LIMIT; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
 template <int DT, bool DENSE, bool VEC>
 __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
 {
     using acc_t = typename std::conditional<DT == T_F32, float, int>::type;
-    __shared__ __align__(16) uint32_t As[TK][TM];
-    __shared__ __align__(16) uint32_t As2[(DT == T_BIN) ? TK : 1][TM];
-    __shared__ __align__(16) uint32_t Bs[TK][TN];
-    __shared__ int s_q[TM], s_nbase[TM], s_iy0[TM], s_ix0[TM];
-    __shared__ int s_rowsum[TM];
+    constexpr int A_BUFS = (DT == T_BIN) ? 2 : 1;
+    extern __shared__ __align__(128) uint32_t g_smem[];    // [stages][B | A | (A2)]
+    constexpr int STAGE_WORDS = GEMM_B_WORDS + A_BUFS * GEMM_A_WORDS;
+    __shared__ __align__(8) unsigned long long s_full[GEMM_STAGES];
+    __shared__ int s_q[TM];
     __shared__ int s_tmp[33];
+    __shared__ unsigned s_tapmask[4];
+    __shared__ unsigned long long s_rmask[TM][2];
+    __shared__ int s_pix0[TM];
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int tile = blockIdx.x, n0 = blockIdx.y * TN;
     if (!DENSE) {
         // this CTA's rows: the tile-th group of TM set bits of the layer's update bitmap
@@ -65,126 +109,182 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         if (tile == 0 && blockIdx.y == 0 && tid == 0) *p.ocount = count;
         if (tile * TM >= count) return;
     }
+    if (tid == 0) {
+        for (int s = 0; s < GEMM_STAGES; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(g_smem_u32(&s_full[s])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 4) s_tapmask[tid] = 0;
+    __syncthreads();
+
+    // ---- per row: the input pixel under tap (0,0) and the usable taps
+    const int taps = p.kh * p.kw;
     if (tid < TM) {
         const int r = tile * TM + tid;
         const int q = DENSE ? (r < p.opixels ? r : -1) : s_q[tid];
         s_q[tid] = q;
-        s_rowsum[tid] = 0;
+        int pix0 = 0;
+        unsigned long long m0 = 0, m1 = 0;
         if (q >= 0) {
             const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
-            s_nbase[tid] = ns * p.h * p.w;
-            s_iy0[tid] = oy * p.stride - p.pad;
-            s_ix0[tid] = ox * p.stride - p.pad;
-        } else {
-            s_nbase[tid] = 0; s_iy0[tid] = -(1 << 20); s_ix0[tid] = -(1 << 20);
+            const int y0 = oy * p.stride - p.pad, x0 = ox * p.stride - p.pad;
+            pix0 = ns * p.h * p.w + y0 * p.w + x0;
+            for (int t0 = 0; t0 < taps; t0 += 8) {          // 8 taps at a time: all bitmap loads first
+                uint32_t word[8];
+                int sh[8];
+                #pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int t = t0 + u, ky = t / p.kw, kx = t - ky * p.kw;
+                    const int iy = y0 + ky, ix = x0 + kx;
+                    const bool in = t < taps && iy >= 0 && iy < p.h && ix >= 0 && ix < p.w;
+                    const int pix = pix0 + ky * p.w + kx;
+                    sh[u] = in ? (pix & 31) : -1;
+                    word[u] = DENSE ? 0xffffffffu : (in ? p.in_act[pix >> 5] : 0u);
+                }
+                #pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (sh[u] >= 0 && ((word[u] >> sh[u]) & 1u)) {
+                        const int t = t0 + u;
+                        if (t < 64) m0 |= 1ull << t; else m1 |= 1ull << (t - 64);
+                    }
+                }
+            }
+        }
+        s_pix0[tid] = pix0;
+        s_rmask[tid][0] = m0; s_rmask[tid][1] = m1;
+        const unsigned a0 = __reduce_or_sync(0xffffffffu, (unsigned)m0), a1 = __reduce_or_sync(0xffffffffu, (unsigned)(m0 >> 32));
+        const unsigned a2 = __reduce_or_sync(0xffffffffu, (unsigned)m1), a3 = __reduce_or_sync(0xffffffffu, (unsigned)(m1 >> 32));
+        if (lane == 0) {
+            if (a0) atomicOr(&s_tapmask[0], a0);
+            if (a1) atomicOr(&s_tapmask[1], a1);
+            if (a2) atomicOr(&s_tapmask[2], a2);
+            if (a3) atomicOr(&s_tapmask[3], a3);
         }
     }
     __syncthreads();
+    const unsigned long long tm0 = (unsigned long long)s_tapmask[0] | (unsigned long long)s_tapmask[1] << 32;
+    const unsigned long long tm1 = (unsigned long long)s_tapmask[2] | (unsigned long long)s_tapmask[3] << 32;
+    const int n_stages = p.kup / TK;
+    auto stage_live = [&](int ks) -> bool {                 // any usable tap among the stage's K units?
+        const int t_lo = (ks * TK) / p.u_in, t_hi = min(taps - 1, (ks * TK + TK - 1) / p.u_in);
+        for (int t = t_lo; t <= t_hi; ++t)
+            if (t < 64 ? (tm0 >> t) & 1ull : (tm1 >> (t - 64)) & 1ull) return true;
+        return false;
+    };
+    auto next_live = [&](int ks) -> int {
+        while (ks < n_stages && !stage_live(ks)) ++ks;
+        return ks;
+    };
 
-    const int a_row = tid >> 2, a_k = (tid & 3) * 4;       // A gather: 4 consecutive units of one row
-    const int b_row = tid >> 4, b_col = (tid & 15) * 4;    // B load: 4 consecutive output channels
-    const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;    // 4x4 outputs per thread
-    const int my_nbase = s_nbase[a_row], my_iy0 = s_iy0[a_row], my_ix0 = s_ix0[a_row];
+    const uint32_t* Du = reinterpret_cast<const uint32_t*>(p.D);
+    const uint32_t* Xu = reinterpret_cast<const uint32_t*>(p.X);
+    const uint32_t* Wu = reinterpret_cast<const uint32_t*>(p.Wk) + (size_t)blockIdx.y * p.kup * TN;   // this N tile's filters
+    const uint32_t smem_base = g_smem_u32(g_smem);
     const uint32_t tail_mask = (p.c_in & 31) ? ((1u << (p.c_in & 31)) - 1u) : 0xffffffffu;
 
+    // issues the copies of stage `ks` into ring slot `slot`
+    auto issue = [&](int ks, int slot) {
+        const uint32_t sB = smem_base + (uint32_t)(slot * STAGE_WORDS) * 4u, sA = sB + GEMM_B_WORDS * 4u;
+        if (tid == 0) {
+            const uint32_t bar = g_smem_u32(&s_full[slot]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot precede the bulk write
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(GEMM_B_WORDS * 4)) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(sB), "l"(Wu + (size_t)ks * GEMM_B_WORDS), "r"((uint32_t)(GEMM_B_WORDS * 4)), "r"(bar) : "memory");
+        }
+        // thread -> (row = tid / 8 [+ 32], piece = tid % 8): 8 lanes cover the 32 K units of one row
+        const int piece = tid & 7;
+        #pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int row = (tid >> 3) + half * 32;
+            const unsigned long long rm0 = s_rmask[row][0], rm1 = s_rmask[row][1];
+            const int pix0 = s_pix0[row];
+            #pragma unroll
+            for (int i = 0; i < (VEC ? 1 : 4); ++i) {
+                const int kk = VEC ? piece * 4 : piece + 8 * i, k = ks * TK + kk;
+                const int tap = k / p.u_in, u = k - tap * p.u_in;
+                const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                const bool use = tap < taps && ((tap < 64 ? rm0 >> tap : rm1 >> (tap - 64)) & 1ull);
+                const size_t off = use ? (size_t)(pix0 + ky * p.w + kx) * p.u_in + u : 0;
+                const int sidx = row * GEMM_LDA + kk;
+                const uint32_t dst = sA + (uint32_t)sidx * 4u;
+                if (DT == T_BIN) {
+                    // first buffer: changed bits (dense: the valid-channel mask, written directly), second: sign bits
+                    if (DENSE) {
+                        uint32_t* d = g_smem + slot * STAGE_WORDS + GEMM_B_WORDS + sidx;
+                        #pragma unroll
+                        for (int j = 0; j < (VEC ? 4 : 1); ++j) d[j] = use ? ((u + j == p.u_in - 1) ? tail_mask : 0xffffffffu) : 0u;
+                    } else if (VEC) g_cp_async16(dst, Du + off, use ? 16u : 0u);
+                    else g_cp_async4(dst, Du + off, use ? 4u : 0u);
+                    if (VEC) g_cp_async16(dst + GEMM_A_WORDS * 4u, Xu + off, use ? 16u : 0u);
+                    else g_cp_async4(dst + GEMM_A_WORDS * 4u, Xu + off, use ? 4u : 0u);
+                } else if (VEC) {
+                    g_cp_async16(dst, (DENSE ? Xu : Du) + off, use ? 16u : 0u);
+                } else {
+                    g_cp_async4(dst, (DENSE ? Xu : Du) + off, use ? 4u : 0u);
+                }
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;    // 4x4 outputs per thread
     acc_t acc[4][4];
     #pragma unroll
     for (int i = 0; i < 4; ++i)
         #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
-    int my_popc = 0;
+    int rowpop[4] = {0, 0, 0, 0};                          // binary: changed (dense: valid) bits of the thread's 4 rows
+    bool ok = true;
 
-    const uint32_t* Du = reinterpret_cast<const uint32_t*>(p.D);
-    const uint32_t* Xu = reinterpret_cast<const uint32_t*>(p.X);
-    const uint32_t* Wu = reinterpret_cast<const uint32_t*>(p.Wk);
-
-    for (int k0 = 0; k0 < p.kup; k0 += TK) {
-        // ---- gather 4 units of A into registers
-        uint32_t a1[4] = {0, 0, 0, 0}, a2[4] = {0, 0, 0, 0};
-        int any = 0;
-        auto locate = [&](int k, int& u) -> long long {     // pixel-row offset (in units) or -1
-            if (k >= p.ku) return -1;
-            const int tap = k / p.u_in;
-            u = k - tap * p.u_in;
-            const int ky = tap / p.kw, kx = tap - ky * p.kw;
-            const int iy = my_iy0 + ky, ix = my_ix0 + kx;
-            if (iy < 0 || iy >= p.h || ix < 0 || ix >= p.w) return -1;
-            const int pix = my_nbase + iy * p.w + ix;
-            if (!DENSE && !bit_test(p.in_act, pix)) return -1;
-            return (long long)pix * p.u_in;
-        };
-        if (VEC) {
-            int u;
-            const long long off = locate(k0 + a_k, u);
-            if (off >= 0) {
-                any = 1;
-                if (DT == T_BIN) {
-                    const uint4 nw = *reinterpret_cast<const uint4*>(Xu + off + u);
-                    uint4 ch;
-                    if (DENSE) {
-                        ch = make_uint4(~0u, ~0u, ~0u, ~0u);
-                        if (u + 3 == p.u_in - 1) ch.w = tail_mask;
-                    } else {
-                        ch = *reinterpret_cast<const uint4*>(Du + off + u);
-                    }
-                    a1[0] = ch.x; a1[1] = ch.y; a1[2] = ch.z; a1[3] = ch.w;
-                    a2[0] = nw.x; a2[1] = nw.y; a2[2] = nw.z; a2[3] = nw.w;
-                } else {
-                    const uint4 v = *reinterpret_cast<const uint4*>((DENSE ? Xu : Du) + off + u);
-                    a1[0] = v.x; a1[1] = v.y; a1[2] = v.z; a1[3] = v.w;
-                }
-            }
-        } else {
+    // prologue: the first GEMM_STAGES - 1 live stages
+    int ks_issue = next_live(0), issued = 0;
+    for (int s = 0; s < GEMM_STAGES - 1; ++s) {
+        if (ks_issue < n_stages) { issue(ks_issue, issued % GEMM_STAGES); ++issued; ks_issue = next_live(ks_issue + 1); }
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    int it = 0;
+    for (int ks = next_live(0); ks < n_stages; ks = next_live(ks + 1), ++it) {
+        const int slot = it % GEMM_STAGES;
+        asm volatile("cp.async.wait_group %0;" ::"n"(GEMM_STAGES - 2) : "memory");   // this thread's copies of stage `it` landed
+        if (ok && !g_mbar_wait(g_smem_u32(&s_full[slot]), (it / GEMM_STAGES) & 1)) ok = false;
+        __syncthreads();                                     // everyone's copies landed; everyone is done with stage it - 1
+        if (ks_issue < n_stages) { issue(ks_issue, issued % GEMM_STAGES); ++issued; ks_issue = next_live(ks_issue + 1); }
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        const uint32_t* Bs = g_smem + slot * STAGE_WORDS;
+        const uint32_t* As = Bs + GEMM_B_WORDS;
+        #pragma unroll 2
+        for (int k4 = 0; k4 < TK; k4 += 4) {
+            uint4 ar[4], an[4];                               // 4 K units of each of the thread's 4 rows
             #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                int u;
-                const long long off = locate(k0 + a_k + i, u);
-                if (off >= 0) {
-                    any = 1;
+                ar[i] = *reinterpret_cast<const uint4*>(&As[(tm + i) * GEMM_LDA + k4]);
+                if (DT == T_BIN) an[i] = *reinterpret_cast<const uint4*>(&As[GEMM_A_WORDS + (tm + i) * GEMM_LDA + k4]);
+            }
+            #pragma unroll
+            for (int kq = 0; kq < 4; ++kq) {
+                const uint4 bw = *reinterpret_cast<const uint4*>(&Bs[(k4 + kq) * TN + tn]);
+                const uint32_t b[4] = {bw.x, bw.y, bw.z, bw.w};
+                #pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t a = kq == 0 ? ar[i].x : kq == 1 ? ar[i].y : kq == 2 ? ar[i].z : ar[i].w;
+                    uint32_t nw = 0;
                     if (DT == T_BIN) {
-                        a2[i] = Xu[off + u];
-                        a1[i] = DENSE ? ((u == p.u_in - 1) ? tail_mask : 0xffffffffu) : Du[off + u];
-                    } else {
-                        a1[i] = (DENSE ? Xu : Du)[off + u];
+                        nw = kq == 0 ? an[i].x : kq == 1 ? an[i].y : kq == 2 ? an[i].z : an[i].w;
+                        rowpop[i] += __popc(a);
+                    }
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (DT == T_F32) acc[i][j] = fmaf(__uint_as_float(a), __uint_as_float(b[j]), acc[i][j]);
+                        else if (DT == T_I8) acc[i][j] = __dp4a((int)a, (int)b[j], (int)acc[i][j]);
+                        else acc[i][j] += __popc(a & (nw ^ b[j]));
                     }
                 }
             }
         }
-        // a stage with no active row contributes nothing: skip it (uniform decision; the barrier
-        // also protects the shared tiles from the previous stage's readers)
-        if (!__syncthreads_or(any)) continue;
-        const uint4 bv = *reinterpret_cast<const uint4*>(Wu + (size_t)(k0 + b_row) * p.np + n0 + b_col);
-        #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            As[a_k + i][a_row] = a1[i];
-            if (DT == T_BIN) { As2[a_k + i][a_row] = a2[i]; my_popc += __popc(a1[i]); }
-        }
-        *reinterpret_cast<uint4*>(&Bs[b_row][b_col]) = bv;
-        __syncthreads();
-        #pragma unroll
-        for (int kk = 0; kk < TK; ++kk) {
-            const uint4 av = *reinterpret_cast<const uint4*>(&As[kk][tm]);
-            const uint4 bw = *reinterpret_cast<const uint4*>(&Bs[kk][tn]);
-            const uint32_t a[4] = {av.x, av.y, av.z, av.w}, b[4] = {bw.x, bw.y, bw.z, bw.w};
-            uint32_t a_nw[4] = {0, 0, 0, 0};
-            if (DT == T_BIN) {
-                const uint4 nv = *reinterpret_cast<const uint4*>(&As2[kk][tm]);
-                a_nw[0] = nv.x; a_nw[1] = nv.y; a_nw[2] = nv.z; a_nw[3] = nv.w;
-            }
-            #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (DT == T_F32) acc[i][j] = fmaf(__uint_as_float(a[i]), __uint_as_float(b[j]), acc[i][j]);
-                    else if (DT == T_I8) acc[i][j] = __dp4a((int)a[i], (int)b[j], (int)acc[i][j]);
-                    else acc[i][j] += __popc(a[i] & (a_nw[i] ^ b[j]));
-                }
-        }
     }
-    if (DT == T_BIN) {
-        if (my_popc) atomicAdd(&s_rowsum[a_row], my_popc);
-    }
-    __syncthreads();
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (!ok) { atomicOr(p.errw, ERRW_TIMEOUT); return; }
 
     // ---- owner-computes update of the stored projection
     #pragma unroll
@@ -203,7 +303,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             } else {
                 int* P = reinterpret_cast<int*>(p.P);
                 int v = (int)acc[i][j];
-                if (DT == T_BIN) v = DENSE ? (s_rowsum[tm + i] - 2 * v) : 2 * (s_rowsum[tm + i] - 2 * v);
+                if (DT == T_BIN) v = DENSE ? (rowpop[i] - 2 * v) : 2 * (rowpop[i] - 2 * v);
                 if (DENSE) P[o] = v + (p.bias ? reinterpret_cast<const int*>(p.bias)[co] : 0);
                 else P[o] += v;
             }
@@ -211,15 +311,39 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     }
 }
 
+static size_t gemm_smem_bytes(int dt)
+{
+    return (size_t)GEMM_STAGES * (GEMM_B_WORDS + (dt == T_BIN ? 2 : 1) * GEMM_A_WORDS) * 4;
+}
+
+template <int DT, bool DENSE>
+static void launch_gemm(const ConvParams& p, dim3 grid, cudaStream_t st)
+{
+    if (p.u_in % 4 == 0) conv_gemm_kernel<DT, DENSE, true><<<grid, CONV_THREADS, gemm_smem_bytes(DT), st>>>(p);
+    else conv_gemm_kernel<DT, DENSE, false><<<grid, CONV_THREADS, gemm_smem_bytes(DT), st>>>(p);
+}
+
+template <int DT>
+static int gemm_allow_smem()
+{
+    const int b = (int)gemm_smem_bytes(DT);
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
+    return RRM_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
-// Filter repack: W[c_out][c_in][kh][kw] -> Wk[k][np] with k = tap * u_in + unit (zero padded).
+// Filter repack: W[c_out][c_in][kh][kw] -> Wk[n tile][k][TN] with k = tap * u_in + unit (zero padded), so
+// that the filter slice of one GEMM stage ([TK][TN] words of one N tile) is one contiguous block.
 // ------------------------------------------------------------------------------------------------
 __global__ void pack_weights_kernel(const void* W, uint32_t* Wk, int dt, int c_in, int c_out, int kh, int kw,
                                     int u_in, int kup, int np)
 {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= kup * np) return;
-    const int k = idx / np, co = idx - k * np;
+    const int nt = idx / (kup * TN), k = (idx / TN) % kup, co = nt * TN + idx % TN;
     uint32_t out = 0;
     const int taps = kh * kw;
     const int tap = k / u_in, u = k - tap * u_in;
@@ -623,6 +747,10 @@ int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bia
                                                     d.dtype == RRM_F32 ? T_F32 : (d.dtype == RRM_I8 ? T_I8 : T_BIN),
                                                     d.c_in, d.c_out, d.kh, d.kw, L.u_in, L.kup, L.np);
     RRM_CUDA_TRY(cudaGetLastError());
+    if (d.kh * d.kw > 128) return RRM_ERR_UNSUPPORTED;       // the kernels keep a row's usable taps in a 128-bit mask
+    RRM_TRY(gemm_allow_smem<T_F32>());
+    RRM_TRY(gemm_allow_smem<T_I8>());
+    RRM_TRY(gemm_allow_smem<T_BIN>());
     if (d.variant != RRM_VARIANT_GATHER && conv_tc_eligible(net, L)) RRM_TRY(conv_tc_create(net, L, W_dev));
     return RRM_OK;
 }
@@ -687,13 +815,6 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
     return RRM_OK;
 }
 
-template <int DT, bool DENSE>
-static void launch_gemm(const ConvParams& p, bool vec, dim3 grid, cudaStream_t st)
-{
-    if (vec) conv_gemm_kernel<DT, DENSE, true><<<grid, CONV_THREADS, 0, st>>>(p);
-    else conv_gemm_kernel<DT, DENSE, false><<<grid, CONV_THREADS, 0, st>>>(p);
-}
-
 template <int PT, int OT, bool DENSE>
 static int launch_epi_k(const EpiParams& e, int blocks, cudaStream_t st)
 {
@@ -732,11 +853,11 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.c_out = d.c_out; p.np = L.np;
     p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
     dim3 grid(ceil_div(L.opixels(), TM), L.np / TN);
-    const bool vec = (L.u_in % 4) == 0;
+    p.errw = net->errw;
     if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, dense, stateless, st));
-    else if (d.dtype == RRM_F32) { if (dense) launch_gemm<T_F32, true>(p, vec, grid, st); else launch_gemm<T_F32, false>(p, vec, grid, st); }
-    else if (d.dtype == RRM_I8) { if (dense) launch_gemm<T_I8, true>(p, vec, grid, st); else launch_gemm<T_I8, false>(p, vec, grid, st); }
-    else { if (dense) launch_gemm<T_BIN, true>(p, vec, grid, st); else launch_gemm<T_BIN, false>(p, vec, grid, st); }
+    else if (d.dtype == RRM_F32) { if (dense) launch_gemm<T_F32, true>(p, grid, st); else launch_gemm<T_F32, false>(p, grid, st); }
+    else if (d.dtype == RRM_I8) { if (dense) launch_gemm<T_I8, true>(p, grid, st); else launch_gemm<T_I8, false>(p, grid, st); }
+    else { if (dense) launch_gemm<T_BIN, true>(p, grid, st); else launch_gemm<T_BIN, false>(p, grid, st); }
 
     EpiParams e;
     e.P = p.P; e.oact = L.oact;

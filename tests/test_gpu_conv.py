@@ -137,6 +137,17 @@ def test_single_layer_shapes(dtype, c_in, c_out, hw, k, s, p):
     _run([sp], video, n=2, stats=True)
 
 
+@pytest.mark.parametrize("dtype", ["i8", "bin"])
+@pytest.mark.parametrize("c_in,c_out,hw,k,s,p", [(16, 70, (13, 13), 3, 1, 1), (8, 12, (17, 15), 5, 2, 2), (64, 16, (10, 10), 3, 1, 1),
+                                                 (3, 6, (35, 35), 11, 4, 0)])
+def test_single_layer_cuda_core_variant(dtype, c_in, c_out, hw, k, s, p):
+    """The CUDA-core (dp4a / popcount) variant on layers that would otherwise take the tensor-core one."""
+    rng = np.random.default_rng(c_in * 1000 + c_out * 10 + k + 1)
+    sp = _spec(dtype, c_in, hw, c_out, k, s, p, rng)
+    video = _video(dtype, c_in, hw, 5, 2, rng)
+    _run([sp], video, n=2, stats=True, variant="gather")
+
+
 @pytest.mark.parametrize("dtype,act,pool,shift", [
     ("f32", "relu", (3, 2, 0), -1), ("f32", "relu", (3, 2, 1), -1), ("f32", "none", (2, 2, 0), -1),
     ("i8", "relu", (3, 2, 0), 9), ("i8", "none", None, 10), ("i8", "sign", (3, 2, 0), -1), ("i8", "none", (3, 2, 1), -1),
