@@ -140,6 +140,7 @@ int fc_seq_stats(Layer& L, unsigned long long* nnz, unsigned long long* groups);
 bool conv_tc_eligible(const rrm_net* net, const Layer& L);
 int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev);
 int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st);
+int zero_projection(void* P, long long words, cudaStream_t st);
 
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);

@@ -38,6 +38,7 @@ struct ConvParams {
     void* P;                  // [opixels][c_out]
     int* errw;
     int n, c_in, h, w, u_in, oh, ow, kh, kw, stride, pad, c_out, np, ku, kup, opixels;
+    int ksplit;               // gridDim.z: CTAs that share one output tile, each with a contiguous range of K stages
 };
 
 __device__ __forceinline__ bool bit_test(const uint32_t* bm, int i) { return (bm[i >> 5] >> (i & 31)) & 1u; }
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     if (!DENSE) {
         // this CTA's rows: the tile-th group of TM set bits of the layer's update bitmap
         const int count = select_rows<TM>(p.oact, (p.opixels + 31) >> 5, tile, s_q, s_tmp);
-        if (tile == 0 && blockIdx.y == 0 && tid == 0) *p.ocount = count;
+        if (tile == 0 && blockIdx.y == 0 && blockIdx.z == 0 && tid == 0) *p.ocount = count;
         if (tile * TM >= count) return;
     }
     if (tid == 0) {
@@ -164,7 +165,9 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     __syncthreads();
     const unsigned long long tm0 = (unsigned long long)s_tapmask[0] | (unsigned long long)s_tapmask[1] << 32;
     const unsigned long long tm1 = (unsigned long long)s_tapmask[2] | (unsigned long long)s_tapmask[3] << 32;
-    const int n_stages = p.kup / TK;
+    // this CTA's share of the K stages
+    const int all_stages = p.kup / TK, per_split = (all_stages + p.ksplit - 1) / p.ksplit;
+    const int s_first = blockIdx.z * per_split, n_stages = min(all_stages, s_first + per_split);
     auto stage_live = [&](int ks) -> bool {                 // any usable tap among the stage's K units?
         const int t_lo = (ks * TK) / p.u_in, t_hi = min(taps - 1, (ks * TK + TK - 1) / p.u_in);
         for (int t = t_lo; t <= t_hi; ++t)
@@ -238,13 +241,13 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     bool ok = true;
 
     // prologue: the first GEMM_STAGES - 1 live stages
-    int ks_issue = next_live(0), issued = 0;
+    int ks_issue = next_live(s_first), issued = 0;
     for (int s = 0; s < GEMM_STAGES - 1; ++s) {
         if (ks_issue < n_stages) { issue(ks_issue, issued % GEMM_STAGES); ++issued; ks_issue = next_live(ks_issue + 1); }
         else asm volatile("cp.async.commit_group;" ::: "memory");
     }
     int it = 0;
-    for (int ks = next_live(0); ks < n_stages; ks = next_live(ks + 1), ++it) {
+    for (int ks = next_live(s_first); ks < n_stages; ks = next_live(ks + 1), ++it) {
         const int slot = it % GEMM_STAGES;
         asm volatile("cp.async.wait_group %0;" ::"n"(GEMM_STAGES - 2) : "memory");   // this thread's copies of stage `it` landed
         if (ok && !g_mbar_wait(g_smem_u32(&s_full[slot]), (it / GEMM_STAGES) & 1)) ok = false;
@@ -286,7 +289,9 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     if (!ok) { atomicOr(p.errw, ERRW_TIMEOUT); return; }
 
-    // ---- owner-computes update of the stored projection
+    // ---- update of the stored projection: the owner of a tile writes it; CTAs that share a tile
+    // (split K) add their partial sums with atomics (dense: onto a zeroed projection, split 0 adds the bias)
+    const bool shared_tile = p.ksplit > 1;
     #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int q = s_q[tm + i];
@@ -298,13 +303,18 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             const size_t o = (size_t)q * p.c_out + co;
             if (DT == T_F32) {
                 float* P = reinterpret_cast<float*>(p.P);
-                if (DENSE) P[o] = acc[i][j] + (p.bias ? reinterpret_cast<const float*>(p.bias)[co] : 0.f);
-                else P[o] += acc[i][j];
+                float v = acc[i][j];
+                if (DENSE && blockIdx.z == 0 && p.bias) v += reinterpret_cast<const float*>(p.bias)[co];
+                if (shared_tile) atomicAdd(P + o, v);
+                else if (DENSE) P[o] = v;
+                else P[o] += v;
             } else {
                 int* P = reinterpret_cast<int*>(p.P);
                 int v = (int)acc[i][j];
                 if (DT == T_BIN) v = DENSE ? (rowpop[i] - 2 * v) : 2 * (rowpop[i] - 2 * v);
-                if (DENSE) P[o] = v + (p.bias ? reinterpret_cast<const int*>(p.bias)[co] : 0);
+                if (DENSE && blockIdx.z == 0 && p.bias) v += reinterpret_cast<const int*>(p.bias)[co];
+                if (shared_tile) atomicAdd(P + o, v);
+                else if (DENSE) P[o] = v;
                 else P[o] += v;
             }
         }
@@ -854,6 +864,15 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
     dim3 grid(ceil_div(L.opixels(), TM), L.np / TN);
     p.errw = net->errw;
+    // split K over CTAs while the tiles alone leave most of the machine idle (each share keeps >= 4 stages)
+    {
+        const int stages = L.kup / TK;
+        int ks = 1;
+        while ((long long)grid.x * grid.y * ks < 2 * 148 && stages / (ks * 2) >= 4) ks *= 2;
+        p.ksplit = ks;
+        grid.z = ks;
+        if (!L.tc_ready && dense && ks > 1) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));
+    }
     if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, dense, stateless, st));
     else if (d.dtype == RRM_F32) { if (dense) launch_gemm<T_F32, true>(p, grid, st); else launch_gemm<T_F32, false>(p, grid, st); }
     else if (d.dtype == RRM_I8) { if (dense) launch_gemm<T_I8, true>(p, grid, st); else launch_gemm<T_I8, false>(p, grid, st); }

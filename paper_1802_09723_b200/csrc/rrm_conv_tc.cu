@@ -503,6 +503,13 @@ __global__ void zero_projection_kernel(int32_t* P, long long total)
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+int zero_projection(void* P, long long words, cudaStream_t st)
+{
+    zero_projection_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(reinterpret_cast<int32_t*>(P), words);
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
 bool conv_tc_eligible(const rrm_net* net, const Layer& L)
 {
     const rrm_layer_desc& d = L.d;
