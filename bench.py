@@ -147,19 +147,26 @@ CONV_WORKLOADS = ("cfg1", "cfg3_f32", "cfg3_i8", "cfg4", "cfg5")
 FFMA_TMACS, DP4A_TMACS, POPC_TBITMACS = 37.2, 74.5, 148.9      # derived ALU peaks: lanes x clock
 
 
-def conv_workload(name, frames=None):
+def conv_workload(name, frames=None, streams=None):
+    """(layer specs, video [F][n]..., n, dtype label).  `streams` overrides the configuration's stream count."""
     import workloads as wl
     if name == "cfg1":
-        return wl.single_conv_f32(), wl.block_redraw_sequence(frames=frames or 8), 1, "f32"
+        n = streams or 1
+        return wl.single_conv_f32(), wl.block_redraw_sequence(frames=frames or 8, n=n), n, "f32"
     if name == "cfg3_f32":
-        return wl.alexnet_convs("f32"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="f32", seed=31), 1, "f32"
+        n = streams or 1
+        return wl.alexnet_convs("f32"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="f32", seed=31, n=n), n, "f32"
     if name == "cfg3_i8":
-        return wl.alexnet_convs("i8"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="i8", seed=32), 1, "i8"
+        n = streams or 1
+        return wl.alexnet_convs("i8"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="i8", seed=32, n=n), n, "i8"
     if name == "cfg4":
-        return (wl.resnet18_convs(), wl.moving_rect_video(frames=frames or 64, hw=224, dtype="i8", seed=41, n=4,
-                                                          bg_redraw=0.02), 4, "i8")
+        n = streams or 4
+        return (wl.resnet18_convs(), wl.moving_rect_video(frames=frames or 64, hw=224, dtype="i8", seed=41, n=n,
+                                                          bg_redraw=0.02), n, "i8")
     if name == "cfg5":
-        return wl.xnor_alexnet_convs(), wl.moving_rect_video(frames=frames or 128, hw=227, dtype="i8", seed=51), 1, "i8+bin"
+        n = streams or 1
+        return (wl.xnor_alexnet_convs(), wl.moving_rect_video(frames=frames or 128, hw=227, dtype="i8", seed=51, n=n),
+                n, "i8+bin")
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -170,7 +177,7 @@ def run_conv(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    specs, video, n, dtype = conv_workload(args.workload, args.frames)
+    specs, video, n, dtype = conv_workload(args.workload, args.frames, args.streams)
     F = video.shape[0]
     net = rrm.net_from_specs(specs, n=n, variant=args.variant)
     frames = [torch.from_numpy(np.ascontiguousarray(video[t])).cuda() for t in range(F)]
@@ -241,6 +248,7 @@ def main():
                     help="cfg2 (default) is the contract line; the others are secondary convolution workloads")
     ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense"])
     ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
+    ap.add_argument("--streams", type=int, default=None, help="independent videos per call (convolution workloads)")
     args = ap.parse_args()
     if args.workload != "cfg2":
         if args.steps == 310:

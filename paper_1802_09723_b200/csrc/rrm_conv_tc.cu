@@ -43,7 +43,8 @@ struct TcParams {
     int* errw;
     int h, w, oh, ow, kw, taps, stride, pad, c_in, c_out, opixels;
     int row_units;            // int8: bytes per input pixel row (multiple of 32); binary: words per pixel
-    int chunks_per_tap;       // 32-byte K chunks per tap
+    int chunks_per_tap;       // 32-byte K chunks per tap (0 for the 4-bytes-per-pixel form)
+    int kpp;                  // K bytes per tap: padded channels per pixel (int8) or 32 x words (binary)
     int slabs;                // total 128-byte slabs of K
     int bn;                   // 64 or 128
     int ksplit;               // gridDim.z
@@ -232,7 +233,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     const int s_begin = split * per, s_end = min(p.slabs, s_begin + per);
     const int cpt = p.chunks_per_tap;
     auto slab_live = [&](int ks) -> bool {
-        const int t_lo = (ks * 4) / cpt, t_hi = min(p.taps - 1, (ks * 4 + 3) / cpt);
+        const int t_lo = (ks * TC_SLAB) / p.kpp, t_hi = min(p.taps - 1, (ks * TC_SLAB + TC_SLAB - 1) / p.kpp);
         for (int t = t_lo; t <= t_hi; ++t)
             if (t < 64 ? (tm0 >> t) & 1ull : (tm1 >> (t - 64)) & 1ull) return true;
         return false;
@@ -257,6 +258,25 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 const int stage = it % TC_STAGES;
                 if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
                 const uint32_t As = base_u32 + stage * (uint32_t)TC_STAGE_BYTES;
+                if (p.kpp == 4) {
+                    // first layers (up to 4 channels = 4 bytes per pixel): a 16-byte piece holds 4 taps, copied one by one
+                    #pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = warp * 32 + i * 4 + rsub;
+                        const unsigned long long rm0 = S->rmask[r][0], rm1 = S->rmask[r][1];
+                        const int pix0 = S->pix0[r];
+                        const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int tap = ks * (TC_SLAB / 4) + piece * 4 + j;
+                            const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                            const bool use = tap < p.taps && ((tap < 64 ? rm0 >> tap : rm1 >> (tap - 64)) & 1ull);
+                            const unsigned char* src = use ? Ab + (size_t)(pix0 + ky * p.w + kx) * 4 : Ab;
+                            asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;"
+                                         ::"r"(As + off + 4u * j), "l"(src), "r"(use ? 4u : 0u) : "memory");
+                        }
+                    }
+                } else {
                 const int kc = ks * 4 + (piece >> 1);       // this lane's 32-byte chunk of K
                 const int tap = kc / cpt, cc = kc - tap * cpt;
                 const int ky = tap / p.kw, kx = tap - ky * p.kw;
@@ -269,6 +289,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                     const unsigned char* src = use ? Ab + (size_t)(S->pix0[r] + tap_off) * p.row_units + byte_off : Ab;
                     const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
                     cp_async16(As + off, src, use ? 16u : 0u);
+                }
                 }
                 cp_async_commit();
                 if (it >= TC_LAG) {
@@ -514,7 +535,7 @@ bool conv_tc_eligible(const rrm_net* net, const Layer& L)
 {
     const rrm_layer_desc& d = L.d;
     const Tensor& in = net->tensors[d.src];
-    if (d.dtype == RRM_I8) { if (in.dtype != T_I8 || in.cs % 32 != 0) return false; }
+    if (d.dtype == RRM_I8) { if (in.dtype != T_I8 || (in.cs % 32 != 0 && in.cs != 4)) return false; }
     else if (d.dtype == RRM_BIN) { if (in.dtype != T_BIN) return false; }
     else return false;
     if (d.kh * d.kw > 128) return false;
@@ -568,6 +589,7 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.c_in = d.c_in; p.c_out = d.c_out; p.opixels = L.opixels();
     p.row_units = bin ? in.cs : in.cs;                       // int8: bytes per pixel; binary: words per pixel
     p.chunks_per_tap = L.tc_kpp / 32;
+    p.kpp = L.tc_kpp;
     p.slabs = L.tc_slabs; p.bn = L.tc_bn;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
     // split K so that a CTA's slabs all fit in its pipeline at once (its gather is then one round trip
