@@ -466,6 +466,69 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
     if (tid < readers.n && s_macs[tid]) atomicAdd(readers.r[tid].macs, s_macs[tid]);
 }
 
+// int8 frames with up to 4 channels (one 4-byte word per pixel): one thread per pixel, plane reads coalesced
+// across the warp, the activity word of 32 consecutive pixels written by one lane from a ballot.
+template <bool DELTA>
+__global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
+                                                            uint32_t* act, int* pnnz, unsigned long long* nnz,
+                                                            unsigned long long* npix, int* errw, int c, int h, int w,
+                                                            int pixels, Readers readers)
+{
+    const int gp = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
+    const int hw = h * w;
+    int cnt = 0;
+    if (gp < pixels) {
+        const int ns = gp / hw, pix = gp - ns * hw;
+        uint32_t nw = 0;
+        for (int ch = 0; ch < c; ++ch) nw |= ((uint32_t)(uint8_t)src[((size_t)ns * c + ch) * hw + pix]) << (8 * ch);
+        if (DELTA) {
+            const uint32_t ow = X[gp];
+            if (nw != ow) {
+                uint32_t dw = 0;
+                #pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int d = (int)(int8_t)(nw >> (8 * j)) - (int)(int8_t)(ow >> (8 * j));
+                    if (d < -128 || d > 127) atomicOr(errw, ERRW_BOUNDS);
+                    dw |= ((uint32_t)d & 0xffu) << (8 * j);
+                    cnt += d != 0;
+                }
+                D[gp] = dw;
+                X[gp] = nw;
+                pnnz[gp] = cnt;
+            }
+        } else {
+            X[gp] = nw;
+        }
+    }
+    if (!DELTA) return;
+    const unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
+    if (m == 0) return;                                      // uniform inside the warp
+    if (lane == 0) act[gp >> 5] = m;                         // gp of lane 0 is a multiple of 32: the word is this warp's alone
+    int tot = cnt;
+    #pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tot += __shfl_down_sync(0xffffffffu, tot, o);
+    if (lane == 0) {
+        atomicAdd(nnz, (unsigned long long)tot);
+        atomicAdd(npix, (unsigned long long)__popc(m));
+    }
+    unsigned long long wsum[MAX_READERS];
+    #pragma unroll
+    for (int i = 0; i < MAX_READERS; ++i) wsum[i] = 0;
+    for (unsigned mm = m; mm; mm &= mm - 1) {
+        const int src_lane = __ffs(mm) - 1;
+        const int pg = __shfl_sync(0xffffffffu, gp, src_lane), cc = __shfl_sync(0xffffffffu, cnt, src_lane);
+        const int x = pg % w, y = (pg / w) % h, ns = pg / hw;
+        unsigned long long macs[MAX_READERS];
+        scatter_changed(readers, ns, y, x, cc, lane, macs);
+        #pragma unroll
+        for (int i = 0; i < MAX_READERS; ++i) wsum[i] += macs[i];
+    }
+    if (lane == 0) {
+        #pragma unroll
+        for (int i = 0; i < MAX_READERS; ++i) if (i < readers.n && wsum[i]) atomicAdd(readers.r[i].macs, wsum[i]);
+    }
+}
+
 // Binary frames arrive already pixel-major and bit-packed: one thread per pixel.
 template <bool DELTA>
 __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X, uint32_t* D, uint32_t* act,
@@ -798,6 +861,14 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
         else import_bin_kernel<false><<<blocks, 256, 0, st>>>((const uint32_t*)frame, (uint32_t*)X, nullptr, nullptr,
                                                               nullptr, nullptr, nullptr, T.cs, T.pixels(), T.h, T.w,
                                                               Readers{});
+    } else if (T.dtype == T_I8 && T.cs == 4) {
+        const int blocks = ceil_div(T.pixels(), 256);
+        if (delta) import_i8_word_kernel<true><<<blocks, 256, 0, st>>>((const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
+                                                                      T.pnnz, T.nnz, T.npix, net->errw, T.c, T.h, T.w,
+                                                                      T.pixels(), T.readers);
+        else import_i8_word_kernel<false><<<blocks, 256, 0, st>>>((const int8_t*)frame, (uint32_t*)X, nullptr, nullptr, nullptr,
+                                                                  nullptr, nullptr, net->errw, T.c, T.h, T.w, T.pixels(),
+                                                                  Readers{});
     } else {
         dim3 grid(ceil_div(hw, IMP_TP), T.n);
         const size_t smem = (size_t)IMP_TP * (T.cs + 1) * T.unit_bytes;

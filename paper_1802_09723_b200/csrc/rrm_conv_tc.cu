@@ -592,11 +592,13 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.kpp = L.tc_kpp;
     p.slabs = L.tc_slabs; p.bn = L.tc_bn;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
-    // split K so that a CTA's slabs all fit in its pipeline at once (its gather is then one round trip
-    // instead of a chain of them), as long as the grid stays within a few waves of the machine
-    int ksplit = ceil_div(L.tc_slabs, TC_STAGES);
-    const int max_ctas = 148 * 2 * 4;
-    while (ksplit > 1 && (long long)m_tiles * L.tc_ntiles * ksplit > max_ctas) --ksplit;
+    // split K towards the point where a CTA's slabs all fit in its pipeline at once
+    // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the
+    // machine needs: once the tiles alone fill it, a tile owned by one CTA saves the adds of shared tiles
+    const int wave = 148 * 2;
+    int ksplit = 1;
+    const int ks_max = ceil_div(L.tc_slabs, TC_STAGES);
+    while (ksplit < ks_max && (long long)m_tiles * L.tc_ntiles * ksplit < wave) ++ksplit;
     ksplit = ceil_div(L.tc_slabs, ceil_div(L.tc_slabs, ksplit));   // no empty shares
     p.ksplit = ksplit;
     if (dense && ksplit > 1) {
