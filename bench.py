@@ -40,6 +40,23 @@ def pingpong(frames):
     return list(range(frames)) + list(range(frames - 2, 0, -1))
 
 
+def whole_job_rate(units_per_rank_step, ms_max_over_ranks, world):
+    """Units per second of the whole job: every rank processes `units_per_rank_step` units per step (weak
+    scaling, replicas), and a step takes as long as the slowest rank."""
+    return world * units_per_rank_step * 1e3 / ms_max_over_ranks
+
+
+def max_over_ranks(ms, world, device=None):
+    """The slowest rank's time (all-reduce MAX over the process group when there is one)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -289,11 +306,7 @@ def main():
         torch.cuda.synchronize()
 
     def reduce_max(ms):
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return ms
+        return max_over_ranks(ms, world, "cuda")
 
     def make(rho, n=1):
         """Layer + the endless back-and-forth walk over the 32-frame sequence, laid out so that chunk k
@@ -380,7 +393,7 @@ def main():
     sampler.start()
     ms = timed_chunks(layer, seq, walk_dev, args.steps, args.warmup, cold=True)
     clocks = sampler.stop()
-    fps = world * T * 1e3 / ms
+    fps = whole_job_rate(T, ms, world)
     bytes_launch = frame_bytes(nnz_mean) * T
     achieved = bytes_launch / (ms * 1e-3) / 1e9
     achieved_unique = chunk_cold_bytes(uniq_mean, T) / (ms * 1e-3) / 1e9

@@ -939,7 +939,9 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     {
         const int stages = L.kup / TK;
         int ks = 1;
-        while ((long long)grid.x * grid.y * ks < 2 * 148 && stages / (ks * 2) >= 4) ks *= 2;
+        // (a delta pass is sized as if half of the tiles had rows: the others leave right after the row scan)
+        const long long tiles = dense ? (long long)grid.x * grid.y : (long long)(grid.x + 1) / 2 * grid.y;
+        while (tiles * ks < 2 * 148 && stages / (ks * 2) >= 2) ks *= 2;
         p.ksplit = ks;
         grid.z = ks;
         if (!L.tc_ready && dense && ks > 1) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));

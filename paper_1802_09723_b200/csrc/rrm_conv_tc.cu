@@ -598,7 +598,9 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     const int wave = 148 * 2;
     int ksplit = 1;
     const int ks_max = ceil_div(L.tc_slabs, TC_STAGES);
-    while (ksplit < ks_max && (long long)m_tiles * L.tc_ntiles * ksplit < wave) ++ksplit;
+    // (a delta pass is sized as if half of the tiles had rows: the others leave right after the row scan)
+    const long long tiles = dense ? (long long)m_tiles * L.tc_ntiles : (long long)(m_tiles + 1) / 2 * L.tc_ntiles;
+    while (ksplit < ks_max && tiles * ksplit < wave) ++ksplit;
     ksplit = ceil_div(L.tc_slabs, ceil_div(L.tc_slabs, ksplit));   // no empty shares
     p.ksplit = ksplit;
     if (dense && ksplit > 1) {
