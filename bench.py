@@ -423,12 +423,14 @@ def main():
             L2, sq, wk, wd, nz, un = make(rho)
             fr = [torch.from_numpy(sq[t]).cuda() for t in range(FRAMES)]
             c_ms = timed_chunks(L2, sq, wd, 124, 10, cold=True)
+            variant = {1: "column gather", 3: "dense on tensor cores (previous chunk's measured density >= 8 %)"}.get(
+                L2.stats(0)["variant"], "?")
             w_ms = timed_chunks(L2, sq, wd, 124, 10, cold=False)
             d_ms = timed_chunks(L2, sq, wd, 31, 3, cold=True, dense=True)
             s_ms = timed_single(L2, sq, fr, 310, 31, cold=True)
             sd_ms = timed_single(L2, sq, fr, 124, 10, cold=True, dense=True)
             by_rho[f"{rho:g}"] = {
-                "nnz_mean_per_frame": nz, "distinct_columns_per_chunk": un,
+                "nnz_mean_per_frame": nz, "distinct_columns_per_chunk": un, "chunk_evaluation": variant,
                 "chunk_cold_us": c_ms * 1e3, "chunk_warm_us": w_ms * 1e3, "dense_chunk_cold_us": d_ms * 1e3,
                 "fps_cold": T * 1e3 / c_ms, "gmacs_dense_equiv_cold": T * DENSE_MACS / c_ms / 1e6,
                 "speedup_vs_own_dense_chunk": d_ms / c_ms,

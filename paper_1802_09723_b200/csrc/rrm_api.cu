@@ -282,6 +282,10 @@ int rrm_net_destroy(rrm_net* net)
 {
     if (!net) return RRM_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
+    for (auto& L : net->layers) {
+        if (L.seq_ev) cudaEventDestroy(L.seq_ev);
+        if (L.seq_stat_host) cudaFreeHost(L.seq_stat_host);
+    }
     if (net->step_exec) cudaGraphExecDestroy(net->step_exec);
     if (net->step_graph) cudaGraphDestroy(net->step_graph);
     if (net->cap_stream) cudaStreamDestroy(net->cap_stream);
@@ -415,7 +419,7 @@ int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
         h->active_in_pixels = (int64_t)tot[1];
         h->active_out_pixels = tot[0] ? (int64_t)frames * d.n : 0;
         h->active_macs = (int64_t)tot[0] * d.c_out;
-        h->variant = RRM_VARIANT_GATHER;
+        h->variant = L.seq_last_T > 0 ? L.seq_last_variant : RRM_VARIANT_GATHER;
         return RRM_OK;
     }
     const Tensor& in = net->tensors[d.src];

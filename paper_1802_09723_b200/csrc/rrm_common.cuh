@@ -96,6 +96,15 @@ struct Layer {
     int seq_cap = 0;                        // frames the scratch arrays hold
     int seq_lanes = 0;                      // 0: pick the slice width per call; 8 / 16 / 32: forced (tuning)
     int seq_last_T = 0;                     // frames of the most recent chunk (0: last call was a single-frame step)
+    // measured density of the previous chunk, read back without stalling the stream: chooses between the
+    // column gather and the dense tensor-core evaluation of the next chunk
+    unsigned* seq_stat_host = nullptr;      // pinned copy of seq_stat
+    int seq_stat_host_cap = 0;              // frames it holds
+    cudaEvent_t seq_ev = nullptr;           // the copy into seq_stat_host has landed
+    bool seq_ev_pending = false;
+    int seq_pending_rows = 0;               // frame x stream rows of the pending copy
+    double seq_density = -1.0;              // non-zero fraction of the last chunk whose counters were read; < 0: unknown
+    int seq_last_variant = RRM_VARIANT_GATHER;
 };
 
 }  // namespace rrm
@@ -135,6 +144,7 @@ bool fc_seq_supported(const Layer& L);
 int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool dense, bool stateless,
                cudaStream_t st);
 int fc_seq_stats(Layer& L, unsigned long long* nnz, unsigned long long* groups);
+int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool stateless, cudaStream_t st);
 
 // ---- rrm_conv_tc.cu
 bool conv_tc_eligible(const rrm_net* net, const Layer& L);

@@ -304,9 +304,64 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
     if (tid == 0) p.counters[s * slices + slice] = 0;
 }
 
+// Non-zero delta entries and active groups of 32 inputs of every (frame, stream) of a chunk: the
+// delta + scan step alone, for chunks that are then evaluated densely.
+__global__ void __launch_bounds__(SQ_THREADS) fc_count_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ xprev,
+                                                            unsigned* stat, int n, int C)
+{
+    __shared__ int s_nnz, s_grp;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int t = blockIdx.x / n, s = blockIdx.x - t * n;
+    if (tid == 0) { s_nnz = 0; s_grp = 0; }
+    __syncthreads();
+    const uint4* xt4 = reinterpret_cast<const uint4*>(x + ((size_t)t * n + s) * C);
+    const uint4* xp4 = reinterpret_cast<const uint4*>(t > 0 ? x + ((size_t)(t - 1) * n + s) * C : xprev + (size_t)s * C);
+    int nnz = 0, grp = 0;
+    for (int base = 0; base < (C >> 4); base += SQ_THREADS) {     // same trip count for every thread: the shuffles below need whole warps
+        const int chunk = base + tid;
+        unsigned m = 0;
+        if (chunk < (C >> 4)) {
+            const uint4 a = __ldg(xt4 + chunk), b = __ldg(xp4 + chunk);
+            m = nonzero_bytes(a.x ^ b.x) | nonzero_bytes(a.y ^ b.y) << 4 | nonzero_bytes(a.z ^ b.z) << 8 | nonzero_bytes(a.w ^ b.w) << 12;
+        }
+        nnz += __popc(m);
+        const unsigned other = __shfl_xor_sync(0xffffffffu, m, 1);
+        grp += ((lane & 1) == 0 && (m | other)) ? 1 : 0;
+    }
+    #pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { nnz += __shfl_down_sync(0xffffffffu, nnz, o); grp += __shfl_down_sync(0xffffffffu, grp, o); }
+    if (lane == 0) { atomicAdd(&s_nnz, nnz); atomicAdd(&s_grp, grp); }
+    __syncthreads();
+    if (tid == 0) { stat[blockIdx.x * 2] = (unsigned)s_nnz; stat[blockIdx.x * 2 + 1] = (unsigned)s_grp; }
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+// From this measured non-zero fraction of the previous chunk on, the next chunk is evaluated densely on the
+// tensor cores (W read once for all frames) instead of by column gather (measured break-even on fc6: ~7 %).
+constexpr double SQ_DENSE_SWITCH = 0.08;
+
+// Copies the chunk's counters to pinned host memory behind the work already on the stream.
+static int seq_read_back(Layer& L, int rows, cudaStream_t st)
+{
+    if (L.seq_ev_pending) return RRM_OK;                     // an older copy is still in flight: keep it
+    if (rows > L.seq_stat_host_cap) {
+        if (L.seq_stat_host) cudaFreeHost(L.seq_stat_host);
+        L.seq_stat_host = nullptr; L.seq_stat_host_cap = 0;
+        if (cudaMallocHost(reinterpret_cast<void**>(&L.seq_stat_host), (size_t)rows * 2 * 4) != cudaSuccess) { cudaGetLastError(); return RRM_OK; }
+        L.seq_stat_host_cap = rows;
+    }
+    if (!L.seq_ev && cudaEventCreateWithFlags(&L.seq_ev, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return RRM_OK; }
+    RRM_CUDA_TRY(cudaMemcpyAsync(L.seq_stat_host, L.seq_stat, (size_t)rows * 2 * 4, cudaMemcpyDeviceToHost, st));
+    RRM_CUDA_TRY(cudaEventRecord(L.seq_ev, st));
+    L.seq_ev_pending = true;
+    L.seq_pending_rows = rows;
+    return RRM_OK;
+}
+
+int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool stateless, cudaStream_t st);
+
 static size_t seq_dyn_smem(int c_in, int lanes) { return (size_t)SQ_WARPS * 16 * lanes * 4 + (size_t)c_in * 4; }
 
 static int seq_ensure(rrm_net* net, Layer& L, int T)
@@ -354,6 +409,7 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
     const int C = L.d.c_in, K = L.d.c_out, n = L.d.n;
     if (T < 1) return RRM_ERR_INVALID_ARG;
     if ((long long)T * n > 65535) return RRM_ERR_CAPACITY;
+    if (dense && stateless && L.tc_ready) return fc_dense_tc_run(net, L, X_dev, Y_dev, T, true, st);
     RRM_TRY(seq_ensure(net, L, T));
     FcSeqParams p;
     p.x = reinterpret_cast<const int8_t*>(X_dev);
@@ -369,13 +425,32 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
         if (stateless) { p.xnext = nullptr; p.P = nullptr; }
         else { p.xnext = L.xs[L.xs_cur ^ 1]; L.xs_cur ^= 1; p.P = reinterpret_cast<int32_t*>(L.P); }
     } else {
+        // ---- which evaluation: the previous chunk's measured density decides (temporal coherence is the
+        // method's premise).  Its counters were copied to pinned memory behind the chunk; they are used
+        // once that copy has landed, and never waited for.
+        if (L.seq_ev_pending && cudaEventQuery(L.seq_ev) == cudaSuccess) {
+            unsigned long long nz = 0;
+            for (int i = 0; i < L.seq_pending_rows; ++i) nz += L.seq_stat_host[2 * i];
+            L.seq_density = (double)nz / ((double)L.seq_pending_rows * C);
+            L.seq_ev_pending = false;
+        }
+        cudaGetLastError();                                  // cudaErrorNotReady from the query is not an error
+        const bool use_dense = L.tc_ready && L.d.variant == RRM_VARIANT_AUTO && (long long)T * n >= 8 &&
+                               L.seq_density >= SQ_DENSE_SWITCH;
+        L.seq_last_T = T;
+        L.seq_last_variant = use_dense ? RRM_VARIANT_DENSE : RRM_VARIANT_GATHER;
+        if (use_dense) {
+            // the results are the same integers: P_t = b + W X_t for every frame, state := last frame
+            fc_count_kernel<<<T * n, SQ_THREADS, 0, st>>>(reinterpret_cast<const int8_t*>(X_dev), L.xs[L.xs_cur], L.seq_stat, n, C);
+            RRM_TRY(fc_dense_tc_run(net, L, X_dev, Y_dev, T, false, st));
+            return seq_read_back(L, T * n, st);
+        }
         p.xprev = L.xs[L.xs_cur];
         p.xnext = L.xs[L.xs_cur ^ 1];
         L.xs_cur ^= 1;
         p.bias = nullptr;
         p.P = reinterpret_cast<int32_t*>(L.P);
         p.stat = L.seq_stat;
-        L.seq_last_T = T;
     }
     // slice width: the widest (fewest redundant scans, one wave of CTAs with a short chain of dependent
     // round trips each), narrowed while the grid would leave a good part of the machine idle
@@ -406,6 +481,50 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
         else fc_seq_kernel<8, false><<<grid, SQ_THREADS, dyn, st>>>(p);
     }
     RRM_CUDA_TRY(cudaGetLastError());
+    if (!dense) RRM_TRY(seq_read_back(L, T * n, st));
+    return RRM_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Dense evaluation of M = frames x streams input rows on the tensor cores: P = X W^T + b is the 1x1
+// "convolution" of an M-pixel image with c_in channels, i.e. exactly what conv_tc_kernel computes from
+// the [c_out][c_in] filters; W is read from HBM once for all rows.
+// ------------------------------------------------------------------------------------------------
+// Pstate (may be nullptr) receives the rows from `state_from` on: the projection of the last frame.
+__global__ void fc_dense_finish_kernel(const int32_t* __restrict__ Pd, void* Y, int32_t* Pstate, long long state_from,
+                                       long long total, int shift, int act)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int v = Pd[i];
+    if (Pstate && i >= state_from) Pstate[i - state_from] = v;
+    if (Y) {
+        if (shift < 0) reinterpret_cast<int32_t*>(Y)[i] = v;
+        else reinterpret_cast<int8_t*>(Y)[i] = (int8_t)seq_apply_f(v, shift, act);
+    }
+}
+
+// stateless: Y only.  Otherwise the stored projection and the snapshot become those of the last frame.
+int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool stateless, cudaStream_t st)
+{
+    const int C = L.d.c_in, K = L.d.c_out, n = L.d.n;
+    RRM_TRY(seq_ensure(net, L, T));
+    Layer Lt = L;                                            // the M-row problem as a 1x1 convolution
+    Lt.d.n = T * n; Lt.d.h = Lt.d.w = 1; Lt.oh = Lt.ow = 1;
+    Lt.P = L.seq_dP;
+    Tensor in;
+    in.dtype = T_I8; in.n = T * n; in.c = C; in.h = in.w = 1; in.cs = C; in.unit_bytes = 1;
+    in.X = const_cast<void*>(X_dev);
+    RRM_TRY(launch_conv_tc(net, Lt, in, true, false, st));
+    const long long total = (long long)T * n * K;
+    fc_dense_finish_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(L.seq_dP, Y_dev, stateless ? nullptr : reinterpret_cast<int32_t*>(L.P),
+                                                                           (long long)(T - 1) * n * K, total, L.d.shift, L.d.act);
+    RRM_CUDA_TRY(cudaGetLastError());
+    if (!stateless) {
+        RRM_CUDA_TRY(cudaMemcpyAsync(L.xs[L.xs_cur ^ 1], reinterpret_cast<const int8_t*>(X_dev) + (size_t)(T - 1) * n * C, (size_t)n * C,
+                                     cudaMemcpyDeviceToDevice, st));
+        L.xs_cur ^= 1;
+    }
     return RRM_OK;
 }
 

@@ -217,3 +217,34 @@ def test_fc6_chunk_longer_than_one_launch_holds():
     spec = wl.fc6_i8()[0]
     seq = wl.fc_run_sequence(frames=41, rho=0.01, seed=29)
     _run_chunks(spec, seq, 1, [40])
+
+
+def test_fc6_dense_chunks_take_over_at_high_measured_density():
+    """At 20 % density the second chunk on is evaluated densely on the tensor cores (the previous chunk's
+    measured density decides); outputs, state and counters stay those of the delta recurrence."""
+    rrm = _rrm()
+    spec = wl.fc6_i8()[0]
+    seq = wl.fc_run_sequence(frames=33, rho=0.20, seed=30)
+    layer = rrm.layer_from_spec(spec)
+    rec = orc.Recurrence([spec])
+    frames = dev(seq)
+    variants = []
+    t0 = 0
+    for T in (8, 8, 8, 8):
+        Y = layer.new_output(frames=T)
+        layer.step_seq(frames[t0:t0 + T], Y, T)
+        nnz = 0
+        for i in range(T):
+            want = orc.dense_forward([spec], seq[t0 + i])[0][1]
+            np.testing.assert_array_equal(Y[i].cpu().numpy().astype(np.int64), want.astype(np.int64))
+            rec.step(seq[t0 + i])
+            nnz += rec.nnz[0]
+        st = layer.stats(0)                       # synchronises: the counters of this chunk are read back by the next call
+        assert st["nnz_elems"] == nnz and st["active_macs"] == nnz * 4096
+        variants.append(st["variant"])
+        t0 += T
+    assert variants[0] == 1 and variants[-1] == 3, variants      # gather first, dense once the density is known
+    Y1 = layer.new_output()
+    layer.step(frames[32], Y1)                    # the state after dense chunks is the recurrence's state
+    np.testing.assert_array_equal(Y1.cpu().numpy(), orc.dense_forward([spec], seq[32])[0][1])
+    layer.close()
