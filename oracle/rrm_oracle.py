@@ -174,10 +174,19 @@ def dense_forward(layers, frame):
 
 # ------------------------------------------------------------- Algorithm 1, literal
 class Recurrence:
-    """Algorithm 1.  State per linear layer: I_prev (zeros at start) and P_prev (= bias)."""
+    """Algorithm 1.  State per linear layer: I_prev (zeros at start) and P_prev (= bias).
 
-    def __init__(self, layers, n=1):
+    eps > 0 (fp32 layers) is the sparsity enhancement of Sec. 3.4: delta entries with |d| < eps are
+    truncated to zero before the sparse product.  Reading: the snapshot still becomes I_t, so the
+    truncated part u is lost and the error accumulates; the decision |d| < eps is taken on the delta
+    computed in fp32 (the kernel's precision).  trunc_l2[l] is l2(u) of the last step for layer l
+    (over all streams of the batch) and e_t the running sum of Eq. 7 since the last reset."""
+
+    def __init__(self, layers, n=1, eps=0.0):
         self.layers = layers
+        self.eps = float(eps)
+        self.trunc_l2 = [0.0] * len(layers)
+        self.e_t = 0.0
         self.I_prev, self.P_prev = [], []
         for s in layers:
             _, dt = _kind(s)
@@ -199,15 +208,40 @@ class Recurrence:
         for l, s in enumerate(layers):
             I = tensors[s.src]
             D = I - self.I_prev[l]                              # Alg. 1: delta of the layer input
+            self.trunc_l2[l] = 0.0
+            if self.eps > 0.0 and s.dtype == "f32":            # Sec. 3.4: truncate small delta entries
+                d32 = I.astype(np.float32) - self.I_prev[l].astype(np.float32)
+                keep = np.abs(d32) >= np.float32(self.eps)
+                u = np.where(keep, 0.0, D)
+                D = np.where(keep, D, 0.0)
+                self.trunc_l2[l] = float(np.sqrt(np.sum(u * u)))
+                self.e_t += self.trunc_l2[l]                   # Eq. 7
             self.nnz[l] = int(np.count_nonzero(D))
             self.macs[l] = delta_accumulate(s, D, self.P_prev[l])   # P_t = P_{t-1} + F*dI
             self.I_prev[l] = I.copy()                           # snapshot the input
             tensors.append(nonlinearity(s, self.P_prev[l], tensors[s.res] if s.res >= 0 else None))
         return tensors, [p.copy() for p in self.P_prev]
 
+    def reset_to(self, frame):
+        """A precise (dense) inference of `frame` replaces the state and clears the accumulated
+        truncated value (Sec. 3.4, last sentence)."""
+        tensors, projs = dense_forward(self.layers, frame)
+        for l, s in enumerate(self.layers):
+            self.I_prev[l] = tensors[s.src].copy()
+            self.P_prev[l] = projs[l].copy()
+        self.e_t = 0.0
+        self.trunc_l2 = [0.0] * len(self.layers)
+        return tensors, projs
+
     def density(self):
         """Per-layer element density rho of the last step's input delta (Table 1)."""
         return [self.nnz[l] / self.I_prev[l].size for l in range(len(self.layers))]
+
+
+def aecs_predict(mu, e_t):
+    """Eq. 8 with H a fourth-order polynomial: e_c = mu[0] + mu[1] e_t + ... + mu[4] e_t^4."""
+    assert len(mu) == 5
+    return float(sum(float(m) * float(e_t) ** k for k, m in enumerate(mu)))
 
 
 # ------------------------------------------------------------- evaluation formulas

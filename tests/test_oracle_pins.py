@@ -304,3 +304,77 @@ def test_generated_stacks_are_not_degenerate():
                 assert 0.1 < frac < 0.9, (s.name, frac)
             elif s.shift >= 0:
                 assert 0.1 < float(np.mean(t > 0)) and float(np.mean(np.abs(t) >= 127)) < 0.2, s.name
+
+
+# ------------------------------------------------------------------ Sec. 3.4: truncation and Eq. 7 / Eq. 8
+def _eps_video(frames=6, c=4, hw=10, seed=5, small=0.004, big=0.3):
+    """Frames whose deltas are a mix of sub-threshold jitter (|d| <= small) and real changes (|d| ~ big)."""
+    rng = np.random.default_rng(seed)
+    v = np.empty((frames, 1, c, hw, hw), dtype=np.float32)
+    v[0] = rng.random((1, c, hw, hw), dtype=np.float32)
+    for t in range(1, frames):
+        jitter = (rng.random((1, c, hw, hw), dtype=np.float32) - 0.5) * np.float32(2 * small)
+        jitter[rng.random((1, c, hw, hw)) < 0.5] = 0
+        v[t] = v[t - 1] + jitter
+        v[t, 0, :, 2:5, 3:7] += np.float32(big) * rng.standard_normal((c, 3, 4)).astype(np.float32)
+    return v
+
+
+def test_truncated_recurrence_loses_exactly_the_filtered_truncated_part():
+    """By linearity, P_eps(T) = dense(X_T) - F * (sum of the truncated parts): an independent route to the
+    truncated recurrence's state (a dropped or doubly counted truncated entry breaks the equality)."""
+    specs = wl.single_conv_f32(c_in=4, c_out=6, hw=10)
+    v = _eps_video()
+    eps = 0.01
+    rec = orc.Recurrence(specs, eps=eps)
+    U = np.zeros((1, 4, 10, 10))
+    prev = np.zeros_like(v[0])
+    l2 = 0.0
+    for t in range(v.shape[0]):
+        rec.step(v[t])
+        d32 = v[t] - prev                                    # fp32 delta decides
+        u = np.where(np.abs(d32) < np.float32(eps), v[t].astype(np.float64) - prev.astype(np.float64), 0.0)
+        U += u
+        l2 += float(np.sqrt((u * u).sum()))
+        prev = v[t]
+    want = orc.dense_forward(specs, v[-1])[1][0] - orc.projection(specs[0], U, with_bias=False)
+    np.testing.assert_allclose(rec.P_prev[0], want, rtol=0, atol=1e-12)
+    assert abs(rec.e_t - l2) <= 1e-12 * max(1.0, l2)
+    assert rec.e_t > 0 and rec.macs[0] < 6 * 4 * 100
+
+
+def test_truncation_hand_case_and_limits():
+    s = wl.LayerSpec("conv", "f32", 1, 2, 2, 1, 1, 1, 1, 0, src=0)
+    s.weight = np.full((1, 1, 1, 1), 2.0, dtype=np.float32)
+    s.bias = np.array([1.0], dtype=np.float32)
+    rec = orc.Recurrence([s], eps=0.01)
+    x0 = np.zeros((1, 1, 2, 2), dtype=np.float32)
+    rec.step(x0)
+    x1 = np.array([0.005, 0.02, -0.003, 0.0], dtype=np.float32).reshape(1, 1, 2, 2)
+    rec.step(x1)
+    # kept: 0.02 -> P = 1 + 2 * 0.02 there; truncated: 0.005 and -0.003 -> l2 = sqrt(25e-6 + 9e-6)
+    np.testing.assert_allclose(rec.P_prev[0].ravel(), [1.0, 1.0 + 2 * float(np.float32(0.02)), 1.0, 1.0], atol=1e-12)
+    assert abs(rec.e_t - np.sqrt(float(np.float32(0.005)) ** 2 + float(np.float32(0.003)) ** 2)) < 1e-12
+    assert rec.nnz[0] == 1
+    # the snapshot moved on to x1: the same frame again has no delta at all, nothing more is truncated
+    e = rec.e_t
+    rec.step(x1)
+    assert rec.nnz[0] == 0 and rec.e_t == e
+    # a precise inference clears the accumulated value and the error
+    _, projs = rec.reset_to(x1)
+    assert rec.e_t == 0.0
+    np.testing.assert_allclose(rec.P_prev[0], projs[0])
+    # eps above every delta: nothing is ever multiplied, P stays at the bias
+    big = orc.Recurrence([s], eps=10.0)
+    big.step(x1)
+    assert big.macs[0] == 0 and np.all(big.P_prev[0] == 1.0)
+    # eps = 0 is the exact recurrence
+    ex = orc.Recurrence([s], eps=0.0)
+    ex.step(x1)
+    np.testing.assert_allclose(ex.P_prev[0], orc.dense_forward([s], x1)[1][0], atol=1e-12)
+
+
+def test_aecs_polynomial():
+    mu = [0.5, -1.0, 2.0, 0.25, -0.125]
+    for e in (0.0, 0.3, 2.0):
+        assert abs(orc.aecs_predict(mu, e) - float(np.polyval(mu[::-1], e))) < 1e-12
