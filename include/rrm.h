@@ -162,6 +162,20 @@ int rrm_net_dense_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int 
 int rrm_net_step_seq_host(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream);
 
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* host_out);
+
+/* ---- approximate mode: sparsity enhancement and accumulated error control (Sec. 3.4) -----------
+ * With eps > 0 every delta entry with |d| < eps is truncated to zero before the sparse product (fp32 stacks
+ * only, RRM_ERR_DTYPE otherwise).  The snapshot still becomes the new frame, so the truncated part u is lost:
+ * the outputs are approximate and the error accumulates until the next rrm_net_keyframe.  eps = 0 (the
+ * default) is the exact recurrence.  Synchronises the device; call it between frames. */
+int rrm_net_set_epsilon(rrm_net* net, float eps);
+/* Eq. 7: *e_t = sum over the frames since the last keyframe and over the linear layers of l2(u), u the
+ * truncated part of the layer's input delta (all streams of the batch together).  last_step_l2 (may be NULL)
+ * receives the [n_layers] terms of the most recent frame.  Synchronises the net's last stream. */
+int rrm_net_truncation(rrm_net* net, double* e_t, double* last_step_l2);
+/* Eq. 8 with H a fourth-order polynomial: mu[0] + mu[1] e_t + ... + mu[4] e_t^4 (host arithmetic).  The paper
+ * fits mu on its data; the caller supplies it and runs rrm_net_keyframe when the estimate passes its threshold. */
+double rrm_aecs_predict(const double mu[5], double e_t);
 /* Copies P_prev of `layer` / the current value of tensor `t` (boundary layout) to dst_dev. */
 int rrm_net_projection(rrm_net* net, int layer, void* P_dev, void* stream);
 int rrm_net_tensor(rrm_net* net, int t, void* dst_dev, void* stream);

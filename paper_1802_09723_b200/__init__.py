@@ -5,7 +5,7 @@ marshals arguments.  Importing it does not load the shared library; the first ca
 and fails loudly if the library is missing or cannot be built.
 """
 from .binding import (RRMError, LayerDesc, Stats, Net, Layer, lib, desc_from_spec, net_from_specs,
-                      layer_from_spec, fc_step_noalloc, KIND, DTYPE, ACT, VARIANT)
+                      layer_from_spec, fc_step_noalloc, aecs_predict, KIND, DTYPE, ACT, VARIANT)
 
 __all__ = ["RRMError", "LayerDesc", "Stats", "Net", "Layer", "lib", "desc_from_spec", "net_from_specs",
-           "layer_from_spec", "fc_step_noalloc", "KIND", "DTYPE", "ACT", "VARIANT"]
+           "layer_from_spec", "fc_step_noalloc", "aecs_predict", "KIND", "DTYPE", "ACT", "VARIANT"]

@@ -83,6 +83,12 @@ def lib():
         f.restype = ctypes.c_int
     L.rrm_fc_step_noalloc.argtypes = [_P, _P, _P, _P, _P] + [ctypes.c_int] * 5 + [_P]
     L.rrm_fc_step_noalloc.restype = ctypes.c_int
+    L.rrm_net_set_epsilon.argtypes = [_P, ctypes.c_float]
+    L.rrm_net_set_epsilon.restype = ctypes.c_int
+    L.rrm_net_truncation.argtypes = [_P, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    L.rrm_net_truncation.restype = ctypes.c_int
+    L.rrm_aecs_predict.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_double]
+    L.rrm_aecs_predict.restype = ctypes.c_double
     L.rrm_net_tensor_bytes.argtypes = [_P, ctypes.c_int]
     L.rrm_net_tensor_bytes.restype = ctypes.c_int64
     L.rrm_strerror.argtypes = [ctypes.c_int]
@@ -177,6 +183,16 @@ class Net:
         _check(lib().rrm_net_step_seq_host(self._h, _ptr(frames_host), _ptr(outs_host), T, _stream(stream)),
                "rrm_net_step_seq_host")
 
+    def set_epsilon(self, eps):
+        _check(lib().rrm_net_set_epsilon(self._h, float(eps)), "rrm_net_set_epsilon")
+
+    def truncation(self):
+        """(e_t of Eq. 7 since the last keyframe, [per-layer l2 of the last frame])."""
+        e = ctypes.c_double()
+        per = (ctypes.c_double * self.n_layers)()
+        _check(lib().rrm_net_truncation(self._h, ctypes.byref(e), per), "rrm_net_truncation")
+        return e.value, list(per)
+
     def stats(self, layer=0):
         s = Stats()
         _check(lib().rrm_net_get_stats(self._h, layer, ctypes.byref(s)), "rrm_net_get_stats")
@@ -237,6 +253,12 @@ def fc_step_noalloc(Wt, Xt, Xprev, P, Y, n, c_in, c_out, shift=-1, act="none", s
     can test the documented limits."""
     return lib().rrm_fc_step_noalloc(_ptr(Wt), _ptr(Xt), _ptr(Xprev), _ptr(P), _ptr(Y), n, c_in, c_out, shift,
                                      ACT[act], _stream(stream))
+
+
+def aecs_predict(mu, e_t):
+    """rrm_aecs_predict: the fourth-order polynomial error estimate of Eq. 8."""
+    arr = (ctypes.c_double * 5)(*[float(m) for m in mu])
+    return lib().rrm_aecs_predict(arr, float(e_t))
 
 
 def net_from_specs(specs, n=1, variant="auto", device="cuda"):

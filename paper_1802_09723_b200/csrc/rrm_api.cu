@@ -123,7 +123,7 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     for (auto& L : net->layers) cleared += (size_t)ceil_div(L.opixels(), 32) * 4;
     cleared = (cleared + 15) & ~(size_t)15;
     const size_t counters_off = cleared;
-    cleared += net->tensors.size() * 16 + net->layers.size() * 16;
+    cleared += net->tensors.size() * 32 + net->layers.size() * 16;
     RRM_TRY(dev_alloc(net, &net->cleared, cleared));
     net->cleared_bytes = cleared;
     char* base = reinterpret_cast<char*>(net->cleared);
@@ -134,13 +134,15 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     for (auto& T : net->tensors) {
         T.nnz = reinterpret_cast<unsigned long long*>(base + off);
         T.npix = reinterpret_cast<unsigned long long*>(base + off + 8);
-        off += 16;
+        T.trunc = reinterpret_cast<double*>(base + off + 16);
+        off += 32;
     }
     for (auto& L : net->layers) {
         L.macs = reinterpret_cast<unsigned long long*>(base + off);
         L.ocount = reinterpret_cast<int*>(base + off + 8);
         off += 16;
     }
+    RRM_TRY(dev_alloc(net, (void**)&net->aecs, (size_t)(1 + n_layers) * 8));
     for (int l = 0; l < n_layers; ++l) RRM_TRY(conv_layer_create(net, net->layers[l], W[l], B ? B[l] : nullptr));
     {
         const char* e = getenv("RRM_NO_GRAPH");
@@ -174,9 +176,9 @@ int build_step_graph(rrm_net* net)
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
-    RRM_TRY(dev_alloc(net, &net->frame_buf, (size_t)bi));
-    RRM_TRY(dev_alloc(net, &net->out_buf, (size_t)bo));
-    RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
+    if (!net->frame_buf) RRM_TRY(dev_alloc(net, &net->frame_buf, (size_t)bi));
+    if (!net->out_buf) RRM_TRY(dev_alloc(net, &net->out_buf, (size_t)bo));
+    if (!net->cap_stream) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
     RRM_CUDA_TRY(cudaStreamBeginCapture(net->cap_stream, cudaStreamCaptureModeThreadLocal));
     const int s = launch_sequence(net, net->frame_buf, net->out_buf, net->cap_stream, false, false);
     cudaGraph_t g = nullptr;
@@ -215,6 +217,8 @@ int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st,
     if (!stateless) RRM_CUDA_TRY(cudaMemsetAsync(net->cleared, 0, net->cleared_bytes, st));
     RRM_TRY(launch_import(net, frame, !dense, stateless, st));
     for (int l = 0; l < (int)net->layers.size(); ++l) RRM_TRY(launch_layer(net, l, dense, stateless, st));
+    if (!dense && net->eps > 0.f) RRM_TRY(launch_aecs(net, st));
+    if (dense && !stateless) RRM_CUDA_TRY(cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, st));   // a precise inference clears e_t
     if (out) RRM_TRY(launch_export_tensor(net, (int)net->layers.size(), out, stateless, st));
     return RRM_OK;
 }
@@ -384,6 +388,38 @@ int rrm_net_step_seq_host(rrm_net* net, const void* frames_host, void* outs_host
 int rrm_step_seq_host(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream)
 {
     return rrm_net_step_seq_host(layer, X_host, Y_host, T, stream);
+}
+
+int rrm_net_set_epsilon(rrm_net* net, float eps)
+{
+    if (!net || !(eps >= 0.f)) return RRM_ERR_INVALID_ARG;
+    if (net->layers[0].fc_fused) return RRM_ERR_UNSUPPORTED;
+    for (auto& L : net->layers) if (L.d.dtype != RRM_F32) return RRM_ERR_DTYPE;
+    if (eps == net->eps) return RRM_OK;
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
+    net->eps = eps;
+    // the threshold is a kernel argument: a captured step has to be captured again
+    if (net->step_exec) { cudaGraphExecDestroy(net->step_exec); net->step_exec = nullptr; }
+    if (net->step_graph) { cudaGraphDestroy(net->step_graph); net->step_graph = nullptr; }
+    return RRM_OK;
+}
+
+int rrm_net_truncation(rrm_net* net, double* e_t, double* last_step_l2)
+{
+    if (!net || !e_t) return RRM_ERR_INVALID_ARG;
+    if (net->layers[0].fc_fused) return RRM_ERR_UNSUPPORTED;
+    RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
+    std::vector<double> h(1 + net->layers.size());
+    RRM_CUDA_TRY(cudaMemcpy(h.data(), net->aecs, h.size() * 8, cudaMemcpyDeviceToHost));
+    *e_t = h[0];
+    if (last_step_l2) for (size_t l = 0; l < net->layers.size(); ++l) last_step_l2[l] = h[1 + l];
+    return RRM_OK;
+}
+
+double rrm_aecs_predict(const double mu[5], double e_t)
+{
+    if (!mu) return 0.0;
+    return mu[0] + e_t * (mu[1] + e_t * (mu[2] + e_t * (mu[3] + e_t * mu[4])));
 }
 
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)

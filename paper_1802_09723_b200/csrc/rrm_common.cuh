@@ -52,6 +52,7 @@ struct Tensor {
     int* pnnz = nullptr;              // per-pixel count of non-zero delta elements (valid where act is set)
     unsigned long long* nnz = nullptr;      // total non-zero delta elements (cleared every step)
     unsigned long long* npix = nullptr;     // active pixels (cleared every step)
+    double* trunc = nullptr;                // fp32: sum of squares of the truncated delta entries (cleared every step)
     void* X2 = nullptr;               // value buffer of the stateless dense path
     bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
     Readers readers{};                // the layers that read it
@@ -127,6 +128,8 @@ struct rrm_net {
     void* frame_buf = nullptr;        // the step's input frame, boundary layout
     void* out_buf = nullptr;          // the step's last tensor, boundary layout
     bool graph_off = false;           // RRM_NO_GRAPH=1: launch kernel by kernel (debugging)
+    float eps = 0.f;                  // Sec. 3.4: fp32 delta entries below it are truncated (0: exact)
+    double* aecs = nullptr;           // [1 + layers]: accumulated truncated value e_t (Eq. 7), then the last step's l2 per layer
     std::vector<void*> allocs;        // everything to free
 };
 
@@ -159,5 +162,6 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
 int launch_export_tensor(rrm_net* net, int t, void* dst_dev, bool stateless, cudaStream_t st);
 int launch_export_projection(rrm_net* net, int l, void* dst_dev, cudaStream_t st);
 int reset_state(rrm_net* net, cudaStream_t st);
+int launch_aecs(rrm_net* net, cudaStream_t st);
 
 }  // namespace rrm

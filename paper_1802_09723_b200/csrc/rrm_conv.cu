@@ -388,7 +388,8 @@ template <typename T, bool DELTA>
 __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ src, T* X, T* D, uint32_t* act,
                                                           int* pnnz, unsigned long long* nnz,
                                                           unsigned long long* npix, int* errw,
-                                                          int c, int cs, int hw, int w, Readers readers)
+                                                          int c, int cs, int hw, int w, Readers readers,
+                                                          float eps, double* trunc)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T* s_x = reinterpret_cast<T*>(smem_raw);               // [IMP_TP][cs + 1]
@@ -404,6 +405,7 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
     }
     __syncthreads();
     const size_t gp0 = (size_t)ns * hw + pix0;
+    float sq = 0.f;                                          // squares of the truncated delta entries
     for (int idx = tid; idx < IMP_TP * cs; idx += 256) {
         const int pl = idx / cs, ch = idx - pl * cs;
         if (pix0 + pl >= hw) continue;
@@ -411,15 +413,19 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
         const T xt = s_x[pl * ld + ch];
         if (DELTA) {
             const T xp = X[o];
+            T dv = (T)(xt - xp);
             if (xt != xp) {
-                atomicAdd(&s_cnt[pl], 1);
-                X[o] = xt;
+                X[o] = xt;                                   // the snapshot always moves on to the new frame
+                bool keep = true;
+                if (sizeof(T) == 4 && eps > 0.f) keep = fabsf((float)dv) >= eps;   // Sec. 3.4: small deltas are truncated
+                if (keep) atomicAdd(&s_cnt[pl], 1);
+                else { sq += (float)dv * (float)dv; dv = (T)0; }
                 if (sizeof(T) == 1) {
                     const int d = (int)xt - (int)xp;
                     if (d < -128 || d > 127) atomicOr(errw, ERRW_BOUNDS);
                 }
             }
-            s_x[pl * ld + ch] = (T)(xt - xp);
+            s_x[pl * ld + ch] = dv;
         } else {
             X[o] = xt;
         }
@@ -449,8 +455,13 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
     }
     // every changed pixel marks the projection pixels of the reading layers that it touches
     __shared__ unsigned long long s_macs[MAX_READERS];
+    __shared__ float s_sq;
     if (tid < MAX_READERS) s_macs[tid] = 0;
+    if (tid == 0) s_sq = 0.f;
     __syncthreads();
+    #pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if (lane == 0 && sq > 0.f) atomicAdd(&s_sq, sq);
     for (int pl = warp; pl < IMP_TP; pl += 8) {
         const int cnt = (pix0 + pl < hw) ? s_cnt[pl] : 0;
         if (cnt == 0) continue;
@@ -464,6 +475,7 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
     }
     __syncthreads();
     if (tid < readers.n && s_macs[tid]) atomicAdd(readers.r[tid].macs, s_macs[tid]);
+    if (tid == 0 && trunc && s_sq > 0.f) atomicAdd(trunc, (double)s_sq);
 }
 
 // int8 frames with up to 4 channels (one 4-byte word per pixel): one thread per pixel, plane reads coalesced
@@ -599,6 +611,8 @@ struct EpiParams {
     int* errw;
     int n, oh, ow, th, tw, c_out, cs, pool_k, pool_s, pool_p, act_fn, shift, theta;
     Readers readers;          // layers that read the output tensor
+    float eps;                // fp32: delta entries below it are truncated to zero (Sec. 3.4)
+    double* trunc;            // fp32: receives the sum of squares of the truncated entries
 };
 
 // PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.  KW: pool window edge (1 = no pool).
@@ -608,9 +622,10 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
     __shared__ unsigned long long s_macs[MAX_READERS];
     __shared__ unsigned int s_nnz, s_npix;
+    __shared__ float s_sq;
     const int lane = threadIdx.x & 31;
     if (threadIdx.x < MAX_READERS) s_macs[threadIdx.x] = 0;
-    if (threadIdx.x == 0) { s_nnz = 0; s_npix = 0; }
+    if (threadIdx.x == 0) { s_nnz = 0; s_npix = 0; s_sq = 0.f; }
     __syncthreads();
     const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int tpix = p.n * p.th * p.tw;
@@ -632,6 +647,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
         on = DENSE ? true : (__ballot_sync(0xffffffffu, upd) != 0);
     }
     int cnt = 0;
+    float sq = 0.f;                                          // squares of the truncated delta entries (fp32)
     if (on) {
         const pt* P = reinterpret_cast<const pt*>(p.P);
         const bool vec = (p.c_out & 3) == 0;
@@ -735,8 +751,13 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                         if (DENSE) X[o + j] = best[j];
                         else {
                             const pt old = X[o + j];
-                            Dp[o + j] = best[j] - old;
-                            if (best[j] != old) { X[o + j] = best[j]; ++cnt; }
+                            pt dv = best[j] - old;
+                            if (best[j] != old) {
+                                X[o + j] = best[j];          // the snapshot always moves on
+                                if (PT == T_F32 && p.eps > 0.f && fabsf((float)dv) < p.eps) { sq += (float)dv * (float)dv; dv = 0; }
+                                else ++cnt;
+                            }
+                            Dp[o + j] = dv;
                         }
                     }
                 }
@@ -745,7 +766,8 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     }
     if (DENSE) return;
     #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    for (int o = 16; o > 0; o >>= 1) { cnt += __shfl_xor_sync(0xffffffffu, cnt, o); sq += __shfl_xor_sync(0xffffffffu, sq, o); }
+    if (PT == T_F32 && lane == 0 && sq > 0.f) atomicAdd(&s_sq, sq);
     if (cnt) {                                               // uniform inside the warp
         if (lane == 0) {
             atomicOr(&p.act[r >> 5], 1u << (r & 31));
@@ -766,6 +788,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
         atomicAdd(p.nnz, (unsigned long long)s_nnz);
         atomicAdd(p.npix, (unsigned long long)s_npix);
     }
+    if (PT == T_F32 && threadIdx.x == 0 && p.trunc && s_sq > 0.f) atomicAdd(p.trunc, (double)s_sq);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -787,6 +810,16 @@ __global__ void fill_projection_kernel(T* P, const T* bias, int c_out, long long
 {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < total) P[i] = bias ? bias[i % c_out] : (T)0;
+}
+
+// Eq. 7, one frame: e_t += sum over the linear layers of l2(truncated part of the layer's input).
+struct AecsParams { const double* sumsq[64]; int n; double* e_t; double* last_l2; };
+__global__ void aecs_accumulate_kernel(AecsParams p)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    double add = 0.0;
+    for (int l = 0; l < p.n; ++l) { const double v = sqrt(*p.sumsq[l]); p.last_l2[l] = v; add += v; }
+    *p.e_t += add;
 }
 
 // ================================================================================================
@@ -880,16 +913,16 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                 cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             }
             if (delta) kd<<<grid, 256, smem, st>>>((const float*)frame, (float*)X, (float*)T.D, T.act, T.pnnz, T.nnz,
-                                                   T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers);
+                                                   T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, net->eps, T.trunc);
             else kn<<<grid, 256, smem, st>>>((const float*)frame, (float*)X, nullptr, nullptr, nullptr, nullptr,
-                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{});
+                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr);
         } else {
             auto kd = import_nchw_kernel<int8_t, true>;
             auto kn = import_nchw_kernel<int8_t, false>;
             if (delta) kd<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, (int8_t*)T.D, T.act, T.pnnz,
-                                                   T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers);
+                                                   T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, 0.f, nullptr);
             else kn<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, nullptr, nullptr, nullptr, nullptr,
-                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{});
+                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr);
         }
     }
     RRM_CUDA_TRY(cudaGetLastError());
@@ -959,11 +992,24 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     e.n = d.n; e.oh = L.oh; e.ow = L.ow; e.th = L.th; e.tw = L.tw; e.c_out = d.c_out; e.cs = out.cs;
     e.pool_k = d.pool_k; e.pool_s = d.pool_s; e.pool_p = d.pool_p; e.act_fn = d.act; e.shift = d.shift; e.theta = d.theta;
     e.readers = dense ? Readers{} : out.readers;
+    e.eps = net->eps; e.trunc = out.trunc;
     const int blocks = ceil_div(out.pixels(), 8);
     int es;
     if (proj_type(L) == T_F32) es = dense ? launch_epi<T_F32, true>(e, out.dtype, blocks, st) : launch_epi<T_F32, false>(e, out.dtype, blocks, st);
     else es = dense ? launch_epi<T_I32, true>(e, out.dtype, blocks, st) : launch_epi<T_I32, false>(e, out.dtype, blocks, st);
     RRM_TRY(es);
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
+int launch_aecs(rrm_net* net, cudaStream_t st)
+{
+    AecsParams a;
+    a.n = (int)net->layers.size();
+    if (a.n > 64) return RRM_ERR_UNSUPPORTED;
+    for (int l = 0; l < a.n; ++l) a.sumsq[l] = net->tensors[net->layers[l].d.src].trunc;
+    a.e_t = net->aecs; a.last_l2 = net->aecs + 1;
+    aecs_accumulate_kernel<<<1, 32, 0, st>>>(a);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
