@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     constexpr int STAGE_WORDS = GEMM_B_WORDS + A_BUFS * GEMM_A_WORDS;
     __shared__ __align__(8) unsigned long long s_full[GEMM_STAGES];
     __shared__ int s_q[TM];
-    __shared__ int s_tmp[33];
+    __shared__ int s_tmp[256 + 34];
     __shared__ unsigned s_tapmask[4];
     __shared__ unsigned long long s_rmask[TM][2];
     __shared__ int s_pix0[TM];

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
     TcSmemTail* S = reinterpret_cast<TcSmemTail*>(base + TC_STAGES * TC_STAGE_BYTES);
     const uint32_t base_u32 = smem_u32(base);
-    __shared__ int s_tmp[33];
+    __shared__ int s_tmp[256 + 34];
     int count = p.opixels;
     if (!DENSE) {
         // this CTA's rows: the tile-th group of 128 set bits of the layer's update bitmap

@@ -42,11 +42,15 @@ __device__ __forceinline__ void scatter_changed(const Readers& R, int ns, int y,
 
 // Rows [tile * TM, tile * TM + TM) of the set bits of bm[0 .. words), in increasing pixel order, go to
 // s_q[0 .. TM) (-1 where the bitmap has fewer).  Returns the total number of set bits.  Every thread
-// of the CTA calls it; s_tmp holds 33 ints.
+// of the CTA calls it (blockDim.x <= 256, TM <= blockDim.x); s_pref holds 256 + 34 ints.
+// Each thread counts a contiguous share of the words; an exclusive prefix sum over the threads tells
+// every row which thread's share holds its bit, and the row walks that share (a few words) itself:
+// all TM rows are located in parallel.
 template <int TM>
-__device__ int select_rows(const uint32_t* __restrict__ bm, int words, int tile, int* s_q, int* s_tmp)
+__device__ int select_rows(const uint32_t* __restrict__ bm, int words, int tile, int* s_q, int* s_pref)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nwarps = (nt + 31) >> 5;
+    int* s_warp = s_pref + 257;
     const int nper = (words + nt - 1) / nt;
     const int lo = min(words, tid * nper), hi = min(words, lo + nper);
     int mine = 0;
@@ -57,26 +61,33 @@ __device__ int select_rows(const uint32_t* __restrict__ bm, int words, int tile,
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
     }
-    if (lane == 31) s_tmp[warp] = incl;
-    if (tid < TM) s_q[tid] = -1;
+    if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
-    int run = incl - mine, total = 0;
+    int before = incl - mine, total = 0;
     for (int w = 0; w < nwarps; ++w) {
-        const int v = s_tmp[w];
-        if (w < warp) run += v;
+        const int v = s_warp[w];
+        if (w < warp) before += v;
         total += v;
     }
-    const int first = tile * TM;
-    if (run < first + TM && run + mine > first) {
-        for (int i = lo; i < hi; ++i) {
-            uint32_t w = __ldg(bm + i);
-            while (w) {
-                const int b = __ffs(w) - 1;
-                w &= w - 1;
-                if (run >= first && run < first + TM) s_q[run - first] = i * 32 + b;
-                ++run;
+    s_pref[tid] = before;                                    // set bits in the shares of threads 0 .. tid-1
+    if (tid == nt - 1) s_pref[nt] = total;
+    __syncthreads();
+    if (tid < TM) {
+        const int rank = tile * TM + tid;
+        int q = -1;
+        if (rank < total) {
+            int t = 0;                                       // largest t with s_pref[t] <= rank
+            for (int step = 128; step > 0; step >>= 1)
+                if (t + step < nt && s_pref[t + step] <= rank) t += step;
+            int k = rank - s_pref[t];
+            for (int i = t * nper; i < words; ++i) {
+                const uint32_t w = __ldg(bm + i);
+                const int c = __popc(w);
+                if (k < c) { q = i * 32 + (int)__fns(w, 0, k + 1); break; }
+                k -= c;
             }
         }
+        s_q[tid] = q;
     }
     __syncthreads();
     return total;
