@@ -654,6 +654,10 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
         const int c_iter = (OT == T_BIN) ? p.cs * 32 : p.cs;
         for (int c0 = 0; c0 < c_iter; c0 += 128) {
             const int c = c0 + lane * 4;
+            // the stored int8 activation word is fetched together with the projection, not after it
+            uint32_t old_word = 0;
+            if (OT == T_I8 && !DENSE && c < p.cs)
+                old_word = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(p.X) + (size_t)r * p.cs + c);
             // ---- the 4-channel words of every window position
             pt v[KW * KW][4];
             #pragma unroll
@@ -729,7 +733,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                     uint32_t* X = reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.X) + o);
                     if (DENSE) *X = nw;
                     else {
-                        const uint32_t ow_ = *X;
+                        const uint32_t ow_ = old_word;
                         uint32_t dw = 0;
                         #pragma unroll
                         for (int j = 0; j < 4; ++j) {
