@@ -46,3 +46,52 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src, f
+
+
+def _desc(**kw):
+    import paper_1802_09723_b200 as rrm
+    d = rrm.LayerDesc()
+    base = dict(kind=0, dtype=0, n=1, c_in=4, h=8, w=8, c_out=4, kh=3, kw=3, stride=1, pad=1, act=0, pool_k=0, pool_s=0,
+                pool_p=0, shift=-1, theta=0, src=0, res=-1, variant=0)
+    base.update(kw)
+    for k, v in base.items():
+        setattr(d, k, v)
+    return d
+
+
+def test_invalid_descriptions_are_rejected_before_any_device_work():
+    """Validation comes first in rrm_layer_create, so these calls return their error codes on a machine
+    without a GPU too (the weight pointer is a dummy that is never dereferenced)."""
+    import paper_1802_09723_b200 as rrm
+    L = rrm.lib()
+    INVALID, SHAPE, DTYPE, UNSUPPORTED = -1, -2, -3, -8
+    dummy = ctypes.c_void_p(16)
+    cases = [
+        (_desc(kind=7), INVALID), (_desc(dtype=9), DTYPE), (_desc(n=0), SHAPE), (_desc(c_out=0), SHAPE),
+        (_desc(stride=0), SHAPE), (_desc(pad=3), SHAPE), (_desc(kh=11, kw=11, h=4, w=4, pad=0), SHAPE),
+        (_desc(kind=1, h=2), SHAPE), (_desc(act=5), INVALID), (_desc(act=2), UNSUPPORTED),
+        (_desc(pool_k=3, pool_s=0), SHAPE), (_desc(pool_k=5, pool_s=2), UNSUPPORTED), (_desc(shift=40, dtype=1), INVALID),
+        (_desc(variant=9), INVALID), (_desc(dtype=1, shift=-1, act=1), UNSUPPORTED),
+    ]
+    for d, want in cases:
+        h = ctypes.c_void_p()
+        got = L.rrm_layer_create(ctypes.byref(h), ctypes.byref(d), dummy, None)
+        assert got == want, ({n: getattr(d, n) for n, _ in d._fields_}, got, want)
+        assert not h.value
+    # a stack whose second layer reads a tensor that does not exist yet, or whose shapes do not chain
+    two = (rrm.LayerDesc * 2)(_desc(), _desc(src=2))
+    W = (ctypes.c_void_p * 2)(16, 16)
+    h = ctypes.c_void_p()
+    assert L.rrm_net_create(ctypes.byref(h), two, 2, W, None) == INVALID
+    two = (rrm.LayerDesc * 2)(_desc(), _desc(src=1, c_in=5))
+    assert L.rrm_net_create(ctypes.byref(h), two, 2, W, None) == SHAPE
+    assert L.rrm_net_set_epsilon(None, ctypes.c_float(0.1)) == INVALID
+    assert L.rrm_step_seq(None, None, None, 4, None) == INVALID
+
+
+def test_error_strings_cover_every_status():
+    import paper_1802_09723_b200 as rrm
+    L = rrm.lib()
+    seen = {L.rrm_strerror(s) for s in range(0, -9, -1)}
+    assert len(seen) == 9 and b"unknown status" not in seen
+    assert L.rrm_strerror(-99) == b"unknown status"
