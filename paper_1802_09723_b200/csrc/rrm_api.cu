@@ -169,24 +169,34 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
 
 int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
 
-// Captures the delta step's launch sequence into a graph (on a private stream: a capture cannot start
-// on the legacy default stream) so that later steps cost one graph launch on the host.
-int build_step_graph(rrm_net* net)
+// Captures one of the per-frame launch sequences into a graph (on a private stream: a capture cannot
+// start on the legacy default stream) so that later frames cost one graph launch on the host.
+int build_graph(rrm_net* net, int kind)
 {
+    const bool dense = kind != 0, stateless = kind == 2;
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
     if (!net->frame_buf) RRM_TRY(dev_alloc(net, &net->frame_buf, (size_t)bi));
     if (!net->out_buf) RRM_TRY(dev_alloc(net, &net->out_buf, (size_t)bo));
+    if (stateless) RRM_TRY(ensure_stateless(net));           // allocations cannot happen inside a capture
     if (!net->cap_stream) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
     RRM_CUDA_TRY(cudaStreamBeginCapture(net->cap_stream, cudaStreamCaptureModeThreadLocal));
-    const int s = launch_sequence(net, net->frame_buf, net->out_buf, net->cap_stream, false, false);
+    const int s = launch_sequence(net, net->frame_buf, net->out_buf, net->cap_stream, dense, stateless);
     cudaGraph_t g = nullptr;
     const cudaError_t e = cudaStreamEndCapture(net->cap_stream, &g);
     if (s != RRM_OK || e != cudaSuccess || !g) { if (g) cudaGraphDestroy(g); cudaGetLastError(); return s != RRM_OK ? s : RRM_ERR_CUDA; }
-    net->step_graph = g;
-    RRM_CUDA_TRY(cudaGraphInstantiate(&net->step_exec, g, 0));
+    net->graph[kind] = g;
+    RRM_CUDA_TRY(cudaGraphInstantiate(&net->exec[kind], g, 0));
     return RRM_OK;
+}
+
+void drop_graphs(rrm_net* net)
+{
+    for (int k = 0; k < 3; ++k) {
+        if (net->exec[k]) { cudaGraphExecDestroy(net->exec[k]); net->exec[k] = nullptr; }
+        if (net->graph[k]) { cudaGraphDestroy(net->graph[k]); net->graph[k] = nullptr; }
+    }
 }
 
 int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
@@ -194,17 +204,18 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
     if (!net || !frame) return RRM_ERR_INVALID_ARG;
     net->last_stream = st;
     if (net->layers[0].fc_fused) return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
-    if (!dense && !stateless && !net->graph_off) {
-        if (!net->step_exec) {
-            const int s = build_step_graph(net);
+    if (!net->graph_off) {
+        const int kind = !dense ? 0 : (stateless ? 2 : 1);
+        if (!net->exec[kind]) {
+            const int s = build_graph(net, kind);
             if (s != RRM_OK) { net->graph_off = true; if (s == RRM_ERR_ALLOC) return s; }
         }
-        if (net->step_exec) {
+        if (net->exec[kind]) {
             int64_t bi = 0, bo = 0;
             tensor_bytes_boundary(net->tensors.front(), &bi);
             tensor_bytes_boundary(net->tensors.back(), &bo);
             RRM_CUDA_TRY(cudaMemcpyAsync(net->frame_buf, frame, (size_t)bi, cudaMemcpyDeviceToDevice, st));
-            RRM_CUDA_TRY(cudaGraphLaunch(net->step_exec, st));
+            RRM_CUDA_TRY(cudaGraphLaunch(net->exec[kind], st));
             if (out) RRM_CUDA_TRY(cudaMemcpyAsync(out, net->out_buf, (size_t)bo, cudaMemcpyDeviceToDevice, st));
             return RRM_OK;
         }
@@ -290,8 +301,7 @@ int rrm_net_destroy(rrm_net* net)
         if (L.seq_ev) cudaEventDestroy(L.seq_ev);
         if (L.seq_stat_host) cudaFreeHost(L.seq_stat_host);
     }
-    if (net->step_exec) cudaGraphExecDestroy(net->step_exec);
-    if (net->step_graph) cudaGraphDestroy(net->step_graph);
+    drop_graphs(net);
     if (net->cap_stream) cudaStreamDestroy(net->cap_stream);
     for (void* p : net->allocs) cudaFree(p);
     delete net;
@@ -398,9 +408,8 @@ int rrm_net_set_epsilon(rrm_net* net, float eps)
     if (eps == net->eps) return RRM_OK;
     RRM_CUDA_TRY(cudaDeviceSynchronize());
     net->eps = eps;
-    // the threshold is a kernel argument: a captured step has to be captured again
-    if (net->step_exec) { cudaGraphExecDestroy(net->step_exec); net->step_exec = nullptr; }
-    if (net->step_graph) { cudaGraphDestroy(net->step_graph); net->step_graph = nullptr; }
+    // the threshold is a kernel argument: captured sequences have to be captured again
+    drop_graphs(net);
     return RRM_OK;
 }
 

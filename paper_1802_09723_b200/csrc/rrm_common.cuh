@@ -121,9 +121,10 @@ struct rrm_net {
     void* stage_in = nullptr;         // device staging for the *_host entry points
     void* stage_out = nullptr;
     int stage_frames = 0;             // frames the staging buffers hold
-    // the per-frame launch sequence of rrm_net_step, captured once and replayed (fixed frame / output buffers)
-    cudaGraph_t step_graph = nullptr;
-    cudaGraphExec_t step_exec = nullptr;
+    // the per-frame launch sequences (0: delta step, 1: keyframe, 2: stateless dense pass), each captured
+    // once and replayed (fixed frame / output buffers)
+    cudaGraph_t graph[3] = {nullptr, nullptr, nullptr};
+    cudaGraphExec_t exec[3] = {nullptr, nullptr, nullptr};
     cudaStream_t cap_stream = nullptr;
     void* frame_buf = nullptr;        // the step's input frame, boundary layout
     void* out_buf = nullptr;          // the step's last tensor, boundary layout
@@ -162,6 +163,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
 int launch_export_tensor(rrm_net* net, int t, void* dst_dev, bool stateless, cudaStream_t st);
 int launch_export_projection(rrm_net* net, int l, void* dst_dev, cudaStream_t st);
 int reset_state(rrm_net* net, cudaStream_t st);
+int ensure_stateless(rrm_net* net);
 int launch_aecs(rrm_net* net, cudaStream_t st);
 
 }  // namespace rrm

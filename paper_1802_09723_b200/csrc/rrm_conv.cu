@@ -875,7 +875,7 @@ int reset_state(rrm_net* net, cudaStream_t st)
     return RRM_OK;
 }
 
-static int ensure_stateless(rrm_net* net)
+int ensure_stateless(rrm_net* net)
 {
     for (auto& T : net->tensors)
         if (!T.X2) RRM_TRY(dev_alloc(net, &T.X2, T.bytes()));
