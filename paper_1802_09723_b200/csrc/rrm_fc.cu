@@ -18,14 +18,6 @@
 
 namespace cg = cooperative_groups;
 
-// Optional phase timestamps for tuning builds (-DRRM_FC_TIMING): CTA (0,0,0) stores clock64() per phase.
-#ifdef RRM_FC_TIMING
-__device__ long long rrm_fc_phase_clock[16];
-#define RRM_FC_PHASE(i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) rrm_fc_phase_clock[i] = clock64(); } while (0)
-#else
-#define RRM_FC_PHASE(i) do { } while (0)
-#endif
-
 namespace rrm {
 
 constexpr int FC_THREADS = 256;
@@ -82,7 +74,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
     int32_t* Ps = p.P + (size_t)s * K + slice * FC_OW;
     const int width = min(FC_OW, K - slice * FC_OW);
 
-    RRM_FC_PHASE(0);
     cluster_arrive_relaxed();                        // waited for just before the first remote store
     // stored projection of this slice: fetched now, needed at the very end
     int p_old = 0;
@@ -100,7 +91,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
             if (xp4) xb[i] = __ldg(xp4 + c_begin + i);
         }
     }
-    RRM_FC_PHASE(1);
     // raw bytes to shared memory (the gather looks the delta of an entry up there) and a 64-bit mask
     // of the non-zero delta bytes of this thread's 64 inputs (a byte differs <=> its delta is non-zero)
     unsigned long long m = 0;
@@ -145,7 +135,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
     s_off[tid] = offset;
     s_mask[tid] = m;
     __syncthreads();
-    RRM_FC_PHASE(2);
     // ---- 2. this CTA's share of the list, one entry per thread: find the thread that scanned entry e
     // (largest t with s_off[t] <= e) and pick the matching set bit of its mask
     const int per_cta = (total + FC_CL - 1) / FC_CL;
@@ -187,7 +176,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
     }
     __syncthreads();
 
-    RRM_FC_PHASE(3);
     // ---- 3. gather the columns of the owned entries: 8 lanes x 16 bytes span the slice, 32 columns in flight
     const int sub = tid & 7, grp = tid >> 3;
     const int o0 = slice * FC_OW + sub * 16;
@@ -234,7 +222,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
                 if (j[u] >= 0) fma16(w[u], (int)s_xt[j[u]] - (int)s_xp[j[u]]);
         }
     }
-    RRM_FC_PHASE(4);
     // ---- 4. reduce: the 4 column groups of a warp by shuffles, the 8 warps through shared memory
     #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -249,7 +236,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
     // ---- 5. across the cluster: every CTA pushes its partial sums into rank 0's shared memory, then
     // arrives at the cluster barrier; only rank 0 waits, adds them onto the projection slice it owns
     // (owner computes, no atomics), applies f and writes Y_t.
-    RRM_FC_PHASE(5);
     cluster_wait();                                  // pairs with the arrive at kernel entry: all CTAs are running
     if (tid < FC_OW) {
         int v = 0;
@@ -257,11 +243,9 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
         for (int w = 0; w < FC_THREADS / 32; ++w) v += s_red[w][tid];
         *cluster.map_shared_rank(&s_part[kg][tid], 0) = v;
     }
-    RRM_FC_PHASE(6);
     cluster_arrive_release();
     if (kg != 0) return;                             // nobody reads a non-zero rank's shared memory
     cluster_wait_acquire();
-    RRM_FC_PHASE(7);
     if (tid < width) {
         int v = p_old;
         #pragma unroll
@@ -273,7 +257,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
             else reinterpret_cast<int8_t*>(p.Y)[oi] = (int8_t)fc_apply_f(v, p.shift, p.act);
         }
     }
-    RRM_FC_PHASE(8);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -624,9 +607,3 @@ extern "C" int rrm_fc_step_noalloc(const int8_t* Wt_dev, const int8_t* Xt_dev, i
     return RRM_OK;
 }
 
-#ifdef RRM_FC_TIMING
-extern "C" int rrm_fc_phase_clocks(long long* host16)
-{
-    return cudaMemcpyFromSymbol(host16, rrm_fc_phase_clock, sizeof(long long) * 16) == cudaSuccess ? 0 : -7;
-}
-#endif
