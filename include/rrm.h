@@ -52,7 +52,12 @@ enum {
 enum { RRM_CONV = 0, RRM_FC = 1 };
 enum { RRM_F32 = 0, RRM_I8 = 1, RRM_BIN = 2 };
 enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2 };
-/* how F*dI is evaluated; AUTO picks per layer */
+/* How F*dI is evaluated.  As a request in rrm_layer_desc.variant: AUTO lets the library pick per layer (tensor
+ * cores for int8 and binary layers, CUDA cores for fp32; for a lone int8 FC layer also: dense evaluation of a chunk
+ * when the previous chunk's measured delta density was high); GATHER forces the CUDA-core / column-gather kernels;
+ * TENSOR is AUTO without the density switch; DENSE on a lone FC layer selects the generic (non-fused) path.
+ * As a report in rrm_stats.variant: what the most recent step ran (GATHER, TENSOR, or DENSE for a chunk that was
+ * evaluated densely). */
 enum { RRM_VARIANT_AUTO = 0, RRM_VARIANT_GATHER = 1, RRM_VARIANT_TENSOR = 2, RRM_VARIANT_DENSE = 3 };
 
 /*
@@ -125,8 +130,11 @@ int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* st
  *   Y_dev  [T] outputs f(P_t), each in the layer's output layout, back to back; may be NULL
  * For a lone int8 FC layer all T input deltas are known up front (dI_t = X_t - X_{t-1}), so the T
  * sparse products W dI_t run in ONE launch and only the running sum P_t = P_{t-1} + W dI_t is
- * serial; other layers and stacks are stepped frame by frame on `stream`.  The first call with a
- * larger T than any before allocates scratch memory (T * N * c_out * 4 bytes); later calls do not.
+ * serial; other layers and stacks are stepped frame by frame on `stream`.  With variant AUTO the
+ * library reads back the measured delta density of each chunk (asynchronously) and evaluates the
+ * next chunk densely on the tensor cores instead when that density was high: outputs, state and
+ * counters are the same integers either way.  The first call with a larger T than any before
+ * allocates scratch memory (T * N * c_out * 4 bytes); later calls do not.
  * T * N must not exceed 65535.  Asynchronous on `stream`.  After the call rrm_get_stats reports the
  * counters summed over the chunk's frames. */
 int rrm_step_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream);
