@@ -51,7 +51,8 @@ enum {
 
 enum { RRM_CONV = 0, RRM_FC = 1 };
 enum { RRM_F32 = 0, RRM_I8 = 1, RRM_BIN = 2 };
-enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2 };
+enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2,
+       RRM_ACT_LEAKY = 3 /* fp32 only: x > 0 ? x : 0.1 x, the leaky ReLU of the YOLOv2-style stacks of Sec. 4.4 */ };
 /* How F*dI is evaluated.  As a request in rrm_layer_desc.variant: AUTO lets the library pick per layer (tensor
  * cores for int8 and binary layers, CUDA cores for fp32; for a lone int8 FC layer also: dense evaluation of a chunk
  * when the previous chunk's measured delta density was high); GATHER forces the CUDA-core / column-gather kernels;

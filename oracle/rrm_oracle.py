@@ -138,6 +138,8 @@ def nonlinearity(spec, P, res=None):
         v = P if res is None else P + res
         if spec.act == "relu":
             v = np.maximum(v, 0.0)
+        elif spec.act == "leaky":                       # leaky ReLU with the slope 0.1 (as an fp32 constant)
+            v = np.where(v > 0.0, v, float(np.float32(0.1)) * v)
         elif spec.act != "none":
             raise ValueError(spec.act)
         return maxpool(v, *spec.pool) if spec.pool is not None else v

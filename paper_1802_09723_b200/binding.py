@@ -10,7 +10,7 @@ from . import build as _build
 
 KIND = {"conv": 0, "fc": 1}
 DTYPE = {"f32": 0, "i8": 1, "bin": 2}
-ACT = {"none": 0, "relu": 1, "sign": 2}
+ACT = {"none": 0, "relu": 1, "sign": 2, "leaky": 3}
 VARIANT = {"auto": 0, "gather": 1, "tensor": 2, "dense": 3}
 
 

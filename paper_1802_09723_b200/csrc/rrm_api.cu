@@ -25,7 +25,8 @@ int validate_desc(const rrm_layer_desc& d, int l, int n_layers)
         return RRM_ERR_SHAPE;
     if (d.h + 2 * d.pad < d.kh || d.w + 2 * d.pad < d.kw) return RRM_ERR_SHAPE;
     if (d.pad >= d.kh || d.pad >= d.kw) return RRM_ERR_SHAPE;
-    if (d.act != RRM_ACT_NONE && d.act != RRM_ACT_RELU && d.act != RRM_ACT_SIGN) return RRM_ERR_INVALID_ARG;
+    if (d.act != RRM_ACT_NONE && d.act != RRM_ACT_RELU && d.act != RRM_ACT_SIGN && d.act != RRM_ACT_LEAKY) return RRM_ERR_INVALID_ARG;
+    if (d.act == RRM_ACT_LEAKY && d.dtype != RRM_F32) return RRM_ERR_UNSUPPORTED;
     if (d.dtype == RRM_F32 && d.act == RRM_ACT_SIGN) return RRM_ERR_UNSUPPORTED;
     if (d.dtype != RRM_F32 && d.shift < 0 && d.act == RRM_ACT_RELU) return RRM_ERR_UNSUPPORTED;
     if (d.shift > 30) return RRM_ERR_INVALID_ARG;

@@ -692,6 +692,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                     if (PT == T_F32) {
                         x += res;
                         if (p.act_fn == RRM_ACT_RELU) x = x > 0 ? x : 0;
+                        else if (p.act_fn == RRM_ACT_LEAKY) x = x > 0 ? x : (pt)(0.1f * (float)x);
                     } else if (OT == T_I8) {
                         int iv = (int)x;
                         if (p.shift > 0) iv = (iv + (1 << (p.shift - 1))) >> p.shift;

@@ -69,7 +69,7 @@ def test_invalid_descriptions_are_rejected_before_any_device_work():
     cases = [
         (_desc(kind=7), INVALID), (_desc(dtype=9), DTYPE), (_desc(n=0), SHAPE), (_desc(c_out=0), SHAPE),
         (_desc(stride=0), SHAPE), (_desc(pad=3), SHAPE), (_desc(kh=11, kw=11, h=4, w=4, pad=0), SHAPE),
-        (_desc(kind=1, h=2), SHAPE), (_desc(act=5), INVALID), (_desc(act=2), UNSUPPORTED),
+        (_desc(kind=1, h=2), SHAPE), (_desc(act=5), INVALID), (_desc(act=2), UNSUPPORTED), (_desc(act=3, dtype=1, shift=4), UNSUPPORTED),
         (_desc(pool_k=3, pool_s=0), SHAPE), (_desc(pool_k=5, pool_s=2), UNSUPPORTED), (_desc(shift=40, dtype=1), INVALID),
         (_desc(variant=9), INVALID), (_desc(dtype=1, shift=-1, act=1), UNSUPPORTED),
     ]

@@ -150,6 +150,7 @@ def test_single_layer_cuda_core_variant(dtype, c_in, c_out, hw, k, s, p):
 
 @pytest.mark.parametrize("dtype,act,pool,shift", [
     ("f32", "relu", (3, 2, 0), -1), ("f32", "relu", (3, 2, 1), -1), ("f32", "none", (2, 2, 0), -1),
+    ("f32", "leaky", None, -1), ("f32", "leaky", (2, 2, 0), -1),
     ("i8", "relu", (3, 2, 0), 9), ("i8", "none", None, 10), ("i8", "sign", (3, 2, 0), -1), ("i8", "none", (3, 2, 1), -1),
     ("bin", "sign", None, -1), ("bin", "sign", (3, 2, 0), -1), ("bin", "none", (3, 2, 0), -1)])
 def test_single_layer_nonlinearities(dtype, act, pool, shift):
@@ -191,6 +192,18 @@ def test_small_stacks_every_frame(name):
     video = wl.moving_rect_video(frames=6, hw=hw, dtype=dt, seed=9, n=n, side=(12, 24),
                                  bg_redraw=0.02 if name == "resnet_i8" else 0.0)
     _run(specs, video, n=n, stats=True, keyframe_at=(4,))
+
+
+# ------------------------------------------------------------------ whole networks: FC layers inside a stack, VGG-16 shape
+@pytest.mark.parametrize("name", ["alexnet_full_i8", "alexnet_full_f32", "vgg16_i8", "vgg16_f32"])
+def test_second_workloads_every_frame(name):
+    dt = "i8" if name.endswith("i8") else "f32"
+    if name.startswith("alexnet_full"):
+        specs, hw = wl.alexnet_full(dt, hw=99, scale=8, classes=80), 99
+    else:
+        specs, hw = wl.vgg16_convs(dt, hw=64, scale=8), 64
+    video = wl.moving_rect_video(frames=5, hw=hw, dtype=dt, seed=12, side=(10, 20))
+    _run(specs, video, stats=True, keyframe_at=(3,))
 
 
 # ------------------------------------------------------------------ full-size configs, sampled frames

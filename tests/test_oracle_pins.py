@@ -378,3 +378,13 @@ def test_aecs_polynomial():
     mu = [0.5, -1.0, 2.0, 0.25, -0.125]
     for e in (0.0, 0.3, 2.0):
         assert abs(orc.aecs_predict(mu, e) - float(np.polyval(mu[::-1], e))) < 1e-12
+
+
+def test_leaky_relu_matches_the_library_routine():
+    import torch
+    s = wl.LayerSpec("conv", "f32", 2, 5, 5, 3, 1, 1, 1, 0, act="leaky", src=0)
+    P = np.random.default_rng(2).standard_normal((1, 3, 5, 5))
+    got = orc.nonlinearity(s, P)
+    want = torch.nn.functional.leaky_relu(torch.from_numpy(P), float(np.float32(0.1))).numpy()
+    np.testing.assert_allclose(got, want, atol=1e-15)
+    assert (got[P < 0] < 0).all() and (got[P > 0] == P[P > 0]).all()

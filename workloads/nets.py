@@ -212,3 +212,39 @@ def xnor_alexnet_convs(seed=5, hw=227, scale=1):
     L.append(LayerSpec("conv", "bin", c[2], h, w, c[3], 3, 3, 1, 1, "sign", None, -1, name="conv4"))
     L.append(LayerSpec("conv", "bin", c[3], h, w, c[4], 3, 3, 1, 1, "none", (3, 2, 0), -1, name="conv5"))
     return _fill(_resolve_src(L), seed)
+
+
+# ---------------------------------------------------------------- whole networks (second workloads)
+def alexnet_full(dtype="i8", seed=6, hw=227, scale=1, classes=1000):
+    """conv1..conv5 as in alexnet_convs plus fc6, fc7, fc8.  An FC layer after a convolution is the
+    convolution whose filter covers the whole map (fc6: 6x6 over the 6x6x256 map); fc7 and fc8 are 1x1
+    convolutions of a 1x1 map."""
+    L = alexnet_convs(dtype, seed=seed, hw=hw, scale=scale)
+    sh = 0 if dtype == "i8" else -1
+    _, (h, w) = out_hw(L[-1])
+    c = L[-1].c_out
+    f = max(8, 4096 // scale)
+    L.append(LayerSpec("conv", dtype, c, h, w, f, h, w, 1, 0, "relu", None, sh, name="fc6"))
+    L.append(LayerSpec("conv", dtype, f, 1, 1, f, 1, 1, 1, 0, "relu", None, sh, name="fc7"))
+    L.append(LayerSpec("conv", dtype, f, 1, 1, max(4, classes // scale), 1, 1, 1, 0, "none", None, -1 if dtype == "i8" else sh,
+                       name="fc8"))
+    for s in L:
+        s.src = -1
+    return _fill(_resolve_src(L), seed)
+
+
+def vgg16_convs(dtype="i8", seed=7, hw=224, scale=1):
+    """The 13 convolutions of a VGG-16-shaped stack (3x3, pad 1, ReLU; 2x2 stride-2 max-pool after
+    conv 2, 4, 7, 10 and 13): the third model of the paper's Table 2."""
+    plan = [(64, False), (64, True), (128, False), (128, True), (256, False), (256, False), (256, True),
+            (512, False), (512, False), (512, True), (512, False), (512, False), (512, True)]
+    sh = 0 if dtype == "i8" else -1
+    L = []
+    c_in, h, w = 3, hw, hw
+    for i, (c, pool) in enumerate(plan):
+        c = max(4, c // scale)
+        L.append(LayerSpec("conv", dtype, c_in, h, w, c, 3, 3, 1, 1, "relu", (2, 2, 0) if pool else None, sh,
+                           name=f"conv{i + 1}"))
+        _, (h, w) = out_hw(L[-1])
+        c_in = c
+    return _fill(_resolve_src(L), seed)
