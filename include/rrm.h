@@ -160,7 +160,12 @@ int rrm_net_destroy(rrm_net* net);
 
 /* Dense pass over the whole stack that resets every layer's state. out_dev may be NULL. */
 int rrm_net_keyframe(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
-/* Algorithm 1, one iteration of the frame loop; out_dev receives the last tensor. */
+/* Algorithm 1, one iteration of the frame loop; out_dev receives the last tensor.  On a stack of at least
+ * 1 GMAC per frame whose layers all ask for RRM_VARIANT_AUTO the library reads back (asynchronously) how many
+ * projection pixels the last delta frame had to update; while that share, weighted by the layers' MACs, is
+ * 75 % or more it evaluates frames densely instead (a precise inference that replaces the state: the same
+ * results), and measures again with a delta frame every 16th frame.  rrm_net_get_stats reports such a frame
+ * with variant RRM_VARIANT_DENSE and its counters as -1 (nothing was counted). */
 int rrm_net_step(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
 /* Dense evaluation of the stack without touching the RRM state. */
 int rrm_net_dense(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);

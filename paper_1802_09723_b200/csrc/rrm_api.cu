@@ -124,6 +124,8 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     for (auto& L : net->layers) cleared += (size_t)ceil_div(L.opixels(), 32) * 4;
     cleared = (cleared + 15) & ~(size_t)15;
     const size_t counters_off = cleared;
+    net->counters_off = counters_off;
+    net->counters_bytes = net->tensors.size() * 32 + net->layers.size() * 16;
     cleared += net->tensors.size() * 32 + net->layers.size() * 16;
     RRM_TRY(dev_alloc(net, &net->cleared, cleared));
     net->cleared_bytes = cleared;
@@ -145,6 +147,17 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     }
     RRM_TRY(dev_alloc(net, (void**)&net->aecs, (size_t)(1 + n_layers) * 8));
     for (int l = 0; l < n_layers; ++l) RRM_TRY(conv_layer_create(net, net->layers[l], W[l], B ? B[l] : nullptr));
+    {
+        // dense evaluation of high-activity frames: only where a frame is real work (>= 1 GMAC), so that the
+        // per-layer counters stay available on small stacks, and only if no layer pins its variant
+        long long macs = 0;
+        bool all_auto = true;
+        for (auto& L : net->layers) {
+            macs += (long long)L.opixels() * L.d.c_out * L.d.c_in * L.d.kh * L.d.kw;
+            all_auto = all_auto && L.d.variant == RRM_VARIANT_AUTO;
+        }
+        net->auto_switch = all_auto && macs >= 1000000000ll;
+    }
     {
         const char* e = getenv("RRM_NO_GRAPH");
         net->graph_off = e && e[0] == '1';
@@ -169,6 +182,7 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
 }
 
 int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
+int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
 
 // Captures one of the per-frame launch sequences into a graph (on a private stream: a capture cannot
 // start on the legacy default stream) so that later frames cost one graph launch on the host.
@@ -200,11 +214,67 @@ void drop_graphs(rrm_net* net)
     }
 }
 
+constexpr double DENSE_SWITCH_ACTIVITY = 0.75;   // MAC-weighted share of projection pixels to update, from which on a frame goes dense
+constexpr int DENSE_SWITCH_REPROBE = 15;         // dense frames in a row before a delta frame measures the activity again
+
+// Copies the step's counters to pinned memory behind the work on the stream (never waited for).
+int activity_read_back(rrm_net* net, cudaStream_t st)
+{
+    if (net->act_pending) return RRM_OK;
+    if (!net->act_host && cudaMallocHost(reinterpret_cast<void**>(&net->act_host), net->counters_bytes) != cudaSuccess) { cudaGetLastError(); return RRM_OK; }
+    if (!net->act_ev && cudaEventCreateWithFlags(&net->act_ev, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return RRM_OK; }
+    RRM_CUDA_TRY(cudaMemcpyAsync(net->act_host, reinterpret_cast<char*>(net->cleared) + net->counters_off, net->counters_bytes,
+                                 cudaMemcpyDeviceToHost, st));
+    RRM_CUDA_TRY(cudaEventRecord(net->act_ev, st));
+    net->act_pending = true;
+    return RRM_OK;
+}
+
+void activity_poll(rrm_net* net)
+{
+    if (!net->act_pending || cudaEventQuery(net->act_ev) != cudaSuccess) { cudaGetLastError(); return; }
+    net->act_pending = false;
+    double num = 0, den = 0;
+    const size_t base = net->tensors.size() * 32;
+    for (size_t l = 0; l < net->layers.size(); ++l) {
+        const Layer& L = net->layers[l];
+        int oc = 0;
+        std::memcpy(&oc, net->act_host + base + l * 16 + 8, 4);
+        const double macs = (double)L.opixels() * L.d.c_out * L.d.c_in * L.d.kh * L.d.kw;
+        num += macs * oc / (double)L.opixels();
+        den += macs;
+    }
+    net->activity = den > 0 ? num / den : -1.0;
+}
+
 int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
 {
     if (!net || !frame) return RRM_ERR_INVALID_ARG;
     net->last_stream = st;
     if (net->layers[0].fc_fused) return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
+    const bool is_step = !dense && !stateless;
+    if (is_step) {
+        // the variant of this frame from the measured activity of the last delta frame (temporal coherence):
+        // a dense pass that replaces the state gives the same results, so the switch is invisible in the outputs
+        net->last_step_dense = false;
+        if (net->auto_switch && net->eps == 0.f) {
+            activity_poll(net);
+            if (net->activity >= DENSE_SWITCH_ACTIVITY && net->dense_streak < DENSE_SWITCH_REPROBE) {
+                ++net->dense_streak;
+                net->last_step_dense = true;
+                dense = true;
+            } else {
+                net->dense_streak = 0;
+            }
+        }
+    }
+    const int s_run = run_sequence(net, frame, out, st, dense, stateless);
+    if (s_run == RRM_OK && is_step && !dense && net->auto_switch) RRM_TRY(activity_read_back(net, st));
+    return s_run;
+}
+
+int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
+{
     if (!net->graph_off) {
         const int kind = !dense ? 0 : (stateless ? 2 : 1);
         if (!net->exec[kind]) {
@@ -303,6 +373,8 @@ int rrm_net_destroy(rrm_net* net)
         if (L.seq_stat_host) cudaFreeHost(L.seq_stat_host);
     }
     drop_graphs(net);
+    if (net->act_ev) cudaEventDestroy(net->act_ev);
+    if (net->act_host) cudaFreeHost(net->act_host);
     if (net->cap_stream) cudaStreamDestroy(net->cap_stream);
     for (void* p : net->allocs) cudaFree(p);
     delete net;
@@ -466,6 +538,12 @@ int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
         h->active_out_pixels = tot[0] ? (int64_t)frames * d.n : 0;
         h->active_macs = (int64_t)tot[0] * d.c_out;
         h->variant = L.seq_last_T > 0 ? L.seq_last_variant : RRM_VARIANT_GATHER;
+        return RRM_OK;
+    }
+    if (net->last_step_dense) {                  // the most recent step was evaluated densely: nothing was counted
+        h->nnz_elems = h->active_in_pixels = h->active_out_pixels = h->active_macs = -1;
+        h->in_pixels = net->tensors[d.src].pixels();
+        h->variant = RRM_VARIANT_DENSE;
         return RRM_OK;
     }
     const Tensor& in = net->tensors[d.src];

@@ -129,6 +129,16 @@ struct rrm_net {
     void* frame_buf = nullptr;        // the step's input frame, boundary layout
     void* out_buf = nullptr;          // the step's last tensor, boundary layout
     bool graph_off = false;           // RRM_NO_GRAPH=1: launch kernel by kernel (debugging)
+    // measured activity of the last delta step, read back without stalling the stream: when nearly every
+    // projection pixel has to be updated anyway, the next frames are evaluated densely (same results, less work)
+    size_t counters_off = 0, counters_bytes = 0;   // the counters inside the cleared arena
+    unsigned char* act_host = nullptr;        // pinned copy of the counters
+    cudaEvent_t act_ev = nullptr;
+    bool act_pending = false;
+    double activity = -1.0;                   // MAC-weighted fraction of projection pixels updated; < 0: unknown
+    int dense_streak = 0;                     // dense frames since the last measured delta frame
+    bool last_step_dense = false;             // the most recent rrm_net_step was evaluated densely
+    bool auto_switch = false;                 // every layer asks for RRM_VARIANT_AUTO and the net is large enough
     float eps = 0.f;                  // Sec. 3.4: fp32 delta entries below it are truncated (0: exact)
     double* aecs = nullptr;           // [1 + layers]: accumulated truncated value e_t (Eq. 7), then the last step's l2 per layer
     std::vector<void*> allocs;        // everything to free

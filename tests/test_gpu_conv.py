@@ -206,6 +206,28 @@ def test_second_workloads_every_frame(name):
     _run(specs, video, stats=True, keyframe_at=(3,))
 
 
+def test_large_stack_goes_dense_while_nearly_every_pixel_changes():
+    """Background noise makes every projection pixel change: after the first measured delta frame the frames
+    are evaluated densely (same results), with a delta frame every 16th frame to measure again."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8")
+    video = wl.moving_rect_video(frames=20, hw=227, dtype="i8", seed=33, n=2, bg_redraw=0.10)
+    net = rrm.net_from_specs(specs, n=2)
+    out = net.new_output()
+    variants = []
+    for t in range(20):
+        net.step(dev(video[t]), out)
+        st = net.stats(1)                     # synchronises, so the next call sees this frame's counters
+        variants.append(st["variant"])
+        assert (st["nnz_elems"] == -1) == (st["variant"] == 3)
+        if t in (0, 1, 2, 16, 19):
+            _compare(specs, net, video[t], t)
+    assert variants[0] == 2                               # the first frame (every pixel new) is a measured delta frame
+    assert all(v == 3 for v in variants[1:16])            # dense while the measured activity is high
+    assert variants[16] == 2 and variants[17] == 3        # one delta frame measures again
+    net.close()
+
+
 # ------------------------------------------------------------------ full-size configs, sampled frames
 def test_cfg3_alexnet_fp32_full_size():
     specs = wl.alexnet_convs("f32")
