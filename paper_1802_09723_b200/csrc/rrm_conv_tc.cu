@@ -254,6 +254,18 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             // int8 rows are copied as they are: asynchronous 16-byte copies (zero-filled where the input
             // pixel is unusable); a slab is handed to the tensor core TC_LAG slabs later, when its copies landed
             const unsigned char* Ab = reinterpret_cast<const unsigned char*>(p.A);
+            // this thread's 8 rows stay the same for the whole K loop: their tap masks, source offsets and
+            // shared-memory offsets live in registers, so a slab costs a few instructions per 16-byte copy
+            unsigned long long rm0[8], rm1[8];
+            int src_row[8];
+            uint32_t dst_row[8];
+            #pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = warp * 32 + i * 4 + rsub;
+                rm0[i] = S->rmask[r][0]; rm1[i] = S->rmask[r][1];
+                src_row[i] = S->pix0[r] * p.row_units;       // fits: a tensor holds fewer than 2^31 values
+                dst_row[i] = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
+            }
             for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
                 const int stage = it % TC_STAGES;
                 if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
@@ -280,15 +292,14 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 const int kc = ks * 4 + (piece >> 1);       // this lane's 32-byte chunk of K
                 const int tap = kc / cpt, cc = kc - tap * cpt;
                 const int ky = tap / p.kw, kx = tap - ky * p.kw;
-                const int tap_off = ky * p.w + kx;
-                const int byte_off = cc * 32 + (piece & 1) * 16;
+                const int slab_off = (ky * p.w + kx) * p.row_units + cc * 32 + (piece & 1) * 16;   // same for the 8 rows
+                const bool tap_ok = tap < p.taps, hi = tap >= 64;
+                const int sh = tap & 63;
                 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const int r = warp * 32 + i * 4 + rsub;
-                    const bool use = tap < p.taps && ((S->rmask[r][tap >> 6] >> (tap & 63)) & 1ull);
-                    const unsigned char* src = use ? Ab + (size_t)(S->pix0[r] + tap_off) * p.row_units + byte_off : Ab;
-                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
-                    cp_async16(As + off, src, use ? 16u : 0u);
+                    const bool use = tap_ok && (((hi ? rm1[i] : rm0[i]) >> sh) & 1ull);
+                    const unsigned char* src = use ? Ab + (src_row[i] + slab_off) : Ab;
+                    cp_async16(As + dst_row[i], src, use ? 16u : 0u);
                 }
                 }
                 cp_async_commit();
@@ -308,23 +319,34 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             const uint32_t* Cu = reinterpret_cast<const uint32_t*>(p.A);
             const uint32_t* Nu = reinterpret_cast<const uint32_t*>(p.Anew);
             uint32_t nw[8], cw[8];
+            unsigned long long bm0[8], bm1[8];               // per-row tap masks, word offsets and store offsets
+            int bsrc[8];
+            uint32_t bdst[8];
+            #pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = warp * 32 + i * 4 + rsub;
+                bm0[i] = S->rmask[r][0]; bm1[i] = S->rmask[r][1];
+                bsrc[i] = S->pix0[r] * p.row_units;
+                bdst[i] = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
+            }
             unsigned usemask = 0;
             int half_valid = 0;
             auto fetch = [&](int ks) {
                 const int kc = ks * 4 + (piece >> 1);
                 const int tap = kc / cpt, cc = kc - tap * cpt;
                 const int ky = tap / p.kw, kx = tap - ky * p.kw;
-                const int tap_off = ky * p.w + kx;
+                const int slab_off = (ky * p.w + kx) * p.row_units + cc;
+                const bool tap_ok = tap < p.taps, hi = tap >= 64;
+                const int sh = tap & 63;
                 const int c_base = cc * 32 + (piece & 1) * 16;
                 half_valid = c_base >= p.c_in ? 0 : (c_base + 16 > p.c_in ? (int)((1u << (p.c_in - c_base)) - 1u) : 0xffff);
                 usemask = 0;
                 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const int r = warp * 32 + i * 4 + rsub;
-                    const bool use = tap < p.taps && ((S->rmask[r][tap >> 6] >> (tap & 63)) & 1ull);
+                    const bool use = tap_ok && (((hi ? bm1[i] : bm0[i]) >> sh) & 1ull);
                     nw[i] = 0; cw[i] = 0;
                     if (use) {
-                        const size_t wi = (size_t)(S->pix0[r] + tap_off) * p.row_units + cc;
+                        const int wi = bsrc[i] + slab_off;
                         nw[i] = Nu[wi];
                         if (!DENSE) cw[i] = Cu[wi];
                         usemask |= 1u << i;
@@ -348,7 +370,6 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 const int shift = (piece & 1) * 16;
                 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const int r = warp * 32 + i * 4 + rsub;
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (use_cur >> i & 1u) {
                         const uint32_t nb = n_cur[i] >> shift;
@@ -361,8 +382,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                         v.z = spread4(pos >> 8) * pm + spread4(neg >> 8) * nm;
                         v.w = spread4(pos >> 12) * pm + spread4(neg >> 12) * nm;
                     }
-                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4*>(As + off) = v;
+                    *reinterpret_cast<uint4*>(As + bdst[i]) = v;
                 }
                 fence_async_smem();                          // generic-proxy stores -> visible to the tensor core
                 mbar_arrive(smem_u32(&S->full[stage]));
