@@ -112,6 +112,9 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     }
     RRM_TRY(dev_alloc(net, (void**)&net->errw, 16));
     if (fused) return RRM_OK;
+    // the import kernel turns 32 pixels x all channels of the frame around in shared memory
+    if (net->tensors[0].dtype != T_BIN && net->tensors[0].cs != 4 &&
+        (size_t)32 * (net->tensors[0].cs + 1) * net->tensors[0].unit_bytes > 200 * 1024) return RRM_ERR_UNSUPPORTED;
 
     // tensors
     size_t cleared = 0;

@@ -2,13 +2,22 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <cstdio>
+#include <cstdlib>
 #include <vector>
 #include "../../include/rrm.h"
+
+// RRM_DEBUG=1 in the environment: a failing CUDA call is named on stderr (call site and error string)
+inline void rrm_note_cuda_error(cudaError_t e, const char* file, int line)
+{
+    static const bool on = getenv("RRM_DEBUG") != nullptr;
+    if (on) fprintf(stderr, "rrm: %s:%d: %s\n", file, line, cudaGetErrorString(e));
+}
 
 #define RRM_CUDA_TRY(expr)                                   \
     do {                                                     \
         cudaError_t e__ = (expr);                            \
-        if (e__ != cudaSuccess) return RRM_ERR_CUDA;         \
+        if (e__ != cudaSuccess) { rrm_note_cuda_error(e__, __FILE__, __LINE__); return RRM_ERR_CUDA; } \
     } while (0)
 
 #define RRM_TRY(expr)                                        \
@@ -90,6 +99,9 @@ struct Layer {
     int8_t* tc_Wimg = nullptr;              // [n_tiles][slabs][bn * 128] shared-memory images of the filter tiles
     int tc_kpp = 0;                         // K bytes per tap (padded channels per pixel)
     int tc_bn = 0, tc_ntiles = 0, tc_slabs = 0;
+    // few-row dense FC on the tensor cores (weights as the M operand, K split over CTAs)
+    int32_t* ft_acc = nullptr;              // [rows][tiles * 128] partial sums, zero between launches
+    unsigned* ft_arrive = nullptr;          // [tiles] arrival counters, zero between launches
     // chunk-of-frames form of the fused FC path
     int32_t* seq_dP = nullptr;              // [seq_cap][n][c_out] per-frame projection deltas
     unsigned* seq_stat = nullptr;           // [seq_cap * n][2] per frame and stream: non-zeros, active groups of 32
@@ -159,6 +171,11 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
                cudaStream_t st);
 int fc_seq_stats(Layer& L, unsigned long long* nnz, unsigned long long* groups);
 int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool stateless, cudaStream_t st);
+
+// ---- rrm_fc_tc.cu
+int fc_tc_create(rrm_net* net, Layer& L);
+bool fc_tc_usable(const Layer& L, int rows);
+int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, bool stateless, unsigned* stat, cudaStream_t st);
 
 // ---- rrm_conv_tc.cu
 bool conv_tc_eligible(const rrm_net* net, const Layer& L);

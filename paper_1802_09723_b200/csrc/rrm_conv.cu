@@ -924,6 +924,10 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
         } else {
             auto kd = import_nchw_kernel<int8_t, true>;
             auto kn = import_nchw_kernel<int8_t, false>;
+            if (smem > 48 * 1024) {
+                cudaFuncSetAttribute(kd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            }
             if (delta) kd<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, (int8_t*)T.D, T.act, T.pnnz,
                                                    T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, 0.f, nullptr);
             else kn<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, nullptr, nullptr, nullptr, nullptr,

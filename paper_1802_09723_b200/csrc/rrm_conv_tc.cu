@@ -21,15 +21,14 @@
 // word and the CTA leaves through the common exit, which frees its tensor memory.
 #include "rrm_common.cuh"
 #include "rrm_rows.cuh"
+#include "rrm_tc.cuh"
 
 namespace rrm {
 
-constexpr int TC_M = 128;
 constexpr int TC_SLAB = 128;                  // bytes of K per stage
 constexpr int TC_STAGES = 3;
 constexpr int TC_THREADS = 192;               // warps 0-3: A producers + epilogue, warp 4: MMA, warp 5: B loader
 constexpr int TC_MAX_BN = 128;
-constexpr unsigned TC_SPIN_LIMIT = 1u << 20;
 
 struct TcParams {
     const void* A;            // int8: delta rows (delta) or values (dense); binary: changed bits (delta) / unused
@@ -50,74 +49,6 @@ struct TcParams {
     int ksplit;               // gridDim.z
 };
 
-// ---- raw PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (unsigned i = 0; i < TC_SPIN_LIMIT; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024
-// bytes apart (the tile starts on a 1024-byte boundary).
-__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);            // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                             // leading byte offset (unused with swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                   // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                             // 128-byte swizzle
-    return d;
-}
-// Instruction descriptor: int8 x int8 -> int32, both operands K-major, M = 128, N = bn.
-__device__ __forceinline__ uint32_t tc_instr_desc(int bn)
-{
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_M >> 4) << 24);
-}
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
 // byte i of the result = bit i of the low nibble of x (0 or 1)
 __device__ __forceinline__ uint32_t spread4(uint32_t x) { return ((x & 0xfu) * 0x00204081u) & 0x01010101u; }
 
@@ -135,13 +66,6 @@ constexpr size_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + sizeof(TcSm
 constexpr int TC_LAG = TC_STAGES - 1;         // slabs whose asynchronous copies may still be in flight
 constexpr int TC_ROW_WORDS = TC_MAX_BN + 4;   // epilogue row buffers: 16-byte aligned rows, staggered over the banks
 static_assert((size_t)TC_M * TC_ROW_WORDS * 4 <= TC_STAGES * TC_STAGE_BYTES, "epilogue rows reuse the stage buffers");
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <bool BIN, bool DENSE>
 __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)

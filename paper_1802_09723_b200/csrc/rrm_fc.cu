@@ -490,7 +490,10 @@ int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_
     L.fc_fused = true;
     RRM_TRY(fc_seq_create(net, L));
     // the dense path (keyframe, rrm_dense) runs on the tensor cores when the inputs are whole 32-byte K chunks
-    if (C % 32 == 0 && L.d.variant != RRM_VARIANT_GATHER) RRM_TRY(conv_tc_create(net, L, W_dev));
+    if (C % 32 == 0 && L.d.variant != RRM_VARIANT_GATHER) {
+        RRM_TRY(conv_tc_create(net, L, W_dev));
+        RRM_TRY(fc_tc_create(net, L));
+    }
     return RRM_OK;
 }
 
@@ -500,8 +503,8 @@ int fc_fused_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, bool de
 {
     const int C = L.d.c_in, K = L.d.c_out, n = L.d.n;
     const int slices = ceil_div(K, FC_OW);
-    // (a handful of rows is served faster by the gather kernel with every entry active)
-    if (dense && L.tc_ready && n >= 4) return fc_dense_tc_run(net, L, X_dev, Y_dev, 1, stateless, st);
+    // (without the few-row tensor-core form a handful of rows is served faster by the gather kernel with every entry active)
+    if (dense && L.tc_ready && (n >= 4 || fc_tc_usable(L, n))) return fc_dense_tc_run(net, L, X_dev, Y_dev, 1, stateless, st);
     FcParams p;
     p.xt = reinterpret_cast<const int8_t*>(X_dev);
     p.Wt = L.Wt;

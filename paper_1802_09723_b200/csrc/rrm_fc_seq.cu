@@ -341,6 +341,9 @@ __global__ void __launch_bounds__(SQ_THREADS) fc_count_kernel(const int8_t* __re
 // From this measured non-zero fraction of the previous chunk on, the next chunk is evaluated densely on the
 // tensor cores (W read once for all frames) instead of by column gather (measured break-even on fc6: ~7 %).
 constexpr double SQ_DENSE_SWITCH = 0.08;
+// ... and for chunks of few rows (one launch that reads W once): rows x non-zero fraction from which on the dense
+// evaluation wins (measured break-even on fc6, 32 rows: 2.2 % non-zeros)
+constexpr double SQ_DENSE_SWITCH_ROWS = 0.75;
 
 // Copies the chunk's counters to pinned host memory behind the work already on the stream.
 static int seq_read_back(Layer& L, int rows, cudaStream_t st)
@@ -435,14 +438,22 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
             L.seq_ev_pending = false;
         }
         cudaGetLastError();                                  // cudaErrorNotReady from the query is not an error
+        // (few rows go through the single-launch form, whose cost is that of reading W once: it wins as soon as
+        // the rows' gathered columns add up to about that many bytes)
         const bool use_dense = L.tc_ready && L.d.variant == RRM_VARIANT_AUTO && (long long)T * n >= 8 &&
-                               L.seq_density >= SQ_DENSE_SWITCH;
+                               (fc_tc_usable(L, T * n) ? L.seq_density * T * n >= SQ_DENSE_SWITCH_ROWS
+                                                       : L.seq_density >= SQ_DENSE_SWITCH);
         L.seq_last_T = T;
         L.seq_last_variant = use_dense ? RRM_VARIANT_DENSE : RRM_VARIANT_GATHER;
         if (use_dense) {
             // the results are the same integers: P_t = b + W X_t for every frame, state := last frame
-            fc_count_kernel<<<T * n, SQ_THREADS, 0, st>>>(reinterpret_cast<const int8_t*>(X_dev), L.xs[L.xs_cur], L.seq_stat, n, C);
-            RRM_TRY(fc_dense_tc_run(net, L, X_dev, Y_dev, T, false, st));
+            if (fc_tc_usable(L, T * n)) {
+                // few rows: one launch streams W once, and its idle warps count the delta entries meanwhile
+                RRM_TRY(fc_tc_run(net, L, X_dev, Y_dev, T * n, false, L.seq_stat, st));
+            } else {
+                fc_count_kernel<<<T * n, SQ_THREADS, 0, st>>>(reinterpret_cast<const int8_t*>(X_dev), L.xs[L.xs_cur], L.seq_stat, n, C);
+                RRM_TRY(fc_dense_tc_run(net, L, X_dev, Y_dev, T, false, st));
+            }
             return seq_read_back(L, T * n, st);
         }
         p.xprev = L.xs[L.xs_cur];
@@ -508,6 +519,8 @@ __global__ void fc_dense_finish_kernel(const int32_t* __restrict__ Pd, void* Y, 
 int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool stateless, cudaStream_t st)
 {
     const int C = L.d.c_in, K = L.d.c_out, n = L.d.n;
+    // a few rows: one launch that streams W once and finishes the outputs itself
+    if (fc_tc_usable(L, T * n)) return fc_tc_run(net, L, X_dev, Y_dev, T * n, stateless, nullptr, st);
     RRM_TRY(seq_ensure(net, L, T));
     Layer Lt = L;                                            // the M-row problem as a 1x1 convolution
     Lt.d.n = T * n; Lt.d.h = Lt.d.w = 1; Lt.oh = Lt.ow = 1;

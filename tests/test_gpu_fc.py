@@ -248,3 +248,52 @@ def test_fc6_dense_chunks_take_over_at_high_measured_density():
     layer.step(frames[32], Y1)                    # the state after dense chunks is the recurrence's state
     np.testing.assert_array_equal(Y1.cpu().numpy(), orc.dense_forward([spec], seq[32])[0][1])
     layer.close()
+
+
+# ------------------------------------------------------------------ few-row dense FC on the tensor cores
+@pytest.mark.parametrize("c_in,c_out,shift,act,n,T", [
+    (9216, 4096, -1, "none", 1, 1),       # one row: the keyframe / rrm_dense of the fc6 shape
+    (9216, 4096, -1, "none", 1, 32),      # one full launch
+    (9216, 4096, -1, "none", 3, 17),      # 51 rows: two launches, the state rows straddle nothing
+    (9216, 4096, -1, "none", 5, 7),       # 35 rows: the last frame's rows straddle the two launches
+    (4096, 1008, 7, "relu", 2, 9),        # outputs not a multiple of 128, int8 outputs through f
+    (4096, 1000, 7, "relu", 2, 9),        # outputs not a multiple of 16: the general layer path, frame by frame
+    (160, 528, 6, "relu", 3, 5),          # K smaller than one share per SM, ragged tiles
+    (2048, 1024, -1, "none", 4, 16),      # 64 rows in one launch
+])
+def test_fc_dense_few_rows_on_tensor_cores(c_in, c_out, shift, act, n, T):
+    """Dense chunks (stateless and keyframe-like) equal Eq. 3 row by row; the state after a stateful dense
+    evaluation is that of the last frame, so a delta step from it is exact."""
+    rrm = _rrm()
+    rng = np.random.default_rng(c_in + c_out + n + T)
+    spec = LayerSpec("fc", "i8", c_in, 1, 1, c_out, act=act, shift=shift, src=0)
+    spec.weight = rng.integers(-127, 128, size=(c_out, c_in, 1, 1)).astype(np.int8)
+    spec.bias = rng.integers(-500, 501, size=c_out).astype(np.int32)
+    seq = wl.fc_run_sequence(frames=T + 1, c_in=c_in, rho=0.3, run=8, seed=c_in + T, n=n)
+    layer = rrm.layer_from_spec(spec, n=n)
+    frames = dev(seq)
+    want = [orc.dense_forward([spec], seq[t]) for t in range(T + 1)]
+    # stateless dense chunk, twice (the scratch accumulators must come back zeroed)
+    for _ in range(2):
+        Y = layer.new_output(frames=T)
+        layer.dense_seq(frames[:T], Y, T)
+        for t in range(T):
+            np.testing.assert_array_equal(Y[t].cpu().numpy().astype(np.int64), want[t][0][1].astype(np.int64), err_msg=f"frame {t}")
+    # a chunk dense enough to be evaluated densely with state: first chunk measures, second one switches
+    Y = layer.new_output(frames=T)
+    layer.step_seq(frames[:T], Y, T)
+    layer.stats(0)
+    layer.step_seq(frames[:T], Y, T)
+    for t in range(T):
+        np.testing.assert_array_equal(Y[t].cpu().numpy().astype(np.int64), want[t][0][1].astype(np.int64), err_msg=f"frame {t}")
+    np.testing.assert_array_equal(layer.projection(0).cpu().numpy().astype(np.int64), want[T - 1][1][0])
+    Y1 = layer.new_output()
+    layer.step(frames[T], Y1)
+    np.testing.assert_array_equal(Y1.cpu().numpy().astype(np.int64), want[T][0][1].astype(np.int64))
+    # keyframe + dense of single frames
+    layer.keyframe(frames[0], Y1)
+    np.testing.assert_array_equal(Y1.cpu().numpy().astype(np.int64), want[0][0][1].astype(np.int64))
+    layer.step(frames[1], Y1)
+    np.testing.assert_array_equal(Y1.cpu().numpy().astype(np.int64), want[1][0][1].astype(np.int64))
+    assert layer.stats(0)["error_word"] == 0
+    layer.close()
