@@ -67,9 +67,10 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-def committed_traffic(rho):
-    """DRAM bytes per launch of the chunk delta-FC kernel from the committed ncu summary, if present."""
-    p = os.path.join(ROOT, "profiles", "fc_seq_fc6_chunk32.txt")
+def committed_traffic(kernel, rho):
+    """DRAM bytes per launch of the chunk kernel that ran, from its committed ncu summary, if present."""
+    p = os.path.join(ROOT, "profiles", {"fc_seq_kernel": "fc_seq_fc6_chunk32.txt",
+                                        "fc_tc_kernel": "fc_tc_fc6_chunk32.txt"}[kernel])
     if not os.path.exists(p):
         return None
     for line in open(p):
@@ -312,10 +313,10 @@ def main():
     def reduce_max(ms):
         return max_over_ranks(ms, world, "cuda")
 
-    def make(rho, n=1):
+    def make(rho, n=1, variant="auto"):
         """Layer + the endless back-and-forth walk over the 32-frame sequence, laid out so that chunk k
         is rows [k*T, (k+1)*T) of one device array (whole number of periods, so it wraps seamlessly)."""
-        desc = rrm.desc_from_spec(spec, n=n)
+        desc = rrm.desc_from_spec(spec, n=n, variant=variant)
         layer = rrm.Net([desc], [W], [B])
         seq = wl.fc_run_sequence(frames=FRAMES, rho=rho, seed=21 + rank, n=n)
         total = period * T // np.gcd(period, T)
@@ -384,6 +385,14 @@ def main():
         # per frame: gathered weight columns + read/modify/write of P + output + X_t, snapshot read, snapshot write
         return nnz_mean * C_OUT + 8 * C_OUT + 4 * C_OUT + 3 * C_IN
 
+    def dense_chunk_bytes(frames):
+        # the dense evaluation of a chunk: W once, the frames, outputs, stored projection, snapshot
+        return C_IN * C_OUT + (frames + 1) * C_IN + frames * 4 * C_OUT + 4 * C_OUT
+
+    EVAL = {1: "column gather", 3: "dense on the tensor cores, W read once (rows x measured density of the previous "
+                                   "chunk >= 0.75)"}
+    KERNEL = {1: "fc_seq_kernel", 3: "fc_tc_kernel"}
+
     def chunk_cold_bytes(uniq_cols, frames):
         # what one chunk launch must fetch with a cold L2: every distinct column once, the frames, per-frame
         # projection deltas (write + read) and outputs, the stored projection
@@ -400,8 +409,9 @@ def main():
     fps = whole_job_rate(T, ms, world)
     bytes_launch = frame_bytes(nnz_mean) * T
     achieved = bytes_launch / (ms * 1e-3) / 1e9
-    achieved_unique = chunk_cold_bytes(uniq_mean, T) / (ms * 1e-3) / 1e9
     st = layer.stats(0)
+    main_variant = st["variant"]
+    own_bytes = dense_chunk_bytes(T) if main_variant == 3 else chunk_cold_bytes(uniq_mean, T)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     nchunks = walk.shape[0] // T
@@ -427,22 +437,28 @@ def main():
             L2, sq, wk, wd, nz, un = make(rho)
             fr = [torch.from_numpy(sq[t]).cuda() for t in range(FRAMES)]
             c_ms = timed_chunks(L2, sq, wd, 124, 10, cold=True)
-            variant = {1: "column gather", 3: "dense on tensor cores (previous chunk's measured density >= 8 %)"}.get(
-                L2.stats(0)["variant"], "?")
+            variant = EVAL.get(L2.stats(0)["variant"], "?")
             w_ms = timed_chunks(L2, sq, wd, 124, 10, cold=False)
             d_ms = timed_chunks(L2, sq, wd, 31, 3, cold=True, dense=True)
             s_ms = timed_single(L2, sq, fr, 310, 31, cold=True)
             sd_ms = timed_single(L2, sq, fr, 124, 10, cold=True, dense=True)
+            LG = make(rho, variant="gather")[0]            # the column-gather kernel whatever the density
+            g_ms = timed_chunks(LG, sq, wd, 124, 10, cold=True)
+            LG.close()
             by_rho[f"{rho:g}"] = {
                 "nnz_mean_per_frame": nz, "distinct_columns_per_chunk": un, "chunk_evaluation": variant,
                 "chunk_cold_us": c_ms * 1e3, "chunk_warm_us": w_ms * 1e3, "dense_chunk_cold_us": d_ms * 1e3,
+                "gather_chunk_cold_us": g_ms * 1e3,
                 "fps_cold": T * 1e3 / c_ms, "gmacs_dense_equiv_cold": T * DENSE_MACS / c_ms / 1e6,
-                "speedup_vs_own_dense_chunk": d_ms / c_ms,
+                "speedup_vs_own_dense_chunk": d_ms / c_ms, "gather_speedup_vs_own_dense_chunk": d_ms / g_ms,
                 "roofline_frac_per_frame_bytes": frame_bytes(nz) * T / (c_ms * 1e-3) / 1e9 / peak,
-                "roofline_frac_distinct_bytes": chunk_cold_bytes(un, T) / (c_ms * 1e-3) / 1e9 / peak,
+                "gather_roofline_frac_per_frame_bytes": frame_bytes(nz) * T / (g_ms * 1e-3) / 1e9 / peak,
+                "gather_roofline_frac_distinct_bytes": chunk_cold_bytes(un, T) / (g_ms * 1e-3) / 1e9 / peak,
+                "dense_chunk_roofline_frac_own_bytes": dense_chunk_bytes(T) / (d_ms * 1e-3) / 1e9 / peak,
                 "single_frame_call_cold_us": s_ms * 1e3, "single_frame_dense_cold_us": sd_ms * 1e3,
                 "single_frame_speedup_vs_own_dense": sd_ms / s_ms,
-                "single_frame_roofline_frac": frame_bytes(nz) / (s_ms * 1e-3) / 1e9 / peak}
+                "single_frame_roofline_frac": frame_bytes(nz) / (s_ms * 1e-3) / 1e9 / peak,
+                "single_frame_dense_roofline_frac": dense_chunk_bytes(1) / (sd_ms * 1e-3) / 1e9 / peak}
             L2.close()
         extra["by_rho"] = by_rho
         streams = {}
@@ -477,7 +493,7 @@ def main():
             "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream per GPU; one step = "
                                    f"one chunk of {T} consecutive frames (one rrm_step_seq call) of the {FRAMES}-frame "
                                    f"sequence walked back and forth",
-                       "frames_per_step": T,
+                       "frames_per_step": T, "evaluation": EVAL.get(main_variant, "?"),
                        "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair",
                        "measured_nnz_mean_per_frame": nnz_mean, "measured_density": nnz_mean / C_IN,
                        "distinct_columns_per_chunk": uniq_mean},
@@ -487,12 +503,15 @@ def main():
                     "d2h_bytes_per_step": T * 4 * C_OUT},
             "gpu_launches": args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": committed_traffic(args.rho), "peak_kind": f"of {peak_kind}",
-                         "kernel": "fc_seq_kernel", "algorithmic_bytes_per_launch": bytes_launch,
-                         "achieved_distinct": achieved_unique, "frac_distinct": achieved_unique / peak,
-                         "distinct_bytes_per_launch": chunk_cold_bytes(uniq_mean, T),
-                         "note": "algorithmic bytes = per-frame bytes x frames per launch; frames of a chunk share "
-                                 "weight columns through L2, so DRAM traffic is the smaller 'distinct' figure"},
+                         "traffic": committed_traffic(KERNEL.get(main_variant, "fc_seq_kernel"), args.rho),
+                         "peak_kind": f"of {peak_kind}",
+                         "kernel": KERNEL.get(main_variant, "?"), "evaluation": EVAL.get(main_variant, "?"),
+                         "algorithmic_bytes_per_launch": bytes_launch,
+                         "own_bytes_per_launch": own_bytes, "achieved_own": own_bytes / (ms * 1e-3) / 1e9,
+                         "frac_own": own_bytes / (ms * 1e-3) / 1e9 / peak,
+                         "note": "algorithmic bytes = the delta-FC's per-frame bytes (gathered columns, projection, "
+                                 "frames) x frames per launch; own bytes = what the kernel that ran has to move with a "
+                                 "cold L2 (dense evaluation: W once for all frames; gather: every distinct column once)"},
             "cpu_baseline": cpu,
             "last_step_stats": st,
         }

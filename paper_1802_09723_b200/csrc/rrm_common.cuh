@@ -102,6 +102,7 @@ struct Layer {
     // few-row dense FC on the tensor cores (weights as the M operand, K split over CTAs)
     int32_t* ft_acc = nullptr;              // [rows][tiles * 128] partial sums, zero between launches
     unsigned* ft_arrive = nullptr;          // [tiles] arrival counters, zero between launches
+    bool ft_cluster = false;                // the K shares of an output block run as one thread-block cluster
     // chunk-of-frames form of the fused FC path
     int32_t* seq_dP = nullptr;              // [seq_cap][n][c_out] per-frame projection deltas
     unsigned* seq_stat = nullptr;           // [seq_cap * n][2] per frame and stream: non-zeros, active groups of 32

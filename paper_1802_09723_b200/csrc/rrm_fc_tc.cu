@@ -76,6 +76,26 @@ __device__ __forceinline__ void ft_finish(const FtParams& p, int row, int o, int
     }
 }
 
+// four consecutive outputs of one row: bias, stored projection, output through f
+__device__ __forceinline__ void ft_finish4(const FtParams& p, int row, int oo, int4 w)
+{
+    if (p.bias) { const int4 b = *reinterpret_cast<const int4*>(p.bias + oo); w.x += b.x; w.y += b.y; w.z += b.z; w.w += b.w; }
+    const size_t at = (size_t)row * p.c_out + oo;
+    if (p.Pstate && row >= p.state_from) *reinterpret_cast<int4*>(p.Pstate + at - (size_t)p.state_from * p.c_out) = w;
+    if (p.Y) {
+        if (p.shift < 0) *reinterpret_cast<int4*>(reinterpret_cast<int32_t*>(p.Y) + at) = w;
+        else {
+            char4 q;
+            q.x = (signed char)ft_apply_f(w.x, p.shift, p.act); q.y = (signed char)ft_apply_f(w.y, p.shift, p.act);
+            q.z = (signed char)ft_apply_f(w.z, p.shift, p.act); q.w = (signed char)ft_apply_f(w.w, p.shift, p.act);
+            *reinterpret_cast<char4*>(reinterpret_cast<int8_t*>(p.Y) + at) = q;
+        }
+    }
+}
+
+// CLUSTER: the CTAs that share an output block (the K shares) form one thread-block cluster and add their
+// partial sums through distributed shared memory; otherwise through the scratch array in global memory.
+template <bool CLUSTER>
 __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const __grid_constant__ CUtensorMap tmapX)
 {
     extern __shared__ unsigned char ft_smem_raw[];
@@ -185,6 +205,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
 
     // ================= epilogue: thread = output (tensor-memory lane), register j = input row
     const int o = mtile * TC_M + (warp & 3) * 32 + lane;     // (only warps 0-3 use it)
+    int* red = reinterpret_cast<int*>(base);                 // [rows][128] partial sums; the ring is free by then
     if (warp < 4) {
         ok = __all_sync(0xffffffffu, ok);
         if (ok && !mbar_wait(smem_u32(&S->done), 0)) { ok = false; atomicOr(p.errw, ERRW_TIMEOUT); }
@@ -208,17 +229,45 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
                     const int row = c0 + j;
                     if (row >= p.rows) break;
                     if (p.ksplit == 1) { if (o < p.c_out) ft_finish(p, row, o, (int)v[j]); }
+                    else if (CLUSTER) red[row * TC_M + (warp & 3) * 32 + lane] = (int)v[j];
                     else atomicAdd(p.acc + (size_t)row * (gridDim.x * TC_M) + o, (int)v[j]);
                 }
             }
         }
-        __threadfence();                                     // the partial sums are out before the arrival below
+        if (!CLUSTER) __threadfence();                       // the partial sums are out before the arrival below
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 4)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)p.tmem_cols) : "memory");
     if (p.ksplit == 1) return;
+
+    if (CLUSTER) {
+        // ================= every CTA of the cluster closes its share of the rows: row r belongs to rank r mod ksplit
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        uint32_t rank;
+        asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+        const int my_rows = (p.rows - (int)rank + p.ksplit - 1) / p.ksplit;
+        const uint32_t red_u32 = smem_u32(red);
+        for (int i = tid; i < my_rows * (TC_M / 4); i += FT_THREADS) {
+            const int row = (int)rank + (i / (TC_M / 4)) * p.ksplit, o4 = (i % (TC_M / 4)) * 4;
+            int4 w = make_int4(0, 0, 0, 0);
+            for (int c = 0; c < p.ksplit; ++c) {
+                uint32_t remote;
+                int4 t;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(red_u32 + (uint32_t)(row * TC_M + o4) * 4u), "r"(c));
+                asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w) : "r"(remote) : "memory");
+                w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
+            }
+            const int oo = mtile * TC_M + o4;
+            if (oo < p.c_out) ft_finish4(p, row, oo, w);
+        }
+        // nobody leaves while its shared memory may still be read
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        return;
+    }
 
     // ================= the last CTA of this output block closes it
     if (tid == 0) S->last = atomicAdd(p.arrive + mtile, 1u) == (unsigned)p.ksplit - 1u;
@@ -243,20 +292,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
             if (i >= total4) continue;
             const int row = i / (TC_M / 4), oo = mtile * TC_M + (i % (TC_M / 4)) * 4;
             *reinterpret_cast<int4*>(p.acc + (size_t)row * ld + oo) = make_int4(0, 0, 0, 0);
-            if (oo >= p.c_out) continue;
-            int4 w = v[u];
-            if (p.bias) { const int4 b = *reinterpret_cast<const int4*>(p.bias + oo); w.x += b.x; w.y += b.y; w.z += b.z; w.w += b.w; }
-            const size_t at = (size_t)row * p.c_out + oo;
-            if (p.Pstate && row >= p.state_from) *reinterpret_cast<int4*>(p.Pstate + at - (size_t)p.state_from * p.c_out) = w;
-            if (p.Y) {
-                if (p.shift < 0) *reinterpret_cast<int4*>(reinterpret_cast<int32_t*>(p.Y) + at) = w;
-                else {
-                    char4 q;
-                    q.x = (signed char)ft_apply_f(w.x, p.shift, p.act); q.y = (signed char)ft_apply_f(w.y, p.shift, p.act);
-                    q.z = (signed char)ft_apply_f(w.z, p.shift, p.act); q.w = (signed char)ft_apply_f(w.w, p.shift, p.act);
-                    *reinterpret_cast<char4*>(reinterpret_cast<int8_t*>(p.Y) + at) = q;
-                }
-            }
+            if (oo < p.c_out) ft_finish4(p, row, oo, v[u]);
         }
     }
     if (tid == 0) p.arrive[mtile] = 0;
@@ -295,6 +331,18 @@ static ft_encode_t ft_encoder()
     return fn;
 }
 
+static void ft_cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* at, int tiles, int ksplit, size_t dyn, cudaStream_t st)
+{
+    cfg.gridDim = dim3(tiles, ksplit);
+    cfg.blockDim = dim3(FT_THREADS);
+    cfg.dynamicSmemBytes = dyn;
+    cfg.stream = st;
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = ksplit; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+}
+
 bool fc_tc_usable(const Layer& L, int rows)
 {
     return L.tc_ready && L.tc_bn == TC_M && L.ft_acc && rows <= 2 * FT_MAX_ROWS && L.d.c_in % 16 == 0;
@@ -310,7 +358,20 @@ int fc_tc_create(rrm_net* net, Layer& L)
     RRM_CUDA_TRY(cudaMemset(a, 0, acc_bytes + arr_bytes));
     L.ft_acc = reinterpret_cast<int32_t*>(a);
     L.ft_arrive = reinterpret_cast<unsigned*>(reinterpret_cast<char*>(a) + acc_bytes);
-    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(FT_SMEM_BUDGET + 2048)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(FT_SMEM_BUDGET + 2048)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(FT_SMEM_BUDGET + 2048)));
+    // the K shares of an output block as one cluster, when all clusters of the grid can be resident at once
+    const FtPlan f = ft_plan(L);
+    L.ft_cluster = false;
+    if (f.ksplit > 1 && f.ksplit <= 8) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        ft_cluster_config(cfg, at, L.tc_ntiles, f.ksplit, FT_SMEM_BUDGET + 2048, nullptr);
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, fc_tc_kernel<true>, &cfg) == cudaSuccess) L.ft_cluster = clusters >= L.tc_ntiles;
+        else cudaGetLastError();
+        if (getenv("RRM_DEBUG")) fprintf(stderr, "rrm: few-row FC: %d tiles x %d K shares, %d clusters can be resident -> %s\n", L.tc_ntiles, f.ksplit, clusters, L.ft_cluster ? "cluster" : "global scratch");
+    }
     return RRM_OK;
 }
 
@@ -364,7 +425,14 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return RRM_ERR_CUDA;
         const size_t dyn = 1024 + (size_t)p.stages * stage_bytes + sizeof(FtSmemTail);
-        fc_tc_kernel<<<dim3(L.tc_ntiles, f.ksplit), FT_THREADS, dyn, st>>>(p, tm);
+        if (L.ft_cluster) {
+            cudaLaunchConfig_t cfg = {};
+            cudaLaunchAttribute at[1];
+            ft_cluster_config(cfg, at, L.tc_ntiles, f.ksplit, dyn, st);
+            RRM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fc_tc_kernel<true>, p, tm));
+        } else {
+            fc_tc_kernel<false><<<dim3(L.tc_ntiles, f.ksplit), FT_THREADS, dyn, st>>>(p, tm);
+        }
     }
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
