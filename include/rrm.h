@@ -143,6 +143,17 @@ int rrm_step_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* 
 int rrm_dense_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream);
 /* rrm_step_seq with HOST buffers (copies in, steps, copies out, synchronises `stream`). */
 int rrm_step_seq_host(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream);
+/* The same without waiting: the call returns once the work is queued.  The copy-in, the frames and the
+ * copy-out of a call run on three streams (two of them the library's own) chained by events, through two
+ * staging slots, so that consecutive calls overlap: chunk k+1 is copied in and chunk k-1 copied out while
+ * chunk k is computed.  X_host and Y_host should be page-locked (pageable memory makes the copies
+ * synchronous); X_host must stay unchanged and Y_host unread until rrm_host_sync (or a later call to
+ * rrm_step_seq_host on the same layer) has returned.  Calls must be issued from one thread, in frame order;
+ * the RRM state advances in that order on `stream`.  The first call, and a call with a larger T than any
+ * before, allocate the staging slots. */
+int rrm_step_seq_host_async(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream);
+/* Waits until every queued rrm_step_seq_host_async call has delivered its outputs to host memory. */
+int rrm_host_sync(rrm_layer* layer);
 
 /* Synchronises the layer's last stream and fills `host_out`. */
 int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out);
@@ -174,6 +185,9 @@ int rrm_net_step_host(rrm_net* net, const void* frame_host, void* out_host, void
 int rrm_net_step_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream);
 int rrm_net_dense_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream);
 int rrm_net_step_seq_host(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream);
+/* As rrm_step_seq_host_async / rrm_host_sync. */
+int rrm_net_step_seq_host_async(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream);
+int rrm_net_host_sync(rrm_net* net);
 
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* host_out);
 

@@ -73,6 +73,10 @@ def lib():
         "rrm_net_step_seq": [_P, _P, _P, ctypes.c_int, _P],
         "rrm_net_dense_seq": [_P, _P, _P, ctypes.c_int, _P],
         "rrm_net_step_seq_host": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_step_seq_host_async": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_net_step_seq_host_async": [_P, _P, _P, ctypes.c_int, _P],
+        "rrm_host_sync": [_P],
+        "rrm_net_host_sync": [_P],
         "rrm_net_get_stats": [_P, ctypes.c_int, ctypes.POINTER(Stats)],
         "rrm_net_projection": [_P, ctypes.c_int, _P, _P],
         "rrm_net_tensor": [_P, ctypes.c_int, _P, _P],
@@ -182,6 +186,14 @@ class Net:
         T = frames_host.shape[0] if T is None else T
         _check(lib().rrm_net_step_seq_host(self._h, _ptr(frames_host), _ptr(outs_host), T, _stream(stream)),
                "rrm_net_step_seq_host")
+
+    def step_seq_host_async(self, frames_host, outs_host=None, T=None, stream=None):
+        T = frames_host.shape[0] if T is None else T
+        _check(lib().rrm_net_step_seq_host_async(self._h, _ptr(frames_host), _ptr(outs_host), T, _stream(stream)),
+               "rrm_net_step_seq_host_async")
+
+    def host_sync(self):
+        _check(lib().rrm_net_host_sync(self._h), "rrm_net_host_sync")
 
     def set_epsilon(self, eps):
         _check(lib().rrm_net_set_epsilon(self._h, float(eps)), "rrm_net_set_epsilon")

@@ -340,6 +340,34 @@ int ensure_stage(rrm_net* net, int frames = 1)
     return RRM_OK;
 }
 
+// Staging slots, copy streams and events of the pipelined host entry point.
+int ensure_pipe(rrm_net* net, int frames)
+{
+    if (!net->h2d_stream) {
+        RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->h2d_stream, cudaStreamNonBlocking));
+        RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->d2h_stream, cudaStreamNonBlocking));
+        for (int s = 0; s < 2; ++s) {
+            RRM_CUDA_TRY(cudaEventCreateWithFlags(&net->ev_in[s], cudaEventDisableTiming));
+            RRM_CUDA_TRY(cudaEventCreateWithFlags(&net->ev_done[s], cudaEventDisableTiming));
+            RRM_CUDA_TRY(cudaEventCreateWithFlags(&net->ev_out[s], cudaEventDisableTiming));
+        }
+    }
+    if (frames <= net->pipe_frames) return RRM_OK;
+    // larger slots: the old ones may still be in use by copies in flight
+    RRM_CUDA_TRY(cudaStreamSynchronize(net->h2d_stream));
+    RRM_CUDA_TRY(cudaStreamSynchronize(net->d2h_stream));
+    if (net->last_stream) RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    for (int s = 0; s < 2; ++s) {
+        RRM_TRY(dev_alloc(net, &net->pipe_in[s], (size_t)bi * frames));
+        RRM_TRY(dev_alloc(net, &net->pipe_out[s], (size_t)bo * frames));
+    }
+    net->pipe_frames = frames;
+    return RRM_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -379,6 +407,13 @@ int rrm_net_destroy(rrm_net* net)
     if (net->act_ev) cudaEventDestroy(net->act_ev);
     if (net->act_host) cudaFreeHost(net->act_host);
     if (net->cap_stream) cudaStreamDestroy(net->cap_stream);
+    if (net->h2d_stream) cudaStreamDestroy(net->h2d_stream);
+    if (net->d2h_stream) cudaStreamDestroy(net->d2h_stream);
+    for (int s = 0; s < 2; ++s) {
+        if (net->ev_in[s]) cudaEventDestroy(net->ev_in[s]);
+        if (net->ev_done[s]) cudaEventDestroy(net->ev_done[s]);
+        if (net->ev_out[s]) cudaEventDestroy(net->ev_out[s]);
+    }
     for (void* p : net->allocs) cudaFree(p);
     delete net;
     return RRM_OK;
@@ -475,6 +510,47 @@ int rrm_step_seq_host(rrm_layer* layer, const void* X_host, void* Y_host, int T,
 {
     return rrm_net_step_seq_host(layer, X_host, Y_host, T, stream);
 }
+
+int rrm_net_step_seq_host_async(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream)
+{
+    if (!net || !frames_host || T < 1) return RRM_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    RRM_TRY(ensure_pipe(net, T));
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    const int s = net->pipe_slot;
+    net->pipe_slot ^= 1;
+    // copy-in, once the kernels that read this slot two calls ago are done (waiting for an event that was never
+    // recorded returns at once)
+    RRM_CUDA_TRY(cudaStreamWaitEvent(net->h2d_stream, net->ev_done[s], 0));
+    RRM_CUDA_TRY(cudaMemcpyAsync(net->pipe_in[s], frames_host, (size_t)bi * T, cudaMemcpyHostToDevice, net->h2d_stream));
+    RRM_CUDA_TRY(cudaEventRecord(net->ev_in[s], net->h2d_stream));
+    // the frames themselves, on the caller's stream: after their copy-in and after the copy-out that last read this
+    // slot's output buffer
+    RRM_CUDA_TRY(cudaStreamWaitEvent(st, net->ev_in[s], 0));
+    RRM_CUDA_TRY(cudaStreamWaitEvent(st, net->ev_out[s], 0));
+    RRM_TRY(run_seq(net, net->pipe_in[s], outs_host ? net->pipe_out[s] : nullptr, T, st, false, false));
+    RRM_CUDA_TRY(cudaEventRecord(net->ev_done[s], st));
+    if (outs_host) {
+        RRM_CUDA_TRY(cudaStreamWaitEvent(net->d2h_stream, net->ev_done[s], 0));
+        RRM_CUDA_TRY(cudaMemcpyAsync(outs_host, net->pipe_out[s], (size_t)bo * T, cudaMemcpyDeviceToHost, net->d2h_stream));
+        RRM_CUDA_TRY(cudaEventRecord(net->ev_out[s], net->d2h_stream));
+    }
+    return RRM_OK;
+}
+int rrm_step_seq_host_async(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream)
+{
+    return rrm_net_step_seq_host_async(layer, X_host, Y_host, T, stream);
+}
+int rrm_net_host_sync(rrm_net* net)
+{
+    if (!net) return RRM_ERR_INVALID_ARG;
+    if (net->last_stream) RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
+    if (net->d2h_stream) RRM_CUDA_TRY(cudaStreamSynchronize(net->d2h_stream));
+    return RRM_OK;
+}
+int rrm_host_sync(rrm_layer* layer) { return rrm_net_host_sync(layer); }
 
 int rrm_net_set_epsilon(rrm_net* net, float eps)
 {

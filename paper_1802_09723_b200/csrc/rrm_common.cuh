@@ -134,6 +134,13 @@ struct rrm_net {
     void* stage_in = nullptr;         // device staging for the *_host entry points
     void* stage_out = nullptr;
     int stage_frames = 0;             // frames the staging buffers hold
+    // pipelined host entry point: two staging slots, copies on streams of their own so that the copy-in of
+    // chunk k+1 and the copy-out of chunk k-1 overlap the kernels of chunk k
+    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    void* pipe_in[2] = {nullptr, nullptr};
+    void* pipe_out[2] = {nullptr, nullptr};
+    int pipe_frames = 0, pipe_slot = 0;
     // the per-frame launch sequences (0: delta step, 1: keyframe, 2: stateless dense pass), each captured
     // once and replayed (fixed frame / output buffers)
     cudaGraph_t graph[3] = {nullptr, nullptr, nullptr};

@@ -212,6 +212,29 @@ def test_fc_chunk_host_entry_point():
     layer.close()
 
 
+def test_fc_chunk_host_entry_point_pipelined():
+    """Chunks queued without waiting (copies and kernels of consecutive calls overlap) deliver the same outputs;
+    every call has host buffers of its own, and the staging slots are reused from the third call on."""
+    rrm = _rrm()
+    spec = wl.fc6_i8(c_in=2048, c_out=1024)[0]
+    seq = wl.fc_run_sequence(frames=31, c_in=2048, rho=0.05, seed=31, n=2)
+    layer = rrm.layer_from_spec(spec, n=2)
+    chunks = [(0, 4), (4, 4), (8, 8), (16, 3), (19, 12)]          # a larger T than before grows the slots mid-way
+    ins = [torch.from_numpy(seq[a:a + T]).pin_memory() for a, T in chunks]
+    outs = [torch.empty((T, 2, 1024, 1, 1), dtype=torch.int32).pin_memory() for _, T in chunks]
+    for (a, T), x, y in zip(chunks, ins, outs):
+        layer.step_seq_host_async(x, y, T)
+    layer.host_sync()
+    for (a, T), y in zip(chunks, outs):
+        for i in range(T):
+            np.testing.assert_array_equal(y[i].numpy(), orc.dense_forward([spec], seq[a + i])[0][1], err_msg=f"frame {a + i}")
+    # the state is that of the last frame: a synchronous step from it is exact
+    Y = layer.new_output()
+    layer.step(dev(seq[30]), Y)
+    np.testing.assert_array_equal(Y.cpu().numpy(), orc.dense_forward([spec], seq[30])[0][1])
+    layer.close()
+
+
 def test_fc6_chunk_longer_than_one_launch_holds():
     """40 frames exceed what one launch's closing sum keeps per thread: the call goes out in pieces."""
     spec = wl.fc6_i8()[0]
