@@ -187,6 +187,75 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
 int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
 int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
 
+// Finds the nodes of a captured sequence that hold the fixed frame / output buffers, so that each launch can
+// point them at the caller's buffers instead of copying through the fixed ones.  Any doubt (an API error, no
+// node found) leaves patch_ok false and the copies in place.
+void find_io_nodes(rrm_net* net, int kind)
+{
+    net->patch_in[kind].clear(); net->patch_out[kind].clear(); net->patch_ok[kind] = false;
+    size_t n = 0;
+    if (cudaGraphGetNodes(net->graph[kind], nullptr, &n) != cudaSuccess || n == 0) { cudaGetLastError(); return; }
+    std::vector<cudaGraphNode_t> nodes(n);
+    if (cudaGraphGetNodes(net->graph[kind], nodes.data(), &n) != cudaSuccess) { cudaGetLastError(); return; }
+    for (cudaGraphNode_t node : nodes) {
+        cudaGraphNodeType type;
+        if (cudaGraphNodeGetType(node, &type) != cudaSuccess) { cudaGetLastError(); return; }
+        if (type == cudaGraphNodeTypeKernel) {
+            cudaKernelNodeParams kp = {};
+            if (cudaGraphKernelNodeGetParams(node, &kp) != cudaSuccess || !kp.kernelParams) { cudaGetLastError(); return; }
+            // the kernel's arguments: count and sizes from the function itself
+            std::vector<void*> args;
+            for (size_t i = 0;; ++i) {
+                size_t off = 0, size = 0;
+                if (cudaFuncGetParamInfo(kp.func, i, &off, &size) != cudaSuccess) { cudaGetLastError(); break; }
+                args.push_back(kp.kernelParams[i]);
+            }
+            for (size_t i = 0; i < args.size(); ++i) {
+                size_t off = 0, size = 0;
+                cudaFuncGetParamInfo(kp.func, i, &off, &size);
+                if (size != sizeof(void*)) continue;
+                void* v = *reinterpret_cast<void* const*>(kp.kernelParams[i]);
+                if (v != net->frame_buf && v != net->out_buf) continue;
+                rrm_net::IoPatch pt;
+                pt.node = node; pt.kp = kp; pt.args = args; pt.index = (int)i;
+                (v == net->frame_buf ? net->patch_in[kind] : net->patch_out[kind]).push_back(pt);
+            }
+        } else if (type == cudaGraphNodeTypeMemcpy) {
+            cudaMemcpy3DParms mp = {};
+            if (cudaGraphMemcpyNodeGetParams(node, &mp) != cudaSuccess) { cudaGetLastError(); return; }
+            if (mp.dstPtr.ptr == net->out_buf && mp.extent.height <= 1 && mp.extent.depth <= 1) {
+                rrm_net::IoPatch pt;
+                pt.node = node; pt.is_copy = true; pt.src = mp.srcPtr.ptr; pt.bytes = mp.extent.width;
+                net->patch_out[kind].push_back(pt);
+            } else if (mp.dstPtr.ptr == net->out_buf || mp.srcPtr.ptr == net->frame_buf) {
+                return;                                      // a copy of another shape: leave everything as it is
+            }
+        }
+    }
+    net->patch_ok[kind] = net->patch_in[kind].size() == 1 && net->patch_out[kind].size() == 1;
+}
+
+// Points the frame / output nodes of the instantiated graph at `frame` and `out`.
+int patch_io(rrm_net* net, int kind, const void* frame, void* out)
+{
+    for (int side = 0; side < 2; ++side) {
+        rrm_net::IoPatch& pt = side == 0 ? net->patch_in[kind][0] : net->patch_out[kind][0];
+        void* target = side == 0 ? const_cast<void*>(frame) : (out ? out : net->out_buf);
+        if (pt.value == target) continue;                    // already there
+        if (pt.is_copy) {
+            RRM_CUDA_TRY(cudaGraphExecMemcpyNodeSetParams1D(net->exec[kind], pt.node, target, pt.src, pt.bytes,
+                                                            cudaMemcpyDeviceToDevice));
+        } else {
+            pt.value = target;
+            pt.args[pt.index] = &pt.value;
+            pt.kp.kernelParams = pt.args.data();
+            RRM_CUDA_TRY(cudaGraphExecKernelNodeSetParams(net->exec[kind], pt.node, &pt.kp));
+        }
+        pt.value = target;
+    }
+    return RRM_OK;
+}
+
 // Captures one of the per-frame launch sequences into a graph (on a private stream: a capture cannot
 // start on the legacy default stream) so that later frames cost one graph launch on the host.
 int build_graph(rrm_net* net, int kind)
@@ -206,12 +275,14 @@ int build_graph(rrm_net* net, int kind)
     if (s != RRM_OK || e != cudaSuccess || !g) { if (g) cudaGraphDestroy(g); cudaGetLastError(); return s != RRM_OK ? s : RRM_ERR_CUDA; }
     net->graph[kind] = g;
     RRM_CUDA_TRY(cudaGraphInstantiate(&net->exec[kind], g, 0));
+    find_io_nodes(net, kind);
     return RRM_OK;
 }
 
 void drop_graphs(rrm_net* net)
 {
     for (int k = 0; k < 3; ++k) {
+        net->patch_in[k].clear(); net->patch_out[k].clear(); net->patch_ok[k] = false;
         if (net->exec[k]) { cudaGraphExecDestroy(net->exec[k]); net->exec[k] = nullptr; }
         if (net->graph[k]) { cudaGraphDestroy(net->graph[k]); net->graph[k] = nullptr; }
     }
@@ -288,6 +359,17 @@ int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bo
             int64_t bi = 0, bo = 0;
             tensor_bytes_boundary(net->tensors.front(), &bi);
             tensor_bytes_boundary(net->tensors.back(), &bo);
+            if (net->patch_ok[kind] && patch_io(net, kind, frame, out) == RRM_OK) {
+                RRM_CUDA_TRY(cudaGraphLaunch(net->exec[kind], st));
+                return RRM_OK;
+            }
+            if (net->patch_ok[kind]) {
+                // an update failed half-way: the graphs are no longer trusted, launch kernel by kernel from now on
+                cudaGetLastError();
+                drop_graphs(net);
+                net->graph_off = true;
+                return launch_sequence(net, frame, out, st, dense, stateless);
+            }
             RRM_CUDA_TRY(cudaMemcpyAsync(net->frame_buf, frame, (size_t)bi, cudaMemcpyDeviceToDevice, st));
             RRM_CUDA_TRY(cudaGraphLaunch(net->exec[kind], st));
             if (out) RRM_CUDA_TRY(cudaMemcpyAsync(out, net->out_buf, (size_t)bo, cudaMemcpyDeviceToDevice, st));

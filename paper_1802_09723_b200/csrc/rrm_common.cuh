@@ -149,6 +149,20 @@ struct rrm_net {
     void* frame_buf = nullptr;        // the step's input frame, boundary layout
     void* out_buf = nullptr;          // the step's last tensor, boundary layout
     bool graph_off = false;           // RRM_NO_GRAPH=1: launch kernel by kernel (debugging)
+    // where a captured sequence reads the frame and writes the output: the nodes (kernel arguments or a copy) that
+    // hold frame_buf / out_buf are re-pointed at the caller's buffers before each launch, which saves the two
+    // device-to-device copies around the graph; empty when the nodes could not be identified
+    struct IoPatch {
+        cudaGraphNode_t node = nullptr;
+        bool is_copy = false;                      // a 1-D copy node (binary outputs) instead of a kernel
+        cudaKernelNodeParams kp = {};
+        std::vector<void*> args;                   // the node's argument pointers, ours to edit
+        int index = -1;                            // which argument is the buffer
+        const void* src = nullptr; size_t bytes = 0;   // copy node: source and size
+        void* value = nullptr;                     // storage the patched argument points to
+    };
+    std::vector<IoPatch> patch_in[3], patch_out[3];
+    bool patch_ok[3] = {false, false, false};
     // measured activity of the last delta step, read back without stalling the stream: when nearly every
     // projection pixel has to be updated anyway, the next frames are evaluated densely (same results, less work)
     size_t counters_off = 0, counters_bytes = 0;   // the counters inside the cleared arena
