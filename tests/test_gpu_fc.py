@@ -283,6 +283,9 @@ def test_fc6_dense_chunks_take_over_at_high_measured_density():
     (4096, 1000, 7, "relu", 2, 9),        # outputs not a multiple of 16: the general layer path, frame by frame
     (160, 528, 6, "relu", 3, 5),          # K smaller than one share per SM, ragged tiles
     (2048, 1024, -1, "none", 4, 16),      # 64 rows in one launch
+    (1024, 256, -1, "none", 8, 25),       # 200 rows: two launches of 100 (112 accumulator columns), clusters of 8 K shares
+    (4096, 128, 5, "relu", 2, 6),         # one output block, 32 K shares: partial sums through the global scratch
+    (128, 256, -1, "none", 2, 5),         # a single K slab: no split, outputs straight from the accumulators
 ])
 def test_fc_dense_few_rows_on_tensor_cores(c_in, c_out, shift, act, n, T):
     """Dense chunks (stateless and keyframe-like) equal Eq. 3 row by row; the state after a stateful dense
