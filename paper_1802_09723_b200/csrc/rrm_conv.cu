@@ -382,7 +382,7 @@ __global__ void pack_weights_kernel(const void* W, uint32_t* Wk, int dt, int c_i
 // One CTA handles 32 consecutive pixels of one stream: coalesced reads along w, transposed through
 // shared memory, coalesced pixel-major writes.
 // ------------------------------------------------------------------------------------------------
-constexpr int IMP_TP = 32;
+constexpr int IMP_TP = 32;                  // pixels per tile = lanes of the warp that marks their footprints
 
 template <typename T, bool DELTA>
 __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ src, T* X, T* D, uint32_t* act,
@@ -462,15 +462,14 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
     #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
     if (lane == 0 && sq > 0.f) atomicAdd(&s_sq, sq);
-    for (int pl = warp; pl < IMP_TP; pl += 8) {
-        const int cnt = (pix0 + pl < hw) ? s_cnt[pl] : 0;
-        if (cnt == 0) continue;
-        const int pix = pix0 + pl;
+    if (warp == 0) {                                         // lane = pixel of the tile
+        const int pix = pix0 + lane;
+        const int cnt = pix < hw ? s_cnt[lane] : 0;
         unsigned long long macs[MAX_READERS];
-        scatter_changed(readers, ns, pix / w, pix % w, cnt, lane, macs);
+        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, macs);
         if (lane == 0) {
             #pragma unroll
-            for (int i = 0; i < MAX_READERS; ++i) if (macs[i]) atomicAdd(&s_macs[i], macs[i]);
+            for (int i = 0; i < MAX_READERS; ++i) if (macs[i]) s_macs[i] = macs[i];
         }
     }
     __syncthreads();
@@ -524,16 +523,9 @@ __global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __res
         atomicAdd(npix, (unsigned long long)__popc(m));
     }
     unsigned long long wsum[MAX_READERS];
-    #pragma unroll
-    for (int i = 0; i < MAX_READERS; ++i) wsum[i] = 0;
-    for (unsigned mm = m; mm; mm &= mm - 1) {
-        const int src_lane = __ffs(mm) - 1;
-        const int pg = __shfl_sync(0xffffffffu, gp, src_lane), cc = __shfl_sync(0xffffffffu, cnt, src_lane);
-        const int x = pg % w, y = (pg / w) % h, ns = pg / hw;
-        unsigned long long macs[MAX_READERS];
-        scatter_changed(readers, ns, y, x, cc, lane, macs);
-        #pragma unroll
-        for (int i = 0; i < MAX_READERS; ++i) wsum[i] += macs[i];
+    {
+        const int ns = gp / hw, pix = gp - ns * hw;
+        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum);
     }
     if (lane == 0) {
         #pragma unroll
@@ -576,16 +568,9 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
     // every changed pixel marks the projection pixels of the reading layers that it touches
     const int lane = threadIdx.x & 31;
     unsigned long long wsum[MAX_READERS];
-    #pragma unroll
-    for (int i = 0; i < MAX_READERS; ++i) wsum[i] = 0;
-    for (unsigned mm = m; mm; mm &= mm - 1) {
-        const int src_lane = __ffs(mm) - 1;
-        const int pix = __shfl_sync(0xffffffffu, gp, src_lane), c = __shfl_sync(0xffffffffu, cnt, src_lane);
-        const int x = pix % w, y = (pix / w) % h, ns = pix / (w * h);
-        unsigned long long macs[MAX_READERS];
-        scatter_changed(readers, ns, y, x, c, lane, macs);
-        #pragma unroll
-        for (int i = 0; i < MAX_READERS; ++i) wsum[i] += macs[i];
+    {
+        const int ns = gp / (w * h), pix = gp - ns * (w * h);
+        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum);
     }
     if (lane == 0) {
         #pragma unroll

@@ -40,6 +40,76 @@ __device__ __forceinline__ void scatter_changed(const Readers& R, int ns, int y,
     }
 }
 
+// The same marking and counting for 32 CONSECUTIVE pixels of a tensor at once, executed by a full warp: lane j
+// owns one pixel (ns, y, x) (consecutive in the flattened [n][h][w] order) with `cnt` non-zero delta elements
+// (0: unchanged or past the end).  Changed pixels come in runs along an image row, so the marking is done per
+// row segment of the warp instead of per pixel: lane j tests candidate projection column ox_min + j of the
+// reading layer against the segment's mask of changed pixels, a ballot gives the columns as a run of bits, and
+// lane r ORs that run into projection row oy_lo + r.  macs[i] (valid in every lane) = the exact
+// multiply-accumulates of all 32 pixels in reader i, as scatter_changed counts them.
+__device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, int y, int x, int cnt, int lane,
+                                                     unsigned long long (&macs)[MAX_READERS])
+{
+    const unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
+    const unsigned seg_starts = __ballot_sync(0xffffffffu, x == 0 || lane == 0);
+    #pragma unroll
+    for (int i = 0; i < MAX_READERS; ++i) {
+        macs[i] = 0;
+        if (i >= R.n) continue;
+        const Reader& c = R.r[i];
+        // this lane's own pixel: rows x columns of projection pixels it meets (for the exact count)
+        if (c.macs) {
+            unsigned long long mine = 0;
+            if (cnt > 0) {
+                const int ay = y + c.pad, ax = x + c.pad;
+                const int rows = min(c.oh - 1, ay / c.stride) - max(0, (ay - c.kh + c.stride) / c.stride) + 1;
+                const int cols = min(c.ow - 1, ax / c.stride) - max(0, (ax - c.kw + c.stride) / c.stride) + 1;
+                if (rows > 0 && cols > 0) mine = (unsigned long long)cnt * rows * cols * c.c_out;
+            }
+            #pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+            macs[i] = mine;
+        }
+        if (m == 0) continue;
+        // one row segment [a, b] of lanes at a time
+        for (unsigned ss = seg_starts; ss; ss &= ss - 1) {
+            const int a = __ffs(ss) - 1;
+            const unsigned rest = ss & (ss - 1);
+            const int b = rest ? __ffs(rest) - 2 : 31;
+            const unsigned seg = (b - a == 31 ? 0xffffffffu : ((1u << (b - a + 1)) - 1u) << a);
+            const unsigned ms = m & seg;
+            if (ms == 0) continue;
+            const int sns = __shfl_sync(0xffffffffu, ns, a), sy = __shfl_sync(0xffffffffu, y, a), xa = __shfl_sync(0xffffffffu, x, a);
+            const int ay = sy + c.pad;
+            const int oy_lo = max(0, (ay - c.kh + c.stride) / c.stride), oy_hi = min(c.oh - 1, ay / c.stride);
+            if (oy_hi < oy_lo) continue;
+            const int x_first = xa + (__ffs(ms) - 1 - a), x_last = xa + (31 - __clz(ms) - a);
+            const int ox_min = max(0, (x_first + c.pad - c.kw + c.stride) / c.stride);
+            const int ox_max = min(c.ow - 1, (x_last + c.pad) / c.stride);
+            for (int c0 = ox_min; c0 <= ox_max; c0 += 32) {
+                const int ox = c0 + lane;
+                bool touched = false;
+                if (ox <= ox_max) {
+                    // input columns under this projection column, as lanes of the segment
+                    const int la = max(a, ox * c.stride - c.pad - xa + a), lb = min(b, ox * c.stride - c.pad + c.kw - 1 - xa + a);
+                    if (la <= lb) {
+                        const unsigned bits = (lb - la == 31 ? 0xffffffffu : ((1u << (lb - la + 1)) - 1u) << la);
+                        touched = (ms & bits) != 0;
+                    }
+                }
+                const unsigned run = __ballot_sync(0xffffffffu, touched);
+                if (run == 0) continue;
+                for (int r = oy_lo + lane; r <= oy_hi; r += 32) {
+                    const int q0 = (sns * c.oh + r) * c.ow + c0;
+                    const unsigned long long v = (unsigned long long)run << (q0 & 31);
+                    atomicOr(&c.oact[q0 >> 5], (unsigned)v);
+                    if (v >> 32) atomicOr(&c.oact[(q0 >> 5) + 1], (unsigned)(v >> 32));
+                }
+            }
+        }
+    }
+}
+
 // Rows [tile * TM, tile * TM + TM) of the set bits of bm[0 .. words), in increasing pixel order, go to
 // s_q[0 .. TM) (-1 where the bitmap has fewer).  Returns the total number of set bits.  Every thread
 // of the CTA calls it (blockDim.x <= 256, TM <= blockDim.x); s_pref holds 256 + 34 ints.
