@@ -601,12 +601,14 @@ struct EpiParams {
 };
 
 // PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.  KW: pool window edge (1 = no pool).
-template <int PT, int OT, bool DENSE, int KW>
+// READERS: some layer reads the output tensor (a last layer's kernel leaves the marking code, and its registers, out).
+template <int PT, int OT, bool DENSE, int KW, bool READERS>
 __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
 {
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
     __shared__ unsigned long long s_macs[MAX_READERS];
     __shared__ unsigned int s_nnz, s_npix;
+    __shared__ int s_cnt[8];                                 // changed elements of the CTA's pixels (one per warp)
     __shared__ float s_sq;
     const int lane = threadIdx.x & 31;
     if (threadIdx.x < MAX_READERS) s_macs[threadIdx.x] = 0;
@@ -758,18 +760,24 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     #pragma unroll
     for (int o = 16; o > 0; o >>= 1) { cnt += __shfl_xor_sync(0xffffffffu, cnt, o); sq += __shfl_xor_sync(0xffffffffu, sq, o); }
     if (PT == T_F32 && lane == 0 && sq > 0.f) atomicAdd(&s_sq, sq);
-    if (cnt) {                                               // uniform inside the warp
-        if (lane == 0) {
-            atomicOr(&p.act[r >> 5], 1u << (r & 31));
-            p.pnnz[r] = cnt;
-            atomicAdd(&s_nnz, (unsigned)cnt);
-            atomicAdd(&s_npix, 1u);
-        }
+    if (lane == 0) s_cnt[threadIdx.x >> 5] = cnt;
+    if (cnt && lane == 0) {                                  // (cnt is uniform inside the warp)
+        atomicOr(&p.act[r >> 5], 1u << (r & 31));
+        p.pnnz[r] = cnt;
+        atomicAdd(&s_nnz, (unsigned)cnt);
+        atomicAdd(&s_npix, 1u);
+    }
+    if (READERS) __syncthreads();
+    // the CTA's 8 consecutive pixels mark the reading layers' projection pixels together (lane = pixel)
+    if (READERS && threadIdx.x < 32) {
+        const int rl = blockIdx.x * (blockDim.x >> 5) + lane;
+        const bool have = lane < (int)(blockDim.x >> 5) && rl < tpix;
         unsigned long long macs[MAX_READERS];
-        scatter_changed(p.readers, ns, ty, tx, cnt, lane, macs);
+        scatter_changed_warp(p.readers, have ? rl / (p.tw * p.th) : 0, have ? (rl / p.tw) % p.th : 0, have ? rl % p.tw : 1,
+                             have ? s_cnt[lane] : 0, lane, macs);
         if (lane == 0) {
             #pragma unroll
-            for (int i = 0; i < MAX_READERS; ++i) if (macs[i]) atomicAdd(&s_macs[i], macs[i]);
+            for (int i = 0; i < MAX_READERS; ++i) s_macs[i] = macs[i];
         }
     }
     __syncthreads();
@@ -926,10 +934,11 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
 template <int PT, int OT, bool DENSE>
 static int launch_epi_k(const EpiParams& e, int blocks, cudaStream_t st)
 {
+    const bool rd = !DENSE && e.readers.n > 0;               // (a dense pass marks nothing)
     switch (e.pool_k > 0 ? e.pool_k : 1) {
-        case 1: epilogue_kernel<PT, OT, DENSE, 1><<<blocks, 256, 0, st>>>(e); break;
-        case 2: epilogue_kernel<PT, OT, DENSE, 2><<<blocks, 256, 0, st>>>(e); break;
-        case 3: epilogue_kernel<PT, OT, DENSE, 3><<<blocks, 256, 0, st>>>(e); break;
+        case 1: if (rd) epilogue_kernel<PT, OT, DENSE, 1, !DENSE><<<blocks, 256, 0, st>>>(e); else epilogue_kernel<PT, OT, DENSE, 1, false><<<blocks, 256, 0, st>>>(e); break;
+        case 2: if (rd) epilogue_kernel<PT, OT, DENSE, 2, !DENSE><<<blocks, 256, 0, st>>>(e); else epilogue_kernel<PT, OT, DENSE, 2, false><<<blocks, 256, 0, st>>>(e); break;
+        case 3: if (rd) epilogue_kernel<PT, OT, DENSE, 3, !DENSE><<<blocks, 256, 0, st>>>(e); else epilogue_kernel<PT, OT, DENSE, 3, false><<<blocks, 256, 0, st>>>(e); break;
         default: return RRM_ERR_UNSUPPORTED;                 // pool windows are 2x2 or 3x3
     }
     return RRM_OK;

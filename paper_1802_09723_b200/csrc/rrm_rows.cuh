@@ -51,11 +51,12 @@ __device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, i
                                                      unsigned long long (&macs)[MAX_READERS])
 {
     const unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
-    const unsigned seg_starts = __ballot_sync(0xffffffffu, x == 0 || lane == 0);
     #pragma unroll
-    for (int i = 0; i < MAX_READERS; ++i) {
-        macs[i] = 0;
-        if (i >= R.n) continue;
+    for (int i = 0; i < MAX_READERS; ++i) macs[i] = 0;
+    if (m == 0) return;                                      // nothing changed: uniform inside the warp
+    const unsigned seg_starts = __ballot_sync(0xffffffffu, x == 0 || lane == 0);
+    #pragma unroll 1
+    for (int i = 0; i < R.n; ++i) {
         const Reader& c = R.r[i];
         // this lane's own pixel: rows x columns of projection pixels it meets (for the exact count)
         if (c.macs) {
@@ -70,7 +71,6 @@ __device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, i
             for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
             macs[i] = mine;
         }
-        if (m == 0) continue;
         // one row segment [a, b] of lanes at a time
         for (unsigned ss = seg_starts; ss; ss &= ss - 1) {
             const int a = __ffs(ss) - 1;
