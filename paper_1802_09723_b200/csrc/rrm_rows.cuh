@@ -5,48 +5,16 @@
 
 namespace rrm {
 
-// Executed by a full warp for ONE changed pixel (ns, y, x) of a tensor with `nnz` non-zero delta
-// elements: marks, in every reading layer's bitmap, the projection pixels whose filter footprint
-// covers the pixel (a layer that adds the tensor as its shortcut is a 1x1 reader), and returns in
-// macs[i] (same value in every lane) the exact multiply-accumulates the pixel implies in reader i:
-// nnz x (output, tap) pairs that meet it x output channels (Table 1 without its border approximation).
-// The projection pixels that meet (y, x) form a rectangle [oy_lo, oy_hi] x [ox_lo, ox_hi]: lane j marks
-// row oy_lo + j as one run of bits (one or two word-wide atomic ORs).
-__device__ __forceinline__ void scatter_changed(const Readers& R, int ns, int y, int x, int nnz, int lane,
-                                                unsigned long long (&macs)[MAX_READERS])
-{
-    #pragma unroll
-    for (int i = 0; i < MAX_READERS; ++i) {
-        macs[i] = 0;
-        if (i >= R.n) continue;
-        const Reader& c = R.r[i];
-        // o * stride - pad + k = coordinate, 0 <= k < kernel  <=>  ceil((coord + pad - kernel + 1) / stride) <= o <= floor((coord + pad) / stride)
-        const int ay = y + c.pad, ax = x + c.pad;
-        const int oy_lo = max(0, (ay - c.kh + c.stride) / c.stride), oy_hi = min(c.oh - 1, ay / c.stride);
-        const int ox_lo = max(0, (ax - c.kw + c.stride) / c.stride), ox_hi = min(c.ow - 1, ax / c.stride);
-        const int rows = oy_hi - oy_lo + 1, cols = ox_hi - ox_lo + 1;
-        if (rows <= 0 || cols <= 0) continue;
-        for (int j = lane; j < rows; j += 32) {
-            const int q0 = (ns * c.oh + oy_lo + j) * c.ow + ox_lo;       // first bit of the run, `cols` bits long
-            int done = 0;
-            while (done < cols) {
-                const int bit = (q0 + done) & 31, take = min(32 - bit, cols - done);
-                const uint32_t m = (take == 32 ? 0xffffffffu : ((1u << take) - 1u)) << bit;
-                atomicOr(&c.oact[(q0 + done) >> 5], m);
-                done += take;
-            }
-        }
-        if (c.macs) macs[i] = (unsigned long long)nnz * rows * cols * c.c_out;
-    }
-}
-
-// The same marking and counting for 32 CONSECUTIVE pixels of a tensor at once, executed by a full warp: lane j
-// owns one pixel (ns, y, x) (consecutive in the flattened [n][h][w] order) with `cnt` non-zero delta elements
-// (0: unchanged or past the end).  Changed pixels come in runs along an image row, so the marking is done per
-// row segment of the warp instead of per pixel: lane j tests candidate projection column ox_min + j of the
-// reading layer against the segment's mask of changed pixels, a ballot gives the columns as a run of bits, and
-// lane r ORs that run into projection row oy_lo + r.  macs[i] (valid in every lane) = the exact
-// multiply-accumulates of all 32 pixels in reader i, as scatter_changed counts them.
+// Executed by a full warp for 32 CONSECUTIVE pixels of a tensor: lane j owns one pixel (ns, y, x) (consecutive in
+// the flattened [n][h][w] order) with `cnt` non-zero delta elements (0: unchanged or past the end).  Marks, in every
+// reading layer's bitmap, the projection pixels whose filter footprint covers a changed pixel (a layer that adds
+// the tensor as its shortcut is a 1x1 reader), and returns in macs[i] (same value in every lane) the exact
+// multiply-accumulates the changed pixels imply in reader i: non-zeros x (output, tap) pairs that meet the pixel x
+// output channels (Table 1 without its border approximation).
+// The projection pixels that meet (y, x) form a rectangle [oy_lo, oy_hi] x [ox_lo, ox_hi], and changed pixels come
+// in runs along an image row, so the marking is done per row segment of the warp, not per pixel: lane j tests
+// candidate projection column ox_min + j against the segment's mask of changed pixels, a ballot gives the columns
+// as a run of bits, and lane r ORs that run into projection row oy_lo + r (one or two word-wide atomic ORs).
 __device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, int y, int x, int cnt, int lane,
                                                      unsigned long long (&macs)[MAX_READERS])
 {
