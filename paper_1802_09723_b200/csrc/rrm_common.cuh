@@ -197,6 +197,7 @@ int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int 
 // ---- rrm_fc_tc.cu
 int fc_tc_create(rrm_net* net, Layer& L);
 bool fc_tc_usable(const Layer& L, int rows);
+int fc_tc_launches(int rows);
 int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, bool stateless, unsigned* stat, cudaStream_t st);
 
 // ---- rrm_conv_tc.cu

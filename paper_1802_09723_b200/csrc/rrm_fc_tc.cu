@@ -25,6 +25,7 @@ constexpr int FT_SLAB = 128;                  // bytes of K per stage
 constexpr int FT_A_BYTES = TC_M * FT_SLAB;    // the W part of a stage
 constexpr int FT_MAX_STAGES = 12;
 constexpr int FT_MAX_ROWS = 128;              // input rows of one launch
+constexpr int FT_MAX_LAUNCHES = 8;            // more rows than this many launches hold go to the convolution kernel
 constexpr size_t FT_SMEM_BUDGET = 220 * 1024;
 
 struct FtSmemTail {
@@ -343,9 +344,11 @@ static void ft_cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* at, 
     cfg.numAttrs = 1;
 }
 
+int fc_tc_launches(int rows) { return ceil_div(rows, FT_MAX_ROWS); }
+
 bool fc_tc_usable(const Layer& L, int rows)
 {
-    return L.tc_ready && L.tc_bn == TC_M && L.ft_acc && rows <= 2 * FT_MAX_ROWS && L.d.c_in % 16 == 0;
+    return L.tc_ready && L.tc_bn == TC_M && L.ft_acc && rows <= FT_MAX_LAUNCHES * FT_MAX_ROWS && L.d.c_in % 16 == 0;
 }
 
 int fc_tc_create(rrm_net* net, Layer& L)
@@ -395,8 +398,9 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
     const int8_t* old_snap = L.xs[L.xs_cur];
     p.n = n;
     if (!stateless) L.xs_cur ^= 1;
-    // two even pieces rather than a full one and a remainder
-    const int piece_max = rows <= FT_MAX_ROWS ? rows : (rows + 1) / 2;
+    // even pieces rather than full ones and a remainder (every launch streams W again, from L2 when it fits)
+    const int pieces = ceil_div(rows, FT_MAX_ROWS);
+    const int piece_max = ceil_div(rows, pieces);
     for (int r0 = 0; r0 < rows; r0 += piece_max) {
         const int piece = rows - r0 < piece_max ? rows - r0 : piece_max;
         p.rows = piece;

@@ -284,6 +284,8 @@ def test_fc6_dense_chunks_take_over_at_high_measured_density():
     (160, 528, 6, "relu", 3, 5),          # K smaller than one share per SM, ragged tiles
     (2048, 1024, -1, "none", 4, 16),      # 64 rows in one launch
     (1024, 256, -1, "none", 8, 25),       # 200 rows: two launches of 100 (112 accumulator columns), clusters of 8 K shares
+    (512, 256, -1, "none", 16, 24),       # 384 rows: three launches of 128
+    (256, 128, -1, "none", 150, 2),       # 300 rows in three launches: the last frame's rows straddle two of them
     (4096, 128, 5, "relu", 2, 6),         # one output block, 32 K shares: partial sums through the global scratch
     (128, 256, -1, "none", 2, 5),         # a single K slab: no split, outputs straight from the accumulators
 ])
