@@ -67,6 +67,16 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def measured_tensor_tmacs():
+    """int8 tensor-core peak in TMAC/s: the measured bf16 burst TFLOP/s x 2 (nominal int8 : bf16 ratio) / 2 (flops per
+    MAC); fallback 1590 TFLOP/s bf16."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["bf16_tflops"]), "measured"
+    except Exception:  # noqa: BLE001
+        return 1590.0, "fallback"
+
+
 def committed_traffic(kernel, rho):
     """DRAM bytes per launch of the chunk kernel that ran, from its committed ncu summary, if present."""
     p = os.path.join(ROOT, "profiles", {"fc_seq_kernel": "fc_seq_fc6_chunk32.txt",
@@ -238,6 +248,36 @@ def run_conv(args):
                           "active_in_pixels": st["active_in_pixels"] / max(1, st["in_pixels"]),
                           "active_out_pixels": st["active_out_pixels"] / max(1, st["out_pixels"]),
                           "active_macs": st["active_macs"], "dense_macs": st["dense_macs"], "variant": st["variant"]})
+    # ---- roofline of the last timed step: per layer the slower of (MACs executed at the unit's peak) and (bytes that
+    # have to move at the HBM peak), summed over the layers, against the measured step time.  Bytes per layer: the delta
+    # rows of the active input pixels once + the projection rows of the pixels to update three times (read and write
+    # by the convolution, read by the epilogue); weights stay in L2 and are left out.
+    hbm, hbm_kind = measured_peaks()
+    tens, tens_kind = measured_tensor_tmacs()
+    unit_bytes = {"f32": 4.0, "i8": 1.0, "bin": 1.0 / 8}
+    mac_peak = {"f32": FFMA_TMACS, "i8": tens, "bin": tens}         # TMAC/s (int8 and binary layers run on the tensor cores)
+    roof_us = mac_us = byte_us = 0.0
+    for l, sp in enumerate(specs):
+        st = net.stats(l)
+        dense_step = st["variant"] == 3
+        macs = st["dense_macs"] if dense_step else st["active_macs"]
+        fin = 1.0 if dense_step else st["active_in_pixels"] / max(1, st["in_pixels"])
+        fout = 1.0 if dense_step else st["active_out_pixels"] / max(1, st["out_pixels"])
+        peak_l = mac_peak[sp.dtype] if (sp.dtype == "f32" or st["variant"] in (2, 3)) else (DP4A_TMACS if sp.dtype == "i8" else POPC_TBITMACS)
+        t_mac = macs / (peak_l * 1e12) * 1e6
+        nbytes = st["in_pixels"] * fin * sp.c_in * unit_bytes[sp.dtype] + st["out_pixels"] * fout * sp.c_out * 4 * (2 if dense_step else 3)
+        t_byte = nbytes / (hbm * 1e9) * 1e6
+        per_layer[l]["roofline_us"] = max(t_mac, t_byte)
+        per_layer[l]["roofline_bound"] = "hbm" if t_byte >= t_mac else ("alu" if sp.dtype == "f32" else "tensor")
+        roof_us += max(t_mac, t_byte); mac_us += t_mac; byte_us += t_byte
+    roofline = {"bound": "hbm" if byte_us >= mac_us else ("alu" if dtype == "f32" else "tensor"),
+                "achieved": roof_us * 1e-3 / ms * (hbm if byte_us >= mac_us else (FFMA_TMACS if dtype == "f32" else tens)),
+                "peak": hbm if byte_us >= mac_us else (FFMA_TMACS if dtype == "f32" else tens),
+                "unit": "GB/s" if byte_us >= mac_us else "TMAC/s", "frac": roof_us * 1e-3 / ms, "traffic": None,
+                "peak_kind": f"of {hbm_kind if byte_us >= mac_us else ('derived' if dtype == 'f32' else tens_kind)}",
+                "roofline_us_per_step": roof_us, "mac_us": mac_us, "byte_us": byte_us,
+                "note": "sum over the layers of max(executed MACs at the unit's peak, algorithmic bytes at the HBM peak) / "
+                        "measured step time; per-layer figures in per_layer_last_step"}
     ms_warm = timed(net.step, args.steps, args.warmup, cold=False)
     ms_dense = timed(net.dense, max(8, args.steps // 4), 3)
     line = {
@@ -251,7 +291,7 @@ def run_conv(args):
         "ms_per_step_warm": ms_warm, "ms_per_step_dense_path": ms_dense, "speedup_vs_own_dense": ms_dense / ms,
         "active_macs_last_step": tot_active, "dense_macs_per_step": dense_macs,
         "active_gmacs_per_s": None if tot_active is None else tot_active / ms / 1e6,
-        "clocks": clocks, "per_layer_last_step": per_layer,
+        "clocks": clocks, "roofline": roofline, "per_layer_last_step": per_layer,
     }
     print(json.dumps(line))
     net.close()
