@@ -280,6 +280,38 @@ def run_conv(args):
                         "measured step time; per-layer figures in per_layer_last_step"}
     ms_warm = timed(net.step, args.steps, args.warmup, cold=False)
     ms_dense = timed(net.dense, max(8, args.steps // 4), 3)
+    # ---- chunks of --seq consecutive frames per call (rrm_net_step_seq: the frames of a chunk overlap layer by layer)
+    seq_extra = {}
+    if args.seq and args.seq > 1:
+        Tq = args.seq
+        total = period * Tq // np.gcd(period, Tq)
+        walk = torch.stack([frames[order[(i + 1) % period]] for i in range(total)])     # frame i+1 of the walk
+        outs = net.new_output(frames=Tq)
+        nchunks = total // Tq
+
+        def timed_seq(call, steps, warmup):
+            net.keyframe(frames[order[0]], out)
+            for i in range(warmup):
+                call(walk[(i % nchunks) * Tq:(i % nchunks + 1) * Tq], outs, Tq)
+            torch.cuda.synchronize()
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for i in range(steps):
+                k = (warmup + i) % nchunks
+                flush.fill_(i & 0xff)
+                evs[i][0].record(stream)
+                call(walk[k * Tq:(k + 1) * Tq], outs, Tq)
+                evs[i][1].record(stream)
+            torch.cuda.synchronize()
+            return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+
+        steps_q = max(4, args.steps // Tq)
+        ms_seq = timed_seq(net.step_seq, steps_q, 3)
+        ms_seq_dense = timed_seq(net.dense_seq, steps_q, 3)
+        seq_extra = {"seq": {"frames_per_call": Tq, "ms_per_call": ms_seq, "ms_per_frame_step": ms_seq / Tq,
+                             "frames_per_sec": n * Tq * 1e3 / ms_seq, "dense_ms_per_call": ms_seq_dense,
+                             "dense_frames_per_sec": n * Tq * 1e3 / ms_seq_dense,
+                             "speedup_vs_own_dense": ms_seq_dense / ms_seq,
+                             "speedup_vs_frame_by_frame": ms * Tq / ms_seq}}
     line = {
         "metric": "frames_per_sec", "value": n * 1e3 / ms, "unit": "frames/s", "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -293,6 +325,7 @@ def run_conv(args):
         "active_gmacs_per_s": None if tot_active is None else tot_active / ms / 1e6,
         "clocks": clocks, "roofline": roofline, "per_layer_last_step": per_layer,
     }
+    line.update(seq_extra)
     print(json.dumps(line))
     net.close()
 
@@ -311,6 +344,7 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense"])
     ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
     ap.add_argument("--streams", type=int, default=None, help="independent videos per call (convolution workloads)")
+    ap.add_argument("--seq", type=int, default=None, help="also time rrm_net_step_seq with this many frames per call (convolution workloads)")
     args = ap.parse_args()
     if args.workload != "cfg2":
         if args.steps == 310:

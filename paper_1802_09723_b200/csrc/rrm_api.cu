@@ -59,6 +59,48 @@ void set_tensor(Tensor& T, int dtype, int n, int c, int h, int w)
     else { T.cs = c; T.unit_bytes = 4; }
 }
 
+// Points every activity bitmap and per-step counter at an arena (one memset clears it): tensors' activity bitmaps,
+// layers' update bitmaps, then the counters.  A net has one arena for frame-by-frame stepping and, for pipelined
+// chunks of frames, one per frame in flight.
+void bind_arena(rrm_net* net, char* base)
+{
+    size_t off = 0;
+    for (auto& T : net->tensors) { T.act = reinterpret_cast<uint32_t*>(base + off); off += (size_t)T.act_words() * 4; }
+    for (auto& L : net->layers) { L.oact = reinterpret_cast<uint32_t*>(base + off); off += (size_t)ceil_div(L.opixels(), 32) * 4; }
+    off = net->counters_off;
+    for (auto& T : net->tensors) {
+        T.nnz = reinterpret_cast<unsigned long long*>(base + off);
+        T.npix = reinterpret_cast<unsigned long long*>(base + off + 8);
+        T.trunc = reinterpret_cast<double*>(base + off + 16);
+        off += 32;
+    }
+    for (auto& L : net->layers) {
+        L.macs = reinterpret_cast<unsigned long long*>(base + off);
+        L.ocount = reinterpret_cast<int*>(base + off + 8);
+        off += 16;
+    }
+    net->bound_arena = base;
+}
+
+// Who reads which tensor: as input (filter footprint) or as shortcut (1x1).  The entries hold arena pointers, so
+// this follows every bind_arena.
+int bind_readers(rrm_net* net)
+{
+    for (auto& T : net->tensors) T.readers.n = 0;
+    for (auto& L : net->layers) {
+        const rrm_layer_desc& d = L.d;
+        auto add = [&](int t, Reader r) -> int {
+            Readers& R = net->tensors[t].readers;
+            if (R.n >= MAX_READERS) return RRM_ERR_UNSUPPORTED;
+            R.r[R.n++] = r;
+            return RRM_OK;
+        };
+        RRM_TRY(add(d.src, Reader{L.oact, L.oh, L.ow, d.kh, d.kw, d.stride, d.pad, d.c_out, L.macs}));
+        if (d.res >= 0) RRM_TRY(add(d.res, Reader{L.oact, L.oh, L.ow, 1, 1, 1, 0, d.c_out, nullptr}));
+    }
+    return RRM_OK;
+}
+
 int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const void* const* W, const void* const* B)
 {
     const int n = descs[0].n;
@@ -132,22 +174,7 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     cleared += net->tensors.size() * 32 + net->layers.size() * 16;
     RRM_TRY(dev_alloc(net, &net->cleared, cleared));
     net->cleared_bytes = cleared;
-    char* base = reinterpret_cast<char*>(net->cleared);
-    size_t off = 0;
-    for (auto& T : net->tensors) { T.act = reinterpret_cast<uint32_t*>(base + off); off += (size_t)T.act_words() * 4; }
-    for (auto& L : net->layers) { L.oact = reinterpret_cast<uint32_t*>(base + off); off += (size_t)ceil_div(L.opixels(), 32) * 4; }
-    off = counters_off;
-    for (auto& T : net->tensors) {
-        T.nnz = reinterpret_cast<unsigned long long*>(base + off);
-        T.npix = reinterpret_cast<unsigned long long*>(base + off + 8);
-        T.trunc = reinterpret_cast<double*>(base + off + 16);
-        off += 32;
-    }
-    for (auto& L : net->layers) {
-        L.macs = reinterpret_cast<unsigned long long*>(base + off);
-        L.ocount = reinterpret_cast<int*>(base + off + 8);
-        off += 16;
-    }
+    bind_arena(net, reinterpret_cast<char*>(net->cleared));
     RRM_TRY(dev_alloc(net, (void**)&net->aecs, (size_t)(1 + n_layers) * 8));
     for (int l = 0; l < n_layers; ++l) RRM_TRY(conv_layer_create(net, net->layers[l], W[l], B ? B[l] : nullptr));
     {
@@ -166,19 +193,7 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         net->graph_off = e && e[0] == '1';
     }
     for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
-    // who reads which tensor: as input (filter footprint) or as shortcut (1x1)
-    for (int l = 0; l < n_layers; ++l) {
-        Layer& L = net->layers[l];
-        const rrm_layer_desc& d = L.d;
-        auto add = [&](int t, Reader r) -> int {
-            Readers& R = net->tensors[t].readers;
-            if (R.n >= MAX_READERS) return RRM_ERR_UNSUPPORTED;
-            R.r[R.n++] = r;
-            return RRM_OK;
-        };
-        RRM_TRY(add(d.src, Reader{L.oact, L.oh, L.ow, d.kh, d.kw, d.stride, d.pad, d.c_out, L.macs}));
-        if (d.res >= 0) RRM_TRY(add(d.res, Reader{L.oact, L.oh, L.ow, 1, 1, 1, 0, d.c_out, nullptr}));
-    }
+    RRM_TRY(bind_readers(net));
     RRM_TRY(reset_state(net, nullptr));
     RRM_CUDA_TRY(cudaDeviceSynchronize());
     return RRM_OK;
@@ -283,6 +298,9 @@ void drop_graphs(rrm_net* net)
 {
     for (int k = 0; k < 3; ++k) {
         net->patch_in[k].clear(); net->patch_out[k].clear(); net->patch_ok[k] = false;
+        if (net->chunk_exec[k]) { cudaGraphExecDestroy(net->chunk_exec[k]); net->chunk_exec[k] = nullptr; }
+        if (net->chunk_graph[k]) { cudaGraphDestroy(net->chunk_graph[k]); net->chunk_graph[k] = nullptr; }
+        net->chunk_T[k] = 0;
         if (net->exec[k]) { cudaGraphExecDestroy(net->exec[k]); net->exec[k] = nullptr; }
         if (net->graph[k]) { cudaGraphDestroy(net->graph[k]); net->graph[k] = nullptr; }
     }
@@ -297,7 +315,7 @@ int activity_read_back(rrm_net* net, cudaStream_t st)
     if (net->act_pending) return RRM_OK;
     if (!net->act_host && cudaMallocHost(reinterpret_cast<void**>(&net->act_host), net->counters_bytes) != cudaSuccess) { cudaGetLastError(); return RRM_OK; }
     if (!net->act_ev && cudaEventCreateWithFlags(&net->act_ev, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return RRM_OK; }
-    RRM_CUDA_TRY(cudaMemcpyAsync(net->act_host, reinterpret_cast<char*>(net->cleared) + net->counters_off, net->counters_bytes,
+    RRM_CUDA_TRY(cudaMemcpyAsync(net->act_host, net->bound_arena + net->counters_off, net->counters_bytes,
                                  cudaMemcpyDeviceToHost, st));
     RRM_CUDA_TRY(cudaEventRecord(net->act_ev, st));
     net->act_pending = true;
@@ -326,6 +344,10 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
     if (!net || !frame) return RRM_ERR_INVALID_ARG;
     net->last_stream = st;
     if (net->layers[0].fc_fused) return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
+    if (net->bound_arena != reinterpret_cast<char*>(net->cleared)) {    // a pipelined chunk left another arena bound
+        bind_arena(net, reinterpret_cast<char*>(net->cleared));
+        RRM_TRY(bind_readers(net));
+    }
     const bool is_step = !dense && !stateless;
     if (is_step) {
         // the variant of this frame from the measured activity of the last delta frame (temporal coherence):
@@ -390,6 +412,165 @@ int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st,
     return RRM_OK;
 }
 
+constexpr int CHUNK_MAX_SLOTS = 24;
+
+// Streams, events, arenas and staging buffers of the pipelined chunk graphs.
+int ensure_chunk(rrm_net* net, int T)
+{
+    const int L = (int)net->layers.size();
+    int slots = L + 2 < CHUNK_MAX_SLOTS ? L + 2 : CHUNK_MAX_SLOTS;
+    if ((int)net->chunk_arena.size() < slots) {
+        if (!net->cap_stream) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
+        while ((int)net->chunk_arena.size() < slots) {
+            void* a = nullptr;
+            RRM_TRY(dev_alloc(net, &a, net->cleared_bytes));
+            net->chunk_arena.push_back(reinterpret_cast<char*>(a));
+            cudaStream_t s = net->cap_stream;
+            if (!net->chunk_streams.empty()) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
+            net->chunk_streams.push_back(s);
+            cudaEvent_t e = nullptr;
+            RRM_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            net->ev_join.push_back(e);
+        }
+        auto make = [&](cudaEvent_t* e) -> int { RRM_CUDA_TRY(cudaEventCreateWithFlags(e, cudaEventDisableTiming)); return RRM_OK; };
+        net->ev_conv.resize(L); net->ev_epi.resize(L);
+        for (int l = 0; l < L; ++l) { RRM_TRY(make(&net->ev_conv[l])); RRM_TRY(make(&net->ev_epi[l])); }
+        RRM_TRY(make(&net->ev_fork)); RRM_TRY(make(&net->ev_export));
+    }
+    if (T > net->chunk_cap) {
+        int64_t bi = 0, bo = 0;
+        tensor_bytes_boundary(net->tensors.front(), &bi);
+        tensor_bytes_boundary(net->tensors.back(), &bo);
+        RRM_CUDA_TRY(cudaDeviceSynchronize());               // the old buffers may be in use by a graph in flight
+        RRM_TRY(dev_alloc(net, &net->chunk_in, (size_t)bi * T));
+        RRM_TRY(dev_alloc(net, &net->chunk_out, (size_t)bo * T));
+        net->chunk_cap = T;
+        for (int k = 0; k < 3; ++k) {                        // graphs hold the old buffers
+            if (net->chunk_exec[k]) { cudaGraphExecDestroy(net->chunk_exec[k]); net->chunk_exec[k] = nullptr; }
+            if (net->chunk_graph[k]) { cudaGraphDestroy(net->chunk_graph[k]); net->chunk_graph[k] = nullptr; }
+            net->chunk_T[k] = 0;
+        }
+    }
+    return RRM_OK;
+}
+
+// T frames as one graph.  Frame t is captured on stream t mod S with arena t mod S; inside a frame the launches
+// follow each other on that stream; across frames:
+//   the convolution of layer l waits for the previous frame's epilogue of layer l (which reads the projection it adds to);
+//   the producer of a tensor (the import for tensor 0, the epilogue of layer l for tensor l+1) waits for the previous
+//   frame's readers of that tensor (convolutions that take it as input, epilogues that add it as shortcut, the export
+//   of the last tensor), because it overwrites the snapshot and the delta rows they read.
+// Everything else of consecutive frames may overlap.
+int build_chunk_graph(rrm_net* net, int kind, int T)
+{
+    const bool dense = kind != 0, stateless = kind == 2;
+    const int L = (int)net->layers.size();
+    RRM_TRY(ensure_chunk(net, T));
+    if (stateless) RRM_TRY(ensure_stateless(net));
+    const int S = (int)net->chunk_arena.size() < T ? (int)net->chunk_arena.size() : T;
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    cudaStream_t origin = net->cap_stream;
+    std::vector<char> conv_rec(L, 0), epi_rec(L, 0);
+    bool export_rec = false;
+    int status = RRM_OK;
+    RRM_CUDA_TRY(cudaStreamBeginCapture(origin, cudaStreamCaptureModeThreadLocal));
+    auto fail = [&](int s) { if (status == RRM_OK) status = s; };
+    auto wait = [&](cudaStream_t s, cudaEvent_t e) { if (cudaStreamWaitEvent(s, e, 0) != cudaSuccess) fail(RRM_ERR_CUDA); };
+    auto record = [&](cudaEvent_t e, cudaStream_t s) { if (cudaEventRecord(e, s) != cudaSuccess) fail(RRM_ERR_CUDA); };
+    record(net->ev_fork, origin);
+    for (int k = 1; k < S; ++k) wait(net->chunk_streams[k], net->ev_fork);
+    // the previous frame's readers of tensor j
+    auto wait_readers = [&](cudaStream_t s, int j) {
+        for (int r = 0; r < L; ++r) {
+            if (net->layers[r].d.src == j && conv_rec[r]) wait(s, net->ev_conv[r]);
+            if (net->layers[r].d.res == j && epi_rec[r]) wait(s, net->ev_epi[r]);
+        }
+        if (j == L && export_rec) wait(s, net->ev_export);
+    };
+    for (int t = 0; t < T && status == RRM_OK; ++t) {
+        cudaStream_t s = net->chunk_streams[t % S];
+        bind_arena(net, net->chunk_arena[t % S]);
+        if (bind_readers(net) != RRM_OK) { fail(RRM_ERR_UNSUPPORTED); break; }
+        // (the frame that used this arena before ran on this same stream: it is complete before the clear)
+        if (!stateless && cudaMemsetAsync(net->bound_arena, 0, net->cleared_bytes, s) != cudaSuccess) fail(RRM_ERR_CUDA);
+        wait_readers(s, 0);
+        { const int q = launch_import(net, reinterpret_cast<const char*>(net->chunk_in) + (size_t)t * bi, !dense, stateless, s); if (q != RRM_OK) fail(q); }
+        for (int l = 0; l < L && status == RRM_OK; ++l) {
+            const std::function<int(int)> hook = [&, l, s](int phase) -> int {
+                if (phase == 0) { if (epi_rec[l]) wait(s, net->ev_epi[l]); }
+                else if (phase == 1) { record(net->ev_conv[l], s); conv_rec[l] = 1; wait_readers(s, l + 1); }
+                else { record(net->ev_epi[l], s); epi_rec[l] = 1; }
+                return status;
+            };
+            const int q = launch_layer(net, l, dense, stateless, s, &hook);
+            if (q != RRM_OK) fail(q);
+        }
+        if (dense && !stateless && cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, s) != cudaSuccess) fail(RRM_ERR_CUDA);
+        { const int q = launch_export_tensor(net, L, reinterpret_cast<char*>(net->chunk_out) + (size_t)t * bo, stateless, s); if (q != RRM_OK) fail(q); }
+        record(net->ev_export, s);
+        export_rec = true;
+    }
+    for (int k = 1; k < S; ++k) { record(net->ev_join[k], net->chunk_streams[k]); wait(origin, net->ev_join[k]); }
+    cudaGraph_t g = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(origin, &g);
+    if (status != RRM_OK || e != cudaSuccess || !g) {
+        if (g) cudaGraphDestroy(g);
+        cudaGetLastError();
+        return status != RRM_OK ? status : RRM_ERR_CUDA;
+    }
+    if (net->chunk_exec[kind]) { cudaGraphExecDestroy(net->chunk_exec[kind]); net->chunk_exec[kind] = nullptr; }
+    if (net->chunk_graph[kind]) cudaGraphDestroy(net->chunk_graph[kind]);
+    net->chunk_graph[kind] = g;
+    RRM_CUDA_TRY(cudaGraphInstantiate(&net->chunk_exec[kind], g, 0));
+    net->chunk_T[kind] = T;
+    return RRM_OK;
+}
+
+// T consecutive frames of a stack as one pipelined graph; RRM_ERR_UNSUPPORTED when the per-frame loop has to do it.
+int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t st, bool dense, bool stateless)
+{
+    if (net->graph_off || net->eps > 0.f || T < 2) return RRM_ERR_UNSUPPORTED;
+    const bool is_step = !dense && !stateless;
+    if (is_step) {
+        // one decision per chunk, from the measured activity of the last delta frame (as rrm_net_step does per frame)
+        net->last_step_dense = false;
+        if (net->auto_switch) {
+            activity_poll(net);
+            if (net->activity >= DENSE_SWITCH_ACTIVITY && net->dense_streak < DENSE_SWITCH_REPROBE) {
+                net->dense_streak += T;
+                net->last_step_dense = true;
+                dense = true;
+            } else {
+                net->dense_streak = 0;
+            }
+        }
+    }
+    const int kind = !dense ? 0 : (stateless ? 2 : 1);
+    if (!net->chunk_exec[kind] || net->chunk_T[kind] != T) {
+        const int s = build_chunk_graph(net, kind, T);
+        if (s != RRM_OK) {
+            cudaGetLastError();
+            bind_arena(net, reinterpret_cast<char*>(net->cleared));
+            RRM_TRY(bind_readers(net));
+            return s == RRM_ERR_ALLOC ? s : RRM_ERR_UNSUPPORTED;
+        }
+    }
+    // the structures describe the last frame of the chunk from here on (statistics, activity read-back)
+    const int S = (int)net->chunk_arena.size() < T ? (int)net->chunk_arena.size() : T;
+    bind_arena(net, net->chunk_arena[(T - 1) % S]);
+    RRM_TRY(bind_readers(net));
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    RRM_CUDA_TRY(cudaMemcpyAsync(net->chunk_in, frames, (size_t)bi * T, cudaMemcpyDeviceToDevice, st));
+    RRM_CUDA_TRY(cudaGraphLaunch(net->chunk_exec[kind], st));
+    if (outs) RRM_CUDA_TRY(cudaMemcpyAsync(outs, net->chunk_out, (size_t)bo * T, cudaMemcpyDeviceToDevice, st));
+    if (is_step && !dense && net->auto_switch) RRM_TRY(activity_read_back(net, st));
+    return RRM_OK;
+}
+
 // T consecutive frames: one launch for the fused FC layer, the per-frame launch sequence otherwise
 int run_seq(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t st, bool dense, bool stateless)
 {
@@ -399,6 +580,12 @@ int run_seq(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t st
     if (L0.fc_fused && fc_seq_supported(L0) && T * net->n >= 4) {
         net->last_stream = st;
         return fc_seq_run(net, L0, frames, outs, T, dense, stateless, st);
+    }
+    if (!L0.fc_fused) {
+        // a stack: the frames of the chunk overlap layer by layer inside one graph
+        net->last_stream = st;
+        const int s = run_chunk(net, frames, outs, T, st, dense, stateless);
+        if (s != RRM_ERR_UNSUPPORTED) return s;
     }
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
@@ -489,6 +676,12 @@ int rrm_net_destroy(rrm_net* net)
     if (net->act_ev) cudaEventDestroy(net->act_ev);
     if (net->act_host) cudaFreeHost(net->act_host);
     if (net->cap_stream) cudaStreamDestroy(net->cap_stream);
+    for (size_t k = 1; k < net->chunk_streams.size(); ++k) cudaStreamDestroy(net->chunk_streams[k]);   // [0] is cap_stream
+    for (cudaEvent_t e : net->ev_conv) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : net->ev_epi) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : net->ev_join) if (e) cudaEventDestroy(e);
+    if (net->ev_fork) cudaEventDestroy(net->ev_fork);
+    if (net->ev_export) cudaEventDestroy(net->ev_export);
     if (net->h2d_stream) cudaStreamDestroy(net->h2d_stream);
     if (net->d2h_stream) cudaStreamDestroy(net->d2h_stream);
     for (int s = 0; s < 2; ++s) {

@@ -4,6 +4,7 @@
 #include <stdint.h>
 #include <cstdio>
 #include <cstdlib>
+#include <functional>
 #include <vector>
 #include "../../include/rrm.h"
 
@@ -128,6 +129,7 @@ struct rrm_net {
     std::vector<rrm::Tensor> tensors;
     int n = 1;
     void* cleared = nullptr;          // arena zeroed at the start of every step
+    char* bound_arena = nullptr;      // the arena the tensors' and layers' bitmap / counter pointers refer to right now
     size_t cleared_bytes = 0;
     int* errw = nullptr;              // device error word
     cudaStream_t last_stream = nullptr;
@@ -163,6 +165,21 @@ struct rrm_net {
     };
     std::vector<IoPatch> patch_in[3], patch_out[3];
     bool patch_ok[3] = {false, false, false};
+    // pipelined chunks of frames (rrm_net_step_seq on a stack): T frames captured as ONE graph in which layer l of
+    // frame t+1 depends only on layer l-1 of frame t+1, on layer l of frame t (its projection) and on the layers of
+    // frame t that read the tensor it overwrites - so consecutive frames overlap layer by layer.  Each frame in
+    // flight has an arena of its own.
+    std::vector<char*> chunk_arena;
+    std::vector<cudaStream_t> chunk_streams;      // capture streams, one per frame in flight ([0] is cap_stream)
+    std::vector<cudaEvent_t> ev_conv, ev_epi;     // per layer: the most recently captured convolution / epilogue
+    std::vector<cudaEvent_t> ev_join;
+    cudaEvent_t ev_fork = nullptr, ev_export = nullptr;
+    cudaGraph_t chunk_graph[3] = {nullptr, nullptr, nullptr};
+    cudaGraphExec_t chunk_exec[3] = {nullptr, nullptr, nullptr};
+    int chunk_T[3] = {0, 0, 0};
+    void* chunk_in = nullptr;
+    void* chunk_out = nullptr;
+    int chunk_cap = 0;                            // frames chunk_in / chunk_out hold
     // measured activity of the last delta step, read back without stalling the stream: when nearly every
     // projection pixel has to be updated anyway, the next frames are evaluated densely (same results, less work)
     size_t counters_off = 0, counters_bytes = 0;   // the counters inside the cleared arena
@@ -209,7 +226,8 @@ int zero_projection(void* P, long long words, cudaStream_t st);
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);
 int launch_import(rrm_net* net, const void* frame_dev, bool delta, bool stateless, cudaStream_t st);
-int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st);
+int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st,
+                 const std::function<int(int)>* hook = nullptr);
 int launch_export_tensor(rrm_net* net, int t, void* dst_dev, bool stateless, cudaStream_t st);
 int launch_export_projection(rrm_net* net, int l, void* dst_dev, cudaStream_t st);
 int reset_state(rrm_net* net, cudaStream_t st);

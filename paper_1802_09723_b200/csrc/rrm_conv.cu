@@ -955,8 +955,11 @@ static int launch_epi(const EpiParams& e, int ot, int blocks, cudaStream_t st)
     }
 }
 
-int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st)
+// hook (may be null): called with 0 before the layer's first launch, with 1 between the convolution and the
+// epilogue, with 2 after the epilogue (the pipelined chunk graph inserts its cross-frame dependencies there).
+int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st, const std::function<int(int)>* hook)
 {
+    if (hook) RRM_TRY((*hook)(0));
     Layer& L = net->layers[l];
     const rrm_layer_desc& d = L.d;
     Tensor& in = net->tensors[d.src];
@@ -987,6 +990,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     else if (d.dtype == RRM_I8) { if (dense) launch_gemm<T_I8, true>(p, grid, st); else launch_gemm<T_I8, false>(p, grid, st); }
     else { if (dense) launch_gemm<T_BIN, true>(p, grid, st); else launch_gemm<T_BIN, false>(p, grid, st); }
 
+    if (hook) RRM_TRY((*hook)(1));
     EpiParams e;
     e.P = p.P; e.oact = L.oact;
     e.resX = res ? (stateless ? res->X2 : res->X) : nullptr;
@@ -1002,6 +1006,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     else es = dense ? launch_epi<T_I32, true>(e, out.dtype, blocks, st) : launch_epi<T_I32, false>(e, out.dtype, blocks, st);
     RRM_TRY(es);
     RRM_CUDA_TRY(cudaGetLastError());
+    if (hook) RRM_TRY((*hook)(2));
     return RRM_OK;
 }
 

@@ -251,3 +251,67 @@ def test_cfg5_xnor_alexnet_128_frames():
     specs = wl.xnor_alexnet_convs()
     video = wl.moving_rect_video(frames=128, hw=227, dtype="i8", seed=51)
     _run(specs, video, check_frames={0, 1, 64, 127})
+
+
+# ------------------------------------------------------------------ chunks of frames through a stack (frames overlap layer by layer)
+@pytest.mark.parametrize("name", ["alex_f32", "alex_i8", "resnet_i8", "xnor", "alexnet_full_i8"])
+def test_stack_chunks_of_frames_equal_frame_by_frame(name):
+    """rrm_net_step_seq on a stack runs the frames of a chunk as one graph in which consecutive frames overlap;
+    every frame's output, the state after each chunk and the last frame's counters are those of Algorithm 1."""
+    rrm = _rrm()
+    if name == "alex_f32":
+        specs, dt, hw = wl.alexnet_convs("f32", hw=99, scale=8), "f32", 99
+    elif name == "alex_i8":
+        specs, dt, hw = wl.alexnet_convs("i8", hw=99, scale=8), "i8", 99
+    elif name == "resnet_i8":
+        specs, dt, hw = wl.resnet18_convs(hw=96, scale=8), "i8", 96
+    elif name == "xnor":
+        specs, dt, hw = wl.xnor_alexnet_convs(hw=99, scale=8), "i8", 99
+    else:
+        specs, dt, hw = wl.alexnet_full("i8", hw=99, scale=8, classes=80), "i8", 99
+    n = 2 if name == "resnet_i8" else 1
+    video = wl.moving_rect_video(frames=17, hw=hw, dtype=dt, seed=19, n=n, side=(12, 24),
+                                 bg_redraw=0.02 if name == "resnet_i8" else 0.0)
+    net = rrm.net_from_specs(specs, n=n)
+    rec = orc.Recurrence(specs, n=n)
+    rec.step(np.full_like(video[0], 0))
+    frames = dev(np.ascontiguousarray(video))
+    t0 = 0
+    for T in (5, 5, 2, 4):                    # the same length twice (graph reuse), then other lengths
+        outs = net.new_output(frames=T)
+        net.step_seq(frames[t0:t0 + T], outs, T)
+        for i in range(T):
+            rec.step(video[t0 + i])
+            want = orc.dense_forward(specs, video[t0 + i])[0][len(specs)]
+            got = outs[i].cpu().numpy()
+            if dt == "f32":
+                assert float(np.abs(got - want).max()) <= F32_TOL * max(1e-30, float(np.abs(want).max())), (t0 + i)
+            elif _out_kind(specs[-1]) == "bin":
+                np.testing.assert_array_equal(unpack_bits_nhwc(got.view(np.uint32), specs[-1].c_out), want, err_msg=f"frame {t0 + i}")
+            else:
+                np.testing.assert_array_equal(got.astype(np.int64), want, err_msg=f"frame {t0 + i}")
+        t0 += T
+        _compare(specs, net, video[t0 - 1], t0 - 1)          # every layer's stored projection and tensor after the chunk
+        for l in range(len(specs)):
+            st = net.stats(l)
+            assert st["error_word"] == 0
+            if dt != "f32" or l == 0:
+                assert st["nnz_elems"] == rec.nnz[l] and st["active_macs"] == rec.macs[l], (t0, l, st)
+    # frame-by-frame stepping carries on from the chunk's state
+    out = net.new_output()
+    net.step(dev(video[16]), out)
+    _compare(specs, net, video[16], 16)
+    # dense chunks leave the state alone
+    outs = net.new_output(frames=3)
+    net.dense_seq(frames[2:5], outs, 3)
+    for i in range(3):
+        want = orc.dense_forward(specs, video[2 + i])[0][len(specs)]
+        got = outs[i].cpu().numpy()
+        if dt == "f32":
+            assert float(np.abs(got - want).max()) <= F32_TOL * max(1e-30, float(np.abs(want).max()))
+        elif _out_kind(specs[-1]) == "bin":
+            np.testing.assert_array_equal(unpack_bits_nhwc(got.view(np.uint32), specs[-1].c_out), want)
+        else:
+            np.testing.assert_array_equal(got.astype(np.int64), want)
+    _compare(specs, net, video[16], 16)
+    net.close()
