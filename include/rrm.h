@@ -131,7 +131,11 @@ int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* st
  *   Y_dev  [T] outputs f(P_t), each in the layer's output layout, back to back; may be NULL
  * For a lone int8 FC layer all T input deltas are known up front (dI_t = X_t - X_{t-1}), so the T
  * sparse products W dI_t run in ONE launch and only the running sum P_t = P_{t-1} + W dI_t is
- * serial; other layers and stacks are stepped frame by frame on `stream`.  With variant AUTO the
+ * serial.  A stack (and a lone layer of another kind) keeps Algorithm 1's order per layer but lets the frames of
+ * the chunk overlap: the T frames are captured as one graph in which layer l of frame t+1 waits only for layer
+ * l-1 of frame t+1, for layer l of frame t (its projection) and for the layers of frame t that read the tensor
+ * it overwrites; the first call with a new T captures that graph (and allocates T frames of staging).  With eps > 0
+ * the frames are stepped one by one.  With variant AUTO the
  * library reads back the measured delta density of each chunk (asynchronously) and evaluates the
  * next chunk densely on the tensor cores instead when that density was high: outputs, state and
  * counters are the same integers either way.  The first call with a larger T than any before
@@ -181,7 +185,8 @@ int rrm_net_step(rrm_net* net, const void* frame_dev, void* out_dev, void* strea
 /* Dense evaluation of the stack without touching the RRM state. */
 int rrm_net_dense(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
 int rrm_net_step_host(rrm_net* net, const void* frame_host, void* out_host, void* stream);
-/* Chunks of T frames, as rrm_step_seq / rrm_dense_seq / rrm_step_seq_host; outs = [T] last tensors. */
+/* Chunks of T frames, as rrm_step_seq / rrm_dense_seq / rrm_step_seq_host; outs = [T] last tensors.  After the call
+ * rrm_net_get_stats reports the counters of the chunk's last frame. */
 int rrm_net_step_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream);
 int rrm_net_dense_seq(rrm_net* net, const void* frames_dev, void* outs_dev, int T, void* stream);
 int rrm_net_step_seq_host(rrm_net* net, const void* frames_host, void* outs_host, int T, void* stream);
