@@ -539,7 +539,7 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
         if (net->auto_switch) {
             activity_poll(net);
             if (net->activity >= DENSE_SWITCH_ACTIVITY && net->dense_streak < DENSE_SWITCH_REPROBE) {
-                net->dense_streak += T;
+                ++net->dense_streak;                         // (counted in calls: a delta chunk measures again after 15 dense ones)
                 net->last_step_dense = true;
                 dense = true;
             } else {
