@@ -315,3 +315,29 @@ def test_stack_chunks_of_frames_equal_frame_by_frame(name):
             np.testing.assert_array_equal(got.astype(np.int64), want)
     _compare(specs, net, video[16], 16)
     net.close()
+
+
+def test_large_stack_chunks_go_dense_while_nearly_every_pixel_changes():
+    """The density switch of a large stack, chunk by chunk: the chunk after a measured high-activity delta chunk is
+    evaluated densely (a sequence of precise inferences that replace the state); outputs and state stay exact."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8")
+    video = wl.moving_rect_video(frames=13, hw=227, dtype="i8", seed=34, n=2, bg_redraw=0.10)
+    net = rrm.net_from_specs(specs, n=2)
+    frames = dev(np.ascontiguousarray(video))
+    variants = []
+    for k in range(3):
+        outs = net.new_output(frames=4)
+        net.step_seq(frames[4 * k:4 * k + 4], outs, 4)
+        st = net.stats(1)                     # synchronises, so the next call sees this chunk's counters
+        variants.append(st["variant"])
+        assert (st["nnz_elems"] == -1) == (st["variant"] == 3)
+        for i in (0, 3):
+            want = orc.dense_forward(specs, video[4 * k + i])[0][len(specs)]
+            np.testing.assert_array_equal(outs[i].cpu().numpy().astype(np.int64), want, err_msg=f"frame {4 * k + i}")
+        _compare(specs, net, video[4 * k + 3], 4 * k + 3)
+    assert variants[0] == 2 and variants[1] == 3 and variants[2] == 3, variants
+    out = net.new_output()
+    net.step(dev(video[12]), out)             # frame by frame from the state the dense chunks left
+    _compare(specs, net, video[12], 12)
+    net.close()
