@@ -305,7 +305,9 @@ def run_conv(args):
             return float(np.mean([a.elapsed_time(b) for a, b in evs]))
 
         steps_q = max(4, args.steps // Tq)
-        ms_seq = timed_seq(net.step_seq, steps_q, 3)
+        # (18 warm-up chunks: a large stack measures its activity with one delta chunk after 15 dense ones, and both
+        # chunk graphs are to be captured before the timed region)
+        ms_seq = timed_seq(net.step_seq, max(steps_q, 16), 18)
         ms_seq_dense = timed_seq(net.dense_seq, steps_q, 3)
         seq_extra = {"seq": {"frames_per_call": Tq, "ms_per_call": ms_seq, "ms_per_frame_step": ms_seq / Tq,
                              "frames_per_sec": n * Tq * 1e3 / ms_seq, "dense_ms_per_call": ms_seq_dense,

@@ -412,19 +412,22 @@ int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st,
     return RRM_OK;
 }
 
-constexpr int CHUNK_MAX_SLOTS = 24;
+constexpr int CHUNK_MAX_SLOTS = 24;             // capture streams = frames in flight
+constexpr int CHUNK_ARENAS = 64;                // arenas of the chunk graphs (>= CHUNK_MAX_SLOTS)
 
 // Streams, events, arenas and staging buffers of the pipelined chunk graphs.
 int ensure_chunk(rrm_net* net, int T)
 {
     const int L = (int)net->layers.size();
     int slots = L + 2 < CHUNK_MAX_SLOTS ? L + 2 : CHUNK_MAX_SLOTS;
-    if ((int)net->chunk_arena.size() < slots) {
+    if (net->chunk_arena.empty()) {
         if (!net->cap_stream) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
-        while ((int)net->chunk_arena.size() < slots) {
-            void* a = nullptr;
-            RRM_TRY(dev_alloc(net, &a, net->cleared_bytes));
-            net->chunk_arena.push_back(reinterpret_cast<char*>(a));
+        // one block of CHUNK_ARENAS arenas: a chunk of up to that many frames gives every frame its own and clears
+        // them all with one memset; longer chunks reuse `slots` of them, each cleared by the frame that takes it
+        void* block = nullptr;
+        RRM_TRY(dev_alloc(net, &block, net->cleared_bytes * CHUNK_ARENAS));
+        for (int a = 0; a < CHUNK_ARENAS; ++a) net->chunk_arena.push_back(reinterpret_cast<char*>(block) + (size_t)a * net->cleared_bytes);
+        while ((int)net->chunk_streams.size() < slots) {
             cudaStream_t s = net->cap_stream;
             if (!net->chunk_streams.empty()) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
             net->chunk_streams.push_back(s);
@@ -467,7 +470,8 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
     const int L = (int)net->layers.size();
     RRM_TRY(ensure_chunk(net, T));
     if (stateless) RRM_TRY(ensure_stateless(net));
-    const int S = (int)net->chunk_arena.size() < T ? (int)net->chunk_arena.size() : T;
+    const int S = (int)net->chunk_streams.size() < T ? (int)net->chunk_streams.size() : T;
+    const bool own_arena = T <= CHUNK_ARENAS;                // every frame has an arena of its own
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
@@ -479,6 +483,7 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
     auto fail = [&](int s) { if (status == RRM_OK) status = s; };
     auto wait = [&](cudaStream_t s, cudaEvent_t e) { if (cudaStreamWaitEvent(s, e, 0) != cudaSuccess) fail(RRM_ERR_CUDA); };
     auto record = [&](cudaEvent_t e, cudaStream_t s) { if (cudaEventRecord(e, s) != cudaSuccess) fail(RRM_ERR_CUDA); };
+    if (own_arena && !stateless && cudaMemsetAsync(net->chunk_arena[0], 0, net->cleared_bytes * T, origin) != cudaSuccess) fail(RRM_ERR_CUDA);
     record(net->ev_fork, origin);
     for (int k = 1; k < S; ++k) wait(net->chunk_streams[k], net->ev_fork);
     // the previous frame's readers of tensor j
@@ -491,10 +496,10 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
     };
     for (int t = 0; t < T && status == RRM_OK; ++t) {
         cudaStream_t s = net->chunk_streams[t % S];
-        bind_arena(net, net->chunk_arena[t % S]);
+        bind_arena(net, net->chunk_arena[own_arena ? t : t % S]);
         if (bind_readers(net) != RRM_OK) { fail(RRM_ERR_UNSUPPORTED); break; }
-        // (the frame that used this arena before ran on this same stream: it is complete before the clear)
-        if (!stateless && cudaMemsetAsync(net->bound_arena, 0, net->cleared_bytes, s) != cudaSuccess) fail(RRM_ERR_CUDA);
+        // (a reused arena: the frame that used it before ran on this same stream, so it is complete before the clear)
+        if (!own_arena && !stateless && cudaMemsetAsync(net->bound_arena, 0, net->cleared_bytes, s) != cudaSuccess) fail(RRM_ERR_CUDA);
         wait_readers(s, 0);
         { const int q = launch_import(net, reinterpret_cast<const char*>(net->chunk_in) + (size_t)t * bi, !dense, stateless, s); if (q != RRM_OK) fail(q); }
         for (int l = 0; l < L && status == RRM_OK; ++l) {
@@ -525,6 +530,12 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
     net->chunk_graph[kind] = g;
     RRM_CUDA_TRY(cudaGraphInstantiate(&net->chunk_exec[kind], g, 0));
     net->chunk_T[kind] = T;
+    if (getenv("RRM_DEBUG")) {
+        size_t nodes = 0;
+        cudaGraphGetNodes(g, nullptr, &nodes);
+        fprintf(stderr, "rrm: chunk graph (%s, %d frames): %zu nodes, %d frames in flight\n",
+                kind == 0 ? "delta" : (kind == 1 ? "keyframes" : "dense"), T, nodes, S);
+    }
     return RRM_OK;
 }
 
@@ -558,8 +569,8 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
         }
     }
     // the structures describe the last frame of the chunk from here on (statistics, activity read-back)
-    const int S = (int)net->chunk_arena.size() < T ? (int)net->chunk_arena.size() : T;
-    bind_arena(net, net->chunk_arena[(T - 1) % S]);
+    const int S = (int)net->chunk_streams.size() < T ? (int)net->chunk_streams.size() : T;
+    bind_arena(net, net->chunk_arena[T <= CHUNK_ARENAS ? T - 1 : (T - 1) % S]);
     RRM_TRY(bind_readers(net));
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
