@@ -341,3 +341,23 @@ def test_large_stack_chunks_go_dense_while_nearly_every_pixel_changes():
     net.step(dev(video[12]), out)             # frame by frame from the state the dense chunks left
     _compare(specs, net, video[12], 12)
     net.close()
+
+
+def test_stack_chunks_through_the_pipelined_host_entry_point():
+    """Host buffers in, host buffers out, calls queued without waiting: a stack's chunks through
+    rrm_net_step_seq_host_async deliver every frame's output."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8", hw=99, scale=8)
+    video = wl.moving_rect_video(frames=12, hw=99, dtype="i8", seed=23, n=1, side=(12, 24))
+    net = rrm.net_from_specs(specs, n=1)
+    ins = [torch.from_numpy(np.ascontiguousarray(video[a:a + 4])).pin_memory() for a in (0, 4, 8)]
+    shape = tuple(net.new_output(frames=4).shape)
+    outs = [torch.empty(shape, dtype=torch.int8).pin_memory() for _ in range(3)]
+    for x, y in zip(ins, outs):
+        net.step_seq_host_async(x, y, 4)
+    net.host_sync()
+    for k, y in enumerate(outs):
+        for i in range(4):
+            want = orc.dense_forward(specs, video[4 * k + i])[0][len(specs)]
+            np.testing.assert_array_equal(y[i].numpy().astype(np.int64), want, err_msg=f"frame {4 * k + i}")
+    net.close()
