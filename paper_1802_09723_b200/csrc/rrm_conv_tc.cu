@@ -112,7 +112,33 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
             const int y0 = oy * p.stride - p.pad, x0 = ox * p.stride - p.pad;
             pix0 = ns * p.h * p.w + y0 * p.w + x0;
-            for (int t0 = 0; t0 < p.taps; t0 += 8) {          // 8 taps at a time: all bitmap loads first
+            if (p.kw <= 32) {
+                // one filter row at a time: its usable taps are a run of consecutive input pixels, whose activity bits
+                // come out of one or two bitmap words together
+                const int kx_lo = max(0, -x0), kx_hi = min(p.kw, p.w - x0), nk = kx_hi - kx_lo;
+                const int kh = p.taps / p.kw;
+                const unsigned run = nk >= 32 ? 0xffffffffu : ((1u << max(nk, 0)) - 1u);
+                for (int ky = 0; ky < kh && nk > 0; ++ky) {
+                    const int iy = y0 + ky;
+                    if (iy < 0 || iy >= p.h) continue;
+                    unsigned bits = run;
+                    if (!DENSE) {
+                        const int g = pix0 + ky * p.w + kx_lo, sh = g & 31;
+                        unsigned long long two = p.in_act[g >> 5];
+                        if (sh + nk > 32) two |= (unsigned long long)p.in_act[(g >> 5) + 1] << 32;
+                        bits = (unsigned)(two >> sh) & run;
+                    }
+                    if (bits == 0) continue;
+                    const int t = ky * p.kw + kx_lo;             // tap index of the run's first bit
+                    if (t < 64) {
+                        m0 |= (unsigned long long)bits << t;
+                        if (t + nk > 64) m1 |= (unsigned long long)bits >> (64 - t);
+                    } else {
+                        m1 |= (unsigned long long)bits << (t - 64);
+                    }
+                }
+            } else
+            for (int t0 = 0; t0 < p.taps; t0 += 8) {          // (very wide filters) 8 taps at a time: all bitmap loads first
                 uint32_t word[8];
                 int sh[8];
                 #pragma unroll
@@ -195,21 +221,25 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
                 const uint32_t As = base_u32 + stage * (uint32_t)TC_STAGE_BYTES;
                 if (p.kpp == 4) {
-                    // first layers (up to 4 channels = 4 bytes per pixel): a 16-byte piece holds 4 taps, copied one by one
+                    // first layers (up to 4 channels = 4 bytes per pixel): a 16-byte piece holds 4 taps, copied one by one;
+                    // where a tap sits relative to the row's first pixel is the same for all 8 rows
+                    int toff[4], tsh[4];
+                    bool tok[4], thi[4];
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int tap = ks * (TC_SLAB / 4) + piece * 4 + j;
+                        const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                        toff[j] = (ky * p.w + kx) * 4;
+                        tok[j] = tap < p.taps; thi[j] = tap >= 64; tsh[j] = tap & 63;
+                    }
                     #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const int r = warp * 32 + i * 4 + rsub;
-                        const unsigned long long rm0 = S->rmask[r][0], rm1 = S->rmask[r][1];
-                        const int pix0 = S->pix0[r];
-                        const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)((piece ^ (r & 7)) << 4);
                         #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const int tap = ks * (TC_SLAB / 4) + piece * 4 + j;
-                            const int ky = tap / p.kw, kx = tap - ky * p.kw;
-                            const bool use = tap < p.taps && ((tap < 64 ? rm0 >> tap : rm1 >> (tap - 64)) & 1ull);
-                            const unsigned char* src = use ? Ab + (size_t)(pix0 + ky * p.w + kx) * 4 : Ab;
+                            const bool use = tok[j] && (((thi[j] ? rm1[i] : rm0[i]) >> tsh[j]) & 1ull);
+                            const unsigned char* src = use ? Ab + (src_row[i] + toff[j]) : Ab;
                             asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;"
-                                         ::"r"(As + off + 4u * j), "l"(src), "r"(use ? 4u : 0u) : "memory");
+                                         ::"r"(As + dst_row[i] + 4u * j), "l"(src), "r"(use ? 4u : 0u) : "memory");
                         }
                     }
                 } else {
