@@ -590,7 +590,8 @@ def main():
             "clocks": clocks,
             "e2e": {"value": world * T * 1e3 / e2e_ms, "unit": "frames/s", "h2d_bytes_per_step": T * C_IN,
                     "d2h_bytes_per_step": T * 4 * C_OUT,
-                    "call": "rrm_step_seq_host_async per step, one rrm_host_sync after the last step",
+                    "call": "rrm_step_seq_host_async per step, one rrm_host_sync after the last step; steps back to back "
+                            "(no L2 flush between them, unlike `value`), timed on the host clock",
                     "value_waiting_every_call": world * T * 1e3 / e2e_sync_ms},
             "gpu_launches": args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
