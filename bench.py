@@ -172,7 +172,7 @@ def run_reference(args, rank, world):
 # One step = one frame through rrm_net_step (Algorithm 1, one iteration of the frame loop).
 # ------------------------------------------------------------------------------------------------
 CONV_WORKLOADS = ("cfg1", "cfg3_f32", "cfg3_i8", "cfg4", "cfg5")
-FFMA_TMACS, DP4A_TMACS, POPC_TBITMACS = 37.2, 74.5, 148.9      # derived ALU peaks: lanes x clock
+FFMA_TMACS, DP4A_TMACS, POPC_TBITMACS = 37.2, 74.5, 148.9      # derived ALU peaks in TMAC/s: lanes per SM x 148 SMs x 1.965 GHz (FFMA 128, dp4a 64 x 4, popc 16 x 32 bits)
 
 
 def conv_workload(name, frames=None, streams=None):
