@@ -294,13 +294,20 @@ int build_graph(rrm_net* net, int kind)
     return RRM_OK;
 }
 
+void drop_chunk_graphs(rrm_net* net, int kind)
+{
+    for (auto& c : net->chunk_graphs[kind]) {
+        if (c.exec) cudaGraphExecDestroy(c.exec);
+        if (c.graph) cudaGraphDestroy(c.graph);
+    }
+    net->chunk_graphs[kind].clear();
+}
+
 void drop_graphs(rrm_net* net)
 {
     for (int k = 0; k < 3; ++k) {
         net->patch_in[k].clear(); net->patch_out[k].clear(); net->patch_ok[k] = false;
-        if (net->chunk_exec[k]) { cudaGraphExecDestroy(net->chunk_exec[k]); net->chunk_exec[k] = nullptr; }
-        if (net->chunk_graph[k]) { cudaGraphDestroy(net->chunk_graph[k]); net->chunk_graph[k] = nullptr; }
-        net->chunk_T[k] = 0;
+        drop_chunk_graphs(net, k);
         if (net->exec[k]) { cudaGraphExecDestroy(net->exec[k]); net->exec[k] = nullptr; }
         if (net->graph[k]) { cudaGraphDestroy(net->graph[k]); net->graph[k] = nullptr; }
     }
@@ -413,6 +420,7 @@ int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st,
 }
 
 constexpr int CHUNK_MAX_SLOTS = 24;             // capture streams = frames in flight
+constexpr size_t CHUNK_GRAPHS_KEPT = 4;         // chunk lengths whose graphs are kept per kind
 constexpr int CHUNK_ARENAS = 64;                // arenas of the chunk graphs (>= CHUNK_MAX_SLOTS)
 
 // Streams, events, arenas and staging buffers of the pipelined chunk graphs.
@@ -448,11 +456,7 @@ int ensure_chunk(rrm_net* net, int T)
         RRM_TRY(dev_alloc(net, &net->chunk_in, (size_t)bi * T));
         RRM_TRY(dev_alloc(net, &net->chunk_out, (size_t)bo * T));
         net->chunk_cap = T;
-        for (int k = 0; k < 3; ++k) {                        // graphs hold the old buffers
-            if (net->chunk_exec[k]) { cudaGraphExecDestroy(net->chunk_exec[k]); net->chunk_exec[k] = nullptr; }
-            if (net->chunk_graph[k]) { cudaGraphDestroy(net->chunk_graph[k]); net->chunk_graph[k] = nullptr; }
-            net->chunk_T[k] = 0;
-        }
+        for (int k = 0; k < 3; ++k) drop_chunk_graphs(net, k);   // graphs hold the old buffers
     }
     return RRM_OK;
 }
@@ -525,11 +529,20 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
         cudaGetLastError();
         return status != RRM_OK ? status : RRM_ERR_CUDA;
     }
-    if (net->chunk_exec[kind]) { cudaGraphExecDestroy(net->chunk_exec[kind]); net->chunk_exec[kind] = nullptr; }
-    if (net->chunk_graph[kind]) cudaGraphDestroy(net->chunk_graph[kind]);
-    net->chunk_graph[kind] = g;
-    RRM_CUDA_TRY(cudaGraphInstantiate(&net->chunk_exec[kind], g, 0));
-    net->chunk_T[kind] = T;
+    // keep the few most recently used chunk lengths (a video's last chunk is usually shorter than the others)
+    auto& cache = net->chunk_graphs[kind];
+    if (cache.size() >= CHUNK_GRAPHS_KEPT) {
+        size_t old = 0;
+        for (size_t i = 1; i < cache.size(); ++i) if (cache[i].used < cache[old].used) old = i;
+        if (cache[old].exec) cudaGraphExecDestroy(cache[old].exec);
+        if (cache[old].graph) cudaGraphDestroy(cache[old].graph);
+        cache.erase(cache.begin() + old);
+    }
+    rrm_net::ChunkGraph c;
+    c.T = T; c.graph = g;
+    if (cudaGraphInstantiate(&c.exec, g, 0) != cudaSuccess) { cudaGraphDestroy(g); cudaGetLastError(); return RRM_ERR_CUDA; }
+    c.used = ++net->chunk_clock;
+    cache.push_back(c);
     if (getenv("RRM_DEBUG")) {
         size_t nodes = 0;
         cudaGraphGetNodes(g, nullptr, &nodes);
@@ -559,7 +572,11 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
         }
     }
     const int kind = !dense ? 0 : (stateless ? 2 : 1);
-    if (!net->chunk_exec[kind] || net->chunk_T[kind] != T) {
+    auto find = [&]() -> rrm_net::ChunkGraph* {
+        for (auto& c : net->chunk_graphs[kind]) if (c.T == T) return &c;
+        return nullptr;
+    };
+    if (!find()) {
         const int s = build_chunk_graph(net, kind, T);
         if (s != RRM_OK) {
             cudaGetLastError();
@@ -576,7 +593,9 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
     RRM_CUDA_TRY(cudaMemcpyAsync(net->chunk_in, frames, (size_t)bi * T, cudaMemcpyDeviceToDevice, st));
-    RRM_CUDA_TRY(cudaGraphLaunch(net->chunk_exec[kind], st));
+    rrm_net::ChunkGraph* cg = find();
+    cg->used = ++net->chunk_clock;
+    RRM_CUDA_TRY(cudaGraphLaunch(cg->exec, st));
     if (outs) RRM_CUDA_TRY(cudaMemcpyAsync(outs, net->chunk_out, (size_t)bo * T, cudaMemcpyDeviceToDevice, st));
     if (is_step && !dense && net->auto_switch) RRM_TRY(activity_read_back(net, st));
     return RRM_OK;

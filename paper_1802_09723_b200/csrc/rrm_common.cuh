@@ -174,9 +174,9 @@ struct rrm_net {
     std::vector<cudaEvent_t> ev_conv, ev_epi;     // per layer: the most recently captured convolution / epilogue
     std::vector<cudaEvent_t> ev_join;
     cudaEvent_t ev_fork = nullptr, ev_export = nullptr;
-    cudaGraph_t chunk_graph[3] = {nullptr, nullptr, nullptr};
-    cudaGraphExec_t chunk_exec[3] = {nullptr, nullptr, nullptr};
-    int chunk_T[3] = {0, 0, 0};
+    struct ChunkGraph { int T = 0; cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr; unsigned long long used = 0; };
+    std::vector<ChunkGraph> chunk_graphs[3];      // per kind (delta / keyframes / dense): the few most recently used chunk lengths
+    unsigned long long chunk_clock = 0;
     void* chunk_in = nullptr;
     void* chunk_out = nullptr;
     int chunk_cap = 0;                            // frames chunk_in / chunk_out hold
