@@ -361,3 +361,30 @@ def test_stack_chunks_through_the_pipelined_host_entry_point():
             want = orc.dense_forward(specs, video[4 * k + i])[0][len(specs)]
             np.testing.assert_array_equal(y[i].numpy().astype(np.int64), want, err_msg=f"frame {4 * k + i}")
     net.close()
+
+
+def test_stack_chunk_longer_than_the_arenas_held():
+    """More frames in one call than there are per-frame arenas: arenas are reused, each cleared by the frame that
+    takes it over; outputs and state are unchanged."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8", hw=67, scale=8)
+    video = wl.moving_rect_video(frames=71, hw=67, dtype="i8", seed=29, n=1, side=(8, 16))
+    net = rrm.net_from_specs(specs, n=1)
+    rec = orc.Recurrence(specs, n=1)
+    rec.step(np.full_like(video[0], 0))
+    frames = dev(np.ascontiguousarray(video))
+    outs = net.new_output(frames=70)
+    net.step_seq(frames[:70], outs, 70)
+    for t in range(70):
+        rec.step(video[t])
+        if t in (0, 1, 33, 64, 65, 69):
+            want = orc.dense_forward(specs, video[t])[0][len(specs)]
+            np.testing.assert_array_equal(outs[t].cpu().numpy().astype(np.int64), want, err_msg=f"frame {t}")
+    _compare(specs, net, video[69], 69)
+    for l in range(len(specs)):
+        st = net.stats(l)
+        assert st["error_word"] == 0 and st["nnz_elems"] == rec.nnz[l] and st["active_macs"] == rec.macs[l], (l, st)
+    out = net.new_output()
+    net.step(dev(video[70]), out)
+    _compare(specs, net, video[70], 70)
+    net.close()
