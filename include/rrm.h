@@ -141,7 +141,7 @@ int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* st
  * counters are the same integers either way.  The first call with a larger T than any before
  * allocates scratch memory (T * N * c_out * 4 bytes); later calls do not.
  * T * N must not exceed 65535.  Asynchronous on `stream`.  After the call rrm_get_stats reports the
- * counters summed over the chunk's frames. */
+ * counters summed over the chunk's frames (lone int8 FC layer) or those of the chunk's last frame (other layers). */
 int rrm_step_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream);
 /* T frames through the dense path, each on its own (Y_t = f(F*X_t + b)); RRM state untouched. */
 int rrm_dense_seq(rrm_layer* layer, const void* X_dev, void* Y_dev, int T, void* stream);
@@ -151,8 +151,8 @@ int rrm_step_seq_host(rrm_layer* layer, const void* X_host, void* Y_host, int T,
  * copy-out of a call run on three streams (two of them the library's own) chained by events, through two
  * staging slots, so that consecutive calls overlap: chunk k+1 is copied in and chunk k-1 copied out while
  * chunk k is computed.  X_host and Y_host should be page-locked (pageable memory makes the copies
- * synchronous); X_host must stay unchanged and Y_host unread until rrm_host_sync (or a later call to
- * rrm_step_seq_host on the same layer) has returned.  Calls must be issued from one thread, in frame order;
+ * synchronous); X_host must stay unchanged and Y_host unread until rrm_host_sync has returned.  Calls must be
+ * issued from one thread, in frame order;
  * the RRM state advances in that order on `stream`.  The first call, and a call with a larger T than any
  * before, allocate the staging slots. */
 int rrm_step_seq_host_async(rrm_layer* layer, const void* X_host, void* Y_host, int T, void* stream);
