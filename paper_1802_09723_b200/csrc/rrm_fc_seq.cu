@@ -438,7 +438,7 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
             L.seq_ev_pending = false;
         }
         cudaGetLastError();                                  // cudaErrorNotReady from the query is not an error
-        // (up to 1024 rows go through the streaming form, 128 rows per launch, each launch at the cost of reading W
+        // (up to 1024 rows go through the streaming form, 256 rows per launch, each launch at the cost of reading W
         // once: it wins as soon as the rows' gathered columns add up to about that many bytes)
         const bool use_dense = L.tc_ready && L.d.variant == RRM_VARIANT_AUTO && (long long)T * n >= 8 &&
                                (fc_tc_usable(L, T * n) ? L.seq_density * T * n >= SQ_DENSE_SWITCH_ROWS * fc_tc_launches(T * n)

@@ -4,7 +4,7 @@
 // The weights are the M operand: a CTA owns 128 outputs and a share of K and streams its slice of W
 // through a deep ring of stages.  A stage holds one 128-byte slab of K: 16 KB of W, filled by one bulk
 // copy of the pre-swizzled tile image the tensor-core convolution already keeps, and the same slab of
-// the input rows (the N operand, 16 to 128 rows), which the copy engine takes straight from the
+// the input rows (the N operand, 16 to 256 rows), which the copy engine takes straight from the
 // caller's [rows][c_in] array through a tensor map that applies the 128-byte swizzle and zero-fills
 // rows and channels past the end.  With W read exactly once the launch is bound by HBM: c_out x c_in bytes.
 // The int32 accumulators leave tensor memory transposed (thread = output, register = row), so for every
@@ -24,8 +24,8 @@ constexpr int FT_THREADS = 192;               // warps 0-3: snapshot, then epilo
 constexpr int FT_SLAB = 128;                  // bytes of K per stage
 constexpr int FT_A_BYTES = TC_M * FT_SLAB;    // the W part of a stage
 constexpr int FT_MAX_STAGES = 12;
-constexpr int FT_MAX_ROWS = 128;              // input rows of one launch
-constexpr int FT_MAX_LAUNCHES = 8;            // more rows than this many launches hold go to the convolution kernel
+constexpr int FT_MAX_ROWS = 256;              // input rows of one launch (the N of one MMA, and the accumulator's columns)
+constexpr int FT_MAX_LAUNCHES = 4;            // more rows than this many launches hold go to the convolution kernel
 constexpr size_t FT_SMEM_BUDGET = 220 * 1024;
 
 struct FtSmemTail {
@@ -405,7 +405,7 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
         const int piece = rows - r0 < piece_max ? rows - r0 : piece_max;
         p.rows = piece;
         p.bn = (piece + 15) & ~15;
-        p.tmem_cols = p.bn <= 32 ? 32 : (p.bn <= 64 ? 64 : 128);
+        p.tmem_cols = p.bn <= 32 ? 32 : (p.bn <= 64 ? 64 : (p.bn <= 128 ? 128 : 256));
         const size_t stage_bytes = (size_t)FT_A_BYTES + (size_t)p.bn * FT_SLAB;
         const int stages = (int)(FT_SMEM_BUDGET / stage_bytes);
         p.stages = stages > FT_MAX_STAGES ? FT_MAX_STAGES : stages;
