@@ -253,6 +253,97 @@ def test_mac_accounting_follows_table_1():
     assert orc.delta_accumulate(cv, D, P) == 4 * 5
 
 
+def _golden(name):
+    vals = {}
+    for line in open(os.path.join(GOLDEN, name)):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, *nums = line.split()
+        vals[key] = np.array([int(v) for v in nums])
+    return vals
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f32"])
+def test_fc_delta_hand_computed_fixture(dtype):
+    """FC branch of Algorithm 1's update on a 3 x 4 matrix whose rows, columns and streams all differ, so a
+    transposed weight index, a swapped stream / input index or a dropped entry changes the result."""
+    v = _golden("hand_fc_delta.txt")
+    fc = LayerSpec("fc", dtype, 4, 1, 1, 3, src=0)
+    fc.weight = v["weight"].reshape(3, 4, 1, 1).astype(np.float32 if dtype == "f32" else np.int8)
+    fc.bias = np.zeros(3, dtype=np.float32 if dtype == "f32" else np.int32)
+    dt = np.float64 if dtype == "f32" else np.int64
+    P = v["p_prev"].reshape(2, 3).astype(dt)
+    macs = orc.delta_accumulate(fc, v["delta"].reshape(2, 4).astype(dt), P)
+    np.testing.assert_array_equal(P.ravel(), v["p_next"].astype(dt))
+    assert macs == int(v["macs"][0])
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f32"])
+def test_fc_delta_equals_matrix_product_of_the_delta(dtype):
+    """Eq. 4 for the FC case: the column-by-column update onto zeros is W dI.  Checked against numpy's
+    matmul (a library routine) and against the dense FC definition without bias, on a ragged c_in x c_out
+    with several streams and mostly-zero deltas."""
+    rng = np.random.default_rng(77)
+    c_in, c_out, n = 37, 13, 3
+    fc = _spec(dtype, c_in, 1, 1, c_out, 1, 1, 0, rng, kind="fc")
+    dt = np.float64 if dtype == "f32" else np.int64
+    D = np.zeros((n, c_in), dtype=dt)
+    for s in range(n):
+        idx = rng.choice(c_in, size=4 + 3 * s, replace=False)
+        D[s, idx] = rng.standard_normal(idx.size) if dtype == "f32" else rng.integers(-254, 255, size=idx.size)
+    P = np.zeros((n, c_out), dtype=dt)
+    macs = orc.delta_accumulate(fc, D, P)
+    Wm = fc.weight.reshape(c_out, c_in).astype(dt)
+    ref = D @ Wm.T
+    nobias = orc.projection(fc, D, with_bias=False).reshape(n, c_out)
+    if dtype == "f32":
+        np.testing.assert_allclose(P, ref, rtol=0, atol=1e-12 * np.abs(ref).max())
+        np.testing.assert_allclose(P, nobias, rtol=0, atol=1e-12 * np.abs(ref).max())
+    else:
+        np.testing.assert_array_equal(P, ref)
+        np.testing.assert_array_equal(P, nobias)
+    assert macs == int(np.count_nonzero(D)) * c_out
+    # an update onto a non-zero projection adds to it (Eq. 5), stream by stream
+    P0 = (rng.standard_normal((n, c_out)) if dtype == "f32" else rng.integers(-1000, 1000, size=(n, c_out))).astype(dt)
+    P1 = P0.copy()
+    orc.delta_accumulate(fc, D, P1)
+    if dtype == "f32":
+        np.testing.assert_allclose(P1 - P0, ref, rtol=0, atol=1e-12 * np.abs(ref).max())
+    else:
+        np.testing.assert_array_equal(P1 - P0, ref)
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f32"])
+def test_fc_recurrence_equals_dense_at_every_frame(dtype):
+    """Algorithm 1 on a lone FC layer (and on an FC -> FC pair) against the dense definition, 5 frames."""
+    rng = np.random.default_rng(12)
+    c_in, c_mid, c_out, n = 48, 20, 9, 2
+    a = _spec(dtype, c_in, 1, 1, c_mid, 1, 1, 0, rng, kind="fc", act="relu", shift=6 if dtype == "i8" else -1)
+    b = _spec(dtype, c_mid, 1, 1, c_out, 1, 1, 0, rng, kind="fc")
+    b.src = 1
+    for layers in ([a], [a, b]):
+        rec = orc.Recurrence(layers, n=n)
+        x = (rng.standard_normal((n, c_in)).astype(np.float32) if dtype == "f32"
+             else rng.integers(0, 128, size=(n, c_in)).astype(np.int8))
+        for t in range(5):
+            if t:
+                j = rng.choice(c_in, size=5, replace=False)
+                x = x.copy()
+                x[:, j] = (rng.standard_normal((n, 5)).astype(np.float32) if dtype == "f32"
+                           else rng.integers(0, 128, size=(n, 5)).astype(np.int8))
+            tens_r, P_r = rec.step(x)
+            tens_d, P_d = orc.dense_forward(layers, x)
+            for l in range(len(layers)):
+                if dtype == "f32":
+                    assert np.abs(P_r[l] - P_d[l]).max() <= 1e-11 * max(1.0, np.abs(P_d[l]).max())
+                else:
+                    np.testing.assert_array_equal(P_r[l], P_d[l])
+            if dtype != "f32":
+                np.testing.assert_array_equal(tens_r[-1], tens_d[-1])
+            if t:
+                assert rec.nnz[0] <= 5 * n and rec.macs[0] == rec.nnz[0] * c_mid
+
+
 def test_int32_accumulator_bound():
     # worst case of the largest contraction used here (fc6: 9216 inputs of magnitude <= 127)
     assert 9216 * 127 * 127 < 2 ** 31
