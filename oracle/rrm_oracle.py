@@ -78,11 +78,32 @@ def _out_dim(i, k, s, p):
 
 
 # --------------------------------------------------------------------- linear part
+_promoted = []      # [(weight array, element type, promoted copy)], most recently used last
+
+
+def _weights(spec, dt):
+    """The layer's filters in the oracle's element type.  The C routines take fp64 / int64 arrays; promoting a
+    large filter bank (fc6: 37.7 M int8 -> 302 MB of int64) costs far more than the recurrence's own work, so
+    the promoted copy of a large, unchanged weight array is kept between calls.  Small arrays are promoted
+    every time (tests edit them in place)."""
+    w = spec.weight
+    if w.size < (1 << 20):
+        return np.ascontiguousarray(w, dtype=dt)
+    for i, (src, t, F) in enumerate(_promoted):
+        if src is w and t == dt:
+            _promoted.append(_promoted.pop(i))
+            return F
+    F = np.ascontiguousarray(w, dtype=dt)
+    _promoted.append((w, dt, F))
+    del _promoted[:-3]
+    return F
+
+
 def projection(spec, I, with_bias=True):
     """Eq. 3: P = F*I + b (conv) or W I + b (FC).  I: [N,C,H,W] (FC: [N,C] or [N,C,1,1])."""
     t, dt = _kind(spec)
     I = np.ascontiguousarray(I, dtype=dt)
-    F = np.ascontiguousarray(spec.weight, dtype=dt)
+    F = _weights(spec, dt)
     b = np.ascontiguousarray(spec.bias, dtype=dt) if with_bias else None
     N = I.shape[0]
     if spec.kind == "fc":
@@ -104,7 +125,7 @@ def delta_accumulate(spec, D, P):
     Updates P in place; returns the multiply-accumulates executed."""
     t, dt = _kind(spec)
     D = np.ascontiguousarray(D, dtype=dt)
-    F = np.ascontiguousarray(spec.weight, dtype=dt)
+    F = _weights(spec, dt)
     assert P.dtype == dt and P.flags["C_CONTIGUOUS"]
     N = D.shape[0]
     if spec.kind == "fc":
