@@ -1,20 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the RRM hot path on B200.
 
-Workload: the int8 delta-FC configuration (AlexNet-fc6 shape 9216 -> 4096, int32 accumulation,
-32-frame sequences whose frames differ in a fraction rho of the inputs, changed entries in runs
-of 32).  One "step" = one chunk of 32 consecutive frames of one stream through the whole hot path
-of the layer (delta + compaction, column-gather product, accumulate + snapshot + output for every
-frame), i.e. one rrm_step_seq call = one kernel launch; the reported value is frames per second.
-Secondary numbers: the same with one frame per call (rrm_step), the library's dense path, other
-densities, several streams per call.
+Workload of the contract line: the int8 delta-FC configuration (AlexNet-fc6 shape 9216 -> 4096, int32
+accumulation, 32-frame sequences whose frames differ in a fraction rho of the inputs, changed entries in runs
+of 32).  One "step" = one chunk of 32 consecutive frames of one stream through the whole hot path of the layer
+(delta + compaction, sparse product, accumulate + snapshot + output for every frame), i.e. one rrm_step_seq call
+= one kernel launch; the reported value is frames per second.  The line also carries, under "conv", compact
+results of the convolution configurations (cfg1, cfg3 int8, cfg4) and, under "by_rho" / "roofline_delta_fc",
+the column-gather kernel forced at 1 / 5 / 20 % density.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--rho 0.05] [--chunk 32] [--impl ours|reference]
+  python bench.py --workload cfg1|cfg3_f32|cfg3_i8|cfg4|cfg5 [--streams N] [--seq T] [--variant auto|tensor|gather]
 
-Timing: every timed step is preceded by an untimed L2 flush (a 256 MiB device write), and is
-bracketed by its own CUDA event pair on the launching stream; ms_per_step is the mean of those
-K durations, max over ranks.  N > 1 runs N independent replicas (one video stream and one layer
-state per GPU, no data-path collective): weak scaling.
+Timing: every timed step is preceded by an untimed L2 flush (a 256 MiB device write) and bracketed by its own
+CUDA event pair on the launching stream; ms_per_step is the MEDIAN of those K durations (mean, min and max are
+printed beside it), max over ranks.  N > 1 runs N independent replicas (one video stream and one layer state
+per GPU, no data-path collective): weak scaling.
 """
 import argparse
 import json
@@ -57,6 +58,13 @@ def max_over_ranks(ms, world, device=None):
     return float(t.item())
 
 
+def summarize(times_ms):
+    """Median (the reported figure: robust against a few slow early steps), mean, min, max of per-step durations."""
+    a = np.asarray(times_ms, dtype=np.float64)
+    return {"median": float(np.median(a)), "mean": float(a.mean()), "min": float(a.min()), "max": float(a.max()),
+            "n": int(a.size)}
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -75,6 +83,19 @@ def measured_tensor_tmacs():
         return float(json.load(open(p))["bf16_tflops"]), "measured"
     except Exception:  # noqa: BLE001
         return 1590.0, "fallback"
+
+
+_ALU = {}
+
+
+def alu_peaks():
+    """FFMA / dp4a / popc peaks in TMAC/s (T bit-MAC/s for popc), measured once per process by the library's
+    micro-kernels (rrm_measure_alu_peak) on the current device."""
+    if not _ALU:
+        import paper_1802_09723_b200 as rrm
+        for k in ("ffma", "dp4a", "popc"):
+            _ALU[k] = rrm.measure_alu_peak(k) / 1e12
+    return dict(_ALU)
 
 
 def committed_traffic(kernel, rho):
@@ -133,9 +154,52 @@ class ClockSampler:
                 "samples": len(mhz)}
 
 
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places where bench.py executes anything under oracle/)
+# ------------------------------------------------------------------------------------------------
+def cpu_fc_baseline(spec, seq, order, budget_s=10.0, max_frames=None):
+    """The oracle's Algorithm-1 recurrence and its dense definition on frames of the same sequence, timed on the
+    host cores.  Returns (recurrence frames/s, frames, dense frames/s, frames, threads)."""
+    from oracle import rrm_oracle as orc
+    period = len(order)
+    rec = orc.Recurrence([spec])
+    rec.step(seq[order[0]])                                   # also promotes the weights once (setup, untimed)
+    orc.dense_forward([spec], seq[order[0]])
+    t0 = time.perf_counter()
+    cnt = 0
+    while (max_frames is None or cnt < max_frames) and time.perf_counter() - t0 < budget_s:
+        rec.step(seq[order[(cnt + 1) % period]])
+        cnt += 1
+    dt = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    dcnt = 0
+    while dcnt < max(4, cnt // 4) and time.perf_counter() - t0 < budget_s / 2:
+        orc.dense_forward([spec], seq[order[(dcnt + 1) % period]])
+        dcnt += 1
+    ddt = time.perf_counter() - t0
+    return cnt / dt, cnt, dcnt / ddt, dcnt, orc.threads()
+
+
+def cpu_stack_baseline(specs, video, n, frames=2):
+    """ms per frame (of every stream) of the oracle's recurrence and of its dense definition on a stack."""
+    from oracle import rrm_oracle as orc
+    rec = orc.Recurrence(specs, n=n)
+    rec.reset_to(video[0])
+    t0 = time.perf_counter()
+    for t in range(1, 1 + frames):
+        rec.step(video[t])
+    ms_rec = (time.perf_counter() - t0) * 1e3 / frames
+    t0 = time.perf_counter()
+    orc.dense_forward(specs, video[1])
+    ms_dense = (time.perf_counter() - t0) * 1e3
+    return {"recurrence_ms_per_frame": ms_rec, "dense_ms_per_frame": ms_dense, "value": n * 1e3 / ms_rec,
+            "dense_value": n * 1e3 / ms_dense, "unit": "frames/s", "cores": orc.threads(), "kind": "oracle",
+            "sample": f"{frames} delta frames after a dense start, and 1 dense frame, of the same video"}
+
+
 def run_reference(args, rank, world):
-    """The CPU oracle, as it stands, on the host cores (rank 0 only).  One reference step is a bounded
-    sample of the GPU arm's step: ONE frame of the chunk; ms_per_step is scaled to a whole chunk."""
+    """The CPU oracle, as it stands, on the host cores (rank 0 only).  One reference step = one chunk of --chunk
+    frames of the same sequence through the oracle's Algorithm-1 recurrence, as in the GPU arm."""
     if rank != 0:
         return
     import workloads as wl
@@ -143,36 +207,47 @@ def run_reference(args, rank, world):
     spec = wl.fc6_i8()[0]
     seq = wl.fc_run_sequence(frames=FRAMES, rho=args.rho, seed=21)
     order = pingpong(FRAMES)
+    period = len(order)
+    T = args.chunk
     rec = orc.Recurrence([spec])
     rec.step(seq[0])
-    for i in range(args.warmup):
-        rec.step(seq[order[(i + 1) % len(order)]])
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        rec.step(seq[order[(args.warmup + i + 1) % len(order)]])
-    dt = time.perf_counter() - t0
-    fps = args.steps / dt
+    pos = 0
+
+    def chunk():
+        nonlocal pos
+        for _ in range(T):
+            pos += 1
+            rec.step(seq[order[pos % period]])
+
+    for _ in range(args.warmup):
+        chunk()
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        chunk()
+        times.append((time.perf_counter() - t0) * 1e3)
+    tm = summarize(times)
+    fps = T * 1e3 / tm["median"]
     print(json.dumps({
         "impl": "reference", "metric": "frames_per_sec", "value": fps, "unit": "frames/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps * args.chunk,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": tm["median"], "ms_per_step_stats": tm,
         "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "i8", "data": "synthetic",
         "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream; one step = one chunk "
-                               f"of {args.chunk} consecutive frames", "frames_per_step": args.chunk},
+                               f"of {T} consecutive frames", "frames_per_step": T},
         "dense_equiv_gmacs": fps * DENSE_MACS / 1e9,
         "cpu_baseline": {"value": fps, "unit": "frames/s", "cores": orc.threads(), "kind": "oracle",
-                         "sample": f"1 frame per step ({args.steps} frames of the same sequence) through the oracle's "
-                                   f"Algorithm-1 recurrence; ms_per_step scaled to {args.chunk} frames"},
+                         "sample": f"{args.steps} chunks of {T} frames of the same sequence through the oracle's "
+                                   f"Algorithm-1 recurrence (weights promoted to int64 once, before the timed region)"},
         "e2e": {"value": fps, "unit": "frames/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
 # ------------------------------------------------------------------------------------------------
-# Secondary workloads (the convolution configurations): python bench.py --workload cfg1|cfg3_f32|...
-# One step = one frame through rrm_net_step (Algorithm 1, one iteration of the frame loop).
+# Convolution configurations.  One step = one frame of every stream through rrm_net_step (Algorithm 1, one
+# iteration of the frame loop).
 # ------------------------------------------------------------------------------------------------
 CONV_WORKLOADS = ("cfg1", "cfg3_f32", "cfg3_i8", "cfg4", "cfg5")
-FFMA_TMACS, DP4A_TMACS, POPC_TBITMACS = 37.2, 74.5, 148.9      # derived ALU peaks in TMAC/s: lanes per SM x 148 SMs x 1.965 GHz (FFMA 128, dp4a 64 x 4, popc 16 x 32 bits)
 
 
 def conv_workload(name, frames=None, streams=None):
@@ -198,17 +273,17 @@ def conv_workload(name, frames=None, streams=None):
     raise SystemExit(f"unknown workload {name}")
 
 
-def run_conv(args):
+def conv_measure(name, variant="auto", steps=60, warmup=5, frames=None, streams=None, seq=None, cpu_frames=0,
+                 sample_clocks=True):
+    """Times one convolution configuration: delta steps (cold and warm L2), the library's own dense path, per-layer
+    densities, Eq. 9 / Eq. 10, the roofline of the step; optionally chunks of `seq` frames and a CPU oracle sample."""
     import torch
     import workloads as wl
     import paper_1802_09723_b200 as rrm
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    specs, video, n, dtype = conv_workload(args.workload, args.frames, args.streams)
+    specs, video, n, dtype = conv_workload(name, frames, streams)
     F = video.shape[0]
-    net = rrm.net_from_specs(specs, n=n, variant=args.variant)
-    frames = [torch.from_numpy(np.ascontiguousarray(video[t])).cuda() for t in range(F)]
+    net = rrm.net_from_specs(specs, n=n, variant=variant)
+    fr = [torch.from_numpy(np.ascontiguousarray(video[t])).cuda() for t in range(F)]
     order = pingpong(F)
     period = len(order)
     out = net.new_output()
@@ -216,120 +291,187 @@ def run_conv(args):
     stream = torch.cuda.current_stream()
     dense_macs = wl.dense_macs(specs) * n
 
-    def timed(call, steps, warmup, cold=True):
-        net.keyframe(frames[order[0]], out)
-        for i in range(warmup):
-            call(frames[order[(i + 1) % period]], out)
+    def timed(call, k, w, cold=True):
+        net.keyframe(fr[order[0]], out)
+        for i in range(w):
+            call(fr[order[(i + 1) % period]], out)
         torch.cuda.synchronize()
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        for i in range(steps):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
+        for i in range(k):
             if cold:
                 flush.fill_(i & 0xff)
             evs[i][0].record(stream)
-            call(frames[order[(warmup + i + 1) % period]], out)
+            call(fr[order[(w + i + 1) % period]], out)
             evs[i][1].record(stream)
         torch.cuda.synchronize()
-        return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+        return summarize([a.elapsed_time(b) for a, b in evs])
 
-    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
-    sampler.start()
-    ms = timed(net.step, args.steps, args.warmup)
-    clocks = sampler.stop()
-    per_layer = []
-    tot_active = 0
-    for l, sp in enumerate(specs):
-        st = net.stats(l)
-        if st["variant"] == 3:                # the last frame was evaluated densely (high measured activity): nothing counted
-            tot_active = None
-            per_layer.append({"layer": sp.name, "variant": "dense (measured activity >= 75 %)", "dense_macs": st["dense_macs"]})
-            continue
-        tot_active += st["active_macs"]
-        per_layer.append({"layer": sp.name, "rho": st["nnz_elems"] / max(1, st["in_elems"]),
-                          "active_in_pixels": st["active_in_pixels"] / max(1, st["in_pixels"]),
-                          "active_out_pixels": st["active_out_pixels"] / max(1, st["out_pixels"]),
-                          "active_macs": st["active_macs"], "dense_macs": st["dense_macs"], "variant": st["variant"]})
-    # ---- roofline of the last timed step: per layer the slower of (MACs executed at the unit's peak) and (bytes that
-    # have to move at the HBM peak), summed over the layers, against the measured step time.  Bytes per layer: the delta
-    # rows of the active input pixels once + the projection rows of the pixels to update three times (read and write
-    # by the convolution, read by the epilogue); weights stay in L2 and are left out.
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0"))) if sample_clocks else None
+    if sampler:
+        sampler.start()
+    tm = timed(net.step, steps, warmup)
+    clocks = sampler.stop() if sampler else None
+    ms = tm["median"]
+    # ---- per-layer counters of the last timed step, Eq. 9 (overall sparsity, MAC-weighted) and Eq. 10 (speedup ratio)
     hbm, hbm_kind = measured_peaks()
     tens, tens_kind = measured_tensor_tmacs()
+    alu = alu_peaks()
     unit_bytes = {"f32": 4.0, "i8": 1.0, "bin": 1.0 / 8}
-    mac_peak = {"f32": FFMA_TMACS, "i8": tens, "bin": tens}         # TMAC/s (int8 and binary layers run on the tensor cores)
+    per_layer, stats = [], []
+    tot_active = 0
+    num_hat = num_in = den = 0.0
     roof_us = mac_us = byte_us = 0.0
     for l, sp in enumerate(specs):
         st = net.stats(l)
+        stats.append(st)
         dense_step = st["variant"] == 3
+        # density of the layer input itself (what a sparse engine without RRM would see): non-zero share of the
+        # tensor the layer reads (binary tensors have no zeros)
+        if sp.dtype == "bin":
+            rho_in = 1.0
+        else:
+            src = net.tensor(sp.src if sp.src >= 0 else l)
+            rho_in = float(torch.count_nonzero(src).item()) / src.numel()
+        entry = {"layer": sp.name, "dense_macs": st["dense_macs"], "rho_input": rho_in,
+                 "variant": {1: "gather", 2: "tensor", 3: "dense"}.get(st["variant"], "?")}
+        if dense_step:
+            tot_active = None
+            entry["note"] = "evaluated densely (measured activity above the switch): no delta counters"
+        else:
+            if tot_active is not None:
+                tot_active += st["active_macs"]
+            entry.update({"rho": st["nnz_elems"] / max(1, st["in_elems"]),
+                          "active_in_pixels": st["active_in_pixels"] / max(1, st["in_pixels"]),
+                          "active_out_pixels": st["active_out_pixels"] / max(1, st["out_pixels"]),
+                          "active_macs": st["active_macs"]})
+            num_hat += entry["rho"] * st["dense_macs"]
+        num_in += rho_in * st["dense_macs"]
+        den += st["dense_macs"]
+        # roofline of this layer: the slower of (MACs executed at the unit's peak) and (bytes that have to move at the
+        # HBM peak).  Bytes: delta rows of the active input pixels once + projection rows of the pixels to update
+        # three times (read and write by the convolution, read by the epilogue); weights stay in L2 and are left out.
         macs = st["dense_macs"] if dense_step else st["active_macs"]
         fin = 1.0 if dense_step else st["active_in_pixels"] / max(1, st["in_pixels"])
         fout = 1.0 if dense_step else st["active_out_pixels"] / max(1, st["out_pixels"])
-        peak_l = mac_peak[sp.dtype] if (sp.dtype == "f32" or st["variant"] in (2, 3)) else (DP4A_TMACS if sp.dtype == "i8" else POPC_TBITMACS)
+        on_tensor = sp.dtype != "f32" and st["variant"] in (2, 3)
+        peak_l = tens if on_tensor else {"f32": alu["ffma"], "i8": alu["dp4a"], "bin": alu["popc"]}[sp.dtype]
         t_mac = macs / (peak_l * 1e12) * 1e6
         nbytes = st["in_pixels"] * fin * sp.c_in * unit_bytes[sp.dtype] + st["out_pixels"] * fout * sp.c_out * 4 * (2 if dense_step else 3)
         t_byte = nbytes / (hbm * 1e9) * 1e6
-        per_layer[l]["roofline_us"] = max(t_mac, t_byte)
-        per_layer[l]["roofline_bound"] = "hbm" if t_byte >= t_mac else ("alu" if sp.dtype == "f32" else "tensor")
+        entry["roofline_us"] = max(t_mac, t_byte)
+        entry["roofline_bound"] = "hbm" if t_byte >= t_mac else ("tensor" if on_tensor else "alu")
         roof_us += max(t_mac, t_byte); mac_us += t_mac; byte_us += t_byte
-    roofline = {"bound": "hbm" if byte_us >= mac_us else ("alu" if dtype == "f32" else "tensor"),
-                "achieved": roof_us * 1e-3 / ms * (hbm if byte_us >= mac_us else (FFMA_TMACS if dtype == "f32" else tens)),
-                "peak": hbm if byte_us >= mac_us else (FFMA_TMACS if dtype == "f32" else tens),
-                "unit": "GB/s" if byte_us >= mac_us else "TMAC/s", "frac": roof_us * 1e-3 / ms, "traffic": None,
-                "peak_kind": f"of {hbm_kind if byte_us >= mac_us else ('derived' if dtype == 'f32' else tens_kind)}",
+        per_layer.append(entry)
+    all_delta = tot_active is not None
+    eq = {"S0_without_rrm": 1.0 - num_in / den,
+          "S_with_rrm": (1.0 - num_hat / den) if all_delta else None,
+          "eta_eq10": (num_in / num_hat) if all_delta and num_hat > 0 else None,
+          "dense_over_active_macs": (dense_macs / tot_active) if all_delta and tot_active else None,
+          "note": "Eq. 9: MAC-weighted sparsity of the layer inputs (S0) and of their deltas (S); Eq. 10: eta = sum(rho MACs) / "
+                  "sum(rho_hat MACs); dense_over_active_macs uses the exact MAC count instead of Table 1's rho x dense MACs"}
+    mac_bound = byte_us < mac_us
+    peak = (alu["ffma"] if dtype == "f32" else tens) if mac_bound else hbm
+    roofline = {"bound": ("alu" if dtype == "f32" else "tensor") if mac_bound else "hbm",
+                "achieved": roof_us * 1e-3 / ms * peak, "peak": peak, "unit": "TMAC/s" if mac_bound else "GB/s",
+                "frac": roof_us * 1e-3 / ms, "traffic": None,
+                "peak_kind": f"of {('measured by rrm_measure_alu_peak' if dtype == 'f32' else tens_kind) if mac_bound else hbm_kind}",
                 "roofline_us_per_step": roof_us, "mac_us": mac_us, "byte_us": byte_us,
                 "note": "sum over the layers of max(executed MACs at the unit's peak, algorithmic bytes at the HBM peak) / "
-                        "measured step time; per-layer figures in per_layer_last_step"}
-    ms_warm = timed(net.step, args.steps, args.warmup, cold=False)
-    ms_dense = timed(net.dense, max(8, args.steps // 4), 3)
-    # ---- chunks of --seq consecutive frames per call (rrm_net_step_seq: the frames of a chunk overlap layer by layer)
-    seq_extra = {}
-    if args.seq and args.seq > 1:
-        Tq = args.seq
+                        "median step time; traffic: no ncu capture of a whole step"}
+    tm_warm = timed(net.step, max(8, steps // 2), 3, cold=False)
+    tm_dense = timed(net.dense, max(8, steps // 3), 3)
+    res = {
+        "workload": name, "streams": n, "variant_requested": variant, "frames_in_video": F,
+        "ms_per_step": ms, "ms_per_step_stats": tm, "frames_per_sec": n * 1e3 / ms,
+        "ms_per_step_warm": tm_warm["median"], "ms_per_step_dense_path": tm_dense["median"],
+        "speedup_vs_own_dense": tm_dense["median"] / ms,
+        "dense_equiv_gmacs": dense_macs / ms / 1e6,
+        "active_macs_last_step": tot_active, "dense_macs_per_step": dense_macs,
+        "eq9_eq10": eq, "roofline": roofline, "per_layer_last_step": per_layer, "clocks": clocks, "dtype": dtype,
+        "alu_peaks_tmacs": alu,
+    }
+    # ---- chunks of `seq` consecutive frames per call (rrm_net_step_seq: the frames of a chunk overlap layer by layer)
+    if seq and seq > 1:
+        Tq = seq
         total = period * Tq // np.gcd(period, Tq)
-        walk = torch.stack([frames[order[(i + 1) % period]] for i in range(total)])     # frame i+1 of the walk
+        walk = torch.stack([fr[order[(i + 1) % period]] for i in range(total)])     # frame i+1 of the walk
         outs = net.new_output(frames=Tq)
         nchunks = total // Tq
 
-        def timed_seq(call, steps, warmup):
-            net.keyframe(frames[order[0]], out)
-            for i in range(warmup):
+        def timed_seq(call, k, w):
+            net.keyframe(fr[order[0]], out)
+            for i in range(w):
                 call(walk[(i % nchunks) * Tq:(i % nchunks + 1) * Tq], outs, Tq)
             torch.cuda.synchronize()
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-            for i in range(steps):
-                k = (warmup + i) % nchunks
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
+            for i in range(k):
+                c = (w + i) % nchunks
                 flush.fill_(i & 0xff)
                 evs[i][0].record(stream)
-                call(walk[k * Tq:(k + 1) * Tq], outs, Tq)
+                call(walk[c * Tq:(c + 1) * Tq], outs, Tq)
                 evs[i][1].record(stream)
             torch.cuda.synchronize()
-            return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+            return summarize([a.elapsed_time(b) for a, b in evs])["median"]
 
-        steps_q = max(4, args.steps // Tq)
+        steps_q = max(4, steps // Tq)
         # (18 warm-up chunks: a large stack measures its activity with one delta chunk after 15 dense ones, and both
         # chunk graphs are to be captured before the timed region)
         ms_seq = timed_seq(net.step_seq, max(steps_q, 16), 18)
         ms_seq_dense = timed_seq(net.dense_seq, steps_q, 3)
-        seq_extra = {"seq": {"frames_per_call": Tq, "ms_per_call": ms_seq, "ms_per_frame_step": ms_seq / Tq,
-                             "frames_per_sec": n * Tq * 1e3 / ms_seq, "dense_ms_per_call": ms_seq_dense,
-                             "dense_frames_per_sec": n * Tq * 1e3 / ms_seq_dense,
-                             "speedup_vs_own_dense": ms_seq_dense / ms_seq,
-                             "speedup_vs_frame_by_frame": ms * Tq / ms_seq}}
-    line = {
-        "metric": "frames_per_sec", "value": n * 1e3 / ms, "unit": "frames/s", "n_gpus": 1, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": dtype, "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {len(specs)} conv layers, {n} stream(s), {F}-frame video walked back and forth; "
-                               f"one step = one frame of every stream through rrm_net_step", "variant": args.variant,
-                   "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair"},
-        "dense_equiv_gmacs": n * 1e3 / ms * (dense_macs / n) / 1e9,
-        "ms_per_step_warm": ms_warm, "ms_per_step_dense_path": ms_dense, "speedup_vs_own_dense": ms_dense / ms,
-        "active_macs_last_step": tot_active, "dense_macs_per_step": dense_macs,
-        "active_gmacs_per_s": None if tot_active is None else tot_active / ms / 1e6,
-        "clocks": clocks, "roofline": roofline, "per_layer_last_step": per_layer,
-    }
-    line.update(seq_extra)
-    print(json.dumps(line))
+        res["seq"] = {"frames_per_call": Tq, "ms_per_call": ms_seq, "ms_per_frame_step": ms_seq / Tq,
+                      "frames_per_sec": n * Tq * 1e3 / ms_seq, "dense_ms_per_call": ms_seq_dense,
+                      "dense_frames_per_sec": n * Tq * 1e3 / ms_seq_dense,
+                      "speedup_vs_own_dense": ms_seq_dense / ms_seq,
+                      "speedup_vs_frame_by_frame": ms * Tq / ms_seq}
     net.close()
+    del fr, flush
+    torch.cuda.empty_cache()
+    if cpu_frames:
+        res["cpu_baseline"] = cpu_stack_baseline(specs, video, n, cpu_frames)
+    return res
+
+
+def run_conv(args):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    r = conv_measure(args.workload, args.variant, args.steps, args.warmup, args.frames, args.streams, args.seq,
+                     cpu_frames=0 if args.quick else 2)
+    n = r["streams"]
+    line = {
+        "metric": "frames_per_sec", "value": r["frames_per_sec"], "unit": "frames/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "ms_per_step_stats": r["ms_per_step_stats"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": r["dtype"], "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {len(r['per_layer_last_step'])} conv layers, {n} stream(s), {r['frames_in_video']}-frame video "
+                               f"walked back and forth; one step = one frame of every stream through rrm_net_step",
+                   "variant": args.variant,
+                   "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair; median"},
+    }
+    for k in ("dense_equiv_gmacs", "ms_per_step_warm", "ms_per_step_dense_path", "speedup_vs_own_dense", "active_macs_last_step",
+              "dense_macs_per_step", "eq9_eq10", "clocks", "roofline", "per_layer_last_step", "alu_peaks_tmacs", "seq", "cpu_baseline"):
+        if k in r:
+            line[k] = r[k]
+    print(json.dumps(line))
+
+
+def compact_conv(r):
+    """The few figures of a convolution configuration that go into the contract line."""
+    out = {k: r[k] for k in ("streams", "variant_requested", "ms_per_step", "frames_per_sec", "ms_per_step_dense_path",
+                             "speedup_vs_own_dense", "dense_equiv_gmacs")}
+    out["rho_per_layer"] = [round(e["rho"], 4) if "rho" in e else None for e in r["per_layer_last_step"]]
+    out["active_out_pixels_per_layer"] = [round(e["active_out_pixels"], 4) if "active_out_pixels" in e else None
+                                          for e in r["per_layer_last_step"]]
+    out["variant_per_layer"] = [e["variant"] for e in r["per_layer_last_step"]]
+    out["S"] = r["eq9_eq10"]["S_with_rrm"]
+    out["S0"] = r["eq9_eq10"]["S0_without_rrm"]
+    out["eta"] = r["eq9_eq10"]["eta_eq10"]
+    out["dense_over_active_macs"] = r["eq9_eq10"]["dense_over_active_macs"]
+    out["roofline_frac"] = r["roofline"]["frac"]
+    out["roofline_bound"] = r["roofline"]["bound"]
+    if "cpu_baseline" in r:
+        out["cpu_baseline"] = r["cpu_baseline"]
+    return out
 
 
 def main():
@@ -340,9 +482,9 @@ def main():
     ap.add_argument("--rho", type=float, default=0.05)
     ap.add_argument("--chunk", type=int, default=FRAMES, help="frames per rrm_step_seq call")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--quick", action="store_true", help="skip the secondary sweeps (profiling runs)")
+    ap.add_argument("--quick", action="store_true", help="skip the secondary sweeps and the CPU legs (profiling runs)")
     ap.add_argument("--workload", default="cfg2", choices=("cfg2",) + CONV_WORKLOADS,
-                    help="cfg2 (default) is the contract line; the others are secondary convolution workloads")
+                    help="cfg2 (default) is the contract line; the others are the convolution configurations")
     ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense"])
     ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
     ap.add_argument("--streams", type=int, default=None, help="independent videos per call (convolution workloads)")
@@ -357,6 +499,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
+        if args.steps == 310:
+            args.steps, args.warmup = 20, 3
         run_reference(args, rank, world)
         return
 
@@ -399,17 +543,18 @@ def main():
         walk = np.stack([seq[order[(i + 1) % period]] for i in range(total)])      # frame i+1 of the walk
         nnz = np.array([np.count_nonzero(seq[order[(i + 1) % period]] != seq[order[i % period]]) / n
                         for i in range(period)])
-        # distinct weight columns one chunk touches (what a cold L2 must fetch), mean over the chunks, stream 0
+        # distinct weight columns one chunk touches (what a cold L2 must fetch; the streams share W), mean over the chunks
         uniq = []
         for k in range(total // T):
             touched = np.zeros(C_IN, dtype=bool)
             for i in range(k * T, (k + 1) * T):
-                touched |= seq[order[(i + 1) % period]][0] != seq[order[i % period]][0]
+                touched |= np.any(seq[order[(i + 1) % period]] != seq[order[i % period]], axis=0).reshape(-1)
             uniq.append(int(touched.sum()))
         return layer, seq, walk, torch.from_numpy(walk).cuda(), float(nnz.mean()), float(np.mean(uniq))
 
     def timed_chunks(layer, seq, walk_dev, steps, warmup, cold, dense=False, frames_per_call=None):
-        """Mean ms per call of rrm_step_seq (or rrm_dense_seq) over chunks of the walk."""
+        """Per-call durations (ms) of rrm_step_seq (or rrm_dense_seq) over chunks of the walk; returns their summary
+        with the median reduced to the max over ranks."""
         tc = T if frames_per_call is None else frames_per_call
         nchunks = walk_dev.shape[0] // tc
         Y = layer.new_output(frames=tc)
@@ -427,7 +572,7 @@ def main():
                 call(walk_dev[k * tc:(k + 1) * tc], Y, tc)
                 evs[i][1].record(stream)
             barrier()
-            ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+            tm = summarize([a.elapsed_time(b) for a, b in evs])
         else:
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
@@ -436,11 +581,12 @@ def main():
                 call(walk_dev[k * tc:(k + 1) * tc], Y, tc)
             b.record(stream)
             barrier()
-            ms = a.elapsed_time(b) / steps
-        return reduce_max(ms)
+            tm = summarize([a.elapsed_time(b) / steps])
+        tm["median"] = reduce_max(tm["median"])
+        return tm
 
     def timed_single(layer, seq, frames, steps, warmup, cold, dense=False):
-        """Mean ms per rrm_step (one frame per call)."""
+        """Median ms per rrm_step (one frame per call)."""
         Y = layer.new_output()
         layer.keyframe(frames[0], Y)
         call = layer.dense if dense else layer.step
@@ -455,7 +601,7 @@ def main():
             call(frames[order[(warmup + i + 1) % period]], Y)
             evs[i][1].record(stream)
         barrier()
-        return reduce_max(float(np.mean([a.elapsed_time(b) for a, b in evs])))
+        return reduce_max(summarize([a.elapsed_time(b) for a, b in evs])["median"])
 
     def frame_bytes(nnz_mean):
         # per frame: gathered weight columns + read/modify/write of P + output + X_t, snapshot read, snapshot write
@@ -465,29 +611,31 @@ def main():
         # the dense evaluation of a chunk: W once, the frames, outputs, stored projection, snapshot
         return C_IN * C_OUT + (frames + 1) * C_IN + frames * 4 * C_OUT + 4 * C_OUT
 
-    EVAL = {1: "column gather", 3: "dense on the tensor cores, W read once (rows x measured density of the previous "
-                                   "chunk >= 0.75)"}
+    def chunk_cold_bytes(uniq_cols, frames, n=1):
+        # what one gather launch must fetch with a cold L2: every distinct column once (the streams share W), the
+        # frames, per-frame projection deltas (write + read) and outputs, the stored projections
+        return uniq_cols * C_OUT + n * ((frames + 2) * C_IN + frames * 12 * C_OUT + 8 * C_OUT)
+
+    EVAL = {1: "column gather (the delta method)", 3: "dense on the tensor cores, W read once (rows x measured density of "
+                                                     "the previous chunk >= rrm_options.fc_dense_rows)"}
     KERNEL = {1: "fc_seq_kernel", 3: "fc_tc_kernel"}
-
-    def chunk_cold_bytes(uniq_cols, frames):
-        # what one chunk launch must fetch with a cold L2: every distinct column once, the frames, per-frame
-        # projection deltas (write + read) and outputs, the stored projection
-        return uniq_cols * C_OUT + (frames + 2) * C_IN + frames * 12 * C_OUT + 8 * C_OUT
-
     peak, peak_kind = measured_peaks()
 
     # ---- primary: one stream per GPU, chunks of T frames per call, rho as asked, cold L2, per-step events
     layer, seq, walk, walk_dev, nnz_mean, uniq_mean = make(args.rho)
+    # (setup, untimed and before the W warm-up steps: lets the library measure the density and settle on its
+    # evaluation, allocate its pinned read-back buffer and scratch)
+    timed_chunks(layer, seq, walk_dev, 4, 4, cold=True)
     sampler = ClockSampler(local)
     sampler.start()
-    ms = timed_chunks(layer, seq, walk_dev, args.steps, args.warmup, cold=True)
+    tm = timed_chunks(layer, seq, walk_dev, args.steps, args.warmup, cold=True)
     clocks = sampler.stop()
+    ms = tm["median"]
     fps = whole_job_rate(T, ms, world)
-    bytes_launch = frame_bytes(nnz_mean) * T
-    achieved = bytes_launch / (ms * 1e-3) / 1e9
     st = layer.stats(0)
     main_variant = st["variant"]
     own_bytes = dense_chunk_bytes(T) if main_variant == 3 else chunk_cold_bytes(uniq_mean, T)
+    achieved = own_bytes / (ms * 1e-3) / 1e9
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     nchunks = walk.shape[0] // T
@@ -520,70 +668,104 @@ def main():
     layer.close()
 
     extra = {}
+    delta_fc = {}
     if not args.quick:
         by_rho = {}
         for rho in RHOS:
             L2, sq, wk, wd, nz, un = make(rho)
             fr = [torch.from_numpy(sq[t]).cuda() for t in range(FRAMES)]
-            c_ms = timed_chunks(L2, sq, wd, 124, 10, cold=True)
-            variant = EVAL.get(L2.stats(0)["variant"], "?")
-            w_ms = timed_chunks(L2, sq, wd, 124, 10, cold=False)
-            d_ms = timed_chunks(L2, sq, wd, 31, 3, cold=True, dense=True)
-            s_ms = timed_single(L2, sq, fr, 310, 31, cold=True)
-            sd_ms = timed_single(L2, sq, fr, 124, 10, cold=True, dense=True)
+            c_ms = timed_chunks(L2, sq, wd, 93, 10, cold=True)["median"]
+            variant = L2.stats(0)["variant"]
+            d_ms = timed_chunks(L2, sq, wd, 31, 3, cold=True, dense=True)["median"]
+            s_ms = timed_single(L2, sq, fr, 186, 31, cold=True)
+            sd_ms = timed_single(L2, sq, fr, 93, 10, cold=True, dense=True)
             LG = make(rho, variant="gather")[0]            # the column-gather kernel whatever the density
-            g_ms = timed_chunks(LG, sq, wd, 124, 10, cold=True)
+            g_ms = timed_chunks(LG, sq, wd, 93, 10, cold=True)["median"]
             LG.close()
+            own = dense_chunk_bytes(T) if variant == 3 else chunk_cold_bytes(un, T)
             by_rho[f"{rho:g}"] = {
-                "nnz_mean_per_frame": nz, "distinct_columns_per_chunk": un, "chunk_evaluation": variant,
-                "chunk_cold_us": c_ms * 1e3, "chunk_warm_us": w_ms * 1e3, "dense_chunk_cold_us": d_ms * 1e3,
-                "gather_chunk_cold_us": g_ms * 1e3,
+                "nnz_mean_per_frame": nz, "distinct_columns_per_chunk": un,
+                "chunk_evaluation": EVAL.get(variant, "?"), "chunk_cold_us": c_ms * 1e3,
                 "fps_cold": T * 1e3 / c_ms, "gmacs_dense_equiv_cold": T * DENSE_MACS / c_ms / 1e6,
-                "speedup_vs_own_dense_chunk": d_ms / c_ms, "gather_speedup_vs_own_dense_chunk": d_ms / g_ms,
-                "roofline_frac_per_frame_bytes": frame_bytes(nz) * T / (c_ms * 1e-3) / 1e9 / peak,
-                "gather_roofline_frac_per_frame_bytes": frame_bytes(nz) * T / (g_ms * 1e-3) / 1e9 / peak,
-                "gather_roofline_frac_distinct_bytes": chunk_cold_bytes(un, T) / (g_ms * 1e-3) / 1e9 / peak,
+                "chunk_roofline_frac_own_bytes": own / (c_ms * 1e-3) / 1e9 / peak,
+                "dense_chunk_cold_us": d_ms * 1e3,
                 "dense_chunk_roofline_frac_own_bytes": dense_chunk_bytes(T) / (d_ms * 1e-3) / 1e9 / peak,
+                "speedup_vs_own_dense_chunk": d_ms / c_ms,
+                "gather_chunk_cold_us": g_ms * 1e3, "gather_speedup_vs_own_dense_chunk": d_ms / g_ms,
                 "single_frame_call_cold_us": s_ms * 1e3, "single_frame_dense_cold_us": sd_ms * 1e3,
                 "single_frame_speedup_vs_own_dense": sd_ms / s_ms,
                 "single_frame_roofline_frac": frame_bytes(nz) / (s_ms * 1e-3) / 1e9 / peak,
                 "single_frame_dense_roofline_frac": dense_chunk_bytes(1) / (sd_ms * 1e-3) / 1e9 / peak}
+            # the contract's kernel (3), the column gather, on its own: the bytes it must fetch from HBM with a cold
+            # L2 (every distinct column of the chunk once) against the HBM peak, and the bytes it serves to the SMs
+            # (every frame's columns; repeats come from L2, so this is a rate, not a fraction of the HBM peak)
+            delta_fc[f"{rho:g}"] = {
+                "kernel": "fc_seq_kernel", "streams": 1, "frames_per_launch": T, "us_per_launch": g_ms * 1e3,
+                "distinct_cold_bytes": chunk_cold_bytes(un, T), "per_frame_bytes_x_frames": frame_bytes(nz) * T,
+                "frac_distinct_cold_bytes": chunk_cold_bytes(un, T) / (g_ms * 1e-3) / 1e9 / peak,
+                "served_gbs_l2_and_hbm": frame_bytes(nz) * T / (g_ms * 1e-3) / 1e9,
+                "faster_than_own_dense_chunk": d_ms / g_ms}
             L2.close()
         extra["by_rho"] = by_rho
+        # more streams per call: the library's choice, and the column gather forced (the multi-stream operating point
+        # of the delta-FC kernel)
         streams = {}
         for n in (4, 16):
             L3, sq, wk, wd, nz, un = make(args.rho, n=n)
-            c_ms = timed_chunks(L3, sq, wd, 62, 5, cold=True)
-            streams[str(n)] = {"chunk_cold_us": c_ms * 1e3, "fps_cold": n * T * 1e3 / c_ms,
-                               "per_frame_bytes_gbs": n * T * frame_bytes(nz) / (c_ms * 1e-3) / 1e9}
+            c_ms = timed_chunks(L3, sq, wd, 31, 5, cold=True)["median"]
+            v3 = L3.stats(0)["variant"]
             L3.close()
+            LG, sq, wk, wd, nz, un = make(args.rho, n=n, variant="gather")
+            g_ms = timed_chunks(LG, sq, wd, 31, 5, cold=True)["median"]
+            LG.close()
+            streams[str(n)] = {"chunk_cold_us": c_ms * 1e3, "fps_cold": n * T * 1e3 / c_ms,
+                               "chunk_evaluation": EVAL.get(v3, "?"), "gather_chunk_cold_us": g_ms * 1e3,
+                               "gather_fps_cold": n * T * 1e3 / g_ms}
+            delta_fc[f"{args.rho:g}_x{n}_streams"] = {
+                "kernel": "fc_seq_kernel", "streams": n, "frames_per_launch": T, "us_per_launch": g_ms * 1e3,
+                "distinct_cold_bytes": chunk_cold_bytes(un, T, n), "per_frame_bytes_x_frames": n * T * frame_bytes(nz),
+                "frac_distinct_cold_bytes": chunk_cold_bytes(un, T, n) / (g_ms * 1e-3) / 1e9 / peak,
+                "served_gbs_l2_and_hbm": n * T * frame_bytes(nz) / (g_ms * 1e-3) / 1e9}
         extra["streams_per_call"] = streams
+        delta_fc["note"] = ("column gather forced (variant GATHER), one launch per chunk, cold L2 before every launch.  "
+                            "frac_distinct_cold_bytes = bytes the launch must fetch from HBM / time / measured HBM peak; "
+                            "served_gbs = all gathered bytes (repeats served by L2) per second: a rate, not an HBM fraction")
+
+    # ---- the convolution configurations, compact (rank 0, one GPU): cfg1, cfg3 int8, cfg4 with the sparse product forced
+    # and as the library chooses
+    conv = None
+    if rank == 0 and world == 1 and not args.quick:
+        conv = {}
+        for key, name, variant, fr_n, cpu_n in (("cfg1", "cfg1", "auto", None, 2), ("cfg3_i8", "cfg3_i8", "auto", 16, 2),
+                                                ("cfg4_delta_forced", "cfg4", "tensor", 8, 1), ("cfg4_auto", "cfg4", "auto", 8, 0)):
+            try:
+                conv[key] = compact_conv(conv_measure(name, variant, steps=30, warmup=5, frames=fr_n, cpu_frames=cpu_n,
+                                                      sample_clocks=False))
+            except Exception as e:  # noqa: BLE001
+                conv[key] = {"error": str(e)}
+        conv["note"] = ("one step = one frame of every stream through rrm_net_step, median of 30 cold-L2 steps; S / S0 / eta: "
+                        "Eq. 9 and Eq. 10 from the measured per-layer densities; cpu_baseline: the oracle on the host cores")
 
     # ---- CPU oracle on the host cores (rank 0, N = 1 only): a bounded sample of the same workload
     cpu = None
     if rank == 0 and world == 1 and not args.quick:
-        from oracle import rrm_oracle as orc
-        rec = orc.Recurrence([spec])
-        rec.step(seq[0])
-        t0 = time.perf_counter()
-        cnt = 0
-        while cnt < 2 * period and time.perf_counter() - t0 < 20.0:
-            rec.step(seq[order[(cnt + 1) % period]])
-            cnt += 1
-        dt = time.perf_counter() - t0
-        cpu = {"value": cnt / dt, "unit": "frames/s", "cores": orc.threads(), "kind": "oracle",
-               "sample": f"{cnt} frames of the same sequence through the oracle's Algorithm-1 recurrence (delta path)"}
+        r_fps, r_n, d_fps, d_n, cores = cpu_fc_baseline(spec, seq, order, budget_s=10.0, max_frames=4 * period)
+        cpu = {"value": r_fps, "unit": "frames/s", "cores": cores, "kind": "oracle",
+               "sample": f"{r_n} frames of the same sequence through the oracle's Algorithm-1 recurrence (delta path); "
+                         f"weights promoted to int64 once, outside the timed region",
+               "dense_value": d_fps, "dense_sample": f"{d_n} frames through the oracle's dense definition (Eq. 3)"}
 
     if rank == 0:
         line = {
             "metric": "frames_per_sec", "value": fps, "unit": "frames/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_stats": tm, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "i8", "data": "synthetic",
             "config": {"workload": f"cfg2 delta-FC int8 fc6 {C_IN}->{C_OUT}, rho={args.rho:g}, 1 stream per GPU; one step = "
                                    f"one chunk of {T} consecutive frames (one rrm_step_seq call) of the {FRAMES}-frame "
                                    f"sequence walked back and forth",
                        "frames_per_step": T, "evaluation": EVAL.get(main_variant, "?"),
-                       "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair",
+                       "l2": "flushed before every timed step (256 MiB write); each step timed by its own event pair; "
+                             "ms_per_step is the median",
                        "measured_nnz_mean_per_frame": nnz_mean, "measured_density": nnz_mean / C_IN,
                        "distinct_columns_per_chunk": uniq_mean},
             "dense_equiv_gmacs": fps * DENSE_MACS / 1e9,
@@ -591,20 +773,20 @@ def main():
             "e2e": {"value": world * T * 1e3 / e2e_ms, "unit": "frames/s", "h2d_bytes_per_step": T * C_IN,
                     "d2h_bytes_per_step": T * 4 * C_OUT,
                     "call": "rrm_step_seq_host_async per step, one rrm_host_sync after the last step; steps back to back "
-                            "(no L2 flush between them, unlike `value`), timed on the host clock",
+                            "(no L2 flush between them, unlike `value`: W stays L2-resident), timed on the host clock",
                     "value_waiting_every_call": world * T * 1e3 / e2e_sync_ms},
             "gpu_launches": args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": committed_traffic(KERNEL.get(main_variant, "fc_seq_kernel"), args.rho),
                          "peak_kind": f"of {peak_kind}",
                          "kernel": KERNEL.get(main_variant, "?"), "evaluation": EVAL.get(main_variant, "?"),
-                         "algorithmic_bytes_per_launch": bytes_launch,
-                         "own_bytes_per_launch": own_bytes, "achieved_own": own_bytes / (ms * 1e-3) / 1e9,
-                         "frac_own": own_bytes / (ms * 1e-3) / 1e9 / peak,
-                         "note": "algorithmic bytes = the delta-FC's per-frame bytes (gathered columns, projection, "
-                                 "frames) x frames per launch; own bytes = what the kernel that ran has to move with a "
-                                 "cold L2 (dense evaluation: W once for all frames; gather: every distinct column once)"},
+                         "algorithmic_bytes_per_launch": own_bytes,
+                         "note": "bytes the kernel that ran must move with a cold L2 (dense evaluation: W once for all "
+                                 "frames + frames, outputs, state; column gather: every distinct column of the chunk once "
+                                 "+ frames, per-frame projection deltas, outputs) / median launch duration"},
+            "roofline_delta_fc": delta_fc or None,
             "cpu_baseline": cpu,
+            "conv": conv,
             "last_step_stats": st,
         }
         line.update(extra)

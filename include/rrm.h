@@ -24,6 +24,9 @@
  *     RRM_BIN (+1 / -1).  Bias: float (RRM_F32) or int32_t.  Weights and bias are copied and
  *     repacked into library-owned device memory at create time; the caller may free its copy.
  *   - One object may be used from one stream at a time.
+ *   - Environment switches, read when an object is created (debugging aids): RRM_NO_GRAPH=1 launches every
+ *     kernel of a stack step on its own instead of replaying a captured CUDA graph; RRM_DEBUG=1 names a failing
+ *     CUDA call (file, line, error string) on stderr and prints the shape of captured chunk graphs.
  */
 #ifndef RRM_H
 #define RRM_H
@@ -97,6 +100,25 @@ typedef struct {
     int32_t error_word;        /* device-side error flags, 0 = none */
 } rrm_stats;
 
+/* Tunables of one object (a layer or a stack).  The paper leaves all of these to the implementation: it only
+ * says that the sparse product pays off below some density (Table 1, Eq. 6) and that a precise inference may
+ * replace the state at any time (Sec. 3.4).  rrm_net_get_options returns the defaults of a fresh object. */
+typedef struct {
+    uint32_t wait_limit;         /* polls a bounded device-side wait (mbarrier, completion of the tensor-core work)
+                                    makes before it gives up, sets the time-out bit of rrm_stats.error_word and lets
+                                    the thread block leave in an orderly way.  Default 2^20.  0 makes every such wait
+                                    give up at once, before the thread block has anything in flight: a test hook */
+    float layer_dense_activity;  /* stacks, variant AUTO: a layer whose measured share of projection pixels to update
+                                    reached this value is evaluated densely in the following frames ... */
+    float layer_delta_activity;  /* ... and goes back to the sparse product once the share has fallen below this one */
+    float stack_dense_activity;  /* whole-stack switch (stacks of >= 1 GMAC per frame): MAC-weighted share from which on
+                                    every layer of the next frames is evaluated densely */
+    int32_t stack_reprobe;       /* dense frames in a row before one delta frame measures the activity again */
+    float fc_dense_rows;         /* lone int8 FC layer, chunks: rows x measured density from which on a chunk is
+                                    evaluated densely on the tensor cores, per launch that evaluation needs */
+    float fc_dense_density;      /* the same for chunks of more rows than the few-row kernel takes: plain density */
+} rrm_options;
+
 /* ---- single layer (Eq. 2-5) ------------------------------------------------------- */
 
 /* Creates a layer with state I_prev = 0, P_prev = bias (Algorithm 1, line 1), so a first
@@ -125,7 +147,7 @@ int rrm_dense(rrm_layer* layer, const void* X_dev, void* Y_dev, void* stream);
 int rrm_step_host(rrm_layer* layer, const void* Xt_host, void* Yt_host, void* stream);
 
 /* A chunk of T consecutive frames in one call: the frame loop of Algorithm 1 for frames t0 .. t0+T-1
- * (Sec. 3.3 notes that a video may be cut into chunks that are processed on their own).  The result
+ * (the end of Sec. 3.2 notes that a video may be cut into chunks that are processed on their own).  The result
  * and the state afterwards are exactly those of T rrm_step calls in a row.
  *   X_dev  [T] frames, each in the layer's input layout, back to back; read-only
  *   Y_dev  [T] outputs f(P_t), each in the layer's output layout, back to back; may be NULL
@@ -159,8 +181,17 @@ int rrm_step_seq_host_async(rrm_layer* layer, const void* X_host, void* Y_host, 
 /* Waits until every queued rrm_step_seq_host_async call has delivered its outputs to host memory. */
 int rrm_host_sync(rrm_layer* layer);
 
-/* Synchronises the layer's last stream and fills `host_out`. */
+/* Synchronises the layer's last stream and fills `host_out`.  Returns RRM_ERR_TIMEOUT when a bounded device wait
+ * ran out since the last rrm_clear_errors (bit 1 of error_word), RRM_ERR_CAPACITY when an int8 delta did not fit a
+ * byte (bit 0): host_out is filled in both cases, and the results of the affected frames are not to be trusted
+ * (a dense pass, rrm_keyframe, restores a consistent state). */
 int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out);
+/* Clears the device error word (synchronises the layer's last stream). */
+int rrm_clear_errors(rrm_layer* layer);
+/* Reads / replaces the tunables.  rrm_set_options synchronises the device and discards the captured launch
+ * sequences (they hold the old values); call it between frames. */
+int rrm_get_options(const rrm_layer* layer, rrm_options* out);
+int rrm_set_options(rrm_layer* layer, const rrm_options* in);
 
 /* Copies the stored projection P_prev (float or int32, [N][C_out][OH][OW]) to P_dev. */
 int rrm_layer_projection(rrm_layer* layer, void* P_dev, void* stream);
@@ -195,6 +226,9 @@ int rrm_net_step_seq_host_async(rrm_net* net, const void* frames_host, void* out
 int rrm_net_host_sync(rrm_net* net);
 
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* host_out);
+int rrm_net_clear_errors(rrm_net* net);
+int rrm_net_get_options(const rrm_net* net, rrm_options* out);
+int rrm_net_set_options(rrm_net* net, const rrm_options* in);
 
 /* ---- approximate mode: sparsity enhancement and accumulated error control (Sec. 3.4) -----------
  * With eps > 0 every delta entry with |d| < eps is truncated to zero before the sparse product (fp32 stacks
@@ -250,6 +284,15 @@ int64_t rrm_net_tensor_bytes(const rrm_net* net, int t);
 #define RRM_FC_NOALLOC_MAX_C_IN 16384
 int rrm_fc_step_noalloc(const int8_t* Wt_dev, const int8_t* Xt_dev, int8_t* Xprev_dev, int32_t* P_dev,
                         void* Y_dev, int n, int c_in, int c_out, int shift, int act, void* stream);
+
+/* ---- measured ALU peaks -------------------------------------------------------------
+ * (No counterpart in the paper: a reporting aid.)  Runs a register-only loop of independent operations on every
+ * SM of the current device and returns the best of five timings as multiply-accumulates per second:
+ *   kind 0  fp32 fused multiply-add                       (the fp32 delta convolution, Table 1's MACs)
+ *   kind 1  dp4a, counted as 4 int8 multiply-accumulates  (int8 layers on the CUDA cores, the delta-FC products)
+ *   kind 2  popc + add, counted as 32 one-bit products    (binary layers on the CUDA cores, Sec. 4.3)
+ * The rooflines of ALU-bound kernels are quoted against these numbers.  Allocates 4 bytes, synchronises. */
+int rrm_measure_alu_peak(int kind, double* macs_per_s);
 
 const char* rrm_strerror(int status);
 

@@ -4,8 +4,8 @@ Every step of the hot path runs in the CUDA kernels of librrm_b200.so; this pack
 marshals arguments.  Importing it does not load the shared library; the first call does,
 and fails loudly if the library is missing or cannot be built.
 """
-from .binding import (RRMError, LayerDesc, Stats, Net, Layer, lib, desc_from_spec, net_from_specs,
-                      layer_from_spec, fc_step_noalloc, aecs_predict, KIND, DTYPE, ACT, VARIANT)
+from .binding import (RRMError, LayerDesc, Stats, Options, Net, Layer, lib, desc_from_spec, net_from_specs,
+                      layer_from_spec, fc_step_noalloc, aecs_predict, measure_alu_peak, KIND, DTYPE, ACT, VARIANT)
 
-__all__ = ["RRMError", "LayerDesc", "Stats", "Net", "Layer", "lib", "desc_from_spec", "net_from_specs",
-           "layer_from_spec", "fc_step_noalloc", "aecs_predict", "KIND", "DTYPE", "ACT", "VARIANT"]
+__all__ = ["RRMError", "LayerDesc", "Stats", "Options", "Net", "Layer", "lib", "desc_from_spec", "net_from_specs",
+           "layer_from_spec", "fc_step_noalloc", "aecs_predict", "measure_alu_peak", "KIND", "DTYPE", "ACT", "VARIANT"]

@@ -33,23 +33,30 @@ class Stats(ctypes.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
+class Options(ctypes.Structure):
+    _fields_ = [("wait_limit", ctypes.c_uint32), ("layer_dense_activity", ctypes.c_float),
+                ("layer_delta_activity", ctypes.c_float), ("stack_dense_activity", ctypes.c_float),
+                ("stack_reprobe", ctypes.c_int32), ("fc_dense_rows", ctypes.c_float), ("fc_dense_density", ctypes.c_float)]
+
+
 _lib = None
 _P = ctypes.c_void_p
 
 
 def lib():
-    """Loads librrm_b200.so (building it with nvcc if absent).  Raises if that fails: there is
-    no fallback implementation."""
+    """Loads librrm_b200.so (building it with nvcc if absent or older than its sources).  Raises if
+    that fails: there is no fallback implementation and a stale library is never loaded."""
     global _lib
     if _lib is not None:
         return _lib
     so = _build.SO
     if _build.needs_build():
+        # never load a library that is older than its sources: a failed rebuild is an error, not a fallback
         try:
             _build.build()
         except Exception as e:  # noqa: BLE001
-            if not os.path.exists(so):
-                raise RRMError(f"librrm_b200.so is missing and could not be built: {e}") from e
+            state = "out of date" if os.path.exists(so) else "missing"
+            raise RRMError(f"librrm_b200.so is {state} and could not be built: {e}") from e
     L = ctypes.CDLL(so)
     sig = {
         "rrm_layer_create": [ctypes.POINTER(_P), ctypes.POINTER(LayerDesc), _P, _P],
@@ -80,6 +87,12 @@ def lib():
         "rrm_net_get_stats": [_P, ctypes.c_int, ctypes.POINTER(Stats)],
         "rrm_net_projection": [_P, ctypes.c_int, _P, _P],
         "rrm_net_tensor": [_P, ctypes.c_int, _P, _P],
+        "rrm_clear_errors": [_P],
+        "rrm_net_clear_errors": [_P],
+        "rrm_get_options": [_P, ctypes.POINTER(Options)],
+        "rrm_set_options": [_P, ctypes.POINTER(Options)],
+        "rrm_net_get_options": [_P, ctypes.POINTER(Options)],
+        "rrm_net_set_options": [_P, ctypes.POINTER(Options)],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -95,6 +108,8 @@ def lib():
     L.rrm_aecs_predict.restype = ctypes.c_double
     L.rrm_net_tensor_bytes.argtypes = [_P, ctypes.c_int]
     L.rrm_net_tensor_bytes.restype = ctypes.c_int64
+    L.rrm_measure_alu_peak.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
+    L.rrm_measure_alu_peak.restype = ctypes.c_int
     L.rrm_strerror.argtypes = [ctypes.c_int]
     L.rrm_strerror.restype = ctypes.c_char_p
     _lib = L
@@ -205,10 +220,35 @@ class Net:
         _check(lib().rrm_net_truncation(self._h, ctypes.byref(e), per), "rrm_net_truncation")
         return e.value, list(per)
 
-    def stats(self, layer=0):
+    def stats(self, layer=0, check=True):
+        """rrm_net_get_stats.  A device-side error since the last clear_errors() (a bounded wait that ran out, an
+        int8 delta outside a byte) comes back as the call's status: raised, or with check=False returned beside the
+        counters under the key "status"."""
         s = Stats()
-        _check(lib().rrm_net_get_stats(self._h, layer, ctypes.byref(s)), "rrm_net_get_stats")
-        return s.as_dict()
+        status = lib().rrm_net_get_stats(self._h, layer, ctypes.byref(s))
+        if check or status not in (0, -5, -6):
+            _check(status, "rrm_net_get_stats")
+        d = s.as_dict()
+        d["status"] = status
+        return d
+
+    def clear_errors(self):
+        _check(lib().rrm_net_clear_errors(self._h), "rrm_net_clear_errors")
+
+    def options(self):
+        o = Options()
+        _check(lib().rrm_net_get_options(self._h, ctypes.byref(o)), "rrm_net_get_options")
+        return {n: getattr(o, n) for n, _ in o._fields_}
+
+    def set_options(self, **kw):
+        """rrm_net_set_options with the named fields replaced (the others keep their current values)."""
+        o = Options()
+        _check(lib().rrm_net_get_options(self._h, ctypes.byref(o)), "rrm_net_get_options")
+        for k, v in kw.items():
+            if k not in dict(o._fields_):
+                raise KeyError(k)
+            setattr(o, k, v)
+        _check(lib().rrm_net_set_options(self._h, ctypes.byref(o)), "rrm_net_set_options")
 
     def tensor_bytes(self, t):
         b = lib().rrm_net_tensor_bytes(self._h, t)
@@ -265,6 +305,13 @@ def fc_step_noalloc(Wt, Xt, Xprev, P, Y, n, c_in, c_out, shift=-1, act="none", s
     can test the documented limits."""
     return lib().rrm_fc_step_noalloc(_ptr(Wt), _ptr(Xt), _ptr(Xprev), _ptr(P), _ptr(Y), n, c_in, c_out, shift,
                                      ACT[act], _stream(stream))
+
+
+def measure_alu_peak(kind):
+    """rrm_measure_alu_peak: measured multiply-accumulates per second of "ffma", "dp4a" or "popc" on the current device."""
+    v = ctypes.c_double()
+    _check(lib().rrm_measure_alu_peak({"ffma": 0, "dp4a": 1, "popc": 2}[kind], ctypes.byref(v)), "rrm_measure_alu_peak")
+    return v.value
 
 
 def aecs_predict(mu, e_t):

@@ -41,6 +41,16 @@ int validate_desc(const rrm_layer_desc& d, int l, int n_layers)
     return RRM_OK;
 }
 
+// Frees a buffer that a larger one is about to replace (the caller has made sure nothing uses it any more).
+void dev_release(rrm_net* net, void** p)
+{
+    if (!*p) return;
+    for (size_t i = 0; i < net->allocs.size(); ++i)
+        if (net->allocs[i] == *p) { net->allocs.erase(net->allocs.begin() + i); break; }
+    cudaFree(*p);
+    *p = nullptr;
+}
+
 int dev_alloc(rrm_net* net, void** p, size_t bytes)
 {
     if (bytes == 0) bytes = 16;
@@ -313,8 +323,6 @@ void drop_graphs(rrm_net* net)
     }
 }
 
-constexpr double DENSE_SWITCH_ACTIVITY = 0.75;   // MAC-weighted share of projection pixels to update, from which on a frame goes dense
-constexpr int DENSE_SWITCH_REPROBE = 15;         // dense frames in a row before a delta frame measures the activity again
 
 // Copies the step's counters to pinned memory behind the work on the stream (never waited for).
 int activity_read_back(rrm_net* net, cudaStream_t st)
@@ -362,7 +370,7 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
         net->last_step_dense = false;
         if (net->auto_switch && net->eps == 0.f) {
             activity_poll(net);
-            if (net->activity >= DENSE_SWITCH_ACTIVITY && net->dense_streak < DENSE_SWITCH_REPROBE) {
+            if (net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
                 ++net->dense_streak;
                 net->last_step_dense = true;
                 dense = true;
@@ -453,10 +461,12 @@ int ensure_chunk(rrm_net* net, int T)
         tensor_bytes_boundary(net->tensors.front(), &bi);
         tensor_bytes_boundary(net->tensors.back(), &bo);
         RRM_CUDA_TRY(cudaDeviceSynchronize());               // the old buffers may be in use by a graph in flight
+        for (int k = 0; k < 3; ++k) drop_chunk_graphs(net, k);   // graphs hold the old buffers
+        dev_release(net, &net->chunk_in);
+        dev_release(net, &net->chunk_out);
         RRM_TRY(dev_alloc(net, &net->chunk_in, (size_t)bi * T));
         RRM_TRY(dev_alloc(net, &net->chunk_out, (size_t)bo * T));
         net->chunk_cap = T;
-        for (int k = 0; k < 3; ++k) drop_chunk_graphs(net, k);   // graphs hold the old buffers
     }
     return RRM_OK;
 }
@@ -562,7 +572,7 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
         net->last_step_dense = false;
         if (net->auto_switch) {
             activity_poll(net);
-            if (net->activity >= DENSE_SWITCH_ACTIVITY && net->dense_streak < DENSE_SWITCH_REPROBE) {
+            if (net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
                 ++net->dense_streak;                         // (counted in calls: a delta chunk measures again after 15 dense ones)
                 net->last_step_dense = true;
                 dense = true;
@@ -633,6 +643,11 @@ int ensure_stage(rrm_net* net, int frames = 1)
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
+    if (net->stage_in) {                                     // growing: the old buffers may still be in use
+        RRM_CUDA_TRY(cudaDeviceSynchronize());
+        dev_release(net, &net->stage_in);
+        dev_release(net, &net->stage_out);
+    }
     RRM_TRY(dev_alloc(net, &net->stage_in, (size_t)bi * frames));
     RRM_TRY(dev_alloc(net, &net->stage_out, (size_t)bo * frames));
     net->stage_frames = frames;
@@ -660,6 +675,8 @@ int ensure_pipe(rrm_net* net, int frames)
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
     for (int s = 0; s < 2; ++s) {
+        dev_release(net, &net->pipe_in[s]);
+        dev_release(net, &net->pipe_out[s]);
         RRM_TRY(dev_alloc(net, &net->pipe_in[s], (size_t)bi * frames));
         RRM_TRY(dev_alloc(net, &net->pipe_out[s], (size_t)bo * frames));
     }
@@ -888,9 +905,20 @@ double rrm_aecs_predict(const double mu[5], double e_t)
     return mu[0] + e_t * (mu[1] + e_t * (mu[2] + e_t * (mu[3] + e_t * mu[4])));
 }
 
+static int stats_fill(rrm_net* net, int layer, rrm_stats* h);
+
 int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
 {
     if (!net || !h || layer < 0 || layer >= (int)net->layers.size()) return RRM_ERR_INVALID_ARG;
+    RRM_TRY(stats_fill(net, layer, h));
+    // device-side errors since the last rrm_net_clear_errors surface here (the steps themselves are asynchronous)
+    if (h->error_word & ERRW_TIMEOUT) return RRM_ERR_TIMEOUT;
+    if (h->error_word & (ERRW_BOUNDS | ERRW_CAPACITY)) return RRM_ERR_CAPACITY;
+    return RRM_OK;
+}
+
+static int stats_fill(rrm_net* net, int layer, rrm_stats* h)
+{
     RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
     std::memset(h, 0, sizeof(*h));
     const Layer& L = net->layers[layer];
@@ -946,6 +974,35 @@ int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* h)
     return RRM_OK;
 }
 int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out) { return rrm_net_get_stats(layer, 0, host_out); }
+
+int rrm_net_clear_errors(rrm_net* net)
+{
+    if (!net) return RRM_ERR_INVALID_ARG;
+    if (net->last_stream) RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
+    RRM_CUDA_TRY(cudaMemset(net->errw, 0, 4));
+    return RRM_OK;
+}
+int rrm_clear_errors(rrm_layer* layer) { return rrm_net_clear_errors(layer); }
+
+int rrm_net_get_options(const rrm_net* net, rrm_options* out)
+{
+    if (!net || !out) return RRM_ERR_INVALID_ARG;
+    *out = net->opt;
+    return RRM_OK;
+}
+int rrm_net_set_options(rrm_net* net, const rrm_options* in)
+{
+    if (!net || !in) return RRM_ERR_INVALID_ARG;
+    if (!(in->layer_dense_activity >= 0.f) || !(in->layer_delta_activity >= 0.f) || in->layer_delta_activity > in->layer_dense_activity ||
+        !(in->stack_dense_activity >= 0.f) || in->stack_reprobe < 1 || !(in->fc_dense_rows >= 0.f) || !(in->fc_dense_density >= 0.f))
+        return RRM_ERR_INVALID_ARG;
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
+    net->opt = *in;
+    drop_graphs(net);                                        // captured sequences hold the old wait limit
+    return RRM_OK;
+}
+int rrm_get_options(const rrm_layer* layer, rrm_options* out) { return rrm_net_get_options(layer, out); }
+int rrm_set_options(rrm_layer* layer, const rrm_options* in) { return rrm_net_set_options(layer, in); }
 
 int rrm_net_projection(rrm_net* net, int layer, void* P_dev, void* stream)
 {

@@ -18,6 +18,7 @@
 // is the library's dense path and the keyframe.
 #include "rrm_common.cuh"
 #include "rrm_rows.cuh"
+#include "rrm_tc.cuh"
 #include <type_traits>
 
 namespace rrm {
@@ -39,6 +40,7 @@ struct ConvParams {
     int* errw;
     int n, c_in, h, w, u_in, oh, ow, kh, kw, stride, pad, c_out, np, ku, kup, opixels;
     int ksplit;               // gridDim.z: CTAs that share one output tile, each with a contiguous range of K stages
+    unsigned wait_limit;      // polls of one bounded wait
 };
 
 __device__ __forceinline__ bool bit_test(const uint32_t* bm, int i) { return (bm[i >> 5] >> (i & 31)) & 1u; }
@@ -61,7 +63,6 @@ __device__ __forceinline__ bool bit_test(const uint32_t* bm, int i) { return (bm
 // Copies of later stages are in flight while the current one is multiplied (4x4 outputs per thread).
 // ------------------------------------------------------------------------------------------------
 constexpr int GEMM_STAGES = 3;
-constexpr unsigned GEMM_SPIN_LIMIT = 1u << 20;
 constexpr int GEMM_LDA = TK + 4;                   // words per activation row in shared memory (16-byte aligned, bank-staggered)
 constexpr int GEMM_A_WORDS = TM * GEMM_LDA, GEMM_B_WORDS = TK * TN;
 
@@ -73,19 +74,6 @@ __device__ __forceinline__ void g_cp_async4(uint32_t dst, const void* src, uint3
 __device__ __forceinline__ void g_cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ bool g_mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (unsigned i = 0; i < GEMM_SPIN_LIMIT; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-    }
-    return false;
 }
 
 template <int DT, bool DENSE, bool VEC>
@@ -275,8 +263,10 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     for (int ks = next_live(s_first); ks < n_stages; ks = next_live(ks + 1), ++it) {
         const int slot = it % GEMM_STAGES;
         asm volatile("cp.async.wait_group %0;" ::"n"(GEMM_STAGES - 2) : "memory");   // this thread's copies of stage `it` landed
-        if (ok && !g_mbar_wait(g_smem_u32(&s_full[slot]), (it / GEMM_STAGES) & 1)) ok = false;
-        __syncthreads();                                     // everyone's copies landed; everyone is done with stage it - 1
+        if (!mbar_wait(g_smem_u32(&s_full[slot]), (it / GEMM_STAGES) & 1, p.wait_limit)) ok = false;
+        // everyone's copies landed; everyone is done with stage it - 1.  A wait that ran out in any thread ends the
+        // loop for all of them: nothing more is issued
+        if (__syncthreads_or(!ok)) { ok = false; break; }
         if (ks_issue < n_stages) { issue(ks_issue, issued % GEMM_STAGES); ++issued; ks_issue = next_live(ks_issue + 1); }
         else asm volatile("cp.async.commit_group;" ::: "memory");
         const uint32_t* Bs = g_smem + slot * STAGE_WORDS;
@@ -312,7 +302,17 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (!ok) { atomicOr(p.errw, ERRW_TIMEOUT); return; }
+    if (!ok) {
+        // giving up: the filter slices still on their way (stages issued, not consumed) must land before the CTA's
+        // shared memory goes away; thread 0 issued them and waits for them, the others wait for thread 0
+        if (tid == 0) {
+            atomicOr(p.errw, ERRW_TIMEOUT);
+            for (int j = it; j < issued; ++j)
+                mbar_wait(g_smem_u32(&s_full[j % GEMM_STAGES]), (j / GEMM_STAGES) & 1, WAIT_LIMIT_DEFAULT);
+        }
+        __syncthreads();
+        return;
+    }
 
     // ---- update of the stored projection: the owner of a tile writes it; CTAs that share a tile
     // (split K) add their partial sums with atomics (dense: onto a zeroed projection, split 0 adds the bias)
@@ -997,6 +997,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     p.n = d.n; p.c_in = d.c_in; p.h = d.h; p.w = d.w; p.u_in = L.u_in; p.oh = L.oh; p.ow = L.ow;
     p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.c_out = d.c_out; p.np = L.np;
     p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
+    p.wait_limit = net->opt.wait_limit;
     dim3 grid(ceil_div(L.opixels(), TM), L.np / TN);
     p.errw = net->errw;
     // split K over CTAs while the tiles alone leave most of the machine idle (each share keeps >= 4 stages)

@@ -47,6 +47,7 @@ struct TcParams {
     int slabs;                // total 128-byte slabs of K
     int bn;                   // 64 or 128
     int ksplit;               // gridDim.z
+    unsigned wait_limit;      // polls of one bounded wait
 };
 
 // byte i of the result = bit i of the low nibble of x (0 or 1)
@@ -54,7 +55,7 @@ __device__ __forceinline__ uint32_t spread4(uint32_t x) { return ((x & 0xfu) * 0
 
 // Dynamic shared memory: [stages][A 16 KB | B 16 KB] on a 1024-byte boundary, then barriers and row tables.
 struct TcSmemTail {
-    unsigned long long full[TC_STAGES], empty[TC_STAGES], done;
+    unsigned long long full[TC_STAGES], bfull[TC_STAGES], empty[TC_STAGES], done;   // A landed / B landed / stage free / all MMAs done
     uint32_t tmem_base;
     int fail;
     unsigned long long tap_mask[2];           // taps with a usable input under at least one row of this tile (up to 128 taps)
@@ -87,7 +88,9 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
 
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) {
-            mbar_init(smem_u32(&S->full[s]), 128 + 1);      // 128 producer threads + the B loader's expect_tx
+            mbar_init(smem_u32(&S->full[s]), 128);          // 128 producer threads
+            mbar_init(smem_u32(&S->bfull[s]), 1);           // the B loader's expect_tx (a barrier of its own, so that the
+                                                            // loader can wait for its copies in flight on a give-up exit)
             mbar_init(smem_u32(&S->empty[s]), 1);           // one tcgen05.commit
         }
         mbar_init(smem_u32(&S->done), 1);
@@ -218,7 +221,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             }
             for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
                 const int stage = it % TC_STAGES;
-                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
+                if (*(volatile int*)&S->fail) break;             // another role gave up: issue nothing more
                 const uint32_t As = base_u32 + stage * (uint32_t)TC_STAGE_BYTES;
                 if (p.kpp == 4) {
                     // first layers (up to 4 channels = 4 bytes per pixel): a 16-byte piece holds 4 taps, copied one by one;
@@ -319,7 +323,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 const int ks_next = next_live(ks + 1);
                 if (ks_next < s_end) fetch(ks_next);
                 const int stage = it % TC_STAGES;
-                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
                 unsigned char* As = base + stage * TC_STAGE_BYTES;
                 const int shift = (piece & 1) * 16;
                 #pragma unroll
@@ -351,13 +355,15 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             int it = 0;
             for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
                 const int stage = it % TC_STAGES;
-                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1)) { ok = false; break; }
-                const uint32_t bar = smem_u32(&S->full[stage]);
+                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / TC_STAGES) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
+                if (*(volatile int*)&S->fail) break;
+                const uint32_t bar = smem_u32(&S->bfull[stage]);
                 mbar_arrive_expect_tx(bar, tile_b_bytes);
                 bulk_copy_g2s(base_u32 + stage * (uint32_t)TC_STAGE_BYTES + TC_M * TC_SLAB,
                               p.Wimg + ((size_t)ntile * p.slabs + ks) * tile_b_bytes, tile_b_bytes, bar);
                 ++it;
             }
+            n_issued = it;
         }
     } else {
         // ================= MMA issuer
@@ -366,7 +372,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             int it = 0;
             for (int ks = next_live(s_begin); ks < s_end; ks = next_live(ks + 1)) {
                 const int stage = it % TC_STAGES;
-                if (!mbar_wait(smem_u32(&S->full[stage]), (it / TC_STAGES) & 1)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&S->full[stage]), (it / TC_STAGES) & 1, p.wait_limit) ||
+                    !mbar_wait(smem_u32(&S->bfull[stage]), (it / TC_STAGES) & 1, p.wait_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_addr = base_u32 + stage * (uint32_t)TC_STAGE_BYTES;
                 const uint64_t adesc = tc_smem_desc(a_addr), bdesc = tc_smem_desc(a_addr + TC_M * TC_SLAB);
@@ -377,9 +384,16 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 ++it;
             }
             if (ok) tc_commit(smem_u32(&S->done));          // all MMAs of this CTA have completed
+            else if (it > 0) {
+                // giving up with MMAs issued: they must have completed before the tensor memory is freed
+                *(volatile int*)&S->fail = 1;               // (before the commit below: the epilogue warps must not take
+                __threadfence_block();                      // the completed barrier for a finished tile)
+                tc_commit(smem_u32(&S->done));
+                mbar_wait(smem_u32(&S->done), 0, WAIT_LIMIT_DEFAULT);
+            }
         }
     }
-    if (!ok) { S->fail = 1; atomicOr(p.errw, ERRW_TIMEOUT); }
+    if (!ok) { *(volatile int*)&S->fail = 1; atomicOr(p.errw, ERRW_TIMEOUT); }
 
     // ================= epilogue: each of the 128 threads of warps 0-3 owns one accumulator row.  It copies
     // the row from tensor memory into shared memory (the stage buffers are free now) and hands it to the
@@ -389,7 +403,9 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     if (warp < 4) {
         ok = __all_sync(0xffffffffu, ok);                   // the tensor-memory loads below need the whole warp
         const bool have = n_issued > 0;                     // identical for all producer threads
-        if (ok && have && !mbar_wait(smem_u32(&S->done), 0)) { ok = false; S->fail = 1; atomicOr(p.errw, ERRW_TIMEOUT); }
+        if (ok && have && !mbar_wait(smem_u32(&S->done), 0, p.wait_limit)) { ok = false; *(volatile int*)&S->fail = 1; atomicOr(p.errw, ERRW_TIMEOUT); }
+        asm volatile("bar.sync 1, 128;" ::: "memory");      // the four warps agree: nobody stores results of a tile that gave up
+        ok = ok && *(volatile int*)&S->fail == 0;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
         const bool atomic = p.ksplit > 1;
@@ -461,6 +477,12 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     }
     tc_fence_before();
     __syncthreads();
+    if (warp == 5 && lane == 0 && S->fail) {
+        // a role gave up: the bulk copies this thread may still have in flight must land before the CTA's shared
+        // memory goes away (at most one per stage; a phase that completed long ago returns at once)
+        for (int j = max(0, n_issued - TC_STAGES); j < n_issued; ++j)
+            mbar_wait(smem_u32(&S->bfull[j % TC_STAGES]), (j / TC_STAGES) & 1, WAIT_LIMIT_DEFAULT);
+    }
     if (warp == 4) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TC_MAX_BN) : "memory");
     }
@@ -534,14 +556,11 @@ int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev)
                                                                       d.c_in, d.c_out, taps, L.tc_kpp, L.tc_slabs, L.tc_bn,
                                                                       L.tc_ntiles);
     RRM_CUDA_TRY(cudaGetLastError());
-    static bool attr_done = false;
-    if (!attr_done) {
-        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
-        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
-        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
-        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
-        attr_done = true;
-    }
+    // (the attribute belongs to the current device's copy of the function: set at every create, it is cheap)
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
     L.tc_ready = true;
     return RRM_OK;
 }
@@ -565,6 +584,7 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.chunks_per_tap = L.tc_kpp / 32;
     p.kpp = L.tc_kpp;
     p.slabs = L.tc_slabs; p.bn = L.tc_bn;
+    p.wait_limit = net->opt.wait_limit;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
     // split K towards the point where a CTA's slabs all fit in its pipeline at once
     // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the

@@ -338,12 +338,10 @@ __global__ void __launch_bounds__(SQ_THREADS) fc_count_kernel(const int8_t* __re
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-// From this measured non-zero fraction of the previous chunk on, the next chunk is evaluated densely on the
-// tensor cores (W read once for all frames) instead of by column gather (measured break-even on fc6: ~7 %).
-constexpr double SQ_DENSE_SWITCH = 0.08;
-// ... and for chunks of few rows (one launch that reads W once): rows x non-zero fraction from which on the dense
-// evaluation wins (measured break-even on fc6, 32 rows: 2.2 % non-zeros)
-constexpr double SQ_DENSE_SWITCH_ROWS = 0.75;
+// The switch between the column gather and the dense tensor-core evaluation of a chunk (W read once for all frames)
+// is rrm_options.fc_dense_density (plain non-zero fraction of the previous chunk; measured break-even on fc6: ~7 %)
+// and, for chunks of few rows (one launch that reads W once), rrm_options.fc_dense_rows (rows x non-zero fraction;
+// measured break-even on fc6, 32 rows: 2.2 % non-zeros).
 
 // Copies the chunk's counters to pinned host memory behind the work already on the stream.
 static int seq_read_back(Layer& L, int rows, cudaStream_t st)
@@ -375,6 +373,15 @@ static int seq_ensure(rrm_net* net, Layer& L, int T)
     void* stat = nullptr;
     if (cudaMalloc(&dP, (size_t)T * n * K * 4) != cudaSuccess) { cudaGetLastError(); return RRM_ERR_ALLOC; }
     if (cudaMalloc(&stat, (size_t)T * n * 2 * 4) != cudaSuccess) { cudaFree(dP); cudaGetLastError(); return RRM_ERR_ALLOC; }
+    if (L.seq_dP) {
+        // growing: the smaller arrays may still be in use by a chunk in flight; after that they are freed
+        cudaDeviceSynchronize();
+        for (void* old : {static_cast<void*>(L.seq_dP), static_cast<void*>(L.seq_stat)}) {
+            for (size_t i = 0; i < net->allocs.size(); ++i)
+                if (net->allocs[i] == old) { net->allocs.erase(net->allocs.begin() + i); break; }
+            cudaFree(old);
+        }
+    }
     net->allocs.push_back(dP);
     net->allocs.push_back(stat);
     L.seq_dP = reinterpret_cast<int32_t*>(dP);
@@ -441,8 +448,8 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
         // (up to 1024 rows go through the streaming form, 256 rows per launch, each launch at the cost of reading W
         // once: it wins as soon as the rows' gathered columns add up to about that many bytes)
         const bool use_dense = L.tc_ready && L.d.variant == RRM_VARIANT_AUTO && (long long)T * n >= 8 &&
-                               (fc_tc_usable(L, T * n) ? L.seq_density * T * n >= SQ_DENSE_SWITCH_ROWS * fc_tc_launches(T * n)
-                                                       : L.seq_density >= SQ_DENSE_SWITCH);
+                               (fc_tc_usable(L, T * n) ? L.seq_density * T * n >= (double)net->opt.fc_dense_rows * fc_tc_launches(T * n)
+                                                       : L.seq_density >= (double)net->opt.fc_dense_density);
         L.seq_last_T = T;
         L.seq_last_variant = use_dense ? RRM_VARIANT_DENSE : RRM_VARIANT_GATHER;
         if (use_dense) {

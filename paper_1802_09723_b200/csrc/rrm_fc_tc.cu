@@ -49,6 +49,7 @@ struct FtParams {
     int n;                    // streams
     int* errw;
     int rows, c_in, c_out, slabs, per, ksplit, bn, stages, tmem_cols, state_from, shift, act;
+    unsigned wait_limit;      // polls of one bounded wait
 };
 
 __device__ __forceinline__ int ft_apply_f(int v, int shift, int act)
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     tc_fence_after();
     const uint32_t tmem = S->tmem_base;
     bool ok = true;
+    int n_loaded = 0;                                        // loader: stages issued
 
     if (warp < 4) {
         // ================= the CTAs of the first output block refresh the input snapshot (their K share of the state rows)
@@ -175,13 +177,14 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
             const int8_t* src = p.Wimg + ((size_t)mtile * p.slabs + s_begin) * FT_A_BYTES;
             for (int it = 0; it < mine; ++it) {
                 const int stage = it % p.stages;
-                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / p.stages) & 1) ^ 1)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / p.stages) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
                 const uint32_t bar = smem_u32(&S->full[stage]);
                 const uint32_t dst = base_u32 + (uint32_t)stage * stage_bytes;
                 mbar_arrive_expect_tx(bar, stage_bytes);
                 asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                              ::"r"(dst + FT_A_BYTES), "l"(&tmapX), "r"((s_begin + it) * FT_SLAB), "r"(0), "r"(bar) : "memory");
                 bulk_copy_g2s(dst, src + (size_t)it * FT_A_BYTES, FT_A_BYTES, bar);
+                n_loaded = it + 1;
             }
         }
     } else {
@@ -190,7 +193,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
             const uint32_t idesc = tc_instr_desc(p.bn);
             for (int it = 0; it < mine; ++it) {
                 const int stage = it % p.stages;
-                if (!mbar_wait(smem_u32(&S->full[stage]), (it / p.stages) & 1)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&S->full[stage]), (it / p.stages) & 1, p.wait_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_addr = base_u32 + (uint32_t)stage * stage_bytes;
                 const uint64_t adesc = tc_smem_desc(a_addr), bdesc = tc_smem_desc(a_addr + FT_A_BYTES);
@@ -198,8 +201,19 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
                 for (int j = 0; j < 4; ++j)                  // 32 bytes of K per MMA: +2 in 16-byte address units
                     tc_mma_i8(tmem, adesc + 2 * j, bdesc + 2 * j, idesc, (it > 0 || j > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&S->empty[stage]));
+                n_loaded = it + 1;                           // (here: MMA groups issued)
             }
             if (ok) tc_commit(smem_u32(&S->done));
+            else {
+                // giving up: flagged first, so that the epilogue warps do not take the barrier for a finished tile;
+                // MMAs already issued must have completed before the tensor memory is freed
+                *(volatile int*)&S->last = -1;
+                __threadfence_block();
+                if (n_loaded > 0) {
+                    tc_commit(smem_u32(&S->done));
+                    mbar_wait(smem_u32(&S->done), 0, WAIT_LIMIT_DEFAULT);
+                }
+            }
         }
     }
     if (!ok) atomicOr(p.errw, ERRW_TIMEOUT);
@@ -209,7 +223,8 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     int* red = reinterpret_cast<int*>(base);                 // [rows][128] partial sums; the ring is free by then
     if (warp < 4) {
         ok = __all_sync(0xffffffffu, ok);
-        if (ok && !mbar_wait(smem_u32(&S->done), 0)) { ok = false; atomicOr(p.errw, ERRW_TIMEOUT); }
+        if (ok && !mbar_wait(smem_u32(&S->done), 0, p.wait_limit)) { ok = false; atomicOr(p.errw, ERRW_TIMEOUT); }
+        ok = ok && *(volatile int*)&S->last != -1;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
         if (ok) {
@@ -239,6 +254,11 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     }
     tc_fence_before();
     __syncthreads();
+    if (warp == 5 && lane == 0 && (!ok || S->last == -1)) {
+        // a role gave up: the loader's copies still in flight must land before the CTA's shared memory goes away
+        for (int j = max(0, n_loaded - p.stages); j < n_loaded; ++j)
+            mbar_wait(smem_u32(&S->full[j % p.stages]), (j / p.stages) & 1, WAIT_LIMIT_DEFAULT);
+    }
     if (warp == 4)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)p.tmem_cols) : "memory");
     if (p.ksplit == 1) return;
@@ -271,7 +291,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     }
 
     // ================= the last CTA of this output block closes it
-    if (tid == 0) S->last = atomicAdd(p.arrive + mtile, 1u) == (unsigned)p.ksplit - 1u;
+    if (tid == 0) S->last = atomicAdd(p.arrive + mtile, 1u) == (unsigned)p.ksplit - 1u;   // (overwrites a give-up mark)
     __syncthreads();
     if (!S->last) return;
     __threadfence();
@@ -393,6 +413,7 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
     p.errw = net->errw;
     p.c_in = C; p.c_out = K; p.slabs = L.tc_slabs; p.per = f.per; p.ksplit = f.ksplit;
     p.shift = L.d.shift; p.act = L.d.act;
+    p.wait_limit = net->opt.wait_limit;
     const size_t ybytes = (size_t)K * (L.d.shift < 0 ? 4 : 1);
     const int state_row = rows - n;                          // first row of the last frame
     const int8_t* old_snap = L.xs[L.xs_cur];

@@ -6,7 +6,7 @@
 
 namespace rrm {
 
-constexpr unsigned TC_SPIN_LIMIT = 1u << 20;    // polls of one mbarrier wait before it gives up
+constexpr unsigned WAIT_LIMIT_DEFAULT = 1u << 20;   // polls of one bounded wait before it gives up (rrm_options.wait_limit)
 constexpr int TC_M = 128;                       // accumulator rows of one MMA tile
 
 // ---- raw PTX wrappers ---------------------------------------------------------------------------
@@ -24,10 +24,11 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait for the phase with the given parity: at most `limit` polls; false when they ran out
+// (limit 0 gives up without polling, which is how a test makes a wait run out with nothing in flight).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned limit)
 {
-    for (unsigned i = 0; i < TC_SPIN_LIMIT; ++i) {
+    for (unsigned i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"

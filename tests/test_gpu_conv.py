@@ -57,7 +57,9 @@ def _compare(specs, net, frame, t, check_tensors=True):
             np.testing.assert_array_equal(T.astype(np.int64), tens_d[l + 1], err_msg=f"frame {t} tensor {l + 1}")
 
 
-def _run(specs, video, n=1, check_frames=None, stats=False, keyframe_at=(), variant="auto"):
+def _run(specs, video, n=1, check_frames=None, stats=False, keyframe_at=(), variant="auto", stats_frames=()):
+    """stats: compare every frame's counters with the literal recurrence (small stacks).  stats_frames: the same at
+    the named frames only, the recurrence being brought to the frame before by a dense pass (full-size stacks)."""
     rrm = _rrm()
     net = rrm.net_from_specs(specs, n=n, variant=variant)
     out = net.new_output()
@@ -81,6 +83,18 @@ def _run(specs, video, n=1, check_frames=None, stats=False, keyframe_at=(), vari
                     if specs[0].dtype != "f32" or l == 0:
                         assert st["nnz_elems"] == rec.nnz[l], (t, l, st, rec.nnz[l])
                         assert st["active_macs"] == rec.macs[l], (t, l, st, rec.macs[l])
+        if t in stats_frames:
+            one = orc.Recurrence(specs, n=n)
+            one.reset_to(video[t - 1])
+            one.step(video[t])
+            for l in range(len(specs)):
+                st = net.stats(l)
+                assert st["error_word"] == 0 and st["variant"] != 3, (t, l, st)
+                assert st["dense_macs"] == orc.layer_macs(specs[l]) * n
+                if specs[0].dtype != "f32" or l == 0:
+                    assert st["nnz_elems"] == one.nnz[l], (t, l, st, one.nnz[l])
+                    assert st["active_macs"] == one.macs[l], (t, l, st, one.macs[l])
+                assert 0 < st["active_out_pixels"] <= st["out_pixels"] and st["nnz_elems"] <= st["in_elems"]
         if check_frames is None or t in check_frames:
             _compare(specs, net, video[t], t)
             # the caller-owned output equals the last tensor
@@ -238,7 +252,7 @@ def test_cfg3_alexnet_fp32_full_size():
 def test_cfg3_alexnet_int8_full_size():
     specs = wl.alexnet_convs("i8")
     video = wl.moving_rect_video(frames=64, hw=227, dtype="i8", seed=32)
-    _run(specs, video, check_frames={0, 1, 30, 63})
+    _run(specs, video, check_frames={0, 1, 30, 63}, stats_frames={30})
 
 
 def test_cfg4_resnet18_int8_batch4():
@@ -247,10 +261,18 @@ def test_cfg4_resnet18_int8_batch4():
     _run(specs, video, n=4, check_frames={0, 1, 63})
 
 
+def test_cfg4_resnet18_int8_batch4_every_frame_through_the_delta_kernels():
+    """The same stack with the delta / dense switch off (variant "tensor"): every frame goes through the sparse
+    product at partial density, every layer's projection is compared at five frames, the counters at two."""
+    specs = wl.resnet18_convs()
+    video = wl.moving_rect_video(frames=64, hw=224, dtype="i8", seed=41, n=4, bg_redraw=0.02)
+    _run(specs, video, n=4, check_frames={0, 1, 16, 32, 63}, stats_frames={16, 63}, variant="tensor")
+
+
 def test_cfg5_xnor_alexnet_128_frames():
     specs = wl.xnor_alexnet_convs()
     video = wl.moving_rect_video(frames=128, hw=227, dtype="i8", seed=51)
-    _run(specs, video, check_frames={0, 1, 64, 127})
+    _run(specs, video, check_frames={0, 1, 64, 127}, stats_frames={64})
 
 
 # ------------------------------------------------------------------ chunks of frames through a stack (frames overlap layer by layer)

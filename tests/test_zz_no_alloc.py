@@ -1,4 +1,4 @@
-"""The allocation-free delta-FC entry point against the ordinary one.
+"""The allocation-free delta-FC entry point against the ordinary one and against the CPU oracle.
 
 Who needs it: callers that cannot allocate device memory - plug-ins whose host hands them a
 fixed memory budget and forbids cudaMalloc afterwards, real-time loops that must not wait on the
@@ -15,6 +15,7 @@ import pytest
 import torch
 
 import workloads as wl
+from oracle import rrm_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
@@ -47,6 +48,9 @@ def test_noalloc_entry_matches_rrm_step_on_consecutive_calls():
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before
         assert torch.equal(Y, Y_ref.reshape(n, c_out)), f"call {t}: output differs from rrm_step"
+        # ... and directly against the CPU oracle's dense evaluation of this frame (Eq. 3), bit for bit
+        want = orc.dense_forward([spec], seq[t])[1][0].reshape(n, c_out)
+        assert np.array_equal(Y.cpu().numpy().astype(np.int64), want), f"call {t}: output differs from the oracle"
         assert torch.equal(P, layer.projection(0).reshape(n, c_out)), f"call {t}: projection differs"
         assert torch.equal(Xprev, x), f"call {t}: snapshot not updated in place"
     layer.close()
