@@ -26,7 +26,9 @@
  *   - One object may be used from one stream at a time.
  *   - Environment switches, read when an object is created (debugging aids): RRM_NO_GRAPH=1 launches every
  *     kernel of a stack step on its own instead of replaying a captured CUDA graph; RRM_DEBUG=1 names a failing
- *     CUDA call (file, line, error string) on stderr and prints the shape of captured chunk graphs.
+ *     CUDA call (file, line, error string) on stderr and prints the shape of captured chunk graphs; RRM_PDL=1
+ *     launches the kernels of a stack step with programmatic dependent launch (each kernel's set-up overlaps its
+ *     predecessor's tail; off by default: measured, it does not pay inside replayed graphs).
  */
 #ifndef RRM_H
 #define RRM_H

@@ -92,7 +92,9 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int tile = blockIdx.x, n0 = blockIdx.y * TN;
+    pdl_launch_dependents();
     if (!DENSE) {
+        pdl_wait();                                          // the update bitmap is the predecessors' work
         // this CTA's rows: the tile-th group of TM set bits of the layer's update bitmap
         const int count = select_rows<TM>(p.oact, (p.opixels + 31) >> 5, tile, s_q, s_tmp);
         if (tile == 0 && blockIdx.y == 0 && blockIdx.z == 0 && tid == 0) *p.ocount = count;
@@ -178,6 +180,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     __syncthreads();
     const unsigned long long tm0 = (unsigned long long)s_tapmask[0] | (unsigned long long)s_tapmask[1] << 32;
     const unsigned long long tm1 = (unsigned long long)s_tapmask[2] | (unsigned long long)s_tapmask[3] << 32;
+    if (DENSE) pdl_wait();                                   // barriers and row tables are set up; the inputs come next
     // this CTA's share of the K stages
     const int all_stages = p.kup / TK, per_split = (all_stages + p.ksplit - 1) / p.ksplit;
     const int s_first = blockIdx.z * per_split, n_stages = min(all_stages, s_first + per_split);
@@ -354,8 +357,8 @@ static size_t gemm_smem_bytes(int dt)
 template <int DT, bool DENSE>
 static void launch_gemm(const ConvParams& p, dim3 grid, cudaStream_t st)
 {
-    if (p.u_in % 4 == 0) conv_gemm_kernel<DT, DENSE, true><<<grid, CONV_THREADS, gemm_smem_bytes(DT), st>>>(p);
-    else conv_gemm_kernel<DT, DENSE, false><<<grid, CONV_THREADS, gemm_smem_bytes(DT), st>>>(p);
+    if (p.u_in % 4 == 0) launch_seq(conv_gemm_kernel<DT, DENSE, true>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, p);
+    else launch_seq(conv_gemm_kernel<DT, DENSE, false>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, p);
 }
 
 template <int DT>
@@ -422,6 +425,8 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
     const int ld = cs + 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ns = blockIdx.y, pix0 = blockIdx.x * IMP_TP;
+    pdl_launch_dependents();
+    pdl_wait();
     if (tid < IMP_TP) s_cnt[tid] = 0;
     for (int ch = warp; ch < cs; ch += 8) {
         T v = 0;
@@ -512,6 +517,8 @@ __global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __res
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
     const int hw = h * w;
+    pdl_launch_dependents();
+    pdl_wait();
     int cnt = 0;
     if (gp < pixels) {
         const int ns = gp / hw, pix = gp - ns * hw;
@@ -565,6 +572,8 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
                                   int h, int w, Readers readers)
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     int cnt = 0;
     if (gp < pixels) {
         for (int k = 0; k < cw; ++k) {
@@ -636,8 +645,10 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     __shared__ int s_cnt[8];                                 // changed elements of the CTA's pixels (one per warp)
     __shared__ float s_sq;
     const int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
     if (threadIdx.x < MAX_READERS) s_macs[threadIdx.x] = 0;
     if (threadIdx.x == 0) { s_nnz = 0; s_npix = 0; s_sq = 0.f; }
+    pdl_wait();                                              // the projection (and its update bitmap) is the convolution's work
     __syncthreads();
     const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int tpix = p.n * p.th * p.tw;
@@ -821,6 +832,8 @@ template <typename T>
 __global__ void export_nchw_kernel(const T* __restrict__ src, T* dst, int c, int cs, int hw, long long total)
 {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     if (i >= total) return;
     const int pix = (int)(i % hw);
     const int ch = (int)((i / hw) % c);
@@ -839,6 +852,8 @@ __global__ void fill_projection_kernel(T* P, const T* bias, int c_out, long long
 struct AecsParams { const double* sumsq[64]; int n; double* e_t; double* last_l2; };
 __global__ void aecs_accumulate_kernel(AecsParams p)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     double add = 0.0;
     for (int l = 0; l < p.n; ++l) { const double v = sqrt(*p.sumsq[l]); p.last_l2[l] = v; add += v; }
@@ -911,18 +926,18 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
     const int hw = T.h * T.w;
     if (T.dtype == T_BIN) {
         const int blocks = ceil_div(T.pixels(), 256);
-        if (delta) import_bin_kernel<true><<<blocks, 256, 0, st>>>((const uint32_t*)frame, (uint32_t*)X, (uint32_t*)T.D,
+        if (delta) launch_seq(import_bin_kernel<true>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, (uint32_t*)T.D,
                                                                   T.act, T.pnnz, T.nnz, T.npix, T.cs, T.pixels(),
                                                                   T.h, T.w, T.readers);
-        else import_bin_kernel<false><<<blocks, 256, 0, st>>>((const uint32_t*)frame, (uint32_t*)X, nullptr, nullptr,
+        else launch_seq(import_bin_kernel<false>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, nullptr, nullptr,
                                                               nullptr, nullptr, nullptr, T.cs, T.pixels(), T.h, T.w,
                                                               Readers{});
     } else if (T.dtype == T_I8 && T.cs == 4) {
         const int blocks = ceil_div(T.pixels(), 256);
-        if (delta) import_i8_word_kernel<true><<<blocks, 256, 0, st>>>((const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
+        if (delta) launch_seq(import_i8_word_kernel<true>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
                                                                       T.pnnz, T.nnz, T.npix, net->errw, T.c, T.h, T.w,
                                                                       T.pixels(), T.readers);
-        else import_i8_word_kernel<false><<<blocks, 256, 0, st>>>((const int8_t*)frame, (uint32_t*)X, nullptr, nullptr, nullptr,
+        else launch_seq(import_i8_word_kernel<false>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, nullptr, nullptr, nullptr,
                                                                   nullptr, nullptr, net->errw, T.c, T.h, T.w, T.pixels(),
                                                                   Readers{});
     } else {
@@ -935,9 +950,9 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                 cudaFuncSetAttribute(kd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             }
-            if (delta) kd<<<grid, 256, smem, st>>>((const float*)frame, (float*)X, (float*)T.D, T.act, T.pnnz, T.nnz,
+            if (delta) launch_seq(kd, dim3(grid), dim3(256), smem, st, (const float*)frame, (float*)X, (float*)T.D, T.act, T.pnnz, T.nnz,
                                                    T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, net->eps, T.trunc);
-            else kn<<<grid, 256, smem, st>>>((const float*)frame, (float*)X, nullptr, nullptr, nullptr, nullptr,
+            else launch_seq(kn, dim3(grid), dim3(256), smem, st, (const float*)frame, (float*)X, nullptr, nullptr, nullptr, nullptr,
                                              nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr);
         } else {
             auto kd = import_nchw_kernel<int8_t, true>;
@@ -946,9 +961,9 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                 cudaFuncSetAttribute(kd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             }
-            if (delta) kd<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, (int8_t*)T.D, T.act, T.pnnz,
+            if (delta) launch_seq(kd, dim3(grid), dim3(256), smem, st, (const int8_t*)frame, (int8_t*)X, (int8_t*)T.D, T.act, T.pnnz,
                                                    T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, 0.f, nullptr);
-            else kn<<<grid, 256, smem, st>>>((const int8_t*)frame, (int8_t*)X, nullptr, nullptr, nullptr, nullptr,
+            else launch_seq(kn, dim3(grid), dim3(256), smem, st, (const int8_t*)frame, (int8_t*)X, nullptr, nullptr, nullptr, nullptr,
                                              nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr);
         }
     }
@@ -961,9 +976,9 @@ static int launch_epi_k(const EpiParams& e, int blocks, cudaStream_t st)
 {
     const bool rd = !DENSE && e.readers.n > 0;               // (a dense pass marks nothing)
     switch (e.pool_k > 0 ? e.pool_k : 1) {
-        case 1: if (rd) epilogue_kernel<PT, OT, DENSE, 1, !DENSE><<<blocks, 256, 0, st>>>(e); else epilogue_kernel<PT, OT, DENSE, 1, false><<<blocks, 256, 0, st>>>(e); break;
-        case 2: if (rd) epilogue_kernel<PT, OT, DENSE, 2, !DENSE><<<blocks, 256, 0, st>>>(e); else epilogue_kernel<PT, OT, DENSE, 2, false><<<blocks, 256, 0, st>>>(e); break;
-        case 3: if (rd) epilogue_kernel<PT, OT, DENSE, 3, !DENSE><<<blocks, 256, 0, st>>>(e); else epilogue_kernel<PT, OT, DENSE, 3, false><<<blocks, 256, 0, st>>>(e); break;
+        case 1: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 1, !DENSE>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 1, false>, dim3(blocks), dim3(256), 0, st, e); break;
+        case 2: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 2, !DENSE>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 2, false>, dim3(blocks), dim3(256), 0, st, e); break;
+        case 3: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 3, !DENSE>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 3, false>, dim3(blocks), dim3(256), 0, st, e); break;
         default: return RRM_ERR_UNSUPPORTED;                 // pool windows are 2x2 or 3x3
     }
     return RRM_OK;
@@ -1043,7 +1058,7 @@ int launch_aecs(rrm_net* net, cudaStream_t st)
     if (a.n > 64) return RRM_ERR_UNSUPPORTED;
     for (int l = 0; l < a.n; ++l) a.sumsq[l] = net->tensors[net->layers[l].d.src].trunc;
     a.e_t = net->aecs; a.last_l2 = net->aecs + 1;
-    aecs_accumulate_kernel<<<1, 32, 0, st>>>(a);
+    launch_seq(aecs_accumulate_kernel, dim3(1), dim3(32), 0, st, a);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
@@ -1059,8 +1074,8 @@ int launch_export_tensor(rrm_net* net, int t, void* dst, bool stateless, cudaStr
     const int hw = T.h * T.w;
     const long long total = (long long)T.n * T.c * hw;
     const int blocks = (int)((total + 255) / 256);
-    if (T.dtype == T_I8) export_nchw_kernel<int8_t><<<blocks, 256, 0, st>>>((const int8_t*)X, (int8_t*)dst, T.c, T.cs, hw, total);
-    else export_nchw_kernel<uint32_t><<<blocks, 256, 0, st>>>((const uint32_t*)X, (uint32_t*)dst, T.c, T.cs, hw, total);
+    if (T.dtype == T_I8) launch_seq(export_nchw_kernel<int8_t>, dim3(blocks), dim3(256), 0, st, (const int8_t*)X, (int8_t*)dst, T.c, T.cs, hw, total);
+    else launch_seq(export_nchw_kernel<uint32_t>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)X, (uint32_t*)dst, T.c, T.cs, hw, total);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
@@ -1070,7 +1085,7 @@ int launch_export_projection(rrm_net* net, int l, void* dst, cudaStream_t st)
     Layer& L = net->layers[l];
     const int hw = L.oh * L.ow;
     const long long total = (long long)L.d.n * L.d.c_out * hw;
-    export_nchw_kernel<uint32_t><<<(int)((total + 255) / 256), 256, 0, st>>>((const uint32_t*)L.P, (uint32_t*)dst,
+    launch_seq(export_nchw_kernel<uint32_t>, dim3((int)((total + 255) / 256)), dim3(256), 0, st, (const uint32_t*)L.P, (uint32_t*)dst,
                                                                             L.d.c_out, L.d.c_out, hw, total);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;

@@ -79,7 +79,9 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     const uint32_t base_u32 = smem_u32(base);
     __shared__ int s_tmp[256 + 34];
     int count = p.opixels;
+    pdl_launch_dependents();
     if (!DENSE) {
+        pdl_wait();                                          // the update bitmap is the predecessors' work
         // this CTA's rows: the tile-th group of 128 set bits of the layer's update bitmap
         count = select_rows<TC_M>(p.oact, (p.opixels + 31) >> 5, tile, S->q, s_tmp);
         if (tile == 0 && ntile == 0 && split == 0 && tid == 0) *p.ocount = count;
@@ -178,6 +180,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (DENSE) pdl_wait();                                   // barriers, tensor memory and row tables are set up; the inputs come next
     const uint32_t tmem = S->tmem_base;
     const unsigned long long tm0 = S->tap_mask[0], tm1 = S->tap_mask[1];
 
@@ -514,6 +517,8 @@ __global__ void pack_weights_tc_kernel(const int8_t* W, int8_t* img, int c_in, i
 __global__ void zero_projection_kernel(int32_t* P, long long total)
 {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();                                              // the predecessor may still read the projection
     if (i < total) P[i] = 0;
 }
 
@@ -522,7 +527,7 @@ __global__ void zero_projection_kernel(int32_t* P, long long total)
 // ------------------------------------------------------------------------------------------------
 int zero_projection(void* P, long long words, cudaStream_t st)
 {
-    zero_projection_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(reinterpret_cast<int32_t*>(P), words);
+    launch_seq(zero_projection_kernel, dim3((unsigned)((words + 255) / 256)), dim3(256), 0, st, reinterpret_cast<int32_t*>(P), words);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
@@ -599,15 +604,15 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.ksplit = ksplit;
     if (dense && ksplit > 1) {
         const long long tot = (long long)L.opixels() * d.c_out;
-        zero_projection_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(p.P, tot);
+        launch_seq(zero_projection_kernel, dim3((unsigned)((tot + 255) / 256)), dim3(256), 0, st, p.P, tot);
     }
     dim3 grid(m_tiles, L.tc_ntiles, ksplit);
     if (bin) {
-        if (dense) conv_tc_kernel<true, true><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(p);
-        else conv_tc_kernel<true, false><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(p);
+        if (dense) launch_seq(conv_tc_kernel<true, true>, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, p);
+        else launch_seq(conv_tc_kernel<true, false>, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, p);
     } else {
-        if (dense) conv_tc_kernel<false, true><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(p);
-        else conv_tc_kernel<false, false><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(p);
+        if (dense) launch_seq(conv_tc_kernel<false, true>, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, p);
+        else launch_seq(conv_tc_kernel<false, false>, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, p);
     }
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
