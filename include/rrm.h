@@ -58,12 +58,18 @@ enum { RRM_CONV = 0, RRM_FC = 1 };
 enum { RRM_F32 = 0, RRM_I8 = 1, RRM_BIN = 2 };
 enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2,
        RRM_ACT_LEAKY = 3 /* fp32 only: x > 0 ? x : 0.1 x, the leaky ReLU of the YOLOv2-style stacks of Sec. 4.4 */ };
-/* How F*dI is evaluated.  As a request in rrm_layer_desc.variant: AUTO lets the library pick per layer (tensor
- * cores for int8 and binary layers, CUDA cores for fp32; for a lone int8 FC layer also: dense evaluation of a chunk
- * when the previous chunk's measured delta density was high); GATHER forces the CUDA-core / column-gather kernels;
- * TENSOR is AUTO without the density switch; DENSE on a lone FC layer selects the generic (non-fused) path.
- * As a report in rrm_stats.variant: what the most recent step ran (GATHER, TENSOR, or DENSE for a chunk that was
- * evaluated densely). */
+/* How F*dI is evaluated.  As a request in rrm_layer_desc.variant: AUTO lets the library pick per layer: the kernel
+ * (tensor cores for int8 and binary layers, CUDA cores for fp32) and, from the measured density, whether the layer
+ * runs the sparse product at all.  In a stack whose layers all ask for AUTO every layer's share of projection
+ * pixels to update is read back after each delta step (asynchronously); a layer whose share reached
+ * rrm_options.layer_dense_activity is evaluated densely inside the following delta steps (P = F*X + b from the
+ * current input replaces its stored projection; its input delta is still formed and counted, and its output delta
+ * still emitted), and returns to the sparse product below rrm_options.layer_delta_activity.  For a lone int8 FC
+ * layer AUTO also means: dense evaluation of a chunk when the previous chunk's measured delta density was high.
+ * GATHER forces the CUDA-core / column-gather kernels; TENSOR is AUTO without any density switch; DENSE on a lone
+ * FC layer selects the generic (non-fused) path.
+ * As a report in rrm_stats.variant: what the most recent step ran for this layer (GATHER, TENSOR, or DENSE for a
+ * layer or chunk that was evaluated densely). */
 enum { RRM_VARIANT_AUTO = 0, RRM_VARIANT_GATHER = 1, RRM_VARIANT_TENSOR = 2, RRM_VARIANT_DENSE = 3 };
 
 /*
@@ -213,7 +219,8 @@ int rrm_net_keyframe(rrm_net* net, const void* frame_dev, void* out_dev, void* s
  * projection pixels the last delta frame had to update; while that share, weighted by the layers' MACs, is
  * 75 % or more it evaluates frames densely instead (a precise inference that replaces the state: the same
  * results), and measures again with a delta frame every 16th frame.  rrm_net_get_stats reports such a frame
- * with variant RRM_VARIANT_DENSE and its counters as -1 (nothing was counted). */
+ * with variant RRM_VARIANT_DENSE and its counters as -1 (nothing was counted).  Below that share the choice is
+ * made layer by layer (see RRM_VARIANT_AUTO): such layers report RRM_VARIANT_DENSE with their counters intact. */
 int rrm_net_step(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);
 /* Dense evaluation of the stack without touching the RRM state. */
 int rrm_net_dense(rrm_net* net, const void* frame_dev, void* out_dev, void* stream);

@@ -197,6 +197,12 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
             all_auto = all_auto && L.d.variant == RRM_VARIANT_AUTO;
         }
         net->auto_switch = all_auto && macs >= 1000000000ll;
+        net->layer_switch = all_auto && n_layers <= 64;
+        // an all-ones bitmap stands in for a layer's update bitmap when the layer is evaluated densely inside a delta step
+        int words = 1;
+        for (auto& L : net->layers) words = words > ceil_div(L.opixels(), 32) ? words : ceil_div(L.opixels(), 32);
+        RRM_TRY(dev_alloc(net, (void**)&net->ones, (size_t)words * 4));
+        RRM_CUDA_TRY(cudaMemset(net->ones, 0xff, (size_t)words * 4));
     }
     {
         const char* e = getenv("RRM_NO_GRAPH");
@@ -209,19 +215,21 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     return RRM_OK;
 }
 
-int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
-int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless);
+int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless,
+                    unsigned long long mask = 0);
+int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless,
+                 unsigned long long mask = 0);
 
 // Finds the nodes of a captured sequence that hold the fixed frame / output buffers, so that each launch can
 // point them at the caller's buffers instead of copying through the fixed ones.  Any doubt (an API error, no
 // node found) leaves patch_ok false and the copies in place.
-void find_io_nodes(rrm_net* net, int kind)
+void find_io_nodes(rrm_net* net, rrm_net::StepGraph& sg)
 {
-    net->patch_in[kind].clear(); net->patch_out[kind].clear(); net->patch_ok[kind] = false;
+    sg.patch_in.clear(); sg.patch_out.clear(); sg.patch_ok = false;
     size_t n = 0;
-    if (cudaGraphGetNodes(net->graph[kind], nullptr, &n) != cudaSuccess || n == 0) { cudaGetLastError(); return; }
+    if (cudaGraphGetNodes(sg.graph, nullptr, &n) != cudaSuccess || n == 0) { cudaGetLastError(); return; }
     std::vector<cudaGraphNode_t> nodes(n);
-    if (cudaGraphGetNodes(net->graph[kind], nodes.data(), &n) != cudaSuccess) { cudaGetLastError(); return; }
+    if (cudaGraphGetNodes(sg.graph, nodes.data(), &n) != cudaSuccess) { cudaGetLastError(); return; }
     for (cudaGraphNode_t node : nodes) {
         cudaGraphNodeType type;
         if (cudaGraphNodeGetType(node, &type) != cudaSuccess) { cudaGetLastError(); return; }
@@ -243,7 +251,7 @@ void find_io_nodes(rrm_net* net, int kind)
                 if (v != net->frame_buf && v != net->out_buf) continue;
                 rrm_net::IoPatch pt;
                 pt.node = node; pt.kp = kp; pt.args = args; pt.index = (int)i;
-                (v == net->frame_buf ? net->patch_in[kind] : net->patch_out[kind]).push_back(pt);
+                (v == net->frame_buf ? sg.patch_in : sg.patch_out).push_back(pt);
             }
         } else if (type == cudaGraphNodeTypeMemcpy) {
             cudaMemcpy3DParms mp = {};
@@ -251,30 +259,30 @@ void find_io_nodes(rrm_net* net, int kind)
             if (mp.dstPtr.ptr == net->out_buf && mp.extent.height <= 1 && mp.extent.depth <= 1) {
                 rrm_net::IoPatch pt;
                 pt.node = node; pt.is_copy = true; pt.src = mp.srcPtr.ptr; pt.bytes = mp.extent.width;
-                net->patch_out[kind].push_back(pt);
+                sg.patch_out.push_back(pt);
             } else if (mp.dstPtr.ptr == net->out_buf || mp.srcPtr.ptr == net->frame_buf) {
                 return;                                      // a copy of another shape: leave everything as it is
             }
         }
     }
-    net->patch_ok[kind] = net->patch_in[kind].size() == 1 && net->patch_out[kind].size() == 1;
+    sg.patch_ok = sg.patch_in.size() == 1 && sg.patch_out.size() == 1;
 }
 
 // Points the frame / output nodes of the instantiated graph at `frame` and `out`.
-int patch_io(rrm_net* net, int kind, const void* frame, void* out)
+int patch_io(rrm_net* net, rrm_net::StepGraph& sg, const void* frame, void* out)
 {
     for (int side = 0; side < 2; ++side) {
-        rrm_net::IoPatch& pt = side == 0 ? net->patch_in[kind][0] : net->patch_out[kind][0];
+        rrm_net::IoPatch& pt = side == 0 ? sg.patch_in[0] : sg.patch_out[0];
         void* target = side == 0 ? const_cast<void*>(frame) : (out ? out : net->out_buf);
         if (pt.value == target) continue;                    // already there
         if (pt.is_copy) {
-            RRM_CUDA_TRY(cudaGraphExecMemcpyNodeSetParams1D(net->exec[kind], pt.node, target, pt.src, pt.bytes,
+            RRM_CUDA_TRY(cudaGraphExecMemcpyNodeSetParams1D(sg.exec, pt.node, target, pt.src, pt.bytes,
                                                             cudaMemcpyDeviceToDevice));
         } else {
             pt.value = target;
             pt.args[pt.index] = &pt.value;
             pt.kp.kernelParams = pt.args.data();
-            RRM_CUDA_TRY(cudaGraphExecKernelNodeSetParams(net->exec[kind], pt.node, &pt.kp));
+            RRM_CUDA_TRY(cudaGraphExecKernelNodeSetParams(sg.exec, pt.node, &pt.kp));
         }
         pt.value = target;
     }
@@ -283,7 +291,15 @@ int patch_io(rrm_net* net, int kind, const void* frame, void* out)
 
 // Captures one of the per-frame launch sequences into a graph (on a private stream: a capture cannot
 // start on the legacy default stream) so that later frames cost one graph launch on the host.
-int build_graph(rrm_net* net, int kind)
+constexpr size_t STEP_GRAPHS_KEPT = 12;         // layer masks whose delta-step graphs are kept
+
+rrm_net::StepGraph* find_step_graph(rrm_net* net, int kind, unsigned long long mask)
+{
+    for (auto& g : net->step_graphs[kind]) if (g.mask == mask) return &g;
+    return nullptr;
+}
+
+int build_graph(rrm_net* net, int kind, unsigned long long mask)
 {
     const bool dense = kind != 0, stateless = kind == 2;
     int64_t bi = 0, bo = 0;
@@ -294,13 +310,23 @@ int build_graph(rrm_net* net, int kind)
     if (stateless) RRM_TRY(ensure_stateless(net));           // allocations cannot happen inside a capture
     if (!net->cap_stream) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
     RRM_CUDA_TRY(cudaStreamBeginCapture(net->cap_stream, cudaStreamCaptureModeThreadLocal));
-    const int s = launch_sequence(net, net->frame_buf, net->out_buf, net->cap_stream, dense, stateless);
+    const int s = launch_sequence(net, net->frame_buf, net->out_buf, net->cap_stream, dense, stateless, mask);
     cudaGraph_t g = nullptr;
     const cudaError_t e = cudaStreamEndCapture(net->cap_stream, &g);
     if (s != RRM_OK || e != cudaSuccess || !g) { if (g) cudaGraphDestroy(g); cudaGetLastError(); return s != RRM_OK ? s : RRM_ERR_CUDA; }
-    net->graph[kind] = g;
-    RRM_CUDA_TRY(cudaGraphInstantiate(&net->exec[kind], g, 0));
-    find_io_nodes(net, kind);
+    auto& cache = net->step_graphs[kind];
+    if (cache.size() >= STEP_GRAPHS_KEPT) {                  // drop the mask that has not been used for the longest time
+        size_t old = 0;
+        for (size_t i = 1; i < cache.size(); ++i) if (cache[i].used < cache[old].used) old = i;
+        if (cache[old].exec) cudaGraphExecDestroy(cache[old].exec);
+        if (cache[old].graph) cudaGraphDestroy(cache[old].graph);
+        cache.erase(cache.begin() + old);
+    }
+    rrm_net::StepGraph sg;
+    sg.mask = mask; sg.graph = g;
+    if (cudaGraphInstantiate(&sg.exec, g, 0) != cudaSuccess) { cudaGraphDestroy(g); cudaGetLastError(); return RRM_ERR_CUDA; }
+    find_io_nodes(net, sg);
+    cache.push_back(std::move(sg));
     return RRM_OK;
 }
 
@@ -316,10 +342,12 @@ void drop_chunk_graphs(rrm_net* net, int kind)
 void drop_graphs(rrm_net* net)
 {
     for (int k = 0; k < 3; ++k) {
-        net->patch_in[k].clear(); net->patch_out[k].clear(); net->patch_ok[k] = false;
         drop_chunk_graphs(net, k);
-        if (net->exec[k]) { cudaGraphExecDestroy(net->exec[k]); net->exec[k] = nullptr; }
-        if (net->graph[k]) { cudaGraphDestroy(net->graph[k]); net->graph[k] = nullptr; }
+        for (auto& g : net->step_graphs[k]) {
+            if (g.exec) cudaGraphExecDestroy(g.exec);
+            if (g.graph) cudaGraphDestroy(g.graph);
+        }
+        net->step_graphs[k].clear();
     }
 }
 
@@ -337,21 +365,30 @@ int activity_read_back(rrm_net* net, cudaStream_t st)
     return RRM_OK;
 }
 
+// Takes in the counters of the last measured delta step, once their copy has landed (never waited for): the
+// MAC-weighted activity of the stack, and per layer the share of projection pixels it had to update, from which
+// the layer's mode in the following steps is chosen (with a hysteresis between the two thresholds).
 void activity_poll(rrm_net* net)
 {
     if (!net->act_pending || cudaEventQuery(net->act_ev) != cudaSuccess) { cudaGetLastError(); return; }
     net->act_pending = false;
     double num = 0, den = 0;
     const size_t base = net->tensors.size() * 32;
+    unsigned long long mask = 0;
     for (size_t l = 0; l < net->layers.size(); ++l) {
-        const Layer& L = net->layers[l];
+        Layer& L = net->layers[l];
         int oc = 0;
         std::memcpy(&oc, net->act_host + base + l * 16 + 8, 4);
         const double macs = (double)L.opixels() * L.d.c_out * L.d.c_in * L.d.kh * L.d.kw;
-        num += macs * oc / (double)L.opixels();
+        L.activity = oc / (double)L.opixels();
+        num += macs * L.activity;
         den += macs;
+        if (L.activity >= net->opt.layer_dense_activity) L.dense_mode = true;
+        else if (L.activity < net->opt.layer_delta_activity) L.dense_mode = false;
+        if (L.dense_mode && l < 64) mask |= 1ull << l;
     }
     net->activity = den > 0 ? num / den : -1.0;
+    net->layer_mask = net->layer_switch ? mask : 0;
 }
 
 int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
@@ -364,63 +401,73 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
         RRM_TRY(bind_readers(net));
     }
     const bool is_step = !dense && !stateless;
+    unsigned long long mask = 0;
     if (is_step) {
-        // the variant of this frame from the measured activity of the last delta frame (temporal coherence):
-        // a dense pass that replaces the state gives the same results, so the switch is invisible in the outputs
+        // how this frame is evaluated follows from the measured activity of the last delta frame (temporal
+        // coherence).  A whole stack of >= 1 GMAC with nearly every pixel changing is evaluated densely (a precise
+        // inference that replaces the state: the same results, and no delta bookkeeping at all); otherwise every
+        // layer on its own runs the sparse product or, above its threshold, a dense evaluation inside the delta step.
         net->last_step_dense = false;
-        if (net->auto_switch && net->eps == 0.f) {
+        if ((net->auto_switch || net->layer_switch) && net->eps == 0.f) {
             activity_poll(net);
-            if (net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
+            if (net->auto_switch && net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
                 ++net->dense_streak;
                 net->last_step_dense = true;
                 dense = true;
             } else {
                 net->dense_streak = 0;
+                mask = net->layer_mask;
             }
         }
+        if (!dense) for (size_t l = 0; l < net->layers.size(); ++l) net->layers[l].ran_dense = l < 64 && (mask >> l & 1ull);
     }
-    const int s_run = run_sequence(net, frame, out, st, dense, stateless);
-    if (s_run == RRM_OK && is_step && !dense && net->auto_switch) RRM_TRY(activity_read_back(net, st));
+    const int s_run = run_sequence(net, frame, out, st, dense, stateless, mask);
+    if (s_run == RRM_OK && is_step && !dense && (net->auto_switch || net->layer_switch) && net->eps == 0.f)
+        RRM_TRY(activity_read_back(net, st));
     return s_run;
 }
 
-int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
+int run_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless,
+                 unsigned long long mask)
 {
     if (!net->graph_off) {
         const int kind = !dense ? 0 : (stateless ? 2 : 1);
-        if (!net->exec[kind]) {
-            const int s = build_graph(net, kind);
+        if (!find_step_graph(net, kind, mask)) {
+            const int s = build_graph(net, kind, mask);
             if (s != RRM_OK) { net->graph_off = true; if (s == RRM_ERR_ALLOC) return s; }
         }
-        if (net->exec[kind]) {
+        if (rrm_net::StepGraph* sg = find_step_graph(net, kind, mask)) {
+            sg->used = ++net->step_clock;
             int64_t bi = 0, bo = 0;
             tensor_bytes_boundary(net->tensors.front(), &bi);
             tensor_bytes_boundary(net->tensors.back(), &bo);
-            if (net->patch_ok[kind] && patch_io(net, kind, frame, out) == RRM_OK) {
-                RRM_CUDA_TRY(cudaGraphLaunch(net->exec[kind], st));
+            if (sg->patch_ok && patch_io(net, *sg, frame, out) == RRM_OK) {
+                RRM_CUDA_TRY(cudaGraphLaunch(sg->exec, st));
                 return RRM_OK;
             }
-            if (net->patch_ok[kind]) {
+            if (sg->patch_ok) {
                 // an update failed half-way: the graphs are no longer trusted, launch kernel by kernel from now on
                 cudaGetLastError();
                 drop_graphs(net);
                 net->graph_off = true;
-                return launch_sequence(net, frame, out, st, dense, stateless);
+                return launch_sequence(net, frame, out, st, dense, stateless, mask);
             }
             RRM_CUDA_TRY(cudaMemcpyAsync(net->frame_buf, frame, (size_t)bi, cudaMemcpyDeviceToDevice, st));
-            RRM_CUDA_TRY(cudaGraphLaunch(net->exec[kind], st));
+            RRM_CUDA_TRY(cudaGraphLaunch(sg->exec, st));
             if (out) RRM_CUDA_TRY(cudaMemcpyAsync(out, net->out_buf, (size_t)bo, cudaMemcpyDeviceToDevice, st));
             return RRM_OK;
         }
     }
-    return launch_sequence(net, frame, out, st, dense, stateless);
+    return launch_sequence(net, frame, out, st, dense, stateless, mask);
 }
 
-int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless)
+int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense, bool stateless,
+                    unsigned long long mask)
 {
     if (!stateless) RRM_CUDA_TRY(cudaMemsetAsync(net->cleared, 0, net->cleared_bytes, st));
     RRM_TRY(launch_import(net, frame, !dense, stateless, st));
-    for (int l = 0; l < (int)net->layers.size(); ++l) RRM_TRY(launch_layer(net, l, dense, stateless, st));
+    for (int l = 0; l < (int)net->layers.size(); ++l)
+        RRM_TRY(launch_layer(net, l, dense, stateless, st, nullptr, !dense && l < 64 && (mask >> l & 1ull)));
     if (!dense && net->eps > 0.f) RRM_TRY(launch_aecs(net, st));
     if (dense && !stateless) RRM_CUDA_TRY(cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, st));   // a precise inference clears e_t
     if (out) RRM_TRY(launch_export_tensor(net, (int)net->layers.size(), out, stateless, st));
@@ -428,7 +475,7 @@ int launch_sequence(rrm_net* net, const void* frame, void* out, cudaStream_t st,
 }
 
 constexpr int CHUNK_MAX_SLOTS = 24;             // capture streams = frames in flight
-constexpr size_t CHUNK_GRAPHS_KEPT = 4;         // chunk lengths whose graphs are kept per kind
+constexpr size_t CHUNK_GRAPHS_KEPT = 8;         // (chunk length, layer mask) pairs whose graphs are kept per kind
 constexpr int CHUNK_ARENAS = 64;                // arenas of the chunk graphs (>= CHUNK_MAX_SLOTS)
 
 // Streams, events, arenas and staging buffers of the pipelined chunk graphs.
@@ -478,7 +525,7 @@ int ensure_chunk(rrm_net* net, int T)
 //   frame's readers of that tensor (convolutions that take it as input, epilogues that add it as shortcut, the export
 //   of the last tensor), because it overwrites the snapshot and the delta rows they read.
 // Everything else of consecutive frames may overlap.
-int build_chunk_graph(rrm_net* net, int kind, int T)
+int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
 {
     const bool dense = kind != 0, stateless = kind == 2;
     const int L = (int)net->layers.size();
@@ -523,7 +570,7 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
                 else { record(net->ev_epi[l], s); epi_rec[l] = 1; }
                 return status;
             };
-            const int q = launch_layer(net, l, dense, stateless, s, &hook);
+            const int q = launch_layer(net, l, dense, stateless, s, &hook, !dense && l < 64 && (mask >> l & 1ull));
             if (q != RRM_OK) fail(q);
         }
         if (dense && !stateless && cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, s) != cudaSuccess) fail(RRM_ERR_CUDA);
@@ -549,7 +596,7 @@ int build_chunk_graph(rrm_net* net, int kind, int T)
         cache.erase(cache.begin() + old);
     }
     rrm_net::ChunkGraph c;
-    c.T = T; c.graph = g;
+    c.T = T; c.mask = mask; c.graph = g;
     if (cudaGraphInstantiate(&c.exec, g, 0) != cudaSuccess) { cudaGraphDestroy(g); cudaGetLastError(); return RRM_ERR_CUDA; }
     c.used = ++net->chunk_clock;
     cache.push_back(c);
@@ -567,27 +614,30 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
 {
     if (net->graph_off || net->eps > 0.f || T < 2) return RRM_ERR_UNSUPPORTED;
     const bool is_step = !dense && !stateless;
+    unsigned long long mask = 0;
     if (is_step) {
         // one decision per chunk, from the measured activity of the last delta frame (as rrm_net_step does per frame)
         net->last_step_dense = false;
-        if (net->auto_switch) {
+        if (net->auto_switch || net->layer_switch) {
             activity_poll(net);
-            if (net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
+            if (net->auto_switch && net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
                 ++net->dense_streak;                         // (counted in calls: a delta chunk measures again after 15 dense ones)
                 net->last_step_dense = true;
                 dense = true;
             } else {
                 net->dense_streak = 0;
+                mask = net->layer_mask;
             }
         }
+        if (!dense) for (size_t l = 0; l < net->layers.size(); ++l) net->layers[l].ran_dense = l < 64 && (mask >> l & 1ull);
     }
     const int kind = !dense ? 0 : (stateless ? 2 : 1);
     auto find = [&]() -> rrm_net::ChunkGraph* {
-        for (auto& c : net->chunk_graphs[kind]) if (c.T == T) return &c;
+        for (auto& c : net->chunk_graphs[kind]) if (c.T == T && c.mask == mask) return &c;
         return nullptr;
     };
     if (!find()) {
-        const int s = build_chunk_graph(net, kind, T);
+        const int s = build_chunk_graph(net, kind, T, mask);
         if (s != RRM_OK) {
             cudaGetLastError();
             bind_arena(net, reinterpret_cast<char*>(net->cleared));
@@ -607,7 +657,7 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
     cg->used = ++net->chunk_clock;
     RRM_CUDA_TRY(cudaGraphLaunch(cg->exec, st));
     if (outs) RRM_CUDA_TRY(cudaMemcpyAsync(outs, net->chunk_out, (size_t)bo * T, cudaMemcpyDeviceToDevice, st));
-    if (is_step && !dense && net->auto_switch) RRM_TRY(activity_read_back(net, st));
+    if (is_step && !dense && (net->auto_switch || net->layer_switch)) RRM_TRY(activity_read_back(net, st));
     return RRM_OK;
 }
 
@@ -970,7 +1020,8 @@ static int stats_fill(rrm_net* net, int layer, rrm_stats* h)
     RRM_CUDA_TRY(cudaMemcpy(&oc, L.ocount, 4, cudaMemcpyDeviceToHost));
     h->active_macs = (int64_t)m;
     h->active_out_pixels = oc;
-    h->variant = L.tc_ready ? RRM_VARIANT_TENSOR : RRM_VARIANT_GATHER;
+    // (a layer that was evaluated densely inside the delta step keeps its counters: the deltas were still formed and counted)
+    h->variant = L.ran_dense ? RRM_VARIANT_DENSE : (L.tc_ready ? RRM_VARIANT_TENSOR : RRM_VARIANT_GATHER);
     return RRM_OK;
 }
 int rrm_get_stats(rrm_layer* layer, rrm_stats* host_out) { return rrm_net_get_stats(layer, 0, host_out); }

@@ -117,6 +117,11 @@ struct Layer {
     int* ocount = nullptr;            // their number (cleared every step, written by the convolution kernel)
     unsigned long long* macs = nullptr;     // exact active multiply-accumulates (cleared every step)
     int opixels() const { return d.n * oh * ow; }
+    // per-layer choice between the sparse product and a dense evaluation inside a delta step, from the measured
+    // share of projection pixels to update (north of rrm_options.layer_dense_activity: dense)
+    bool dense_mode = false;          // how the layer runs in the next delta step
+    bool ran_dense = false;           // how it ran in the most recent one
+    double activity = -1.0;           // last measured share; < 0: unknown
     // fused FC path (int8 FC reading the external input)
     bool fc_fused = false;
     int8_t* Wt = nullptr;             // [c_in][c_out] transposed weights
@@ -172,10 +177,6 @@ struct rrm_net {
     void* pipe_in[2] = {nullptr, nullptr};
     void* pipe_out[2] = {nullptr, nullptr};
     int pipe_frames = 0, pipe_slot = 0;
-    // the per-frame launch sequences (0: delta step, 1: keyframe, 2: stateless dense pass), each captured
-    // once and replayed (fixed frame / output buffers)
-    cudaGraph_t graph[3] = {nullptr, nullptr, nullptr};
-    cudaGraphExec_t exec[3] = {nullptr, nullptr, nullptr};
     cudaStream_t cap_stream = nullptr;
     void* frame_buf = nullptr;        // the step's input frame, boundary layout
     void* out_buf = nullptr;          // the step's last tensor, boundary layout
@@ -192,8 +193,21 @@ struct rrm_net {
         const void* src = nullptr; size_t bytes = 0;   // copy node: source and size
         void* value = nullptr;                     // storage the patched argument points to
     };
-    std::vector<IoPatch> patch_in[3], patch_out[3];
-    bool patch_ok[3] = {false, false, false};
+    // the per-frame launch sequences (0: delta step, 1: keyframe, 2: stateless dense pass), each captured once and
+    // replayed (fixed frame / output buffers).  A delta step exists in one form per layer mask (bit l: layer l is
+    // evaluated densely inside the step); the few most recently used masks are kept.
+    struct StepGraph {
+        unsigned long long mask = 0, used = 0;
+        cudaGraph_t graph = nullptr;
+        cudaGraphExec_t exec = nullptr;
+        std::vector<IoPatch> patch_in, patch_out;
+        bool patch_ok = false;
+    };
+    std::vector<StepGraph> step_graphs[3];
+    unsigned long long step_clock = 0;
+    unsigned long long layer_mask = 0;            // the mask of the next delta step
+    bool layer_switch = false;                    // every layer asks for RRM_VARIANT_AUTO: the per-layer choice is on
+    uint32_t* ones = nullptr;                     // an all-ones bitmap as long as the longest update bitmap
     // pipelined chunks of frames (rrm_net_step_seq on a stack): T frames captured as ONE graph in which layer l of
     // frame t+1 depends only on layer l-1 of frame t+1, on layer l of frame t (its projection) and on the layers of
     // frame t that read the tensor it overwrites - so consecutive frames overlap layer by layer.  Each frame in
@@ -203,7 +217,7 @@ struct rrm_net {
     std::vector<cudaEvent_t> ev_conv, ev_epi;     // per layer: the most recently captured convolution / epilogue
     std::vector<cudaEvent_t> ev_join;
     cudaEvent_t ev_fork = nullptr, ev_export = nullptr;
-    struct ChunkGraph { int T = 0; cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr; unsigned long long used = 0; };
+    struct ChunkGraph { int T = 0; unsigned long long mask = 0; cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr; unsigned long long used = 0; };
     std::vector<ChunkGraph> chunk_graphs[3];      // per kind (delta / keyframes / dense): the few most recently used chunk lengths
     unsigned long long chunk_clock = 0;
     void* chunk_in = nullptr;
@@ -250,14 +264,15 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
 // ---- rrm_conv_tc.cu
 bool conv_tc_eligible(const rrm_net* net, const Layer& L);
 int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev);
-int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st);
+int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st,
+                   const uint32_t* count_bitmap = nullptr);
 int zero_projection(void* P, long long words, cudaStream_t st);
 
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);
 int launch_import(rrm_net* net, const void* frame_dev, bool delta, bool stateless, cudaStream_t st);
 int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st,
-                 const std::function<int(int)>* hook = nullptr);
+                 const std::function<int(int)>* hook = nullptr, bool dense_in_step = false);
 int launch_export_tensor(rrm_net* net, int t, void* dst_dev, bool stateless, cudaStream_t st);
 int launch_export_projection(rrm_net* net, int l, void* dst_dev, cudaStream_t st);
 int reset_state(rrm_net* net, cudaStream_t st);

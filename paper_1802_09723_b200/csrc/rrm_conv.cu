@@ -41,7 +41,26 @@ struct ConvParams {
     int n, c_in, h, w, u_in, oh, ow, kh, kw, stride, pad, c_out, np, ku, kup, opixels;
     int ksplit;               // gridDim.z: CTAs that share one output tile, each with a contiguous range of K stages
     unsigned wait_limit;      // polls of one bounded wait
+    const uint32_t* count_bitmap;   // dense evaluation inside a delta step: the layer's update bitmap, whose set bits the
+                                    // first CTA counts into *ocount (the measured activity); nullptr otherwise
 };
+
+// The number of set bits of bm[0 .. words) -> *out, by one CTA (the activity of a layer that is evaluated densely).
+__device__ __forceinline__ void count_bits_cta(const uint32_t* __restrict__ bm, int words, int* out, int* s_scratch)
+{
+    int c = 0;
+    for (int i = threadIdx.x; i < words; i += blockDim.x) c += __popc(__ldg(bm + i));
+    #pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if ((threadIdx.x & 31) == 0) s_scratch[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int w = 0; w < (int)((blockDim.x + 31) >> 5); ++w) t += s_scratch[w];
+        *out = t;
+    }
+    __syncthreads();
+}
 
 __device__ __forceinline__ bool bit_test(const uint32_t* bm, int i) { return (bm[i >> 5] >> (i & 31)) & 1u; }
 
@@ -181,6 +200,8 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     const unsigned long long tm0 = (unsigned long long)s_tapmask[0] | (unsigned long long)s_tapmask[1] << 32;
     const unsigned long long tm1 = (unsigned long long)s_tapmask[2] | (unsigned long long)s_tapmask[3] << 32;
     if (DENSE) pdl_wait();                                   // barriers and row tables are set up; the inputs come next
+    if (DENSE && p.count_bitmap && tile == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+        count_bits_cta(p.count_bitmap, (p.opixels + 31) >> 5, p.ocount, s_tmp);
     // this CTA's share of the K stages
     const int all_stages = p.kup / TK, per_split = (all_stages + p.ksplit - 1) / p.ksplit;
     const int s_first = blockIdx.z * per_split, n_stages = min(all_stages, s_first + per_split);
@@ -997,9 +1018,15 @@ static int launch_epi(const EpiParams& e, int ot, int blocks, cudaStream_t st)
 
 // hook (may be null): called with 0 before the layer's first launch, with 1 between the convolution and the
 // epilogue, with 2 after the epilogue (the pipelined chunk graph inserts its cross-frame dependencies there).
-int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st, const std::function<int(int)>* hook)
+// dense_in_step: the layer is evaluated densely inside a delta step (its measured activity is above the
+// threshold): P = F*X + b from the input's current value replaces the stored projection (a precise inference of
+// this layer), and the epilogue still compares f(P) with the stored output and emits the next layer's delta.
+int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st, const std::function<int(int)>* hook,
+                 bool dense_in_step)
 {
     if (hook) RRM_TRY((*hook)(0));
+    const bool step_dense = dense_in_step && !dense && !stateless;
+    const bool conv_dense = dense || step_dense;
     Layer& L = net->layers[l];
     const rrm_layer_desc& d = L.d;
     Tensor& in = net->tensors[d.src];
@@ -1013,6 +1040,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.c_out = d.c_out; p.np = L.np;
     p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
     p.wait_limit = net->opt.wait_limit;
+    p.count_bitmap = step_dense ? L.oact : nullptr;
     dim3 grid(ceil_div(L.opixels(), TM), L.np / TN);
     p.errw = net->errw;
     // split K over CTAs while the tiles alone leave most of the machine idle (each share keeps >= 4 stages)
@@ -1020,20 +1048,20 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
         const int stages = L.kup / TK;
         int ks = 1;
         // (a delta pass is sized as if half of the tiles had rows: the others leave right after the row scan)
-        const long long tiles = dense ? (long long)grid.x * grid.y : (long long)(grid.x + 1) / 2 * grid.y;
+        const long long tiles = conv_dense ? (long long)grid.x * grid.y : (long long)(grid.x + 1) / 2 * grid.y;
         while (tiles * ks < 2 * 148 && stages / (ks * 2) >= 2) ks *= 2;
         p.ksplit = ks;
         grid.z = ks;
-        if (!L.tc_ready && dense && ks > 1) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));
+        if (!L.tc_ready && conv_dense && ks > 1) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));
     }
-    if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, dense, stateless, st));
-    else if (d.dtype == RRM_F32) { if (dense) launch_gemm<T_F32, true>(p, grid, st); else launch_gemm<T_F32, false>(p, grid, st); }
-    else if (d.dtype == RRM_I8) { if (dense) launch_gemm<T_I8, true>(p, grid, st); else launch_gemm<T_I8, false>(p, grid, st); }
-    else { if (dense) launch_gemm<T_BIN, true>(p, grid, st); else launch_gemm<T_BIN, false>(p, grid, st); }
+    if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, conv_dense, stateless, st, p.count_bitmap));
+    else if (d.dtype == RRM_F32) { if (conv_dense) launch_gemm<T_F32, true>(p, grid, st); else launch_gemm<T_F32, false>(p, grid, st); }
+    else if (d.dtype == RRM_I8) { if (conv_dense) launch_gemm<T_I8, true>(p, grid, st); else launch_gemm<T_I8, false>(p, grid, st); }
+    else { if (conv_dense) launch_gemm<T_BIN, true>(p, grid, st); else launch_gemm<T_BIN, false>(p, grid, st); }
 
     if (hook) RRM_TRY((*hook)(1));
     EpiParams e;
-    e.P = p.P; e.oact = L.oact;
+    e.P = p.P; e.oact = step_dense ? net->ones : L.oact;     // (dense inside a delta step: every window is looked at)
     e.resX = res ? (stateless ? res->X2 : res->X) : nullptr;
     e.X = stateless ? out.X2 : out.X; e.D = out.D; e.act = out.act; e.pnnz = out.pnnz; e.nnz = out.nnz;
     e.npix = out.npix; e.errw = out.has_consumer ? net->errw : nullptr;

@@ -48,6 +48,8 @@ struct TcParams {
     int bn;                   // 64 or 128
     int ksplit;               // gridDim.z
     unsigned wait_limit;      // polls of one bounded wait
+    const uint32_t* count_bitmap;   // dense evaluation inside a delta step: the layer's update bitmap, whose set bits the
+                                    // first CTA counts into *ocount (the measured activity); nullptr otherwise
 };
 
 // byte i of the result = bit i of the low nibble of x (0 or 1)
@@ -181,6 +183,16 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
     __syncthreads();
     tc_fence_after();
     if (DENSE) pdl_wait();                                   // barriers, tensor memory and row tables are set up; the inputs come next
+    if (DENSE && p.count_bitmap && tile == 0 && ntile == 0 && split == 0) {
+        // (uniform for the whole CTA) the layer's activity is still measured while it is evaluated densely
+        int c = 0;
+        for (int i = tid; i < ((p.opixels + 31) >> 5); i += TC_THREADS) c += __popc(__ldg(p.count_bitmap + i));
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+        if (lane == 0) s_tmp[warp] = c;
+        __syncthreads();
+        if (tid == 0) { int t = 0; for (int w = 0; w < TC_THREADS / 32; ++w) t += s_tmp[w]; *p.ocount = t; }
+    }
     const uint32_t tmem = S->tmem_base;
     const unsigned long long tm0 = S->tap_mask[0], tm1 = S->tap_mask[1];
 
@@ -571,7 +583,8 @@ int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev)
 }
 
 // F*dI (dense: F*X + b) on the tensor cores; P is updated in place (dense: overwritten).
-int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st)
+int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st,
+                   const uint32_t* count_bitmap)
 {
     const rrm_layer_desc& d = L.d;
     TcParams p;
@@ -590,6 +603,7 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.kpp = L.tc_kpp;
     p.slabs = L.tc_slabs; p.bn = L.tc_bn;
     p.wait_limit = net->opt.wait_limit;
+    p.count_bitmap = count_bitmap;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
     // split K towards the point where a CTA's slabs all fit in its pipeline at once
     // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the

@@ -89,7 +89,7 @@ def _run(specs, video, n=1, check_frames=None, stats=False, keyframe_at=(), vari
             one.step(video[t])
             for l in range(len(specs)):
                 st = net.stats(l)
-                assert st["error_word"] == 0 and st["variant"] != 3, (t, l, st)
+                assert st["error_word"] == 0 and st["nnz_elems"] != -1, (t, l, st)
                 assert st["dense_macs"] == orc.layer_macs(specs[l]) * n
                 if specs[0].dtype != "f32" or l == 0:
                     assert st["nnz_elems"] == one.nnz[l], (t, l, st, one.nnz[l])
@@ -228,17 +228,68 @@ def test_large_stack_goes_dense_while_nearly_every_pixel_changes():
     video = wl.moving_rect_video(frames=20, hw=227, dtype="i8", seed=33, n=2, bg_redraw=0.10)
     net = rrm.net_from_specs(specs, n=2)
     out = net.new_output()
-    variants = []
+    variants, counted = [], []
     for t in range(20):
         net.step(dev(video[t]), out)
         st = net.stats(1)                     # synchronises, so the next call sees this frame's counters
         variants.append(st["variant"])
-        assert (st["nnz_elems"] == -1) == (st["variant"] == 3)
+        counted.append(st["nnz_elems"] != -1)
         if t in (0, 1, 2, 16, 19):
             _compare(specs, net, video[t], t)
-    assert variants[0] == 2                               # the first frame (every pixel new) is a measured delta frame
-    assert all(v == 3 for v in variants[1:16])            # dense while the measured activity is high
-    assert variants[16] == 2 and variants[17] == 3        # one delta frame measures again
+    assert variants[0] == 2 and counted[0]                # the first frame (every pixel new) is a measured delta frame
+    assert all(v == 3 for v in variants[1:16]) and not any(counted[1:16])   # the whole stack dense while the measured activity is high
+    # one delta frame measures again; its layers, all above their own threshold, are evaluated densely inside it and
+    # still count their deltas
+    assert variants[16] == 3 and counted[16]
+    assert variants[17] == 3 and not counted[17]
+    net.close()
+
+
+@pytest.mark.parametrize("name", ["alex_i8", "resnet_i8", "alex_f32", "xnor"])
+def test_layers_choose_between_sparse_and_dense_evaluation_from_their_measured_activity(name):
+    """Per-layer choice (variant AUTO): with the thresholds lowered, the layers whose share of projection pixels to
+    update is high run a dense evaluation inside the delta step while the others run the sparse product.  Outputs,
+    stored projections and counters stay those of Algorithm 1 at every frame, whatever the mix."""
+    rrm = _rrm()
+    if name == "alex_i8":
+        specs, dt, hw, n = wl.alexnet_convs("i8", hw=99, scale=8), "i8", 99, 1
+    elif name == "resnet_i8":
+        specs, dt, hw, n = wl.resnet18_convs(hw=96, scale=8), "i8", 96, 2
+    elif name == "alex_f32":
+        specs, dt, hw, n = wl.alexnet_convs("f32", hw=99, scale=8), "f32", 99, 1
+    else:
+        specs, dt, hw, n = wl.xnor_alexnet_convs(hw=99, scale=8), "i8", 99, 1
+    video = wl.moving_rect_video(frames=9, hw=hw, dtype=dt, seed=23, n=n, side=(12, 24))
+    net = rrm.net_from_specs(specs, n=n)
+    rec = orc.Recurrence(specs, n=n)
+    rec.step(np.full_like(video[0], 0))
+    out = net.new_output()
+    mixes = set()
+    for t in range(video.shape[0]):
+        net.step(dev(video[t]), out)
+        rec.step(video[t])
+        vs, acts = [], []
+        for l in range(len(specs)):
+            st = net.stats(l)                 # synchronises: the next step's choice sees this frame's counters
+            vs.append(st["variant"])
+            acts.append(st["active_out_pixels"] / st["out_pixels"])
+            assert st["error_word"] == 0
+            if dt != "f32" or l == 0:
+                assert st["nnz_elems"] == rec.nnz[l] and st["active_macs"] == rec.macs[l], (t, l, st, rec.nnz[l], rec.macs[l])
+        mixes.add(tuple(v == 3 for v in vs))
+        _compare(specs, net, video[t], t)
+        if t == 2:
+            # thresholds between this video's measured per-layer activities, so that the layers really split
+            a = sorted(set(acts))
+            assert len(a) >= 2, acts
+            thr = 0.5 * (a[len(a) // 2 - 1] + a[len(a) // 2])
+            net.set_options(layer_dense_activity=thr, layer_delta_activity=0.95 * thr)
+    assert any(any(m) and not all(m) for m in mixes), mixes       # some frame ran a real mix of the two evaluations
+    # ... and a chunk of frames with the mix chosen at its start
+    more = wl.moving_rect_video(frames=13, hw=hw, dtype=dt, seed=23, n=n, side=(12, 24))
+    outs = net.new_output(frames=4)
+    net.step_seq(dev(np.ascontiguousarray(more[9:13])), outs, 4)
+    _compare(specs, net, more[12], 12)
     net.close()
 
 
@@ -253,6 +304,27 @@ def test_cfg3_alexnet_int8_full_size():
     specs = wl.alexnet_convs("i8")
     video = wl.moving_rect_video(frames=64, hw=227, dtype="i8", seed=32)
     _run(specs, video, check_frames={0, 1, 30, 63}, stats_frames={30})
+
+
+def test_cfg3_alexnet_int8_early_layers_sparse_late_layers_dense():
+    """On the moving-rectangle video the first layers update a fifth to a half of their projection pixels, the last
+    ones nearly all: with the default thresholds the library settles on the sparse product for conv1-2 and a dense
+    evaluation for conv5, inside the same delta step."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8")
+    video = wl.moving_rect_video(frames=20, hw=227, dtype="i8", seed=32)
+    net = rrm.net_from_specs(specs)
+    out = net.new_output()
+    # (frame 0 changes every pixel, so this stack of > 1 GMAC is evaluated densely as a whole for the next 15 frames;
+    # frame 16 measures again, and from frame 17 on every layer follows its own activity)
+    for t in range(20):
+        net.step(dev(video[t]), out)
+        vs = [net.stats(l)["variant"] for l in range(len(specs))]
+    assert vs[0] == 2 and vs[1] == 2 and vs[4] == 3, vs
+    act = [net.stats(l)["active_out_pixels"] / net.stats(l)["out_pixels"] for l in range(len(specs))]
+    assert act[0] < 0.6 and act[4] > 0.75, act
+    _compare(specs, net, video[19], 19)
+    net.close()
 
 
 def test_cfg4_resnet18_int8_batch4():
