@@ -274,7 +274,7 @@ def conv_workload(name, frames=None, streams=None):
 
 
 def conv_measure(name, variant="auto", steps=60, warmup=5, frames=None, streams=None, seq=None, cpu_frames=0,
-                 sample_clocks=True):
+                 sample_clocks=True, options=None):
     """Times one convolution configuration: delta steps (cold and warm L2), the library's own dense path, per-layer
     densities, Eq. 9 / Eq. 10, the roofline of the step; optionally chunks of `seq` frames and a CPU oracle sample."""
     import torch
@@ -283,6 +283,8 @@ def conv_measure(name, variant="auto", steps=60, warmup=5, frames=None, streams=
     specs, video, n, dtype = conv_workload(name, frames, streams)
     F = video.shape[0]
     net = rrm.net_from_specs(specs, n=n, variant=variant)
+    if options:
+        net.set_options(**options)
     fr = [torch.from_numpy(np.ascontiguousarray(video[t])).cuda() for t in range(F)]
     order = pingpong(F)
     period = len(order)
@@ -436,8 +438,12 @@ def run_conv(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    options = {}
+    for kv in args.opt or []:
+        k, v = kv.split("=")
+        options[k] = int(v) if k in ("wait_limit", "stack_reprobe") else float(v)
     r = conv_measure(args.workload, args.variant, args.steps, args.warmup, args.frames, args.streams, args.seq,
-                     cpu_frames=0 if args.quick else 2)
+                     cpu_frames=0 if args.quick else 2, options=options)
     n = r["streams"]
     line = {
         "metric": "frames_per_sec", "value": r["frames_per_sec"], "unit": "frames/s", "n_gpus": 1, "steps": args.steps,
@@ -488,6 +494,7 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense"])
     ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
     ap.add_argument("--streams", type=int, default=None, help="independent videos per call (convolution workloads)")
+    ap.add_argument("--opt", action="append", help="rrm_options field=value (convolution workloads), e.g. --opt layer_dense_activity=0.9")
     ap.add_argument("--seq", type=int, default=None, help="also time rrm_net_step_seq with this many frames per call (convolution workloads)")
     args = ap.parse_args()
     if args.workload != "cfg2":

@@ -117,8 +117,9 @@ typedef struct {
                                     the thread block leave in an orderly way.  Default 2^20.  0 makes every such wait
                                     give up at once, before the thread block has anything in flight: a test hook */
     float layer_dense_activity;  /* stacks, variant AUTO: a layer whose measured share of projection pixels to update
-                                    reached this value is evaluated densely in the following frames ... */
-    float layer_delta_activity;  /* ... and goes back to the sparse product once the share has fallen below this one */
+                                    reached this value (default 0.97) is evaluated densely in the following frames ... */
+    float layer_delta_activity;  /* ... and goes back to the sparse product once the share has fallen below this one
+                                    (default 0.90) */
     float stack_dense_activity;  /* whole-stack switch (stacks of >= 1 GMAC per frame): MAC-weighted share from which on
                                     every layer of the next frames is evaluated densely */
     int32_t stack_reprobe;       /* dense frames in a row before one delta frame measures the activity again */

@@ -24,11 +24,16 @@ Readings of points the paper leaves open (these bind the CUDA path too):
   - '*' is cross-correlation with zero padding; filters are [C_out][C_in][kh][kw].
   - an element is "non-zero" iff the two frames' values differ (threshold eps = 0).
 Parity unpinned by the paper (not in it; fixed here by definition and hand-checked
-tiny cases): the int8 requantisation rule, the sign threshold, pooling order.
+tiny cases): the int8 requantisation rule, the sign threshold, pooling order, the integer
+form of an explicit batch normalisation.
   - int8: q = clamp((P + 2^(s-1)) >> s, -127, 127) (arithmetic shift), then + shortcut,
     then ReLU (clamp to [0,127]) or clamp to [-127,127], then max-pool.
   - binary: inputs/weights are +-1, padding is 0; sign(v) = +1 iff v >= theta, taken on
     the max-pooled int32 projection.
+  - explicit batch normalisation (the non-linear layer the paper's Discussion names, Sec. 4.5):
+    at inference a per-channel affine applied to the full projection P_t before anything else of
+    f.  fp32: y = scale * P + shift.  int8: integer multiplier and offset inside the
+    requantisation, q = clamp((P * scale + shift + 2^(s-1)) >> s, -127, 127), 64-bit exact.
 """
 import ctypes
 import os
@@ -155,7 +160,11 @@ def requant(P, shift):
 
 def nonlinearity(spec, P, res=None):
     """The map f of Eq. 1 for one layer: I_{t,l+1} = f(P_tl)."""
+    bn = getattr(spec, "bn_scale", None) is not None
     if spec.dtype == "f32":
+        if bn:                                           # explicit batch normalisation: per-channel affine first
+            P = (np.asarray(spec.bn_scale, dtype=np.float64).reshape(1, -1, 1, 1) * P
+                 + np.asarray(spec.bn_shift, dtype=np.float64).reshape(1, -1, 1, 1))
         v = P if res is None else P + res
         if spec.act == "relu":
             v = np.maximum(v, 0.0)
@@ -169,9 +178,14 @@ def nonlinearity(spec, P, res=None):
     if spec.act == "sign":
         v = maxpool(P, *spec.pool) if spec.pool is not None else P
         return np.where(v >= spec.theta, 1, -1).astype(np.int64)
+    assert not bn or (spec.shift >= 0 and spec.act != "sign"), "integer affine is defined inside the requantisation only"
     if spec.shift < 0:
         assert res is None and spec.act == "none"
         return maxpool(P, *spec.pool) if spec.pool is not None else P
+    if bn:                                               # integer multiplier and offset, exact in int64
+        P = (P.astype(np.int64) * np.asarray(spec.bn_scale, dtype=np.int64).reshape(1, -1, 1, 1)
+             + np.asarray(spec.bn_shift, dtype=np.int64).reshape(1, -1, 1, 1))
+        assert np.all(np.abs(P) < 2 ** 62)
     v = requant(P, spec.shift)
     if res is not None:
         v = v + res

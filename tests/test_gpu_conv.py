@@ -308,12 +308,13 @@ def test_cfg3_alexnet_int8_full_size():
 
 def test_cfg3_alexnet_int8_early_layers_sparse_late_layers_dense():
     """On the moving-rectangle video the first layers update a fifth to a half of their projection pixels, the last
-    ones nearly all: with the default thresholds the library settles on the sparse product for conv1-2 and a dense
-    evaluation for conv5, inside the same delta step."""
+    ones nearly all: with the thresholds at 0.75 / 0.60 the library settles on the sparse product for conv1-2 and a
+    dense evaluation for conv5, inside the same delta step."""
     rrm = _rrm()
     specs = wl.alexnet_convs("i8")
     video = wl.moving_rect_video(frames=20, hw=227, dtype="i8", seed=32)
     net = rrm.net_from_specs(specs)
+    net.set_options(layer_dense_activity=0.75, layer_delta_activity=0.60)
     out = net.new_output()
     # (frame 0 changes every pixel, so this stack of > 1 GMAC is evaluated densely as a whole for the next 15 frames;
     # frame 16 measures again, and from frame 17 on every layer follows its own activity)

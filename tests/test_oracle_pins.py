@@ -479,3 +479,63 @@ def test_leaky_relu_matches_the_library_routine():
     want = torch.nn.functional.leaky_relu(torch.from_numpy(P), float(np.float32(0.1))).numpy()
     np.testing.assert_allclose(got, want, atol=1e-15)
     assert (got[P < 0] < 0).all() and (got[P > 0] == P[P > 0]).all()
+
+
+# ------------------------------------------------------------------ explicit batch normalisation as part of f (Sec. 4.5)
+def test_explicit_bn_hand_cases():
+    # fp32: y = scale * P + shift per channel, then ReLU
+    s = LayerSpec("conv", "f32", 1, 1, 2, 2, act="relu", src=0)
+    s.bn_scale = np.array([2.0, -1.0], dtype=np.float32)
+    s.bn_shift = np.array([0.5, 0.25], dtype=np.float32)
+    P = np.array([[[[1.0, -3.0]], [[4.0, -2.0]]]])            # [1, 2 channels, 1, 2]
+    # channel 0: 2*1+0.5 = 2.5, 2*(-3)+0.5 = -5.5 -> 0 ; channel 1: -4+0.25 = -3.75 -> 0, 2+0.25 = 2.25
+    np.testing.assert_allclose(orc.nonlinearity(s, P).ravel(), [2.5, 0.0, 0.0, 2.25], atol=1e-15)
+    # int8: q = clamp((P*m + a + 2^(s-1)) >> s, -127, 127), then + shortcut, then ReLU
+    q = LayerSpec("conv", "i8", 1, 1, 1, 3, act="relu", shift=4, src=0)
+    q.bn_scale = np.array([3, 1, 5], dtype=np.int32)
+    q.bn_shift = np.array([-8, 7, 0], dtype=np.int32)
+    P = np.array([[[[10]], [[-30]], [[1000]]]])
+    # ch0: 30-8+8 = 30 >> 4 = 1 ; ch1: -30+7+8 = -15 >> 4 = -1 (arithmetic shift) ; ch2: 5000+8 >> 4 = 313 -> 127
+    res = np.array([[[[0]], [[3]], [[-100]]]])
+    # + shortcut: 1, 2, 27 ; ReLU keeps them
+    np.testing.assert_array_equal(orc.nonlinearity(q, P, res=res).ravel(), [1, 2, 27])
+    q.act = "none"
+    np.testing.assert_array_equal(orc.nonlinearity(q, P).ravel(), [1, -1, 127])
+
+
+def test_unfolded_bn_equals_the_folded_stack():
+    """An affine after a linear layer folds into it: scale * (F*I + b) + shift = (scale F)*I + (scale b + shift).
+    The oracle's unfolded stack must agree with its own evaluation of the folded one (in fp64; the folded
+    filters are rounded to fp32, hence the tolerance), through ReLU and pooling, at every layer."""
+    specs = wl.with_explicit_bn(wl.alexnet_convs("f32", hw=67, scale=16))
+    folded = wl.fold_bn_f32(specs)
+    assert all(f.bn_scale is None for f in folded) and all(s.bn_scale is not None for s in specs)
+    frame = wl.moving_rect_video(frames=1, hw=67, dtype="f32", seed=5)[0]
+    tu, _ = orc.dense_forward(specs, frame)
+    tf, _ = orc.dense_forward(folded, frame)
+    for a, b in zip(tu[1:], tf[1:]):
+        assert np.abs(a - b).max() <= 1e-5 * max(1.0, np.abs(b).max())
+    # and the affine really acts: without it the tensors differ
+    plain = wl.alexnet_convs("f32", hw=67, scale=16)
+    tp, _ = orc.dense_forward(plain, frame)
+    assert np.abs(tp[1] - tu[1]).max() > 1e-3
+
+
+@pytest.mark.parametrize("net", ["alex_f32", "resnet_i8"])
+def test_recurrence_with_explicit_bn_equals_dense(net):
+    rng = np.random.default_rng(7)
+    layers = wl.with_explicit_bn(wl.alexnet_convs("f32", hw=67, scale=16) if net == "alex_f32" else wl.resnet18_convs(hw=64, scale=8))
+    seq = _seq_for(layers, 4, rng)
+    rec = orc.Recurrence(layers)
+    for frame in seq:
+        tens_r, P_r = rec.step(frame)
+        tens_d, P_d = orc.dense_forward(layers, frame)
+        for l in range(len(layers)):
+            if layers[l].dtype == "f32":
+                assert np.abs(P_r[l] - P_d[l]).max() <= 1e-11 * max(1.0, np.abs(P_d[l]).max())
+            else:
+                np.testing.assert_array_equal(P_r[l], P_d[l])
+                np.testing.assert_array_equal(tens_r[l + 1], tens_d[l + 1])
+    if net == "resnet_i8":       # the integer affine keeps the activations alive
+        t = tens_d[-1]
+        assert 0.05 < float(np.mean(t > 0)) and float(np.mean(np.abs(t) >= 127)) < 0.3

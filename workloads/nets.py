@@ -4,9 +4,12 @@ A network is a list of LayerSpec.  Tensor 0 is the network input; layer l produc
 tensor l+1.  `src` names the tensor a layer reads, `res` (or -1) a tensor that is
 added to the requantised projection before the activation (ResNet shortcut).
 
-Nonlinear map f of a layer, in order: [requant by `shift`] -> [+ res] -> act -> pool,
+Nonlinear map f of a layer, in order: [per-channel affine] -> [requant by `shift`] -> [+ res] -> act -> pool,
 except act == "sign", where pooling comes first and the sign is taken last.
 `shift == -1` on an integer layer means "emit the raw int32 projection".
+The per-channel affine (`bn_scale`, `bn_shift`, both None = absent) is an explicit, unfolded batch
+normalisation at inference: fp32 layers y = scale * P + shift; int8 layers use integer multipliers and
+offsets inside the requantisation, q = clamp((P * scale + shift + 2^(s-1)) >> s, -127, 127).
 """
 from dataclasses import dataclass, field
 import math
@@ -34,6 +37,8 @@ class LayerSpec:
     name: str = ""
     weight: np.ndarray = field(default=None, repr=False)   # [c_out, c_in, kh, kw]
     bias: np.ndarray = field(default=None, repr=False)     # [c_out] f32 or int32
+    bn_scale: np.ndarray = field(default=None, repr=False)  # [c_out] f32 (fp32 layers) or int32 multipliers (int8 layers), or None
+    bn_shift: np.ndarray = field(default=None, repr=False)  # [c_out] f32 or int32 offsets, or None
 
 
 def out_hw(s: LayerSpec):
@@ -248,3 +253,37 @@ def vgg16_convs(dtype="i8", seed=7, hw=224, scale=1):
         _, (h, w) = out_hw(L[-1])
         c_in = c
     return _fill(_resolve_src(L), seed)
+
+
+# ---------------------------------------------------------------- explicit (unfolded) batch normalisation
+def with_explicit_bn(layers, seed=8):
+    """Gives every layer of a stack an explicit per-channel affine after its projection (batch normalisation at
+    inference, not folded into the filters).  fp32 layers: scale in [0.5, 1.5], shift ~ N(0, 0.1).  int8 layers with
+    a requantisation: integer multipliers in [24, 40] with the layer's shift raised by 5 (so the affine is about a
+    factor one) and small integer offsets.  Layers of other kinds are left as they are.  Modifies `layers` in place."""
+    rng = _rng(seed)
+    for s in layers:
+        if s.dtype == "f32":
+            s.bn_scale = (0.5 + rng.random(s.c_out)).astype(np.float32)
+            s.bn_shift = (rng.standard_normal(s.c_out) * 0.1).astype(np.float32)
+        elif s.dtype == "i8" and s.shift >= 0 and s.act != "sign":
+            s.bn_scale = rng.integers(24, 41, size=s.c_out).astype(np.int32)
+            s.shift += 5
+            s.bn_shift = rng.integers(-(1 << (s.shift - 1)), (1 << (s.shift - 1)) + 1, size=s.c_out).astype(np.int32)
+    return layers
+
+
+def fold_bn_f32(layers):
+    """The same fp32 stack with every explicit affine folded into filters and bias (F' = scale * F,
+    b' = scale * b + shift, in fp64 rounded to fp32): what a deployment that folds batch normalisation runs."""
+    import copy
+    out = []
+    for s in layers:
+        t = copy.copy(s)
+        if s.dtype == "f32" and s.bn_scale is not None:
+            sc = s.bn_scale.astype(np.float64)
+            t.weight = (s.weight.astype(np.float64) * sc.reshape(-1, 1, 1, 1)).astype(np.float32)
+            t.bias = (s.bias.astype(np.float64) * sc + s.bn_shift.astype(np.float64)).astype(np.float32)
+            t.bn_scale = t.bn_shift = None
+        out.append(t)
+    return out
