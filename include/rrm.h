@@ -67,10 +67,15 @@ enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2,
  * still emitted), and returns to the sparse product below rrm_options.layer_delta_activity.  For a lone int8 FC
  * layer AUTO also means: dense evaluation of a chunk when the previous chunk's measured delta density was high.
  * GATHER forces the CUDA-core / column-gather kernels; TENSOR is AUTO without any density switch; DENSE on a lone
- * FC layer selects the generic (non-fused) path.
+ * FC layer selects the generic (non-fused) path; SPARSE_W: see the enumerator.
  * As a report in rrm_stats.variant: what the most recent step ran for this layer (GATHER, TENSOR, or DENSE for a
  * layer or chunk that was evaluated densely). */
-enum { RRM_VARIANT_AUTO = 0, RRM_VARIANT_GATHER = 1, RRM_VARIANT_TENSOR = 2, RRM_VARIANT_DENSE = 3 };
+enum { RRM_VARIANT_AUTO = 0, RRM_VARIANT_GATHER = 1, RRM_VARIANT_TENSOR = 2, RRM_VARIANT_DENSE = 3,
+       RRM_VARIANT_SPARSE_W = 4 /* lone int8 FC layer: weight-sparse x delta-sparse product (Sec. 3.5 / 4.3: the
+                                   compressed models EIE runs).  The zero weights of W (a pruned model) are dropped
+                                   at create time: every (input, 512-output slice) keeps a 128-bit map of its
+                                   non-zero groups of four outputs and only those groups' bytes, so a non-zero
+                                   delta entry gathers a fraction of its column.  Results are the same integers */ };
 
 /*
  * One linear layer and the nonlinear map f that follows it (Eq. 1).
@@ -239,6 +244,17 @@ int rrm_net_get_stats(rrm_net* net, int layer, rrm_stats* host_out);
 int rrm_net_clear_errors(rrm_net* net);
 int rrm_net_get_options(const rrm_net* net, rrm_options* out);
 int rrm_net_set_options(rrm_net* net, const rrm_options* in);
+
+/* ---- explicit batch normalisation as part of f (the non-linear layer the paper's Discussion names, Sec. 4.5) ----
+ * At inference batch normalisation is a per-channel affine on the full projection P_t; it can be folded into
+ * the filters, or kept explicit: then f of `layer` becomes [affine] -> [requant] -> [+ residual] -> act -> pool.
+ *   RRM_F32 layers: float scale[c_out], shift[c_out]:        y = scale * P + shift
+ *   RRM_I8 layers with shift >= 0: int32 m[c_out], a[c_out]: q = clamp((P*m + a + 2^(shift-1)) >> shift, -127, 127),
+ *                                                            evaluated in 64 bits
+ * Other layers: RRM_ERR_UNSUPPORTED.  Both device arrays are copied.  NULL, NULL removes the affine.  Because f
+ * changes, the call puts the stack back into its fresh state (as after rrm_net_create); it synchronises the
+ * device and discards the captured launch sequences: call it right after creating the stack. */
+int rrm_net_set_affine(rrm_net* net, int layer, const void* scale_dev, const void* shift_dev);
 
 /* ---- approximate mode: sparsity enhancement and accumulated error control (Sec. 3.4) -----------
  * With eps > 0 every delta entry with |d| < eps is truncated to zero before the sparse product (fp32 stacks

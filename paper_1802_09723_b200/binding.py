@@ -11,7 +11,7 @@ from . import build as _build
 KIND = {"conv": 0, "fc": 1}
 DTYPE = {"f32": 0, "i8": 1, "bin": 2}
 ACT = {"none": 0, "relu": 1, "sign": 2, "leaky": 3}
-VARIANT = {"auto": 0, "gather": 1, "tensor": 2, "dense": 3}
+VARIANT = {"auto": 0, "gather": 1, "tensor": 2, "dense": 3, "sparse_w": 4}
 
 
 class RRMError(RuntimeError):
@@ -87,6 +87,7 @@ def lib():
         "rrm_net_get_stats": [_P, ctypes.c_int, ctypes.POINTER(Stats)],
         "rrm_net_projection": [_P, ctypes.c_int, _P, _P],
         "rrm_net_tensor": [_P, ctypes.c_int, _P, _P],
+        "rrm_net_set_affine": [_P, ctypes.c_int, _P, _P],
         "rrm_clear_errors": [_P],
         "rrm_net_clear_errors": [_P],
         "rrm_get_options": [_P, ctypes.POINTER(Options)],
@@ -213,6 +214,10 @@ class Net:
     def set_epsilon(self, eps):
         _check(lib().rrm_net_set_epsilon(self._h, float(eps)), "rrm_net_set_epsilon")
 
+    def set_affine(self, layer, scale, shift):
+        """rrm_net_set_affine: explicit per-channel affine (unfolded batch normalisation) as the first step of f."""
+        _check(lib().rrm_net_set_affine(self._h, layer, _ptr(scale), _ptr(shift)), "rrm_net_set_affine")
+
     def truncation(self):
         """(e_t of Eq. 7 since the last keyframe, [per-layer l2 of the last frame])."""
         e = ctypes.c_double()
@@ -326,7 +331,12 @@ def net_from_specs(specs, n=1, variant="auto", device="cuda"):
     Ws = [torch.from_numpy(np.ascontiguousarray(s.weight)).to(device) for s in specs]
     Bs = [torch.from_numpy(np.ascontiguousarray(s.bias)).to(device) for s in specs]
     torch.cuda.synchronize()
-    return Net(descs, Ws, Bs)
+    net = Net(descs, Ws, Bs)
+    for l, s in enumerate(specs):
+        if getattr(s, "bn_scale", None) is not None:
+            net.set_affine(l, torch.from_numpy(np.ascontiguousarray(s.bn_scale)).to(device),
+                           torch.from_numpy(np.ascontiguousarray(s.bn_shift)).to(device))
+    return net
 
 
 def layer_from_spec(spec, n=1, variant="auto", device="cuda"):

@@ -36,7 +36,8 @@ int validate_desc(const rrm_layer_desc& d, int l, int n_layers)
     if (d.res > l) return RRM_ERR_INVALID_ARG;
     if (d.res >= 0 && (d.pool_k > 0 || d.act == RRM_ACT_SIGN)) return RRM_ERR_UNSUPPORTED;
     if (d.res >= 0 && d.dtype != RRM_F32 && d.shift < 0) return RRM_ERR_UNSUPPORTED;
-    if (d.variant < RRM_VARIANT_AUTO || d.variant > RRM_VARIANT_DENSE) return RRM_ERR_INVALID_ARG;
+    if (d.variant < RRM_VARIANT_AUTO || d.variant > RRM_VARIANT_SPARSE_W) return RRM_ERR_INVALID_ARG;
+    if (d.variant == RRM_VARIANT_SPARSE_W && (n_layers != 1 || d.kind != RRM_FC || d.dtype != RRM_I8)) return RRM_ERR_UNSUPPORTED;
     (void)n_layers;
     return RRM_OK;
 }
@@ -164,6 +165,7 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
     }
     RRM_TRY(dev_alloc(net, (void**)&net->errw, 16));
     if (fused) return RRM_OK;
+    if (descs[0].variant == RRM_VARIANT_SPARSE_W) return RRM_ERR_UNSUPPORTED;   // (shapes the fused FC path does not take)
     // the import kernel turns 32 pixels x all channels of the frame around in shared memory
     if (net->tensors[0].dtype != T_BIN && net->tensors[0].cs != 4 &&
         (size_t)32 * (net->tensors[0].cs + 1) * net->tensors[0].unit_bytes > 200 * 1024) return RRM_ERR_UNSUPPORTED;
@@ -395,7 +397,11 @@ int run(rrm_net* net, const void* frame, void* out, cudaStream_t st, bool dense,
 {
     if (!net || !frame) return RRM_ERR_INVALID_ARG;
     net->last_stream = st;
-    if (net->layers[0].fc_fused) return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
+    if (net->layers[0].fc_fused) {
+        // (the weight-sparse form lives in the chunk kernel: a single frame is a chunk of one)
+        if (net->layers[0].Wsp) return fc_seq_run(net, net->layers[0], frame, out, 1, dense, stateless, st);
+        return fc_fused_run(net, net->layers[0], frame, out, dense, stateless, st);
+    }
     if (net->bound_arena != reinterpret_cast<char*>(net->cleared)) {    // a pipelined chunk left another arena bound
         bind_arena(net, reinterpret_cast<char*>(net->cleared));
         RRM_TRY(bind_readers(net));
@@ -667,7 +673,7 @@ int run_seq(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t st
     if (!net || !frames || T < 1) return RRM_ERR_INVALID_ARG;
     Layer& L0 = net->layers[0];
     // (a chunk too small to fill the machine goes frame by frame through the split-list kernel instead)
-    if (L0.fc_fused && fc_seq_supported(L0) && T * net->n >= 4) {
+    if (L0.fc_fused && fc_seq_supported(L0) && (T * net->n >= 4 || L0.Wsp)) {
         net->last_stream = st;
         return fc_seq_run(net, L0, frames, outs, T, dense, stateless, st);
     }
@@ -934,6 +940,33 @@ int rrm_net_set_epsilon(rrm_net* net, float eps)
     net->eps = eps;
     // the threshold is a kernel argument: captured sequences have to be captured again
     drop_graphs(net);
+    return RRM_OK;
+}
+
+int rrm_net_set_affine(rrm_net* net, int layer, const void* scale_dev, const void* shift_dev)
+{
+    if (!net || layer < 0 || layer >= (int)net->layers.size() || (!scale_dev) != (!shift_dev)) return RRM_ERR_INVALID_ARG;
+    Layer& L = net->layers[layer];
+    if (L.fc_fused) return RRM_ERR_UNSUPPORTED;
+    // the integer form lives inside the requantisation: layers that emit raw projections or signs have none
+    if (L.d.dtype != RRM_F32 && (L.d.shift < 0 || L.d.act == RRM_ACT_SIGN)) return RRM_ERR_UNSUPPORTED;
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
+    const size_t bytes = (size_t)L.d.c_out * 4;
+    if (scale_dev) {
+        if (!L.bn_scale) { RRM_TRY(dev_alloc(net, &L.bn_scale, bytes)); RRM_TRY(dev_alloc(net, &L.bn_shift, bytes)); }
+        RRM_CUDA_TRY(cudaMemcpy(L.bn_scale, scale_dev, bytes, cudaMemcpyDeviceToDevice));
+        RRM_CUDA_TRY(cudaMemcpy(L.bn_shift, shift_dev, bytes, cudaMemcpyDeviceToDevice));
+    } else {
+        dev_release(net, &L.bn_scale);
+        dev_release(net, &L.bn_shift);
+    }
+    drop_graphs(net);                                        // captured sequences hold the old arguments
+    if (net->bound_arena != reinterpret_cast<char*>(net->cleared)) {
+        bind_arena(net, reinterpret_cast<char*>(net->cleared));
+        RRM_TRY(bind_readers(net));
+    }
+    RRM_TRY(reset_state(net, nullptr));                      // f changed: back to the fresh state, consistent with the new f
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
     return RRM_OK;
 }
 

@@ -110,6 +110,8 @@ struct Layer {
     int np = 0;                       // c_out padded to GEMM_TN
     void* Wk = nullptr;               // packed filters [kup][np] units
     void* bias = nullptr;             // float or int32 [c_out]
+    void* bn_scale = nullptr;         // explicit per-channel affine applied to P before the rest of f (batch
+    void* bn_shift = nullptr;         // normalisation at inference): float, or int32 multiplier / offset; nullptr: none
     void* P = nullptr;                // projection [n*oh*ow][c_out] float or int32
     void* P2 = nullptr;               // projection buffer of the stateless dense path
     uint32_t* oact = nullptr;         // bitmap of projection pixels to update (cleared every step, set by the
@@ -129,6 +131,11 @@ struct Layer {
     int xs_cur = 0;
     void* fc_scratch = nullptr;             // per-stream non-zero lists of the two-kernel form
     unsigned long long* fc_nnz = nullptr;   // [0] nnz elements, [1] active groups of 32 (cleared by the kernel's last CTA)
+    // weight-sparse form (RRM_VARIANT_SPARSE_W): per (input, 512-output slice) a record of sp_stride words:
+    // 4 words = map of the non-zero groups of four outputs, then those groups' weights, packed
+    uint32_t* Wsp = nullptr;
+    int sp_stride = 0;
+    long long sp_words = 0;                 // packed weight words of the whole matrix (for reporting)
     // tensor-core variant (int8 / binary layers whose input rows are whole 32-byte K chunks)
     bool tc_ready = false;
     int8_t* tc_Wimg = nullptr;              // [n_tiles][slabs][bn * 128] shared-memory images of the filter tiles
@@ -252,6 +259,7 @@ int fc_fused_projection(rrm_net* net, Layer& L, void* P_dev, cudaStream_t st);
 
 // ---- rrm_fc_seq.cu
 int fc_seq_create(rrm_net* net, Layer& L);
+int fc_sparse_w_create(rrm_net* net, Layer& L);
 bool fc_seq_supported(const Layer& L);
 int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool dense, bool stateless,
                cudaStream_t st);

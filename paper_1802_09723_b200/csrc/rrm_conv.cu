@@ -653,6 +653,8 @@ struct EpiParams {
     Readers readers;          // layers that read the output tensor
     float eps;                // fp32: delta entries below it are truncated to zero (Sec. 3.4)
     double* trunc;            // fp32: receives the sum of squares of the truncated entries
+    const void* bn_scale;     // explicit batch normalisation, the first step of f: per-channel float scale / shift
+    const void* bn_shift;     // (fp32) or int32 multiplier / offset inside the requantisation (int8); nullptr: none
 };
 
 // PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.  KW: pool window edge (1 = no pool).
@@ -717,12 +719,17 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                     for (int j = 0; j < 4; ++j) if (c + j < p.c_out) v[wi][j] = P[o + j];
                 }
             }
-            // ---- f: [requant] -> [+ shortcut] -> act -> max over the window (sign: max first, threshold last)
+            // ---- f: [affine] -> [requant] -> [+ shortcut] -> act -> max over the window (sign: max first, threshold last)
             pt best[4];
             #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const bool live = c + j < p.c_out;
                 pt res = 0;
+                pt bn_m = 1, bn_a = 0;                       // the channel's affine (Sec. 4.5: BN as part of f)
+                if (live && p.bn_scale) {
+                    bn_m = reinterpret_cast<const pt*>(p.bn_scale)[c + j];
+                    bn_a = reinterpret_cast<const pt*>(p.bn_shift)[c + j];
+                }
                 if (live && p.resX) {
                     if (PT == T_F32) res = (pt)reinterpret_cast<const float*>(p.resX)[(size_t)r * p.cs + c + j];
                     else if (OT == T_I8) res = (pt)reinterpret_cast<const int8_t*>(p.resX)[(size_t)r * p.cs + c + j];
@@ -734,13 +741,20 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                     if (!(inside >> wi & 1u)) continue;
                     pt x = v[wi][j];
                     if (PT == T_F32) {
+                        if (p.bn_scale) x = (pt)fmaf((float)x, (float)bn_m, (float)bn_a);
                         x += res;
                         if (p.act_fn == RRM_ACT_RELU) x = x > 0 ? x : 0;
                         else if (p.act_fn == RRM_ACT_LEAKY) x = x > 0 ? x : (pt)(0.1f * (float)x);
                     } else if (OT == T_I8) {
                         int iv = (int)x;
-                        if (p.shift > 0) iv = (iv + (1 << (p.shift - 1))) >> p.shift;
-                        iv = max(-127, min(127, iv));
+                        if (p.bn_scale) {                    // integer multiplier and offset inside the requantisation, 64-bit exact
+                            long long t = (long long)iv * (long long)(int)bn_m + (long long)(int)bn_a;
+                            if (p.shift > 0) t = (t + (1ll << (p.shift - 1))) >> p.shift;
+                            iv = (int)max(-127ll, min(127ll, t));
+                        } else {
+                            if (p.shift > 0) iv = (iv + (1 << (p.shift - 1))) >> p.shift;
+                            iv = max(-127, min(127, iv));
+                        }
                         iv += (int)res;
                         iv = (p.act_fn == RRM_ACT_RELU) ? max(0, min(127, iv)) : max(-127, min(127, iv));
                         x = (pt)iv;
@@ -1069,6 +1083,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     e.pool_k = d.pool_k; e.pool_s = d.pool_s; e.pool_p = d.pool_p; e.act_fn = d.act; e.shift = d.shift; e.theta = d.theta;
     e.readers = dense ? Readers{} : out.readers;
     e.eps = net->eps; e.trunc = out.trunc;
+    e.bn_scale = L.bn_scale; e.bn_shift = L.bn_shift;
     const int blocks = ceil_div(out.pixels(), 8);
     int es;
     if (proj_type(L) == T_F32) es = dense ? launch_epi<T_F32, true>(e, out.dtype, blocks, st) : launch_epi<T_F32, false>(e, out.dtype, blocks, st);

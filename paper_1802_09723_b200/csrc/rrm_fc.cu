@@ -489,6 +489,7 @@ int fc_fused_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_
     L.xs_cur = 0;
     L.fc_fused = true;
     RRM_TRY(fc_seq_create(net, L));
+    if (L.d.variant == RRM_VARIANT_SPARSE_W) return fc_sparse_w_create(net, L);
     // the dense path (keyframe, rrm_dense) runs on the tensor cores when the inputs are whole 32-byte K chunks
     if (C % 32 == 0 && L.d.variant != RRM_VARIANT_GATHER) {
         RRM_TRY(conv_tc_create(net, L, W_dev));

@@ -19,6 +19,7 @@
 //      writes Y_0 .. Y_{T-1}.
 // Cost: the weight columns of the non-zero entries (HBM; frames of a chunk share columns through L2).
 #include "rrm_common.cuh"
+#include <cstring>
 
 namespace rrm {
 
@@ -40,6 +41,8 @@ struct FcSeqParams {
     unsigned* counters;      // [n][slices], zero on entry, zero again on exit
     unsigned* stat;          // [T*n][2]: non-zero entries / active groups of 32 inputs per frame, or nullptr
     int T, n, c_in, c_out, shift, act;
+    const uint32_t* Wsp;     // weight-sparse form: [c_in][slices] records of sp_stride words (map, then packed groups)
+    int sp_stride;
 };
 
 __device__ __forceinline__ int seq_apply_f(int v, int shift, int act)
@@ -85,9 +88,15 @@ __device__ __forceinline__ void fma16(int (&acc)[16], const uint4& w, int d)
 // redundant scans.  The host picks LANES from the size of the chunk.
 // DEEP: 16 instead of 8 loads in flight per lane at 2 instead of 3 CTAs per SM; pays when the whole
 // grid is resident at once (each CTA's chain of round trips is what the launch waits for).
-template <int LANES, bool DEEP>
+// SW (LANES = 32 only): the weights are in the weight-sparse form (Sec. 3.5: EIE keeps the pruned weights of a
+// compressed model in compressed columns).  A lane owns 16 outputs = 4 groups of four; the record of (input j, this
+// slice) starts with a 128-bit map (bit 4 * lane + g: group g of that lane holds a non-zero weight) followed by the
+// 4-byte words of the non-zero groups, in map order.  All lanes load the map (one 16-byte broadcast), find their
+// word offset by counting the map bits below their own, and load only their non-zero groups.
+template <int LANES, bool DEEP, bool SW>
 __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqParams p)
 {
+    static_assert(!SW || LANES == 32, "the weight-sparse records are laid out for 512-output slices");
     constexpr int OW = 16 * LANES;                 // outputs per CTA
     constexpr int CPW = 32 / LANES;                // columns per warp-wide load
     constexpr int CPR = CPW * SQ_WARPS;            // columns per CTA-wide round
@@ -124,9 +133,10 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
     // while the frame is on its way: touch one line in every 2 MiB of the weights, so that the
     // address translations the gather will need are fetched now instead of on its first loads
     {
-        const size_t wbytes = (size_t)C * K;
+        const size_t wbytes = SW ? (size_t)C * slices * p.sp_stride * 4 : (size_t)C * K;
         const size_t off = (size_t)tid << 21;
-        if (off < wbytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.Wt + off));
+        const char* wptr = SW ? reinterpret_cast<const char*>(p.Wsp) : reinterpret_cast<const char*>(p.Wt);
+        if (off < wbytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(wptr + off));
         // likewise the stored projection (or the bias), which only the closing sum reads
         const int32_t* pp = p.bias ? p.bias + slice * OW : p.P + (size_t)s * K + slice * OW;
         if (t == 0 && tid * 32 < width) asm volatile("prefetch.global.L2 [%0];" ::"l"(pp + tid * 32));
@@ -196,7 +206,60 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
     int acc[16];
     #pragma unroll
     for (int i = 0; i < 16; ++i) acc[i] = 0;
-    if (o0 < K) {                                            // K is a multiple of 16
+    if (SW) {
+        constexpr int SW_U = DEEP ? 8 : 4;                   // entries in flight per warp (one column slice per warp-wide step)
+        const int nib_shift = 4 * (lane & 7), nib_word = lane >> 3;
+        for (int e = warp; e < total; e += SW_U * SQ_WARPS) {
+            uint32_t ent[SW_U];
+            uint4 map[SW_U];
+            #pragma unroll
+            for (int u = 0; u < SW_U; ++u) {
+                const int eu = e + u * SQ_WARPS;
+                ent[u] = eu < total ? s_list[eu] : 0xffffffffu;
+            }
+            #pragma unroll
+            for (int u = 0; u < SW_U; ++u)
+                map[u] = ent[u] != 0xffffffffu
+                             ? __ldg(reinterpret_cast<const uint4*>(p.Wsp + ((size_t)(ent[u] & 0xffffu) * slices + slice) * p.sp_stride))
+                             : make_uint4(0, 0, 0, 0);
+            uint32_t wv[SW_U][4];
+            unsigned nib[SW_U];
+            #pragma unroll
+            for (int u = 0; u < SW_U; ++u) {
+                const uint32_t m0 = map[u].x, m1 = map[u].y, m2 = map[u].z, m3 = map[u].w;
+                const uint32_t mine = nib_word == 0 ? m0 : (nib_word == 1 ? m1 : (nib_word == 2 ? m2 : m3));
+                nib[u] = (mine >> nib_shift) & 0xfu;
+                // words of the lanes before this one
+                int before = __popc(mine & ((1u << nib_shift) - 1u));
+                if (nib_word > 0) before += __popc(m0);
+                if (nib_word > 1) before += __popc(m1);
+                if (nib_word > 2) before += __popc(m2);
+                const uint32_t* words = p.Wsp + ((size_t)(ent[u] & 0xffffu) * slices + slice) * p.sp_stride + 4 + before;
+                #pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    wv[u][g] = 0;
+                    if (nib[u] >> g & 1u) wv[u][g] = __ldg(words + __popc(nib[u] & ((1u << g) - 1u)));
+                }
+            }
+            #pragma unroll
+            for (int u = 0; u < SW_U; ++u) {
+                if (nib[u] == 0) continue;
+                const int d = (int)(ent[u] >> 16) - 256;
+                const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
+                const int dl = d - dh;
+                const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
+                #pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    if (!(nib[u] >> g & 1u)) continue;
+                    #pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        acc[g * 4 + b] = __dp4a((int)wv[u][g], (int)(lb << (8 * b)), acc[g * 4 + b]);
+                        if (dh != 0) acc[g * 4 + b] = __dp4a((int)wv[u][g], (int)(hb << (8 * b)), acc[g * 4 + b]);
+                    }
+                }
+            }
+        }
+    } else if (o0 < K) {                                     // K is a multiple of 16
         const int8_t* wbase = p.Wt + o0;
         for (int e = grp; e < total; e += SQ_U * CPR) {
             uint32_t ent[SQ_U];
@@ -399,14 +462,18 @@ int fc_seq_create(rrm_net* net, Layer& L)
     net->allocs.push_back(c);
     RRM_CUDA_TRY(cudaMemset(c, 0, (size_t)n * slices * 4));
     L.seq_counters = reinterpret_cast<unsigned*>(c);
-    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
-    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
-    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<16, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)seq_dyn_smem(SQ_MAX_C_IN, 16)));
-    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<8, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)seq_dyn_smem(SQ_MAX_C_IN, 8)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
+    RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
     return seq_ensure(net, L, 1);
 }
 
@@ -428,6 +495,7 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
     p.Y = Y_dev;
     p.counters = L.seq_counters;
     p.T = T; p.n = n; p.c_in = C; p.c_out = K; p.shift = L.d.shift; p.act = L.d.act;
+    p.Wsp = L.Wsp; p.sp_stride = L.sp_stride;
     if (dense) {
         p.xprev = nullptr;
         p.bias = reinterpret_cast<const int32_t*>(L.bias);
@@ -451,7 +519,7 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
                                (fc_tc_usable(L, T * n) ? L.seq_density * T * n >= (double)net->opt.fc_dense_rows * fc_tc_launches(T * n)
                                                        : L.seq_density >= (double)net->opt.fc_dense_density);
         L.seq_last_T = T;
-        L.seq_last_variant = use_dense ? RRM_VARIANT_DENSE : RRM_VARIANT_GATHER;
+        L.seq_last_variant = use_dense ? RRM_VARIANT_DENSE : (L.Wsp ? RRM_VARIANT_SPARSE_W : RRM_VARIANT_GATHER);
         if (use_dense) {
             // the results are the same integers: P_t = b + W X_t for every frame, state := last frame
             if (fc_tc_usable(L, T * n)) {
@@ -472,7 +540,7 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
     }
     // slice width: the widest (fewest redundant scans, one wave of CTAs with a short chain of dependent
     // round trips each), narrowed while the grid would leave a good part of the machine idle
-    int lanes = L.seq_lanes;
+    int lanes = L.Wsp ? 32 : L.seq_lanes;
     if (lanes == 0) {
         lanes = 32;
         while (lanes > 8 && (long long)ceil_div(K, 16 * lanes) * T * n < 200) lanes /= 2;
@@ -493,10 +561,12 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
         p.T = piece;
         dim3 grid(ceil_div(K, 16 * lanes), piece * n);
         const size_t dyn = seq_dyn_smem(C, lanes);
-        if (lanes == 32 && grid.x * grid.y <= 2 * 148) fc_seq_kernel<32, true><<<grid, SQ_THREADS, dyn, st>>>(p);
-        else if (lanes == 32) fc_seq_kernel<32, false><<<grid, SQ_THREADS, dyn, st>>>(p);
-        else if (lanes == 16) fc_seq_kernel<16, false><<<grid, SQ_THREADS, dyn, st>>>(p);
-        else fc_seq_kernel<8, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+        if (L.Wsp && grid.x * grid.y <= 2 * 148) fc_seq_kernel<32, true, true><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else if (L.Wsp) fc_seq_kernel<32, false, true><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else if (lanes == 32 && grid.x * grid.y <= 2 * 148) fc_seq_kernel<32, true, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else if (lanes == 32) fc_seq_kernel<32, false, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else if (lanes == 16) fc_seq_kernel<16, false, false><<<grid, SQ_THREADS, dyn, st>>>(p);
+        else fc_seq_kernel<8, false, false><<<grid, SQ_THREADS, dyn, st>>>(p);
     }
     RRM_CUDA_TRY(cudaGetLastError());
     if (!dense) RRM_TRY(seq_read_back(L, T * n, st));
@@ -545,6 +615,78 @@ int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int 
                                      cudaMemcpyDeviceToDevice, st));
         L.xs_cur ^= 1;
     }
+    return RRM_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Weight-sparse form: packs Wt[c_in][c_out] into records per (input, 512-output slice).  One warp per record; lane L
+// owns outputs 16 L .. 16 L + 15 of the slice = 4 groups of four.  WRITE = false only finds the longest record.
+// ------------------------------------------------------------------------------------------------
+template <bool WRITE>
+__global__ void __launch_bounds__(256) fc_sparse_w_pack_kernel(const int8_t* __restrict__ Wt, uint32_t* rec, int C, int K, int slices,
+                                                               int stride, int* max_words, unsigned long long* total_words)
+{
+    const int lane = threadIdx.x & 31;
+    const long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= (long long)C * slices) return;                  // uniform inside the warp
+    const int j = (int)(r / slices), slice = (int)(r - (long long)j * slices);
+    const int o = slice * 512 + lane * 16;
+    uint4 w = make_uint4(0, 0, 0, 0);
+    if (o < K) w = *reinterpret_cast<const uint4*>(Wt + (size_t)j * K + o);      // K is a multiple of 16
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    unsigned nib = 0;
+    #pragma unroll
+    for (int g = 0; g < 4; ++g) if (ww[g]) nib |= 1u << g;
+    const int cnt = __popc(nib);
+    int incl = cnt;
+    #pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (!WRITE) {
+        if (lane == 0) { atomicMax(max_words, total); atomicAdd(total_words, (unsigned long long)total); }
+        return;
+    }
+    uint32_t* out = rec + (size_t)r * stride;
+    unsigned m = nib << (4 * (lane & 7));                    // the 8 lanes of a map word OR their nibbles together
+    m |= __shfl_xor_sync(0xffffffffu, m, 1);
+    m |= __shfl_xor_sync(0xffffffffu, m, 2);
+    m |= __shfl_xor_sync(0xffffffffu, m, 4);
+    if ((lane & 7) == 0) out[lane >> 3] = m;
+    int at = 4 + incl - cnt;
+    #pragma unroll
+    for (int g = 0; g < 4; ++g) if (nib >> g & 1u) out[at++] = ww[g];
+}
+
+int fc_sparse_w_create(rrm_net* net, Layer& L)
+{
+    const int C = L.d.c_in, K = L.d.c_out;
+    const int slices = ceil_div(K, 512);
+    const long long records = (long long)C * slices;
+    int* d_max = nullptr;
+    if (cudaMalloc(&d_max, 16) != cudaSuccess) { cudaGetLastError(); return RRM_ERR_ALLOC; }
+    RRM_CUDA_TRY(cudaMemset(d_max, 0, 16));
+    const unsigned blocks = (unsigned)((records + 7) / 8);
+    fc_sparse_w_pack_kernel<false><<<blocks, 256>>>(L.Wt, nullptr, C, K, slices, 0, d_max, reinterpret_cast<unsigned long long*>(d_max + 2));
+    int h[4] = {0, 0, 0, 0};
+    const cudaError_t e = cudaMemcpy(h, d_max, 16, cudaMemcpyDeviceToHost);
+    cudaFree(d_max);
+    if (e != cudaSuccess) { cudaGetLastError(); return RRM_ERR_CUDA; }
+    L.sp_stride = 4 + round_up(h[0] > 0 ? h[0] : 1, 4);      // 16-byte aligned records
+    std::memcpy(&L.sp_words, &h[2], 8);
+    void* rec = nullptr;
+    if (cudaMalloc(&rec, (size_t)records * L.sp_stride * 4) != cudaSuccess) { cudaGetLastError(); return RRM_ERR_ALLOC; }
+    net->allocs.push_back(rec);
+    RRM_CUDA_TRY(cudaMemset(rec, 0, (size_t)records * L.sp_stride * 4));
+    fc_sparse_w_pack_kernel<true><<<blocks, 256>>>(L.Wt, reinterpret_cast<uint32_t*>(rec), C, K, slices, L.sp_stride, nullptr, nullptr);
+    RRM_CUDA_TRY(cudaGetLastError());
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
+    L.Wsp = reinterpret_cast<uint32_t*>(rec);
+    if (getenv("RRM_DEBUG"))
+        fprintf(stderr, "rrm: weight-sparse FC: %lld records of %d words, %lld packed weight words (%.1f %% of the dense bytes incl. maps)\n",
+                records, L.sp_stride, L.sp_words, 100.0 * (L.sp_words * 4.0 + records * 16.0) / ((double)C * K));
     return RRM_OK;
 }
 

@@ -483,3 +483,56 @@ def test_stack_chunk_longer_than_the_arenas_held():
     net.step(dev(video[70]), out)
     _compare(specs, net, video[70], 70)
     net.close()
+
+
+# ------------------------------------------------------------------ explicit batch normalisation as part of f (Sec. 4.5)
+@pytest.mark.parametrize("name", ["alex_f32", "resnet_i8", "vgg_i8"])
+def test_explicit_bn_stacks_every_frame(name):
+    """Stacks whose layers keep their batch normalisation explicit (per-channel affine before requantisation /
+    activation / pooling): projections, tensors and counters against the oracle at every frame, a keyframe in between."""
+    if name == "alex_f32":
+        specs, dt, hw, n = wl.alexnet_convs("f32", hw=99, scale=8), "f32", 99, 1
+    elif name == "resnet_i8":
+        specs, dt, hw, n = wl.resnet18_convs(hw=96, scale=8), "i8", 96, 2
+    else:
+        specs, dt, hw, n = wl.vgg16_convs("i8", hw=64, scale=8), "i8", 64, 1
+    wl.with_explicit_bn(specs)
+    assert all(s.bn_scale is not None for s in specs)
+    video = wl.moving_rect_video(frames=6, hw=hw, dtype=dt, seed=29, n=n, side=(10, 20))
+    _run(specs, video, n=n, stats=True, keyframe_at=(3,))
+
+
+def test_explicit_bn_equals_the_folded_stack_on_the_gpu():
+    """fp32: the stack with its affines unfolded and the stack with them folded into filters and bias give the same
+    tensors within the fp32 tolerance, on the library's delta path."""
+    rrm = _rrm()
+    specs = wl.with_explicit_bn(wl.alexnet_convs("f32", hw=99, scale=8))
+    folded = wl.fold_bn_f32(specs)
+    video = wl.moving_rect_video(frames=5, hw=99, dtype="f32", seed=30, side=(10, 20))
+    a, b = rrm.net_from_specs(specs), rrm.net_from_specs(folded)
+    oa, ob = a.new_output(), b.new_output()
+    for t in range(5):
+        a.step(dev(video[t]), oa)
+        b.step(dev(video[t]), ob)
+        scale = float(ob.abs().max())
+        assert float((oa - ob).abs().max()) <= 5 * F32_TOL * max(scale, 1e-6), t
+    # removing the affine again gives the plain stack's fresh state
+    plain = wl.alexnet_convs("f32", hw=99, scale=8)
+    for l in range(len(specs)):
+        a.set_affine(l, None, None)
+    a.step(dev(video[0]), oa)
+    want = orc.dense_forward(plain, video[0])[0][len(plain)]
+    assert float(np.abs(oa.cpu().numpy() - want).max()) <= F32_TOL * float(np.abs(want).max())
+    a.close(); b.close()
+
+
+def test_affine_is_rejected_where_it_is_not_defined():
+    rrm = _rrm()
+    specs = wl.xnor_alexnet_convs(hw=99, scale=8)
+    net = rrm.net_from_specs(specs)
+    z = torch.zeros(specs[0].c_out, dtype=torch.int32, device="cuda")
+    with pytest.raises(rrm.RRMError):
+        net.set_affine(0, z, z)               # a sign layer
+    with pytest.raises(rrm.RRMError):
+        net.set_affine(0, z, None)
+    net.close()

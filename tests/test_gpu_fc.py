@@ -325,3 +325,65 @@ def test_fc_dense_few_rows_on_tensor_cores(c_in, c_out, shift, act, n, T):
     np.testing.assert_array_equal(Y1.cpu().numpy().astype(np.int64), want[1][0][1].astype(np.int64))
     assert layer.stats(0)["error_word"] == 0
     layer.close()
+
+
+# ------------------------------------------------------------------ weight-sparse x delta-sparse (Sec. 3.5 / 4.3)
+@pytest.mark.parametrize("rho", [0.01, 0.05, 0.20])
+def test_weight_sparse_fc_is_bit_exact_at_every_density(rho):
+    """A magnitude-pruned layer (10 % of the weights kept) in the weight-sparse form: chunks, single frames, the
+    keyframe and the stateless dense path all give the integers of the dense FC definition on the pruned matrix;
+    the counters are those of Algorithm 1 (Table 1 counts whole columns)."""
+    import paper_1802_09723_b200 as rrm
+    c_in, c_out, n, F = 2048, 1040, 2, 12                     # two full 512-output slices and a ragged third
+    spec = wl.fc6_i8_pruned(c_in=c_in, c_out=c_out, keep=0.10)[0]
+    assert 0.08 < float(np.mean(spec.weight != 0)) < 0.12
+    seq = wl.fc_run_sequence(frames=F, c_in=c_in, rho=rho, seed=61, n=n)
+    seq[5] = seq[4]                                            # a frame with nothing to do
+    layer = rrm.layer_from_spec(spec, n=n, variant="sparse_w")
+    frames = dev(seq)
+    want = [orc.dense_forward([spec], seq[t])[1][0].reshape(n, c_out) for t in range(F)]
+    Y = layer.new_output(frames=4)
+    t0 = 0
+    for T in (4, 4, 1, 3):
+        layer.step_seq(frames[t0:t0 + T], Y[:T], T)
+        for i in range(T):
+            np.testing.assert_array_equal(Y[i].cpu().numpy().astype(np.int64).reshape(n, c_out), want[t0 + i], err_msg=f"frame {t0 + i}")
+        st = layer.stats(0)
+        nnz = sum(int(np.count_nonzero(seq[t] != (seq[t - 1] if t else np.zeros_like(seq[0])))) for t in range(t0, t0 + T))
+        assert st["variant"] == 4 and st["nnz_elems"] == nnz and st["active_macs"] == nnz * c_out and st["error_word"] == 0, st
+        t0 += T
+    np.testing.assert_array_equal(layer.projection(0).cpu().numpy().astype(np.int64).reshape(n, c_out), want[t0 - 1])
+    # frame-by-frame stepping, a keyframe, and the stateless dense path on the same weights
+    y1 = layer.new_output()
+    layer.keyframe(frames[2], y1)
+    np.testing.assert_array_equal(y1.cpu().numpy().astype(np.int64).reshape(n, c_out), want[2])
+    for t in (3, 4, 5):
+        layer.step(frames[t], y1)
+        np.testing.assert_array_equal(y1.cpu().numpy().astype(np.int64).reshape(n, c_out), want[t])
+    layer.dense(frames[9], y1)
+    np.testing.assert_array_equal(y1.cpu().numpy().astype(np.int64).reshape(n, c_out), want[9])
+    layer.step(frames[6], y1)                                  # the state was left alone by the dense path
+    np.testing.assert_array_equal(y1.cpu().numpy().astype(np.int64).reshape(n, c_out), want[6])
+    layer.close()
+
+
+def test_weight_sparse_fc_full_range_deltas_and_unpruned_weights():
+    """The form does not depend on the matrix being sparse (a dense matrix packs every group) and takes deltas
+    outside the int8 range like the column gather does."""
+    import paper_1802_09723_b200 as rrm
+    c_in, c_out = 512, 512
+    spec = wl.fc6_i8(c_in=c_in, c_out=c_out)[0]
+    rng = np.random.default_rng(3)
+    seq = rng.integers(-127, 128, size=(4, 1, c_in)).astype(np.int8)
+    seq[2, 0, ::2] = seq[1, 0, ::2]
+    layer = rrm.layer_from_spec(spec, variant="sparse_w")
+    Y = layer.new_output(frames=4)
+    layer.step_seq(dev(seq), Y, 4)
+    for t in range(4):
+        np.testing.assert_array_equal(Y[t].cpu().numpy().astype(np.int64).reshape(1, c_out),
+                                      orc.dense_forward([spec], seq[t])[1][0].reshape(1, c_out))
+    layer.close()
+    # the variant exists for a lone int8 FC layer only
+    conv = wl.single_conv_f32(c_in=4, c_out=4, hw=8)
+    with pytest.raises(rrm.RRMError):
+        rrm.net_from_specs(conv, variant="sparse_w")

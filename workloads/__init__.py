@@ -7,13 +7,13 @@ inputs from here, so the two sides see byte-identical tensors.
 
 All draws use numpy's counter-based Philox generator keyed by an integer seed.
 """
-from .nets import (LayerSpec, single_conv_f32, fc6_i8, alexnet_convs, resnet18_convs,
+from .nets import (LayerSpec, single_conv_f32, fc6_i8, fc6_i8_pruned, alexnet_convs, resnet18_convs,
                    xnor_alexnet_convs, alexnet_full, vgg16_convs, out_hw, tensor_shapes, dense_macs,
                    with_explicit_bn, fold_bn_f32)
 from .video import (block_redraw_sequence, fc_run_sequence, moving_rect_video)
 
 __all__ = [
-    "LayerSpec", "single_conv_f32", "fc6_i8", "alexnet_convs", "resnet18_convs",
+    "LayerSpec", "single_conv_f32", "fc6_i8", "fc6_i8_pruned", "alexnet_convs", "resnet18_convs",
     "xnor_alexnet_convs", "alexnet_full", "vgg16_convs", "out_hw", "tensor_shapes", "dense_macs",
     "with_explicit_bn", "fold_bn_f32",
     "block_redraw_sequence", "fc_run_sequence", "moving_rect_video",

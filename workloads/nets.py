@@ -155,6 +155,18 @@ def fc6_i8(seed=2, c_in=9216, c_out=4096):
     return _resolve_src([s])
 
 
+def fc6_i8_pruned(seed=2, c_in=9216, c_out=4096, keep=0.10):
+    """The same layer after magnitude pruning: only the fraction `keep` of the weights with the largest magnitude
+    stays, the rest is zero (unstructured, as deep compression leaves a layer; stands in for the compressed
+    AlexNet of the paper's Table 4, whose trained weights are not available)."""
+    s = fc6_i8(seed, c_in, c_out)[0]
+    mag = np.abs(s.weight.astype(np.int16))
+    thr = np.quantile(mag, 1.0 - keep)
+    s.weight = np.where(mag > thr, s.weight, 0).astype(np.int8)
+    s.name = "fc6_pruned"
+    return [s]
+
+
 # ---------------------------------------------------------------- config 3
 def alexnet_convs(dtype="f32", seed=3, hw=227, scale=1):
     """conv1..conv5 of an AlexNet-shaped stack (groups=1, no LRN, 3x3 s2 floor pools
