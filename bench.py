@@ -540,11 +540,11 @@ def main():
     def reduce_max(ms):
         return max_over_ranks(ms, world, "cuda")
 
-    def make(rho, n=1, variant="auto"):
+    def make(rho, n=1, variant="auto", weights=None):
         """Layer + the endless back-and-forth walk over the 32-frame sequence, laid out so that chunk k
         is rows [k*T, (k+1)*T) of one device array (whole number of periods, so it wraps seamlessly)."""
         desc = rrm.desc_from_spec(spec, n=n, variant=variant)
-        layer = rrm.Net([desc], [W], [B])
+        layer = rrm.Net([desc], [W if weights is None else weights], [B])
         seq = wl.fc_run_sequence(frames=FRAMES, rho=rho, seed=21 + rank, n=n)
         total = period * T // np.gcd(period, T)
         walk = np.stack([seq[order[(i + 1) % period]] for i in range(total)])      # frame i+1 of the walk
@@ -737,6 +737,43 @@ def main():
         delta_fc["note"] = ("column gather forced (variant GATHER), one launch per chunk, cold L2 before every launch.  "
                             "frac_distinct_cold_bytes = bytes the launch must fetch from HBM / time / measured HBM peak; "
                             "served_gbs = all gathered bytes (repeats served by L2) per second: a rate, not an HBM fraction")
+
+    # ---- weight-sparse x delta-sparse (Sec. 3.5 / 4.3): fc6 magnitude-pruned to 10 %, the weight-sparse form against
+    # the column gather and the dense tensor-core pass on the same pruned matrix
+    if not args.quick:
+        pr = wl.fc6_i8_pruned(keep=0.10)[0]
+        Wp = torch.from_numpy(pr.weight).cuda()
+        kept = float(np.mean(pr.weight != 0))
+        groups = float(np.mean(np.any(pr.weight.reshape(C_OUT // 4, 4, C_IN) != 0, axis=1)))   # non-zero groups of four outputs
+        sw = {"weights_kept": kept, "nonzero_groups_of_4": groups,
+              "bytes_per_gathered_column": {"dense": C_OUT, "weight_sparse": groups * C_OUT + 16 * (C_OUT // 512)}}
+        for rho in RHOS:
+            row = {}
+            for nm, var in (("weight_sparse", "sparse_w"), ("column_gather", "gather"), ("library_auto", "auto")):
+                Lp, sq, wk, wd, nz, un = make(rho, variant=var, weights=Wp)
+                row[nm + "_us"] = timed_chunks(Lp, sq, wd, 62, 10, cold=True)["median"] * 1e3
+                Lp.close()
+            row["nnz_mean_per_frame"] = nz
+            row["weight_sparse_bytes_per_chunk"] = T * (nz * sw["bytes_per_gathered_column"]["weight_sparse"] + 12 * C_OUT + 3 * C_IN)
+            row["column_gather_bytes_per_chunk"] = T * frame_bytes(nz)
+            row["speedup_vs_column_gather"] = row["column_gather_us"] / row["weight_sparse_us"]
+            row["speedup_vs_library_auto"] = row["library_auto_us"] / row["weight_sparse_us"]
+            sw[f"{rho:g}"] = row
+        Lp, sq, wk, wd, nz, un = make(args.rho, n=16, variant="sparse_w", weights=Wp)
+        s16 = timed_chunks(Lp, sq, wd, 31, 5, cold=True)["median"] * 1e3
+        Lp.close()
+        Lp, sq, wk, wd, nz, un = make(args.rho, n=16, variant="gather", weights=Wp)
+        g16 = timed_chunks(Lp, sq, wd, 31, 5, cold=True)["median"] * 1e3
+        Lp.close()
+        Lp, sq, wk, wd, nz, un = make(args.rho, n=16, variant="auto", weights=Wp)
+        a16 = timed_chunks(Lp, sq, wd, 31, 5, cold=True)["median"] * 1e3
+        Lp.close()
+        sw[f"{args.rho:g}_x16_streams"] = {"weight_sparse_us": s16, "column_gather_us": g16, "library_auto_us": a16,
+                                           "speedup_vs_column_gather": g16 / s16, "speedup_vs_library_auto": a16 / s16}
+        sw["note"] = ("one launch per 32-frame chunk, cold L2, median; library_auto = what RRM_VARIANT_AUTO runs on the pruned "
+                      "matrix stored densely (column gather or the dense tensor-core chunk)")
+        extra["weight_sparse_fc"] = sw
+        del Wp
 
     # ---- the convolution configurations, compact (rank 0, one GPU): cfg1, cfg3 int8, cfg4 with the sparse product forced
     # and as the library chooses

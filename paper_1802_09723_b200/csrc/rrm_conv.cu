@@ -335,6 +335,50 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
                 mbar_wait(g_smem_u32(&s_full[j % GEMM_STAGES]), (j / GEMM_STAGES) & 1, WAIT_LIMIT_DEFAULT);
         }
         __syncthreads();
+        if (!(DT == T_F32 && p.ksplit > 1)) return;          // (an fp32 share still meets its cluster at the barriers below)
+    }
+
+    // ---- fp32 with the K range split over CTAs: the shares of a tile form one thread-block cluster and their partial
+    // sums meet through distributed shared memory in a FIXED order (share 0, 1, ...), so the stored projection is
+    // reproducible bit for bit and no float atomics are needed.  Every share parks its partial tile in its own
+    // shared memory; share r then adds up rows [r * TM / shares, (r + 1) * TM / shares) of all shares and updates
+    // the projection for them.
+    if (DT == T_F32 && p.ksplit > 1) {
+        float* tilebuf = reinterpret_cast<float*>(g_smem);   // [TM][TN]; the ring is free: every issued stage was consumed
+        __syncthreads();
+        #pragma unroll
+        for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<float4*>(&tilebuf[(tm + i) * TN + tn]) = make_float4((float)acc[i][0], (float)acc[i][1], (float)acc[i][2], (float)acc[i][3]);
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        const int rank = blockIdx.z, rows_per = TM / p.ksplit;
+        const uint32_t tile_u32 = g_smem_u32(tilebuf);
+        float* P = reinterpret_cast<float*>(p.P);
+        for (int item = tid; item < rows_per * (TN / 4); item += CONV_THREADS) {
+            const int row = rank * rows_per + item / (TN / 4), c4 = (item % (TN / 4)) * 4;
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int z = 0; z < p.ksplit; ++z) {
+                uint32_t remote;
+                float4 v;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(tile_u32 + (uint32_t)(row * TN + c4) * 4u), "r"(z));
+                asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+            }
+            const int q = s_q[row];
+            if (q < 0 || !ok) continue;
+            const float sv[4] = {sum.x, sum.y, sum.z, sum.w};
+            #pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int co = n0 + c4 + j;
+                if (co >= p.c_out) continue;
+                const size_t o = (size_t)q * p.c_out + co;
+                if (DENSE) P[o] = sv[j] + (p.bias ? reinterpret_cast<const float*>(p.bias)[co] : 0.f);
+                else P[o] += sv[j];
+            }
+        }
+        // nobody leaves while its tile may still be read
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         return;
     }
 
@@ -350,12 +394,11 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             const int co = n0 + tn + j;
             if (co >= p.c_out) continue;
             const size_t o = (size_t)q * p.c_out + co;
-            if (DT == T_F32) {
+            if (DT == T_F32) {                                 // (a tile owned by one CTA; shared fp32 tiles were closed above)
                 float* P = reinterpret_cast<float*>(p.P);
                 float v = acc[i][j];
-                if (DENSE && blockIdx.z == 0 && p.bias) v += reinterpret_cast<const float*>(p.bias)[co];
-                if (shared_tile) atomicAdd(P + o, v);
-                else if (DENSE) P[o] = v;
+                if (DENSE && p.bias) v += reinterpret_cast<const float*>(p.bias)[co];
+                if (DENSE) P[o] = v;
                 else P[o] += v;
             } else {
                 int* P = reinterpret_cast<int*>(p.P);
@@ -378,14 +421,21 @@ static size_t gemm_smem_bytes(int dt)
 template <int DT, bool DENSE>
 static void launch_gemm(const ConvParams& p, dim3 grid, cudaStream_t st)
 {
-    if (p.u_in % 4 == 0) launch_seq(conv_gemm_kernel<DT, DENSE, true>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, p);
-    else launch_seq(conv_gemm_kernel<DT, DENSE, false>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, p);
+    const int cluster_z = (DT == T_F32 && p.ksplit > 1) ? p.ksplit : 1;       // fp32 shares of a tile: one cluster
+    if (p.u_in % 4 == 0) launch_seq_cluster(conv_gemm_kernel<DT, DENSE, true>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, cluster_z, p);
+    else launch_seq_cluster(conv_gemm_kernel<DT, DENSE, false>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, cluster_z, p);
 }
 
 template <int DT>
 static int gemm_allow_smem()
 {
     const int b = (int)gemm_smem_bytes(DT);
+    if (DT == T_F32) {                                       // clusters of 16 CTAs are beyond the portable size of 8
+        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, true, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, false, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, true, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, false, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    }
     RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
     RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
     RRM_CUDA_TRY(cudaFuncSetAttribute(conv_gemm_kernel<DT, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b));
@@ -909,6 +959,20 @@ static int dev_alloc(rrm_net* net, void** p, size_t bytes, bool zero = true)
 
 static int proj_type(const Layer& L) { return L.d.dtype == RRM_F32 ? T_F32 : T_I32; }
 
+// CTAs that share one output tile of the CUDA-core kernel, each with a contiguous range of K stages: K is split
+// while the tiles alone leave most of the machine idle (each share keeps >= 2 stages).  A delta pass is sized as
+// if half of the tiles had rows: the others leave right after the row scan.
+static int gemm_ksplit(const Layer& L, bool dense)
+{
+    const int stages = L.kup / TK;
+    const long long gx = ceil_div(L.opixels(), TM), gy = L.np / TN;
+    const long long tiles = dense ? gx * gy : (gx + 1) / 2 * gy;
+    int ks = 1;
+    while (tiles * ks < 2 * 148 && stages / (ks * 2) >= 2) ks *= 2;
+    if (L.d.dtype == RRM_F32 && ks > 16) ks = 16;            // fp32 shares form a thread-block cluster (at most 16 CTAs on this GPU)
+    return ks;
+}
+
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev)
 {
     const rrm_layer_desc& d = L.d;
@@ -927,6 +991,7 @@ int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bia
                                                     d.c_in, d.c_out, d.kh, d.kw, L.u_in, L.kup, L.np);
     RRM_CUDA_TRY(cudaGetLastError());
     if (d.kh * d.kw > 128) return RRM_ERR_UNSUPPORTED;       // the kernels keep a row's usable taps in a 128-bit mask
+
     RRM_TRY(gemm_allow_smem<T_F32>());
     RRM_TRY(gemm_allow_smem<T_I8>());
     RRM_TRY(gemm_allow_smem<T_BIN>());
@@ -1057,16 +1122,12 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     p.count_bitmap = step_dense ? L.oact : nullptr;
     dim3 grid(ceil_div(L.opixels(), TM), L.np / TN);
     p.errw = net->errw;
-    // split K over CTAs while the tiles alone leave most of the machine idle (each share keeps >= 4 stages)
     {
-        const int stages = L.kup / TK;
-        int ks = 1;
-        // (a delta pass is sized as if half of the tiles had rows: the others leave right after the row scan)
-        const long long tiles = conv_dense ? (long long)grid.x * grid.y : (long long)(grid.x + 1) / 2 * grid.y;
-        while (tiles * ks < 2 * 148 && stages / (ks * 2) >= 2) ks *= 2;
+        const int ks = gemm_ksplit(L, conv_dense);
         p.ksplit = ks;
         grid.z = ks;
-        if (!L.tc_ready && conv_dense && ks > 1) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));
+        // (integer shares add onto a zeroed projection; fp32 shares meet in their cluster's shared memory, in a fixed order)
+        if (!L.tc_ready && conv_dense && ks > 1 && d.dtype != RRM_F32) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));
     }
     if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, conv_dense, stateless, st, p.count_bitmap));
     else if (d.dtype == RRM_F32) { if (conv_dense) launch_gemm<T_F32, true>(p, grid, st); else launch_gemm<T_F32, false>(p, grid, st); }

@@ -536,3 +536,27 @@ def test_affine_is_rejected_where_it_is_not_defined():
     with pytest.raises(rrm.RRMError):
         net.set_affine(0, z, None)
     net.close()
+
+
+# ------------------------------------------------------------------ fp32 results are reproducible bit for bit
+@pytest.mark.parametrize("name", ["cfg1", "alex_f32"])
+def test_fp32_projections_are_bitwise_reproducible(name):
+    """Layers whose K range is split over CTAs add their shares' partial sums in a fixed order, so two runs over the
+    same frames leave bit-identical projections (the race detector of last resort: any unordered float addition or
+    data race would show here)."""
+    rrm = _rrm()
+    if name == "cfg1":
+        specs, video = wl.single_conv_f32(), wl.block_redraw_sequence()
+    else:
+        specs, video = wl.alexnet_convs("f32", hw=131, scale=4), wl.moving_rect_video(frames=6, hw=131, dtype="f32", seed=3, side=(12, 24))
+    runs = []
+    for rep in range(3):
+        net = rrm.net_from_specs(specs, variant="tensor")      # (no density switch: every frame through the delta kernels)
+        out = net.new_output()
+        for t in range(video.shape[0]):
+            net.step(dev(video[t]), out)
+        runs.append([net.projection(l).clone() for l in range(len(specs))] + [out.clone()])
+        net.close()
+    for other in runs[1:]:
+        for a, b in zip(runs[0], other):
+            assert torch.equal(a, b)
