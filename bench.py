@@ -6,8 +6,9 @@ accumulation, 32-frame sequences whose frames differ in a fraction rho of the in
 of 32).  One "step" = one chunk of 32 consecutive frames of one stream through the whole hot path of the layer
 (delta + compaction, sparse product, accumulate + snapshot + output for every frame), i.e. one rrm_step_seq call
 = one kernel launch; the reported value is frames per second.  The line also carries, under "conv", compact
-results of the convolution configurations (cfg1, cfg3 int8, cfg4) and, under "by_rho" / "roofline_delta_fc",
-the column-gather kernel forced at 1 / 5 / 20 % density.
+results of the convolution configurations (cfg1, cfg3 fp32 / int8, cfg4, cfg5) and, under "by_rho" /
+"roofline_delta_fc" / "weight_sparse_fc", the column-gather kernel forced at 1 / 5 / 20 % density and the
+weight-sparse form on a pruned matrix.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--rho 0.05] [--chunk 32] [--impl ours|reference]
   python bench.py --workload cfg1|cfg3_f32|cfg3_i8|cfg4|cfg5 [--streams N] [--seq T] [--variant auto|tensor|gather]
@@ -780,7 +781,8 @@ def main():
     conv = None
     if rank == 0 and world == 1 and not args.quick:
         conv = {}
-        for key, name, variant, fr_n, cpu_n in (("cfg1", "cfg1", "auto", None, 2), ("cfg3_i8", "cfg3_i8", "auto", 16, 2),
+        for key, name, variant, fr_n, cpu_n in (("cfg1", "cfg1", "auto", None, 2), ("cfg3_f32", "cfg3_f32", "auto", 16, 1),
+                                                ("cfg3_i8", "cfg3_i8", "auto", 16, 2), ("cfg5", "cfg5", "auto", 16, 1),
                                                 ("cfg4_delta_forced", "cfg4", "tensor", 8, 1), ("cfg4_auto", "cfg4", "auto", 8, 0)):
             try:
                 conv[key] = compact_conv(conv_measure(name, variant, steps=30, warmup=5, frames=fr_n, cpu_frames=cpu_n,

@@ -19,6 +19,7 @@
 #include "rrm_common.cuh"
 #include "rrm_rows.cuh"
 #include "rrm_tc.cuh"
+#include "rrm_dev.cuh"
 #include <type_traits>
 
 namespace rrm {
@@ -139,51 +140,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
             const int y0 = oy * p.stride - p.pad, x0 = ox * p.stride - p.pad;
             pix0 = ns * p.h * p.w + y0 * p.w + x0;
-            if (p.kw <= 32) {
-                // one filter row at a time: its usable taps are a run of consecutive input pixels, whose activity bits
-                // come out of one or two bitmap words together
-                const int kx_lo = max(0, -x0), kx_hi = min(p.kw, p.w - x0), nk = kx_hi - kx_lo;
-                const unsigned run = nk >= 32 ? 0xffffffffu : ((1u << max(nk, 0)) - 1u);
-                for (int ky = 0; ky < p.kh && nk > 0; ++ky) {
-                    const int iy = y0 + ky;
-                    if (iy < 0 || iy >= p.h) continue;
-                    unsigned bits = run;
-                    if (!DENSE) {
-                        const int g = pix0 + ky * p.w + kx_lo, sh = g & 31;
-                        unsigned long long two = p.in_act[g >> 5];
-                        if (sh + nk > 32) two |= (unsigned long long)p.in_act[(g >> 5) + 1] << 32;
-                        bits = (unsigned)(two >> sh) & run;
-                    }
-                    if (bits == 0) continue;
-                    const int t = ky * p.kw + kx_lo;             // tap index of the run's first bit
-                    if (t < 64) {
-                        m0 |= (unsigned long long)bits << t;
-                        if (t + nk > 64) m1 |= (unsigned long long)bits >> (64 - t);
-                    } else {
-                        m1 |= (unsigned long long)bits << (t - 64);
-                    }
-                }
-            } else
-            for (int t0 = 0; t0 < taps; t0 += 8) {          // (very wide filters) 8 taps at a time: all bitmap loads first
-                uint32_t word[8];
-                int sh[8];
-                #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int t = t0 + u, ky = t / p.kw, kx = t - ky * p.kw;
-                    const int iy = y0 + ky, ix = x0 + kx;
-                    const bool in = t < taps && iy >= 0 && iy < p.h && ix >= 0 && ix < p.w;
-                    const int pix = pix0 + ky * p.w + kx;
-                    sh[u] = in ? (pix & 31) : -1;
-                    word[u] = DENSE ? 0xffffffffu : (in ? p.in_act[pix >> 5] : 0u);
-                }
-                #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (sh[u] >= 0 && ((word[u] >> sh[u]) & 1u)) {
-                        const int t = t0 + u;
-                        if (t < 64) m0 |= 1ull << t; else m1 |= 1ull << (t - 64);
-                    }
-                }
-            }
+            row_tap_masks<DENSE>(p.in_act, pix0, y0, x0, p.h, p.w, p.kh, p.kw, m0, m1);
         }
         s_pix0[tid] = pix0;
         s_rmask[tid][0] = m0; s_rmask[tid][1] = m1;

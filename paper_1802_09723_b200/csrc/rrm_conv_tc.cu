@@ -22,6 +22,7 @@
 #include "rrm_common.cuh"
 #include "rrm_rows.cuh"
 #include "rrm_tc.cuh"
+#include "rrm_dev.cuh"
 
 namespace rrm {
 
@@ -119,52 +120,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             const int ox = q % p.ow, oy = (q / p.ow) % p.oh, ns = q / (p.ow * p.oh);
             const int y0 = oy * p.stride - p.pad, x0 = ox * p.stride - p.pad;
             pix0 = ns * p.h * p.w + y0 * p.w + x0;
-            if (p.kw <= 32) {
-                // one filter row at a time: its usable taps are a run of consecutive input pixels, whose activity bits
-                // come out of one or two bitmap words together
-                const int kx_lo = max(0, -x0), kx_hi = min(p.kw, p.w - x0), nk = kx_hi - kx_lo;
-                const int kh = p.taps / p.kw;
-                const unsigned run = nk >= 32 ? 0xffffffffu : ((1u << max(nk, 0)) - 1u);
-                for (int ky = 0; ky < kh && nk > 0; ++ky) {
-                    const int iy = y0 + ky;
-                    if (iy < 0 || iy >= p.h) continue;
-                    unsigned bits = run;
-                    if (!DENSE) {
-                        const int g = pix0 + ky * p.w + kx_lo, sh = g & 31;
-                        unsigned long long two = p.in_act[g >> 5];
-                        if (sh + nk > 32) two |= (unsigned long long)p.in_act[(g >> 5) + 1] << 32;
-                        bits = (unsigned)(two >> sh) & run;
-                    }
-                    if (bits == 0) continue;
-                    const int t = ky * p.kw + kx_lo;             // tap index of the run's first bit
-                    if (t < 64) {
-                        m0 |= (unsigned long long)bits << t;
-                        if (t + nk > 64) m1 |= (unsigned long long)bits >> (64 - t);
-                    } else {
-                        m1 |= (unsigned long long)bits << (t - 64);
-                    }
-                }
-            } else
-            for (int t0 = 0; t0 < p.taps; t0 += 8) {          // (very wide filters) 8 taps at a time: all bitmap loads first
-                uint32_t word[8];
-                int sh[8];
-                #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int t = t0 + u, ky = t / p.kw, kx = t - ky * p.kw;
-                    const int iy = y0 + ky, ix = x0 + kx;
-                    const bool in = t < p.taps && iy >= 0 && iy < p.h && ix >= 0 && ix < p.w;
-                    const int pix = pix0 + ky * p.w + kx;
-                    sh[u] = in ? (pix & 31) : -1;
-                    word[u] = DENSE ? 0xffffffffu : (in ? p.in_act[pix >> 5] : 0u);
-                }
-                #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (sh[u] >= 0 && ((word[u] >> sh[u]) & 1u)) {
-                        const int t = t0 + u;
-                        if (t < 64) m0 |= 1ull << t; else m1 |= 1ull << (t - 64);
-                    }
-                }
-            }
+            row_tap_masks<DENSE>(p.in_act, pix0, y0, x0, p.h, p.w, p.taps / p.kw, p.kw, m0, m1);
         }
         S->pix0[tid] = pix0;
         S->rmask[tid][0] = m0; S->rmask[tid][1] = m1;
@@ -608,11 +564,10 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     // split K towards the point where a CTA's slabs all fit in its pipeline at once
     // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the
     // machine needs: once the tiles alone fill it, a tile owned by one CTA saves the adds of shared tiles
-    const int wave = 148 * 2;
+    const int wave = 148;                                    // (measured: one CTA per SM is enough; more shares only add reductions)
     int ksplit = 1;
     const int ks_max = ceil_div(L.tc_slabs, TC_STAGES);
-    // (a delta pass is sized as if half of the tiles had rows: the others leave right after the row scan)
-    const long long tiles = dense ? (long long)m_tiles * L.tc_ntiles : (long long)(m_tiles + 1) / 2 * L.tc_ntiles;
+    const long long tiles = (long long)m_tiles * L.tc_ntiles;
     while (ksplit < ks_max && tiles * ksplit < wave) ++ksplit;
     ksplit = ceil_div(L.tc_slabs, ceil_div(L.tc_slabs, ksplit));   // no empty shares
     p.ksplit = ksplit;

@@ -13,6 +13,7 @@
 //   4. one CTA per stream writes the new snapshot into the other half of a ping-pong pair.
 // Cost is HBM-bound: nnz * C_out weight bytes per frame.
 #include "rrm_common.cuh"
+#include "rrm_dev.cuh"
 #include <cooperative_groups.h>
 #include <mutex>
 
@@ -38,13 +39,6 @@ struct FcParams {
     unsigned long long* stat;// [n][2]: nnz elements, active groups of 32 inputs (or nullptr)
     int c_in, c_out, shift, act;
 };
-
-__device__ __forceinline__ int fc_apply_f(int v, int shift, int act) {
-    if (shift > 0) v = (v + (1 << (shift - 1))) >> shift;
-    v = max(-127, min(127, v));
-    if (act == RRM_ACT_RELU) v = max(v, 0);
-    return v;
-}
 
 // Split cluster barrier.  Every thread alternates arrive and wait; a thread may exit after an arrive.
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
@@ -99,17 +93,7 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
         if (c_begin + i < nchunks) {
             reinterpret_cast<uint4*>(s_xt)[c_begin + i] = xa[i];
             reinterpret_cast<uint4*>(s_xp)[c_begin + i] = xb[i];
-            unsigned cm;
-            if (xp4) {
-                auto nib = [](unsigned v) {           // one flag bit per non-zero byte, packed into 4 bits
-                    v |= v >> 4; v |= v >> 2; v |= v >> 1;
-                    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
-                };
-                cm = nib(xa[i].x ^ xb[i].x) | nib(xa[i].y ^ xb[i].y) << 4 | nib(xa[i].z ^ xb[i].z) << 8 |
-                     nib(xa[i].w ^ xb[i].w) << 12;
-            } else {
-                cm = 0xffffu;
-            }
+            const unsigned cm = xp4 ? differing_bytes(xa[i], xb[i]) : 0xffffu;
             m |= (unsigned long long)cm << (16 * i);
         }
     }
@@ -184,26 +168,6 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
     #pragma unroll
     for (int i = 0; i < 16; ++i) acc[i] = 0;
     const int8_t* wbase = p.Wt + o0;
-    // acc[i] += w_i * d for the 16 int8 weights in w: dp4a against a selector that holds d in one
-    // byte lane; a delta outside int8 range (|d| <= 254) is split into two in-range halves.
-    auto fma16 = [&](const uint4& w, int d) {
-        const unsigned ww[4] = {w.x, w.y, w.z, w.w};
-        const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
-        const int dl = d - dh;
-        const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
-        #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            #pragma unroll
-            for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
-        }
-        if (dh != 0) {
-            #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
-            }
-        }
-    };
     if (o_ok) {
         constexpr int U = 8;                           // columns in flight per thread
         for (int e = grp; e < mine; e += U * FC_GROUPS) {
@@ -219,7 +183,7 @@ __global__ void __cluster_dims__(FC_CL, 1, 1) __launch_bounds__(FC_THREADS) fc_d
                 w[u] = j[u] >= 0 ? __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)j[u] * K)) : make_uint4(0, 0, 0, 0);
             #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (j[u] >= 0) fma16(w[u], (int)s_xt[j[u]] - (int)s_xp[j[u]]);
+                if (j[u] >= 0) fma16(acc, w[u], (int)s_xt[j[u]] - (int)s_xp[j[u]]);
         }
     }
     // ---- 4. reduce: the 4 column groups of a warp by shuffles, the 8 warps through shared memory
@@ -294,14 +258,7 @@ __global__ void __launch_bounds__(FC_THREADS) fc_scan_kernel(FcParams p, void* s
             reinterpret_cast<uint4*>(s_xp)[c_begin + i] = b;
             // the thread that read a chunk of the snapshot is the one that overwrites it: in place is safe
             if (p.xnext) reinterpret_cast<uint4*>(p.xnext + (size_t)s * C)[c_begin + i] = a;
-            unsigned cm = 0xffffu;
-            if (xp4) {
-                auto nib = [](unsigned v) {
-                    v |= v >> 4; v |= v >> 2; v |= v >> 1;
-                    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
-                };
-                cm = nib(a.x ^ b.x) | nib(a.y ^ b.y) << 4 | nib(a.z ^ b.z) << 8 | nib(a.w ^ b.w) << 12;
-            }
+            const unsigned cm = xp4 ? differing_bytes(a, b) : 0xffffu;
             m |= (unsigned long long)cm << (16 * i);
         }
     }
@@ -374,24 +331,6 @@ __global__ void __launch_bounds__(FC_THREADS) fc_gather_kernel(FcParams p, const
     #pragma unroll
     for (int i = 0; i < 16; ++i) acc[i] = 0;
     const int8_t* wbase = p.Wt + o0;
-    auto fma16 = [&](const uint4& w, int d) {
-        const unsigned ww[4] = {w.x, w.y, w.z, w.w};
-        const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
-        const int dl = d - dh;
-        const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
-        #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            #pragma unroll
-            for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
-        }
-        if (dh != 0) {
-            #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
-            }
-        }
-    };
     if (o0 < K) {
         constexpr int U = 8;
         for (int e = grp; e < total; e += U * FC_GROUPS) {
@@ -408,7 +347,7 @@ __global__ void __launch_bounds__(FC_THREADS) fc_gather_kernel(FcParams p, const
                                              : make_uint4(0, 0, 0, 0);
             #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (ent[u] != 0xffffffffu) fma16(w[u], (int)(ent[u] >> 16) - 256);
+                if (ent[u] != 0xffffffffu) fma16(acc, w[u], (int)(ent[u] >> 16) - 256);
         }
     }
     #pragma unroll

@@ -19,6 +19,7 @@
 //      writes Y_0 .. Y_{T-1}.
 // Cost: the weight columns of the non-zero entries (HBM; frames of a chunk share columns through L2).
 #include "rrm_common.cuh"
+#include "rrm_dev.cuh"
 #include <cstring>
 
 namespace rrm {
@@ -44,43 +45,6 @@ struct FcSeqParams {
     const uint32_t* Wsp;     // weight-sparse form: [c_in][slices] records of sp_stride words (map, then packed groups)
     int sp_stride;
 };
-
-__device__ __forceinline__ int seq_apply_f(int v, int shift, int act)
-{
-    if (shift > 0) v = (v + (1 << (shift - 1))) >> shift;
-    v = max(-127, min(127, v));
-    if (act == RRM_ACT_RELU) v = max(v, 0);
-    return v;
-}
-
-// one flag bit per non-zero byte of v, packed into the low 4 bits
-__device__ __forceinline__ unsigned nonzero_bytes(unsigned v)
-{
-    v |= v >> 4; v |= v >> 2; v |= v >> 1;
-    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
-}
-
-// acc[i] += w_i * d for the 16 int8 weights in w: dp4a against a selector holding d in one byte
-// lane; a delta outside int8 range (|d| <= 254) is split into two in-range halves.
-__device__ __forceinline__ void fma16(int (&acc)[16], const uint4& w, int d)
-{
-    const unsigned ww[4] = {w.x, w.y, w.z, w.w};
-    const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
-    const int dl = d - dh;
-    const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
-    #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(lb << (8 * b)), acc[q * 4 + b]);
-    }
-    if (dh != 0) {
-        #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            #pragma unroll
-            for (int b = 0; b < 4; ++b) acc[q * 4 + b] = __dp4a((int)ww[q], (int)(hb << (8 * b)), acc[q * 4 + b]);
-        }
-    }
-}
 
 // LANES: lanes of a warp that span one column slice (16 bytes each): the CTA owns OW = 16 * LANES
 // outputs and a warp-wide load fetches 32 / LANES columns.  Narrow slices mean more CTAs and fewer
@@ -149,9 +113,7 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
         if (i * SQ_THREADS >= nchunks) break;                // uniform
         unsigned m = 0;
         if (chunk < nchunks)
-            m = xp4 ? (nonzero_bytes(a[i].x ^ b[i].x) | nonzero_bytes(a[i].y ^ b[i].y) << 4 |
-                       nonzero_bytes(a[i].z ^ b[i].z) << 8 | nonzero_bytes(a[i].w ^ b[i].w) << 12)
-                    : 0xffffu;
+            m = xp4 ? differing_bytes(a[i], b[i]) : 0xffffu;
         const int local = __popc(m);
         int incl = local;
         #pragma unroll
@@ -355,8 +317,8 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
                     *reinterpret_cast<int4*>(reinterpret_cast<int32_t*>(p.Y) + oi) = v;
                 } else {
                     char4 q;
-                    q.x = (signed char)seq_apply_f(v.x, p.shift, p.act); q.y = (signed char)seq_apply_f(v.y, p.shift, p.act);
-                    q.z = (signed char)seq_apply_f(v.z, p.shift, p.act); q.w = (signed char)seq_apply_f(v.w, p.shift, p.act);
+                    q.x = (signed char)fc_apply_f(v.x, p.shift, p.act); q.y = (signed char)fc_apply_f(v.y, p.shift, p.act);
+                    q.z = (signed char)fc_apply_f(v.z, p.shift, p.act); q.w = (signed char)fc_apply_f(v.w, p.shift, p.act);
                     *reinterpret_cast<char4*>(reinterpret_cast<int8_t*>(p.Y) + oi) = q;
                 }
             }
@@ -385,7 +347,7 @@ __global__ void __launch_bounds__(SQ_THREADS) fc_count_kernel(const int8_t* __re
         unsigned m = 0;
         if (chunk < (C >> 4)) {
             const uint4 a = __ldg(xt4 + chunk), b = __ldg(xp4 + chunk);
-            m = nonzero_bytes(a.x ^ b.x) | nonzero_bytes(a.y ^ b.y) << 4 | nonzero_bytes(a.z ^ b.z) << 8 | nonzero_bytes(a.w ^ b.w) << 12;
+            m = differing_bytes(a, b);
         }
         nnz += __popc(m);
         const unsigned other = __shfl_xor_sync(0xffffffffu, m, 1);
@@ -588,7 +550,7 @@ __global__ void fc_dense_finish_kernel(const int32_t* __restrict__ Pd, void* Y, 
     if (Pstate && i >= state_from) Pstate[i - state_from] = v;
     if (Y) {
         if (shift < 0) reinterpret_cast<int32_t*>(Y)[i] = v;
-        else reinterpret_cast<int8_t*>(Y)[i] = (int8_t)seq_apply_f(v, shift, act);
+        else reinterpret_cast<int8_t*>(Y)[i] = (int8_t)fc_apply_f(v, shift, act);
     }
 }
 

@@ -17,6 +17,7 @@
 #include <cuda.h>
 #include "rrm_common.cuh"
 #include "rrm_tc.cuh"
+#include "rrm_dev.cuh"
 
 namespace rrm {
 
@@ -52,21 +53,6 @@ struct FtParams {
     unsigned wait_limit;      // polls of one bounded wait
 };
 
-__device__ __forceinline__ int ft_apply_f(int v, int shift, int act)
-{
-    if (shift > 0) v = (v + (1 << (shift - 1))) >> shift;
-    v = max(-127, min(127, v));
-    if (act == RRM_ACT_RELU) v = max(v, 0);
-    return v;
-}
-
-// one flag bit per non-zero byte of v, packed into the low 4 bits
-__device__ __forceinline__ unsigned ft_nonzero_bytes(unsigned v)
-{
-    v |= v >> 4; v |= v >> 2; v |= v >> 1;
-    return ((v & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
-}
-
 __device__ __forceinline__ void ft_finish(const FtParams& p, int row, int o, int v)
 {
     if (p.bias) v += p.bias[o];
@@ -74,7 +60,7 @@ __device__ __forceinline__ void ft_finish(const FtParams& p, int row, int o, int
     if (p.Pstate && row >= p.state_from) p.Pstate[i - (size_t)p.state_from * p.c_out] = v;
     if (p.Y) {
         if (p.shift < 0) reinterpret_cast<int32_t*>(p.Y)[i] = v;
-        else reinterpret_cast<int8_t*>(p.Y)[i] = (int8_t)ft_apply_f(v, p.shift, p.act);
+        else reinterpret_cast<int8_t*>(p.Y)[i] = (int8_t)fc_apply_f(v, p.shift, p.act);
     }
 }
 
@@ -88,8 +74,8 @@ __device__ __forceinline__ void ft_finish4(const FtParams& p, int row, int oo, i
         if (p.shift < 0) *reinterpret_cast<int4*>(reinterpret_cast<int32_t*>(p.Y) + at) = w;
         else {
             char4 q;
-            q.x = (signed char)ft_apply_f(w.x, p.shift, p.act); q.y = (signed char)ft_apply_f(w.y, p.shift, p.act);
-            q.z = (signed char)ft_apply_f(w.z, p.shift, p.act); q.w = (signed char)ft_apply_f(w.w, p.shift, p.act);
+            q.x = (signed char)fc_apply_f(w.x, p.shift, p.act); q.y = (signed char)fc_apply_f(w.y, p.shift, p.act);
+            q.z = (signed char)fc_apply_f(w.z, p.shift, p.act); q.w = (signed char)fc_apply_f(w.w, p.shift, p.act);
             *reinterpret_cast<char4*>(reinterpret_cast<int8_t*>(p.Y) + at) = q;
         }
     }
@@ -156,8 +142,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
                     unsigned m = 0;
                     if (chunk < c16) {
                         const uint4 a = __ldg(xt4 + chunk), b = __ldg(xp4 + chunk);
-                        m = ft_nonzero_bytes(a.x ^ b.x) | ft_nonzero_bytes(a.y ^ b.y) << 4 | ft_nonzero_bytes(a.z ^ b.z) << 8 |
-                            ft_nonzero_bytes(a.w ^ b.w) << 12;
+                        m = differing_bytes(a, b);
                     }
                     nnz += __popc(m);
                     const unsigned other = __shfl_xor_sync(0xffffffffu, m, 1);
