@@ -492,7 +492,8 @@ def main():
     ap.add_argument("--quick", action="store_true", help="skip the secondary sweeps and the CPU legs (profiling runs)")
     ap.add_argument("--workload", default="cfg2", choices=("cfg2",) + CONV_WORKLOADS,
                     help="cfg2 (default) is the contract line; the others are the convolution configurations")
-    ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense", "sparse_w"],
+                    help="rrm_layer_desc.variant of the timed object (default: the library chooses)")
     ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
     ap.add_argument("--streams", type=int, default=None, help="independent videos per call (convolution workloads)")
     ap.add_argument("--opt", action="append", help="rrm_options field=value (convolution workloads), e.g. --opt layer_dense_activity=0.9")
@@ -630,7 +631,7 @@ def main():
     peak, peak_kind = measured_peaks()
 
     # ---- primary: one stream per GPU, chunks of T frames per call, rho as asked, cold L2, per-step events
-    layer, seq, walk, walk_dev, nnz_mean, uniq_mean = make(args.rho)
+    layer, seq, walk, walk_dev, nnz_mean, uniq_mean = make(args.rho, variant=args.variant)
     # (setup, untimed and before the W warm-up steps: lets the library measure the density and settle on its
     # evaluation, allocate its pinned read-back buffer and scratch)
     timed_chunks(layer, seq, walk_dev, 4, 4, cold=True)
