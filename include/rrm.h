@@ -313,7 +313,7 @@ int rrm_fc_step_noalloc(const int8_t* Wt_dev, const int8_t* Xt_dev, int8_t* Xpre
 
 /* ---- measured ALU peaks -------------------------------------------------------------
  * (No counterpart in the paper: a reporting aid.)  Runs a register-only loop of independent operations on every
- * SM of the current device and returns the best of five timings as multiply-accumulates per second:
+ * SM of the current device and returns the best of four timings as multiply-accumulates per second:
  *   kind 0  fp32 fused multiply-add                       (the fp32 delta convolution, Table 1's MACs)
  *   kind 1  dp4a, counted as 4 int8 multiply-accumulates  (int8 layers on the CUDA cores, the delta-FC products)
  *   kind 2  popc + add, counted as 32 one-bit products    (binary layers on the CUDA cores, Sec. 4.3)

@@ -641,9 +641,10 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
 }
 
 // ------------------------------------------------------------------------------------------------
-// Epilogue: f on the stored projection, next layer's delta.  One warp per output-tensor pixel; a lane
-// owns 4 neighbouring channels at a time, so the 4-channel words of all window positions are fetched
-// with independent 128-bit loads (one memory round trip per 128 channels).
+// Epilogue: f on the stored projection, next layer's delta.  A pixel of the output tensor belongs to `wpp` warps
+// of one CTA (1, 2, 4 or 8: the chunks of 128 channels are dealt out to them, so that a pixel of a wide layer
+// costs one memory round trip, not one per chunk); a lane owns 4 neighbouring channels at a time, so the
+// 4-channel words of all window positions are fetched with independent 128-bit loads.
 // ------------------------------------------------------------------------------------------------
 struct EpiParams {
     const void* P;            // [opixels][c_out] float / int
@@ -657,6 +658,7 @@ struct EpiParams {
     unsigned long long* npix;
     int* errw;
     int n, oh, ow, th, tw, c_out, cs, pool_k, pool_s, pool_p, act_fn, shift, theta;
+    int wpp;                  // warps that share one output pixel (1, 2, 4 or 8); a CTA of 8 warps holds 8 / wpp pixels
     Readers readers;          // layers that read the output tensor
     float eps;                // fp32: delta entries below it are truncated to zero (Sec. 3.4)
     double* trunc;            // fp32: receives the sum of squares of the truncated entries
@@ -672,15 +674,18 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
     __shared__ unsigned long long s_macs[MAX_READERS];
     __shared__ unsigned int s_nnz, s_npix;
-    __shared__ int s_cnt[8];                                 // changed elements of the CTA's pixels (one per warp)
+    __shared__ int s_cnt[8];                                 // changed elements of the CTA's pixels
     __shared__ float s_sq;
     const int lane = threadIdx.x & 31;
     pdl_launch_dependents();
     if (threadIdx.x < MAX_READERS) s_macs[threadIdx.x] = 0;
+    if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) { s_nnz = 0; s_npix = 0; s_sq = 0.f; }
     pdl_wait();                                              // the projection (and its update bitmap) is the convolution's work
     __syncthreads();
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int ppc = (blockDim.x >> 5) / p.wpp;               // pixels per CTA
+    const int slot = (threadIdx.x >> 5) / p.wpp, sub = (threadIdx.x >> 5) % p.wpp;   // this warp's pixel of the CTA, and its share of the chunks
+    const int r = blockIdx.x * ppc + slot;
     const int tpix = p.n * p.th * p.tw;
     const int tx = r % p.tw, ty = (r / p.tw) % p.th, ns = r / (p.tw * p.th);
     const int st = KW > 1 ? p.pool_s : 1, pp = KW > 1 ? p.pool_p : 0;
@@ -705,7 +710,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
         const pt* P = reinterpret_cast<const pt*>(p.P);
         const bool vec = (p.c_out & 3) == 0;
         const int c_iter = (OT == T_BIN) ? p.cs * 32 : p.cs;
-        for (int c0 = 0; c0 < c_iter; c0 += 128) {
+        for (int c0 = sub * 128; c0 < c_iter; c0 += p.wpp * 128) {
             const int c = c0 + lane * 4;
             // the stored int8 activation word is fetched together with the projection, not after it
             uint32_t old_word = 0;
@@ -838,18 +843,18 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     #pragma unroll
     for (int o = 16; o > 0; o >>= 1) { cnt += __shfl_xor_sync(0xffffffffu, cnt, o); sq += __shfl_xor_sync(0xffffffffu, sq, o); }
     if (PT == T_F32 && lane == 0 && sq > 0.f) atomicAdd(&s_sq, sq);
-    if (lane == 0) s_cnt[threadIdx.x >> 5] = cnt;
-    if (cnt && lane == 0) {                                  // (cnt is uniform inside the warp)
+    if (cnt && lane == 0) atomicAdd(&s_cnt[slot], cnt);      // (cnt is uniform inside the warp) the pixel's warps add up
+    __syncthreads();
+    if (sub == 0 && lane == 0 && r < tpix && s_cnt[slot]) {
         atomicOr(&p.act[r >> 5], 1u << (r & 31));
-        p.pnnz[r] = cnt;
-        atomicAdd(&s_nnz, (unsigned)cnt);
+        p.pnnz[r] = s_cnt[slot];
+        atomicAdd(&s_nnz, (unsigned)s_cnt[slot]);
         atomicAdd(&s_npix, 1u);
     }
-    if (READERS) __syncthreads();
-    // the CTA's 8 consecutive pixels mark the reading layers' projection pixels together (lane = pixel)
+    // the CTA's consecutive pixels mark the reading layers' projection pixels together (lane = pixel)
     if (READERS && threadIdx.x < 32) {
-        const int rl = blockIdx.x * (blockDim.x >> 5) + lane;
-        const bool have = lane < (int)(blockDim.x >> 5) && rl < tpix;
+        const int rl = blockIdx.x * ppc + lane;
+        const bool have = lane < ppc && rl < tpix;
         unsigned long long macs[MAX_READERS];
         scatter_changed_warp(p.readers, have ? rl / (p.tw * p.th) : 0, have ? (rl / p.tw) % p.th : 0, have ? rl % p.tw : 1,
                              have ? s_cnt[lane] : 0, lane, macs);
@@ -1102,7 +1107,11 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     e.readers = dense ? Readers{} : out.readers;
     e.eps = net->eps; e.trunc = out.trunc;
     e.bn_scale = L.bn_scale; e.bn_shift = L.bn_shift;
-    const int blocks = ceil_div(out.pixels(), 8);
+    {
+        const int chunks = ceil_div(out.dtype == T_BIN ? out.cs * 32 : out.cs, 128);
+        e.wpp = chunks >= 8 ? 8 : (chunks > 2 ? 4 : (chunks > 1 ? 2 : 1));
+    }
+    const int blocks = ceil_div(out.pixels(), 8 / e.wpp);
     int es;
     if (proj_type(L) == T_F32) es = dense ? launch_epi<T_F32, true>(e, out.dtype, blocks, st) : launch_epi<T_F32, false>(e, out.dtype, blocks, st);
     else es = dense ? launch_epi<T_I32, true>(e, out.dtype, blocks, st) : launch_epi<T_I32, false>(e, out.dtype, blocks, st);

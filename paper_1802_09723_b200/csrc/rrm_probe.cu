@@ -8,7 +8,7 @@ namespace rrm {
 
 constexpr int PROBE_THREADS = 256;
 constexpr int PROBE_CHAINS = 8;               // independent dependency chains per thread
-constexpr int PROBE_ITERS = 4096;             // loop trips; each does PROBE_CHAINS x 4 operations per thread
+constexpr int PROBE_ITERS = 1024;             // loop trips; each does PROBE_CHAINS x 4 operations per thread
 
 // KIND 0: fp32 fused multiply-add; 1: dp4a (four int8 multiply-accumulates); 2: popc of a 32-bit word and an add
 // (32 one-bit multiply-accumulates, the inner operation of the binary convolution).
@@ -52,7 +52,7 @@ static int probe_run(double* ops_per_s)
     RRM_CUDA_TRY(cudaEventCreate(&e1));
     const int blocks = sms * 8;                               // 8 x 256 threads = every warp slot of an SM
     double best = 0.0;
-    for (int rep = 0; rep < 5; ++rep) {                       // the first repetitions also serve as warm-up
+    for (int rep = 0; rep < 4; ++rep) {                       // the first repetitions also serve as warm-up
         cudaEventRecord(e0);
         alu_probe_kernel<KIND><<<blocks, PROBE_THREADS>>>(17u + rep, sink);
         cudaEventRecord(e1);
