@@ -122,9 +122,12 @@ typedef struct {
                                     the thread block leave in an orderly way.  Default 2^20.  0 makes every such wait
                                     give up at once, before the thread block has anything in flight: a test hook */
     float layer_dense_activity;  /* stacks, variant AUTO: a layer whose measured share of projection pixels to update
-                                    reached this value (default 0.97) is evaluated densely in the following frames ... */
+                                    reached this value is evaluated densely in the following frames ...  Default
+                                    1.01, i.e. never: on the stacks measured so far the sparse product of a single
+                                    layer was never slower than its dense evaluation inside a delta step; lower it
+                                    (e.g. to 0.75) to turn the per-layer choice on */
     float layer_delta_activity;  /* ... and goes back to the sparse product once the share has fallen below this one
-                                    (default 0.90) */
+                                    (default 1.005) */
     float stack_dense_activity;  /* whole-stack switch (stacks of >= 1 GMAC per frame): MAC-weighted share from which on
                                     every layer of the next frames is evaluated densely */
     int32_t stack_reprobe;       /* dense frames in a row before one delta frame measures the activity again */

@@ -547,6 +547,7 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
     bool export_rec = false;
     int status = RRM_OK;
     RRM_CUDA_TRY(cudaStreamBeginCapture(origin, cudaStreamCaptureModeThreadLocal));
+    net->many_in_flight = true;
     auto fail = [&](int s) { if (status == RRM_OK) status = s; };
     auto wait = [&](cudaStream_t s, cudaEvent_t e) { if (cudaStreamWaitEvent(s, e, 0) != cudaSuccess) fail(RRM_ERR_CUDA); };
     auto record = [&](cudaEvent_t e, cudaStream_t s) { if (cudaEventRecord(e, s) != cudaSuccess) fail(RRM_ERR_CUDA); };
@@ -587,6 +588,7 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
     for (int k = 1; k < S; ++k) { record(net->ev_join[k], net->chunk_streams[k]); wait(origin, net->ev_join[k]); }
     cudaGraph_t g = nullptr;
     const cudaError_t e = cudaStreamEndCapture(origin, &g);
+    net->many_in_flight = false;
     if (status != RRM_OK || e != cudaSuccess || !g) {
         if (g) cudaGraphDestroy(g);
         cudaGetLastError();

@@ -206,6 +206,8 @@ struct rrm_net {
     void* frame_buf = nullptr;        // the step's input frame, boundary layout
     void* out_buf = nullptr;          // the step's last tensor, boundary layout
     bool graph_off = false;           // RRM_NO_GRAPH=1: launch kernel by kernel (debugging)
+    bool many_in_flight = false;      // set while a chunk graph is captured: its launches share the machine with those of
+                                      // neighbouring frames, so grids are sized for throughput instead of latency
     // where a captured sequence reads the frame and writes the output: the nodes (kernel arguments or a copy) that
     // hold frame_buf / out_buf are re-pointed at the caller's buffers before each launch, which saves the two
     // device-to-device copies around the graph; empty when the nodes could not be identified
@@ -258,10 +260,11 @@ struct rrm_net {
     int dense_streak = 0;                     // dense frames since the last measured delta frame
     bool last_step_dense = false;             // the most recent rrm_net_step was evaluated densely
     bool auto_switch = false;                 // every layer asks for RRM_VARIANT_AUTO and the net is large enough
-    // the defaults rrm_net_get_options reports.  (The per-layer thresholds sit this high because, measured on B200, a
-    // dense evaluation of one layer inside a delta step is never faster than its sparse product below ~95 % activity:
-    // what a delta step pays for is change detection and marking, which only a dense pass of the whole stack drops.)
-    rrm_options opt = {1u << 20, 0.97f, 0.90f, 0.75f, 15, 0.75f, 0.08f};
+    // the defaults rrm_net_get_options reports.  (The per-layer thresholds are above 1, i.e. the per-layer choice is off
+    // until the caller lowers them: measured on B200, a dense evaluation of one layer inside a delta step is never
+    // faster than its sparse product, not even with every pixel active.  What a delta step pays for is change
+    // detection and marking, which only a dense pass of the whole stack drops.)
+    rrm_options opt = {1u << 20, 1.01f, 1.005f, 0.75f, 15, 0.75f, 0.08f};
     float eps = 0.f;                  // Sec. 3.4: fp32 delta entries below it are truncated (0: exact)
     double* aecs = nullptr;           // [1 + layers]: accumulated truncated value e_t (Eq. 7), then the last step's l2 per layer
     std::vector<void*> allocs;        // everything to free

@@ -668,7 +668,8 @@ struct EpiParams {
 
 // PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.  KW: pool window edge (1 = no pool).
 // READERS: some layer reads the output tensor (a last layer's kernel leaves the marking code, and its registers, out).
-template <int PT, int OT, bool DENSE, int KW, bool READERS>
+// BN: f starts with the explicit per-channel affine (the kernels of layers without one are compiled without it).
+template <int PT, int OT, bool DENSE, int KW, bool READERS, bool BN>
 __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
 {
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
@@ -738,7 +739,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                 const bool live = c + j < p.c_out;
                 pt res = 0;
                 pt bn_m = 1, bn_a = 0;                       // the channel's affine (Sec. 4.5: BN as part of f)
-                if (live && p.bn_scale) {
+                if (BN && live) {
                     bn_m = reinterpret_cast<const pt*>(p.bn_scale)[c + j];
                     bn_a = reinterpret_cast<const pt*>(p.bn_shift)[c + j];
                 }
@@ -753,13 +754,13 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                     if (!(inside >> wi & 1u)) continue;
                     pt x = v[wi][j];
                     if (PT == T_F32) {
-                        if (p.bn_scale) x = (pt)fmaf((float)x, (float)bn_m, (float)bn_a);
+                        if (BN) x = (pt)fmaf((float)x, (float)bn_m, (float)bn_a);
                         x += res;
                         if (p.act_fn == RRM_ACT_RELU) x = x > 0 ? x : 0;
                         else if (p.act_fn == RRM_ACT_LEAKY) x = x > 0 ? x : (pt)(0.1f * (float)x);
                     } else if (OT == T_I8) {
                         int iv = (int)x;
-                        if (p.bn_scale) {                    // integer multiplier and offset inside the requantisation, 64-bit exact
+                        if (BN) {                            // integer multiplier and offset inside the requantisation, 64-bit exact
                             long long t = (long long)iv * (long long)(int)bn_m + (long long)(int)bn_a;
                             if (p.shift > 0) t = (t + (1ll << (p.shift - 1))) >> p.shift;
                             iv = (int)max(-127ll, min(127ll, t));
@@ -1033,17 +1034,25 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
     return RRM_OK;
 }
 
-template <int PT, int OT, bool DENSE>
-static int launch_epi_k(const EpiParams& e, int blocks, cudaStream_t st)
+template <int PT, int OT, bool DENSE, bool BN>
+static int launch_epi_kb(const EpiParams& e, int blocks, cudaStream_t st)
 {
     const bool rd = !DENSE && e.readers.n > 0;               // (a dense pass marks nothing)
     switch (e.pool_k > 0 ? e.pool_k : 1) {
-        case 1: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 1, !DENSE>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 1, false>, dim3(blocks), dim3(256), 0, st, e); break;
-        case 2: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 2, !DENSE>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 2, false>, dim3(blocks), dim3(256), 0, st, e); break;
-        case 3: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 3, !DENSE>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 3, false>, dim3(blocks), dim3(256), 0, st, e); break;
+        case 1: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 1, !DENSE, BN>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 1, false, BN>, dim3(blocks), dim3(256), 0, st, e); break;
+        case 2: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 2, !DENSE, BN>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 2, false, BN>, dim3(blocks), dim3(256), 0, st, e); break;
+        case 3: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 3, !DENSE, BN>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 3, false, BN>, dim3(blocks), dim3(256), 0, st, e); break;
         default: return RRM_ERR_UNSUPPORTED;                 // pool windows are 2x2 or 3x3
     }
     return RRM_OK;
+}
+
+template <int PT, int OT, bool DENSE>
+static int launch_epi_k(const EpiParams& e, int blocks, cudaStream_t st)
+{
+    // (the affine exists for fp32 outputs and for requantised int8 outputs only)
+    if ((OT == T_F32 || OT == T_I8) && e.bn_scale) return launch_epi_kb<PT, OT, DENSE, (OT == T_F32 || OT == T_I8)>(e, blocks, st);
+    return launch_epi_kb<PT, OT, DENSE, false>(e, blocks, st);
 }
 
 template <int PT, bool DENSE>
@@ -1109,7 +1118,9 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     e.bn_scale = L.bn_scale; e.bn_shift = L.bn_shift;
     {
         const int chunks = ceil_div(out.dtype == T_BIN ? out.cs * 32 : out.cs, 128);
-        e.wpp = chunks >= 8 ? 8 : (chunks > 2 ? 4 : (chunks > 1 ? 2 : 1));
+        // (several warps per pixel shorten a lone frame's step; inside a chunk graph, where launches of several frames
+        // overlap anyway, one warp per pixel does the same work with fewer CTAs)
+        e.wpp = net->many_in_flight ? 1 : (chunks >= 8 ? 8 : (chunks > 2 ? 4 : (chunks > 1 ? 2 : 1)));
     }
     const int blocks = ceil_div(out.pixels(), 8 / e.wpp);
     int es;

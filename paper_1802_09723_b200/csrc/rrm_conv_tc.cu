@@ -564,7 +564,9 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     // split K towards the point where a CTA's slabs all fit in its pipeline at once
     // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the
     // machine needs: once the tiles alone fill it, a tile owned by one CTA saves the adds of shared tiles
-    const int wave = 148;                                    // (measured: one CTA per SM is enough; more shares only add reductions)
+    // (measured: for one frame at a time one CTA per SM is enough, more shares only add reductions; inside a chunk
+    // graph, where the layers of several frames run side by side, half of that gives the best frames per second)
+    const int wave = net->many_in_flight ? 74 : 148;
     int ksplit = 1;
     const int ks_max = ceil_div(L.tc_slabs, TC_STAGES);
     const long long tiles = (long long)m_tiles * L.tc_ntiles;

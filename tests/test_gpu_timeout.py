@@ -24,7 +24,7 @@ def test_options_round_trip_and_validation():
     layer = rrm.layer_from_spec(wl.fc6_i8(c_in=256, c_out=128)[0])
     o = layer.options()
     assert o["wait_limit"] == 1 << 20 and abs(o["stack_dense_activity"] - 0.75) < 1e-6 and o["stack_reprobe"] == 15
-    assert abs(o["layer_dense_activity"] - 0.97) < 1e-6 and abs(o["layer_delta_activity"] - 0.90) < 1e-6
+    assert o["layer_dense_activity"] > 1.0 and o["layer_delta_activity"] > 1.0            # the per-layer choice is opt-in
     layer.set_options(wait_limit=123, fc_dense_rows=0.5)
     o2 = layer.options()
     assert o2["wait_limit"] == 123 and abs(o2["fc_dense_rows"] - 0.5) < 1e-6 and o2["stack_reprobe"] == 15
