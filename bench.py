@@ -494,6 +494,8 @@ def main():
                     help="cfg2 (default) is the contract line; the others are the convolution configurations")
     ap.add_argument("--variant", default="auto", choices=["auto", "gather", "tensor", "dense", "sparse_w"],
                     help="rrm_layer_desc.variant of the timed object (default: the library chooses)")
+    ap.add_argument("--pruned", type=float, default=None, help="contract workload on a magnitude-pruned matrix (fraction of weights kept); "
+                                                               "for profiling the weight-sparse form: --pruned 0.1 --variant sparse_w")
     ap.add_argument("--frames", type=int, default=None, help="frames of the synthetic video (convolution workloads)")
     ap.add_argument("--streams", type=int, default=None, help="independent videos per call (convolution workloads)")
     ap.add_argument("--opt", action="append", help="rrm_options field=value (convolution workloads), e.g. --opt layer_dense_activity=0.9")
@@ -524,7 +526,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     rrm.lib()
-    spec = wl.fc6_i8()[0]
+    spec = wl.fc6_i8_pruned(keep=args.pruned)[0] if args.pruned else wl.fc6_i8()[0]
     W = torch.from_numpy(spec.weight).cuda()
     B = torch.from_numpy(spec.bias).cuda()
     order = pingpong(FRAMES)
@@ -748,7 +750,7 @@ def main():
         kept = float(np.mean(pr.weight != 0))
         groups = float(np.mean(np.any(pr.weight.reshape(C_OUT // 4, 4, C_IN) != 0, axis=1)))   # non-zero groups of four outputs
         sw = {"weights_kept": kept, "nonzero_groups_of_4": groups,
-              "bytes_per_gathered_column": {"dense": C_OUT, "weight_sparse": groups * C_OUT + 16 * (C_OUT // 512)}}
+              "bytes_per_gathered_column": {"dense": C_OUT, "weight_sparse": groups * C_OUT + 32 * (C_OUT // 512)}}
         for rho in RHOS:
             row = {}
             for nm, var in (("weight_sparse", "sparse_w"), ("column_gather", "gather"), ("library_auto", "auto")):

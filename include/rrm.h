@@ -73,8 +73,8 @@ enum { RRM_ACT_NONE = 0, RRM_ACT_RELU = 1, RRM_ACT_SIGN = 2,
 enum { RRM_VARIANT_AUTO = 0, RRM_VARIANT_GATHER = 1, RRM_VARIANT_TENSOR = 2, RRM_VARIANT_DENSE = 3,
        RRM_VARIANT_SPARSE_W = 4 /* lone int8 FC layer: weight-sparse x delta-sparse product (Sec. 3.5 / 4.3: the
                                    compressed models EIE runs).  The zero weights of W (a pruned model) are dropped
-                                   at create time: every (input, 512-output slice) keeps a 128-bit map of its
-                                   non-zero groups of four outputs and only those groups' bytes, so a non-zero
+                                   at create time: every (input, 512-output slice) keeps a 32-byte header (a 128-bit
+                                   map of its non-zero groups of four outputs) and only those groups' bytes, so a non-zero
                                    delta entry gathers a fraction of its column.  Results are the same integers */ };
 
 /*

@@ -150,7 +150,7 @@ struct Layer {
     void* fc_scratch = nullptr;             // per-stream non-zero lists of the two-kernel form
     unsigned long long* fc_nnz = nullptr;   // [0] nnz elements, [1] active groups of 32 (cleared by the kernel's last CTA)
     // weight-sparse form (RRM_VARIANT_SPARSE_W): per (input, 512-output slice) a record of sp_stride words:
-    // 4 words = map of the non-zero groups of four outputs, then those groups' weights, packed
+    // 8 words of header (map of the non-zero groups of four outputs, running counts), then those groups' weights, packed
     uint32_t* Wsp = nullptr;
     int sp_stride = 0;
     long long sp_words = 0;                 // packed weight words of the whole matrix (for reporting)

@@ -29,6 +29,7 @@ constexpr int SQ_WARPS = SQ_THREADS / 32;
 constexpr int SQ_TAIL = 16;                    // frames one thread of the closing sum holds (chunks of up to 2 * SQ_TAIL frames)
 constexpr int SQ_PT = 4;                       // 16-byte chunks scanned per thread
 constexpr int SQ_MAX_C_IN = 16 * SQ_PT * SQ_THREADS;   // 16384 (entry format: 14-bit index)
+constexpr int SW_RING = 12;                    // weight-sparse form: records in flight per warp
 
 struct FcSeqParams {
     const int8_t* x;         // [T][n][c_in] frames of the chunk
@@ -54,8 +55,8 @@ struct FcSeqParams {
 // grid is resident at once (each CTA's chain of round trips is what the launch waits for).
 // SW (LANES = 32 only): the weights are in the weight-sparse form (Sec. 3.5: EIE keeps the pruned weights of a
 // compressed model in compressed columns).  A lane owns 16 outputs = 4 groups of four; the record of (input j, this
-// slice) starts with a 128-bit map (bit 4 * lane + g: group g of that lane holds a non-zero weight) followed by the
-// 4-byte words of the non-zero groups, in map order.  All lanes load the map (one 16-byte broadcast), find their
+// slice) starts with a 128-bit map (bit 4 * lane + g: group g of that lane holds a non-zero weight) and the running
+// word counts of the map's four words, followed (from byte 32 on) by the 4-byte words of the non-zero groups, in map order.  All lanes load the map (one 16-byte broadcast), find their
 // word offset by counting the map bits below their own, and load only their non-zero groups.
 template <int LANES, bool DEEP, bool SW>
 __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqParams p)
@@ -169,58 +170,74 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
     #pragma unroll
     for (int i = 0; i < 16; ++i) acc[i] = 0;
     if (SW) {
-        constexpr int SW_U = DEEP ? 8 : 4;                   // entries in flight per warp (one column slice per warp-wide step)
+        // Every warp streams the records of its list entries (entry warp, warp + 8, ...) through a ring of SW_RING slots
+        // in shared memory with 16-byte asynchronous copies: one memory round trip per record, SW_RING records in flight.
+        // A whole record (fixed stride: the longest record of the matrix) is fetched, map and packed groups together.
+        const int stride_b = p.sp_stride * 4, pieces = stride_b >> 4;
+        unsigned char* ringbuf = s_dyn + (size_t)SQ_WARPS * OW * 4 + (size_t)C * 4 + (size_t)warp * SW_RING * stride_b;
+        const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(ringbuf);
         const int nib_shift = 4 * (lane & 7), nib_word = lane >> 3;
-        for (int e = warp; e < total; e += SW_U * SQ_WARPS) {
-            uint32_t ent[SW_U];
-            uint4 map[SW_U];
+        const int mine_n = total > warp ? (total - warp + SQ_WARPS - 1) / SQ_WARPS : 0;
+        auto issue = [&](int i) {
+            if (i < mine_n) {
+                const uint32_t ent = s_list[warp + i * SQ_WARPS];
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(p.Wsp + ((size_t)(ent & 0xffffu) * slices + slice) * p.sp_stride);
+                for (int pc = lane; pc < pieces; pc += 32)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_u32 + (uint32_t)((i % SW_RING) * stride_b + pc * 16)), "l"(src + pc * 16) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        for (int i = 0; i < SW_RING - 2; ++i) issue(i);
+        // two records per turn: their decode chains (map -> offsets -> words -> products) overlap
+        for (int i = 0; i < mine_n; i += 2) {
+            issue(i + SW_RING - 2);                          // (refill the two slots read in the previous turn: every lane is past them)
+            issue(i + SW_RING - 1);
+            asm volatile("cp.async.wait_group %0;" ::"n"(SW_RING - 2) : "memory");
+            __syncwarp();                                    // the pieces the other lanes copied are visible too
+            uint32_t wg[2][4];
+            int dl[2], dh[2];
             #pragma unroll
-            for (int u = 0; u < SW_U; ++u) {
-                const int eu = e + u * SQ_WARPS;
-                ent[u] = eu < total ? s_list[eu] : 0xffffffffu;
+            for (int r = 0; r < 2; ++r) {
+                const bool have = i + r < mine_n;            // (an odd tail: the second record is absent, all its words zero)
+                const unsigned char* slot = ringbuf + ((i + r) % SW_RING) * stride_b;
+                const uint4 map = have ? *reinterpret_cast<const uint4*>(slot) : make_uint4(0, 0, 0, 0);
+                const uint32_t mine = nib_word == 0 ? map.x : (nib_word == 1 ? map.y : (nib_word == 2 ? map.z : map.w));
+                const unsigned nib = (mine >> nib_shift) & 0xfu;
+                // branch-free: a lane reads its (up to four) groups with predicated loads, absent groups are zero words
+                // (the record carries the running counts of its map words, and the offsets inside a nibble are sums of
+                // bits: one population count per record and lane - that pipe is the narrow one)
+                const uint32_t cum = have ? reinterpret_cast<const uint32_t*>(slot)[4] : 0u;
+                const int before = __popc(mine & ((1u << nib_shift) - 1u)) + (nib_word == 0 ? 0 : (int)((cum >> (8 * (nib_word - 1))) & 0xffu));
+                const uint32_t* words = reinterpret_cast<const uint32_t*>(slot) + 8 + before;
+                const unsigned b0 = nib & 1u, b01 = b0 + ((nib >> 1) & 1u), b012 = b01 + ((nib >> 2) & 1u);
+                wg[r][0] = (nib & 1u) ? words[0] : 0u;
+                wg[r][1] = (nib & 2u) ? words[b0] : 0u;
+                wg[r][2] = (nib & 4u) ? words[b01] : 0u;
+                wg[r][3] = (nib & 8u) ? words[b012] : 0u;
+                const uint32_t ent = have ? s_list[warp + (i + r) * SQ_WARPS] : (256u << 16);
+                const int d = (int)(ent >> 16) - 256;        // (the same for every lane: the branch below is uniform)
+                dh[r] = (d >= -128 && d <= 127) ? 0 : d / 2;
+                dl[r] = d - dh[r];
             }
             #pragma unroll
-            for (int u = 0; u < SW_U; ++u)
-                map[u] = ent[u] != 0xffffffffu
-                             ? __ldg(reinterpret_cast<const uint4*>(p.Wsp + ((size_t)(ent[u] & 0xffffu) * slices + slice) * p.sp_stride))
-                             : make_uint4(0, 0, 0, 0);
-            uint32_t wv[SW_U][4];
-            unsigned nib[SW_U];
-            #pragma unroll
-            for (int u = 0; u < SW_U; ++u) {
-                const uint32_t m0 = map[u].x, m1 = map[u].y, m2 = map[u].z, m3 = map[u].w;
-                const uint32_t mine = nib_word == 0 ? m0 : (nib_word == 1 ? m1 : (nib_word == 2 ? m2 : m3));
-                nib[u] = (mine >> nib_shift) & 0xfu;
-                // words of the lanes before this one
-                int before = __popc(mine & ((1u << nib_shift) - 1u));
-                if (nib_word > 0) before += __popc(m0);
-                if (nib_word > 1) before += __popc(m1);
-                if (nib_word > 2) before += __popc(m2);
-                const uint32_t* words = p.Wsp + ((size_t)(ent[u] & 0xffffu) * slices + slice) * p.sp_stride + 4 + before;
+            for (int r = 0; r < 2; ++r) {
                 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    wv[u][g] = 0;
-                    if (nib[u] >> g & 1u) wv[u][g] = __ldg(words + __popc(nib[u] & ((1u << g) - 1u)));
-                }
-            }
-            #pragma unroll
-            for (int u = 0; u < SW_U; ++u) {
-                if (nib[u] == 0) continue;
-                const int d = (int)(ent[u] >> 16) - 256;
-                const int dh = (d >= -128 && d <= 127) ? 0 : d / 2;
-                const int dl = d - dh;
-                const unsigned lb = (unsigned)dl & 0xffu, hb = (unsigned)dh & 0xffu;
-                #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    if (!(nib[u] >> g & 1u)) continue;
+                for (int half = 0; half < 2; ++half) {
+                    if (half == 1 && dh[r] == 0) break;
+                    const unsigned sel = (unsigned)(half ? dh[r] : dl[r]) & 0xffu;
+                    const int s0 = (int)sel, s1 = (int)(sel << 8), s2 = (int)(sel << 16), s3 = (int)(sel << 24);
                     #pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        acc[g * 4 + b] = __dp4a((int)wv[u][g], (int)(lb << (8 * b)), acc[g * 4 + b]);
-                        if (dh != 0) acc[g * 4 + b] = __dp4a((int)wv[u][g], (int)(hb << (8 * b)), acc[g * 4 + b]);
+                    for (int g = 0; g < 4; ++g) {
+                        acc[g * 4 + 0] = __dp4a((int)wg[r][g], s0, acc[g * 4 + 0]);
+                        acc[g * 4 + 1] = __dp4a((int)wg[r][g], s1, acc[g * 4 + 1]);
+                        acc[g * 4 + 2] = __dp4a((int)wg[r][g], s2, acc[g * 4 + 2]);
+                        acc[g * 4 + 3] = __dp4a((int)wg[r][g], s3, acc[g * 4 + 3]);
                     }
                 }
             }
+            __syncwarp();
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (o0 < K) {                                     // K is a multiple of 16
         const int8_t* wbase = p.Wt + o0;
         for (int e = grp; e < total; e += SQ_U * CPR) {
@@ -388,7 +405,11 @@ static int seq_read_back(Layer& L, int rows, cudaStream_t st)
 
 int fc_dense_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bool stateless, cudaStream_t st);
 
-static size_t seq_dyn_smem(int c_in, int lanes) { return (size_t)SQ_WARPS * 16 * lanes * 4 + (size_t)c_in * 4; }
+// (sp_stride > 0: the weight-sparse form adds every warp's ring of records)
+static size_t seq_dyn_smem(int c_in, int lanes, int sp_stride = 0)
+{
+    return (size_t)SQ_WARPS * 16 * lanes * 4 + (size_t)c_in * 4 + (size_t)SQ_WARPS * SW_RING * sp_stride * 4;
+}
 
 static int seq_ensure(rrm_net* net, Layer& L, int T)
 {
@@ -432,10 +453,11 @@ int fc_seq_create(rrm_net* net, Layer& L)
                                       (int)seq_dyn_smem(SQ_MAX_C_IN, 16)));
     RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<8, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)seq_dyn_smem(SQ_MAX_C_IN, 8)));
+    // (weight-sparse form: up to 136 words per record, the stride of a matrix without zeros)
     RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32, 136)));
     RRM_CUDA_TRY(cudaFuncSetAttribute(fc_seq_kernel<32, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32)));
+                                      (int)seq_dyn_smem(SQ_MAX_C_IN, 32, 136)));
     return seq_ensure(net, L, 1);
 }
 
@@ -522,7 +544,7 @@ int fc_seq_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int T, bo
         p.stat = dense ? nullptr : L.seq_stat + (size_t)t0 * n * 2;
         p.T = piece;
         dim3 grid(ceil_div(K, 16 * lanes), piece * n);
-        const size_t dyn = seq_dyn_smem(C, lanes);
+        const size_t dyn = seq_dyn_smem(C, lanes, L.Wsp ? L.sp_stride : 0);
         if (L.Wsp && grid.x * grid.y <= 2 * 148) fc_seq_kernel<32, true, true><<<grid, SQ_THREADS, dyn, st>>>(p);
         else if (L.Wsp) fc_seq_kernel<32, false, true><<<grid, SQ_THREADS, dyn, st>>>(p);
         else if (lanes == 32 && grid.x * grid.y <= 2 * 148) fc_seq_kernel<32, true, false><<<grid, SQ_THREADS, dyn, st>>>(p);
@@ -617,7 +639,10 @@ __global__ void __launch_bounds__(256) fc_sparse_w_pack_kernel(const int8_t* __r
     m |= __shfl_xor_sync(0xffffffffu, m, 2);
     m |= __shfl_xor_sync(0xffffffffu, m, 4);
     if ((lane & 7) == 0) out[lane >> 3] = m;
-    int at = 4 + incl - cnt;
+    // word 4: the number of packed words before map word 1, 2 and 3 (one byte each); words 5-7 unused
+    const int c0 = __shfl_sync(0xffffffffu, incl, 7), c1 = __shfl_sync(0xffffffffu, incl, 15), c2 = __shfl_sync(0xffffffffu, incl, 23);
+    if (lane == 0) out[4] = (uint32_t)c0 | (uint32_t)c1 << 8 | (uint32_t)c2 << 16;
+    int at = 8 + incl - cnt;
     #pragma unroll
     for (int g = 0; g < 4; ++g) if (nib >> g & 1u) out[at++] = ww[g];
 }
@@ -636,7 +661,7 @@ int fc_sparse_w_create(rrm_net* net, Layer& L)
     const cudaError_t e = cudaMemcpy(h, d_max, 16, cudaMemcpyDeviceToHost);
     cudaFree(d_max);
     if (e != cudaSuccess) { cudaGetLastError(); return RRM_ERR_CUDA; }
-    L.sp_stride = 4 + round_up(h[0] > 0 ? h[0] : 1, 4);      // 16-byte aligned records
+    L.sp_stride = 8 + round_up(h[0] > 0 ? h[0] : 1, 4);      // 32-byte header, 16-byte aligned records
     std::memcpy(&L.sp_words, &h[2], 8);
     void* rec = nullptr;
     if (cudaMalloc(&rec, (size_t)records * L.sp_stride * 4) != cudaSuccess) { cudaGetLastError(); return RRM_ERR_ALLOC; }
@@ -648,7 +673,7 @@ int fc_sparse_w_create(rrm_net* net, Layer& L)
     L.Wsp = reinterpret_cast<uint32_t*>(rec);
     if (getenv("RRM_DEBUG"))
         fprintf(stderr, "rrm: weight-sparse FC: %lld records of %d words, %lld packed weight words (%.1f %% of the dense bytes incl. maps)\n",
-                records, L.sp_stride, L.sp_words, 100.0 * (L.sp_words * 4.0 + records * 16.0) / ((double)C * K));
+                records, L.sp_stride, L.sp_words, 100.0 * (L.sp_words * 4.0 + records * 32.0) / ((double)C * K));
     return RRM_OK;
 }
 
