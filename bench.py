@@ -742,6 +742,82 @@ def main():
                             "frac_distinct_cold_bytes = bytes the launch must fetch from HBM / time / measured HBM peak; "
                             "served_gbs = all gathered bytes (repeats served by L2) per second: a rate, not an HBM fraction")
 
+    # ---- the same delta-FC kernels on a layer large enough to be bound by bytes: 16384 -> 16384 int8 (268 MB of
+    # weights, twice the L2: gathered columns come from HBM whatever ran before), one frame per call (rrm_step) and a
+    # chunk of 8 frames, the column gather forced.  fc6's 37.7 MB take 5.8 us at the HBM peak, less than the fixed cost
+    # of a launch, which is why its fractions stay low; this row shows what the kernels reach once the bytes dominate.
+    if not args.quick and rank == 0 and world == 1:
+        try:
+            CB, KB = 16384, 16384
+            big = wl.fc6_i8(seed=7, c_in=CB, c_out=KB)[0]
+            Wb = torch.from_numpy(big.weight).cuda()
+            Bb = torch.from_numpy(big.bias).cuda()
+            rows = {}
+            for rho in (0.05, 0.20):
+                Lb = rrm.Net([rrm.desc_from_spec(big, n=1, variant="gather")], [Wb], [Bb])
+                sq = wl.fc_run_sequence(frames=9, c_in=CB, rho=rho, seed=77)
+                fr = [torch.from_numpy(sq[t]).cuda() for t in range(9)]
+                ordb = pingpong(9)
+                Yb = Lb.new_output()
+                Lb.keyframe(fr[0], Yb)
+                for i in range(4):
+                    Lb.step(fr[ordb[(i + 1) % len(ordb)]], Yb)
+                torch.cuda.synchronize()
+                evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(24)]
+                for i in range(24):
+                    flush.fill_(i & 0xff)
+                    evs[i][0].record(stream)
+                    Lb.step(fr[ordb[(5 + i) % len(ordb)]], Yb)
+                    evs[i][1].record(stream)
+                torch.cuda.synchronize()
+                us = summarize([a.elapsed_time(b) for a, b in evs])["median"] * 1e3
+                nnz = float(np.mean([np.count_nonzero(sq[ordb[(k + 1) % len(ordb)]] != sq[ordb[k % len(ordb)]]) for k in range(len(ordb))]))
+                nbytes = nnz * KB + 12 * KB + 3 * CB
+                rows[f"{rho:g}"] = {"kernel": "fc_delta_i8_kernel", "frames_per_launch": 1, "nnz_mean_per_frame": nnz,
+                                    "us_per_launch": us, "algorithmic_bytes_per_launch": nbytes,
+                                    "achieved_gbs": nbytes / (us * 1e-6) / 1e9, "frac": nbytes / (us * 1e-6) / 1e9 / peak}
+                # chunks of Tb frames per launch (fc_seq_kernel): distinct columns of the chunk once from HBM, repeats from L2
+                for Tb in (4, 8):
+                    walkb = np.stack([sq[ordb[(i + 1) % len(ordb)]] for i in range(len(ordb) * Tb)])
+                    wdb = torch.from_numpy(walkb).cuda()
+                    ncb = wdb.shape[0] // Tb
+                    Ycb = Lb.new_output(frames=Tb)
+                    Lb.keyframe(fr[0], Yb)
+                    for i in range(3):
+                        Lb.step_seq(wdb[(i % ncb) * Tb:(i % ncb + 1) * Tb], Ycb, Tb)
+                    torch.cuda.synchronize()
+                    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(16)]
+                    for i in range(16):
+                        k = (3 + i) % ncb
+                        flush.fill_(i & 0xff)
+                        evs[i][0].record(stream)
+                        Lb.step_seq(wdb[k * Tb:(k + 1) * Tb], Ycb, Tb)
+                        evs[i][1].record(stream)
+                    torch.cuda.synchronize()
+                    usc = summarize([a.elapsed_time(b) for a, b in evs])["median"] * 1e3
+                    uniq = []
+                    for k in range(ncb):
+                        touched = np.zeros(CB, dtype=bool)
+                        for i in range(k * Tb, (k + 1) * Tb):
+                            prev = walkb[i - 1] if i else sq[ordb[0]]
+                            touched |= (walkb[i] != prev).reshape(-1)
+                        uniq.append(int(touched.sum()))
+                    db = float(np.mean(uniq)) * KB + Tb * (12 * KB + CB) + 2 * CB
+                    rows[f"{rho:g}_chunk{Tb}"] = {"kernel": "fc_seq_kernel", "frames_per_launch": Tb, "us_per_launch": usc,
+                                                  "distinct_cold_bytes": db, "per_frame_bytes_x_frames": Tb * nbytes,
+                                                  "frac_distinct_cold_bytes": db / (usc * 1e-6) / 1e9 / peak,
+                                                  "served_gbs_l2_and_hbm": Tb * nbytes / (usc * 1e-6) / 1e9}
+                    del wdb
+                Lb.close()
+            rows["note"] = (f"int8 FC {CB}->{KB} (268 MB of weights, larger than L2), one stream, column gather forced, cold L2, "
+                            f"medians; one frame per rrm_step call (bytes = gathered columns + projection + frames, all from HBM) "
+                            f"and chunks of 4 / 8 frames per rrm_step_seq call (distinct columns once from HBM)")
+            extra["roofline_delta_fc_large_layer"] = rows
+            del Wb, Bb
+            torch.cuda.empty_cache()
+        except Exception as e:  # noqa: BLE001
+            extra["roofline_delta_fc_large_layer"] = {"error": str(e)}
+
     # ---- weight-sparse x delta-sparse (Sec. 3.5 / 4.3): fc6 magnitude-pruned to 10 %, the weight-sparse form against
     # the column gather and the dense tensor-core pass on the same pruned matrix
     if not args.quick:
