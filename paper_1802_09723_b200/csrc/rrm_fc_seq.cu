@@ -239,23 +239,36 @@ __global__ void __launch_bounds__(SQ_THREADS, DEEP ? 2 : 3) fc_seq_kernel(FcSeqP
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (o0 < K) {                                     // K is a multiple of 16
+        // Two half-batches in flight alternately: while one half's columns are multiplied, the other half's loads
+        // are already on their way (the memory system is never left idle behind the arithmetic).
+        constexpr int HB = SQ_U / 2;                         // columns per half-batch and lane
         const int8_t* wbase = p.Wt + o0;
-        for (int e = grp; e < total; e += SQ_U * CPR) {
-            uint32_t ent[SQ_U];
-            uint4 w[SQ_U];
+        uint32_t entA[HB], entB[HB];
+        uint4 wA[HB], wB[HB];
+        auto fetch = [&](int e, uint32_t (&ent)[HB], uint4 (&w)[HB]) {
             #pragma unroll
-            for (int u = 0; u < SQ_U; ++u) {
+            for (int u = 0; u < HB; ++u) {
                 const int eu = e + u * CPR;
                 ent[u] = eu < total ? s_list[eu] : 0xffffffffu;
             }
             #pragma unroll
-            for (int u = 0; u < SQ_U; ++u)
+            for (int u = 0; u < HB; ++u)
                 w[u] = ent[u] != 0xffffffffu
                            ? __ldg(reinterpret_cast<const uint4*>(wbase + (size_t)(ent[u] & 0xffffu) * K))
                            : make_uint4(0, 0, 0, 0);
+        };
+        auto consume = [&](const uint32_t (&ent)[HB], const uint4 (&w)[HB]) {
             #pragma unroll
-            for (int u = 0; u < SQ_U; ++u)
+            for (int u = 0; u < HB; ++u)
                 if (ent[u] != 0xffffffffu) fma16(acc, w[u], (int)(ent[u] >> 16) - 256);
+        };
+        constexpr int STEP = HB * CPR;                       // list entries one half-batch of the CTA covers
+        fetch(grp, entA, wA);
+        for (int e = grp; e < total; e += 2 * STEP) {
+            fetch(e + STEP, entB, wB);
+            consume(entA, wA);
+            fetch(e + 2 * STEP, entA, wA);
+            consume(entB, wB);
         }
     }
     // ---- 3. add the partial sums: the column groups of a warp by shuffles, the warps through shared memory
