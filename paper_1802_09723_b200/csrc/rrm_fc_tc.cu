@@ -15,7 +15,6 @@
 // Every mbarrier wait is bounded; a wait that runs out sets ERRW_TIMEOUT and the CTA still takes part
 // in the arrival protocol and frees its tensor memory.
 #include <cuda.h>
-#include <cstddef>
 #include "rrm_common.cuh"
 #include "rrm_tc.cuh"
 #include "rrm_dev.cuh"
@@ -35,10 +34,7 @@ struct FtSmemTail {
     uint32_t tmem_base;
     int last;
     int cnt_nnz, cnt_grp;     // per-row counters of the delta scan
-    __align__(16) int bias[TC_M];   // the bias of this CTA's output block, fetched while W streams (read four at a time)
 };
-
-static_assert(offsetof(FtSmemTail, bias) % 16 == 0, "the bias is read with 16-byte shared-memory loads");
 
 struct FtParams {
     const int8_t* Wimg;       // [m_tiles][slabs][128 x 128] swizzled tile images
@@ -57,10 +53,9 @@ struct FtParams {
     unsigned wait_limit;      // polls of one bounded wait
 };
 
-// (bias: the output block's bias in shared memory, indexed by the output's position inside the block)
-__device__ __forceinline__ void ft_finish(const FtParams& p, const int* bias, int row, int o, int v)
+__device__ __forceinline__ void ft_finish(const FtParams& p, int row, int o, int v)
 {
-    v += bias[o & (TC_M - 1)];
+    if (p.bias) v += p.bias[o];
     const size_t i = (size_t)row * p.c_out + o;
     if (p.Pstate && row >= p.state_from) p.Pstate[i - (size_t)p.state_from * p.c_out] = v;
     if (p.Y) {
@@ -70,9 +65,9 @@ __device__ __forceinline__ void ft_finish(const FtParams& p, const int* bias, in
 }
 
 // four consecutive outputs of one row: bias, stored projection, output through f
-__device__ __forceinline__ void ft_finish4(const FtParams& p, const int* bias, int row, int oo, int4 w)
+__device__ __forceinline__ void ft_finish4(const FtParams& p, int row, int oo, int4 w)
 {
-    { const int4 b = *reinterpret_cast<const int4*>(bias + (oo & (TC_M - 1))); w.x += b.x; w.y += b.y; w.z += b.z; w.w += b.w; }
+    if (p.bias) { const int4 b = *reinterpret_cast<const int4*>(p.bias + oo); w.x += b.x; w.y += b.y; w.z += b.z; w.w += b.w; }
     const size_t at = (size_t)row * p.c_out + oo;
     if (p.Pstate && row >= p.state_from) *reinterpret_cast<int4*>(p.Pstate + at - (size_t)p.state_from * p.c_out) = w;
     if (p.Y) {
@@ -101,21 +96,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     const uint32_t stage_bytes = FT_A_BYTES + b_bytes;
     FtSmemTail* S = reinterpret_cast<FtSmemTail*>(base + (size_t)p.stages * stage_bytes);
 
-    bool ok = true;
-    int n_loaded = 0;                                        // loader: stages issued
-    // one slab into its ring stage: a 16 KB bulk copy of W and a tensor copy of the input rows (loader thread only)
-    auto load_slab = [&](int it) {
-        const int stage = it % p.stages;
-        const uint32_t bar = smem_u32(&S->full[stage]);
-        const uint32_t dst = base_u32 + (uint32_t)stage * stage_bytes;
-        mbar_arrive_expect_tx(bar, stage_bytes);
-        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                     ::"r"(dst + FT_A_BYTES), "l"(&tmapX), "r"((s_begin + it) * FT_SLAB), "r"(0), "r"(bar) : "memory");
-        bulk_copy_g2s(dst, p.Wimg + ((size_t)mtile * p.slabs + s_begin + it) * FT_A_BYTES, FT_A_BYTES, bar);
-    };
-    if (tid == 5 * 32) {
-        // the loader thread sets the barriers up itself and fills the whole ring at once (a fresh stage needs no
-        // wait): W is on its way while the other warps allocate tensor memory and fetch the bias
+    if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&S->full[s]), 1);            // the loader's expect_tx
             mbar_init(smem_u32(&S->empty[s]), 1);           // one tcgen05.commit
@@ -123,12 +104,6 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
         mbar_init(smem_u32(&S->done), 1);
         S->last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (p.wait_limit > 0)                               // (limit 0: the test hook, every wait gives up, nothing is issued)
-            for (; n_loaded < mine && n_loaded < p.stages; ++n_loaded) load_slab(n_loaded);
-    }
-    if (tid < TC_M) {
-        const int o = mtile * TC_M + tid;
-        S->bias[tid] = (p.bias && o < p.c_out) ? p.bias[o] : 0;
     }
     if (warp == 4) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -139,6 +114,8 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S->tmem_base;
+    bool ok = true;
+    int n_loaded = 0;                                        // loader: stages issued
 
     if (warp < 4) {
         // ================= the CTAs of the first output block refresh the input snapshot (their K share of the state rows)
@@ -182,10 +159,16 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
     } else if (warp == 5) {
         // ================= loader: per slab one 16 KB bulk copy of W and one tensor copy of the input rows
         if (lane == 0) {
-            for (int it = n_loaded; it < mine; ++it) {       // (the first ring-full of slabs went out before the set-up barrier)
+            const int8_t* src = p.Wimg + ((size_t)mtile * p.slabs + s_begin) * FT_A_BYTES;
+            for (int it = 0; it < mine; ++it) {
                 const int stage = it % p.stages;
                 if (!mbar_wait(smem_u32(&S->empty[stage]), ((it / p.stages) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
-                load_slab(it);
+                const uint32_t bar = smem_u32(&S->full[stage]);
+                const uint32_t dst = base_u32 + (uint32_t)stage * stage_bytes;
+                mbar_arrive_expect_tx(bar, stage_bytes);
+                asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                             ::"r"(dst + FT_A_BYTES), "l"(&tmapX), "r"((s_begin + it) * FT_SLAB), "r"(0), "r"(bar) : "memory");
+                bulk_copy_g2s(dst, src + (size_t)it * FT_A_BYTES, FT_A_BYTES, bar);
                 n_loaded = it + 1;
             }
         }
@@ -246,7 +229,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
                 for (int j = 0; j < 32; ++j) {
                     const int row = c0 + j;
                     if (row >= p.rows) break;
-                    if (p.ksplit == 1) { if (o < p.c_out) ft_finish(p, S->bias, row, o, (int)v[j]); }
+                    if (p.ksplit == 1) { if (o < p.c_out) ft_finish(p, row, o, (int)v[j]); }
                     else if (CLUSTER) red[row * TC_M + (warp & 3) * 32 + lane] = (int)v[j];
                     else atomicAdd(p.acc + (size_t)row * (gridDim.x * TC_M) + o, (int)v[j]);
                 }
@@ -284,7 +267,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
                 w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
             }
             const int oo = mtile * TC_M + o4;
-            if (oo < p.c_out) ft_finish4(p, S->bias, row, oo, w);
+            if (oo < p.c_out) ft_finish4(p, row, oo, w);
         }
         // nobody leaves while its shared memory may still be read
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -315,7 +298,7 @@ __global__ void __launch_bounds__(FT_THREADS, 1) fc_tc_kernel(FtParams p, const 
             if (i >= total4) continue;
             const int row = i / (TC_M / 4), oo = mtile * TC_M + (i % (TC_M / 4)) * 4;
             *reinterpret_cast<int4*>(p.acc + (size_t)row * ld + oo) = make_int4(0, 0, 0, 0);
-            if (oo < p.c_out) ft_finish4(p, S->bias, row, oo, v[u]);
+            if (oo < p.c_out) ft_finish4(p, row, oo, v[u]);
         }
     }
     if (tid == 0) p.arrive[mtile] = 0;
