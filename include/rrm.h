@@ -28,7 +28,10 @@
  *     kernel of a stack step on its own instead of replaying a captured CUDA graph; RRM_DEBUG=1 names a failing
  *     CUDA call (file, line, error string) on stderr and prints the shape of captured chunk graphs; RRM_PDL=1
  *     launches the kernels of a stack step with programmatic dependent launch (each kernel's set-up overlaps its
- *     predecessor's tail; off by default: measured, it does not pay inside replayed graphs).
+ *     predecessor's tail; off by default: measured, it does not pay inside replayed graphs); RRM_CHUNK_INPLACE=1
+ *     makes the delta chunks of a stack (rrm_net_step_seq) add each frame's product straight onto the stored
+ *     projection, as single steps do, instead of keeping it in a per-frame buffer that the epilogue merges (the
+ *     default, which lets the convolution of frame t+1 run beside the epilogue of frame t; same results).
  */
 #ifndef RRM_H
 #define RRM_H

@@ -77,7 +77,7 @@ void bind_arena(rrm_net* net, char* base)
 {
     size_t off = 0;
     for (auto& T : net->tensors) { T.act = reinterpret_cast<uint32_t*>(base + off); off += (size_t)T.act_words() * 4; }
-    for (auto& L : net->layers) { L.oact = reinterpret_cast<uint32_t*>(base + off); off += (size_t)ceil_div(L.opixels(), 32) * 4; }
+    for (auto& L : net->layers) { L.oact = reinterpret_cast<uint32_t*>(base + off); L.oact_off = off; off += (size_t)ceil_div(L.opixels(), 32) * 4; }
     off = net->counters_off;
     for (auto& T : net->tensors) {
         T.nnz = reinterpret_cast<unsigned long long*>(base + off);
@@ -205,10 +205,13 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         for (auto& L : net->layers) words = words > ceil_div(L.opixels(), 32) ? words : ceil_div(L.opixels(), 32);
         RRM_TRY(dev_alloc(net, (void**)&net->ones, (size_t)words * 4));
         RRM_CUDA_TRY(cudaMemset(net->ones, 0xff, (size_t)words * 4));
+        RRM_TRY(dev_alloc(net, (void**)&net->zeros, (size_t)words * 4));
     }
     {
         const char* e = getenv("RRM_NO_GRAPH");
         net->graph_off = e && e[0] == '1';
+        e = getenv("RRM_CHUNK_INPLACE");
+        net->chunk_in_place = e && e[0] == '1';
     }
     for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
     RRM_TRY(bind_readers(net));
@@ -488,7 +491,8 @@ constexpr int CHUNK_ARENAS = 64;                // arenas of the chunk graphs (>
 int ensure_chunk(rrm_net* net, int T)
 {
     const int L = (int)net->layers.size();
-    int slots = L + 2 < CHUNK_MAX_SLOTS ? L + 2 : CHUNK_MAX_SLOTS;
+    // (a frame is ~2 L + 2 launches long and, with the split projection, a new one can start every one or two of them)
+    int slots = 2 * L + 2 < CHUNK_MAX_SLOTS ? 2 * L + 2 : CHUNK_MAX_SLOTS;
     if (net->chunk_arena.empty()) {
         if (!net->cap_stream) RRM_CUDA_TRY(cudaStreamCreateWithFlags(&net->cap_stream, cudaStreamNonBlocking));
         // one block of CHUNK_ARENAS arenas: a chunk of up to that many frames gives every frame its own and clears
@@ -505,9 +509,9 @@ int ensure_chunk(rrm_net* net, int T)
             net->ev_join.push_back(e);
         }
         auto make = [&](cudaEvent_t* e) -> int { RRM_CUDA_TRY(cudaEventCreateWithFlags(e, cudaEventDisableTiming)); return RRM_OK; };
-        net->ev_conv.resize(L); net->ev_epi.resize(L);
-        for (int l = 0; l < L; ++l) { RRM_TRY(make(&net->ev_conv[l])); RRM_TRY(make(&net->ev_epi[l])); }
-        RRM_TRY(make(&net->ev_fork)); RRM_TRY(make(&net->ev_export));
+        net->ev_conv.resize(CHUNK_RING * L); net->ev_epi.resize(CHUNK_RING * L);
+        for (int l = 0; l < CHUNK_RING * L; ++l) { RRM_TRY(make(&net->ev_conv[l])); RRM_TRY(make(&net->ev_epi[l])); }
+        RRM_TRY(make(&net->ev_fork)); RRM_TRY(make(&net->ev_export)); RRM_TRY(make(&net->ev_import));
     }
     if (T > net->chunk_cap) {
         int64_t bi = 0, bo = 0;
@@ -525,11 +529,21 @@ int ensure_chunk(rrm_net* net, int T)
 }
 
 // T frames as one graph.  Frame t is captured on stream t mod S with arena t mod S; inside a frame the launches
-// follow each other on that stream; across frames:
+// follow each other on that stream.  Across frames, in the in-place form (keyframes, dense passes, delta chunks with
+// a layer evaluated densely, RRM_CHUNK_INPLACE=1):
 //   the convolution of layer l waits for the previous frame's epilogue of layer l (which reads the projection it adds to);
 //   the producer of a tensor (the import for tensor 0, the epilogue of layer l for tensor l+1) waits for the previous
 //   frame's readers of that tensor (convolutions that take it as input, epilogues that add it as shortcut, the export
 //   of the last tensor), because it overwrites the snapshot and the delta rows they read.
+// Delta chunks otherwise take the split form, which removes both waits from the frame-to-frame cycle (a layer then
+// advances one frame per epilogue instead of one per convolution + epilogue):
+//   the convolution of frame t adds its product into delta-projection buffer t mod R (R = CHUNK_RING) and waits only
+//   for the epilogue of frame t-R+1, whose merge role zeroed that buffer; the epilogue evaluates f from (projection
+//   as of t-1) + (the product), writes the merged rows to the other projection buffer and waits for the epilogue of
+//   frame t-1;
+//   delta rows (and the new rows of binary tensors) cycle through R sets, so a producer waits for the convolutions
+//   of frame t-R that read its tensor, and for the previous frame's shortcut readers and export, which read the
+//   snapshot it overwrites in place.
 // Everything else of consecutive frames may overlap.
 int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
 {
@@ -537,14 +551,18 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
     const int L = (int)net->layers.size();
     RRM_TRY(ensure_chunk(net, T));
     if (stateless) RRM_TRY(ensure_stateless(net));
+    const bool split = kind == 0 && mask == 0 && !net->chunk_in_place;
+    if (split) RRM_TRY(ensure_split(net));
     const int S = (int)net->chunk_streams.size() < T ? (int)net->chunk_streams.size() : T;
     const bool own_arena = T <= CHUNK_ARENAS;                // every frame has an arena of its own
+    const int R = CHUNK_RING;
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);
     tensor_bytes_boundary(net->tensors.back(), &bo);
     cudaStream_t origin = net->cap_stream;
-    std::vector<char> conv_rec(L, 0), epi_rec(L, 0);
-    bool export_rec = false;
+    // [slot * L + l]: an event of that layer has been recorded for a frame of that ring slot (in-place form: slot 0 only)
+    std::vector<char> conv_rec(R * L, 0), epi_rec(R * L, 0);
+    bool export_rec = false, import_rec = false;
     int status = RRM_OK;
     RRM_CUDA_TRY(cudaStreamBeginCapture(origin, cudaStreamCaptureModeThreadLocal));
     net->many_in_flight = true;
@@ -552,40 +570,74 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
     auto wait = [&](cudaStream_t s, cudaEvent_t e) { if (cudaStreamWaitEvent(s, e, 0) != cudaSuccess) fail(RRM_ERR_CUDA); };
     auto record = [&](cudaEvent_t e, cudaStream_t s) { if (cudaEventRecord(e, s) != cudaSuccess) fail(RRM_ERR_CUDA); };
     if (own_arena && !stateless && cudaMemsetAsync(net->chunk_arena[0], 0, net->cleared_bytes * T, origin) != cudaSuccess) fail(RRM_ERR_CUDA);
+    // the second projection buffers start as copies of the stored projections; whichever buffer the first frame reads,
+    // the last frame's merge lands in the stored one
+    if (split) { const int q = launch_copy_projections(net, origin); if (q != RRM_OK) fail(q); }
     record(net->ev_fork, origin);
     for (int k = 1; k < S; ++k) wait(net->chunk_streams[k], net->ev_fork);
-    // the previous frame's readers of tensor j
-    auto wait_readers = [&](cudaStream_t s, int j) {
+    // what the producer of tensor j waits for in a frame of ring slot `cur` (the previous frame has slot `prv`)
+    auto wait_readers = [&](cudaStream_t s, int j, int cur, int prv) {
         for (int r = 0; r < L; ++r) {
-            if (net->layers[r].d.src == j && conv_rec[r]) wait(s, net->ev_conv[r]);
-            if (net->layers[r].d.res == j && epi_rec[r]) wait(s, net->ev_epi[r]);
+            // (split form: slot `cur` still holds the events of frame t-R, whose convolutions read the set of delta
+            // rows about to be overwritten)
+            if (net->layers[r].d.src == j && conv_rec[cur * L + r]) wait(s, net->ev_conv[cur * L + r]);
+            if (net->layers[r].d.res == j && epi_rec[prv * L + r]) wait(s, net->ev_epi[prv * L + r]);
         }
         if (j == L && export_rec) wait(s, net->ev_export);
     };
     for (int t = 0; t < T && status == RRM_OK; ++t) {
         cudaStream_t s = net->chunk_streams[t % S];
+        const int cur = split ? t % R : 0, prv = split ? (t + R - 1) % R : 0, nxt = split ? (t + 1) % R : 0;
+        char* const prev_arena = net->chunk_arena[own_arena ? (t > 0 ? t - 1 : 0) : (t + S - 1) % S];
         bind_arena(net, net->chunk_arena[own_arena ? t : t % S]);
         if (bind_readers(net) != RRM_OK) { fail(RRM_ERR_UNSUPPORTED); break; }
-        // (a reused arena: the frame that used it before ran on this same stream, so it is complete before the clear)
-        if (!own_arena && !stateless && cudaMemsetAsync(net->bound_arena, 0, net->cleared_bytes, s) != cudaSuccess) fail(RRM_ERR_CUDA);
-        wait_readers(s, 0);
+        if (!own_arena && !stateless) {
+            // a reused arena: the frame that used it before ran on this same stream, so it is complete before the clear;
+            // in the split form the frame after that one read its update bitmaps as well
+            if (split && t >= S) wait(s, net->ev_join[(t + 1) % S]);
+            if (cudaMemsetAsync(net->bound_arena, 0, net->cleared_bytes, s) != cudaSuccess) fail(RRM_ERR_CUDA);
+        }
+        if (split) for (auto& X : net->tensors) { X.D = X.Dring[cur]; X.Xn_cur = X.Xn[cur]; }
+        wait_readers(s, 0, cur, prv);
+        if (split && import_rec) wait(s, net->ev_import);        // (the import reads and overwrites the input's snapshot)
         { const int q = launch_import(net, reinterpret_cast<const char*>(net->chunk_in) + (size_t)t * bi, !dense, stateless, s); if (q != RRM_OK) fail(q); }
+        if (split) { record(net->ev_import, s); import_rec = true; }
         for (int l = 0; l < L && status == RRM_OK; ++l) {
+            Layer& Y = net->layers[l];
+            SplitProjection sp{};
+            if (split) {
+                // frame T-1 writes the stored projection, the frames before it alternate
+                const bool to_stored = ((T - 1 - t) & 1) == 0;
+                sp.dP = Y.dP[cur];
+                sp.R = to_stored ? Y.Palt : Y.P;
+                sp.Q = to_stored ? Y.P : Y.Palt;
+                sp.Z = Y.dP[prv];
+                sp.prev_oact = t > 0 ? reinterpret_cast<const uint32_t*>(prev_arena + Y.oact_off) : net->zeros;
+            }
             const std::function<int(int)> hook = [&, l, s](int phase) -> int {
-                if (phase == 0) { if (epi_rec[l]) wait(s, net->ev_epi[l]); }
-                else if (phase == 1) { record(net->ev_conv[l], s); conv_rec[l] = 1; wait_readers(s, l + 1); }
-                else { record(net->ev_epi[l], s); epi_rec[l] = 1; }
+                if (phase == 0) {
+                    // split form: slot `nxt` holds the epilogue of frame t-R+1, whose merge role zeroed the buffer this product goes to
+                    if (epi_rec[nxt * L + l]) wait(s, net->ev_epi[nxt * L + l]);
+                } else if (phase == 1) {
+                    record(net->ev_conv[cur * L + l], s); conv_rec[cur * L + l] = 1;
+                    wait_readers(s, l + 1, cur, prv);
+                    if (split && epi_rec[prv * L + l]) wait(s, net->ev_epi[prv * L + l]);   // frame t-1: projection buffers, the output's snapshot
+                } else { record(net->ev_epi[cur * L + l], s); epi_rec[cur * L + l] = 1; }
                 return status;
             };
-            const int q = launch_layer(net, l, dense, stateless, s, &hook, !dense && l < 64 && (mask >> l & 1ull));
+            const int q = launch_layer(net, l, dense, stateless, s, &hook, !dense && l < 64 && (mask >> l & 1ull), split ? &sp : nullptr);
             if (q != RRM_OK) fail(q);
         }
         if (dense && !stateless && cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, s) != cudaSuccess) fail(RRM_ERR_CUDA);
         { const int q = launch_export_tensor(net, L, reinterpret_cast<char*>(net->chunk_out) + (size_t)t * bo, stateless, s); if (q != RRM_OK) fail(q); }
         record(net->ev_export, s);
         export_rec = true;
+        if (split && !own_arena) record(net->ev_join[t % S], s);                // the frame is complete (its arena may be cleared one frame later)
     }
+    if (split) for (auto& X : net->tensors) { X.D = X.Dring[0]; X.Xn_cur = nullptr; }
     for (int k = 1; k < S; ++k) { record(net->ev_join[k], net->chunk_streams[k]); wait(origin, net->ev_join[k]); }
+    // the last frame's products were merged but not zeroed (the arena bound now is that frame's)
+    if (split && status == RRM_OK) { const int q = launch_zero_delta_projections(net, (T - 1) % CHUNK_RING, origin); if (q != RRM_OK) fail(q); }
     cudaGraph_t g = nullptr;
     const cudaError_t e = cudaStreamEndCapture(origin, &g);
     net->many_in_flight = false;
@@ -784,6 +836,7 @@ int rrm_net_destroy(rrm_net* net)
     for (size_t k = 1; k < net->chunk_streams.size(); ++k) cudaStreamDestroy(net->chunk_streams[k]);   // [0] is cap_stream
     for (cudaEvent_t e : net->ev_conv) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : net->ev_epi) if (e) cudaEventDestroy(e);
+    if (net->ev_import) cudaEventDestroy(net->ev_import);
     for (cudaEvent_t e : net->ev_join) if (e) cudaEventDestroy(e);
     if (net->ev_fork) cudaEventDestroy(net->ev_fork);
     if (net->ev_export) cudaEventDestroy(net->ev_export);
@@ -1066,6 +1119,8 @@ int rrm_net_clear_errors(rrm_net* net)
     if (!net) return RRM_ERR_INVALID_ARG;
     if (net->last_stream) RRM_CUDA_TRY(cudaStreamSynchronize(net->last_stream));
     RRM_CUDA_TRY(cudaMemset(net->errw, 0, 4));
+    RRM_TRY(clear_split(net, nullptr));          // (a pipelined chunk that gave up may have left products unmerged)
+    RRM_CUDA_TRY(cudaDeviceSynchronize());
     return RRM_OK;
 }
 int rrm_clear_errors(rrm_layer* layer) { return rrm_net_clear_errors(layer); }

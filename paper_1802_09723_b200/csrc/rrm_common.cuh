@@ -98,6 +98,8 @@ struct Reader {
 constexpr int MAX_READERS = 4;
 struct Readers { Reader r[MAX_READERS]; int n; };
 
+constexpr int CHUNK_RING = 4;         // sets of delta rows / delta-projection buffers a pipelined chunk cycles through
+
 struct Tensor {
     int dtype = T_F32;
     int n = 0, c = 0, h = 0, w = 0;
@@ -111,6 +113,13 @@ struct Tensor {
     unsigned long long* npix = nullptr;     // active pixels (cleared every step)
     double* trunc = nullptr;                // fp32: sum of squares of the truncated delta entries (cleared every step)
     void* X2 = nullptr;               // value buffer of the stateless dense path
+    // pipelined chunks: consecutive frames write their delta rows into a ring of sets ([0] is the set D points at
+    // outside the capture of such a chunk), so that a producer does not wait for the previous frames' readers
+    void* Dring[CHUNK_RING] = {};
+    // binary tensors: the sparse product needs the new value of a changed bit (its sign) next to the delta rows, so the
+    // pipelined chunk keeps a copy of the new rows per frame parity; Xn_cur is set only while such a chunk is captured
+    void* Xn[CHUNK_RING] = {};
+    void* Xn_cur = nullptr;
     bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
     Readers readers{};                // the layers that read it
     int pixels() const { return n * h * w; }
@@ -132,6 +141,12 @@ struct Layer {
     void* bn_shift = nullptr;         // normalisation at inference): float, or int32 multiplier / offset; nullptr: none
     void* P = nullptr;                // projection [n*oh*ow][c_out] float or int32
     void* P2 = nullptr;               // projection buffer of the stateless dense path
+    // pipelined delta chunks: the convolution of a frame adds into a delta-projection buffer of its own (one of a ring,
+    // zero between uses) and the epilogue merges it, reading the projection from one buffer and writing it to the
+    // other, so that the convolution of frame t+1 does not wait for the epilogue of frame t
+    void* Palt = nullptr;             // the second projection buffer (a copy of P is made at the start of a chunk)
+    void* dP[CHUNK_RING] = {};
+    size_t oact_off = 0;              // offset of the update bitmap inside an arena
     uint32_t* oact = nullptr;         // bitmap of projection pixels to update (cleared every step, set by the
                                       // kernels that produce the layer's input and shortcut tensors)
     int* ocount = nullptr;            // their number (cleared every step, written by the convolution kernel)
@@ -241,7 +256,12 @@ struct rrm_net {
     // flight has an arena of its own.
     std::vector<char*> chunk_arena;
     std::vector<cudaStream_t> chunk_streams;      // capture streams, one per frame in flight ([0] is cap_stream)
-    std::vector<cudaEvent_t> ev_conv, ev_epi;     // per layer: the most recently captured convolution / epilogue
+    // [slot * layers + l]: the most recently captured convolution / epilogue of layer l among the frames of ring slot
+    // `slot` (frame mod CHUNK_RING in the split form; slot 0 only otherwise)
+    std::vector<cudaEvent_t> ev_conv, ev_epi;
+    cudaEvent_t ev_import = nullptr;
+    bool chunk_in_place = false;                  // RRM_CHUNK_INPLACE=1: delta chunks add into the stored projection (no delta-projection buffers)
+    uint32_t* zeros = nullptr;                    // an all-zero bitmap as long as the longest update bitmap
     std::vector<cudaEvent_t> ev_join;
     cudaEvent_t ev_fork = nullptr, ev_export = nullptr;
     struct ChunkGraph { int T = 0; unsigned long long mask = 0; cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr; unsigned long long used = 0; };
@@ -297,18 +317,31 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
 bool conv_tc_eligible(const rrm_net* net, const Layer& L);
 int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev);
 int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st,
-                   const uint32_t* count_bitmap = nullptr);
+                   const uint32_t* count_bitmap = nullptr, void* P_dst = nullptr);
 int zero_projection(void* P, long long words, cudaStream_t st);
 
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);
 int launch_import(rrm_net* net, const void* frame_dev, bool delta, bool stateless, cudaStream_t st);
+// Where a delta step of one layer keeps its projection when the frames of a chunk are pipelined (null: in place).
+struct SplitProjection {
+    void* dP;                         // the convolution adds here (zero wherever the frame has no update)
+    const void* R;                    // the projection as of the previous frame
+    void* Q;                          // receives R + dP at the pixels updated in this frame or in the previous one
+    void* Z;                          // the previous frame's delta-projection buffer, zeroed at that frame's updated pixels
+    const uint32_t* prev_oact;        // the previous frame's update bitmap
+};
 int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st,
-                 const std::function<int(int)>* hook = nullptr, bool dense_in_step = false);
+                 const std::function<int(int)>* hook = nullptr, bool dense_in_step = false,
+                 const SplitProjection* split = nullptr);
 int launch_export_tensor(rrm_net* net, int t, void* dst_dev, bool stateless, cudaStream_t st);
 int launch_export_projection(rrm_net* net, int l, void* dst_dev, cudaStream_t st);
 int reset_state(rrm_net* net, cudaStream_t st);
 int ensure_stateless(rrm_net* net);
 int launch_aecs(rrm_net* net, cudaStream_t st);
+int ensure_split(rrm_net* net);
+int launch_copy_projections(rrm_net* net, cudaStream_t st);
+int launch_zero_delta_projections(rrm_net* net, int slot, cudaStream_t st);
+int clear_split(rrm_net* net, cudaStream_t st);
 
 }  // namespace rrm

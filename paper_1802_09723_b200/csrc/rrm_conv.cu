@@ -597,7 +597,7 @@ __global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __res
 template <bool DELTA>
 __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X, uint32_t* D, uint32_t* act,
                                   int* pnnz, unsigned long long* nnz, unsigned long long* npix, int cw, int pixels,
-                                  int h, int w, Readers readers)
+                                  int h, int w, Readers readers, uint32_t* Xn)
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x;
     pdl_launch_dependents();
@@ -612,6 +612,7 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
                 cnt += __popc(ch);
             }
             X[(size_t)gp * cw + k] = xt;
+            if (DELTA && Xn) Xn[(size_t)gp * cw + k] = xt;   // (pipelined chunk: the frame's own copy of the new rows)
         }
         if (DELTA && cnt) {
             atomicOr(&act[gp >> 5], 1u << (gp & 31));
@@ -664,21 +665,78 @@ struct EpiParams {
     double* trunc;            // fp32: receives the sum of squares of the truncated entries
     const void* bn_scale;     // explicit batch normalisation, the first step of f: per-channel float scale / shift
     const void* bn_shift;     // (fp32) or int32 multiplier / offset inside the requantisation (int8); nullptr: none
+    // SPLIT form (pipelined chunks): P is the projection as of the previous frame and is only read; the frame's product
+    // waits in dP (zero wherever oact has no bit).  CTAs from f_blocks on merge: Q = P + dP at the pixels of oact and
+    // of oact_prev (the other buffer missed the previous frame's update), and Z, the previous frame's dP, is zeroed
+    // at the pixels of oact_prev so that the buffer can be added into again.
+    const void* dP;
+    void* Q;
+    void* Z;
+    void* Xn;                 // binary outputs: receives a copy of the new rows of the pixels looked at (or nullptr)
+    const uint32_t* oact_prev;
+    int f_blocks;             // CTAs that evaluate f
+    int opix;                 // projection pixels
 };
 
 // PT: projection type (T_F32 or T_I32).  OT: output tensor storage type.  KW: pool window edge (1 = no pool).
 // READERS: some layer reads the output tensor (a last layer's kernel leaves the marking code, and its registers, out).
 // BN: f starts with the explicit per-channel affine (the kernels of layers without one are compiled without it).
-template <int PT, int OT, bool DENSE, int KW, bool READERS, bool BN>
+// SPLIT: the projection is read from one buffer plus the frame's delta projection and merged into another (see EpiParams).
+template <int PT, int OT, bool DENSE, int KW, bool READERS, bool BN, bool SPLIT>
 __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
 {
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
+    using pt4 = typename std::conditional<PT == T_F32, float4, int4>::type;
     __shared__ unsigned long long s_macs[MAX_READERS];
     __shared__ unsigned int s_nnz, s_npix;
     __shared__ int s_cnt[8];                                 // changed elements of the CTA's pixels
     __shared__ float s_sq;
     const int lane = threadIdx.x & 31;
     pdl_launch_dependents();
+    if (SPLIT && (int)blockIdx.x >= p.f_blocks) {
+        // ---- merge role: a CTA per word of the update bitmaps, a warp per four of its pixels, whose rows are in flight together
+        pdl_wait();
+        const int w = (int)blockIdx.x - p.f_blocks;
+        const unsigned bp = p.oact_prev[w];
+        const unsigned u = (p.oact[w] | bp) >> ((threadIdx.x >> 5) * 4);
+        if ((u & 15u) == 0) return;
+        const unsigned zp = bp >> ((threadIdx.x >> 5) * 4);
+        const pt* R = reinterpret_cast<const pt*>(p.P);
+        const pt* dP = reinterpret_cast<const pt*>(p.dP);
+        pt* Q = reinterpret_cast<pt*>(p.Q);
+        pt* Z = reinterpret_cast<pt*>(p.Z);
+        const size_t row0 = (size_t)(w * 32 + (threadIdx.x >> 5) * 4) * p.c_out;
+        if ((p.c_out & 3) == 0) {
+            for (int c = lane * 4; c < p.c_out; c += 128) {
+                pt4 r[4], d[4];
+                #pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (!(u >> k & 1u)) continue;
+                    r[k] = *reinterpret_cast<const pt4*>(R + row0 + (size_t)k * p.c_out + c);
+                    d[k] = *reinterpret_cast<const pt4*>(dP + row0 + (size_t)k * p.c_out + c);
+                }
+                #pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (!(u >> k & 1u)) continue;
+                    pt4 t = r[k];
+                    t.x += d[k].x; t.y += d[k].y; t.z += d[k].z; t.w += d[k].w;
+                    *reinterpret_cast<pt4*>(Q + row0 + (size_t)k * p.c_out + c) = t;
+                    if (zp >> k & 1u) { pt4 z; z.x = z.y = z.z = z.w = 0; *reinterpret_cast<pt4*>(Z + row0 + (size_t)k * p.c_out + c) = z; }
+                }
+            }
+        } else {
+            #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (!(u >> k & 1u)) continue;
+                for (int c = lane; c < p.c_out; c += 32) {
+                    const size_t o = row0 + (size_t)k * p.c_out + c;
+                    Q[o] = R[o] + dP[o];
+                    if (zp >> k & 1u) Z[o] = 0;
+                }
+            }
+        }
+        return;
+    }
     if (threadIdx.x < MAX_READERS) s_macs[threadIdx.x] = 0;
     if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) { s_nnz = 0; s_npix = 0; s_sq = 0.f; }
@@ -693,7 +751,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
     const int y0 = ty * st - pp, x0 = tx * st - pp;
     const int qbase = ns * p.oh * p.ow;
     // window positions inside the projection (bit wy * KW + wx), and whether any of them was updated
-    unsigned inside = 0;
+    unsigned inside = 0, updm = 0;
     bool on = false;
     if (r < tpix) {
         bool mine = false, upd = false;
@@ -703,7 +761,8 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
             if (mine && !DENSE) { const int q = qbase + y * p.ow + x; upd = (p.oact[q >> 5] >> (q & 31)) & 1u; }
         }
         inside = __ballot_sync(0xffffffffu, mine);
-        on = DENSE ? true : (__ballot_sync(0xffffffffu, upd) != 0);
+        updm = __ballot_sync(0xffffffffu, upd);
+        on = DENSE ? true : updm != 0;
     }
     int cnt = 0;
     float sq = 0.f;                                          // squares of the truncated delta entries (fp32)
@@ -730,6 +789,14 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                 } else {
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) if (c + j < p.c_out) v[wi][j] = P[o + j];
+                }
+                if (SPLIT && (updm >> wi & 1u)) {            // this frame's product is still on its own
+                    const pt* dP = reinterpret_cast<const pt*>(p.dP);
+                    if (vec) { const pt4 t = *reinterpret_cast<const pt4*>(dP + o); v[wi][0] += t.x; v[wi][1] += t.y; v[wi][2] += t.z; v[wi][3] += t.w; }
+                    else {
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) if (c + j < p.c_out) v[wi][j] += dP[o + j];
+                    }
                 }
             }
             // ---- f: [affine] -> [requant] -> [+ shortcut] -> act -> max over the window (sign: max first, threshold last)
@@ -794,6 +861,7 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                         const uint32_t ch = word ^ X[o];
                         reinterpret_cast<uint32_t*>(p.D)[o] = ch;
                         X[o] = word;
+                        if (SPLIT && p.Xn) reinterpret_cast<uint32_t*>(p.Xn)[o] = word;
                         cnt += __popc(ch);
                     }
                 }
@@ -897,6 +965,44 @@ __global__ void fill_projection_kernel(T* P, const T* bias, int c_out, long long
 }
 
 // Eq. 7, one frame: e_t += sum over the linear layers of l2(truncated part of the layer's input).
+// Copies of whole projections (start of a pipelined chunk: the second buffer of every layer), one launch for up to 32 layers.
+struct CopyJobs { const int* src[32]; int* dst[32]; long long words[32]; int n; };
+__global__ void __launch_bounds__(256) copy_projections_kernel(CopyJobs j)
+{
+    const int k = blockIdx.y;
+    const long long n = j.words[k], step = (long long)gridDim.x * blockDim.x;
+    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
+    if ((n & 3) == 0) {
+        const int4* s = reinterpret_cast<const int4*>(j.src[k]);
+        int4* d = reinterpret_cast<int4*>(j.dst[k]);
+        for (long long i = i0; i < n / 4; i += step) d[i] = s[i];
+    } else {
+        for (long long i = i0; i < n; i += step) j.dst[k][i] = j.src[k][i];
+    }
+}
+
+// End of a pipelined chunk: the last frame's delta projections go back to zero (rows of the pixels in `bits`).
+struct ZeroJobs { int* dst[32]; const uint32_t* bits[32]; int words[32]; int c_out[32]; int n; };
+__global__ void __launch_bounds__(256) zero_rows_kernel(ZeroJobs j)
+{
+    const int k = blockIdx.y, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int c_out = j.c_out[k];
+    for (int w = blockIdx.x * 8 + (threadIdx.x >> 5); w < j.words[k]; w += gridDim.x * 8) {
+        unsigned u = j.bits[k][w];
+        while (u) {
+            const int q = w * 32 + __ffs(u) - 1;
+            u &= u - 1;
+            int* row = j.dst[k] + (size_t)q * c_out;
+            if ((c_out & 3) == 0) for (int c = lane * 4; c < c_out; c += 128) *reinterpret_cast<int4*>(row + c) = make_int4(0, 0, 0, 0);
+            else for (int c = lane; c < c_out; c += 32) row[c] = 0;
+        }
+    }
+}
+
 struct AecsParams { const double* sumsq[64]; int n; double* e_t; double* last_l2; };
 __global__ void aecs_accumulate_kernel(AecsParams p)
 {
@@ -991,10 +1097,10 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
         const int blocks = ceil_div(T.pixels(), 256);
         if (delta) launch_seq(import_bin_kernel<true>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, (uint32_t*)T.D,
                                                                   T.act, T.pnnz, T.nnz, T.npix, T.cs, T.pixels(),
-                                                                  T.h, T.w, T.readers);
+                                                                  T.h, T.w, T.readers, (uint32_t*)(stateless ? nullptr : T.Xn_cur));
         else launch_seq(import_bin_kernel<false>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, nullptr, nullptr,
                                                               nullptr, nullptr, nullptr, T.cs, T.pixels(), T.h, T.w,
-                                                              Readers{});
+                                                              Readers{}, (uint32_t*)nullptr);
     } else if (T.dtype == T_I8 && T.cs == 4) {
         const int blocks = ceil_div(T.pixels(), 256);
         if (delta) launch_seq(import_i8_word_kernel<true>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
@@ -1034,14 +1140,26 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
     return RRM_OK;
 }
 
+template <int PT, int OT, bool DENSE, bool BN, int KW>
+static void launch_epi_kw(const EpiParams& e, int blocks, cudaStream_t st)
+{
+    const bool rd = !DENSE && e.readers.n > 0;               // (a dense pass marks nothing)
+    if (!DENSE && e.dP) {                                    // pipelined chunk: f from P + dP, merge CTAs behind the f CTAs
+        if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, KW, !DENSE, BN, !DENSE>, dim3(blocks), dim3(256), 0, st, e);
+        else launch_seq(epilogue_kernel<PT, OT, DENSE, KW, false, BN, !DENSE>, dim3(blocks), dim3(256), 0, st, e);
+    } else {
+        if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, KW, !DENSE, BN, false>, dim3(blocks), dim3(256), 0, st, e);
+        else launch_seq(epilogue_kernel<PT, OT, DENSE, KW, false, BN, false>, dim3(blocks), dim3(256), 0, st, e);
+    }
+}
+
 template <int PT, int OT, bool DENSE, bool BN>
 static int launch_epi_kb(const EpiParams& e, int blocks, cudaStream_t st)
 {
-    const bool rd = !DENSE && e.readers.n > 0;               // (a dense pass marks nothing)
     switch (e.pool_k > 0 ? e.pool_k : 1) {
-        case 1: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 1, !DENSE, BN>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 1, false, BN>, dim3(blocks), dim3(256), 0, st, e); break;
-        case 2: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 2, !DENSE, BN>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 2, false, BN>, dim3(blocks), dim3(256), 0, st, e); break;
-        case 3: if (rd) launch_seq(epilogue_kernel<PT, OT, DENSE, 3, !DENSE, BN>, dim3(blocks), dim3(256), 0, st, e); else launch_seq(epilogue_kernel<PT, OT, DENSE, 3, false, BN>, dim3(blocks), dim3(256), 0, st, e); break;
+        case 1: launch_epi_kw<PT, OT, DENSE, BN, 1>(e, blocks, st); break;
+        case 2: launch_epi_kw<PT, OT, DENSE, BN, 2>(e, blocks, st); break;
+        case 3: launch_epi_kw<PT, OT, DENSE, BN, 3>(e, blocks, st); break;
         default: return RRM_ERR_UNSUPPORTED;                 // pool windows are 2x2 or 3x3
     }
     return RRM_OK;
@@ -1071,10 +1189,12 @@ static int launch_epi(const EpiParams& e, int ot, int blocks, cudaStream_t st)
 // dense_in_step: the layer is evaluated densely inside a delta step (its measured activity is above the
 // threshold): P = F*X + b from the input's current value replaces the stored projection (a precise inference of
 // this layer), and the epilogue still compares f(P) with the stored output and emits the next layer's delta.
+// split (delta steps of pipelined chunks): the product goes to a delta-projection buffer and the epilogue merges it.
 int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t st, const std::function<int(int)>* hook,
-                 bool dense_in_step)
+                 bool dense_in_step, const SplitProjection* split)
 {
     if (hook) RRM_TRY((*hook)(0));
+    if (split && (dense || stateless || dense_in_step)) return RRM_ERR_INVALID_ARG;
     const bool step_dense = dense_in_step && !dense && !stateless;
     const bool conv_dense = dense || step_dense;
     Layer& L = net->layers[l];
@@ -1084,8 +1204,8 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     Tensor* res = d.res >= 0 ? &net->tensors[d.res] : nullptr;
 
     ConvParams p;
-    p.D = in.D; p.X = stateless ? in.X2 : in.X; p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
-    p.Wk = L.Wk; p.bias = L.bias; p.P = stateless ? L.P2 : L.P;
+    p.D = in.D; p.X = stateless ? in.X2 : (split && in.Xn_cur ? in.Xn_cur : in.X); p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
+    p.Wk = L.Wk; p.bias = L.bias; p.P = split ? split->dP : (stateless ? L.P2 : L.P);
     p.n = d.n; p.c_in = d.c_in; p.h = d.h; p.w = d.w; p.u_in = L.u_in; p.oh = L.oh; p.ow = L.ow;
     p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.c_out = d.c_out; p.np = L.np;
     p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
@@ -1100,14 +1220,16 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
         // (integer shares add onto a zeroed projection; fp32 shares meet in their cluster's shared memory, in a fixed order)
         if (!L.tc_ready && conv_dense && ks > 1 && d.dtype != RRM_F32) RRM_TRY(zero_projection(p.P, (long long)L.opixels() * d.c_out, st));
     }
-    if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, conv_dense, stateless, st, p.count_bitmap));
+    if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, conv_dense, stateless, st, p.count_bitmap, split ? split->dP : nullptr));
     else if (d.dtype == RRM_F32) { if (conv_dense) launch_gemm<T_F32, true>(p, grid, st); else launch_gemm<T_F32, false>(p, grid, st); }
     else if (d.dtype == RRM_I8) { if (conv_dense) launch_gemm<T_I8, true>(p, grid, st); else launch_gemm<T_I8, false>(p, grid, st); }
     else { if (conv_dense) launch_gemm<T_BIN, true>(p, grid, st); else launch_gemm<T_BIN, false>(p, grid, st); }
 
     if (hook) RRM_TRY((*hook)(1));
     EpiParams e;
-    e.P = p.P; e.oact = step_dense ? net->ones : L.oact;     // (dense inside a delta step: every window is looked at)
+    e.P = split ? split->R : p.P; e.oact = step_dense ? net->ones : L.oact;     // (dense inside a delta step: every window is looked at)
+    e.dP = split ? split->dP : nullptr; e.Q = split ? split->Q : nullptr; e.Z = split ? split->Z : nullptr;
+    e.oact_prev = split ? split->prev_oact : nullptr; e.opix = L.opixels(); e.Xn = split ? out.Xn_cur : nullptr;
     e.resX = res ? (stateless ? res->X2 : res->X) : nullptr;
     e.X = stateless ? out.X2 : out.X; e.D = out.D; e.act = out.act; e.pnnz = out.pnnz; e.nnz = out.nnz;
     e.npix = out.npix; e.errw = out.has_consumer ? net->errw : nullptr;
@@ -1124,13 +1246,86 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
         const bool latency_bound = !net->many_in_flight && out.pixels() <= 8 * 2 * 148;
         e.wpp = !latency_bound ? 1 : (chunks >= 8 ? 8 : (chunks > 2 ? 4 : (chunks > 1 ? 2 : 1)));
     }
-    const int blocks = ceil_div(out.pixels(), 8 / e.wpp);
+    e.f_blocks = ceil_div(out.pixels(), 8 / e.wpp);
+    const int blocks = e.f_blocks + (split ? ceil_div(L.opixels(), 32) : 0);   // merge CTAs: one per word of the update bitmap
     int es;
     if (proj_type(L) == T_F32) es = dense ? launch_epi<T_F32, true>(e, out.dtype, blocks, st) : launch_epi<T_F32, false>(e, out.dtype, blocks, st);
     else es = dense ? launch_epi<T_I32, true>(e, out.dtype, blocks, st) : launch_epi<T_I32, false>(e, out.dtype, blocks, st);
     RRM_TRY(es);
     RRM_CUDA_TRY(cudaGetLastError());
     if (hook) RRM_TRY((*hook)(2));
+    return RRM_OK;
+}
+
+// The buffers of the pipelined delta chunks (second projection, the rings of delta projections and of delta rows).
+int ensure_split(rrm_net* net)
+{
+    for (auto& L : net->layers) {
+        const size_t bytes = (size_t)L.opixels() * L.d.c_out * 4;
+        if (!L.Palt) RRM_TRY(dev_alloc(net, &L.Palt, bytes, false));
+        for (int k = 0; k < CHUNK_RING; ++k) if (!L.dP[k]) RRM_TRY(dev_alloc(net, &L.dP[k], bytes));      // zero
+    }
+    for (auto& T : net->tensors) {
+        if (!T.Dring[0]) T.Dring[0] = T.D;
+        for (int k = 1; k < CHUNK_RING; ++k) if (!T.Dring[k]) RRM_TRY(dev_alloc(net, &T.Dring[k], T.bytes()));
+        if (T.dtype == T_BIN) for (int k = 0; k < CHUNK_RING; ++k) if (!T.Xn[k]) RRM_TRY(dev_alloc(net, &T.Xn[k], T.bytes()));
+    }
+    return RRM_OK;
+}
+
+// P -> Palt for every layer.
+int launch_copy_projections(rrm_net* net, cudaStream_t st)
+{
+    const int n = (int)net->layers.size();
+    for (int l0 = 0; l0 < n; l0 += 32) {
+        CopyJobs j;
+        j.n = n - l0 < 32 ? n - l0 : 32;
+        long long most = 0;
+        for (int k = 0; k < j.n; ++k) {
+            const Layer& L = net->layers[l0 + k];
+            j.src[k] = reinterpret_cast<const int*>(L.P);
+            j.dst[k] = reinterpret_cast<int*>(L.Palt);
+            j.words[k] = (long long)L.opixels() * L.d.c_out;
+            most = most > j.words[k] ? most : j.words[k];
+        }
+        for (int k = j.n; k < 32; ++k) { j.src[k] = nullptr; j.dst[k] = nullptr; j.words[k] = 0; }
+        long long gx = (most / 4 + 255) / 256;
+        gx = gx < 1 ? 1 : (gx > 148 ? 148 : gx);                 // (a few 16-byte words per thread at most layers' sizes)
+        launch_seq(copy_projections_kernel, dim3((unsigned)gx, (unsigned)j.n), dim3(256), 0, st, j);
+    }
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
+// Zeroes delta-projection buffer `slot` of every layer at the pixels of the bound arena's update bitmaps.
+int launch_zero_delta_projections(rrm_net* net, int slot, cudaStream_t st)
+{
+    const int n = (int)net->layers.size();
+    for (int l0 = 0; l0 < n; l0 += 32) {
+        ZeroJobs j;
+        j.n = n - l0 < 32 ? n - l0 : 32;
+        int most = 1;
+        for (int k = 0; k < 32; ++k) {
+            if (k < j.n) {
+                const Layer& L = net->layers[l0 + k];
+                j.dst[k] = reinterpret_cast<int*>(L.dP[slot]); j.bits[k] = L.oact;
+                j.words[k] = ceil_div(L.opixels(), 32); j.c_out[k] = L.d.c_out;
+                most = most > j.words[k] ? most : j.words[k];
+            } else { j.dst[k] = nullptr; j.bits[k] = nullptr; j.words[k] = 0; j.c_out[k] = 0; }
+        }
+        const int gx = ceil_div(most, 8) < 148 ? ceil_div(most, 8) : 148;
+        launch_seq(zero_rows_kernel, dim3((unsigned)gx, (unsigned)j.n), dim3(256), 0, st, j);
+    }
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
+// All delta-projection buffers back to zero (after a step that gave up may have left rows behind).
+int clear_split(rrm_net* net, cudaStream_t st)
+{
+    for (auto& L : net->layers)
+        for (int k = 0; k < CHUNK_RING; ++k)
+            if (L.dP[k]) RRM_CUDA_TRY(cudaMemsetAsync(L.dP[k], 0, (size_t)L.opixels() * L.d.c_out * 4, st));
     return RRM_OK;
 }
 

@@ -538,19 +538,20 @@ int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev)
     return RRM_OK;
 }
 
-// F*dI (dense: F*X + b) on the tensor cores; P is updated in place (dense: overwritten).
+// F*dI (dense: F*X + b) on the tensor cores; P is updated in place (dense: overwritten).  P_dst (delta only): the
+// product is added there instead of onto the stored projection.
 int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st,
-                   const uint32_t* count_bitmap)
+                   const uint32_t* count_bitmap, void* P_dst)
 {
     const rrm_layer_desc& d = L.d;
     TcParams p;
     const bool bin = d.dtype == RRM_BIN;
     const void* X = stateless ? in.X2 : in.X;
     p.A = bin ? in.D : (dense ? X : in.D);
-    p.Anew = X;
+    p.Anew = (!dense && !stateless && in.Xn_cur) ? in.Xn_cur : X;    // (pipelined chunk: this frame's copy of the new rows)
     p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
     p.Wimg = L.tc_Wimg; p.bias = reinterpret_cast<const int32_t*>(L.bias);
-    p.P = reinterpret_cast<int32_t*>(stateless ? L.P2 : L.P);
+    p.P = reinterpret_cast<int32_t*>(P_dst && !dense ? P_dst : (stateless ? L.P2 : L.P));
     p.errw = net->errw;
     p.h = d.h; p.w = d.w; p.oh = L.oh; p.ow = L.ow; p.kw = d.kw; p.taps = d.kh * d.kw; p.stride = d.stride; p.pad = d.pad;
     p.c_in = d.c_in; p.c_out = d.c_out; p.opixels = L.opixels();
