@@ -98,6 +98,15 @@ struct Reader {
 constexpr int MAX_READERS = 4;
 struct Readers { Reader r[MAX_READERS]; int n; };
 
+// Several consecutive frames in one launch (frame = blockIdx.z; frames <= 1: the ordinary single-frame launch): where
+// frame g's data lie relative to frame 0's.
+struct SeqFrames {
+    int frames;
+    long long in_stride;      // elements between consecutive frames at the boundary (the frame before frame 0 lies one stride earlier)
+    long long row_stride;     // bytes between the frames' sets of delta rows (and of new rows)
+    long long arena_stride;   // bytes between the frames' arenas (bitmaps, counters)
+};
+
 constexpr int CHUNK_RING = 4;         // sets of delta rows / delta-projection buffers a pipelined chunk cycles through
 
 struct Tensor {
@@ -317,12 +326,12 @@ int fc_tc_run(rrm_net* net, Layer& L, const void* X_dev, void* Y_dev, int rows, 
 bool conv_tc_eligible(const rrm_net* net, const Layer& L);
 int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev);
 int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st,
-                   const uint32_t* count_bitmap = nullptr, void* P_dst = nullptr);
+                   const uint32_t* count_bitmap = nullptr, void* P_dst = nullptr, int frames = 1, long long arena_stride = 0);
 int zero_projection(void* P, long long words, cudaStream_t st);
 
 // ---- rrm_conv.cu
 int conv_layer_create(rrm_net* net, Layer& L, const void* W_dev, const void* bias_dev);
-int launch_import(rrm_net* net, const void* frame_dev, bool delta, bool stateless, cudaStream_t st);
+int launch_import(rrm_net* net, const void* frame_dev, bool delta, bool stateless, cudaStream_t st, int frames = 1, long long arena_stride = 0);
 // Where a delta step of one layer keeps its projection when the frames of a chunk are pipelined (null: in place).
 struct SplitProjection {
     void* dP;                         // the convolution adds here (zero wherever the frame has no update)

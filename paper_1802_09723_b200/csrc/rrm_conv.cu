@@ -44,6 +44,12 @@ struct ConvParams {
     unsigned wait_limit;      // polls of one bounded wait
     const uint32_t* count_bitmap;   // dense evaluation inside a delta step: the layer's update bitmap, whose set bits the
                                     // first CTA counts into *ocount (the measured activity); nullptr otherwise
+    // several frames in one launch (delta only, K not split; gridDim.z = frames): frame g reads its delta rows, new
+    // rows and bitmaps, and stores its product, at these distances from frame 0's
+    int frames;
+    long long row_stride;     // bytes between the frames' sets of delta rows (and of new rows)
+    long long arena_stride;   // bytes between the frames' arenas (bitmaps, counters)
+    long long p_stride;       // elements between the frames' products
 };
 
 // The number of set bits of bm[0 .. words) -> *out, by one CTA (the activity of a layer that is evaluated densely).
@@ -112,12 +118,23 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int tile = blockIdx.x, n0 = blockIdx.y * TN;
+    const bool batched = !DENSE && p.frames > 1;             // gridDim.z counts frames, not shares of K
+    const int zshare = batched ? 0 : blockIdx.z;
+    if (batched && blockIdx.z > 0) {
+        const long long g = blockIdx.z;
+        p.D = reinterpret_cast<const char*>(p.D) + g * p.row_stride;
+        p.X = reinterpret_cast<const char*>(p.X) + g * p.row_stride;
+        p.in_act = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.in_act) + g * p.arena_stride);
+        p.oact = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.oact) + g * p.arena_stride);
+        p.ocount = reinterpret_cast<int*>(reinterpret_cast<char*>(p.ocount) + g * p.arena_stride);
+        p.P = reinterpret_cast<char*>(p.P) + g * p.p_stride * 4;
+    }
     pdl_launch_dependents();
     if (!DENSE) {
         pdl_wait();                                          // the update bitmap is the predecessors' work
         // this CTA's rows: the tile-th group of TM set bits of the layer's update bitmap
         const int count = select_rows<TM>(p.oact, (p.opixels + 31) >> 5, tile, s_q, s_tmp);
-        if (tile == 0 && blockIdx.y == 0 && blockIdx.z == 0 && tid == 0) *p.ocount = count;
+        if (tile == 0 && blockIdx.y == 0 && zshare == 0 && tid == 0) *p.ocount = count;
         if (tile * TM >= count) return;
     }
     if (tid == 0) {
@@ -157,11 +174,11 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     const unsigned long long tm0 = (unsigned long long)s_tapmask[0] | (unsigned long long)s_tapmask[1] << 32;
     const unsigned long long tm1 = (unsigned long long)s_tapmask[2] | (unsigned long long)s_tapmask[3] << 32;
     if (DENSE) pdl_wait();                                   // barriers and row tables are set up; the inputs come next
-    if (DENSE && p.count_bitmap && tile == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+    if (DENSE && p.count_bitmap && tile == 0 && blockIdx.y == 0 && zshare == 0)
         count_bits_cta(p.count_bitmap, (p.opixels + 31) >> 5, p.ocount, s_tmp);
     // this CTA's share of the K stages
     const int all_stages = p.kup / TK, per_split = (all_stages + p.ksplit - 1) / p.ksplit;
-    const int s_first = blockIdx.z * per_split, n_stages = min(all_stages, s_first + per_split);
+    const int s_first = zshare * per_split, n_stages = min(all_stages, s_first + per_split);
     auto stage_live = [&](int ks) -> bool {                 // any usable tap among the stage's K units?
         const int t_lo = (ks * TK) / p.u_in, t_hi = min(taps - 1, (ks * TK + TK - 1) / p.u_in);
         for (int t = t_lo; t <= t_hi; ++t)
@@ -308,7 +325,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             *reinterpret_cast<float4*>(&tilebuf[(tm + i) * TN + tn]) = make_float4((float)acc[i][0], (float)acc[i][1], (float)acc[i][2], (float)acc[i][3]);
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-        const int rank = blockIdx.z, rows_per = TM / p.ksplit;
+        const int rank = zshare, rows_per = TM / p.ksplit;
         const uint32_t tile_u32 = g_smem_u32(tilebuf);
         float* P = reinterpret_cast<float*>(p.P);
         for (int item = tid; item < rows_per * (TN / 4); item += CONV_THREADS) {
@@ -355,15 +372,15 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
                 float* P = reinterpret_cast<float*>(p.P);
                 float v = acc[i][j];
                 if (DENSE && p.bias) v += reinterpret_cast<const float*>(p.bias)[co];
-                if (DENSE) P[o] = v;
+                if (DENSE || batched) P[o] = v;            // (several frames per launch: the product is stored, not added)
                 else P[o] += v;
             } else {
                 int* P = reinterpret_cast<int*>(p.P);
                 int v = (int)acc[i][j];
                 if (DT == T_BIN) v = DENSE ? (rowpop[i] - 2 * v) : 2 * (rowpop[i] - 2 * v);
-                if (DENSE && blockIdx.z == 0 && p.bias) v += reinterpret_cast<const int*>(p.bias)[co];
+                if (DENSE && zshare == 0 && p.bias) v += reinterpret_cast<const int*>(p.bias)[co];
                 if (shared_tile) atomicAdd(P + o, v);
-                else if (DENSE) P[o] = v;
+                else if (DENSE || batched) P[o] = v;
                 else P[o] += v;
             }
         }
@@ -438,6 +455,17 @@ __global__ void pack_weights_kernel(const void* W, uint32_t* Wk, int dt, int c_i
 // One CTA handles 32 consecutive pixels of one stream: coalesced reads along w, transposed through
 // shared memory, coalesced pixel-major writes.
 // ------------------------------------------------------------------------------------------------
+// the readers' bitmaps and counters of frame g's arena
+__device__ __forceinline__ void shift_readers(Readers& R, long long bytes)
+{
+    #pragma unroll
+    for (int i = 0; i < MAX_READERS; ++i) {
+        if (i >= R.n) break;
+        R.r[i].oact = shift_bytes(R.r[i].oact, bytes);
+        if (R.r[i].macs) R.r[i].macs = shift_bytes(R.r[i].macs, bytes);
+    }
+}
+
 constexpr int IMP_TP = 32;                  // pixels per tile = lanes of the warp that marks their footprints
 
 template <typename T, bool DELTA>
@@ -445,21 +473,38 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
                                                           int* pnnz, unsigned long long* nnz,
                                                           unsigned long long* npix, int* errw,
                                                           int c, int cs, int hw, int w, Readers readers,
-                                                          float eps, double* trunc)
+                                                          float eps, double* trunc, SeqFrames sf)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    T* s_x = reinterpret_cast<T*>(smem_raw);               // [IMP_TP][cs + 1]
+    T* s_x = reinterpret_cast<T*>(smem_raw);               // [IMP_TP][cs + 1] (several frames per launch: a second tile, the frame before)
     __shared__ int s_cnt[IMP_TP];
     const int ld = cs + 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ns = blockIdx.y, pix0 = blockIdx.x * IMP_TP;
+    // several frames per launch: frame g is compared with frame g-1 at the boundary, not with the snapshot, which
+    // only the last frame writes (all of it)
+    const bool seq = DELTA && sf.frames > 1;
+    T* s_p = s_x + IMP_TP * ld;
+    if (seq) {
+        const long long g = blockIdx.z;
+        src += g * sf.in_stride;
+        D = shift_bytes(D, g * sf.row_stride);
+        act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
+        npix = shift_bytes(npix, g * sf.arena_stride);
+        shift_readers(readers, g * sf.arena_stride);
+    }
+    const bool write_x = !seq || (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
     if (tid < IMP_TP) s_cnt[tid] = 0;
     for (int ch = warp; ch < cs; ch += 8) {
-        T v = 0;
-        if (ch < c && pix0 + lane < hw) v = src[((size_t)ns * c + ch) * hw + pix0 + lane];
+        T v = 0, pv = 0;
+        if (ch < c && pix0 + lane < hw) {
+            v = src[((size_t)ns * c + ch) * hw + pix0 + lane];
+            if (seq) pv = (src - sf.in_stride)[((size_t)ns * c + ch) * hw + pix0 + lane];
+        }
         s_x[lane * ld + ch] = v;
+        if (seq) s_p[lane * ld + ch] = pv;
     }
     __syncthreads();
     const size_t gp0 = (size_t)ns * hw + pix0;
@@ -470,10 +515,11 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
         const size_t o = (gp0 + pl) * cs + ch;
         const T xt = s_x[pl * ld + ch];
         if (DELTA) {
-            const T xp = X[o];
+            const T xp = seq ? s_p[pl * ld + ch] : X[o];
             T dv = (T)(xt - xp);
+            if (seq && write_x) X[o] = xt;
             if (xt != xp) {
-                X[o] = xt;                                   // the snapshot always moves on to the new frame
+                if (!seq) X[o] = xt;                         // the snapshot always moves on to the new frame
                 bool keep = true;
                 if (sizeof(T) == 4 && eps > 0.f) keep = fabsf((float)dv) >= eps;   // Sec. 3.4: small deltas are truncated
                 if (keep) atomicAdd(&s_cnt[pl], 1);
@@ -541,19 +587,31 @@ template <bool DELTA>
 __global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
                                                             uint32_t* act, int* pnnz, unsigned long long* nnz,
                                                             unsigned long long* npix, int* errw, int c, int h, int w,
-                                                            int pixels, Readers readers)
+                                                            int pixels, Readers readers, SeqFrames sf)
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
     const int hw = h * w;
+    const bool seq = DELTA && sf.frames > 1;                 // (see import_nchw_kernel)
+    if (seq) {
+        const long long g = blockIdx.z;
+        src += g * sf.in_stride;
+        D = shift_bytes(D, g * sf.row_stride);
+        act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
+        npix = shift_bytes(npix, g * sf.arena_stride);
+        shift_readers(readers, g * sf.arena_stride);
+    }
+    const bool write_x = !seq || (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
     int cnt = 0;
     if (gp < pixels) {
         const int ns = gp / hw, pix = gp - ns * hw;
-        uint32_t nw = 0;
+        uint32_t nw = 0, pw = 0;
         for (int ch = 0; ch < c; ++ch) nw |= ((uint32_t)(uint8_t)src[((size_t)ns * c + ch) * hw + pix]) << (8 * ch);
+        if (seq) for (int ch = 0; ch < c; ++ch) pw |= ((uint32_t)(uint8_t)(src - sf.in_stride)[((size_t)ns * c + ch) * hw + pix]) << (8 * ch);
         if (DELTA) {
-            const uint32_t ow = X[gp];
+            const uint32_t ow = seq ? pw : X[gp];
+            if (seq && write_x) X[gp] = nw;
             if (nw != ow) {
                 uint32_t dw = 0;
                 #pragma unroll
@@ -564,7 +622,7 @@ __global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __res
                     cnt += d != 0;
                 }
                 D[gp] = dw;
-                X[gp] = nw;
+                if (!seq) X[gp] = nw;
                 pnnz[gp] = cnt;
             }
         } else {
@@ -597,9 +655,20 @@ __global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __res
 template <bool DELTA>
 __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X, uint32_t* D, uint32_t* act,
                                   int* pnnz, unsigned long long* nnz, unsigned long long* npix, int cw, int pixels,
-                                  int h, int w, Readers readers, uint32_t* Xn)
+                                  int h, int w, Readers readers, uint32_t* Xn, SeqFrames sf)
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool seq = DELTA && sf.frames > 1;                 // (see import_nchw_kernel)
+    if (seq) {
+        const long long g = blockIdx.z;
+        src += g * sf.in_stride;
+        D = shift_bytes(D, g * sf.row_stride);
+        if (Xn) Xn = shift_bytes(Xn, g * sf.row_stride);
+        act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
+        npix = shift_bytes(npix, g * sf.arena_stride);
+        shift_readers(readers, g * sf.arena_stride);
+    }
+    const bool write_x = !seq || (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
     int cnt = 0;
@@ -607,11 +676,11 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
         for (int k = 0; k < cw; ++k) {
             const uint32_t xt = src[(size_t)gp * cw + k];
             if (DELTA) {
-                const uint32_t ch = xt ^ X[(size_t)gp * cw + k];
+                const uint32_t ch = xt ^ (seq ? (src - sf.in_stride)[(size_t)gp * cw + k] : X[(size_t)gp * cw + k]);
                 D[(size_t)gp * cw + k] = ch;
                 cnt += __popc(ch);
             }
-            X[(size_t)gp * cw + k] = xt;
+            if (write_x) X[(size_t)gp * cw + k] = xt;
             if (DELTA && Xn) Xn[(size_t)gp * cw + k] = xt;   // (pipelined chunk: the frame's own copy of the new rows)
         }
         if (DELTA && cnt) {
@@ -800,49 +869,16 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
                 }
             }
             // ---- f: [affine] -> [requant] -> [+ shortcut] -> act -> max over the window (sign: max first, threshold last)
-            pt best[4];
-            #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const bool live = c + j < p.c_out;
-                pt res = 0;
-                pt bn_m = 1, bn_a = 0;                       // the channel's affine (Sec. 4.5: BN as part of f)
-                if (BN && live) {
-                    bn_m = reinterpret_cast<const pt*>(p.bn_scale)[c + j];
-                    bn_a = reinterpret_cast<const pt*>(p.bn_shift)[c + j];
-                }
-                if (live && p.resX) {
-                    if (PT == T_F32) res = (pt)reinterpret_cast<const float*>(p.resX)[(size_t)r * p.cs + c + j];
-                    else if (OT == T_I8) res = (pt)reinterpret_cast<const int8_t*>(p.resX)[(size_t)r * p.cs + c + j];
-                }
-                bool have = false;
-                pt b = 0;
+            pt best[4], res[4] = {0, 0, 0, 0};
+            if (p.resX) {
                 #pragma unroll
-                for (int wi = 0; wi < KW * KW; ++wi) {
-                    if (!(inside >> wi & 1u)) continue;
-                    pt x = v[wi][j];
-                    if (PT == T_F32) {
-                        if (BN) x = (pt)fmaf((float)x, (float)bn_m, (float)bn_a);
-                        x += res;
-                        if (p.act_fn == RRM_ACT_RELU) x = x > 0 ? x : 0;
-                        else if (p.act_fn == RRM_ACT_LEAKY) x = x > 0 ? x : (pt)(0.1f * (float)x);
-                    } else if (OT == T_I8) {
-                        int iv = (int)x;
-                        if (BN) {                            // integer multiplier and offset inside the requantisation, 64-bit exact
-                            long long t = (long long)iv * (long long)(int)bn_m + (long long)(int)bn_a;
-                            if (p.shift > 0) t = (t + (1ll << (p.shift - 1))) >> p.shift;
-                            iv = (int)max(-127ll, min(127ll, t));
-                        } else {
-                            if (p.shift > 0) iv = (iv + (1 << (p.shift - 1))) >> p.shift;
-                            iv = max(-127, min(127, iv));
-                        }
-                        iv += (int)res;
-                        iv = (p.act_fn == RRM_ACT_RELU) ? max(0, min(127, iv)) : max(-127, min(127, iv));
-                        x = (pt)iv;
-                    }
-                    if (!have || x > b) { b = x; have = true; }
+                for (int j = 0; j < 4; ++j) {
+                    if (c + j >= p.c_out) continue;
+                    if (PT == T_F32) res[j] = (pt)reinterpret_cast<const float*>(p.resX)[(size_t)r * p.cs + c + j];
+                    else if (OT == T_I8) res[j] = (pt)reinterpret_cast<const int8_t*>(p.resX)[(size_t)r * p.cs + c + j];
                 }
-                best[j] = live ? b : (pt)0;
             }
+            epi_f<PT, OT, KW, BN, pt>(v, inside, c, res, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, best);
             // ---- compare with the stored activation, emit delta row and snapshot
             if (OT == T_BIN) {
                 unsigned bits = 0;
@@ -1087,31 +1123,42 @@ int ensure_stateless(rrm_net* net)
     return RRM_OK;
 }
 
-int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, cudaStream_t st)
+// frames > 1 (delta only): `frame` is the first of that many consecutive frames at the boundary, the frame before it
+// lies right in front of them; frame g's delta rows, new rows and arena follow frame 0's (the bound ones) at the
+// tensor's size / arena_stride bytes each.  The snapshot ends up as the last frame.
+int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, cudaStream_t st, int frames, long long arena_stride)
 {
     if (stateless) RRM_TRY(ensure_stateless(net));
     Tensor& T = net->tensors[0];
     void* X = stateless ? T.X2 : T.X;
     const int hw = T.h * T.w;
+    const bool seq = frames > 1 && delta && !stateless;
+    const unsigned gz = seq ? (unsigned)frames : 1u;
+    SeqFrames sf{};
+    if (seq) {
+        sf.frames = frames; sf.row_stride = (long long)T.bytes(); sf.arena_stride = arena_stride;
+        sf.in_stride = T.dtype == T_BIN ? (long long)T.pixels() * T.cs : (long long)T.n * T.c * hw;
+    }
     if (T.dtype == T_BIN) {
         const int blocks = ceil_div(T.pixels(), 256);
-        if (delta) launch_seq(import_bin_kernel<true>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, (uint32_t*)T.D,
+        if (delta) launch_seq(import_bin_kernel<true>, dim3(blocks, 1, gz), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, (uint32_t*)T.D,
                                                                   T.act, T.pnnz, T.nnz, T.npix, T.cs, T.pixels(),
-                                                                  T.h, T.w, T.readers, (uint32_t*)(stateless ? nullptr : T.Xn_cur));
+                                                                  T.h, T.w, T.readers, (uint32_t*)(stateless ? nullptr : T.Xn_cur), sf);
         else launch_seq(import_bin_kernel<false>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)frame, (uint32_t*)X, nullptr, nullptr,
                                                               nullptr, nullptr, nullptr, T.cs, T.pixels(), T.h, T.w,
-                                                              Readers{}, (uint32_t*)nullptr);
+                                                              Readers{}, (uint32_t*)nullptr, sf);
     } else if (T.dtype == T_I8 && T.cs == 4) {
         const int blocks = ceil_div(T.pixels(), 256);
-        if (delta) launch_seq(import_i8_word_kernel<true>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
+        if (delta) launch_seq(import_i8_word_kernel<true>, dim3(blocks, 1, gz), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
                                                                       T.pnnz, T.nnz, T.npix, net->errw, T.c, T.h, T.w,
-                                                                      T.pixels(), T.readers);
+                                                                      T.pixels(), T.readers, sf);
         else launch_seq(import_i8_word_kernel<false>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, nullptr, nullptr, nullptr,
                                                                   nullptr, nullptr, net->errw, T.c, T.h, T.w, T.pixels(),
-                                                                  Readers{});
+                                                                  Readers{}, sf);
     } else {
-        dim3 grid(ceil_div(hw, IMP_TP), T.n);
-        const size_t smem = (size_t)IMP_TP * (T.cs + 1) * T.unit_bytes;
+        dim3 grid(ceil_div(hw, IMP_TP), T.n, gz);
+        const size_t smem = (size_t)IMP_TP * (T.cs + 1) * T.unit_bytes * (seq ? 2 : 1);
+        if (smem > 200 * 1024) return RRM_ERR_UNSUPPORTED;
         if (T.dtype == T_F32) {
             auto kd = import_nchw_kernel<float, true>;
             auto kn = import_nchw_kernel<float, false>;
@@ -1120,9 +1167,9 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                 cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             }
             if (delta) launch_seq(kd, dim3(grid), dim3(256), smem, st, (const float*)frame, (float*)X, (float*)T.D, T.act, T.pnnz, T.nnz,
-                                                   T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, net->eps, T.trunc);
+                                                   T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, net->eps, T.trunc, sf);
             else launch_seq(kn, dim3(grid), dim3(256), smem, st, (const float*)frame, (float*)X, nullptr, nullptr, nullptr, nullptr,
-                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr);
+                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr, sf);
         } else {
             auto kd = import_nchw_kernel<int8_t, true>;
             auto kn = import_nchw_kernel<int8_t, false>;
@@ -1131,9 +1178,9 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                 cudaFuncSetAttribute(kn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             }
             if (delta) launch_seq(kd, dim3(grid), dim3(256), smem, st, (const int8_t*)frame, (int8_t*)X, (int8_t*)T.D, T.act, T.pnnz,
-                                                   T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, 0.f, nullptr);
+                                                   T.nnz, T.npix, net->errw, T.c, T.cs, hw, T.w, T.readers, 0.f, nullptr, sf);
             else launch_seq(kn, dim3(grid), dim3(256), smem, st, (const int8_t*)frame, (int8_t*)X, nullptr, nullptr, nullptr, nullptr,
-                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr);
+                                             nullptr, net->errw, T.c, T.cs, hw, T.w, Readers{}, 0.f, nullptr, sf);
         }
     }
     RRM_CUDA_TRY(cudaGetLastError());
@@ -1203,7 +1250,8 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     Tensor& out = net->tensors[l + 1];
     Tensor* res = d.res >= 0 ? &net->tensors[d.res] : nullptr;
 
-    ConvParams p;
+    ConvParams p{};
+    p.frames = 1;
     p.D = in.D; p.X = stateless ? in.X2 : (split && in.Xn_cur ? in.Xn_cur : in.X); p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
     p.Wk = L.Wk; p.bias = L.bias; p.P = split ? split->dP : (stateless ? L.P2 : L.P);
     p.n = d.n; p.c_in = d.c_in; p.h = d.h; p.w = d.w; p.u_in = L.u_in; p.oh = L.oh; p.ow = L.ow;
@@ -1226,7 +1274,7 @@ int launch_layer(rrm_net* net, int l, bool dense, bool stateless, cudaStream_t s
     else { if (conv_dense) launch_gemm<T_BIN, true>(p, grid, st); else launch_gemm<T_BIN, false>(p, grid, st); }
 
     if (hook) RRM_TRY((*hook)(1));
-    EpiParams e;
+    EpiParams e{};
     e.P = split ? split->R : p.P; e.oact = step_dense ? net->ones : L.oact;     // (dense inside a delta step: every window is looked at)
     e.dP = split ? split->dP : nullptr; e.Q = split ? split->Q : nullptr; e.Z = split ? split->Z : nullptr;
     e.oact_prev = split ? split->prev_oact : nullptr; e.opix = L.opixels(); e.Xn = split ? out.Xn_cur : nullptr;

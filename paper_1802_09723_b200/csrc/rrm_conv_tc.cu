@@ -51,6 +51,13 @@ struct TcParams {
     unsigned wait_limit;      // polls of one bounded wait
     const uint32_t* count_bitmap;   // dense evaluation inside a delta step: the layer's update bitmap, whose set bits the
                                     // first CTA counts into *ocount (the measured activity); nullptr otherwise
+    // several frames in one launch (delta only; gridDim.z = frames x ksplit): frame g reads its delta rows, new rows
+    // and bitmaps, and writes its product, at these distances from frame 0's
+    int frames;
+    long long row_stride;     // bytes between the frames' sets of delta rows (and of new rows)
+    long long arena_stride;   // bytes between the frames' arenas (bitmaps, counters)
+    long long p_stride;       // elements between the frames' products
+    int store;                // delta: the product is stored, not added (ksplit 1: every row written belongs to one CTA)
 };
 
 // byte i of the result = bit i of the low nibble of x (0 or 1)
@@ -76,7 +83,16 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
 {
     extern __shared__ unsigned char tc_smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tile = blockIdx.x, ntile = blockIdx.y, split = blockIdx.z;
+    const int tile = blockIdx.x, ntile = blockIdx.y;
+    const int frame = (!DENSE && p.frames > 1) ? blockIdx.z / p.ksplit : 0, split = blockIdx.z - frame * p.ksplit;
+    if (!DENSE && frame > 0) {
+        p.A = reinterpret_cast<const char*>(p.A) + frame * p.row_stride;
+        p.Anew = reinterpret_cast<const char*>(p.Anew) + frame * p.row_stride;
+        p.in_act = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.in_act) + frame * p.arena_stride);
+        p.oact = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.oact) + frame * p.arena_stride);
+        p.ocount = reinterpret_cast<int*>(reinterpret_cast<char*>(p.ocount) + frame * p.arena_stride);
+        p.P += frame * p.p_stride;
+    }
     unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
     TcSmemTail* S = reinterpret_cast<TcSmemTail*>(base + TC_STAGES * TC_STAGE_BYTES);
     const uint32_t base_u32 = smem_u32(base);
@@ -425,6 +441,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                         if (DENSE) {
                             const int b = (split == 0 && p.bias) ? p.bias[co] : 0;
                             if (atomic) atomicAdd(dst, val + b); else *dst = val + b;
+                        } else if (p.store) {
+                            *dst = val;
                         } else if (val != 0) {
                             atomicAdd(dst, val);
                         }
@@ -435,7 +453,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                 fence_async_smem();                          // this thread's row -> visible to the copy engine
                 int32_t* dst = p.P + (size_t)q * p.c_out + n0;
                 const uint32_t bytes = (uint32_t)ncols * 4u;
-                if (DENSE && !atomic)
+                if ((DENSE && !atomic) || (!DENSE && p.store))
                     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                                  ::"l"(dst), "r"(smem_u32(row)), "r"(bytes) : "memory");
                 else                                         // with a split K of a dense pass the projection was zeroed beforehand
@@ -540,11 +558,14 @@ int conv_tc_create(rrm_net* net, Layer& L, const void* W_dev)
 
 // F*dI (dense: F*X + b) on the tensor cores; P is updated in place (dense: overwritten).  P_dst (delta only): the
 // product is added there instead of onto the stored projection.
+// frames > 1 (delta only): that many frames in one launch; the tensor's delta rows and new rows, the bound arena and
+// P_dst are frame 0's, the other frames' lie the tensor's size / arena_stride bytes and one projection further each;
+// K is not split and the products are stored.
 int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool stateless, cudaStream_t st,
-                   const uint32_t* count_bitmap, void* P_dst)
+                   const uint32_t* count_bitmap, void* P_dst, int frames, long long arena_stride)
 {
     const rrm_layer_desc& d = L.d;
-    TcParams p;
+    TcParams p{};
     const bool bin = d.dtype == RRM_BIN;
     const void* X = stateless ? in.X2 : in.X;
     p.A = bin ? in.D : (dense ? X : in.D);
@@ -561,6 +582,10 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.slabs = L.tc_slabs; p.bn = L.tc_bn;
     p.wait_limit = net->opt.wait_limit;
     p.count_bitmap = count_bitmap;
+    const bool batched = frames > 1 && !dense;
+    p.frames = batched ? frames : 1;
+    p.row_stride = (long long)in.bytes(); p.arena_stride = arena_stride; p.p_stride = (long long)L.opixels() * d.c_out;
+    p.store = batched ? 1 : 0;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
     // split K towards the point where a CTA's slabs all fit in its pipeline at once
     // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the
@@ -571,14 +596,14 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     int ksplit = 1;
     const int ks_max = ceil_div(L.tc_slabs, TC_STAGES);
     const long long tiles = (long long)m_tiles * L.tc_ntiles;
-    while (ksplit < ks_max && tiles * ksplit < wave) ++ksplit;
+    while (!batched && ksplit < ks_max && tiles * ksplit < wave) ++ksplit;
     ksplit = ceil_div(L.tc_slabs, ceil_div(L.tc_slabs, ksplit));   // no empty shares
     p.ksplit = ksplit;
     if (dense && ksplit > 1) {
         const long long tot = (long long)L.opixels() * d.c_out;
         launch_seq(zero_projection_kernel, dim3((unsigned)((tot + 255) / 256)), dim3(256), 0, st, p.P, tot);
     }
-    dim3 grid(m_tiles, L.tc_ntiles, ksplit);
+    dim3 grid(m_tiles, L.tc_ntiles, ksplit * p.frames);
     if (bin) {
         if (dense) launch_seq(conv_tc_kernel<true, true>, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, p);
         else launch_seq(conv_tc_kernel<true, false>, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, p);

@@ -3,6 +3,7 @@
 // the two convolution kernels.
 #pragma once
 #include <cstdint>
+#include <type_traits>
 #include <cuda_runtime.h>
 #include "../../include/rrm.h"
 
@@ -106,6 +107,61 @@ __device__ __forceinline__ void row_tap_masks(const uint32_t* __restrict__ in_ac
                 if (t < 64) m0 |= 1ull << t; else m1 |= 1ull << (t - 64);
             }
         }
+    }
+}
+
+// pointer + byte offset
+template <typename P>
+__device__ __forceinline__ P* shift_bytes(P* p, long long bytes)
+{
+    return reinterpret_cast<P*>(reinterpret_cast<char*>(const_cast<typename std::remove_const<P>::type*>(p)) + bytes);
+}
+
+// f of Algorithm 1 on the 4 neighbouring channels c .. c+3 of one output pixel: [affine] -> [requantisation] -> [+ shortcut]
+// -> activation -> max over the pool window (a sign activation takes the max first, its threshold is the caller's).
+// v: the projection at the window's positions (bit wi of `inside`: position wi lies inside the projection);
+// res: the shortcut's values; PT: projection type, OT: output storage type, KW: window edge, BN: the explicit
+// per-channel affine of Sec. 4.5 (fp32: y = scale * P + shift; int8: multiplier and offset inside the requantisation).
+template <int PT, int OT, int KW, bool BN, typename pt>
+__device__ __forceinline__ void epi_f(const pt (&v)[KW * KW][4], unsigned inside, int c, const pt (&res)[4], int c_out,
+                                      int act_fn, int shift, const void* bn_scale, const void* bn_shift, pt (&best)[4])
+{
+    #pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool live = c + j < c_out;
+        pt bn_m = 1, bn_a = 0;
+        if (BN && live) {
+            bn_m = reinterpret_cast<const pt*>(bn_scale)[c + j];
+            bn_a = reinterpret_cast<const pt*>(bn_shift)[c + j];
+        }
+        bool have = false;
+        pt b = 0;
+        #pragma unroll
+        for (int wi = 0; wi < KW * KW; ++wi) {
+            if (!(inside >> wi & 1u)) continue;
+            pt x = v[wi][j];
+            if (PT == T_F32) {
+                if (BN) x = (pt)fmaf((float)x, (float)bn_m, (float)bn_a);
+                x += res[j];
+                if (act_fn == RRM_ACT_RELU) x = x > 0 ? x : 0;
+                else if (act_fn == RRM_ACT_LEAKY) x = x > 0 ? x : (pt)(0.1f * (float)x);
+            } else if (OT == T_I8) {
+                int iv = (int)x;
+                if (BN) {                                    // 64-bit exact
+                    long long t = (long long)iv * (long long)(int)bn_m + (long long)(int)bn_a;
+                    if (shift > 0) t = (t + (1ll << (shift - 1))) >> shift;
+                    iv = (int)max(-127ll, min(127ll, t));
+                } else {
+                    if (shift > 0) iv = (iv + (1 << (shift - 1))) >> shift;
+                    iv = max(-127, min(127, iv));
+                }
+                iv += (int)res[j];
+                iv = (act_fn == RRM_ACT_RELU) ? max(0, min(127, iv)) : max(-127, min(127, iv));
+                x = (pt)iv;
+            }
+            if (!have || x > b) { b = x; have = true; }
+        }
+        best[j] = live ? b : (pt)0;
     }
 }
 
