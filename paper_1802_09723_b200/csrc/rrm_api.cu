@@ -212,6 +212,8 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         net->graph_off = e && e[0] == '1';
         e = getenv("RRM_CHUNK_INPLACE");
         net->chunk_in_place = e && e[0] == '1';
+        e = getenv("RRM_CHUNK_PIPELINED");
+        net->chunk_pipelined = e && e[0] == '1';
     }
     for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
     RRM_TRY(bind_readers(net));
@@ -519,11 +521,85 @@ int ensure_chunk(rrm_net* net, int T)
         tensor_bytes_boundary(net->tensors.back(), &bo);
         RRM_CUDA_TRY(cudaDeviceSynchronize());               // the old buffers may be in use by a graph in flight
         for (int k = 0; k < 3; ++k) drop_chunk_graphs(net, k);   // graphs hold the old buffers
-        dev_release(net, &net->chunk_in);
+        dev_release(net, &net->chunk_in_raw);
         dev_release(net, &net->chunk_out);
-        RRM_TRY(dev_alloc(net, &net->chunk_in, (size_t)bi * T));
+        {
+            // room for one frame in front of the chunk (the layer-by-layer form compares frame 0 with it), aligned
+            const size_t front = ((size_t)bi + 255) & ~(size_t)255;
+            RRM_TRY(dev_alloc(net, &net->chunk_in_raw, front + (size_t)bi * T));
+            net->chunk_in = reinterpret_cast<char*>(net->chunk_in_raw) + front;
+        }
         RRM_TRY(dev_alloc(net, &net->chunk_out, (size_t)bo * T));
         net->chunk_cap = T;
+    }
+    return RRM_OK;
+}
+
+// Inserts a captured chunk graph into the cache of its kind (the few most recently used are kept).
+static int keep_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask, cudaGraph_t g, int last_arena)
+{
+    auto& cache = net->chunk_graphs[kind];
+    if (cache.size() >= CHUNK_GRAPHS_KEPT) {
+        size_t old = 0;
+        for (size_t i = 1; i < cache.size(); ++i) if (cache[i].used < cache[old].used) old = i;
+        if (cache[old].exec) cudaGraphExecDestroy(cache[old].exec);
+        if (cache[old].graph) cudaGraphDestroy(cache[old].graph);
+        cache.erase(cache.begin() + old);
+    }
+    rrm_net::ChunkGraph c;
+    c.T = T; c.mask = mask; c.graph = g; c.last_arena = last_arena;
+    if (cudaGraphInstantiate(&c.exec, g, 0) != cudaSuccess) { cudaGraphDestroy(g); cudaGetLastError(); return RRM_ERR_CUDA; }
+    c.used = ++net->chunk_clock;
+    cache.push_back(c);
+    return RRM_OK;
+}
+
+// A delta chunk layer by layer: every kernel takes all frames of the chunk (at most seq_max_frames() per launch; a
+// longer chunk goes in equal parts one after the other).  2 L + 5 launches per part, no frame-to-frame edges.
+// RRM_ERR_UNSUPPORTED: the stack has shortcuts or would need too much memory (the frame-pipelined graph serves it).
+static int build_seq_graph(rrm_net* net, int T)
+{
+    const int L = (int)net->layers.size();
+    RRM_TRY(ensure_chunk(net, T));
+    RRM_TRY(ensure_frame_batch(net));
+    const int parts = ceil_div(T, seq_max_frames()), per = ceil_div(T, parts);       // (T >= 2: every part holds >= 2 frames)
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    const long long stride = (long long)net->cleared_bytes;
+    cudaStream_t st = net->cap_stream;
+    std::vector<void*> keep_D;
+    for (auto& X : net->tensors) keep_D.push_back(X.D);
+    int status = RRM_OK, last_arena = 0;
+    auto fail = [&](int s) { if (status == RRM_OK && s != RRM_OK) status = s; };
+    RRM_CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    for (int m0 = 0; m0 < T && status == RRM_OK; m0 += per) {
+        const int F = T - m0 < per ? T - m0 : per;
+        if (cudaMemsetAsync(net->chunk_arena[0], 0, net->cleared_bytes * F, st) != cudaSuccess) fail(RRM_ERR_CUDA);
+        fail(launch_copy_projections(net, st));              // the epilogues read the projections from the copies and write the stored ones
+        bind_arena(net, net->chunk_arena[0]);
+        if (bind_readers(net) != RRM_OK) { fail(RRM_ERR_UNSUPPORTED); break; }
+        for (auto& X : net->tensors) { X.D = X.Dall; X.Xn_cur = X.Xnall; }
+        char* in0 = reinterpret_cast<char*>(net->chunk_in) + (size_t)m0 * bi;
+        if (m0 == 0) fail(launch_export_tensor(net, 0, in0 - bi, false, st));        // the frame before the chunk = the input's snapshot
+        fail(launch_import(net, in0, true, false, st, F, stride));
+        for (int l = 0; l < L && status == RRM_OK; ++l) fail(launch_layer_seq(net, l, F, stride, st));
+        fail(launch_export_seq(net, F, reinterpret_cast<char*>(net->chunk_out) + (size_t)m0 * bo, st));
+        last_arena = F - 1;
+    }
+    for (size_t i = 0; i < net->tensors.size(); ++i) { net->tensors[i].D = keep_D[i]; net->tensors[i].Xn_cur = nullptr; }
+    cudaGraph_t g = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(st, &g);
+    if (status != RRM_OK || e != cudaSuccess || !g) {
+        if (g) cudaGraphDestroy(g);
+        cudaGetLastError();
+        return status != RRM_OK ? status : RRM_ERR_CUDA;
+    }
+    RRM_TRY(keep_chunk_graph(net, 0, T, 0, g, last_arena));
+    if (getenv("RRM_DEBUG")) {
+        size_t nodes = 0;
+        cudaGraphGetNodes(g, nullptr, &nodes);
+        fprintf(stderr, "rrm: chunk graph (delta, %d frames, layer by layer): %zu nodes, %d part(s)\n", T, nodes, parts);
     }
     return RRM_OK;
 }
@@ -549,6 +625,11 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
 {
     const bool dense = kind != 0, stateless = kind == 2;
     const int L = (int)net->layers.size();
+    if (kind == 0 && mask == 0 && !net->chunk_in_place && !net->chunk_pipelined) {
+        const int s = build_seq_graph(net, T);
+        if (s != RRM_ERR_UNSUPPORTED && s != RRM_ERR_ALLOC) return s;
+        cudaGetLastError();
+    }
     RRM_TRY(ensure_chunk(net, T));
     if (stateless) RRM_TRY(ensure_stateless(net));
     const bool split = kind == 0 && mask == 0 && !net->chunk_in_place;
@@ -647,19 +728,7 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
         return status != RRM_OK ? status : RRM_ERR_CUDA;
     }
     // keep the few most recently used chunk lengths (a video's last chunk is usually shorter than the others)
-    auto& cache = net->chunk_graphs[kind];
-    if (cache.size() >= CHUNK_GRAPHS_KEPT) {
-        size_t old = 0;
-        for (size_t i = 1; i < cache.size(); ++i) if (cache[i].used < cache[old].used) old = i;
-        if (cache[old].exec) cudaGraphExecDestroy(cache[old].exec);
-        if (cache[old].graph) cudaGraphDestroy(cache[old].graph);
-        cache.erase(cache.begin() + old);
-    }
-    rrm_net::ChunkGraph c;
-    c.T = T; c.mask = mask; c.graph = g;
-    if (cudaGraphInstantiate(&c.exec, g, 0) != cudaSuccess) { cudaGraphDestroy(g); cudaGetLastError(); return RRM_ERR_CUDA; }
-    c.used = ++net->chunk_clock;
-    cache.push_back(c);
+    RRM_TRY(keep_chunk_graph(net, kind, T, mask, g, own_arena ? T - 1 : (T - 1) % S));
     if (getenv("RRM_DEBUG")) {
         size_t nodes = 0;
         cudaGraphGetNodes(g, nullptr, &nodes);
@@ -706,8 +775,7 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
         }
     }
     // the structures describe the last frame of the chunk from here on (statistics, activity read-back)
-    const int S = (int)net->chunk_streams.size() < T ? (int)net->chunk_streams.size() : T;
-    bind_arena(net, net->chunk_arena[T <= CHUNK_ARENAS ? T - 1 : (T - 1) % S]);
+    bind_arena(net, net->chunk_arena[find()->last_arena]);
     RRM_TRY(bind_readers(net));
     int64_t bi = 0, bo = 0;
     tensor_bytes_boundary(net->tensors.front(), &bi);

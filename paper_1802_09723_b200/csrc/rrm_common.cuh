@@ -129,6 +129,11 @@ struct Tensor {
     // pipelined chunk keeps a copy of the new rows per frame parity; Xn_cur is set only while such a chunk is captured
     void* Xn[CHUNK_RING] = {};
     void* Xn_cur = nullptr;
+    // delta chunks taken layer by layer over all frames (rrm_conv_seq.cu): per-frame delta rows, per-frame new rows
+    // (binary tensors), and for the stack's last tensor every frame's full rows; SEQ_MAX_FRAMES of each
+    void* Dall = nullptr;
+    void* Xnall = nullptr;
+    void* Xfull = nullptr;
     bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
     Readers readers{};                // the layers that read it
     int pixels() const { return n * h * w; }
@@ -156,6 +161,7 @@ struct Layer {
     void* Palt = nullptr;             // the second projection buffer (a copy of P is made at the start of a chunk)
     void* dP[CHUNK_RING] = {};
     size_t oact_off = 0;              // offset of the update bitmap inside an arena
+    void* dPall = nullptr;            // per-frame products of the layer-by-layer chunk form
     uint32_t* oact = nullptr;         // bitmap of projection pixels to update (cleared every step, set by the
                                       // kernels that produce the layer's input and shortcut tensors)
     int* ocount = nullptr;            // their number (cleared every step, written by the convolution kernel)
@@ -269,14 +275,18 @@ struct rrm_net {
     // `slot` (frame mod CHUNK_RING in the split form; slot 0 only otherwise)
     std::vector<cudaEvent_t> ev_conv, ev_epi;
     cudaEvent_t ev_import = nullptr;
+    bool seq_ready = false;                       // the buffers of the layer-by-layer chunk form exist
+    bool chunk_pipelined = false;                 // RRM_CHUNK_PIPELINED=1: delta chunks overlap frames instead of batching them per layer
     bool chunk_in_place = false;                  // RRM_CHUNK_INPLACE=1: delta chunks add into the stored projection (no delta-projection buffers)
     uint32_t* zeros = nullptr;                    // an all-zero bitmap as long as the longest update bitmap
     std::vector<cudaEvent_t> ev_join;
     cudaEvent_t ev_fork = nullptr, ev_export = nullptr;
-    struct ChunkGraph { int T = 0; unsigned long long mask = 0; cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr; unsigned long long used = 0; };
+    struct ChunkGraph { int T = 0; unsigned long long mask = 0; cudaGraph_t graph = nullptr; cudaGraphExec_t exec = nullptr; unsigned long long used = 0;
+                        int last_arena = 0; /* the arena that holds the chunk's last frame */ };
     std::vector<ChunkGraph> chunk_graphs[3];      // per kind (delta / keyframes / dense): the few most recently used chunk lengths
     unsigned long long chunk_clock = 0;
-    void* chunk_in = nullptr;
+    void* chunk_in = nullptr;                     // T frames at the boundary; one more frame fits right in front of them
+    void* chunk_in_raw = nullptr;                 // (the allocation chunk_in points into)
     void* chunk_out = nullptr;
     int chunk_cap = 0;                            // frames chunk_in / chunk_out hold
     // measured activity of the last delta step, read back without stalling the stream: when nearly every
@@ -349,6 +359,13 @@ int reset_state(rrm_net* net, cudaStream_t st);
 int ensure_stateless(rrm_net* net);
 int launch_aecs(rrm_net* net, cudaStream_t st);
 int ensure_split(rrm_net* net);
+int launch_layer_seq(rrm_net* net, int l, int frames, long long arena_stride, cudaStream_t st);
+int launch_export_seq(rrm_net* net, int frames, void* dst_dev, cudaStream_t st);
+
+// ---- rrm_conv_seq.cu
+int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride, cudaStream_t st);
+int ensure_frame_batch(rrm_net* net);
+int seq_max_frames();
 int launch_copy_projections(rrm_net* net, cudaStream_t st);
 int launch_zero_delta_projections(rrm_net* net, int slot, cudaStream_t st);
 int clear_split(rrm_net* net, cudaStream_t st);

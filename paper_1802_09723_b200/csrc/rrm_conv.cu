@@ -455,17 +455,6 @@ __global__ void pack_weights_kernel(const void* W, uint32_t* Wk, int dt, int c_i
 // One CTA handles 32 consecutive pixels of one stream: coalesced reads along w, transposed through
 // shared memory, coalesced pixel-major writes.
 // ------------------------------------------------------------------------------------------------
-// the readers' bitmaps and counters of frame g's arena
-__device__ __forceinline__ void shift_readers(Readers& R, long long bytes)
-{
-    #pragma unroll
-    for (int i = 0; i < MAX_READERS; ++i) {
-        if (i >= R.n) break;
-        R.r[i].oact = shift_bytes(R.r[i].oact, bytes);
-        if (R.r[i].macs) R.r[i].macs = shift_bytes(R.r[i].macs, bytes);
-    }
-}
-
 constexpr int IMP_TP = 32;                  // pixels per tile = lanes of the warp that marks their footprints
 
 template <typename T, bool DELTA>
@@ -981,9 +970,12 @@ __global__ void __launch_bounds__(256) epilogue_kernel(EpiParams p)
 // Exports to the boundary layout.
 // ------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void export_nchw_kernel(const T* __restrict__ src, T* dst, int c, int cs, int hw, long long total)
+__global__ void export_nchw_kernel(const T* __restrict__ src, T* dst, int c, int cs, int hw, long long total,
+                                   long long src_stride = 0, long long dst_stride = 0)   // elements between frames (frame = blockIdx.y)
 {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    src += blockIdx.y * src_stride;
+    dst += blockIdx.y * dst_stride;
     pdl_launch_dependents();
     pdl_wait();
     if (i >= total) return;
@@ -1400,10 +1392,61 @@ int launch_export_tensor(rrm_net* net, int t, void* dst, bool stateless, cudaStr
     const int hw = T.h * T.w;
     const long long total = (long long)T.n * T.c * hw;
     const int blocks = (int)((total + 255) / 256);
-    if (T.dtype == T_I8) launch_seq(export_nchw_kernel<int8_t>, dim3(blocks), dim3(256), 0, st, (const int8_t*)X, (int8_t*)dst, T.c, T.cs, hw, total);
-    else launch_seq(export_nchw_kernel<uint32_t>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)X, (uint32_t*)dst, T.c, T.cs, hw, total);
+    if (T.dtype == T_I8) launch_seq(export_nchw_kernel<int8_t>, dim3(blocks), dim3(256), 0, st, (const int8_t*)X, (int8_t*)dst, T.c, T.cs, hw, total, 0ll, 0ll);
+    else launch_seq(export_nchw_kernel<uint32_t>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)X, (uint32_t*)dst, T.c, T.cs, hw, total, 0ll, 0ll);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
+}
+
+// Every frame's output of the layer-by-layer chunk form (the last tensor's full rows) to the boundary layout.
+int launch_export_seq(rrm_net* net, int frames, void* dst, cudaStream_t st)
+{
+    Tensor& T = net->tensors.back();
+    if (!T.Xfull) return RRM_ERR_INVALID_ARG;
+    if (T.dtype == T_BIN) {
+        RRM_CUDA_TRY(cudaMemcpyAsync(dst, T.Xfull, T.bytes() * frames, cudaMemcpyDeviceToDevice, st));
+        return RRM_OK;
+    }
+    const int hw = T.h * T.w;
+    const long long total = (long long)T.n * T.c * hw;
+    const dim3 grid((unsigned)((total + 255) / 256), (unsigned)frames);
+    if (T.dtype == T_I8) launch_seq(export_nchw_kernel<int8_t>, grid, dim3(256), 0, st, (const int8_t*)T.Xfull, (int8_t*)dst, T.c, T.cs, hw, total,
+                                    (long long)T.bytes(), total);
+    else launch_seq(export_nchw_kernel<uint32_t>, grid, dim3(256), 0, st, (const uint32_t*)T.Xfull, (uint32_t*)dst, T.c, T.cs, hw, total,
+                    (long long)T.bytes() / 4, total);
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
+// Layer l over `frames` consecutive frames in two launches: the sparse products of all frames, each stored in a buffer
+// of its own (rows of the updated pixels), then the epilogue that walks the frames in order (rrm_conv_seq.cu).  The
+// bound arena and the tensors' D / Xn_cur are frame 0's.
+int launch_layer_seq(rrm_net* net, int l, int frames, long long arena_stride, cudaStream_t st)
+{
+    Layer& L = net->layers[l];
+    const rrm_layer_desc& d = L.d;
+    Tensor& in = net->tensors[d.src];
+    if (!L.dPall || frames < 1) return RRM_ERR_INVALID_ARG;
+    if (L.tc_ready) RRM_TRY(launch_conv_tc(net, L, in, false, false, st, nullptr, L.dPall, frames, arena_stride));
+    else {
+        ConvParams p{};
+        p.D = in.D; p.X = in.Xn_cur ? in.Xn_cur : in.X; p.in_act = in.act; p.oact = L.oact; p.ocount = L.ocount;
+        p.Wk = L.Wk; p.bias = L.bias; p.P = L.dPall;
+        p.n = d.n; p.c_in = d.c_in; p.h = d.h; p.w = d.w; p.u_in = L.u_in; p.oh = L.oh; p.ow = L.ow;
+        p.kh = d.kh; p.kw = d.kw; p.stride = d.stride; p.pad = d.pad; p.c_out = d.c_out; p.np = L.np;
+        p.ku = L.ku; p.kup = L.kup; p.opixels = L.opixels();
+        p.wait_limit = net->opt.wait_limit;
+        p.errw = net->errw;
+        p.ksplit = 1;
+        p.frames = frames > 1 ? frames : 2;                  // (one frame still takes the storing form: the kernel tests frames > 1)
+        p.row_stride = (long long)in.bytes(); p.arena_stride = arena_stride; p.p_stride = (long long)L.opixels() * d.c_out;
+        dim3 grid(ceil_div(L.opixels(), TM), L.np / TN, frames);
+        if (d.dtype == RRM_F32) launch_gemm<T_F32, false>(p, grid, st);
+        else if (d.dtype == RRM_I8) launch_gemm<T_I8, false>(p, grid, st);
+        else launch_gemm<T_BIN, false>(p, grid, st);
+    }
+    RRM_CUDA_TRY(cudaGetLastError());
+    return launch_epilogue_seq(net, l, frames, arena_stride, st);
 }
 
 int launch_export_projection(rrm_net* net, int l, void* dst, cudaStream_t st)
@@ -1412,7 +1455,7 @@ int launch_export_projection(rrm_net* net, int l, void* dst, cudaStream_t st)
     const int hw = L.oh * L.ow;
     const long long total = (long long)L.d.n * L.d.c_out * hw;
     launch_seq(export_nchw_kernel<uint32_t>, dim3((int)((total + 255) / 256)), dim3(256), 0, st, (const uint32_t*)L.P, (uint32_t*)dst,
-                                                                            L.d.c_out, L.d.c_out, hw, total);
+                                                                            L.d.c_out, L.d.c_out, hw, total, 0ll, 0ll);
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }

@@ -1,0 +1,413 @@
+// A chunk of consecutive frames through a stack, layer by layer (rrm_net_step_seq on delta chunks; the remark at the
+// end of Sec. 3.2: a video may be handed over in chunks).
+//
+// Algorithm 1 is serial in t only through the state a layer keeps: the T input deltas of layer 0 are known as soon as
+// the chunk is, and once a layer has emitted its T output deltas the next layer's T sparse products F*dI_t are
+// independent of one another.  So every kernel of a step takes all frames of the chunk in one launch:
+//   import      frame g against frame g-1 at the boundary (rrm_conv.cu), delta rows and bitmaps per frame;
+//   convolution frame = blockIdx.z: the product of frame g is stored in a buffer of its own, rows of updated pixels only;
+//   epilogue    (here) lane g of a warp is frame g: P_g = P_before + sum_{t<=g} F*dI_t (Eq. 5 unrolled) is an inclusive
+//               prefix sum over the lanes, f is evaluated in every lane at once, the previous frame's output comes
+//               from the neighbouring lane, and lane g emits frame g's delta row, bitmap bit and counters; further
+//               CTAs of the same launch add the products of all frames onto the stored projection.
+// A 32-frame chunk of a five-layer stack is 15 launches instead of 384, and the chains of dependent memory round trips
+// that bound a single-frame launch are paid once per layer and chunk instead of once per layer and frame.
+#include "rrm_common.cuh"
+#include "rrm_rows.cuh"
+#include "rrm_dev.cuh"
+#include <type_traits>
+
+namespace rrm {
+
+constexpr int SEQ_MAX_FRAMES = 32;            // frames per launch: one lane of a warp per frame
+
+struct EpiSeqParams {
+    const void* P;            // the projection as of the frame before the chunk (a copy: read only)
+    void* Q;                  // the stored projection: receives P + the products of all frames at the updated pixels
+    const void* dP;           // frame 0's product (rows of the pixels in frame 0's update bitmap)
+    const uint32_t* oact;     // frame 0's update bitmap
+    void* X;                  // the output tensor's snapshot: read as the value before the chunk, left as the last frame's
+    void* D;                  // frame 0's delta rows of the output tensor
+    void* Xn;                 // frame 0's new rows (binary outputs that a layer reads: the sign of a changed bit) or nullptr
+    void* Xfull;              // or nullptr: receives every pixel's row of every frame (the stack's last tensor)
+    uint32_t* act;            // frame 0's activity bitmap of the output tensor
+    unsigned long long* nnz;
+    unsigned long long* npix;
+    int* errw;
+    int n, oh, ow, th, tw, c_out, cs, pool_k, pool_s, pool_p, act_fn, shift, theta;
+    Readers readers;          // layers that read the output tensor (frame 0's arena)
+    const void* bn_scale;
+    const void* bn_shift;
+    int frames;
+    long long row_stride;     // bytes between the frames' delta rows / new rows / full rows of the output tensor
+    long long arena_stride;   // bytes between the frames' arenas
+    long long p_stride;       // elements between the frames' products
+    int f_blocks;             // CTAs that evaluate f (one output pixel each); the CTAs behind them merge, one per bitmap word
+    int opix;                 // projection pixels
+};
+
+// Inclusive prefix sum over the lanes of a warp (lane g: sum of lanes 0 .. g), in a fixed order: the merge role and the
+// f role use the same one, so the stored projection is bit for bit the one f saw for the last frame (fp32).
+template <typename pt>
+__device__ __forceinline__ void scan4(pt (&d)[4], int lane)
+{
+    #pragma unroll
+    for (int k = 1; k < 32; k <<= 1) {
+        #pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const pt t = __shfl_up_sync(0xffffffffu, d[j], k);
+            if (lane >= k) d[j] += t;
+        }
+    }
+}
+
+// 4 neighbouring elements at P + o (o a multiple of 4 when vec); elements from `limit` on read as zero
+template <typename pt, typename pt4>
+__device__ __forceinline__ void load4(const pt* P, size_t o, bool vec, int c, int limit, pt (&v)[4])
+{
+    v[0] = v[1] = v[2] = v[3] = 0;
+    if (c >= limit) return;
+    if (vec) { const pt4 t = *reinterpret_cast<const pt4*>(P + o); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+    else {
+        #pragma unroll
+        for (int j = 0; j < 4; ++j) if (c + j < limit) v[j] = P[o + j];
+    }
+}
+
+template <int PT, int OT, int KW, bool READERS, bool BN>
+__global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
+{
+    using pt = typename std::conditional<PT == T_F32, float, int>::type;
+    using pt4 = typename std::conditional<PT == T_F32, float4, int4>::type;
+    __shared__ int s_cnt[SEQ_MAX_FRAMES];                    // changed elements of the CTA's pixel, per frame
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool vec = (p.c_out & 3) == 0;
+    pdl_launch_dependents();
+    pdl_wait();
+    if ((int)blockIdx.x >= p.f_blocks) {
+        // ---- merge role: lane g holds frame g's word of the update bitmap; a warp takes four of the word's 32 pixels
+        // and adds the frames' products in frame order, as single steps would (lanes over the channels)
+        const int w = (int)blockIdx.x - p.f_blocks;
+        unsigned bits = 0;
+        if (lane < p.frames) bits = shift_bytes(p.oact, lane * p.arena_stride)[w];
+        const pt* R = reinterpret_cast<const pt*>(p.P);
+        const pt* dP = reinterpret_cast<const pt*>(p.dP);
+        pt* Q = reinterpret_cast<pt*>(p.Q);
+        #pragma unroll 1
+        for (int k = 0; k < 4; ++k) {
+            const int b = warp * 4 + k;
+            const unsigned in_frames = __ballot_sync(0xffffffffu, (bits >> b) & 1u);
+            if (in_frames == 0) continue;
+            const size_t row = (size_t)(w * 32 + b) * p.c_out;
+            for (int c = lane * 4; c < p.c_out; c += 128) {
+                pt acc[4];
+                load4<pt, pt4>(R, row + c, vec, c, p.c_out, acc);
+                unsigned m = in_frames;
+                while (m) {                                  // four frames' rows in flight at a time
+                    int g[4];
+                    pt d[4][4];
+                    #pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        g[i] = -1;
+                        if (m) { g[i] = __ffs(m) - 1; m &= m - 1; }
+                    }
+                    #pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        d[i][0] = d[i][1] = d[i][2] = d[i][3] = 0;
+                        if (g[i] >= 0) load4<pt, pt4>(dP + (size_t)g[i] * p.p_stride, row + c, vec, c, p.c_out, d[i]);
+                    }
+                    #pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (g[i] < 0) continue;
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) acc[j] += d[i][j];
+                    }
+                }
+                if (vec) { pt4 t; t.x = acc[0]; t.y = acc[1]; t.z = acc[2]; t.w = acc[3]; *reinterpret_cast<pt4*>(Q + row + c) = t; }
+                else {
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) if (c + j < p.c_out) Q[row + c + j] = acc[j];
+                }
+            }
+        }
+        return;
+    }
+    if (threadIdx.x < SEQ_MAX_FRAMES) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    // ---- f role: this CTA's output pixel; lane = frame
+    const int r = blockIdx.x;
+    const int tx = r % p.tw, ty = (r / p.tw) % p.th, ns = r / (p.tw * p.th);
+    const int st = KW > 1 ? p.pool_s : 1, pp = KW > 1 ? p.pool_p : 0;
+    const int y0 = ty * st - pp, x0 = tx * st - pp;
+    const int qbase = ns * p.oh * p.ow;
+    // window positions inside the projection (bit wy * KW + wx); ub: the positions this lane's frame updates
+    unsigned inside, ub = 0;
+    {
+        bool mine = false;
+        if (lane < KW * KW) {
+            const int y = y0 + lane / KW, x = x0 + lane % KW;
+            mine = y >= 0 && y < p.oh && x >= 0 && x < p.ow;
+        }
+        inside = __ballot_sync(0xffffffffu, mine);
+        if (lane < p.frames) {
+            const uint32_t* oa = shift_bytes(p.oact, lane * p.arena_stride);
+            #pragma unroll
+            for (int wi = 0; wi < KW * KW; ++wi) {
+                if (!(inside >> wi & 1u)) continue;
+                const int q = qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW;
+                if ((oa[q >> 5] >> (q & 31)) & 1u) ub |= 1u << wi;
+            }
+        }
+    }
+    const unsigned on_frames = __ballot_sync(0xffffffffu, ub != 0);
+    const unsigned posmask = __reduce_or_sync(0xffffffffu, ub);       // positions some frame updates
+    const bool full = p.Xfull != nullptr;
+    if (on_frames || full) {
+        const bool live = lane < p.frames;                   // this lane stands for a frame
+        const bool on = (on_frames >> lane) & 1u;            // ... whose window was updated: it emits a delta row
+        const bool last = lane == p.frames - 1;
+        const pt* P = reinterpret_cast<const pt*>(p.P);
+        const pt* dPg = reinterpret_cast<const pt*>(p.dP) + (size_t)(live ? lane : 0) * p.p_stride;
+        const long long roff = (long long)(live ? lane : 0) * p.row_stride;
+        int cnt = 0;
+        // f on channels c .. c+3 in every frame at once: per window position the frames' products are prefix-summed
+        // over the lanes and added to the projection before the chunk; then the pointwise part of f, then the max
+        auto eval = [&](int c, pt (&best)[4]) {
+            bool have = false;
+            const pt res[4] = {0, 0, 0, 0};                  // (stacks with shortcuts do not take this path)
+            #pragma unroll
+            for (int wi = 0; wi < KW * KW; ++wi) {
+                if (!(inside >> wi & 1u)) continue;
+                const size_t o = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out + c;
+                pt x[1][4];
+                load4<pt, pt4>(P, o, vec, c, p.c_out, x[0]);
+                if (posmask >> wi & 1u) {
+                    pt d[4] = {0, 0, 0, 0};
+                    if (ub >> wi & 1u) load4<pt, pt4>(dPg, o, vec, c, p.c_out, d);
+                    scan4(d, lane);
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) x[0][j] += d[j];
+                }
+                pt y[4];
+                epi_f<PT, OT, 1, BN, pt>(x, 1u, c, res, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
+                #pragma unroll
+                for (int j = 0; j < 4; ++j) best[j] = (!have || y[j] > best[j]) ? y[j] : best[j];
+                have = true;
+            }
+        };
+        if (OT == T_BIN) {
+            for (int u = warp; u < p.cs; u += 8) {           // one 32-channel word of the output per turn
+                uint32_t word = 0;
+                for (int qd = 0; qd < 8; ++qd) {
+                    const int c = u * 32 + qd * 4;
+                    if (c >= p.c_out) break;
+                    pt best[4] = {0, 0, 0, 0};
+                    eval(c, best);
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) if (c + j < p.c_out && (int)best[j] >= p.theta) word |= 1u << (qd * 4 + j);
+                }
+                const size_t o = (size_t)r * p.cs + u;
+                uint32_t prev = __shfl_up_sync(0xffffffffu, word, 1);
+                if (lane == 0) prev = reinterpret_cast<const uint32_t*>(p.X)[o];
+                const uint32_t ch = word ^ prev;
+                if (live) {
+                    if (on) {
+                        shift_bytes(reinterpret_cast<uint32_t*>(p.D), roff)[o] = ch;
+                        if (p.Xn) shift_bytes(reinterpret_cast<uint32_t*>(p.Xn), roff)[o] = word;
+                        cnt += __popc(ch);
+                    }
+                    if (full) shift_bytes(reinterpret_cast<uint32_t*>(p.Xfull), roff)[o] = word;
+                }
+                __syncwarp();                                // every lane has read the old word
+                if (last && on_frames) reinterpret_cast<uint32_t*>(p.X)[o] = word;
+            }
+        } else {
+            const int units = (p.cs + 3) >> 2;
+            for (int u = warp; u < units; u += 8) {          // four channels of the output per turn
+                const int c = u * 4;
+                const size_t o = (size_t)r * p.cs + c;
+                pt best[4] = {0, 0, 0, 0};
+                eval(c, best);
+                if (OT == T_I8) {                            // (cs is a multiple of 4)
+                    const uint32_t nw = ((uint32_t)(int)best[0] & 0xffu) | ((uint32_t)(int)best[1] & 0xffu) << 8 |
+                                        ((uint32_t)(int)best[2] & 0xffu) << 16 | ((uint32_t)(int)best[3] & 0xffu) << 24;
+                    uint32_t ow_ = __shfl_up_sync(0xffffffffu, nw, 1);
+                    if (lane == 0) ow_ = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(p.X) + o);
+                    if (live) {
+                        if (on) {
+                            uint32_t dw = 0;
+                            #pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int nv = (int)(int8_t)(nw >> (8 * j)), ov = (int)(int8_t)(ow_ >> (8 * j));
+                                const int d = nv - ov;
+                                if (p.errw && (d < -128 || d > 127)) atomicOr(p.errw, ERRW_BOUNDS);
+                                dw |= ((uint32_t)d & 0xffu) << (8 * j);
+                                cnt += nv != ov;
+                            }
+                            *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.D), roff) + o) = dw;
+                        }
+                        if (full) *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xfull), roff) + o) = nw;
+                    }
+                    __syncwarp();
+                    if (last && on_frames) *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.X) + o) = nw;
+                } else {
+                    pt old[4];
+                    if (PT == T_F32) {
+                        // a frame that leaves the window alone keeps the value of the frame before it, bit for bit (its
+                        // own f would see the same projection, but the snapshot may stem from a differently rounded sum)
+                        const unsigned below = on_frames & (0xffffffffu >> (31 - lane));
+                        const int src = below ? 31 - __clz(below) : -1;      // the nearest frame at or below this one that re-evaluates
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const pt carried = __shfl_sync(0xffffffffu, best[j], src < 0 ? 0 : src);
+                            best[j] = src < 0 ? ((c + j < p.cs) ? reinterpret_cast<const pt*>(p.X)[o + j] : (pt)0) : carried;
+                        }
+                    }
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        old[j] = __shfl_up_sync(0xffffffffu, best[j], 1);
+                        if (lane == 0) old[j] = (c + j < p.cs) ? reinterpret_cast<const pt*>(p.X)[o + j] : (pt)0;
+                    }
+                    if (live) {
+                        pt* Dg = shift_bytes(reinterpret_cast<pt*>(p.D), roff);
+                        pt* Fg = full ? shift_bytes(reinterpret_cast<pt*>(p.Xfull), roff) : nullptr;
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (c + j >= p.cs) break;
+                            if (on) { Dg[o + j] = best[j] - old[j]; cnt += best[j] != old[j]; }
+                            if (full) Fg[o + j] = best[j];
+                        }
+                    }
+                    __syncwarp();
+                    if (last && on_frames) {
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) if (c + j < p.cs) reinterpret_cast<pt*>(p.X)[o + j] = best[j];
+                    }
+                }
+            }
+        }
+        if (cnt) atomicAdd(&s_cnt[lane], cnt);
+    }
+    __syncthreads();
+    // ---- per frame in which the pixel changed: activity bit, counters, marks in the reading layers' update bitmaps
+    for (int g = warp; g < p.frames; g += 8) {
+        const int cnt = s_cnt[g];
+        if (cnt == 0) continue;                              // uniform inside the warp
+        const long long off = g * p.arena_stride;
+        if (lane == 0) {
+            atomicOr(shift_bytes(p.act, off) + (r >> 5), 1u << (r & 31));
+            atomicAdd(shift_bytes(p.nnz, off), (unsigned long long)cnt);
+            atomicAdd(shift_bytes(p.npix, off), 1ull);
+        }
+        if (READERS) {
+            Readers R = p.readers;
+            shift_readers(R, off);
+            unsigned long long macs[MAX_READERS];
+            // (lane 0 carries the pixel; the other lanes stand for unchanged neighbours of the same image row)
+            scatter_changed_warp(R, ns, ty, lane == 0 ? tx : 1, lane == 0 ? cnt : 0, lane, macs);
+            if (lane == 0) {
+                #pragma unroll
+                for (int i = 0; i < MAX_READERS; ++i) if (i < R.n && R.r[i].macs && macs[i]) atomicAdd(R.r[i].macs, macs[i]);
+            }
+        }
+    }
+}
+
+// ================================================================================================
+// host side
+// ================================================================================================
+template <int PT, int OT, bool BN, int KW>
+static void launch_epi_seq_kw(const EpiSeqParams& e, int blocks, cudaStream_t st)
+{
+    if (e.readers.n > 0) launch_seq(epilogue_seq_kernel<PT, OT, KW, true, BN>, dim3(blocks), dim3(256), 0, st, e);
+    else launch_seq(epilogue_seq_kernel<PT, OT, KW, false, BN>, dim3(blocks), dim3(256), 0, st, e);
+}
+
+template <int PT, int OT, bool BN>
+static int launch_epi_seq_b(const EpiSeqParams& e, int blocks, cudaStream_t st)
+{
+    switch (e.pool_k > 0 ? e.pool_k : 1) {
+        case 1: launch_epi_seq_kw<PT, OT, BN, 1>(e, blocks, st); break;
+        case 2: launch_epi_seq_kw<PT, OT, BN, 2>(e, blocks, st); break;
+        case 3: launch_epi_seq_kw<PT, OT, BN, 3>(e, blocks, st); break;
+        default: return RRM_ERR_UNSUPPORTED;
+    }
+    return RRM_OK;
+}
+
+template <int PT, int OT>
+static int launch_epi_seq_t(const EpiSeqParams& e, int blocks, cudaStream_t st)
+{
+    if ((OT == T_F32 || OT == T_I8) && e.bn_scale) return launch_epi_seq_b<PT, OT, (OT == T_F32 || OT == T_I8)>(e, blocks, st);
+    return launch_epi_seq_b<PT, OT, false>(e, blocks, st);
+}
+
+// The epilogue of layer l over `frames` consecutive frames (the bound arena is frame 0's).
+int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride, cudaStream_t st)
+{
+    Layer& L = net->layers[l];
+    const rrm_layer_desc& d = L.d;
+    Tensor& out = net->tensors[l + 1];
+    if (frames < 1 || frames > SEQ_MAX_FRAMES || d.res >= 0 || !L.Palt || !L.dPall || !out.Dall) return RRM_ERR_INVALID_ARG;
+    EpiSeqParams e{};
+    e.P = L.Palt; e.Q = L.P; e.dP = L.dPall; e.oact = L.oact;
+    e.X = out.X; e.D = out.Dall;
+    e.Xn = (out.dtype == T_BIN && out.has_consumer) ? out.Xnall : nullptr;
+    e.Xfull = (l + 1 == (int)net->layers.size()) ? out.Xfull : nullptr;
+    e.act = out.act; e.nnz = out.nnz; e.npix = out.npix;
+    e.errw = out.has_consumer ? net->errw : nullptr;
+    e.n = d.n; e.oh = L.oh; e.ow = L.ow; e.th = L.th; e.tw = L.tw; e.c_out = d.c_out; e.cs = out.cs;
+    e.pool_k = d.pool_k; e.pool_s = d.pool_s; e.pool_p = d.pool_p; e.act_fn = d.act; e.shift = d.shift; e.theta = d.theta;
+    e.readers = out.readers;
+    e.bn_scale = L.bn_scale; e.bn_shift = L.bn_shift;
+    e.frames = frames; e.row_stride = (long long)out.bytes(); e.arena_stride = arena_stride;
+    e.p_stride = (long long)L.opixels() * d.c_out;
+    e.f_blocks = out.pixels();
+    e.opix = L.opixels();
+    const int blocks = e.f_blocks + ceil_div(L.opixels(), 32);
+    int s;
+    if (d.dtype == RRM_F32) s = launch_epi_seq_t<T_F32, T_F32>(e, blocks, st);
+    else if (out.dtype == T_I8) s = launch_epi_seq_t<T_I32, T_I8>(e, blocks, st);
+    else if (out.dtype == T_BIN) s = launch_epi_seq_t<T_I32, T_BIN>(e, blocks, st);
+    else s = launch_epi_seq_t<T_I32, T_I32>(e, blocks, st);
+    RRM_TRY(s);
+    RRM_CUDA_TRY(cudaGetLastError());
+    return RRM_OK;
+}
+
+int seq_max_frames() { return SEQ_MAX_FRAMES; }
+
+// Can delta chunks of this stack run layer by layer over all frames?  (No shortcuts: a layer that adds another
+// tensor would need that tensor's value at every frame.)  Buffers for SEQ_MAX_FRAMES frames: per tensor the delta
+// rows (binary tensors: the new rows too; the last tensor: every frame's full rows), per layer the products.
+int ensure_frame_batch(rrm_net* net)
+{
+    if (net->seq_ready) return RRM_OK;
+    for (auto& L : net->layers) if (L.d.res >= 0) return RRM_ERR_UNSUPPORTED;
+    const size_t G = SEQ_MAX_FRAMES;
+    size_t need = 0;
+    for (auto& T : net->tensors) need += T.bytes() * G * (T.dtype == T_BIN ? 2 : 1);
+    need += net->tensors.back().bytes() * G;
+    for (auto& L : net->layers) need += (size_t)L.opixels() * L.d.c_out * 4 * (G + 1);
+    if (need > ((size_t)8 << 30)) return RRM_ERR_UNSUPPORTED;          // (a stack this large keeps the frame-pipelined form)
+    auto alloc = [&](void** p, size_t bytes) -> int {
+        if (*p) return RRM_OK;
+        if (cudaMalloc(p, bytes ? bytes : 16) != cudaSuccess) { *p = nullptr; cudaGetLastError(); return RRM_ERR_ALLOC; }
+        net->allocs.push_back(*p);
+        return RRM_OK;
+    };
+    for (auto& T : net->tensors) {
+        RRM_TRY(alloc(&T.Dall, T.bytes() * G));
+        if (T.dtype == T_BIN) RRM_TRY(alloc(&T.Xnall, T.bytes() * G));
+    }
+    RRM_TRY(alloc(&net->tensors.back().Xfull, net->tensors.back().bytes() * G));
+    for (auto& L : net->layers) {
+        const size_t bytes = (size_t)L.opixels() * L.d.c_out * 4;
+        RRM_TRY(alloc(&L.Palt, bytes));
+        RRM_TRY(alloc(&L.dPall, bytes * G));
+    }
+    net->seq_ready = true;
+    return RRM_OK;
+}
+
+}  // namespace rrm

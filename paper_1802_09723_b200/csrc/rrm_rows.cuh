@@ -2,6 +2,7 @@
 // that read it, and how a CTA finds its rows in a layer's bitmap of projection pixels to update.
 #pragma once
 #include "rrm_common.cuh"
+#include "rrm_dev.cuh"
 
 namespace rrm {
 
@@ -75,6 +76,17 @@ __device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, i
                 }
             }
         }
+    }
+}
+
+// the readers' bitmaps and counters of frame g's arena
+__device__ __forceinline__ void shift_readers(Readers& R, long long bytes)
+{
+    #pragma unroll
+    for (int i = 0; i < MAX_READERS; ++i) {
+        if (i >= R.n) break;
+        R.r[i].oact = shift_bytes(R.r[i].oact, bytes);
+        if (R.r[i].macs) R.r[i].macs = shift_bytes(R.r[i].macs, bytes);
     }
 }
 
