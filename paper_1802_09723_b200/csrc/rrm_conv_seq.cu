@@ -42,7 +42,7 @@ struct EpiSeqParams {
     long long row_stride;     // bytes between the frames' delta rows / new rows / full rows of the output tensor
     long long arena_stride;   // bytes between the frames' arenas
     long long p_stride;       // elements between the frames' products
-    int f_blocks;             // CTAs that evaluate f (one output pixel each); the CTAs behind them merge, one per bitmap word
+    int f_blocks;             // CTAs that evaluate f (one output pixel each); the CTAs behind them merge, eight projection pixels each
     int opix;                 // projection pixels
 };
 
@@ -85,49 +85,46 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
     pdl_launch_dependents();
     pdl_wait();
     if ((int)blockIdx.x >= p.f_blocks) {
-        // ---- merge role: lane g holds frame g's word of the update bitmap; a warp takes four of the word's 32 pixels
-        // and adds the frames' products in frame order, as single steps would (lanes over the channels)
-        const int w = (int)blockIdx.x - p.f_blocks;
-        unsigned bits = 0;
-        if (lane < p.frames) bits = shift_bytes(p.oact, lane * p.arena_stride)[w];
+        // ---- merge role: a warp per projection pixel; lane g looks the pixel up in frame g's update bitmap, then the
+        // lanes spread over the channels and add the frames' products in frame order, as single steps would
+        const int q = ((int)blockIdx.x - p.f_blocks) * 8 + warp;
+        if (q >= p.opix) return;
+        bool mine = false;
+        if (lane < p.frames) mine = (shift_bytes(p.oact, lane * p.arena_stride)[q >> 5] >> (q & 31)) & 1u;
+        const unsigned in_frames = __ballot_sync(0xffffffffu, mine);
+        if (in_frames == 0) return;
         const pt* R = reinterpret_cast<const pt*>(p.P);
         const pt* dP = reinterpret_cast<const pt*>(p.dP);
         pt* Q = reinterpret_cast<pt*>(p.Q);
-        #pragma unroll 1
-        for (int k = 0; k < 4; ++k) {
-            const int b = warp * 4 + k;
-            const unsigned in_frames = __ballot_sync(0xffffffffu, (bits >> b) & 1u);
-            if (in_frames == 0) continue;
-            const size_t row = (size_t)(w * 32 + b) * p.c_out;
-            for (int c = lane * 4; c < p.c_out; c += 128) {
-                pt acc[4];
-                load4<pt, pt4>(R, row + c, vec, c, p.c_out, acc);
-                unsigned m = in_frames;
-                while (m) {                                  // four frames' rows in flight at a time
-                    int g[4];
-                    pt d[4][4];
-                    #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        g[i] = -1;
-                        if (m) { g[i] = __ffs(m) - 1; m &= m - 1; }
-                    }
-                    #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        d[i][0] = d[i][1] = d[i][2] = d[i][3] = 0;
-                        if (g[i] >= 0) load4<pt, pt4>(dP + (size_t)g[i] * p.p_stride, row + c, vec, c, p.c_out, d[i]);
-                    }
-                    #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        if (g[i] < 0) continue;
-                        #pragma unroll
-                        for (int j = 0; j < 4; ++j) acc[j] += d[i][j];
-                    }
+        const size_t row = (size_t)q * p.c_out;
+        for (int c = lane * 4; c < p.c_out; c += 128) {
+            pt acc[4];
+            load4<pt, pt4>(R, row + c, vec, c, p.c_out, acc);
+            unsigned m = in_frames;
+            while (m) {                                      // eight frames' rows in flight at a time
+                int g[8];
+                pt d[8][4];
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    g[i] = -1;
+                    if (m) { g[i] = __ffs(m) - 1; m &= m - 1; }
                 }
-                if (vec) { pt4 t; t.x = acc[0]; t.y = acc[1]; t.z = acc[2]; t.w = acc[3]; *reinterpret_cast<pt4*>(Q + row + c) = t; }
-                else {
-                    #pragma unroll
-                    for (int j = 0; j < 4; ++j) if (c + j < p.c_out) Q[row + c + j] = acc[j];
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    d[i][0] = d[i][1] = d[i][2] = d[i][3] = 0;
+                    if (g[i] >= 0) load4<pt, pt4>(dP + (size_t)g[i] * p.p_stride, row + c, vec, c, p.c_out, d[i]);
                 }
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (g[i] < 0) continue;
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[j] += d[i][j];
+                }
+            }
+            if (vec) { pt4 t; t.x = acc[0]; t.y = acc[1]; t.z = acc[2]; t.w = acc[3]; *reinterpret_cast<pt4*>(Q + row + c) = t; }
+            else {
+                #pragma unroll
+                for (int j = 0; j < 4; ++j) if (c + j < p.c_out) Q[row + c + j] = acc[j];
             }
         }
         return;
@@ -170,45 +167,68 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         const pt* dPg = reinterpret_cast<const pt*>(p.dP) + (size_t)(live ? lane : 0) * p.p_stride;
         const long long roff = (long long)(live ? lane : 0) * p.row_stride;
         int cnt = 0;
-        // f on channels c .. c+3 in every frame at once: per window position the frames' products are prefix-summed
-        // over the lanes and added to the projection before the chunk; then the pointwise part of f, then the max
-        auto eval = [&](int c, pt (&best)[4]) {
-            bool have = false;
+        // f on NQ groups of four channels in every frame at once.  All loads of a turn are issued before anything is
+        // done with them (a turn is one memory round trip); then, per window position, the frames' products are
+        // prefix-summed over the lanes and added to the projection before the chunk, the pointwise part of f follows,
+        // and the max over the window.  c[q] < 0: no such group.
+        constexpr int NQ = KW == 1 ? 4 : (KW == 2 ? 2 : 1);
+        auto eval = [&](const int (&c)[NQ], pt (&best)[NQ][4]) {
             const pt res[4] = {0, 0, 0, 0};                  // (stacks with shortcuts do not take this path)
+            pt x[NQ][KW * KW][4], d[NQ][KW * KW][4];
             #pragma unroll
-            for (int wi = 0; wi < KW * KW; ++wi) {
-                if (!(inside >> wi & 1u)) continue;
-                const size_t o = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out + c;
-                pt x[1][4];
-                load4<pt, pt4>(P, o, vec, c, p.c_out, x[0]);
-                if (posmask >> wi & 1u) {
-                    pt d[4] = {0, 0, 0, 0};
-                    if (ub >> wi & 1u) load4<pt, pt4>(dPg, o, vec, c, p.c_out, d);
-                    scan4(d, lane);
-                    #pragma unroll
-                    for (int j = 0; j < 4; ++j) x[0][j] += d[j];
-                }
-                pt y[4];
-                epi_f<PT, OT, 1, BN, pt>(x, 1u, c, res, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
+            for (int q = 0; q < NQ; ++q) {
                 #pragma unroll
-                for (int j = 0; j < 4; ++j) best[j] = (!have || y[j] > best[j]) ? y[j] : best[j];
-                have = true;
+                for (int wi = 0; wi < KW * KW; ++wi) {
+                    x[q][wi][0] = x[q][wi][1] = x[q][wi][2] = x[q][wi][3] = 0;
+                    d[q][wi][0] = d[q][wi][1] = d[q][wi][2] = d[q][wi][3] = 0;
+                    if (c[q] < 0 || !(inside >> wi & 1u)) continue;
+                    const size_t o = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out + c[q];
+                    load4<pt, pt4>(P, o, vec, c[q], p.c_out, x[q][wi]);
+                    if (ub >> wi & 1u) load4<pt, pt4>(dPg, o, vec, c[q], p.c_out, d[q][wi]);
+                }
+            }
+            #pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                bool have = false;
+                best[q][0] = best[q][1] = best[q][2] = best[q][3] = 0;
+                if (c[q] < 0) continue;                      // uniform inside the warp
+                #pragma unroll
+                for (int wi = 0; wi < KW * KW; ++wi) {
+                    if (!(inside >> wi & 1u)) continue;
+                    if (posmask >> wi & 1u) {
+                        scan4(d[q][wi], lane);
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) x[q][wi][j] += d[q][wi][j];
+                    }
+                    pt y[4];
+                    const pt (&x1)[1][4] = reinterpret_cast<const pt (&)[1][4]>(x[q][wi]);
+                    epi_f<PT, OT, 1, BN, pt>(x1, 1u, c[q], res, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) best[q][j] = (!have || y[j] > best[q][j]) ? y[j] : best[q][j];
+                    have = true;
+                }
             }
         };
         if (OT == T_BIN) {
             for (int u = warp; u < p.cs; u += 8) {           // one 32-channel word of the output per turn
+                const size_t o = (size_t)r * p.cs + u;
+                const uint32_t before = reinterpret_cast<const uint32_t*>(p.X)[o];
                 uint32_t word = 0;
-                for (int qd = 0; qd < 8; ++qd) {
-                    const int c = u * 32 + qd * 4;
-                    if (c >= p.c_out) break;
-                    pt best[4] = {0, 0, 0, 0};
+                for (int qd = 0; qd < 8; qd += NQ) {
+                    int c[NQ];
+                    #pragma unroll
+                    for (int q = 0; q < NQ; ++q) { c[q] = u * 32 + (qd + q) * 4; if (c[q] >= p.c_out) c[q] = -1; }
+                    if (c[0] < 0) break;
+                    pt best[NQ][4];
                     eval(c, best);
                     #pragma unroll
-                    for (int j = 0; j < 4; ++j) if (c + j < p.c_out && (int)best[j] >= p.theta) word |= 1u << (qd * 4 + j);
+                    for (int q = 0; q < NQ; ++q) {
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) if (c[q] >= 0 && c[q] + j < p.c_out && (int)best[q][j] >= p.theta) word |= 1u << ((qd + q) * 4 + j);
+                    }
                 }
-                const size_t o = (size_t)r * p.cs + u;
                 uint32_t prev = __shfl_up_sync(0xffffffffu, word, 1);
-                if (lane == 0) prev = reinterpret_cast<const uint32_t*>(p.X)[o];
+                if (lane == 0) prev = before;
                 const uint32_t ch = word ^ prev;
                 if (live) {
                     if (on) {
@@ -218,70 +238,88 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                     }
                     if (full) shift_bytes(reinterpret_cast<uint32_t*>(p.Xfull), roff)[o] = word;
                 }
-                __syncwarp();                                // every lane has read the old word
-                if (last && on_frames) reinterpret_cast<uint32_t*>(p.X)[o] = word;
+                if (last && on_frames) reinterpret_cast<uint32_t*>(p.X)[o] = word;       // (every lane read the old word before the turn's shuffles)
             }
         } else {
             const int units = (p.cs + 3) >> 2;
-            for (int u = warp; u < units; u += 8) {          // four channels of the output per turn
-                const int c = u * 4;
-                const size_t o = (size_t)r * p.cs + c;
-                pt best[4] = {0, 0, 0, 0};
+            for (int u0 = warp * NQ; u0 < units; u0 += 8 * NQ) {   // NQ groups of four output channels per turn
+                int c[NQ];
+                #pragma unroll
+                for (int q = 0; q < NQ; ++q) c[q] = (u0 + q < units) ? (u0 + q) * 4 : -1;
+                // the output's value before the chunk (lane 0's previous frame), fetched with the turn's other loads
+                uint32_t before_w[NQ];
+                pt before[NQ][4];
+                #pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    before_w[q] = 0;
+                    before[q][0] = before[q][1] = before[q][2] = before[q][3] = 0;
+                    if (c[q] < 0) continue;
+                    const size_t o = (size_t)r * p.cs + c[q];
+                    if (OT == T_I8) before_w[q] = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(p.X) + o);
+                    else {
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) if (c[q] + j < p.cs) before[q][j] = reinterpret_cast<const pt*>(p.X)[o + j];
+                    }
+                }
+                pt best[NQ][4];
                 eval(c, best);
-                if (OT == T_I8) {                            // (cs is a multiple of 4)
-                    const uint32_t nw = ((uint32_t)(int)best[0] & 0xffu) | ((uint32_t)(int)best[1] & 0xffu) << 8 |
-                                        ((uint32_t)(int)best[2] & 0xffu) << 16 | ((uint32_t)(int)best[3] & 0xffu) << 24;
-                    uint32_t ow_ = __shfl_up_sync(0xffffffffu, nw, 1);
-                    if (lane == 0) ow_ = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(p.X) + o);
-                    if (live) {
-                        if (on) {
-                            uint32_t dw = 0;
+                #pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (c[q] < 0) continue;                  // uniform inside the warp
+                    const size_t o = (size_t)r * p.cs + c[q];
+                    if (OT == T_I8) {                        // (cs is a multiple of 4)
+                        const uint32_t nw = ((uint32_t)(int)best[q][0] & 0xffu) | ((uint32_t)(int)best[q][1] & 0xffu) << 8 |
+                                            ((uint32_t)(int)best[q][2] & 0xffu) << 16 | ((uint32_t)(int)best[q][3] & 0xffu) << 24;
+                        uint32_t ow_ = __shfl_up_sync(0xffffffffu, nw, 1);
+                        if (lane == 0) ow_ = before_w[q];
+                        if (live) {
+                            if (on) {
+                                uint32_t dw = 0;
+                                #pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const int nv = (int)(int8_t)(nw >> (8 * j)), ov = (int)(int8_t)(ow_ >> (8 * j));
+                                    const int dd = nv - ov;
+                                    if (p.errw && (dd < -128 || dd > 127)) atomicOr(p.errw, ERRW_BOUNDS);
+                                    dw |= ((uint32_t)dd & 0xffu) << (8 * j);
+                                    cnt += nv != ov;
+                                }
+                                *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.D), roff) + o) = dw;
+                            }
+                            if (full) *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xfull), roff) + o) = nw;
+                        }
+                        if (last && on_frames) *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.X) + o) = nw;
+                    } else {
+                        pt old[4];
+                        if (PT == T_F32) {
+                            // a frame that leaves the window alone keeps the value of the frame before it, bit for bit (its
+                            // own f would see the same projection, but the snapshot may stem from a differently rounded sum)
+                            const unsigned below = on_frames & (0xffffffffu >> (31 - lane));
+                            const int src = below ? 31 - __clz(below) : -1;      // the nearest frame at or below this one that re-evaluates
                             #pragma unroll
                             for (int j = 0; j < 4; ++j) {
-                                const int nv = (int)(int8_t)(nw >> (8 * j)), ov = (int)(int8_t)(ow_ >> (8 * j));
-                                const int d = nv - ov;
-                                if (p.errw && (d < -128 || d > 127)) atomicOr(p.errw, ERRW_BOUNDS);
-                                dw |= ((uint32_t)d & 0xffu) << (8 * j);
-                                cnt += nv != ov;
+                                const pt carried = __shfl_sync(0xffffffffu, best[q][j], src < 0 ? 0 : src);
+                                best[q][j] = src < 0 ? before[q][j] : carried;
                             }
-                            *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.D), roff) + o) = dw;
                         }
-                        if (full) *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xfull), roff) + o) = nw;
-                    }
-                    __syncwarp();
-                    if (last && on_frames) *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.X) + o) = nw;
-                } else {
-                    pt old[4];
-                    if (PT == T_F32) {
-                        // a frame that leaves the window alone keeps the value of the frame before it, bit for bit (its
-                        // own f would see the same projection, but the snapshot may stem from a differently rounded sum)
-                        const unsigned below = on_frames & (0xffffffffu >> (31 - lane));
-                        const int src = below ? 31 - __clz(below) : -1;      // the nearest frame at or below this one that re-evaluates
                         #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const pt carried = __shfl_sync(0xffffffffu, best[j], src < 0 ? 0 : src);
-                            best[j] = src < 0 ? ((c + j < p.cs) ? reinterpret_cast<const pt*>(p.X)[o + j] : (pt)0) : carried;
+                            old[j] = __shfl_up_sync(0xffffffffu, best[q][j], 1);
+                            if (lane == 0) old[j] = before[q][j];
                         }
-                    }
-                    #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        old[j] = __shfl_up_sync(0xffffffffu, best[j], 1);
-                        if (lane == 0) old[j] = (c + j < p.cs) ? reinterpret_cast<const pt*>(p.X)[o + j] : (pt)0;
-                    }
-                    if (live) {
-                        pt* Dg = shift_bytes(reinterpret_cast<pt*>(p.D), roff);
-                        pt* Fg = full ? shift_bytes(reinterpret_cast<pt*>(p.Xfull), roff) : nullptr;
-                        #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if (c + j >= p.cs) break;
-                            if (on) { Dg[o + j] = best[j] - old[j]; cnt += best[j] != old[j]; }
-                            if (full) Fg[o + j] = best[j];
+                        if (live) {
+                            pt* Dg = shift_bytes(reinterpret_cast<pt*>(p.D), roff);
+                            pt* Fg = full ? shift_bytes(reinterpret_cast<pt*>(p.Xfull), roff) : nullptr;
+                            #pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if (c[q] + j >= p.cs) break;
+                                if (on) { Dg[o + j] = best[q][j] - old[j]; cnt += best[q][j] != old[j]; }
+                                if (full) Fg[o + j] = best[q][j];
+                            }
                         }
-                    }
-                    __syncwarp();
-                    if (last && on_frames) {
-                        #pragma unroll
-                        for (int j = 0; j < 4; ++j) if (c + j < p.cs) reinterpret_cast<pt*>(p.X)[o + j] = best[j];
+                        if (last && on_frames) {
+                            #pragma unroll
+                            for (int j = 0; j < 4; ++j) if (c[q] + j < p.cs) reinterpret_cast<pt*>(p.X)[o + j] = best[q][j];
+                        }
                     }
                 }
             }
@@ -364,7 +402,7 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
     e.p_stride = (long long)L.opixels() * d.c_out;
     e.f_blocks = out.pixels();
     e.opix = L.opixels();
-    const int blocks = e.f_blocks + ceil_div(L.opixels(), 32);
+    const int blocks = e.f_blocks + ceil_div(L.opixels(), 8);       // merge CTAs: a warp per projection pixel
     int s;
     if (d.dtype == RRM_F32) s = launch_epi_seq_t<T_F32, T_F32>(e, blocks, st);
     else if (out.dtype == T_I8) s = launch_epi_seq_t<T_I32, T_I8>(e, blocks, st);
