@@ -559,3 +559,68 @@ def test_fp32_projections_are_bitwise_reproducible(name):
     for other in runs[1:]:
         for a, b in zip(runs[0], other):
             assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ chunk forms: layer by layer, frame-pipelined, in place
+def _two_layer_stack(dtype, rng):
+    """Layer 0 reads a multi-channel input of the given type (the import kernels of every input layout) and pools with
+    a window that leaves trailing projection rows outside every window; layer 1 reads its output."""
+    if dtype == "bin":
+        a = _spec("bin", 40, (15, 14), 36, 3, 1, 1, rng, act="sign", pool=(3, 2, 0), theta=2)
+        b = _spec("bin", 36, (7, 6), 20, 3, 1, 1, rng, act="sign", theta=1)
+    elif dtype == "i8":
+        a = _spec("i8", 16, (16, 14), 40, 3, 1, 1, rng, act="relu", pool=(3, 2, 0), shift=11)
+        b = _spec("i8", 40, (7, 6), 24, 3, 1, 1, rng, act="none")
+    else:
+        a = _spec("f32", 12, (16, 14), 40, 3, 1, 1, rng, act="relu", pool=(2, 2, 0))
+        b = _spec("f32", 40, (8, 7), 24, 3, 1, 1, rng, act="leaky")
+    b.src = 1
+    return [a, b]
+
+
+@pytest.mark.parametrize("form", ["layer_by_layer", "pipelined", "in_place"])
+@pytest.mark.parametrize("dtype", ["f32", "i8", "bin"])
+def test_chunk_forms_agree_with_the_oracle(dtype, form, monkeypatch):
+    """rrm_net_step_seq on a delta chunk has three forms (every kernel over all frames of the chunk; frames
+    overlapping in one graph with the frame's product kept apart; the same adding in place).  Each must give every
+    frame's output, the state after the chunk and the last frame's counters of Algorithm 1 - also across a frame
+    without change and a frame in which everything changes, for every input layout, two streams."""
+    if form == "pipelined":
+        monkeypatch.setenv("RRM_CHUNK_PIPELINED", "1")
+    elif form == "in_place":
+        monkeypatch.setenv("RRM_CHUNK_INPLACE", "1")
+    rrm = _rrm()
+    rng = np.random.default_rng({"f32": 5, "i8": 6, "bin": 7}[dtype])
+    specs = _two_layer_stack(dtype, rng)
+    s0 = specs[0]
+    video = _video(dtype, s0.c_in, (s0.h, s0.w), 10, 2, rng)
+    net = rrm.net_from_specs(specs, n=2)
+    rec = orc.Recurrence(specs, n=2)
+    rec.step(np.full_like(video[0], -1 if dtype == "bin" else 0))
+    packed = [_frame_to_dev(specs, video[t]) for t in range(video.shape[0])]
+    t0 = 0
+    for T in (4, 3, 2):
+        frames = torch.stack(packed[t0:t0 + T]).contiguous()
+        outs = net.new_output(frames=T)
+        net.step_seq(frames, outs, T)
+        for i in range(T):
+            rec.step(video[t0 + i])
+            want = orc.dense_forward(specs, video[t0 + i])[0][len(specs)]
+            got = outs[i].cpu().numpy()
+            if dtype == "f32":
+                assert float(np.abs(got - want).max()) <= F32_TOL * max(1e-30, float(np.abs(want).max())), t0 + i
+            elif dtype == "bin":
+                np.testing.assert_array_equal(unpack_bits_nhwc(got.view(np.uint32), specs[-1].c_out), want, err_msg=f"frame {t0 + i}")
+            else:
+                np.testing.assert_array_equal(got.astype(np.int64), want, err_msg=f"frame {t0 + i}")
+        t0 += T
+        _compare(specs, net, video[t0 - 1], t0 - 1)
+        for l in range(len(specs)):
+            st = net.stats(l)
+            assert st["error_word"] == 0
+            if dtype != "f32" or l == 0:
+                assert st["nnz_elems"] == rec.nnz[l] and st["active_macs"] == rec.macs[l], (form, t0, l, st, rec.nnz[l], rec.macs[l])
+    out = net.new_output()
+    net.step(packed[9], out)                  # a single step carries on from the chunk's state
+    _compare(specs, net, video[9], 9)
+    net.close()
