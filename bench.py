@@ -476,6 +476,11 @@ def compact_conv(r):
     out["dense_over_active_macs"] = r["eq9_eq10"]["dense_over_active_macs"]
     out["roofline_frac"] = r["roofline"]["frac"]
     out["roofline_bound"] = r["roofline"]["bound"]
+    if "seq" in r:
+        q = r["seq"]
+        out["chunk"] = {"frames_per_call": q["frames_per_call"], "ms_per_frame": q["ms_per_frame_step"],
+                        "dense_ms_per_frame": q["dense_ms_per_call"] / q["frames_per_call"], "frames_per_sec": q["frames_per_sec"],
+                        "speedup_vs_own_dense": q["speedup_vs_own_dense"], "speedup_vs_frame_by_frame": q["speedup_vs_frame_by_frame"]}
     if "cpu_baseline" in r:
         out["cpu_baseline"] = r["cpu_baseline"]
     return out
@@ -865,11 +870,13 @@ def main():
                                                 ("cfg4_delta_forced", "cfg4", "tensor", 8, 1), ("cfg4_auto", "cfg4", "auto", 8, 0)):
             try:
                 conv[key] = compact_conv(conv_measure(name, variant, steps=30, warmup=5, frames=fr_n, cpu_frames=cpu_n,
-                                                      sample_clocks=False))
+                                                      sample_clocks=False, seq=None if name == "cfg4" else FRAMES))
             except Exception as e:  # noqa: BLE001
                 conv[key] = {"error": str(e)}
         conv["note"] = ("one step = one frame of every stream through rrm_net_step, median of 30 cold-L2 steps; S / S0 / eta: "
-                        "Eq. 9 and Eq. 10 from the measured per-layer densities; cpu_baseline: the oracle on the host cores")
+                        "Eq. 9 and Eq. 10 from the measured per-layer densities; chunk: 32 consecutive frames per rrm_net_step_seq "
+                        "call (delta) / rrm_net_dense_seq call (dense), cold L2, median, per frame; cpu_baseline: the oracle on "
+                        "the host cores")
 
     # ---- CPU oracle on the host cores (rank 0, N = 1 only): a bounded sample of the same workload
     cpu = None
