@@ -6,11 +6,11 @@
 // independent of one another.  So every kernel of a step takes all frames of the chunk in one launch:
 //   import      frame g against frame g-1 at the boundary (rrm_conv.cu), delta rows and bitmaps per frame;
 //   convolution frame = blockIdx.z: the product of frame g is stored in a buffer of its own, rows of updated pixels only;
-//   epilogue    (here) lane g of a warp is frame g: P_g = P_before + sum_{t<=g} F*dI_t (Eq. 5 unrolled) is an inclusive
-//               prefix sum over the lanes, f is evaluated in every lane at once, the previous frame's output comes
-//               from the neighbouring lane, and lane g emits frame g's delta row, bitmap bit and counters; further
-//               CTAs of the same launch add the products of all frames onto the stored projection.
-// A 32-frame chunk of a five-layer stack is 15 launches instead of 384, and the chains of dependent memory round trips
+//   projection  (here) lane g of a warp is frame g: P_g = P_before + sum_{t<=g} F*dI_t (Eq. 5 unrolled) is an inclusive
+//               prefix sum over the lanes, once per updated projection pixel; the last frame's goes to the stored projection;
+//   epilogue    (here) lane = frame again: f is evaluated in every frame at once, the previous frame's output comes
+//               from the neighbouring lane, and lane g emits frame g's delta row, bitmap bit and counters.
+// A 32-frame chunk of a five-layer stack is 20 launches instead of 384, and the chains of dependent memory round trips
 // that bound a single-frame launch are paid once per layer and chunk instead of once per layer and frame.
 #include "rrm_common.cuh"
 #include "rrm_rows.cuh"
@@ -42,7 +42,6 @@ struct EpiSeqParams {
     long long row_stride;     // bytes between the frames' delta rows / new rows / full rows of the output tensor
     long long arena_stride;   // bytes between the frames' arenas
     long long p_stride;       // elements between the frames' products
-    int f_blocks;             // CTAs that evaluate f (one output pixel each); the CTAs behind them merge, eight projection pixels each
     int opix;                 // projection pixels
 };
 
@@ -74,6 +73,75 @@ __device__ __forceinline__ void load4(const pt* P, size_t o, bool vec, int c, in
     }
 }
 
+// The projections of all frames, once per projection pixel: P_g = P_before + sum_{t<=g} F*dI_t (Eq. 5 unrolled) as an
+// inclusive prefix sum over the lanes (lane g = frame g).  P_g overwrites frame g's product where frame g updated
+// the pixel; the last frame's value goes to the stored projection.  A CTA per pixel of the union of the frames'
+// update bitmaps, its warps spread over the channels.
+struct ProjSeqParams {
+    const void* R;            // the projection before the chunk (a copy: read only)
+    void* Q;                  // the stored projection
+    void* dP;                 // frame 0's product; in: F*dI_g, out: P_g
+    const uint32_t* oact;     // frame 0's update bitmap
+    int frames, c_out, opix;
+    long long arena_stride, p_stride;
+};
+
+template <int PT>
+__global__ void __launch_bounds__(256) project_seq_kernel(ProjSeqParams p)
+{
+    using pt = typename std::conditional<PT == T_F32, float, int>::type;
+    using pt4 = typename std::conditional<PT == T_F32, float4, int4>::type;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool vec = (p.c_out & 3) == 0;
+    const int q = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
+    bool mine = false;
+    if (lane < p.frames) mine = (shift_bytes(p.oact, lane * p.arena_stride)[q >> 5] >> (q & 31)) & 1u;
+    if (!__any_sync(0xffffffffu, mine)) return;              // (the same in every warp of the CTA)
+    const pt* R = reinterpret_cast<const pt*>(p.R);
+    pt* Q = reinterpret_cast<pt*>(p.Q);
+    pt* dPg = reinterpret_cast<pt*>(p.dP) + (size_t)(lane < p.frames ? lane : 0) * p.p_stride;
+    const size_t row = (size_t)q * p.c_out;
+    const int quads = (p.c_out + 3) >> 2;
+    constexpr int NQ = 4;                                    // groups of four channels per turn (one memory round trip)
+    for (int u0 = warp * NQ; u0 < quads; u0 += 8 * NQ) {
+        pt base[NQ][4], d[NQ][4];
+        #pragma unroll
+        for (int k = 0; k < NQ; ++k) {
+            const int c = (u0 + k) * 4;
+            base[k][0] = base[k][1] = base[k][2] = base[k][3] = 0;
+            d[k][0] = d[k][1] = d[k][2] = d[k][3] = 0;
+            if (u0 + k >= quads) continue;
+            load4<pt, pt4>(R, row + c, vec, c, p.c_out, base[k]);
+            if (mine) load4<pt, pt4>(dPg, row + c, vec, c, p.c_out, d[k]);
+        }
+        #pragma unroll
+        for (int k = 0; k < NQ; ++k) {
+            const int c = (u0 + k) * 4;
+            if (u0 + k >= quads) continue;                   // uniform inside the warp
+            scan4(d[k], lane);
+            #pragma unroll
+            for (int j = 0; j < 4; ++j) d[k][j] += base[k][j];
+            if (mine || lane == 31) {
+                pt* dst = mine ? dPg : Q;
+                if (vec) {
+                    pt4 t; t.x = d[k][0]; t.y = d[k][1]; t.z = d[k][2]; t.w = d[k][3];
+                    *reinterpret_cast<pt4*>(dst + row + c) = t;
+                    if (mine && lane == 31) *reinterpret_cast<pt4*>(Q + row + c) = t;
+                } else {
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (c + j >= p.c_out) continue;
+                        dst[row + c + j] = d[k][j];
+                        if (mine && lane == 31) Q[row + c + j] = d[k][j];
+                    }
+                }
+            }
+        }
+    }
+}
+
 template <int PT, int OT, int KW, bool READERS, bool BN>
 __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
 {
@@ -84,51 +152,6 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
     const bool vec = (p.c_out & 3) == 0;
     pdl_launch_dependents();
     pdl_wait();
-    if ((int)blockIdx.x >= p.f_blocks) {
-        // ---- merge role: a warp per projection pixel; lane g looks the pixel up in frame g's update bitmap, then the
-        // lanes spread over the channels and add the frames' products in frame order, as single steps would
-        const int q = ((int)blockIdx.x - p.f_blocks) * 8 + warp;
-        if (q >= p.opix) return;
-        bool mine = false;
-        if (lane < p.frames) mine = (shift_bytes(p.oact, lane * p.arena_stride)[q >> 5] >> (q & 31)) & 1u;
-        const unsigned in_frames = __ballot_sync(0xffffffffu, mine);
-        if (in_frames == 0) return;
-        const pt* R = reinterpret_cast<const pt*>(p.P);
-        const pt* dP = reinterpret_cast<const pt*>(p.dP);
-        pt* Q = reinterpret_cast<pt*>(p.Q);
-        const size_t row = (size_t)q * p.c_out;
-        for (int c = lane * 4; c < p.c_out; c += 128) {
-            pt acc[4];
-            load4<pt, pt4>(R, row + c, vec, c, p.c_out, acc);
-            unsigned m = in_frames;
-            while (m) {                                      // eight frames' rows in flight at a time
-                int g[8];
-                pt d[8][4];
-                #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    g[i] = -1;
-                    if (m) { g[i] = __ffs(m) - 1; m &= m - 1; }
-                }
-                #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    d[i][0] = d[i][1] = d[i][2] = d[i][3] = 0;
-                    if (g[i] >= 0) load4<pt, pt4>(dP + (size_t)g[i] * p.p_stride, row + c, vec, c, p.c_out, d[i]);
-                }
-                #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (g[i] < 0) continue;
-                    #pragma unroll
-                    for (int j = 0; j < 4; ++j) acc[j] += d[i][j];
-                }
-            }
-            if (vec) { pt4 t; t.x = acc[0]; t.y = acc[1]; t.z = acc[2]; t.w = acc[3]; *reinterpret_cast<pt4*>(Q + row + c) = t; }
-            else {
-                #pragma unroll
-                for (int j = 0; j < 4; ++j) if (c + j < p.c_out) Q[row + c + j] = acc[j];
-            }
-        }
-        return;
-    }
     if (threadIdx.x < SEQ_MAX_FRAMES) s_cnt[threadIdx.x] = 0;
     __syncthreads();
     // ---- f role: this CTA's output pixel; lane = frame
@@ -157,34 +180,37 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         }
     }
     const unsigned on_frames = __ballot_sync(0xffffffffu, ub != 0);
-    const unsigned posmask = __reduce_or_sync(0xffffffffu, ub);       // positions some frame updates
     const bool full = p.Xfull != nullptr;
     if (on_frames || full) {
         const bool live = lane < p.frames;                   // this lane stands for a frame
         const bool on = (on_frames >> lane) & 1u;            // ... whose window was updated: it emits a delta row
         const bool last = lane == p.frames - 1;
         const pt* P = reinterpret_cast<const pt*>(p.P);
-        const pt* dPg = reinterpret_cast<const pt*>(p.dP) + (size_t)(live ? lane : 0) * p.p_stride;
+        const pt* dP = reinterpret_cast<const pt*>(p.dP);
+        unsigned uf[KW * KW];                                // per window position: the frames that update it
+        #pragma unroll
+        for (int wi = 0; wi < KW * KW; ++wi) uf[wi] = __ballot_sync(0xffffffffu, (ub >> wi) & 1u);
         const long long roff = (long long)(live ? lane : 0) * p.row_stride;
         int cnt = 0;
-        // f on NQ groups of four channels in every frame at once.  All loads of a turn are issued before anything is
-        // done with them (a turn is one memory round trip); then, per window position, the frames' products are
-        // prefix-summed over the lanes and added to the projection before the chunk, the pointwise part of f follows,
-        // and the max over the window.  c[q] < 0: no such group.
+        // f on NQ groups of four channels in every frame at once (a turn is one memory round trip): per window position
+        // the frame's projection is fetched, the pointwise part of f applied, then the max over the window.
+        // c[q] < 0: no such group.
         constexpr int NQ = KW == 1 ? 4 : (KW == 2 ? 2 : 1);
         auto eval = [&](const int (&c)[NQ], pt (&best)[NQ][4]) {
             const pt res[4] = {0, 0, 0, 0};                  // (stacks with shortcuts do not take this path)
-            pt x[NQ][KW * KW][4], d[NQ][KW * KW][4];
+            pt x[NQ][KW * KW][4];
             #pragma unroll
             for (int q = 0; q < NQ; ++q) {
                 #pragma unroll
                 for (int wi = 0; wi < KW * KW; ++wi) {
                     x[q][wi][0] = x[q][wi][1] = x[q][wi][2] = x[q][wi][3] = 0;
-                    d[q][wi][0] = d[q][wi][1] = d[q][wi][2] = d[q][wi][3] = 0;
                     if (c[q] < 0 || !(inside >> wi & 1u)) continue;
                     const size_t o = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out + c[q];
-                    load4<pt, pt4>(P, o, vec, c[q], p.c_out, x[q][wi]);
-                    if (ub >> wi & 1u) load4<pt, pt4>(dPg, o, vec, c[q], p.c_out, d[q][wi]);
+                    // the position's projection in this lane's frame: that of the latest frame up to it that updated the
+                    // position (written there by project_seq_kernel), else the projection before the chunk
+                    const unsigned upto = uf[wi] & (0xffffffffu >> (31 - lane));
+                    const pt* src = upto ? dP + (size_t)(31 - __clz(upto)) * p.p_stride : P;
+                    load4<pt, pt4>(src, o, vec, c[q], p.c_out, x[q][wi]);
                 }
             }
             #pragma unroll
@@ -195,11 +221,6 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                 #pragma unroll
                 for (int wi = 0; wi < KW * KW; ++wi) {
                     if (!(inside >> wi & 1u)) continue;
-                    if (posmask >> wi & 1u) {
-                        scan4(d[q][wi], lane);
-                        #pragma unroll
-                        for (int j = 0; j < 4; ++j) x[q][wi][j] += d[q][wi][j];
-                    }
                     pt y[4];
                     const pt (&x1)[1][4] = reinterpret_cast<const pt (&)[1][4]>(x[q][wi]);
                     epi_f<PT, OT, 1, BN, pt>(x1, 1u, c[q], res, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
@@ -210,7 +231,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
             }
         };
         if (OT == T_BIN) {
-            for (int u = warp; u < p.cs; u += 8) {           // one 32-channel word of the output per turn
+            for (int u = blockIdx.y * 8 + warp; u < p.cs; u += 8 * gridDim.y) {   // one 32-channel word of the output per turn
                 const size_t o = (size_t)r * p.cs + u;
                 const uint32_t before = reinterpret_cast<const uint32_t*>(p.X)[o];
                 uint32_t word = 0;
@@ -242,7 +263,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
             }
         } else {
             const int units = (p.cs + 3) >> 2;
-            for (int u0 = warp * NQ; u0 < units; u0 += 8 * NQ) {   // NQ groups of four output channels per turn
+            for (int u0 = (blockIdx.y * 8 + warp) * NQ; u0 < units; u0 += 8 * NQ * gridDim.y) {   // NQ groups of four output channels per turn
                 int c[NQ];
                 #pragma unroll
                 for (int q = 0; q < NQ; ++q) c[q] = (u0 + q < units) ? (u0 + q) * 4 : -1;
@@ -327,25 +348,40 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         if (cnt) atomicAdd(&s_cnt[lane], cnt);
     }
     __syncthreads();
-    // ---- per frame in which the pixel changed: activity bit, counters, marks in the reading layers' update bitmaps
-    for (int g = warp; g < p.frames; g += 8) {
-        const int cnt = s_cnt[g];
-        if (cnt == 0) continue;                              // uniform inside the warp
-        const long long off = g * p.arena_stride;
-        if (lane == 0) {
-            atomicOr(shift_bytes(p.act, off) + (r >> 5), 1u << (r & 31));
+    // ---- per frame in which the pixel changed (lane = frame once more, all frames at once): activity bit, counters,
+    // and in every reading layer's update bitmap of that frame the projection pixels whose filter footprint covers this
+    // pixel, with the exact multiply-accumulates they imply (non-zeros x covering (output, tap) pairs x output channels)
+    if (warp == 0) {
+        const int cnt = lane < p.frames ? s_cnt[lane] : 0;
+        if (cnt > 0) {
+            const long long off = lane * p.arena_stride;
+            // (the CTAs of the grid's y dimension share the pixel, each with a slice of the channels: counts add up, marks
+            // are idempotent, and whoever sets the activity bit first counts the pixel)
+            const unsigned had = atomicOr(shift_bytes(p.act, off) + (r >> 5), 1u << (r & 31));
             atomicAdd(shift_bytes(p.nnz, off), (unsigned long long)cnt);
-            atomicAdd(shift_bytes(p.npix, off), 1ull);
-        }
-        if (READERS) {
-            Readers R = p.readers;
-            shift_readers(R, off);
-            unsigned long long macs[MAX_READERS];
-            // (lane 0 carries the pixel; the other lanes stand for unchanged neighbours of the same image row)
-            scatter_changed_warp(R, ns, ty, lane == 0 ? tx : 1, lane == 0 ? cnt : 0, lane, macs);
-            if (lane == 0) {
-                #pragma unroll
-                for (int i = 0; i < MAX_READERS; ++i) if (i < R.n && R.r[i].macs && macs[i]) atomicAdd(R.r[i].macs, macs[i]);
+            if (!(had >> (r & 31) & 1u)) atomicAdd(shift_bytes(p.npix, off), 1ull);
+            if (READERS) {
+                #pragma unroll 1
+                for (int i = 0; i < p.readers.n; ++i) {
+                    const Reader& rd = p.readers.r[i];
+                    const int ay = ty + rd.pad, ax = tx + rd.pad;
+                    const int oy_lo = max(0, (ay - rd.kh + rd.stride) / rd.stride), oy_hi = min(rd.oh - 1, ay / rd.stride);
+                    const int ox_lo = max(0, (ax - rd.kw + rd.stride) / rd.stride), ox_hi = min(rd.ow - 1, ax / rd.stride);
+                    if (oy_hi < oy_lo || ox_hi < ox_lo) continue;
+                    uint32_t* bm = shift_bytes(rd.oact, off);
+                    for (int oy = oy_lo; oy <= oy_hi; ++oy) {
+                        int q0 = (ns * rd.oh + oy) * rd.ow + ox_lo, left = ox_hi - ox_lo + 1;
+                        while (left > 0) {                   // the run of columns, word by word
+                            const int bit = q0 & 31, take = min(left, 32 - bit);
+                            const unsigned run = (take == 32 ? 0xffffffffu : ((1u << take) - 1u)) << bit;
+                            atomicOr(&bm[q0 >> 5], run);
+                            q0 += take; left -= take;
+                        }
+                    }
+                    if (rd.macs)
+                        atomicAdd(shift_bytes(rd.macs, off),
+                                  (unsigned long long)cnt * (unsigned long long)((oy_hi - oy_lo + 1) * (ox_hi - ox_lo + 1)) * (unsigned long long)rd.c_out);
+                }
             }
         }
     }
@@ -357,8 +393,13 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
 template <int PT, int OT, bool BN, int KW>
 static void launch_epi_seq_kw(const EpiSeqParams& e, int blocks, cudaStream_t st)
 {
-    if (e.readers.n > 0) launch_seq(epilogue_seq_kernel<PT, OT, KW, true, BN>, dim3(blocks), dim3(256), 0, st, e);
-    else launch_seq(epilogue_seq_kernel<PT, OT, KW, false, BN>, dim3(blocks), dim3(256), 0, st, e);
+    // a pixel's channels are dealt out to so many CTAs that a warp has about two turns (memory round trips) to make
+    constexpr int NQ = KW == 1 ? 4 : (KW == 2 ? 2 : 1);
+    const int turns = OT == T_BIN ? ceil_div(e.cs, 8) : ceil_div(ceil_div(e.cs, 4), 8 * NQ);    // per warp of a lone CTA
+    int slices = ceil_div(turns, 2);
+    slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
+    if (e.readers.n > 0) launch_seq(epilogue_seq_kernel<PT, OT, KW, true, BN>, dim3(blocks, slices), dim3(256), 0, st, e);
+    else launch_seq(epilogue_seq_kernel<PT, OT, KW, false, BN>, dim3(blocks, slices), dim3(256), 0, st, e);
 }
 
 template <int PT, int OT, bool BN>
@@ -400,9 +441,16 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
     e.bn_scale = L.bn_scale; e.bn_shift = L.bn_shift;
     e.frames = frames; e.row_stride = (long long)out.bytes(); e.arena_stride = arena_stride;
     e.p_stride = (long long)L.opixels() * d.c_out;
-    e.f_blocks = out.pixels();
     e.opix = L.opixels();
-    const int blocks = e.f_blocks + ceil_div(L.opixels(), 8);       // merge CTAs: a warp per projection pixel
+    {
+        ProjSeqParams q{};
+        q.R = L.Palt; q.Q = L.P; q.dP = L.dPall; q.oact = L.oact;
+        q.frames = frames; q.c_out = d.c_out; q.opix = L.opixels();
+        q.arena_stride = arena_stride; q.p_stride = e.p_stride;
+        if (d.dtype == RRM_F32) launch_seq(project_seq_kernel<T_F32>, dim3(L.opixels()), dim3(256), 0, st, q);
+        else launch_seq(project_seq_kernel<T_I32>, dim3(L.opixels()), dim3(256), 0, st, q);
+    }
+    const int blocks = out.pixels();                         // a CTA per output pixel
     int s;
     if (d.dtype == RRM_F32) s = launch_epi_seq_t<T_F32, T_F32>(e, blocks, st);
     else if (out.dtype == T_I8) s = launch_epi_seq_t<T_I32, T_I8>(e, blocks, st);
