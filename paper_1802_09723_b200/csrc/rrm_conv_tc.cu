@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
         const int ncols = min(p.bn, p.c_out - n0);
         const bool bulk = (p.c_out & 3) == 0;
         int* row = reinterpret_cast<int*>(base) + r * TC_ROW_WORDS;
-        if (ok && (have || DENSE)) {
+        if (ok && (have || DENSE || p.store)) {             // (a stored product is written even if it is all zero)
             for (int c0 = 0; c0 < p.bn; c0 += 32) {
                 uint32_t v[32];
                 if (have) {
