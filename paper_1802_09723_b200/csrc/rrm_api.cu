@@ -556,7 +556,7 @@ static int keep_chunk_graph(rrm_net* net, int kind, int T, unsigned long long ma
 
 // A delta chunk layer by layer: every kernel takes all frames of the chunk (at most seq_max_frames() per launch; a
 // longer chunk goes in equal parts one after the other).  2 L + 5 launches per part, no frame-to-frame edges.
-// RRM_ERR_UNSUPPORTED: the stack has shortcuts or would need too much memory (the frame-pipelined graph serves it).
+// RRM_ERR_UNSUPPORTED: the stack would need too much memory or adds its input as a shortcut (the frame-pipelined graph serves it).
 static int build_seq_graph(rrm_net* net, int T)
 {
     const int L = (int)net->layers.size();
@@ -577,6 +577,8 @@ static int build_seq_graph(rrm_net* net, int T)
         const int F = T - m0 < per ? T - m0 : per;
         if (cudaMemsetAsync(net->chunk_arena[0], 0, net->cleared_bytes * F, st) != cudaSuccess) fail(RRM_ERR_CUDA);
         fail(launch_copy_projections(net, st));              // the epilogues read the projections from the copies and write the stored ones
+        for (auto& X : net->tensors)                         // a shortcut's reader needs the value before the chunk
+            if (X.shortcut_source && cudaMemcpyAsync(X.Xbefore, X.X, X.bytes(), cudaMemcpyDeviceToDevice, st) != cudaSuccess) fail(RRM_ERR_CUDA);
         bind_arena(net, net->chunk_arena[0]);
         if (bind_readers(net) != RRM_OK) { fail(RRM_ERR_UNSUPPORTED); break; }
         for (auto& X : net->tensors) { X.D = X.Dall; X.Xn_cur = X.Xnall; }

@@ -134,6 +134,8 @@ struct Tensor {
     void* Dall = nullptr;
     void* Xnall = nullptr;
     void* Xfull = nullptr;
+    void* Xbefore = nullptr;          // tensors added as a shortcut: the value before the chunk (the snapshot moves on before the reader runs)
+    bool shortcut_source = false;
     bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
     Readers readers{};                // the layers that read it
     int pixels() const { return n * h * w; }

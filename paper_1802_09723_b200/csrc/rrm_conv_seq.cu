@@ -30,6 +30,12 @@ struct EpiSeqParams {
     void* D;                  // frame 0's delta rows of the output tensor
     void* Xn;                 // frame 0's new rows (binary outputs that a layer reads: the sign of a changed bit) or nullptr
     void* Xfull;              // or nullptr: receives every pixel's row of every frame (the stack's last tensor)
+    // shortcut (the layer adds another tensor of the output's shape before the activation): that tensor's value before
+    // the chunk, frame 0's new rows of it and frame 0's activity bitmap of it; nullptr: none
+    const void* res_before;
+    const void* res_new;
+    const uint32_t* res_act;
+    long long res_stride;     // bytes between the frames' new rows of the shortcut tensor
     uint32_t* act;            // frame 0's activity bitmap of the output tensor
     unsigned long long* nnz;
     unsigned long long* npix;
@@ -190,6 +196,12 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         unsigned uf[KW * KW];                                // per window position: the frames that update it
         #pragma unroll
         for (int wi = 0; wi < KW * KW; ++wi) uf[wi] = __ballot_sync(0xffffffffu, (ub >> wi) & 1u);
+        unsigned res_upto = 0;                               // the frames up to this lane's in which the shortcut's pixel changed
+        if (p.res_before) {
+            bool ch = false;
+            if (live) ch = (shift_bytes(p.res_act, lane * p.arena_stride)[r >> 5] >> (r & 31)) & 1u;
+            res_upto = __ballot_sync(0xffffffffu, ch) & (0xffffffffu >> (31 - lane));
+        }
         const long long roff = (long long)(live ? lane : 0) * p.row_stride;
         int cnt = 0;
         // f on NQ groups of four channels in every frame at once (a turn is one memory round trip): per window position
@@ -197,10 +209,22 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         // c[q] < 0: no such group.
         constexpr int NQ = KW == 1 ? 4 : (KW == 2 ? 2 : 1);
         auto eval = [&](const int (&c)[NQ], pt (&best)[NQ][4]) {
-            const pt res[4] = {0, 0, 0, 0};                  // (stacks with shortcuts do not take this path)
-            pt x[NQ][KW * KW][4];
+            pt x[NQ][KW * KW][4], res[NQ][4];
             #pragma unroll
             for (int q = 0; q < NQ; ++q) {
+                res[q][0] = res[q][1] = res[q][2] = res[q][3] = 0;
+                if (p.res_before && c[q] >= 0) {
+                    // the shortcut's value in this lane's frame: the new row of the latest frame up to it in which the
+                    // shortcut's pixel changed, else the value before the chunk
+                    const char* src = res_upto ? reinterpret_cast<const char*>(p.res_new) + (long long)(31 - __clz(res_upto)) * p.res_stride
+                                               : reinterpret_cast<const char*>(p.res_before);
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (c[q] + j >= p.c_out) continue;
+                        if (PT == T_F32) res[q][j] = (pt)reinterpret_cast<const float*>(src)[(size_t)r * p.cs + c[q] + j];
+                        else if (OT == T_I8) res[q][j] = (pt)reinterpret_cast<const int8_t*>(src)[(size_t)r * p.cs + c[q] + j];
+                    }
+                }
                 #pragma unroll
                 for (int wi = 0; wi < KW * KW; ++wi) {
                     x[q][wi][0] = x[q][wi][1] = x[q][wi][2] = x[q][wi][3] = 0;
@@ -223,7 +247,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                     if (!(inside >> wi & 1u)) continue;
                     pt y[4];
                     const pt (&x1)[1][4] = reinterpret_cast<const pt (&)[1][4]>(x[q][wi]);
-                    epi_f<PT, OT, 1, BN, pt>(x1, 1u, c[q], res, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
+                    epi_f<PT, OT, 1, BN, pt>(x1, 1u, c[q], res[q], p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) best[q][j] = (!have || y[j] > best[q][j]) ? y[j] : best[q][j];
                     have = true;
@@ -305,6 +329,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                                     cnt += nv != ov;
                                 }
                                 *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.D), roff) + o) = dw;
+                                if (p.Xn) *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xn), roff) + o) = nw;
                             }
                             if (full) *reinterpret_cast<uint32_t*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xfull), roff) + o) = nw;
                         }
@@ -330,10 +355,11 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                         if (live) {
                             pt* Dg = shift_bytes(reinterpret_cast<pt*>(p.D), roff);
                             pt* Fg = full ? shift_bytes(reinterpret_cast<pt*>(p.Xfull), roff) : nullptr;
+                            pt* Ng = p.Xn ? shift_bytes(reinterpret_cast<pt*>(p.Xn), roff) : nullptr;
                             #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 if (c[q] + j >= p.cs) break;
-                                if (on) { Dg[o + j] = best[q][j] - old[j]; cnt += best[q][j] != old[j]; }
+                                if (on) { Dg[o + j] = best[q][j] - old[j]; cnt += best[q][j] != old[j]; if (Ng) Ng[o + j] = best[q][j]; }
                                 if (full) Fg[o + j] = best[q][j];
                             }
                         }
@@ -427,11 +453,16 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
     Layer& L = net->layers[l];
     const rrm_layer_desc& d = L.d;
     Tensor& out = net->tensors[l + 1];
-    if (frames < 1 || frames > SEQ_MAX_FRAMES || d.res >= 0 || !L.Palt || !L.dPall || !out.Dall) return RRM_ERR_INVALID_ARG;
+    if (frames < 1 || frames > SEQ_MAX_FRAMES || !L.Palt || !L.dPall || !out.Dall) return RRM_ERR_INVALID_ARG;
     EpiSeqParams e{};
     e.P = L.Palt; e.Q = L.P; e.dP = L.dPall; e.oact = L.oact;
     e.X = out.X; e.D = out.Dall;
-    e.Xn = (out.dtype == T_BIN && out.has_consumer) ? out.Xnall : nullptr;
+    e.Xn = ((out.dtype == T_BIN && out.has_consumer) || out.shortcut_source) ? out.Xnall : nullptr;
+    if (d.res >= 0) {
+        const Tensor& rt = net->tensors[d.res];
+        if (!rt.Xbefore || !rt.Xnall) return RRM_ERR_INVALID_ARG;
+        e.res_before = rt.Xbefore; e.res_new = rt.Xnall; e.res_act = rt.act; e.res_stride = (long long)rt.bytes();
+    }
     e.Xfull = (l + 1 == (int)net->layers.size()) ? out.Xfull : nullptr;
     e.act = out.act; e.nnz = out.nnz; e.npix = out.npix;
     e.errw = out.has_consumer ? net->errw : nullptr;
@@ -463,16 +494,18 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
 
 int seq_max_frames() { return SEQ_MAX_FRAMES; }
 
-// Can delta chunks of this stack run layer by layer over all frames?  (No shortcuts: a layer that adds another
-// tensor would need that tensor's value at every frame.)  Buffers for SEQ_MAX_FRAMES frames: per tensor the delta
+// Can delta chunks of this stack run layer by layer over all frames?  Buffers for SEQ_MAX_FRAMES frames: per tensor the delta
 // rows (binary tensors: the new rows too; the last tensor: every frame's full rows), per layer the products.
 int ensure_frame_batch(rrm_net* net)
 {
     if (net->seq_ready) return RRM_OK;
-    for (auto& L : net->layers) if (L.d.res >= 0) return RRM_ERR_UNSUPPORTED;
+    for (auto& L : net->layers) {
+        if (L.d.res == 0) return RRM_ERR_UNSUPPORTED;       // (the input itself as a shortcut: the import keeps no per-frame rows of it)
+        if (L.d.res > 0) net->tensors[L.d.res].shortcut_source = true;
+    }
     const size_t G = SEQ_MAX_FRAMES;
     size_t need = 0;
-    for (auto& T : net->tensors) need += T.bytes() * G * (T.dtype == T_BIN ? 2 : 1);
+    for (auto& T : net->tensors) need += T.bytes() * (G * ((T.dtype == T_BIN || T.shortcut_source) ? 2 : 1) + 1);
     need += net->tensors.back().bytes() * G;
     for (auto& L : net->layers) need += (size_t)L.opixels() * L.d.c_out * 4 * (G + 1);
     if (need > ((size_t)8 << 30)) return RRM_ERR_UNSUPPORTED;          // (a stack this large keeps the frame-pipelined form)
@@ -484,7 +517,8 @@ int ensure_frame_batch(rrm_net* net)
     };
     for (auto& T : net->tensors) {
         RRM_TRY(alloc(&T.Dall, T.bytes() * G));
-        if (T.dtype == T_BIN) RRM_TRY(alloc(&T.Xnall, T.bytes() * G));
+        if (T.dtype == T_BIN || T.shortcut_source) RRM_TRY(alloc(&T.Xnall, T.bytes() * G));
+        if (T.shortcut_source) RRM_TRY(alloc(&T.Xbefore, T.bytes()));
     }
     RRM_TRY(alloc(&net->tensors.back().Xfull, net->tensors.back().bytes() * G));
     for (auto& L : net->layers) {
