@@ -32,6 +32,9 @@
  *     makes the delta chunks of a stack (rrm_net_step_seq) add each frame's product straight onto the stored
  *     projection, as single steps do, instead of keeping it in a per-frame buffer that the epilogue merges (the
  *     default, which lets the convolution of frame t+1 run beside the epilogue of frame t; same results).
+ *     Long delta chunks of few streams (from 16 frames on with up to 2 streams, from 32 on with up to 4) do not
+ *     overlap frames at all: every kernel of a layer takes all frames of the chunk in one launch.
+ *     RRM_CHUNK_BY_LAYER=1 makes every delta chunk take that form, RRM_CHUNK_PIPELINED=1 none (same results).
  */
 #ifndef RRM_H
 #define RRM_H

@@ -214,6 +214,8 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         net->chunk_in_place = e && e[0] == '1';
         e = getenv("RRM_CHUNK_PIPELINED");
         net->chunk_pipelined = e && e[0] == '1';
+        e = getenv("RRM_CHUNK_BY_LAYER");
+        net->chunk_by_layer = e && e[0] == '1';
     }
     for (auto& L : net->layers) net->tensors[L.d.src].has_consumer = true;
     RRM_TRY(bind_readers(net));
@@ -627,14 +629,22 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
 {
     const bool dense = kind != 0, stateless = kind == 2;
     const int L = (int)net->layers.size();
-    if (kind == 0 && mask == 0 && !net->chunk_in_place && !net->chunk_pipelined) {
+    // Delta chunks go layer by layer over all frames where that pays: its epilogue gives every frame a lane of a warp, so
+    // short chunks waste lanes, and with many streams per call the frame-pipelined graph's kernels are large enough by
+    // themselves (measured on cfg1 and cfg3 int8, 1-8 streams x 8-32 frames: ahead from 16 frames on with up to 2
+    // streams, from 32 frames on with up to 4)
+    const int per_launch = T < seq_max_frames() ? T : seq_max_frames();
+    const bool by_layer = net->chunk_by_layer || (per_launch >= 16 && net->n <= 2) || (per_launch >= 32 && net->n <= 4);
+    if (kind == 0 && mask == 0 && !net->chunk_in_place && !net->chunk_pipelined && by_layer) {
         const int s = build_seq_graph(net, T);
         if (s != RRM_ERR_UNSUPPORTED && s != RRM_ERR_ALLOC) return s;
         cudaGetLastError();
     }
     RRM_TRY(ensure_chunk(net, T));
     if (stateless) RRM_TRY(ensure_stateless(net));
-    const bool split = kind == 0 && mask == 0 && !net->chunk_in_place;
+    // (with many streams per call the merge work of the split form costs more than the overlap gains: measured level at 8
+    // streams, behind at 16 on cfg3 int8)
+    const bool split = kind == 0 && mask == 0 && !net->chunk_in_place && net->n <= 8;
     if (split) RRM_TRY(ensure_split(net));
     const int S = (int)net->chunk_streams.size() < T ? (int)net->chunk_streams.size() : T;
     const bool own_arena = T <= CHUNK_ARENAS;                // every frame has an arena of its own

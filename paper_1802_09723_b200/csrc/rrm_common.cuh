@@ -278,6 +278,7 @@ struct rrm_net {
     std::vector<cudaEvent_t> ev_conv, ev_epi;
     cudaEvent_t ev_import = nullptr;
     bool seq_ready = false;                       // the buffers of the layer-by-layer chunk form exist
+    bool chunk_by_layer = false;                  // RRM_CHUNK_BY_LAYER=1: delta chunks always go layer by layer over all frames (where the stack allows)
     bool chunk_pipelined = false;                 // RRM_CHUNK_PIPELINED=1: delta chunks overlap frames instead of batching them per layer
     bool chunk_in_place = false;                  // RRM_CHUNK_INPLACE=1: delta chunks add into the stored projection (no delta-projection buffers)
     uint32_t* zeros = nullptr;                    // an all-zero bitmap as long as the longest update bitmap

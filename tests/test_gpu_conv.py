@@ -348,10 +348,15 @@ def test_cfg5_xnor_alexnet_128_frames():
 
 
 # ------------------------------------------------------------------ chunks of frames through a stack (frames overlap layer by layer)
+@pytest.mark.parametrize("by_layer", [False, True])
 @pytest.mark.parametrize("name", ["alex_f32", "alex_i8", "resnet_i8", "xnor", "alexnet_full_i8"])
-def test_stack_chunks_of_frames_equal_frame_by_frame(name):
-    """rrm_net_step_seq on a stack runs the frames of a chunk as one graph in which consecutive frames overlap;
-    every frame's output, the state after each chunk and the last frame's counters are those of Algorithm 1."""
+def test_stack_chunks_of_frames_equal_frame_by_frame(name, by_layer, monkeypatch):
+    """rrm_net_step_seq on a stack runs the frames of a chunk as one graph in which consecutive frames overlap, or
+    (by_layer: forced here, chosen by the library for long chunks of few streams) every layer over all frames of the
+    chunk in one launch; every frame's output, the state after each chunk and the last frame's counters are those of
+    Algorithm 1."""
+    if by_layer:
+        monkeypatch.setenv("RRM_CHUNK_BY_LAYER", "1")
     rrm = _rrm()
     if name == "alex_f32":
         specs, dt, hw = wl.alexnet_convs("f32", hw=99, scale=8), "f32", 99
@@ -585,7 +590,9 @@ def test_chunk_forms_agree_with_the_oracle(dtype, form, monkeypatch):
     overlapping in one graph with the frame's product kept apart; the same adding in place).  Each must give every
     frame's output, the state after the chunk and the last frame's counters of Algorithm 1 - also across a frame
     without change and a frame in which everything changes, for every input layout, two streams."""
-    if form == "pipelined":
+    if form == "layer_by_layer":
+        monkeypatch.setenv("RRM_CHUNK_BY_LAYER", "1")
+    elif form == "pipelined":
         monkeypatch.setenv("RRM_CHUNK_PIPELINED", "1")
     elif form == "in_place":
         monkeypatch.setenv("RRM_CHUNK_INPLACE", "1")
