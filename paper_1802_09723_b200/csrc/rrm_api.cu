@@ -608,6 +608,91 @@ static int build_seq_graph(rrm_net* net, int T)
     return RRM_OK;
 }
 
+// A dense chunk batched over its frames.  The frames of a dense chunk are independent, and T frames of n streams at
+// the boundary are laid out exactly like one frame of n*T streams: every kernel of the stateless dense pass is launched
+// once for up to DENSE_BATCH frames, on buffers of that size.  kind 1 (the state becomes the last frame) adds one
+// stateful dense pass of the last frame.  RRM_ERR_UNSUPPORTED: too large (the frame-pipelined graph serves it).
+constexpr int DENSE_BATCH = 32;
+
+static int ensure_dense_batch(rrm_net* net)
+{
+    if (net->dense_batch_ready) return RRM_OK;
+    size_t need = 0;
+    for (auto& X : net->tensors) {
+        if ((long long)X.pixels() * DENSE_BATCH * (long long)X.cs > (1ll << 31) - 1) return RRM_ERR_UNSUPPORTED;
+        need += X.bytes() * DENSE_BATCH;
+    }
+    for (auto& Y : net->layers) {
+        if ((long long)Y.opixels() * DENSE_BATCH * (long long)Y.d.c_out > (1ll << 31) - 1) return RRM_ERR_UNSUPPORTED;
+        need += (size_t)Y.opixels() * Y.d.c_out * 4 * DENSE_BATCH;
+    }
+    if (need > ((size_t)8 << 30)) return RRM_ERR_UNSUPPORTED;
+    for (auto& X : net->tensors) if (!X.X2b) RRM_TRY(dev_alloc(net, &X.X2b, X.bytes() * DENSE_BATCH));
+    for (auto& Y : net->layers) if (!Y.P2b) RRM_TRY(dev_alloc(net, &Y.P2b, (size_t)Y.opixels() * Y.d.c_out * 4 * DENSE_BATCH));
+    net->dense_batch_ready = true;
+    return RRM_OK;
+}
+
+static int build_dense_batch_graph(rrm_net* net, int kind, int T)
+{
+    const int L = (int)net->layers.size();
+    RRM_TRY(ensure_chunk(net, T));
+    RRM_TRY(ensure_stateless(net));
+    RRM_TRY(ensure_dense_batch(net));
+    const int parts = ceil_div(T, DENSE_BATCH), per = ceil_div(T, parts);
+    int64_t bi = 0, bo = 0;
+    tensor_bytes_boundary(net->tensors.front(), &bi);
+    tensor_bytes_boundary(net->tensors.back(), &bo);
+    cudaStream_t st = net->cap_stream;
+    const int n0 = net->n;
+    // the stack with F times as many streams, on the large buffers (restored below)
+    auto scale = [&](int F) {
+        net->n = n0 * F;
+        for (auto& X : net->tensors) { X.n = n0 * F; std::swap(X.X2, X.X2b); }
+        for (auto& Y : net->layers) { Y.d.n = n0 * F; std::swap(Y.P2, Y.P2b); }
+    };
+    auto unscale = [&]() {
+        net->n = n0;
+        for (auto& X : net->tensors) { X.n = n0; std::swap(X.X2, X.X2b); }
+        for (auto& Y : net->layers) { Y.d.n = n0; std::swap(Y.P2, Y.P2b); }
+    };
+    int status = RRM_OK;
+    auto fail = [&](int s) { if (status == RRM_OK && s != RRM_OK) status = s; };
+    RRM_CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    if (cudaMemsetAsync(net->chunk_arena[0], 0, net->cleared_bytes, st) != cudaSuccess) fail(RRM_ERR_CUDA);
+    for (int m0 = 0; m0 < T && status == RRM_OK; m0 += per) {
+        const int F = T - m0 < per ? T - m0 : per;
+        scale(F);
+        fail(launch_import(net, reinterpret_cast<const char*>(net->chunk_in) + (size_t)m0 * bi, false, true, st));
+        for (int l = 0; l < L && status == RRM_OK; ++l) fail(launch_layer(net, l, true, true, st));
+        fail(launch_export_tensor(net, L, reinterpret_cast<char*>(net->chunk_out) + (size_t)m0 * bo, true, st));
+        unscale();
+    }
+    if (kind == 1 && status == RRM_OK) {
+        // the state becomes the last frame (a precise inference: the accumulated truncation error is cleared)
+        bind_arena(net, net->chunk_arena[0]);
+        if (bind_readers(net) != RRM_OK) fail(RRM_ERR_UNSUPPORTED);
+        fail(launch_import(net, reinterpret_cast<const char*>(net->chunk_in) + (size_t)(T - 1) * bi, false, false, st));
+        for (int l = 0; l < L && status == RRM_OK; ++l) fail(launch_layer(net, l, true, false, st));
+        if (cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, st) != cudaSuccess) fail(RRM_ERR_CUDA);
+    }
+    cudaGraph_t g = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(st, &g);
+    if (status != RRM_OK || e != cudaSuccess || !g) {
+        if (g) cudaGraphDestroy(g);
+        cudaGetLastError();
+        return status != RRM_OK ? status : RRM_ERR_CUDA;
+    }
+    RRM_TRY(keep_chunk_graph(net, kind, T, 0, g, 0));
+    if (getenv("RRM_DEBUG")) {
+        size_t nodes = 0;
+        cudaGraphGetNodes(g, nullptr, &nodes);
+        fprintf(stderr, "rrm: chunk graph (%s, %d frames, batched over the frames): %zu nodes, %d part(s)\n",
+                kind == 1 ? "keyframes" : "dense", T, nodes, parts);
+    }
+    return RRM_OK;
+}
+
 // T frames as one graph.  Frame t is captured on stream t mod S with arena t mod S; inside a frame the launches
 // follow each other on that stream.  Across frames, in the in-place form (keyframes, dense passes, delta chunks with
 // a layer evaluated densely, RRM_CHUNK_INPLACE=1):
@@ -637,6 +722,11 @@ int build_chunk_graph(rrm_net* net, int kind, int T, unsigned long long mask)
     const bool by_layer = net->chunk_by_layer || (per_launch >= 16 && net->n <= 2) || (per_launch >= 32 && net->n <= 4);
     if (kind == 0 && mask == 0 && !net->chunk_in_place && !net->chunk_pipelined && by_layer) {
         const int s = build_seq_graph(net, T);
+        if (s != RRM_ERR_UNSUPPORTED && s != RRM_ERR_ALLOC) return s;
+        cudaGetLastError();
+    }
+    if (kind != 0 && !net->chunk_pipelined) {
+        const int s = build_dense_batch_graph(net, kind, T);
         if (s != RRM_ERR_UNSUPPORTED && s != RRM_ERR_ALLOC) return s;
         cudaGetLastError();
     }

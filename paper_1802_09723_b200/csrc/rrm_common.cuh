@@ -134,6 +134,7 @@ struct Tensor {
     void* Dall = nullptr;
     void* Xnall = nullptr;
     void* Xfull = nullptr;
+    void* X2b = nullptr;              // value buffer of a dense chunk batched over its frames (as many frames' worth as a launch takes)
     void* Xbefore = nullptr;          // tensors added as a shortcut: the value before the chunk (the snapshot moves on before the reader runs)
     bool shortcut_source = false;
     bool has_consumer = false;        // some layer reads this tensor (its int8 deltas must fit a byte)
@@ -163,6 +164,7 @@ struct Layer {
     void* Palt = nullptr;             // the second projection buffer (a copy of P is made at the start of a chunk)
     void* dP[CHUNK_RING] = {};
     size_t oact_off = 0;              // offset of the update bitmap inside an arena
+    void* P2b = nullptr;              // projection buffer of a dense chunk batched over its frames
     void* dPall = nullptr;            // per-frame products of the layer-by-layer chunk form
     uint32_t* oact = nullptr;         // bitmap of projection pixels to update (cleared every step, set by the
                                       // kernels that produce the layer's input and shortcut tensors)
@@ -277,6 +279,7 @@ struct rrm_net {
     // `slot` (frame mod CHUNK_RING in the split form; slot 0 only otherwise)
     std::vector<cudaEvent_t> ev_conv, ev_epi;
     cudaEvent_t ev_import = nullptr;
+    bool dense_batch_ready = false;               // the buffers of the frame-batched dense chunk exist
     bool seq_ready = false;                       // the buffers of the layer-by-layer chunk form exist
     bool chunk_by_layer = false;                  // RRM_CHUNK_BY_LAYER=1: delta chunks always go layer by layer over all frames (where the stack allows)
     bool chunk_pipelined = false;                 // RRM_CHUNK_PIPELINED=1: delta chunks overlap frames instead of batching them per layer
