@@ -573,7 +573,7 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
 // int8 frames with up to 4 channels (one 4-byte word per pixel): one thread per pixel, plane reads coalesced
 // across the warp, the activity word of 32 consecutive pixels written by one lane from a ballot.
 template <bool DELTA>
-__global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
+__global__ void __launch_bounds__(256, 6) import_i8_word_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
                                                             uint32_t* act, int* pnnz, unsigned long long* nnz,
                                                             unsigned long long* npix, int* errw, int c, int h, int w,
                                                             int pixels, Readers readers, SeqFrames sf)

@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         constexpr int NQ = KW == 1 ? 4 : (KW == 2 ? 2 : 1);
         auto eval = [&](const int (&c)[NQ], pt (&best)[NQ][4]) {
             pt x[NQ][KW * KW][4], res[NQ][4];
+            pt dsum[KW == 1 ? NQ : 1][4];                    // no pool window: this frame's product, prefix-summed below
             #pragma unroll
             for (int q = 0; q < NQ; ++q) {
                 res[q][0] = res[q][1] = res[q][2] = res[q][3] = 0;
@@ -232,9 +233,35 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                     const size_t o = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out + c[q];
                     // the position's projection in this lane's frame: that of the latest frame up to it that updated the
                     // position (written there by project_seq_kernel), else the projection before the chunk
-                    const unsigned upto = uf[wi] & (0xffffffffu >> (31 - lane));
-                    const pt* src = upto ? dP + (size_t)(31 - __clz(upto)) * p.p_stride : P;
-                    load4<pt, pt4>(src, o, vec, c[q], p.c_out, x[q][wi]);
+                    if (KW == 1) {
+                        // without a pool window a projection pixel belongs to one output pixel, so the prefix sum over the
+                        // frames is taken right here (project_seq_kernel is not run for such a layer)
+                        load4<pt, pt4>(P, o, vec, c[q], p.c_out, x[q][wi]);
+                        dsum[q][0] = dsum[q][1] = dsum[q][2] = dsum[q][3] = 0;
+                        if (ub & 1u) load4<pt, pt4>(dP + (size_t)lane * p.p_stride, o, vec, c[q], p.c_out, dsum[q]);
+                    } else {
+                        const unsigned upto = uf[wi] & (0xffffffffu >> (31 - lane));
+                        const pt* src = upto ? dP + (size_t)(31 - __clz(upto)) * p.p_stride : P;
+                        load4<pt, pt4>(src, o, vec, c[q], p.c_out, x[q][wi]);
+                    }
+                }
+            }
+            if (KW == 1 && on_frames) {
+                pt* Q = reinterpret_cast<pt*>(p.Q);
+                #pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (c[q] < 0) continue;                  // uniform inside the warp
+                    scan4(dsum[q], lane);
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) x[q][0][j] += dsum[q][j];
+                    if (lane == 31 && c[q] < p.c_out) {      // the sum over all frames: the stored projection (not for padding channels)
+                        const size_t o = (size_t)(qbase + y0 * p.ow + x0) * p.c_out + c[q];
+                        if (vec) { pt4 t; t.x = x[q][0][0]; t.y = x[q][0][1]; t.z = x[q][0][2]; t.w = x[q][0][3]; *reinterpret_cast<pt4*>(Q + o) = t; }
+                        else {
+                            #pragma unroll
+                            for (int j = 0; j < 4; ++j) if (c[q] + j < p.c_out) Q[o + j] = x[q][0][j];
+                        }
+                    }
                 }
             }
             #pragma unroll
@@ -473,7 +500,7 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
     e.frames = frames; e.row_stride = (long long)out.bytes(); e.arena_stride = arena_stride;
     e.p_stride = (long long)L.opixels() * d.c_out;
     e.opix = L.opixels();
-    {
+    if (d.pool_k > 1) {                                      // (without a pool window the epilogue sums the frames' products itself)
         ProjSeqParams q{};
         q.R = L.Palt; q.Q = L.P; q.dP = L.dPall; q.oact = L.oact;
         q.frames = frames; q.c_out = d.c_out; q.opix = L.opixels();
