@@ -573,34 +573,22 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
 // int8 frames with up to 4 channels (one 4-byte word per pixel): one thread per pixel, plane reads coalesced
 // across the warp, the activity word of 32 consecutive pixels written by one lane from a ballot.
 template <bool DELTA>
-__global__ void __launch_bounds__(256, 6) import_i8_word_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
+__global__ void __launch_bounds__(256) import_i8_word_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
                                                             uint32_t* act, int* pnnz, unsigned long long* nnz,
                                                             unsigned long long* npix, int* errw, int c, int h, int w,
-                                                            int pixels, Readers readers, SeqFrames sf)
+                                                            int pixels, Readers readers)
 {
     const int gp = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
     const int hw = h * w;
-    const bool seq = DELTA && sf.frames > 1;                 // (see import_nchw_kernel)
-    if (seq) {
-        const long long g = blockIdx.z;
-        src += g * sf.in_stride;
-        D = shift_bytes(D, g * sf.row_stride);
-        act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
-        npix = shift_bytes(npix, g * sf.arena_stride);
-        shift_readers(readers, g * sf.arena_stride);
-    }
-    const bool write_x = !seq || (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
     int cnt = 0;
     if (gp < pixels) {
         const int ns = gp / hw, pix = gp - ns * hw;
-        uint32_t nw = 0, pw = 0;
+        uint32_t nw = 0;
         for (int ch = 0; ch < c; ++ch) nw |= ((uint32_t)(uint8_t)src[((size_t)ns * c + ch) * hw + pix]) << (8 * ch);
-        if (seq) for (int ch = 0; ch < c; ++ch) pw |= ((uint32_t)(uint8_t)(src - sf.in_stride)[((size_t)ns * c + ch) * hw + pix]) << (8 * ch);
         if (DELTA) {
-            const uint32_t ow = seq ? pw : X[gp];
-            if (seq && write_x) X[gp] = nw;
+            const uint32_t ow = X[gp];
             if (nw != ow) {
                 uint32_t dw = 0;
                 #pragma unroll
@@ -611,7 +599,7 @@ __global__ void __launch_bounds__(256, 6) import_i8_word_kernel(const int8_t* __
                     cnt += d != 0;
                 }
                 D[gp] = dw;
-                if (!seq) X[gp] = nw;
+                X[gp] = nw;
                 pnnz[gp] = cnt;
             }
         } else {
@@ -637,6 +625,81 @@ __global__ void __launch_bounds__(256, 6) import_i8_word_kernel(const int8_t* __
     if (lane == 0) {
         #pragma unroll
         for (int i = 0; i < MAX_READERS; ++i) if (i < readers.n && wsum[i]) atomicAdd(readers.r[i].macs, wsum[i]);
+    }
+}
+
+// The same for several consecutive frames in one launch (frame = blockIdx.z): frame g is compared with frame g-1 at
+// the boundary (see import_nchw_kernel), the snapshot is written by the last frame.  A warp takes 128 consecutive
+// pixels, lane l the pixels l, l + 32, l + 64, l + 96 of them: all 24 plane reads of a thread are in flight together,
+// and each group of 32 pixels still owns its activity word.
+__global__ void __launch_bounds__(256, 4) import_i8_word_frames_kernel(const int8_t* __restrict__ src, uint32_t* X, uint32_t* D,
+                                                                      uint32_t* act, unsigned long long* nnz,
+                                                                      unsigned long long* npix, int* errw, int c, int h, int w,
+                                                                      int pixels, Readers readers, SeqFrames sf)
+{
+    const int lane = threadIdx.x & 31;
+    const int base = (blockIdx.x * 8 + (threadIdx.x >> 5)) * 128;
+    const int hw = h * w;
+    {
+        const long long g = blockIdx.z;
+        src += g * sf.in_stride;
+        D = shift_bytes(D, g * sf.row_stride);
+        act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
+        npix = shift_bytes(npix, g * sf.arena_stride);
+        shift_readers(readers, g * sf.arena_stride);
+    }
+    const bool write_x = (int)blockIdx.z == sf.frames - 1;
+    pdl_launch_dependents();
+    pdl_wait();
+    uint32_t nw[4], pw[4];
+    #pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int gp = base + 32 * k + lane;
+        nw[k] = pw[k] = 0;
+        if (gp >= pixels) continue;
+        const int ns = gp / hw, pix = gp - ns * hw;
+        for (int ch = 0; ch < c; ++ch) {
+            const size_t o = ((size_t)ns * c + ch) * hw + pix;
+            nw[k] |= ((uint32_t)(uint8_t)src[o]) << (8 * ch);
+            pw[k] |= ((uint32_t)(uint8_t)(src - sf.in_stride)[o]) << (8 * ch);
+        }
+    }
+    #pragma unroll 1
+    for (int k = 0; k < 4; ++k) {
+        const int gp = base + 32 * k + lane;
+        if (base + 32 * k >= pixels) break;                  // uniform inside the warp
+        int cnt = 0;
+        if (gp < pixels) {
+            if (write_x) X[gp] = nw[k];
+            if (nw[k] != pw[k]) {
+                uint32_t dw = 0;
+                #pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int d = (int)(int8_t)(nw[k] >> (8 * j)) - (int)(int8_t)(pw[k] >> (8 * j));
+                    if (d < -128 || d > 127) atomicOr(errw, ERRW_BOUNDS);
+                    dw |= ((uint32_t)d & 0xffu) << (8 * j);
+                    cnt += d != 0;
+                }
+                D[gp] = dw;
+            }
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
+        if (m == 0) continue;                                // uniform inside the warp
+        if (lane == 0) act[gp >> 5] = m;                     // gp of lane 0 is a multiple of 32: the word is this group's alone
+        const int tot = __reduce_add_sync(0xffffffffu, cnt);
+        if (lane == 0) {
+            atomicAdd(nnz, (unsigned long long)tot);
+            atomicAdd(npix, (unsigned long long)__popc(m));
+        }
+        unsigned long long wsum[MAX_READERS];
+        {
+            const int ns = gp / hw, pix = gp - ns * hw;
+            scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum);
+        }
+        if (lane == 0) {
+            #pragma unroll
+            for (int i = 0; i < MAX_READERS; ++i) if (i < readers.n && readers.r[i].macs && wsum[i]) atomicAdd(readers.r[i].macs, wsum[i]);
+        }
     }
 }
 
@@ -1141,12 +1204,14 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
                                                               Readers{}, (uint32_t*)nullptr, sf);
     } else if (T.dtype == T_I8 && T.cs == 4) {
         const int blocks = ceil_div(T.pixels(), 256);
-        if (delta) launch_seq(import_i8_word_kernel<true>, dim3(blocks, 1, gz), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
+        if (seq) launch_seq(import_i8_word_frames_kernel, dim3(ceil_div(T.pixels(), 1024), 1, gz), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X,
+                            (uint32_t*)T.D, T.act, T.nnz, T.npix, net->errw, T.c, T.h, T.w, T.pixels(), T.readers, sf);
+        else if (delta) launch_seq(import_i8_word_kernel<true>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, (uint32_t*)T.D, T.act,
                                                                       T.pnnz, T.nnz, T.npix, net->errw, T.c, T.h, T.w,
-                                                                      T.pixels(), T.readers, sf);
+                                                                      T.pixels(), T.readers);
         else launch_seq(import_i8_word_kernel<false>, dim3(blocks), dim3(256), 0, st, (const int8_t*)frame, (uint32_t*)X, nullptr, nullptr, nullptr,
                                                                   nullptr, nullptr, net->errw, T.c, T.h, T.w, T.pixels(),
-                                                                  Readers{}, sf);
+                                                                  Readers{});
     } else {
         dim3 grid(ceil_div(hw, IMP_TP), T.n, gz);
         const size_t smem = (size_t)IMP_TP * (T.cs + 1) * T.unit_bytes * (seq ? 2 : 1);
