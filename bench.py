@@ -248,7 +248,7 @@ def run_reference(args, rank, world):
 # Convolution configurations.  One step = one frame of every stream through rrm_net_step (Algorithm 1, one
 # iteration of the frame loop).
 # ------------------------------------------------------------------------------------------------
-CONV_WORKLOADS = ("cfg1", "cfg3_f32", "cfg3_i8", "cfg4", "cfg5")
+CONV_WORKLOADS = ("cfg1", "cfg3_f32", "cfg3_i8", "cfg4", "cfg5", "cfg3_i8_quiet")
 
 
 def conv_workload(name, frames=None, streams=None):
@@ -263,6 +263,12 @@ def conv_workload(name, frames=None, streams=None):
     if name == "cfg3_i8":
         n = streams or 1
         return wl.alexnet_convs("i8"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="i8", seed=32, n=n), n, "i8"
+    if name == "cfg3_i8_quiet":
+        # not one of the contract's configurations: the cfg3 stack on a quieter video (one 24-32 px rectangle moving
+        # 1-2 px per frame instead of three of 32-64 px moving 1-4 px), to show how the delta path follows the density
+        n = streams or 1
+        return (wl.alexnet_convs("i8"), wl.moving_rect_video(frames=frames or 64, hw=227, dtype="i8", seed=33, n=n, n_rect=1,
+                                                             side=(24, 32), speed=(1, 2)), n, "i8")
     if name == "cfg4":
         n = streams or 4
         return (wl.resnet18_convs(), wl.moving_rect_video(frames=frames or 64, hw=224, dtype="i8", seed=41, n=n,
@@ -866,7 +872,8 @@ def main():
     if rank == 0 and world == 1 and not args.quick:
         conv = {}
         for key, name, variant, fr_n, cpu_n in (("cfg1", "cfg1", "auto", None, 2), ("cfg3_f32", "cfg3_f32", "auto", 16, 1),
-                                                ("cfg3_i8", "cfg3_i8", "auto", 16, 2), ("cfg5", "cfg5", "auto", 16, 1),
+                                                ("cfg3_i8", "cfg3_i8", "auto", 16, 2), ("cfg3_i8_quiet_video", "cfg3_i8_quiet", "auto", 16, 0),
+                                                ("cfg5", "cfg5", "auto", 16, 1),
                                                 ("cfg4_delta_forced", "cfg4", "tensor", 8, 1), ("cfg4_auto", "cfg4", "auto", 8, 0)):
             try:
                 conv[key] = compact_conv(conv_measure(name, variant, steps=30, warmup=5, frames=fr_n, cpu_frames=cpu_n,
@@ -875,8 +882,9 @@ def main():
                 conv[key] = {"error": str(e)}
         conv["note"] = ("one step = one frame of every stream through rrm_net_step, median of 30 cold-L2 steps; S / S0 / eta: "
                         "Eq. 9 and Eq. 10 from the measured per-layer densities; chunk: 32 consecutive frames per rrm_net_step_seq "
-                        "call (delta) / rrm_net_dense_seq call (dense), cold L2, median, per frame; cpu_baseline: the oracle on "
-                        "the host cores")
+                        "call (delta) / rrm_net_dense_seq call (dense), cold L2, median, per frame; cfg3_i8_quiet_video: the cfg3 "
+                        "stack on a quieter video (one 24-32 px rectangle moving 1-2 px per frame), not a contract configuration; "
+                        "cpu_baseline: the oracle on the host cores")
 
     # ---- CPU oracle on the host cores (rank 0, N = 1 only): a bounded sample of the same workload
     cpu = None
