@@ -74,7 +74,10 @@ struct TcSmemTail {
 };
 constexpr size_t TC_STAGE_BYTES = (size_t)TC_M * TC_SLAB + (size_t)TC_MAX_BN * TC_SLAB;
 constexpr size_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + sizeof(TcSmemTail);
-constexpr int TC_LAG = TC_STAGES - 1;         // slabs whose asynchronous copies may still be in flight
+constexpr int TC_LAG = 1;                     // a slab is handed to the tensor core when the next one has been issued (its copies
+                                              // have landed by then); handing it over one slab later still, with the third stage's
+                                              // copies in flight too, left the stage's MMAs too little time to commit before the
+                                              // producers want the stage back (measured: 3-5 % slower steps)
 constexpr int TC_ROW_WORDS = TC_MAX_BN + 4;   // epilogue row buffers: 16-byte aligned rows, staggered over the banks
 static_assert((size_t)TC_M * TC_ROW_WORDS * 4 <= TC_STAGES * TC_STAGE_BYTES, "epilogue rows reuse the stage buffers");
 
