@@ -506,6 +506,40 @@ def test_explicit_bn_stacks_every_frame(name):
     _run(specs, video, n=n, stats=True, keyframe_at=(3,))
 
 
+@pytest.mark.parametrize("by_layer", [False, True])
+@pytest.mark.parametrize("name", ["alex_f32", "resnet_i8"])
+def test_explicit_bn_stacks_in_chunks(name, by_layer, monkeypatch):
+    """The same stacks through rrm_net_step_seq, frame-pipelined and layer by layer over all frames of a chunk:
+    every frame's output, then projections and tensors after the chunk."""
+    if by_layer:
+        monkeypatch.setenv("RRM_CHUNK_BY_LAYER", "1")
+    rrm = _rrm()
+    if name == "alex_f32":
+        specs, dt, hw, n = wl.alexnet_convs("f32", hw=99, scale=8), "f32", 99, 1
+    else:
+        specs, dt, hw, n = wl.resnet18_convs(hw=96, scale=8), "i8", 96, 2
+    wl.with_explicit_bn(specs)
+    video = wl.moving_rect_video(frames=9, hw=hw, dtype=dt, seed=37, n=n, side=(10, 20))
+    net = rrm.net_from_specs(specs, n=n)
+    frames = dev(np.ascontiguousarray(video))
+    t0 = 0
+    for T in (5, 4):
+        outs = net.new_output(frames=T)
+        net.step_seq(frames[t0:t0 + T], outs, T)
+        for i in range(T):
+            want = orc.dense_forward(specs, video[t0 + i])[0][len(specs)]
+            got = outs[i].cpu().numpy()
+            if dt == "f32":
+                assert float(np.abs(got - want).max()) <= F32_TOL * max(1e-30, float(np.abs(want).max())), t0 + i
+            else:
+                np.testing.assert_array_equal(got.astype(np.int64), want, err_msg=f"frame {t0 + i}")
+        t0 += T
+        _compare(specs, net, video[t0 - 1], t0 - 1)
+    for l in range(len(specs)):
+        assert net.stats(l)["error_word"] == 0
+    net.close()
+
+
 def test_explicit_bn_equals_the_folded_stack_on_the_gpu():
     """fp32: the stack with its affines unfolded and the stack with them folded into filters and bias give the same
     tensors within the fp32 tolerance, on the library's delta path."""
