@@ -140,6 +140,12 @@ typedef struct {
     float fc_dense_rows;         /* lone int8 FC layer, chunks: rows x measured density from which on a chunk is
                                     evaluated densely on the tensor cores, per launch that evaluation needs */
     float fc_dense_density;      /* the same for chunks of more rows than the few-row kernel takes: plain density */
+    float chunk_dense_activity;  /* stacks whose layers all run on the tensor cores, variant AUTO, chunks of 16 or more
+                                    frames of up to 4 streams (rrm_net_step_seq): MAC-weighted share of projection
+                                    pixels to update from which on the next chunks are evaluated densely, batched over
+                                    their frames (same results; a delta chunk measures again after stack_reprobe dense
+                                    ones).  Default 0.40: measured, the two kinds of chunk are level at about a third
+                                    of the pixels active */
 } rrm_options;
 
 /* ---- single layer (Eq. 2-5) ------------------------------------------------------- */

@@ -36,7 +36,8 @@ class Stats(ctypes.Structure):
 class Options(ctypes.Structure):
     _fields_ = [("wait_limit", ctypes.c_uint32), ("layer_dense_activity", ctypes.c_float),
                 ("layer_delta_activity", ctypes.c_float), ("stack_dense_activity", ctypes.c_float),
-                ("stack_reprobe", ctypes.c_int32), ("fc_dense_rows", ctypes.c_float), ("fc_dense_density", ctypes.c_float)]
+                ("stack_reprobe", ctypes.c_int32), ("fc_dense_rows", ctypes.c_float), ("fc_dense_density", ctypes.c_float),
+                ("chunk_dense_activity", ctypes.c_float)]
 
 
 _lib = None

@@ -200,6 +200,11 @@ int build_net(rrm_net* net, const rrm_layer_desc* descs, int n_layers, const voi
         }
         net->auto_switch = all_auto && macs >= 1000000000ll;
         net->layer_switch = all_auto && n_layers <= 64;
+        {
+            bool all_tc = true;
+            for (auto& L : net->layers) all_tc = all_tc && L.tc_ready;
+            net->chunk_switch = all_auto && all_tc && n_layers <= 64;
+        }
         // an all-ones bitmap stands in for a layer's update bitmap when the layer is evaluated densely inside a delta step
         int words = 1;
         for (auto& L : net->layers) words = words > ceil_div(L.opixels(), 32) ? words : ceil_div(L.opixels(), 32);
@@ -669,11 +674,12 @@ static int build_dense_batch_graph(rrm_net* net, int kind, int T)
         unscale();
     }
     if (kind == 1 && status == RRM_OK) {
-        // the state becomes the last frame (a precise inference: the accumulated truncation error is cleared)
+        // the state becomes the last frame (a precise inference: the accumulated truncation error is cleared): its
+        // tensors and projections are copied out of the last part's batched buffers
         bind_arena(net, net->chunk_arena[0]);
         if (bind_readers(net) != RRM_OK) fail(RRM_ERR_UNSUPPORTED);
-        fail(launch_import(net, reinterpret_cast<const char*>(net->chunk_in) + (size_t)(T - 1) * bi, false, false, st));
-        for (int l = 0; l < L && status == RRM_OK; ++l) fail(launch_layer(net, l, true, false, st));
+        const int last_part_frames = T - (parts - 1) * per;
+        fail(launch_copy_state_from_batch(net, last_part_frames - 1, st));
         if (cudaMemsetAsync(net->aecs, 0, (1 + net->layers.size()) * 8, st) != cudaSuccess) fail(RRM_ERR_CUDA);
     }
     cudaGraph_t g = nullptr;
@@ -851,7 +857,12 @@ int run_chunk(rrm_net* net, const void* frames, void* outs, int T, cudaStream_t 
         net->last_step_dense = false;
         if (net->auto_switch || net->layer_switch) {
             activity_poll(net);
-            if (net->auto_switch && net->activity >= net->opt.stack_dense_activity && net->dense_streak < net->opt.stack_reprobe) {
+            // long chunks of few streams have a batched dense form that needs no change detection, marking or prefix
+            // sums: on tensor-core stacks it is ahead from a lower activity on than the whole-stack switch of single steps
+            const bool long_chunk = net->chunk_switch && T >= 16 && net->n <= 4 && !net->chunk_pipelined;
+            const bool go_dense = (net->auto_switch && net->activity >= net->opt.stack_dense_activity) ||
+                                  (long_chunk && net->activity >= net->opt.chunk_dense_activity);
+            if (go_dense && net->dense_streak < net->opt.stack_reprobe) {
                 ++net->dense_streak;                         // (counted in calls: a delta chunk measures again after 15 dense ones)
                 net->last_step_dense = true;
                 dense = true;
@@ -1305,7 +1316,8 @@ int rrm_net_set_options(rrm_net* net, const rrm_options* in)
 {
     if (!net || !in) return RRM_ERR_INVALID_ARG;
     if (!(in->layer_dense_activity >= 0.f) || !(in->layer_delta_activity >= 0.f) || in->layer_delta_activity > in->layer_dense_activity ||
-        !(in->stack_dense_activity >= 0.f) || in->stack_reprobe < 1 || !(in->fc_dense_rows >= 0.f) || !(in->fc_dense_density >= 0.f))
+        !(in->stack_dense_activity >= 0.f) || in->stack_reprobe < 1 || !(in->fc_dense_rows >= 0.f) || !(in->fc_dense_density >= 0.f) ||
+        !(in->chunk_dense_activity >= 0.f))
         return RRM_ERR_INVALID_ARG;
     RRM_CUDA_TRY(cudaDeviceSynchronize());
     net->opt = *in;

@@ -305,11 +305,12 @@ struct rrm_net {
     int dense_streak = 0;                     // dense frames since the last measured delta frame
     bool last_step_dense = false;             // the most recent rrm_net_step was evaluated densely
     bool auto_switch = false;                 // every layer asks for RRM_VARIANT_AUTO and the net is large enough
+    bool chunk_switch = false;                // every layer asks for RRM_VARIANT_AUTO and runs on the tensor cores: long chunks may go dense
     // the defaults rrm_net_get_options reports.  (The per-layer thresholds are above 1, i.e. the per-layer choice is off
     // until the caller lowers them: measured on B200, a dense evaluation of one layer inside a delta step is never
     // faster than its sparse product, not even with every pixel active.  What a delta step pays for is change
     // detection and marking, which only a dense pass of the whole stack drops.)
-    rrm_options opt = {1u << 20, 1.01f, 1.005f, 0.75f, 15, 0.75f, 0.08f};
+    rrm_options opt = {1u << 20, 1.01f, 1.005f, 0.75f, 15, 0.75f, 0.08f, 0.40f};
     float eps = 0.f;                  // Sec. 3.4: fp32 delta entries below it are truncated (0: exact)
     double* aecs = nullptr;           // [1 + layers]: accumulated truncated value e_t (Eq. 7), then the last step's l2 per layer
     std::vector<void*> allocs;        // everything to free
@@ -373,6 +374,7 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
 int ensure_frame_batch(rrm_net* net);
 int seq_max_frames();
 int launch_copy_projections(rrm_net* net, cudaStream_t st);
+int launch_copy_state_from_batch(rrm_net* net, int slot, cudaStream_t st);
 int launch_zero_delta_projections(rrm_net* net, int slot, cudaStream_t st);
 int clear_split(rrm_net* net, cudaStream_t st);
 

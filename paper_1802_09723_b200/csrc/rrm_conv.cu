@@ -21,6 +21,8 @@
 #include "rrm_tc.cuh"
 #include "rrm_dev.cuh"
 #include <type_traits>
+#include <array>
+#include <vector>
 
 namespace rrm {
 
@@ -1431,6 +1433,43 @@ int clear_split(rrm_net* net, cudaStream_t st)
     for (auto& L : net->layers)
         for (int k = 0; k < CHUNK_RING; ++k)
             if (L.dP[k]) RRM_CUDA_TRY(cudaMemsetAsync(L.dP[k], 0, (size_t)L.opixels() * L.d.c_out * 4, st));
+    return RRM_OK;
+}
+
+// The state becomes frame `slot` of a dense pass that was batched over frames: every tensor's value and every layer's
+// projection are copied out of the batched buffers.
+int launch_copy_state_from_batch(rrm_net* net, int slot, cudaStream_t st)
+{
+    std::vector<std::array<const void*, 2>> ptr;
+    std::vector<long long> words;
+    for (auto& T : net->tensors) {
+        if (!T.X2b) return RRM_ERR_INVALID_ARG;
+        ptr.push_back({reinterpret_cast<const char*>(T.X2b) + (size_t)slot * T.bytes(), T.X});
+        words.push_back((long long)(T.bytes() / 4));
+    }
+    for (auto& L : net->layers) {
+        if (!L.P2b) return RRM_ERR_INVALID_ARG;
+        const size_t bytes = (size_t)L.opixels() * L.d.c_out * 4;
+        ptr.push_back({reinterpret_cast<const char*>(L.P2b) + (size_t)slot * bytes, L.P});
+        words.push_back((long long)(bytes / 4));
+    }
+    for (size_t j0 = 0; j0 < ptr.size(); j0 += 32) {
+        CopyJobs j;
+        j.n = (int)(ptr.size() - j0 < 32 ? ptr.size() - j0 : 32);
+        long long most = 0;
+        for (int k = 0; k < 32; ++k) {
+            if (k < j.n) {
+                j.src[k] = reinterpret_cast<const int*>(ptr[j0 + k][0]);
+                j.dst[k] = reinterpret_cast<int*>(const_cast<void*>(ptr[j0 + k][1]));
+                j.words[k] = words[j0 + k];
+                most = most > j.words[k] ? most : j.words[k];
+            } else { j.src[k] = nullptr; j.dst[k] = nullptr; j.words[k] = 0; }
+        }
+        long long gx = (most / 4 + 255) / 256;
+        gx = gx < 1 ? 1 : (gx > 148 ? 148 : gx);
+        launch_seq(copy_projections_kernel, dim3((unsigned)gx, (unsigned)j.n), dim3(256), 0, st, j);
+    }
+    RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
 

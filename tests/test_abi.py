@@ -39,7 +39,7 @@ def test_null_arguments_are_rejected_without_a_device():
     assert L.rrm_net_tensor_bytes(None, 0) == -1
     assert L.rrm_net_get_options(None, None) == -1 and L.rrm_net_set_options(None, None) == -1
     assert L.rrm_net_clear_errors(None) == -1
-    assert ctypes.sizeof(rrm.Options) == 7 * 4
+    assert ctypes.sizeof(rrm.Options) == 8 * 4
 
 
 def test_product_package_does_not_import_the_oracle():

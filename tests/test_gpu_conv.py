@@ -442,6 +442,35 @@ def test_large_stack_chunks_go_dense_while_nearly_every_pixel_changes():
     net.close()
 
 
+def test_long_chunks_of_a_tensor_core_stack_go_dense_from_the_measured_activity():
+    """rrm_options.chunk_dense_activity: after a delta chunk that measured a high share of pixels to update, the next
+    long chunks of an int8 stack are evaluated densely, batched over their frames; outputs and state stay exact, and
+    with the threshold out of reach the library stays on the delta path."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8", hw=99, scale=8)
+    video = wl.moving_rect_video(frames=65, hw=99, dtype="i8", seed=43, n=1, side=(12, 24), bg_redraw=0.10)
+    net = rrm.net_from_specs(specs, n=1)
+    assert abs(net.options()["chunk_dense_activity"] - 0.40) < 1e-6
+    frames = dev(np.ascontiguousarray(video))
+    variants = []
+    for k in range(4):
+        if k == 3:
+            net.set_options(chunk_dense_activity=2.0)
+        outs = net.new_output(frames=16)
+        net.step_seq(frames[16 * k:16 * k + 16], outs, 16)
+        st = net.stats(1)                     # synchronises, so the next call sees this chunk's counters
+        variants.append(st["variant"])
+        for i in (0, 7, 15):
+            want = orc.dense_forward(specs, video[16 * k + i])[0][len(specs)]
+            np.testing.assert_array_equal(outs[i].cpu().numpy().astype(np.int64), want, err_msg=f"frame {16 * k + i}")
+        _compare(specs, net, video[16 * k + 15], 16 * k + 15)
+    assert variants[0] != 3 and variants[1] == 3 and variants[2] == 3 and variants[3] != 3, variants
+    out = net.new_output()
+    net.step(dev(video[64]), out)
+    _compare(specs, net, video[64], 64)
+    net.close()
+
+
 def test_stack_chunks_through_the_pipelined_host_entry_point():
     """Host buffers in, host buffers out, calls queued without waiting: a stack's chunks through
     rrm_net_step_seq_host_async deliver every frame's output."""
