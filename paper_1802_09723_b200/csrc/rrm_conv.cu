@@ -482,8 +482,8 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
         D = shift_bytes(D, g * sf.row_stride);
         act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
         npix = shift_bytes(npix, g * sf.arena_stride);
-        shift_readers(readers, g * sf.arena_stride);
     }
+    const long long arena_off = seq ? (long long)blockIdx.z * sf.arena_stride : 0;
     const bool write_x = !seq || (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
@@ -561,14 +561,14 @@ __global__ void __launch_bounds__(256) import_nchw_kernel(const T* __restrict__ 
         const int pix = pix0 + lane;
         const int cnt = pix < hw ? s_cnt[lane] : 0;
         unsigned long long macs[MAX_READERS];
-        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, macs);
+        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, macs, arena_off);
         if (lane == 0) {
             #pragma unroll
             for (int i = 0; i < MAX_READERS; ++i) if (macs[i]) s_macs[i] = macs[i];
         }
     }
     __syncthreads();
-    if (tid < readers.n && s_macs[tid]) atomicAdd(readers.r[tid].macs, s_macs[tid]);
+    if (tid < readers.n && s_macs[tid] && readers.r[tid].macs) atomicAdd(shift_bytes(readers.r[tid].macs, arena_off), s_macs[tid]);
     if (tid == 0 && trunc && s_sq > 0.f) atomicAdd(trunc, (double)s_sq);
 }
 
@@ -648,8 +648,8 @@ __global__ void __launch_bounds__(256, 4) import_i8_word_frames_kernel(const int
         D = shift_bytes(D, g * sf.row_stride);
         act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
         npix = shift_bytes(npix, g * sf.arena_stride);
-        shift_readers(readers, g * sf.arena_stride);
     }
+    const long long arena_off = (long long)blockIdx.z * sf.arena_stride;
     const bool write_x = (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
@@ -696,11 +696,12 @@ __global__ void __launch_bounds__(256, 4) import_i8_word_frames_kernel(const int
         unsigned long long wsum[MAX_READERS];
         {
             const int ns = gp / hw, pix = gp - ns * hw;
-            scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum);
+            scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum, arena_off);
         }
         if (lane == 0) {
             #pragma unroll
-            for (int i = 0; i < MAX_READERS; ++i) if (i < readers.n && readers.r[i].macs && wsum[i]) atomicAdd(readers.r[i].macs, wsum[i]);
+            for (int i = 0; i < MAX_READERS; ++i)
+                if (i < readers.n && readers.r[i].macs && wsum[i]) atomicAdd(shift_bytes(readers.r[i].macs, arena_off), wsum[i]);
         }
     }
 }
@@ -720,8 +721,8 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
         if (Xn) Xn = shift_bytes(Xn, g * sf.row_stride);
         act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
         npix = shift_bytes(npix, g * sf.arena_stride);
-        shift_readers(readers, g * sf.arena_stride);
     }
+    const long long arena_off = seq ? (long long)blockIdx.z * sf.arena_stride : 0;
     const bool write_x = !seq || (int)blockIdx.z == sf.frames - 1;
     pdl_launch_dependents();
     pdl_wait();
@@ -756,11 +757,12 @@ __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X,
     unsigned long long wsum[MAX_READERS];
     {
         const int ns = gp / (w * h), pix = gp - ns * (w * h);
-        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum);
+        scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum, arena_off);
     }
     if (lane == 0) {
         #pragma unroll
-        for (int i = 0; i < MAX_READERS; ++i) if (i < readers.n && wsum[i]) atomicAdd(readers.r[i].macs, wsum[i]);
+        for (int i = 0; i < MAX_READERS; ++i)
+            if (i < readers.n && readers.r[i].macs && wsum[i]) atomicAdd(shift_bytes(readers.r[i].macs, arena_off), wsum[i]);
     }
 }
 

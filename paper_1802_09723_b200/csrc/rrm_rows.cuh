@@ -16,8 +16,10 @@ namespace rrm {
 // in runs along an image row, so the marking is done per row segment of the warp, not per pixel: lane j tests
 // candidate projection column ox_min + j against the segment's mask of changed pixels, a ballot gives the columns
 // as a run of bits, and lane r ORs that run into projection row oy_lo + r (one or two word-wide atomic ORs).
+// arena_off: byte offset of the arena whose bitmaps are marked from the one the readers' pointers refer to (several
+// frames per launch: frame g's arena).
 __device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, int y, int x, int cnt, int lane,
-                                                     unsigned long long (&macs)[MAX_READERS])
+                                                     unsigned long long (&macs)[MAX_READERS], long long arena_off = 0)
 {
     const unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
     #pragma unroll
@@ -71,22 +73,12 @@ __device__ __forceinline__ void scatter_changed_warp(const Readers& R, int ns, i
                 for (int r = oy_lo + lane; r <= oy_hi; r += 32) {
                     const int q0 = (sns * c.oh + r) * c.ow + c0;
                     const unsigned long long v = (unsigned long long)run << (q0 & 31);
-                    atomicOr(&c.oact[q0 >> 5], (unsigned)v);
-                    if (v >> 32) atomicOr(&c.oact[(q0 >> 5) + 1], (unsigned)(v >> 32));
+                    uint32_t* bm = shift_bytes(c.oact, arena_off);
+                    atomicOr(&bm[q0 >> 5], (unsigned)v);
+                    if (v >> 32) atomicOr(&bm[(q0 >> 5) + 1], (unsigned)(v >> 32));
                 }
             }
         }
-    }
-}
-
-// the readers' bitmaps and counters of frame g's arena
-__device__ __forceinline__ void shift_readers(Readers& R, long long bytes)
-{
-    #pragma unroll
-    for (int i = 0; i < MAX_READERS; ++i) {
-        if (i >= R.n) break;
-        R.r[i].oact = shift_bytes(R.r[i].oact, bytes);
-        if (R.r[i].macs) R.r[i].macs = shift_bytes(R.r[i].macs, bytes);
     }
 }
 
