@@ -58,6 +58,9 @@ struct TcParams {
     long long arena_stride;   // bytes between the frames' arenas (bitmaps, counters)
     long long p_stride;       // elements between the frames' products
     int store;                // delta: the product is stored, not added (ksplit 1: every row written belongs to one CTA)
+    // ceil(2^32 / d) for d = chunks_per_tap and d = kw: the K loop divides by them in every iteration of every role,
+    // and its single-thread roles are bound by the length of their instruction chains (exact for the small operands here)
+    unsigned magic_cpt, magic_kw;
 };
 
 // byte i of the result = bit i of the low nibble of x (0 or 1)
@@ -69,6 +72,7 @@ struct TcSmemTail {
     uint32_t tmem_base;
     int fail;
     unsigned long long tap_mask[2];           // taps with a usable input under at least one row of this tile (up to 128 taps)
+    uint32_t live[8];                         // bit r: slab s_begin + r has a usable tap (the first 256 slabs of the CTA's range)
     unsigned long long rmask[TC_M][2];        // per row: taps whose input pixel is inside the image (and changed, delta mode)
     int q[TC_M], pix0[TC_M];                  // projection pixel of the row; input pixel under tap (0,0) (may be outside)
 };
@@ -120,6 +124,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
         mbar_init(smem_u32(&S->done), 1);
         S->fail = 0;
         S->tap_mask[0] = S->tap_mask[1] = 0ull;
+        for (int i = 0; i < 8; ++i) S->live[i] = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 4) {                                        // tensor memory for the accumulator tile
@@ -181,10 +186,25 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             if (t < 64 ? (tm0 >> t) & 1ull : (tm1 >> (t - 64)) & 1ull) return true;
         return false;
     };
+    // which slabs are live is worked out once, by all threads, and kept as a bitmap: the roles' loops then find their
+    // next slab with a shift instead of divisions (ranges beyond 256 slabs test the rest slab by slab)
+    const int n_range = s_end - s_begin;
+    for (int r = tid; r < min(n_range, 256); r += TC_THREADS)
+        if (slab_live(s_begin + r)) atomicOr(&S->live[r >> 5], 1u << (r & 31));
+    __syncthreads();
     auto next_live = [&](int ks) -> int {                   // first live slab >= ks, or s_end
+        int r = ks - s_begin;
+        while (r < min(n_range, 256)) {
+            const uint32_t wbits = S->live[r >> 5] >> (r & 31);
+            if (wbits) return s_begin + r + __ffs(wbits) - 1;
+            r = (r | 31) + 1;
+        }
+        ks = s_begin + max(r, ks - s_begin);
         while (ks < s_end && !slab_live(ks)) ++ks;
-        return ks;
+        return min(ks, s_end);
     };
+    auto div_cpt = [&](int x) -> int { return p.magic_cpt ? (int)__umulhi((unsigned)x, p.magic_cpt) : x; };   // (0: the divisor is 1)
+    auto div_kw = [&](int x) -> int { return p.magic_kw ? (int)__umulhi((unsigned)x, p.magic_kw) : x; };
     const uint32_t tile_b_bytes = (uint32_t)p.bn * TC_SLAB;
     bool ok = true;
     int n_issued = 0;                                       // slabs that went through the pipeline (same in every role)
@@ -222,7 +242,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const int tap = ks * (TC_SLAB / 4) + piece * 4 + j;
-                        const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                        const int ky = div_kw(tap), kx = tap - ky * p.kw;
                         toff[j] = (ky * p.w + kx) * 4;
                         tok[j] = tap < p.taps; thi[j] = tap >= 64; tsh[j] = tap & 63;
                     }
@@ -238,8 +258,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
                     }
                 } else {
                 const int kc = ks * 4 + (piece >> 1);       // this lane's 32-byte chunk of K
-                const int tap = kc / cpt, cc = kc - tap * cpt;
-                const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                const int tap = div_cpt(kc), cc = kc - tap * cpt;
+                const int ky = div_kw(tap), kx = tap - ky * p.kw;
                 const int slab_off = (ky * p.w + kx) * p.row_units + cc * 32 + (piece & 1) * 16;   // same for the 8 rows
                 const bool tap_ok = tap < p.taps, hi = tap >= 64;
                 const int sh = tap & 63;
@@ -281,8 +301,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) conv_tc_kernel(TcParams p)
             int half_valid = 0;
             auto fetch = [&](int ks) {
                 const int kc = ks * 4 + (piece >> 1);
-                const int tap = kc / cpt, cc = kc - tap * cpt;
-                const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                const int tap = div_cpt(kc), cc = kc - tap * cpt;
+                const int ky = div_kw(tap), kx = tap - ky * p.kw;
                 const int slab_off = (ky * p.w + kx) * p.row_units + cc;
                 const bool tap_ok = tap < p.taps, hi = tap >= 64;
                 const int sh = tap & 63;
@@ -589,6 +609,8 @@ int launch_conv_tc(rrm_net* net, Layer& L, const Tensor& in, bool dense, bool st
     p.frames = batched ? frames : 1;
     p.row_stride = (long long)in.bytes(); p.arena_stride = arena_stride; p.p_stride = (long long)L.opixels() * d.c_out;
     p.store = batched ? 1 : 0;
+    p.magic_cpt = p.chunks_per_tap > 1 ? (unsigned)(((1ull << 32) + p.chunks_per_tap - 1) / p.chunks_per_tap) : 0u;
+    p.magic_kw = p.kw > 1 ? (unsigned)(((1ull << 32) + p.kw - 1) / p.kw) : 0u;
     const int m_tiles = ceil_div(L.opixels(), TC_M);
     // split K towards the point where a CTA's slabs all fit in its pipeline at once
     // (its gather is then one round trip instead of a chain of them) - but no further than one wave of the
