@@ -471,6 +471,36 @@ def test_long_chunks_of_a_tensor_core_stack_go_dense_from_the_measured_activity(
     net.close()
 
 
+def test_dense_chunks_longer_than_one_batch():
+    """Dense chunks are batched over their frames, 32 at most per launch: a chunk of 40 frames of two streams goes in
+    two parts.  rrm_net_dense_seq leaves the state alone; a chunk that the density switch evaluates densely leaves
+    the state at its last frame."""
+    rrm = _rrm()
+    specs = wl.alexnet_convs("i8", hw=67, scale=8)
+    video = wl.moving_rect_video(frames=81, hw=67, dtype="i8", seed=47, n=2, side=(8, 16))
+    net = rrm.net_from_specs(specs, n=2)
+    frames = dev(np.ascontiguousarray(video))
+    out = net.new_output()
+    net.keyframe(frames[0], out)
+    outs = net.new_output(frames=40)
+    net.dense_seq(frames[1:41], outs, 40)
+    for i in (0, 19, 20, 39):
+        want = orc.dense_forward(specs, video[1 + i])[0][len(specs)]
+        np.testing.assert_array_equal(outs[i].cpu().numpy().astype(np.int64), want, err_msg=f"frame {1 + i}")
+    _compare(specs, net, video[0], 0)                       # the state is still the keyframe's
+    net.set_options(chunk_dense_activity=0.0)               # every measured activity sends the next chunk to the dense evaluation
+    net.step_seq(frames[1:41], outs, 40)                    # (nothing measured yet: the delta path)
+    assert net.stats(1)["variant"] != 3
+    _compare(specs, net, video[40], 40)
+    net.step_seq(frames[41:81], outs, 40)
+    assert net.stats(1)["variant"] == 3
+    for i in (0, 21, 39):
+        want = orc.dense_forward(specs, video[41 + i])[0][len(specs)]
+        np.testing.assert_array_equal(outs[i].cpu().numpy().astype(np.int64), want, err_msg=f"frame {41 + i}")
+    _compare(specs, net, video[80], 80)
+    net.close()
+
+
 def test_stack_chunks_through_the_pipelined_host_entry_point():
     """Host buffers in, host buffers out, calls queued without waiting: a stack's chunks through
     rrm_net_step_seq_host_async deliver every frame's output."""
