@@ -165,6 +165,8 @@ struct Layer {
     void* dP[CHUNK_RING] = {};
     size_t oact_off = 0;              // offset of the update bitmap inside an arena
     void* P2b = nullptr;              // projection buffer of a dense chunk batched over its frames
+    void* Aall = nullptr;             // pooled int8 layers of that form: f before the pool window of every frame's projection, as bytes
+                                      // ([0]: of the projection before the chunk, every pixel; [1 + g]: frame g's updated pixels)
     void* dPall = nullptr;            // per-frame products of the layer-by-layer chunk form
     uint32_t* oact = nullptr;         // bitmap of projection pixels to update (cleared every step, set by the
                                       // kernels that produce the layer's input and shortcut tensors)

@@ -49,6 +49,9 @@ struct EpiSeqParams {
     long long arena_stride;   // bytes between the frames' arenas
     long long p_stride;       // elements between the frames' products
     int opix;                 // projection pixels
+    const int8_t* A0;         // epilogue_seq_pool8_kernel: the pointwise part of f as bytes, before the chunk (every projection pixel) ...
+    const int8_t* A;          // ... and of frame 0 (updated pixels), the frames a_stride bytes apart
+    long long a_stride;
 };
 
 // Inclusive prefix sum over the lanes of a warp (lane g: sum of lanes 0 .. g), in a fixed order: the merge role and the
@@ -90,9 +93,18 @@ struct ProjSeqParams {
     const uint32_t* oact;     // frame 0's update bitmap
     int frames, c_out, opix;
     long long arena_stride, p_stride;
+    // ACT (int8 outputs behind a pool window): the pointwise part of f ([affine] -> requantisation -> activation) is
+    // applied here, once per projection pixel, and kept as bytes: A0 for the projection before the chunk (every pixel),
+    // A + g * a_stride for frame g (its updated pixels); the epilogue then only takes maxima of bytes
+    int8_t* A0;
+    int8_t* A;
+    long long a_stride;
+    int act_fn, shift;
+    const void* bn_scale;
+    const void* bn_shift;
 };
 
-template <int PT>
+template <int PT, bool ACT, bool BN>
 __global__ void __launch_bounds__(256) project_seq_kernel(ProjSeqParams p)
 {
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
@@ -104,7 +116,8 @@ __global__ void __launch_bounds__(256) project_seq_kernel(ProjSeqParams p)
     pdl_wait();
     bool mine = false;
     if (lane < p.frames) mine = (shift_bytes(p.oact, lane * p.arena_stride)[q >> 5] >> (q & 31)) & 1u;
-    if (!__any_sync(0xffffffffu, mine)) return;              // (the same in every warp of the CTA)
+    const bool any = __any_sync(0xffffffffu, mine);          // (the same in every warp of the CTA)
+    if (!any && !ACT) return;
     const pt* R = reinterpret_cast<const pt*>(p.R);
     pt* Q = reinterpret_cast<pt*>(p.Q);
     pt* dPg = reinterpret_cast<pt*>(p.dP) + (size_t)(lane < p.frames ? lane : 0) * p.p_stride;
@@ -126,9 +139,28 @@ __global__ void __launch_bounds__(256) project_seq_kernel(ProjSeqParams p)
         for (int k = 0; k < NQ; ++k) {
             const int c = (u0 + k) * 4;
             if (u0 + k >= quads) continue;                   // uniform inside the warp
+            if (ACT) {
+                // f before the pool window, as bytes: of the projection before the chunk (lane 0 writes it) ...
+                pt y[4];
+                const pt none[4] = {0, 0, 0, 0};
+                const pt (&b1)[1][4] = reinterpret_cast<const pt (&)[1][4]>(base[k]);
+                epi_f<PT, T_I8, 1, BN, pt>(b1, 1u, c, none, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
+                if (lane == 0)
+                    *reinterpret_cast<uint32_t*>(p.A0 + row + c) = ((uint32_t)(int)y[0] & 0xffu) | ((uint32_t)(int)y[1] & 0xffu) << 8 |
+                                                                   ((uint32_t)(int)y[2] & 0xffu) << 16 | ((uint32_t)(int)y[3] & 0xffu) << 24;
+                if (!any) continue;                          // a pixel no frame updates: nothing else to do
+            }
             scan4(d[k], lane);
             #pragma unroll
             for (int j = 0; j < 4; ++j) d[k][j] += base[k][j];
+            if (ACT && mine) {                               // ... and of this lane's frame
+                pt y[4];
+                const pt none[4] = {0, 0, 0, 0};
+                const pt (&d1)[1][4] = reinterpret_cast<const pt (&)[1][4]>(d[k]);
+                epi_f<PT, T_I8, 1, BN, pt>(d1, 1u, c, none, p.c_out, p.act_fn, p.shift, p.bn_scale, p.bn_shift, y);
+                *reinterpret_cast<uint32_t*>(p.A + (long long)lane * p.a_stride + row + c) =
+                    ((uint32_t)(int)y[0] & 0xffu) | ((uint32_t)(int)y[1] & 0xffu) << 8 | ((uint32_t)(int)y[2] & 0xffu) << 16 | ((uint32_t)(int)y[3] & 0xffu) << 24;
+            }
             if (mine || lane == 31) {
                 pt* dst = mine ? dPg : Q;
                 if (vec) {
@@ -142,6 +174,49 @@ __global__ void __launch_bounds__(256) project_seq_kernel(ProjSeqParams p)
                         dst[row + c + j] = d[k][j];
                         if (mine && lane == 31) Q[row + c + j] = d[k][j];
                     }
+                }
+            }
+        }
+    }
+}
+
+// Per frame in which the CTA's output pixel r changed (lane = frame, all frames at once): activity bit, counters, and in
+// every reading layer's update bitmap of that frame the projection pixels whose filter footprint covers the pixel, with
+// the exact multiply-accumulates they imply (non-zeros x covering (output, tap) pairs x output channels).
+template <bool READERS>
+__device__ __forceinline__ void seq_mark_frames(const EpiSeqParams& p, const int* s_cnt, int r, int ns, int ty, int tx, int lane, int warp)
+{
+    if (warp != 0) return;
+    {
+        const int cnt = lane < p.frames ? s_cnt[lane] : 0;
+        if (cnt > 0) {
+            const long long off = lane * p.arena_stride;
+            // (the CTAs of the grid's y dimension share the pixel, each with a slice of the channels: counts add up, marks
+            // are idempotent, and whoever sets the activity bit first counts the pixel)
+            const unsigned had = atomicOr(shift_bytes(p.act, off) + (r >> 5), 1u << (r & 31));
+            atomicAdd(shift_bytes(p.nnz, off), (unsigned long long)cnt);
+            if (!(had >> (r & 31) & 1u)) atomicAdd(shift_bytes(p.npix, off), 1ull);
+            if (READERS) {
+                #pragma unroll 1
+                for (int i = 0; i < p.readers.n; ++i) {
+                    const Reader& rd = p.readers.r[i];
+                    const int ay = ty + rd.pad, ax = tx + rd.pad;
+                    const int oy_lo = max(0, (ay - rd.kh + rd.stride) / rd.stride), oy_hi = min(rd.oh - 1, ay / rd.stride);
+                    const int ox_lo = max(0, (ax - rd.kw + rd.stride) / rd.stride), ox_hi = min(rd.ow - 1, ax / rd.stride);
+                    if (oy_hi < oy_lo || ox_hi < ox_lo) continue;
+                    uint32_t* bm = shift_bytes(rd.oact, off);
+                    for (int oy = oy_lo; oy <= oy_hi; ++oy) {
+                        int q0 = (ns * rd.oh + oy) * rd.ow + ox_lo, left = ox_hi - ox_lo + 1;
+                        while (left > 0) {                   // the run of columns, word by word
+                            const int bit = q0 & 31, take = min(left, 32 - bit);
+                            const unsigned run = (take == 32 ? 0xffffffffu : ((1u << take) - 1u)) << bit;
+                            atomicOr(&bm[q0 >> 5], run);
+                            q0 += take; left -= take;
+                        }
+                    }
+                    if (rd.macs)
+                        atomicAdd(shift_bytes(rd.macs, off),
+                                  (unsigned long long)cnt * (unsigned long long)((oy_hi - oy_lo + 1) * (ox_hi - ox_lo + 1)) * (unsigned long long)rd.c_out);
                 }
             }
         }
@@ -401,43 +476,105 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
         if (cnt) atomicAdd(&s_cnt[lane], cnt);
     }
     __syncthreads();
-    // ---- per frame in which the pixel changed (lane = frame once more, all frames at once): activity bit, counters,
-    // and in every reading layer's update bitmap of that frame the projection pixels whose filter footprint covers this
-    // pixel, with the exact multiply-accumulates they imply (non-zeros x covering (output, tap) pairs x output channels)
-    if (warp == 0) {
-        const int cnt = lane < p.frames ? s_cnt[lane] : 0;
-        if (cnt > 0) {
-            const long long off = lane * p.arena_stride;
-            // (the CTAs of the grid's y dimension share the pixel, each with a slice of the channels: counts add up, marks
-            // are idempotent, and whoever sets the activity bit first counts the pixel)
-            const unsigned had = atomicOr(shift_bytes(p.act, off) + (r >> 5), 1u << (r & 31));
-            atomicAdd(shift_bytes(p.nnz, off), (unsigned long long)cnt);
-            if (!(had >> (r & 31) & 1u)) atomicAdd(shift_bytes(p.npix, off), 1ull);
-            if (READERS) {
-                #pragma unroll 1
-                for (int i = 0; i < p.readers.n; ++i) {
-                    const Reader& rd = p.readers.r[i];
-                    const int ay = ty + rd.pad, ax = tx + rd.pad;
-                    const int oy_lo = max(0, (ay - rd.kh + rd.stride) / rd.stride), oy_hi = min(rd.oh - 1, ay / rd.stride);
-                    const int ox_lo = max(0, (ax - rd.kw + rd.stride) / rd.stride), ox_hi = min(rd.ow - 1, ax / rd.stride);
-                    if (oy_hi < oy_lo || ox_hi < ox_lo) continue;
-                    uint32_t* bm = shift_bytes(rd.oact, off);
-                    for (int oy = oy_lo; oy <= oy_hi; ++oy) {
-                        int q0 = (ns * rd.oh + oy) * rd.ow + ox_lo, left = ox_hi - ox_lo + 1;
-                        while (left > 0) {                   // the run of columns, word by word
-                            const int bit = q0 & 31, take = min(left, 32 - bit);
-                            const unsigned run = (take == 32 ? 0xffffffffu : ((1u << take) - 1u)) << bit;
-                            atomicOr(&bm[q0 >> 5], run);
-                            q0 += take; left -= take;
-                        }
-                    }
-                    if (rd.macs)
-                        atomicAdd(shift_bytes(rd.macs, off),
-                                  (unsigned long long)cnt * (unsigned long long)((oy_hi - oy_lo + 1) * (ox_hi - ox_lo + 1)) * (unsigned long long)rd.c_out);
-                }
+    seq_mark_frames<READERS>(p, s_cnt, r, ns, ty, tx, lane, warp);
+}
+
+// The epilogue of an int8 layer behind a pool window whose projection kernel has already applied the pointwise part of
+// f (EpiSeqParams.A0 / A: bytes): lane = frame; per window position the lane takes its frame's row (the latest frame up
+// to it that updated the position, else the row before the chunk), the window's max is a byte-wise max of 16 channels
+// at a time, the previous frame's output comes from the neighbouring lane.  c_out is a multiple of 16.
+template <int KW, bool READERS>
+__global__ void __launch_bounds__(256) epilogue_seq_pool8_kernel(EpiSeqParams p)
+{
+    __shared__ int s_cnt[SEQ_MAX_FRAMES];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_launch_dependents();
+    pdl_wait();
+    if (threadIdx.x < SEQ_MAX_FRAMES) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const int r = blockIdx.x;
+    const int tx = r % p.tw, ty = (r / p.tw) % p.th, ns = r / (p.tw * p.th);
+    const int y0 = ty * p.pool_s - p.pool_p, x0 = tx * p.pool_s - p.pool_p;
+    const int qbase = ns * p.oh * p.ow;
+    unsigned inside, ub = 0;
+    {
+        bool mine = false;
+        if (lane < KW * KW) {
+            const int y = y0 + lane / KW, x = x0 + lane % KW;
+            mine = y >= 0 && y < p.oh && x >= 0 && x < p.ow;
+        }
+        inside = __ballot_sync(0xffffffffu, mine);
+        if (lane < p.frames) {
+            const uint32_t* oa = shift_bytes(p.oact, lane * p.arena_stride);
+            #pragma unroll
+            for (int wi = 0; wi < KW * KW; ++wi) {
+                if (!(inside >> wi & 1u)) continue;
+                const int q = qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW;
+                if ((oa[q >> 5] >> (q & 31)) & 1u) ub |= 1u << wi;
             }
         }
     }
+    const unsigned on_frames = __ballot_sync(0xffffffffu, ub != 0);
+    const bool full = p.Xfull != nullptr;
+    if (on_frames || full) {
+        const bool live = lane < p.frames, on = (on_frames >> lane) & 1u, last = lane == p.frames - 1;
+        const long long roff = (long long)(live ? lane : 0) * p.row_stride;
+        // per window position: the row this lane's frame sees
+        const int8_t* rowp[KW * KW];
+        #pragma unroll
+        for (int wi = 0; wi < KW * KW; ++wi) {
+            const unsigned uf = __ballot_sync(0xffffffffu, (ub >> wi) & 1u);
+            const unsigned upto = uf & (0xffffffffu >> (31 - lane));
+            const size_t pos = (size_t)(qbase + (y0 + wi / KW) * p.ow + x0 + wi % KW) * p.c_out;
+            rowp[wi] = (upto ? p.A + (long long)(31 - __clz(upto)) * p.a_stride : p.A0) + pos;
+        }
+        int cnt = 0;
+        const int units = p.cs >> 4;                         // (cs is a multiple of 32)
+        for (int u = blockIdx.y * 8 + warp; u < units; u += 8 * gridDim.y) {
+            const int c = u * 16;
+            const size_t o = (size_t)r * p.cs + c;
+            const uint4 before = *reinterpret_cast<const uint4*>(reinterpret_cast<const int8_t*>(p.X) + o);
+            uint4 best = make_uint4(0, 0, 0, 0);
+            if (c < p.c_out) {                               // (channels past c_out are padding: zero)
+                uint4 v[KW * KW];
+                #pragma unroll
+                for (int wi = 0; wi < KW * KW; ++wi)
+                    if (inside >> wi & 1u) v[wi] = *reinterpret_cast<const uint4*>(rowp[wi] + c);
+                bool have = false;
+                #pragma unroll
+                for (int wi = 0; wi < KW * KW; ++wi) {
+                    if (!(inside >> wi & 1u)) continue;
+                    if (!have) best = v[wi];
+                    else {
+                        best.x = __vmaxs4(best.x, v[wi].x); best.y = __vmaxs4(best.y, v[wi].y);
+                        best.z = __vmaxs4(best.z, v[wi].z); best.w = __vmaxs4(best.w, v[wi].w);
+                    }
+                    have = true;
+                }
+            }
+            uint4 old;
+            old.x = __shfl_up_sync(0xffffffffu, best.x, 1); old.y = __shfl_up_sync(0xffffffffu, best.y, 1);
+            old.z = __shfl_up_sync(0xffffffffu, best.z, 1); old.w = __shfl_up_sync(0xffffffffu, best.w, 1);
+            if (lane == 0) old = before;
+            if (live) {
+                if (on) {
+                    uint4 dw;
+                    dw.x = __vsub4(best.x, old.x); dw.y = __vsub4(best.y, old.y); dw.z = __vsub4(best.z, old.z); dw.w = __vsub4(best.w, old.w);
+                    // a difference outside a byte shows as a wrapped subtraction that differs from the saturating one
+                    if (p.errw && (dw.x != __vsubss4(best.x, old.x) || dw.y != __vsubss4(best.y, old.y) ||
+                                   dw.z != __vsubss4(best.z, old.z) || dw.w != __vsubss4(best.w, old.w))) atomicOr(p.errw, ERRW_BOUNDS);
+                    cnt += __popc(nonzero_bytes(dw.x)) + __popc(nonzero_bytes(dw.y)) + __popc(nonzero_bytes(dw.z)) + __popc(nonzero_bytes(dw.w));
+                    *reinterpret_cast<uint4*>(shift_bytes(reinterpret_cast<int8_t*>(p.D), roff) + o) = dw;
+                    if (p.Xn) *reinterpret_cast<uint4*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xn), roff) + o) = best;
+                }
+                if (full) *reinterpret_cast<uint4*>(shift_bytes(reinterpret_cast<int8_t*>(p.Xfull), roff) + o) = best;
+            }
+            if (last && on_frames) *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.X) + o) = best;
+        }
+        if (cnt) atomicAdd(&s_cnt[lane], cnt);
+    }
+    __syncthreads();
+    seq_mark_frames<READERS>(p, s_cnt, r, ns, ty, tx, lane, warp);
 }
 
 // ================================================================================================
@@ -500,17 +637,33 @@ int launch_epilogue_seq(rrm_net* net, int l, int frames, long long arena_stride,
     e.frames = frames; e.row_stride = (long long)out.bytes(); e.arena_stride = arena_stride;
     e.p_stride = (long long)L.opixels() * d.c_out;
     e.opix = L.opixels();
+    // int8 outputs behind a pool window: the projection kernel applies the pointwise part of f and the epilogue works on bytes
+    const bool bytes = L.Aall != nullptr;
     if (d.pool_k > 1) {                                      // (without a pool window the epilogue sums the frames' products itself)
         ProjSeqParams q{};
         q.R = L.Palt; q.Q = L.P; q.dP = L.dPall; q.oact = L.oact;
         q.frames = frames; q.c_out = d.c_out; q.opix = L.opixels();
         q.arena_stride = arena_stride; q.p_stride = e.p_stride;
-        if (d.dtype == RRM_F32) launch_seq(project_seq_kernel<T_F32>, dim3(L.opixels()), dim3(256), 0, st, q);
-        else launch_seq(project_seq_kernel<T_I32>, dim3(L.opixels()), dim3(256), 0, st, q);
+        if (bytes) {
+            q.a_stride = (long long)L.opixels() * d.c_out;
+            q.A0 = reinterpret_cast<int8_t*>(L.Aall); q.A = q.A0 + q.a_stride;
+            q.act_fn = d.act; q.shift = d.shift; q.bn_scale = L.bn_scale; q.bn_shift = L.bn_shift;
+            e.A0 = q.A0; e.A = q.A; e.a_stride = q.a_stride;
+            if (L.bn_scale) launch_seq(project_seq_kernel<T_I32, true, true>, dim3(L.opixels()), dim3(256), 0, st, q);
+            else launch_seq(project_seq_kernel<T_I32, true, false>, dim3(L.opixels()), dim3(256), 0, st, q);
+        } else if (d.dtype == RRM_F32) launch_seq(project_seq_kernel<T_F32, false, false>, dim3(L.opixels()), dim3(256), 0, st, q);
+        else launch_seq(project_seq_kernel<T_I32, false, false>, dim3(L.opixels()), dim3(256), 0, st, q);
     }
     const int blocks = out.pixels();                         // a CTA per output pixel
-    int s;
-    if (d.dtype == RRM_F32) s = launch_epi_seq_t<T_F32, T_F32>(e, blocks, st);
+    int s = RRM_OK;
+    if (bytes) {
+        const int slices = ceil_div(ceil_div(out.cs >> 4, 8), 2) < 1 ? 1 : ceil_div(ceil_div(out.cs >> 4, 8), 2);
+        const bool rd = e.readers.n > 0;
+        if (d.pool_k == 2) { if (rd) launch_seq(epilogue_seq_pool8_kernel<2, true>, dim3(blocks, slices), dim3(256), 0, st, e); else launch_seq(epilogue_seq_pool8_kernel<2, false>, dim3(blocks, slices), dim3(256), 0, st, e); }
+        else if (d.pool_k == 3) { if (rd) launch_seq(epilogue_seq_pool8_kernel<3, true>, dim3(blocks, slices), dim3(256), 0, st, e); else launch_seq(epilogue_seq_pool8_kernel<3, false>, dim3(blocks, slices), dim3(256), 0, st, e); }
+        else s = RRM_ERR_UNSUPPORTED;
+    }
+    else if (d.dtype == RRM_F32) s = launch_epi_seq_t<T_F32, T_F32>(e, blocks, st);
     else if (out.dtype == T_I8) s = launch_epi_seq_t<T_I32, T_I8>(e, blocks, st);
     else if (out.dtype == T_BIN) s = launch_epi_seq_t<T_I32, T_BIN>(e, blocks, st);
     else s = launch_epi_seq_t<T_I32, T_I32>(e, blocks, st);
@@ -552,6 +705,10 @@ int ensure_frame_batch(rrm_net* net)
         const size_t bytes = (size_t)L.opixels() * L.d.c_out * 4;
         RRM_TRY(alloc(&L.Palt, bytes));
         RRM_TRY(alloc(&L.dPall, bytes * G));
+        // int8 outputs behind a 2x2 / 3x3 pool window, no shortcut, channels in whole groups of 16: f before the window as bytes
+        const Tensor& out = net->tensors[(&L - &net->layers[0]) + 1];
+        if (out.dtype == T_I8 && (L.d.pool_k == 2 || L.d.pool_k == 3) && L.d.res < 0 && L.d.c_out % 16 == 0 && L.d.dtype != RRM_F32)
+            RRM_TRY(alloc(&L.Aall, (size_t)L.opixels() * L.d.c_out * (G + 1)));
     }
     net->seq_ready = true;
     return RRM_OK;
