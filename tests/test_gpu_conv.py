@@ -416,6 +416,60 @@ def test_stack_chunks_of_frames_equal_frame_by_frame(name, by_layer, monkeypatch
     net.close()
 
 
+@pytest.mark.parametrize("name", ["cfg1", "cfg3_f32", "cfg3_i8", "cfg5", "cfg4"])
+def test_full_size_stacks_in_chunks_of_32_frames(name):
+    """The full-size configurations in the launch configuration the bench times for chunks: 32 frames per
+    rrm_net_step_seq call.  First chunk and second chunk on the delta path (thresholds out of reach), the third as the
+    library chooses; sampled frames' outputs against the dense definition, every layer's state after each chunk, and
+    the last frame's counters of the second chunk against Algorithm 1 brought to the frame before by a dense pass."""
+    rrm = _rrm()
+    n = 1
+    if name == "cfg1":
+        specs, dt, hw = wl.single_conv_f32(), "f32", 56
+    elif name == "cfg3_f32":
+        specs, dt, hw = wl.alexnet_convs("f32"), "f32", 227
+    elif name == "cfg3_i8":
+        specs, dt, hw = wl.alexnet_convs("i8"), "i8", 227
+    elif name == "cfg5":
+        specs, dt, hw = wl.xnor_alexnet_convs(), "i8", 227
+    else:
+        specs, dt, hw, n = wl.resnet18_convs(), "i8", 224, 4
+    if name == "cfg1":
+        video = wl.block_redraw_sequence(frames=96, seed=61)
+    else:
+        video = wl.moving_rect_video(frames=96, hw=hw, dtype=dt, seed=61, n=n, bg_redraw=0.02 if name == "cfg4" else 0.0)
+    net = rrm.net_from_specs(specs, n=n)
+    defaults = net.options()
+    net.set_options(chunk_dense_activity=2.0, stack_dense_activity=2.0)
+    frames = dev(np.ascontiguousarray(video))
+    outs = net.new_output(frames=32)
+    for k in range(3):
+        if k == 2:
+            net.set_options(chunk_dense_activity=defaults["chunk_dense_activity"], stack_dense_activity=defaults["stack_dense_activity"])
+        net.step_seq(frames[32 * k:32 * k + 32], outs, 32)
+        sts = [net.stats(l) for l in range(len(specs))]
+        assert all(st["error_word"] == 0 for st in sts)
+        for i in ((0, 13, 31) if k < 2 else (0, 31)):
+            want = orc.dense_forward(specs, video[32 * k + i])[0][len(specs)]
+            got = outs[i].cpu().numpy()
+            if dt == "f32":
+                assert float(np.abs(got - want).max()) <= F32_TOL * max(1e-30, float(np.abs(want).max())), (k, i)
+            elif _out_kind(specs[-1]) == "bin":
+                np.testing.assert_array_equal(unpack_bits_nhwc(got.view(np.uint32), specs[-1].c_out), want, err_msg=f"chunk {k} frame {i}")
+            else:
+                np.testing.assert_array_equal(got.astype(np.int64), want, err_msg=f"chunk {k} frame {i}")
+        _compare(specs, net, video[32 * k + 31], 32 * k + 31)
+        if k == 1:
+            one = orc.Recurrence(specs, n=n)
+            one.reset_to(video[62])
+            one.step(video[63])
+            for l, st in enumerate(sts):
+                assert st["variant"] != 3 and st["nnz_elems"] != -1, (l, st)
+                if dt != "f32" or l == 0:
+                    assert st["nnz_elems"] == one.nnz[l] and st["active_macs"] == one.macs[l], (l, st, one.nnz[l], one.macs[l])
+    net.close()
+
+
 def test_large_stack_chunks_go_dense_while_nearly_every_pixel_changes():
     """The density switch of a large stack, chunk by chunk: the chunk after a measured high-activity delta chunk is
     evaluated densely (a sequence of precise inferences that replace the state); outputs and state stay exact."""
