@@ -52,6 +52,7 @@ struct ConvParams {
     long long row_stride;     // bytes between the frames' sets of delta rows (and of new rows)
     long long arena_stride;   // bytes between the frames' arenas (bitmaps, counters)
     long long p_stride;       // elements between the frames' products
+    unsigned magic_u, magic_kw;     // ceil(2^32 / u_in), ceil(2^32 / kw): quotients by a multiply-high (0: the divisor is 1); set by launch_gemm
 };
 
 // The number of set bits of bm[0 .. words) -> *out, by one CTA (the activity of a layer that is evaluated densely).
@@ -115,6 +116,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     __shared__ int s_q[TM];
     __shared__ int s_tmp[256 + 34];
     __shared__ unsigned s_tapmask[4];
+    __shared__ uint32_t s_live[8];                           // bit r: stage s_first + r has a usable tap (the first 256 stages of the CTA's range)
     __shared__ unsigned long long s_rmask[TM][2];
     __shared__ int s_pix0[TM];
 
@@ -145,6 +147,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < 4) s_tapmask[tid] = 0;
+    if (tid < 8) s_live[tid] = 0;
     __syncthreads();
 
     // ---- per row: the input pixel under tap (0,0) and the usable taps
@@ -181,15 +184,30 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     // this CTA's share of the K stages
     const int all_stages = p.kup / TK, per_split = (all_stages + p.ksplit - 1) / p.ksplit;
     const int s_first = zshare * per_split, n_stages = min(all_stages, s_first + per_split);
+    auto div_u = [&](int x) -> int { return p.magic_u ? (int)__umulhi((unsigned)x, p.magic_u) : x; };
+    auto div_kw = [&](int x) -> int { return p.magic_kw ? (int)__umulhi((unsigned)x, p.magic_kw) : x; };
     auto stage_live = [&](int ks) -> bool {                 // any usable tap among the stage's K units?
-        const int t_lo = (ks * TK) / p.u_in, t_hi = min(taps - 1, (ks * TK + TK - 1) / p.u_in);
+        const int t_lo = div_u(ks * TK), t_hi = min(taps - 1, div_u(ks * TK + TK - 1));
         for (int t = t_lo; t <= t_hi; ++t)
             if (t < 64 ? (tm0 >> t) & 1ull : (tm1 >> (t - 64)) & 1ull) return true;
         return false;
     };
-    auto next_live = [&](int ks) -> int {
+    // which stages are live is worked out once, by all threads, and kept as a bitmap: the loop then finds its next
+    // stage with a shift (ranges beyond 256 stages test the rest stage by stage)
+    const int n_range = max(0, n_stages - s_first);
+    for (int r = tid; r < min(n_range, 256); r += CONV_THREADS)
+        if (stage_live(s_first + r)) atomicOr(&s_live[r >> 5], 1u << (r & 31));
+    __syncthreads();
+    auto next_live = [&](int ks) -> int {                   // first live stage >= ks, or n_stages
+        int r = ks - s_first;
+        while (r < min(n_range, 256)) {
+            const uint32_t wbits = s_live[r >> 5] >> (r & 31);
+            if (wbits) return s_first + r + __ffs(wbits) - 1;
+            r = (r | 31) + 1;
+        }
+        ks = s_first + max(r, ks - s_first);
         while (ks < n_stages && !stage_live(ks)) ++ks;
-        return ks;
+        return min(ks, n_stages);
     };
 
     const uint32_t* Du = reinterpret_cast<const uint32_t*>(p.D);
@@ -218,8 +236,8 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             #pragma unroll
             for (int i = 0; i < (VEC ? 1 : 4); ++i) {
                 const int kk = VEC ? piece * 4 : piece + 8 * i, k = ks * TK + kk;
-                const int tap = k / p.u_in, u = k - tap * p.u_in;
-                const int ky = tap / p.kw, kx = tap - ky * p.kw;
+                const int tap = div_u(k), u = k - tap * p.u_in;
+                const int ky = div_kw(tap), kx = tap - ky * p.kw;
                 const bool use = tap < taps && ((tap < 64 ? rm0 >> tap : rm1 >> (tap - 64)) & 1ull);
                 const size_t off = use ? (size_t)(pix0 + ky * p.w + kx) * p.u_in + u : 0;
                 const int sidx = row * GEMM_LDA + kk;
@@ -395,9 +413,13 @@ static size_t gemm_smem_bytes(int dt)
 }
 
 template <int DT, bool DENSE>
-static void launch_gemm(const ConvParams& p, dim3 grid, cudaStream_t st)
+static void launch_gemm(const ConvParams& p_in, dim3 grid, cudaStream_t st)
 {
+    ConvParams p = p_in;
     const int cluster_z = (DT == T_F32 && p.ksplit > 1) ? p.ksplit : 1;       // fp32 shares of a tile: one cluster
+    // (exact while the dividend stays below 2^32 / divisor: K units and taps are far below that)
+    p.magic_u = p.u_in > 1 ? (unsigned)(((1ull << 32) + p.u_in - 1) / p.u_in) : 0u;
+    p.magic_kw = p.kw > 1 ? (unsigned)(((1ull << 32) + p.kw - 1) / p.kw) : 0u;
     if (p.u_in % 4 == 0) launch_seq_cluster(conv_gemm_kernel<DT, DENSE, true>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, cluster_z, p);
     else launch_seq_cluster(conv_gemm_kernel<DT, DENSE, false>, dim3(grid), dim3(CONV_THREADS), gemm_smem_bytes(DT), st, cluster_z, p);
 }
