@@ -119,26 +119,50 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     __shared__ uint32_t s_live[8];                           // bit r: stage s_first + r has a usable tap (the first 256 stages of the CTA's range)
     __shared__ unsigned long long s_rmask[TM][2];
     __shared__ int s_pix0[TM];
+    __shared__ int s_fcnt[32];                               // several frames per launch: every frame's number of rows
 
     const int tid = threadIdx.x, lane = tid & 31;
-    const int tile = blockIdx.x, n0 = blockIdx.y * TN;
+    int tile = blockIdx.x;
+    const int n0 = blockIdx.y * TN;
     const bool batched = !DENSE && p.frames > 1;             // gridDim.z counts frames, not shares of K
     const int zshare = batched ? 0 : blockIdx.z;
-    if (batched && blockIdx.z > 0) {
-        const long long g = blockIdx.z;
-        p.D = reinterpret_cast<const char*>(p.D) + g * p.row_stride;
-        p.X = reinterpret_cast<const char*>(p.X) + g * p.row_stride;
-        p.in_act = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.in_act) + g * p.arena_stride);
-        p.oact = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.oact) + g * p.arena_stride);
-        p.ocount = reinterpret_cast<int*>(reinterpret_cast<char*>(p.ocount) + g * p.arena_stride);
-        p.P = reinterpret_cast<char*>(p.P) + g * p.p_stride * 4;
-    }
     pdl_launch_dependents();
     if (!DENSE) {
         pdl_wait();                                          // the update bitmap is the predecessors' work
+        if (batched) {
+            // Which (frame, tile) this CTA takes: the tiles that have rows, numbered frame by frame, go to the CTAs in
+            // launch order (gridDim.x * gridDim.z of them per N tile), so that the CTAs with work come first and spread
+            // evenly over the SMs instead of landing wherever an active frame's block index happens to fall.  Every
+            // CTA counts all frames' update bitmaps for that (a few words per frame and lane).
+            const int words = (p.opixels + 31) >> 5, nfr = (int)gridDim.z;
+            for (int g = tid >> 5; g < nfr; g += CONV_THREADS / 32) {
+                const uint32_t* bm = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.oact) + (long long)g * p.arena_stride);
+                int c = 0;
+                for (int i = lane; i < words; i += 32) c += __popc(__ldg(bm + i));
+                c = __reduce_add_sync(0xffffffffu, c);
+                if (lane == 0) s_fcnt[g] = c;
+            }
+            __syncthreads();
+            int id = (int)(blockIdx.z * gridDim.x + blockIdx.x), frame = -1;
+            if (id == 0 && blockIdx.y == 0 && tid < nfr)     // every frame's count, also of frames without a tile
+                *reinterpret_cast<int*>(reinterpret_cast<char*>(p.ocount) + (long long)tid * p.arena_stride) = s_fcnt[tid];
+            for (int g = 0; g < nfr; ++g) {
+                const int t = (s_fcnt[g] + TM - 1) / TM;
+                if (id < t) { frame = g; break; }
+                id -= t;
+            }
+            if (frame < 0) return;
+            tile = id;
+            const long long g = frame;
+            p.D = reinterpret_cast<const char*>(p.D) + g * p.row_stride;
+            p.X = reinterpret_cast<const char*>(p.X) + g * p.row_stride;
+            p.in_act = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.in_act) + g * p.arena_stride);
+            p.oact = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.oact) + g * p.arena_stride);
+            p.P = reinterpret_cast<char*>(p.P) + g * p.p_stride * 4;
+        }
         // this CTA's rows: the tile-th group of TM set bits of the layer's update bitmap
         const int count = select_rows<TM>(p.oact, (p.opixels + 31) >> 5, tile, s_q, s_tmp);
-        if (tile == 0 && blockIdx.y == 0 && zshare == 0 && tid == 0) *p.ocount = count;
+        if (!batched && tile == 0 && blockIdx.y == 0 && zshare == 0 && tid == 0) *p.ocount = count;
         if (tile * TM >= count) return;
     }
     if (tid == 0) {
@@ -289,7 +313,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         else asm volatile("cp.async.commit_group;" ::: "memory");
         const uint32_t* Bs = g_smem + slot * STAGE_WORDS;
         const uint32_t* As = Bs + GEMM_B_WORDS;
-        #pragma unroll 2
+        #pragma unroll 4
         for (int k4 = 0; k4 < TK; k4 += 4) {
             uint4 ar[4], an[4];                               // 4 K units of each of the thread's 4 rows
             #pragma unroll
