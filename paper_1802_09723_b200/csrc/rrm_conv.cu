@@ -29,7 +29,9 @@ namespace rrm {
 constexpr int TM = 64;            // projection pixels per CTA
 constexpr int TN = GEMM_TN;       // output channels per CTA
 constexpr int TK = GEMM_TK;       // K units per stage
-constexpr int CONV_THREADS = 256;
+constexpr int CONV_THREADS = 128;
+constexpr int RM = TM * 16 / CONV_THREADS;   // rows of the tile per thread (x 4 output channels): 16 threads span the TN = 64 channels
+static_assert(TN == 64 && CONV_THREADS >= TM && TM % (CONV_THREADS / 8) == 0, "thread layout of conv_gemm_kernel");
 
 struct ConvParams {
     const void* D;            // delta rows (delta mode) / unused (dense)
@@ -89,7 +91,7 @@ __device__ __forceinline__ bool bit_test(const uint32_t* bm, int i) { return (bm
 //     are usable is decided once per row (a 128-bit mask in shared memory), so the gather addresses
 //     depend on no further load;
 //   - stages none of whose taps is usable under any row of the tile are skipped.
-// Copies of later stages are in flight while the current one is multiplied (4x4 outputs per thread).
+// Copies of later stages are in flight while the current one is multiplied (RM x 4 outputs per thread).
 // ------------------------------------------------------------------------------------------------
 constexpr int GEMM_STAGES = 3;
 constexpr int GEMM_LDA = TK + 4;                   // words per activation row in shared memory (16-byte aligned, bank-staggered)
@@ -250,11 +252,11 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(sB), "l"(Wu + (size_t)ks * GEMM_B_WORDS), "r"((uint32_t)(GEMM_B_WORDS * 4)), "r"(bar) : "memory");
         }
-        // thread -> (row = tid / 8 [+ 32], piece = tid % 8): 8 lanes cover the 32 K units of one row
+        // thread -> (row = tid / 8 [+ a pass of CONV_THREADS / 8 rows], piece = tid % 8): 8 lanes cover the 32 K units of one row
         const int piece = tid & 7;
         #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int row = (tid >> 3) + half * 32;
+        for (int half = 0; half < TM / (CONV_THREADS / 8); ++half) {
+            const int row = (tid >> 3) + half * (CONV_THREADS / 8);
             const unsigned long long rm0 = s_rmask[row][0], rm1 = s_rmask[row][1];
             const int pix0 = s_pix0[row];
             #pragma unroll
@@ -286,13 +288,15 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
-    const int tm = (tid >> 4) * 4, tn = (tid & 15) * 4;    // 4x4 outputs per thread
-    acc_t acc[4][4];
+    const int tm = (tid >> 4) * RM, tn = (tid & 15) * 4;   // RM x 4 outputs per thread
+    acc_t acc[RM][4];
+    int rowpop[RM];                                        // binary: changed (dense: valid) bits of the thread's rows
     #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < RM; ++i) {
+        rowpop[i] = 0;
         #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
-    int rowpop[4] = {0, 0, 0, 0};                          // binary: changed (dense: valid) bits of the thread's 4 rows
+    }
     bool ok = true;
 
     // prologue: the first GEMM_STAGES - 1 live stages
@@ -315,9 +319,9 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         const uint32_t* As = Bs + GEMM_B_WORDS;
         #pragma unroll 4
         for (int k4 = 0; k4 < TK; k4 += 4) {
-            uint4 ar[4], an[4];                               // 4 K units of each of the thread's 4 rows
+            uint4 ar[RM], an[RM];                             // 4 K units of each of the thread's rows
             #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < RM; ++i) {
                 ar[i] = *reinterpret_cast<const uint4*>(&As[(tm + i) * GEMM_LDA + k4]);
                 if (DT == T_BIN) an[i] = *reinterpret_cast<const uint4*>(&As[GEMM_A_WORDS + (tm + i) * GEMM_LDA + k4]);
             }
@@ -326,7 +330,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
                 const uint4 bw = *reinterpret_cast<const uint4*>(&Bs[(k4 + kq) * TN + tn]);
                 const uint32_t b[4] = {bw.x, bw.y, bw.z, bw.w};
                 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < RM; ++i) {
                     const uint32_t a = kq == 0 ? ar[i].x : kq == 1 ? ar[i].y : kq == 2 ? ar[i].z : ar[i].w;
                     uint32_t nw = 0;
                     if (DT == T_BIN) {
@@ -365,7 +369,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
         float* tilebuf = reinterpret_cast<float*>(g_smem);   // [TM][TN]; the ring is free: every issued stage was consumed
         __syncthreads();
         #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < RM; ++i)
             *reinterpret_cast<float4*>(&tilebuf[(tm + i) * TN + tn]) = make_float4((float)acc[i][0], (float)acc[i][1], (float)acc[i][2], (float)acc[i][3]);
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -404,7 +408,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     // (split K) add their partial sums with atomics (dense: onto a zeroed projection, split 0 adds the bias)
     const bool shared_tile = p.ksplit > 1;
     #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < RM; ++i) {
         const int q = s_q[tm + i];
         if (q < 0) continue;
         #pragma unroll
