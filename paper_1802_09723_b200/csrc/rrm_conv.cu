@@ -107,6 +107,18 @@ __device__ __forceinline__ void g_cp_async16(uint32_t dst, const void* src, uint
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 
+// Two fp32 multiply-adds per instruction (each rounded as fmaf rounds): acc = a * b + acc on both halves of 64-bit pairs.
+__device__ __forceinline__ unsigned long long g_pack2(uint32_t lo, uint32_t hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void g_fma2(unsigned long long& acc, unsigned long long a, unsigned long long b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+
 template <int DT, bool DENSE, bool VEC>
 __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
 {
@@ -290,10 +302,12 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
 
     const int tm = (tid >> 4) * RM, tn = (tid & 15) * 4;   // RM x 4 outputs per thread
     acc_t acc[RM][4];
+    unsigned long long acc2[RM][2];                        // fp32: the same accumulators as pairs (channels 0-1, 2-3)
     int rowpop[RM];                                        // binary: changed (dense: valid) bits of the thread's rows
     #pragma unroll
     for (int i = 0; i < RM; ++i) {
         rowpop[i] = 0;
+        acc2[i][0] = acc2[i][1] = 0ull;
         #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
     }
@@ -337,17 +351,32 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
                         nw = kq == 0 ? an[i].x : kq == 1 ? an[i].y : kq == 2 ? an[i].z : an[i].w;
                         rowpop[i] += __popc(a);
                     }
-                    #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (DT == T_F32) acc[i][j] = fmaf(__uint_as_float(a), __uint_as_float(b[j]), acc[i][j]);
-                        else if (DT == T_I8) acc[i][j] = __dp4a((int)a, (int)b[j], (int)acc[i][j]);
-                        else acc[i][j] += __popc(a & (nw ^ b[j]));
+                    if (DT == T_F32) {
+                        const unsigned long long aa = g_pack2(a, a);
+                        g_fma2(acc2[i][0], aa, g_pack2(b[0], b[1]));
+                        g_fma2(acc2[i][1], aa, g_pack2(b[2], b[3]));
+                    } else {
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (DT == T_I8) acc[i][j] = __dp4a((int)a, (int)b[j], (int)acc[i][j]);
+                            else acc[i][j] += __popc(a & (nw ^ b[j]));
+                        }
                     }
                 }
             }
         }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (DT == T_F32) {
+        #pragma unroll
+        for (int i = 0; i < RM; ++i)
+            #pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t lo, hi;
+                asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(acc2[i][h]));
+                acc[i][2 * h] = (acc_t)__uint_as_float(lo); acc[i][2 * h + 1] = (acc_t)__uint_as_float(hi);
+            }
+    }
     if (!ok) {
         // giving up: the filter slices still on their way (stages issued, not consumed) must land before the CTA's
         // shared memory goes away; thread 0 issued them and waits for them, the others wait for thread 0
