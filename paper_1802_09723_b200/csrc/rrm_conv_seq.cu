@@ -403,7 +403,10 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                     if (c[q] < 0) continue;
                     const size_t o = (size_t)r * p.cs + c[q];
                     if (OT == T_I8) before_w[q] = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const int8_t*>(p.X) + o);
-                    else {
+                    else if ((p.cs & 3) == 0) {              // (rows of whole 16-byte groups: one load)
+                        const pt4 t = *reinterpret_cast<const pt4*>(reinterpret_cast<const pt*>(p.X) + o);
+                        before[q][0] = t.x; before[q][1] = t.y; before[q][2] = t.z; before[q][3] = t.w;
+                    } else {
                         #pragma unroll
                         for (int j = 0; j < 4; ++j) if (c[q] + j < p.cs) before[q][j] = reinterpret_cast<const pt*>(p.X)[o + j];
                     }
@@ -454,20 +457,36 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
                             old[j] = __shfl_up_sync(0xffffffffu, best[q][j], 1);
                             if (lane == 0) old[j] = before[q][j];
                         }
+                        const bool v4 = (p.cs & 3) == 0;     // rows of whole 16-byte groups: one store per row and group
+                        pt4 bv; bv.x = best[q][0]; bv.y = best[q][1]; bv.z = best[q][2]; bv.w = best[q][3];
                         if (live) {
                             pt* Dg = shift_bytes(reinterpret_cast<pt*>(p.D), roff);
                             pt* Fg = full ? shift_bytes(reinterpret_cast<pt*>(p.Xfull), roff) : nullptr;
                             pt* Ng = p.Xn ? shift_bytes(reinterpret_cast<pt*>(p.Xn), roff) : nullptr;
-                            #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                if (c[q] + j >= p.cs) break;
-                                if (on) { Dg[o + j] = best[q][j] - old[j]; cnt += best[q][j] != old[j]; if (Ng) Ng[o + j] = best[q][j]; }
-                                if (full) Fg[o + j] = best[q][j];
+                            if (v4) {
+                                if (on) {
+                                    pt4 dv; dv.x = best[q][0] - old[0]; dv.y = best[q][1] - old[1]; dv.z = best[q][2] - old[2]; dv.w = best[q][3] - old[3];
+                                    *reinterpret_cast<pt4*>(Dg + o) = dv;
+                                    #pragma unroll
+                                    for (int j = 0; j < 4; ++j) cnt += best[q][j] != old[j];
+                                    if (Ng) *reinterpret_cast<pt4*>(Ng + o) = bv;
+                                }
+                                if (full) *reinterpret_cast<pt4*>(Fg + o) = bv;
+                            } else {
+                                #pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    if (c[q] + j >= p.cs) break;
+                                    if (on) { Dg[o + j] = best[q][j] - old[j]; cnt += best[q][j] != old[j]; if (Ng) Ng[o + j] = best[q][j]; }
+                                    if (full) Fg[o + j] = best[q][j];
+                                }
                             }
                         }
                         if (last && on_frames) {
-                            #pragma unroll
-                            for (int j = 0; j < 4; ++j) if (c[q] + j < p.cs) reinterpret_cast<pt*>(p.X)[o + j] = best[q][j];
+                            if (v4) *reinterpret_cast<pt4*>(reinterpret_cast<pt*>(p.X) + o) = bv;
+                            else {
+                                #pragma unroll
+                                for (int j = 0; j < 4; ++j) if (c[q] + j < p.cs) reinterpret_cast<pt*>(p.X)[o + j] = best[q][j];
+                            }
                         }
                     }
                 }
