@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
     using pt = typename std::conditional<PT == T_F32, float, int>::type;
     using pt4 = typename std::conditional<PT == T_F32, float4, int4>::type;
     __shared__ int s_cnt[SEQ_MAX_FRAMES];                    // changed elements of the CTA's pixel, per frame
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (int)(blockDim.x >> 5);
     const bool vec = (p.c_out & 3) == 0;
     pdl_launch_dependents();
     pdl_wait();
@@ -357,7 +357,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
             }
         };
         if (OT == T_BIN) {
-            for (int u = blockIdx.y * 8 + warp; u < p.cs; u += 8 * gridDim.y) {   // one 32-channel word of the output per turn
+            for (int u = blockIdx.y * nwarps + warp; u < p.cs; u += nwarps * gridDim.y) {   // one 32-channel word of the output per turn
                 const size_t o = (size_t)r * p.cs + u;
                 const uint32_t before = reinterpret_cast<const uint32_t*>(p.X)[o];
                 uint32_t word = 0;
@@ -389,7 +389,7 @@ __global__ void __launch_bounds__(256) epilogue_seq_kernel(EpiSeqParams p)
             }
         } else {
             const int units = (p.cs + 3) >> 2;
-            for (int u0 = (blockIdx.y * 8 + warp) * NQ; u0 < units; u0 += 8 * NQ * gridDim.y) {   // NQ groups of four output channels per turn
+            for (int u0 = (blockIdx.y * nwarps + warp) * NQ; u0 < units; u0 += nwarps * NQ * gridDim.y) {   // NQ groups of four output channels per turn
                 int c[NQ];
                 #pragma unroll
                 for (int q = 0; q < NQ; ++q) c[q] = (u0 + q < units) ? (u0 + q) * 4 : -1;
@@ -607,8 +607,11 @@ static void launch_epi_seq_kw(const EpiSeqParams& e, int blocks, cudaStream_t st
     const int turns = OT == T_BIN ? ceil_div(e.cs, 8) : ceil_div(ceil_div(e.cs, 4), 8 * NQ);    // per warp of a lone CTA
     int slices = ceil_div(turns, 2);
     slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
-    if (e.readers.n > 0) launch_seq(epilogue_seq_kernel<PT, OT, KW, true, BN>, dim3(blocks, slices), dim3(256), 0, st, e);
-    else launch_seq(epilogue_seq_kernel<PT, OT, KW, false, BN>, dim3(blocks, slices), dim3(256), 0, st, e);
+    // (a layer of few channels: no more warps than have a turn to make)
+    const int busy = OT == T_BIN ? e.cs : ceil_div(ceil_div(e.cs, 4), NQ);
+    const int threads = 32 * (busy < 1 ? 1 : (busy > 8 ? 8 : busy));
+    if (e.readers.n > 0) launch_seq(epilogue_seq_kernel<PT, OT, KW, true, BN>, dim3(blocks, slices), dim3(threads), 0, st, e);
+    else launch_seq(epilogue_seq_kernel<PT, OT, KW, false, BN>, dim3(blocks, slices), dim3(threads), 0, st, e);
 }
 
 template <int PT, int OT, bool BN>
