@@ -138,8 +138,8 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
     const int tid = threadIdx.x, lane = tid & 31;
     int tile = blockIdx.x;
     const int n0 = blockIdx.y * TN;
-    const bool batched = !DENSE && p.frames > 1;             // gridDim.z counts frames, not shares of K
-    const int zshare = batched ? 0 : blockIdx.z;
+    const bool batched = !DENSE && p.frames > 1;             // gridDim.z counts frames x shares of K (shares: fp32 only)
+    const int zshare = batched ? (int)(blockIdx.z % p.ksplit) : (int)blockIdx.z;
     pdl_launch_dependents();
     if (!DENSE) {
         pdl_wait();                                          // the update bitmap is the predecessors' work
@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
             // launch order (gridDim.x * gridDim.z of them per N tile), so that the CTAs with work come first and spread
             // evenly over the SMs instead of landing wherever an active frame's block index happens to fall.  Every
             // CTA counts all frames' update bitmaps for that (a few words per frame and lane).
-            const int words = (p.opixels + 31) >> 5, nfr = (int)gridDim.z;
+            const int words = (p.opixels + 31) >> 5, nfr = (int)gridDim.z / p.ksplit;
             for (int g = tid >> 5; g < nfr; g += CONV_THREADS / 32) {
                 const uint32_t* bm = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(p.oact) + (long long)g * p.arena_stride);
                 int c = 0;
@@ -157,8 +157,8 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
                 if (lane == 0) s_fcnt[g] = c;
             }
             __syncthreads();
-            int id = (int)(blockIdx.z * gridDim.x + blockIdx.x), frame = -1;
-            if (id == 0 && blockIdx.y == 0 && tid < nfr)     // every frame's count, also of frames without a tile
+            int id = (int)((blockIdx.z / p.ksplit) * gridDim.x + blockIdx.x), frame = -1;   // (the shares of a tile agree)
+            if (id == 0 && blockIdx.y == 0 && zshare == 0 && tid < nfr)     // every frame's count, also of frames without a tile
                 *reinterpret_cast<int*>(reinterpret_cast<char*>(p.ocount) + (long long)tid * p.arena_stride) = s_fcnt[tid];
             for (int g = 0; g < nfr; ++g) {
                 const int t = (s_fcnt[g] + TM - 1) / TM;
@@ -424,6 +424,7 @@ __global__ void __launch_bounds__(CONV_THREADS) conv_gemm_kernel(ConvParams p)
                 if (co >= p.c_out) continue;
                 const size_t o = (size_t)q * p.c_out + co;
                 if (DENSE) P[o] = sv[j] + (p.bias ? reinterpret_cast<const float*>(p.bias)[co] : 0.f);
+                else if (batched) P[o] = sv[j];              // (several frames per launch: the product is stored, not added)
                 else P[o] += sv[j];
             }
         }
@@ -1626,6 +1627,14 @@ int launch_layer_seq(rrm_net* net, int l, int frames, long long arena_stride, cu
         p.frames = frames > 1 ? frames : 2;                  // (one frame still takes the storing form: the kernel tests frames > 1)
         p.row_stride = (long long)in.bytes(); p.arena_stride = arena_stride; p.p_stride = (long long)L.opixels() * d.c_out;
         dim3 grid(ceil_div(L.opixels(), TM), L.np / TN, frames);
+        if (d.dtype == RRM_F32) {
+            // fp32 with a grid of less than ~3 waves: 2 or 4 shares of K per tile (a cluster that adds its partial tiles in
+            // a fixed order), while a share keeps at least 4 stages: CTAs with rows are few and long otherwise
+            const long long ctas = (long long)grid.x * grid.y * grid.z, slots = 4ll * 148;
+            const int stages = L.kup / TK;
+            while (p.ksplit < 4 && ctas * p.ksplit < 3 * slots && stages / (p.ksplit * 2) >= 4) p.ksplit *= 2;
+            grid.z = frames * p.ksplit;
+        }
         if (d.dtype == RRM_F32) launch_gemm<T_F32, false>(p, grid, st);
         else if (d.dtype == RRM_I8) launch_gemm<T_I8, false>(p, grid, st);
         else launch_gemm<T_BIN, false>(p, grid, st);
