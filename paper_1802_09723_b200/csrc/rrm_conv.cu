@@ -1132,6 +1132,29 @@ __global__ void export_nchw_kernel(const T* __restrict__ src, T* dst, int c, int
     dst[i] = src[(ns * hw + pix) * cs + ch];
 }
 
+// The same through a 32 x 32 tile in shared memory (4-byte elements): rows read along the channels, planes written
+// along the pixels, both coalesced.  grid = (pixel tiles, channel tiles x n, frames), block = (32, 8).
+__global__ void __launch_bounds__(256) export_nchw_tiled_kernel(const uint32_t* __restrict__ src, uint32_t* dst, int c, int cs, int hw,
+                                                                int ctiles, long long src_stride, long long dst_stride)
+{
+    __shared__ uint32_t tile[32][33];
+    const int p0 = blockIdx.x * 32, c0 = (int)(blockIdx.y % ctiles) * 32;
+    const long long ns = blockIdx.y / ctiles;
+    src += blockIdx.z * src_stride;
+    dst += blockIdx.z * dst_stride;
+    pdl_launch_dependents();
+    pdl_wait();
+    for (int k = threadIdx.y; k < 32; k += 8) {
+        const int pix = p0 + k, ch = c0 + (int)threadIdx.x;
+        if (pix < hw && ch < c) tile[k][threadIdx.x] = src[(ns * hw + pix) * cs + ch];
+    }
+    __syncthreads();
+    for (int k = threadIdx.y; k < 32; k += 8) {
+        const int ch = c0 + k, pix = p0 + (int)threadIdx.x;
+        if (pix < hw && ch < c) dst[(ns * c + ch) * hw + pix] = tile[threadIdx.x][k];
+    }
+}
+
 template <typename T>
 __global__ void fill_projection_kernel(T* P, const T* bias, int c_out, long long total)
 {
@@ -1579,7 +1602,11 @@ int launch_export_tensor(rrm_net* net, int t, void* dst, bool stateless, cudaStr
     const long long total = (long long)T.n * T.c * hw;
     const int blocks = (int)((total + 255) / 256);
     if (T.dtype == T_I8) launch_seq(export_nchw_kernel<int8_t>, dim3(blocks), dim3(256), 0, st, (const int8_t*)X, (int8_t*)dst, T.c, T.cs, hw, total, 0ll, 0ll);
-    else launch_seq(export_nchw_kernel<uint32_t>, dim3(blocks), dim3(256), 0, st, (const uint32_t*)X, (uint32_t*)dst, T.c, T.cs, hw, total, 0ll, 0ll);
+    else {
+        const int ctiles = ceil_div(T.c, 32);
+        launch_seq(export_nchw_tiled_kernel, dim3(ceil_div(hw, 32), ctiles * T.n, 1), dim3(32, 8), 0, st, (const uint32_t*)X, (uint32_t*)dst,
+                   T.c, T.cs, hw, ctiles, 0ll, 0ll);
+    }
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
@@ -1598,8 +1625,11 @@ int launch_export_seq(rrm_net* net, int frames, void* dst, cudaStream_t st)
     const dim3 grid((unsigned)((total + 255) / 256), (unsigned)frames);
     if (T.dtype == T_I8) launch_seq(export_nchw_kernel<int8_t>, grid, dim3(256), 0, st, (const int8_t*)T.Xfull, (int8_t*)dst, T.c, T.cs, hw, total,
                                     (long long)T.bytes(), total);
-    else launch_seq(export_nchw_kernel<uint32_t>, grid, dim3(256), 0, st, (const uint32_t*)T.Xfull, (uint32_t*)dst, T.c, T.cs, hw, total,
-                    (long long)T.bytes() / 4, total);
+    else {
+        const int ctiles = ceil_div(T.c, 32);
+        launch_seq(export_nchw_tiled_kernel, dim3(ceil_div(hw, 32), ctiles * T.n, frames), dim3(32, 8), 0, st, (const uint32_t*)T.Xfull, (uint32_t*)dst,
+                   T.c, T.cs, hw, ctiles, (long long)T.bytes() / 4, total);
+    }
     RRM_CUDA_TRY(cudaGetLastError());
     return RRM_OK;
 }
