@@ -786,6 +786,79 @@ __global__ void __launch_bounds__(256, 4) import_i8_word_frames_kernel(const int
     }
 }
 
+// fp32 frames of at most 4 channels, several frames per launch, no truncation (Sec. 3.4 off): the same walk as
+// import_i8_word_frames_kernel - a thread per pixel reads its channel planes of frame g and g - 1 (coalesced along the
+// pixels), writes the delta row of a changed pixel and, in the last frame, the snapshot.
+__global__ void __launch_bounds__(256, 4) import_f32_px_frames_kernel(const float* __restrict__ src, float* X, float* D, uint32_t* act,
+                                                                     unsigned long long* nnz, unsigned long long* npix,
+                                                                     int c, int h, int w, int pixels, Readers readers, SeqFrames sf)
+{
+    const int lane = threadIdx.x & 31;
+    const int base = (blockIdx.x * 8 + (threadIdx.x >> 5)) * 128;
+    const int hw = h * w;
+    {
+        const long long g = blockIdx.z;
+        src += g * sf.in_stride;
+        D = shift_bytes(D, g * sf.row_stride);
+        act = shift_bytes(act, g * sf.arena_stride); nnz = shift_bytes(nnz, g * sf.arena_stride);
+        npix = shift_bytes(npix, g * sf.arena_stride);
+    }
+    const long long arena_off = (long long)blockIdx.z * sf.arena_stride;
+    const bool write_x = (int)blockIdx.z == sf.frames - 1;
+    pdl_launch_dependents();
+    pdl_wait();
+    float nv[4][4], pv[4][4];
+    #pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int gp = base + 32 * k + lane;
+        #pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            nv[k][ch] = pv[k][ch] = 0.f;
+            if (gp >= pixels || ch >= c) continue;
+            const int ns = gp / hw, pix = gp - ns * hw;
+            const size_t o = ((size_t)ns * c + ch) * hw + pix;
+            nv[k][ch] = src[o];
+            pv[k][ch] = (src - sf.in_stride)[o];
+        }
+    }
+    #pragma unroll 1
+    for (int k = 0; k < 4; ++k) {
+        const int gp = base + 32 * k + lane;
+        if (base + 32 * k >= pixels) break;                  // uniform inside the warp
+        int cnt = 0;
+        if (gp < pixels) {
+            #pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                if (ch >= c) break;
+                if (write_x) X[(size_t)gp * c + ch] = nv[k][ch];
+                cnt += nv[k][ch] != pv[k][ch];
+            }
+            if (cnt) {
+                #pragma unroll
+                for (int ch = 0; ch < 4; ++ch) if (ch < c) D[(size_t)gp * c + ch] = nv[k][ch] - pv[k][ch];
+            }
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
+        if (m == 0) continue;                                // uniform inside the warp
+        if (lane == 0) act[gp >> 5] = m;                     // gp of lane 0 is a multiple of 32: the word is this group's alone
+        const int tot = __reduce_add_sync(0xffffffffu, cnt);
+        if (lane == 0) {
+            atomicAdd(nnz, (unsigned long long)tot);
+            atomicAdd(npix, (unsigned long long)__popc(m));
+        }
+        unsigned long long wsum[MAX_READERS];
+        {
+            const int ns = gp / hw, pix = gp - ns * hw;
+            scatter_changed_warp(readers, ns, pix / w, pix % w, cnt, lane, wsum, arena_off);
+        }
+        if (lane == 0) {
+            #pragma unroll
+            for (int i = 0; i < MAX_READERS; ++i)
+                if (i < readers.n && readers.r[i].macs && wsum[i]) atomicAdd(shift_bytes(readers.r[i].macs, arena_off), wsum[i]);
+        }
+    }
+}
+
 // Binary frames arrive already pixel-major and bit-packed: one thread per pixel.
 template <bool DELTA>
 __global__ void import_bin_kernel(const uint32_t* __restrict__ src, uint32_t* X, uint32_t* D, uint32_t* act,
@@ -1323,7 +1396,10 @@ int launch_import(rrm_net* net, const void* frame, bool delta, bool stateless, c
         dim3 grid(ceil_div(hw, IMP_TP), T.n, gz);
         const size_t smem = (size_t)IMP_TP * (T.cs + 1) * T.unit_bytes * (seq ? 2 : 1);
         if (smem > 200 * 1024) return RRM_ERR_UNSUPPORTED;
-        if (T.dtype == T_F32) {
+        if (T.dtype == T_F32 && seq && T.c <= 4 && !(net->eps > 0.f)) {
+            launch_seq(import_f32_px_frames_kernel, dim3(ceil_div(T.pixels(), 1024), 1, gz), dim3(256), 0, st, (const float*)frame, (float*)X,
+                       (float*)T.D, T.act, T.nnz, T.npix, T.c, T.h, T.w, T.pixels(), T.readers, sf);
+        } else if (T.dtype == T_F32) {
             auto kd = import_nchw_kernel<float, true>;
             auto kn = import_nchw_kernel<float, false>;
             if (smem > 48 * 1024) {
